@@ -1,0 +1,472 @@
+/*
+ * g10_oracle.c -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, single-threaded CPU restatement of the compile-time planning path of G10
+ * (tensor vitality analysis, Section 4.2; GPU memory pressure, Section 4.3; the smart tensor
+ * eviction loop, Algorithm 1).  It exists so that the CUDA library can be compared against
+ * something written directly from the paper's definitions.  It shares no code, header, table or
+ * helper with the CUDA path, and nothing outside tests / the smoke check / the benchmark's CPU
+ * baseline may call it.
+ *
+ * Everything is integer.  Times are nanoseconds, sizes are bytes.  "u128" is an exact unsigned
+ * 128-bit integer.  Where the paper leaves a point open the reading taken is stated next to the
+ * code that implements it.
+ *
+ * Pins (tests that tie each function to something other than itself):
+ *   g10o_slot_clock, g10o_vitality, g10o_pressure : dense kernel-by-tensor matrix brute force,
+ *       closed forms for the MLP-chain trace, conservation of byte-slots.
+ *   g10o_geometry : hand-worked examples, dense per-nanosecond brute force on toy traces.
+ *   g10o_plan (plain tier) : three hand-worked traces, an independent arbitrary-precision Python
+ *       restatement on random toy traces, plan invariants (excess-area identity, channel budgets,
+ *       residency at every use).  The paper prints no numeric example of Algorithm 1 (its figures
+ *       did not survive), so agreement with the paper's own numbers is "parity unpinned".
+ *   g10o_plan (lazy tier) : must equal the plain tier bit for bit.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef unsigned __int128 u128;
+
+enum { DEST_SSD = 0, DEST_HOST = 1 };
+enum { CH_SSD_OUT = 0, CH_SSD_IN = 1, CH_HOST_OUT = 2, CH_HOST_IN = 3 };
+enum { ST_ALREADY_FITS = 0, ST_FIT = 1, ST_EXHAUSTED = 2, ST_ITERATION_LIMIT = 3 };
+
+#define T_SATURATE ((int64_t)1 << 62)
+
+typedef struct {
+    int32_t period, tensor, dest;
+    int32_t absent_first, absent_last;
+    int32_t iteration;
+    int64_t evict_issue_ns, prefetch_issue_ns, transfer_ns;
+} g10o_migration;
+
+/* ------------------------------------------------------------------------------------------
+ * Slot clock (Section 4.2: kernel execution times measure the inactive periods).
+ * Reading: kernels run back to back in trace order, so kernel k occupies [start[k], start[k+1]).
+ * ---------------------------------------------------------------------------------------- */
+void g10o_slot_clock(int64_t K, const int64_t *kernel_ns, int64_t *start /* [K+1] */)
+{
+    start[0] = 0;
+    for (int64_t k = 0; k < K; ++k) start[k + 1] = start[k] + kernel_ns[k];
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Tensor vitality (Section 4.2).
+ * A tensor is active while a kernel that lists it (input or output) runs.  U_i is the sorted set
+ * of distinct kernels listing tensor i (a kernel that lists a tensor twice, as an in-place
+ * operator does, uses it once).  Born at min U_i, dead after max U_i.  Between two consecutive
+ * uses u < v with at least one kernel in between (v - u >= 2) the tensor is inactive and not
+ * dead: one inactive period (i, u, v).  Periods are numbered by (tensor, u) ascending.
+ * Returns 0, or -1 if uses_cap / periods_cap is too small (counts[] still holds the need).
+ * ---------------------------------------------------------------------------------------- */
+int32_t g10o_vitality(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t *kernel_tensors,
+                      int32_t *first_use, int32_t *last_use, int32_t *num_uses,
+                      int64_t *use_ptr /* [N+1] */, int32_t *uses, int64_t uses_cap,
+                      int64_t *period_ptr /* [N+1] */, int32_t *period_tensor, int32_t *period_prev_use,
+                      int32_t *period_next_use, int64_t periods_cap, int64_t *counts /* [2] */)
+{
+    int32_t *seen = (int32_t *)malloc(sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
+    int64_t *fill = (int64_t *)malloc(sizeof(int64_t) * (size_t)(N > 0 ? N : 1));
+    for (int64_t i = 0; i < N; ++i) { seen[i] = -1; num_uses[i] = 0; }
+    /* |U_i| : kernels are visited in increasing order, so a repeat inside one kernel is caught
+       by remembering the last kernel that listed the tensor. */
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t e = kernel_ptr[k]; e < kernel_ptr[k + 1]; ++e) {
+            int32_t i = kernel_tensors[e];
+            if (seen[i] != (int32_t)k) { seen[i] = (int32_t)k; num_uses[i] += 1; }
+        }
+    use_ptr[0] = 0;
+    for (int64_t i = 0; i < N; ++i) use_ptr[i + 1] = use_ptr[i] + num_uses[i];
+    counts[0] = use_ptr[N];
+    int32_t rc = 0;
+    if (use_ptr[N] > uses_cap) rc = -1;
+    if (rc == 0) {
+        for (int64_t i = 0; i < N; ++i) { seen[i] = -1; fill[i] = use_ptr[i]; }
+        for (int64_t k = 0; k < K; ++k)
+            for (int64_t e = kernel_ptr[k]; e < kernel_ptr[k + 1]; ++e) {
+                int32_t i = kernel_tensors[e];
+                if (seen[i] != (int32_t)k) { seen[i] = (int32_t)k; uses[fill[i]++] = (int32_t)k; }
+            }
+    }
+    /* born / dead, and the inactive periods */
+    int64_t np = 0;
+    period_ptr[0] = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        if (num_uses[i] == 0) { first_use[i] = -1; last_use[i] = -1; }
+        else if (rc == 0) { first_use[i] = uses[use_ptr[i]]; last_use[i] = uses[use_ptr[i + 1] - 1]; }
+        if (rc == 0)
+            for (int64_t j = use_ptr[i]; j + 1 < use_ptr[i + 1]; ++j) {
+                int32_t u = uses[j], v = uses[j + 1];
+                if (v - u >= 2) {
+                    if (np < periods_cap) { period_tensor[np] = (int32_t)i; period_prev_use[np] = u; period_next_use[np] = v; }
+                    np += 1;
+                }
+            }
+        period_ptr[i + 1] = np;
+    }
+    counts[1] = np;
+    if (np > periods_cap) rc = -1;
+    free(seen); free(fill);
+    return rc;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * GPU memory pressure before any migration (Section 4.3: "the total size of non-evicted tensors
+ * in GPU memory at time T").  Written as the definition: every tensor adds its size to every
+ * slot it is alive in.  An intermediate tensor lives from its birth to its death; a global
+ * tensor (weights) is allocated at the start of the program and is never freed, so it lives in
+ * every slot, provided the trace uses it at all.  peak_slot is the lowest slot holding the peak
+ * (-1 when there are no slots).
+ * ---------------------------------------------------------------------------------------- */
+void g10o_pressure(int64_t K, int64_t N, const int64_t *tensor_bytes, const uint8_t *tensor_global,
+                   const int32_t *first_use, const int32_t *last_use,
+                   int64_t *pressure /* [K] */, int64_t *peak_bytes, int32_t *peak_slot)
+{
+    for (int64_t k = 0; k < K; ++k) pressure[k] = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        if (first_use[i] < 0) continue;
+        int64_t lo = first_use[i], hi = last_use[i];
+        if (tensor_global && tensor_global[i]) { lo = 0; hi = K - 1; }
+        for (int64_t k = lo; k <= hi; ++k) pressure[k] += tensor_bytes[i];
+    }
+    int64_t pk = 0; int32_t ps = -1;
+    for (int64_t k = 0; k < K; ++k) if (ps < 0 || pressure[k] > pk) { pk = pressure[k]; ps = (int32_t)k; }
+    *peak_bytes = pk; *peak_slot = ps;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Candidate geometry for one period and one destination.
+ * Transfer time t = ceil(bytes * 1e9 / bandwidth) ns (Algorithm 1: tensor_size / BW), the same in
+ * both directions.  The eviction starts when the period starts, t_r = end of kernel u (Algorithm 1
+ * schedules the pre-eviction at t_r) and occupies [t_r, t_r + t).  The prefetch is issued at the
+ * latest safe prefetch time t_end - t (Section 4.4), t_end = start of kernel v, and occupies
+ * [t_end - t, t_end).  The tensor counts as absent from GPU memory exactly in the slots that lie
+ * wholly between the two windows: from a' = first slot starting at or after t_r + t, to
+ * b' = the slot before the one in which the prefetch window begins.  Invalid (never a candidate)
+ * when the two transfers do not fit into the period (2t > L) or no whole slot is left (a' > b').
+ * ---------------------------------------------------------------------------------------- */
+static int64_t transfer_ns(int64_t bytes, uint64_t bw)
+{
+    u128 num = (u128)(uint64_t)bytes * (u128)1000000000u;
+    u128 q = num / bw;
+    if (q * bw != num) q += 1;
+    if (q > (u128)T_SATURATE) return T_SATURATE;
+    return (int64_t)q;
+}
+
+typedef struct { int64_t t; int32_t a_abs, b_abs; int valid; } geo_t;
+
+static geo_t geometry_one(int64_t K, const int64_t *start, int64_t bytes, int32_t u, int32_t v, uint64_t bw)
+{
+    geo_t g; g.valid = 0; g.a_abs = -1; g.b_abs = -2;
+    g.t = transfer_ns(bytes, bw);
+    int64_t t_r = start[u + 1], t_end = start[v];
+    int64_t L = t_end - t_r;
+    if (g.t > L || 2 * g.t > L) return g;                 /* (first test keeps 2t from overflowing) */
+    int64_t ap = u + 1;                                   /* first k in [0,K] with start[k] >= t_r + t */
+    while (ap <= K && start[ap] < t_r + g.t) ++ap;
+    int64_t j = v;                                        /* last j in [0,K] with start[j] <= t_end - t */
+    while (j >= 0 && start[j] > t_end - g.t) --j;
+    int64_t bp = j - 1;
+    if (ap > bp) return g;
+    g.valid = 1; g.a_abs = (int32_t)ap; g.b_abs = (int32_t)bp;
+    return g;
+}
+
+/* transfer_ns[X*Pn+p], absent_first[X*Pn+p], absent_last[X*Pn+p] for X = 0 (SSD), 1 (HOST);
+   an invalid pair has absent_first = -1, absent_last = -2. */
+void g10o_geometry(int64_t K, int64_t Pn, const int64_t *start, const int64_t *tensor_bytes,
+                   const int32_t *period_tensor, const int32_t *period_prev_use, const int32_t *period_next_use,
+                   uint64_t host_bw, uint64_t ssd_bw,
+                   int64_t *out_transfer_ns, int32_t *out_absent_first, int32_t *out_absent_last)
+{
+    for (int X = 0; X < 2; ++X)
+        for (int64_t p = 0; p < Pn; ++p) {
+            geo_t g = geometry_one(K, start, tensor_bytes[period_tensor[p]], period_prev_use[p], period_next_use[p],
+                                   X == DEST_SSD ? ssd_bw : host_bw);
+            out_transfer_ns[X * Pn + p] = g.t;
+            out_absent_first[X * Pn + p] = g.a_abs;
+            out_absent_last[X * Pn + p] = g.b_abs;
+        }
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Planner state and scoring (Section 4.3, Algorithm 1).
+ * ---------------------------------------------------------------------------------------- */
+typedef struct {
+    int64_t K, Pn;
+    const int64_t *start, *dur, *bytes;
+    const int32_t *per_tensor, *per_u, *per_v;
+    geo_t *geo[2];
+    int64_t *P;            /* current pressure per slot                                  */
+    int64_t *busy[4];      /* ns of each slot already given to a transfer, per channel   */
+    int64_t *hocc;         /* bytes parked in host memory per slot                       */
+    int64_t cap;
+    uint64_t host_capacity;
+} plan_state;
+
+/* overlap of the time window [w0, w1) with slot k */
+static int64_t overlap(const plan_state *S, int64_t w0, int64_t w1, int64_t k)
+{
+    int64_t lo = w0 > S->start[k] ? w0 : S->start[k];
+    int64_t hi = w1 < S->start[k + 1] ? w1 : S->start[k + 1];
+    return hi > lo ? hi - lo : 0;
+}
+
+/* Bandwidth budget (Algorithm 1 asks whether the traffic to a device "is full" during the
+   transfer).  Reading: each slot offers dur[k] ns of channel time per device and direction; a
+   transfer may be booked iff, in every slot its window touches, the time already booked plus the
+   window's overlap with that slot stays within dur[k]. */
+static int channel_free(const plan_state *S, int ch, int64_t w0, int64_t w1, int64_t k0, int64_t k1)
+{
+    for (int64_t k = k0; k <= k1; ++k)
+        if (S->busy[ch][k] + overlap(S, w0, w1, k) > S->dur[k]) return 0;
+    return 1;
+}
+
+static int admissible(const plan_state *S, int64_t p, int X)
+{
+    const geo_t *g = &S->geo[X][p];
+    if (!g->valid) return 0;
+    int64_t a = S->per_u[p] + 1, b = S->per_v[p] - 1;
+    int64_t t_r = S->start[a], t_end = S->start[b + 1];
+    int out = X == DEST_SSD ? CH_SSD_OUT : CH_HOST_OUT, in = X == DEST_SSD ? CH_SSD_IN : CH_HOST_IN;
+    if (!channel_free(S, out, t_r, t_r + g->t, a, g->a_abs - 1)) return 0;
+    if (!channel_free(S, in, t_end - g->t, t_end, g->b_abs + 1, b)) return 0;
+    if (X == DEST_HOST && S->host_capacity != 0) {
+        /* "host mem isn't full during periods[0]": the tensor sits in host memory for the whole period */
+        uint64_t s = (uint64_t)S->bytes[S->per_tensor[p]];
+        for (int64_t k = a; k <= b; ++k)
+            if ((uint64_t)S->hocc[k] + s > S->host_capacity) return 0;
+    }
+    return 1;
+}
+
+/* Benefit of evicting during the period with destination X: the part of the pressure curve above
+   the capacity line that disappears (the shaded area of the paper's state-transition figure),
+   in byte*ns: sum over absent slots of min(size, excess) * dur. */
+static u128 benefit_of(const plan_state *S, int64_t p, int X)
+{
+    const geo_t *g = &S->geo[X][p];
+    int64_t s = S->bytes[S->per_tensor[p]];
+    u128 acc = 0;
+    for (int64_t k = g->a_abs; k <= g->b_abs; ++k) {
+        int64_t ex = S->P[k] - S->cap;
+        if (ex <= 0) continue;
+        if (ex > s) ex = s;
+        acc += (u128)(uint64_t)ex * (u128)(uint64_t)S->dur[k];
+    }
+    return acc;
+}
+
+/* Destination rule: SSD first (large capacity); host memory only when the SSD cannot take the
+   transfer (its channel is saturated in the window, or the tensor cannot go out and come back
+   within the period) and the host link and host memory can.  Returns -1 if neither works. */
+static int choose_destination(const plan_state *S, int64_t p)
+{
+    if (admissible(S, p, DEST_SSD)) return DEST_SSD;
+    if (admissible(S, p, DEST_HOST)) return DEST_HOST;
+    return -1;
+}
+
+/* p beats q iff benefit_p / cost_p > benefit_q / cost_q, exact; ties go to the lower index */
+static int beats(u128 bp, int64_t cp, int64_t ip, u128 bq, int64_t cq, int64_t iq)
+{
+    u128 l = bp * (u128)(uint64_t)cq, r = bq * (u128)(uint64_t)cp;
+    if (l != r) return l > r;
+    return ip < iq;
+}
+
+static void commit(plan_state *S, int64_t p, int X)
+{
+    const geo_t *g = &S->geo[X][p];
+    int64_t s = S->bytes[S->per_tensor[p]];
+    int64_t a = S->per_u[p] + 1, b = S->per_v[p] - 1;
+    int64_t t_r = S->start[a], t_end = S->start[b + 1];
+    int out = X == DEST_SSD ? CH_SSD_OUT : CH_HOST_OUT, in = X == DEST_SSD ? CH_SSD_IN : CH_HOST_IN;
+    for (int64_t k = g->a_abs; k <= g->b_abs; ++k) S->P[k] -= s;
+    for (int64_t k = a; k <= g->a_abs - 1; ++k) S->busy[out][k] += overlap(S, t_r, t_r + g->t, k);
+    for (int64_t k = g->b_abs + 1; k <= b; ++k) S->busy[in][k] += overlap(S, t_end - g->t, t_end, k);
+    if (X == DEST_HOST) for (int64_t k = a; k <= b; ++k) S->hocc[k] += s;
+}
+
+static void peak_of(const int64_t *P, int64_t K, int64_t *pk, int64_t *ps)
+{
+    *pk = 0; *ps = -1;
+    for (int64_t k = 0; k < K; ++k) if (*ps < 0 || P[k] > *pk) { *pk = P[k]; *ps = k; }
+}
+
+/* ---- a binary max-heap of (bound ratio, index) for the lazy tier --------------------------- */
+typedef struct { u128 ben; int64_t cost; int64_t idx; } hnode;
+static int hbeats(const hnode *x, const hnode *y) { return beats(x->ben, x->cost, x->idx, y->ben, y->cost, y->idx); }
+static void hpush(hnode *h, int64_t *n, hnode v)
+{
+    int64_t i = (*n)++; h[i] = v;
+    while (i > 0) { int64_t par = (i - 1) / 2; if (!hbeats(&h[i], &h[par])) break; hnode t = h[i]; h[i] = h[par]; h[par] = t; i = par; }
+}
+static hnode hpop(hnode *h, int64_t *n)
+{
+    hnode top = h[0]; h[0] = h[--(*n)];
+    int64_t i = 0;
+    for (;;) {
+        int64_t l = 2 * i + 1, r = l + 1, m = i;
+        if (l < *n && hbeats(&h[l], &h[m])) m = l;
+        if (r < *n && hbeats(&h[r], &h[m])) m = r;
+        if (m == i) break;
+        hnode t = h[i]; h[i] = h[m]; h[m] = t; i = m;
+    }
+    return top;
+}
+
+/* Lazy tier.  For a fixed destination the absent range and the cost never change, pressure only
+   falls, and booked channel time / host occupancy only rise: each destination's ratio can only
+   fall and a destination once refused stays refused.  So the larger of the ratios of the
+   destinations still open to a period bounds every score the period can have later (it may fall
+   back from SSD to host, and a host transfer is cheaper).  lazy_eval computes, against the
+   current state, that bound and the period's true score (first admissible destination, SSD
+   before host).  Returns 0 when no destination is left or the bound has no benefit: the period
+   can be forgotten. */
+static int lazy_eval(const plan_state *S, int64_t p, char *open, hnode *bound, u128 *tb, int64_t *tc, int *tX)
+{
+    int have = 0;
+    *tX = -1; *tb = 0; *tc = 1;
+    for (int X = 0; X < 2; ++X) {
+        if (!open[2 * p + X]) continue;
+        if (!admissible(S, p, X)) { open[2 * p + X] = 0; continue; }
+        u128 b = benefit_of(S, p, X);
+        int64_t c = 2 * S->geo[X][p].t;
+        if (*tX < 0) { *tX = X; *tb = b; *tc = c; }
+        if (!have || beats(b, c, 0, bound->ben, bound->cost, 0)) { bound->ben = b; bound->cost = c; }
+        have = 1;
+    }
+    bound->idx = p;
+    return have && bound->ben > 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * The planner (Algorithm 1).  Each iteration: stop if the peak fits; score every live period;
+ * take the best benefit/cost ratio; book it; erase the period.  Stops EXHAUSTED when no live
+ * period has a positive benefit ("no more beneficial eviction candidates").
+ *   lazy = 0 : the definition (every live period is rescored every iteration).
+ *   lazy = 1 : same result, periods rescored only when their stale bound is on top of a heap.
+ * win_benefit (optional, 2 words per record: low, high) and win_cost (optional) report the
+ * winner's score for the invariant tests.
+ * summary[8] = { migrations, scoring rounds, exit status, final peak, final peak slot,
+ *                bytes to SSD, bytes to host, 0 }.
+ * Returns 0, or -1 if out_cap is too small (summary[0] then holds the number needed).
+ * ---------------------------------------------------------------------------------------- */
+int32_t g10o_plan(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t *kernel_tensors,
+                  const int64_t *tensor_bytes, const int64_t *kernel_ns, const uint8_t *tensor_global,
+                  uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
+                  uint64_t host_capacity_bytes, int64_t max_iterations, int32_t lazy,
+                  g10o_migration *out, int64_t out_cap, int64_t *final_pressure /* [K] */,
+                  int64_t *summary /* [8] */, uint64_t *win_benefit, int64_t *win_cost)
+{
+    int64_t E = K > 0 ? kernel_ptr[K] : 0;
+    size_t nN = (size_t)(N > 0 ? N : 1), nK = (size_t)(K > 0 ? K : 1), nE = (size_t)(E > 0 ? E : 1);
+    int64_t *start = (int64_t *)malloc(sizeof(int64_t) * (nK + 1));
+    int32_t *first = (int32_t *)malloc(4 * nN), *last = (int32_t *)malloc(4 * nN), *nuse = (int32_t *)malloc(4 * nN);
+    int64_t *use_ptr = (int64_t *)malloc(8 * (nN + 1)), *per_ptr = (int64_t *)malloc(8 * (nN + 1));
+    int32_t *uses = (int32_t *)malloc(4 * nE);
+    int32_t *pt = (int32_t *)malloc(4 * nE), *pu = (int32_t *)malloc(4 * nE), *pv = (int32_t *)malloc(4 * nE);
+    int64_t counts[2];
+    g10o_slot_clock(K, kernel_ns, start);
+    g10o_vitality(K, N, kernel_ptr, kernel_tensors, first, last, nuse, use_ptr, uses, E, per_ptr, pt, pu, pv, E, counts);
+    int64_t Pn = counts[1];
+    int64_t pk; int32_t ps32;
+    g10o_pressure(K, N, tensor_bytes, tensor_global, first, last, final_pressure, &pk, &ps32);
+
+    plan_state S;
+    S.K = K; S.Pn = Pn; S.start = start; S.dur = kernel_ns; S.bytes = tensor_bytes;
+    S.per_tensor = pt; S.per_u = pu; S.per_v = pv; S.P = final_pressure;
+    S.host_capacity = host_capacity_bytes;
+    size_t nP = (size_t)(Pn > 0 ? Pn : 1);
+    for (int X = 0; X < 2; ++X) {
+        S.geo[X] = (geo_t *)malloc(sizeof(geo_t) * nP);
+        for (int64_t p = 0; p < Pn; ++p)
+            S.geo[X][p] = geometry_one(K, start, tensor_bytes[pt[p]], pu[p], pv[p], X == DEST_SSD ? ssd_bw : host_bw);
+    }
+    for (int c = 0; c < 4; ++c) S.busy[c] = (int64_t *)calloc(nK, 8);
+    S.hocc = (int64_t *)calloc(nK, 8);
+    char *alive = (char *)malloc(nP);
+    memset(alive, 1, nP);
+
+    int64_t limit = (max_iterations <= 0 || max_iterations > Pn) ? Pn : max_iterations;
+    int64_t n_mig = 0, n_rounds = 0, status = -1, bytes_to[2] = {0, 0};
+    int32_t rc = 0;
+    /* a capacity of 2^63 or more can never be exceeded by an int64 pressure */
+    int fits_always = gpu_capacity_bytes >= ((uint64_t)1 << 63);
+    S.cap = fits_always ? INT64_MAX : (int64_t)gpu_capacity_bytes;
+
+    hnode *heap = NULL, *popped = NULL; int64_t hn = 0; char *open = NULL;
+    if (lazy) {
+        heap = (hnode *)malloc(sizeof(hnode) * nP);
+        open = (char *)malloc(2 * nP);
+        memset(open, 1, 2 * nP);
+        popped = (hnode *)malloc(sizeof(hnode) * nP);
+        for (int64_t p = 0; p < Pn; ++p) {
+            hnode nd; u128 tb; int64_t tc; int tX;
+            if (lazy_eval(&S, p, open, &nd, &tb, &tc, &tX)) hpush(heap, &hn, nd);
+        }
+    }
+
+    for (int64_t it = 0;; ++it) {
+        int64_t cur_peak, cur_slot;
+        peak_of(S.P, K, &cur_peak, &cur_slot);
+        if (fits_always || cur_peak <= S.cap) { status = n_mig == 0 ? ST_ALREADY_FITS : ST_FIT; break; }
+        if (it >= limit) { status = limit < Pn ? ST_ITERATION_LIMIT : ST_EXHAUSTED; break; }
+        n_rounds += 1;
+        int64_t best = -1; int bestX = -1; u128 bestB = 0; int64_t bestC = 1;
+        if (!lazy) {
+            for (int64_t p = 0; p < Pn; ++p) {
+                if (!alive[p]) continue;
+                int X = choose_destination(&S, p);
+                if (X < 0) continue;
+                u128 b = benefit_of(&S, p, X);
+                if (b == 0) continue;
+                int64_t c = 2 * S.geo[X][p].t;
+                if (best < 0 || beats(b, c, p, bestB, bestC, best)) { best = p; bestX = X; bestB = b; bestC = c; }
+            }
+        } else {
+            /* Pop while the top bound could still beat the best true score seen this iteration;
+               every popped period is rescored against the current state.  What stays in the heap
+               has bound <= best, hence true score <= best. */
+            int64_t npop = 0;
+            while (hn > 0 && (best < 0 || beats(heap[0].ben, heap[0].cost, heap[0].idx, bestB, bestC, best))) {
+                hnode top = hpop(heap, &hn);
+                hnode bd; u128 tb; int64_t tc; int tX;
+                if (!lazy_eval(&S, top.idx, open, &bd, &tb, &tc, &tX)) continue;
+                popped[npop++] = bd;
+                if (tb > 0 && (best < 0 || beats(tb, tc, top.idx, bestB, bestC, best))) {
+                    best = top.idx; bestX = tX; bestB = tb; bestC = tc;
+                }
+            }
+            for (int64_t j = 0; j < npop; ++j) if (popped[j].idx != best) hpush(heap, &hn, popped[j]);
+        }
+        if (best < 0) { status = ST_EXHAUSTED; break; }
+        if (n_mig < out_cap) {
+            const geo_t *g = &S.geo[bestX][best];
+            g10o_migration *m = &out[n_mig];
+            m->period = (int32_t)best; m->tensor = pt[best]; m->dest = bestX;
+            m->absent_first = g->a_abs; m->absent_last = g->b_abs; m->iteration = (int32_t)it;
+            m->evict_issue_ns = start[pu[best] + 1]; m->prefetch_issue_ns = start[pv[best]] - g->t; m->transfer_ns = g->t;
+            if (win_benefit) { win_benefit[2 * n_mig] = (uint64_t)bestB; win_benefit[2 * n_mig + 1] = (uint64_t)(bestB >> 64); }
+            if (win_cost) win_cost[n_mig] = bestC;
+        } else rc = -1;
+        commit(&S, best, bestX);
+        alive[best] = 0;
+        bytes_to[bestX] += tensor_bytes[pt[best]];
+        n_mig += 1;
+    }
+    int64_t fpk, fps;
+    peak_of(S.P, K, &fpk, &fps);
+    summary[0] = n_mig; summary[1] = n_rounds; summary[2] = status; summary[3] = fpk; summary[4] = fps;
+    summary[5] = bytes_to[DEST_SSD]; summary[6] = bytes_to[DEST_HOST]; summary[7] = 0;
+
+    free(start); free(first); free(last); free(nuse); free(use_ptr); free(per_ptr); free(uses);
+    free(pt); free(pu); free(pv); free(S.geo[0]); free(S.geo[1]);
+    for (int c = 0; c < 4; ++c) free(S.busy[c]);
+    free(S.hocc); free(alive); free(heap); free(open); free(popped);
+    return rc;
+}

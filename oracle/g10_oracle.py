@@ -1,0 +1,130 @@
+"""ctypes front end of the CPU oracle (g10_oracle.c) -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
+It compiles g10_oracle.c with gcc on first use and exposes the oracle's functions on numpy
+arrays.  It imports nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from types import SimpleNamespace
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "g10_oracle.c")
+_LIB = os.path.join(_HERE, "libg10_oracle.so")
+
+MIGRATION_DTYPE = np.dtype([
+    ("period", "<i4"), ("tensor", "<i4"), ("dest", "<i4"),
+    ("absent_first", "<i4"), ("absent_last", "<i4"), ("iteration", "<i4"),
+    ("evict_issue_ns", "<i8"), ("prefetch_issue_ns", "<i8"), ("transfer_ns", "<i8"),
+])
+assert MIGRATION_DTYPE.itemsize == 48
+
+STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", _LIB, _SRC])
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(C.c_void_p) if a is not None else None
+
+
+def _c(a, dt):
+    return np.ascontiguousarray(a, dtype=dt)
+
+
+def slot_clock(kernel_ns):
+    dur = _c(kernel_ns, np.int64)
+    start = np.zeros(dur.shape[0] + 1, dtype=np.int64)
+    lib().g10o_slot_clock(C.c_int64(dur.shape[0]), _p(dur), _p(start))
+    return start
+
+
+def vitality(kernel_ptr, kernel_tensors, N):
+    ptr = _c(kernel_ptr, np.int64)
+    kt = _c(kernel_tensors, np.int32)
+    K, E = ptr.shape[0] - 1, kt.shape[0]
+    first = np.zeros(N, np.int32); last = np.zeros(N, np.int32); nuse = np.zeros(N, np.int32)
+    use_ptr = np.zeros(N + 1, np.int64); uses = np.zeros(max(E, 1), np.int32)
+    per_ptr = np.zeros(N + 1, np.int64)
+    pt = np.zeros(max(E, 1), np.int32); pu = np.zeros(max(E, 1), np.int32); pv = np.zeros(max(E, 1), np.int32)
+    counts = np.zeros(2, np.int64)
+    rc = lib().g10o_vitality(C.c_int64(K), C.c_int64(N), _p(ptr), _p(kt), _p(first), _p(last), _p(nuse),
+                             _p(use_ptr), _p(uses), C.c_int64(E), _p(per_ptr), _p(pt), _p(pu), _p(pv),
+                             C.c_int64(E), _p(counts))
+    assert rc == 0
+    e2, pn = int(counts[0]), int(counts[1])
+    return SimpleNamespace(first_use=first, last_use=last, num_uses=nuse, use_ptr=use_ptr, uses=uses[:e2].copy(),
+                           period_ptr=per_ptr, period_tensor=pt[:pn].copy(), period_prev_use=pu[:pn].copy(),
+                           period_next_use=pv[:pn].copy(), counts=counts)
+
+
+def pressure(K, tensor_bytes, tensor_global, first_use, last_use):
+    tb = _c(tensor_bytes, np.int64)
+    tg = _c(tensor_global, np.uint8) if tensor_global is not None else None
+    f = _c(first_use, np.int32); l = _c(last_use, np.int32)
+    P = np.zeros(K, np.int64)
+    peak = C.c_int64(0); slot = C.c_int32(0)
+    lib().g10o_pressure(C.c_int64(K), C.c_int64(tb.shape[0]), _p(tb), _p(tg), _p(f), _p(l), _p(P),
+                        C.byref(peak), C.byref(slot))
+    return P, int(peak.value), int(slot.value)
+
+
+def geometry(start, tensor_bytes, period_tensor, period_prev_use, period_next_use, host_bw, ssd_bw):
+    st = _c(start, np.int64); tb = _c(tensor_bytes, np.int64)
+    pt = _c(period_tensor, np.int32); pu = _c(period_prev_use, np.int32); pv = _c(period_next_use, np.int32)
+    Pn = pt.shape[0]
+    t = np.zeros((2, Pn), np.int64); a = np.zeros((2, Pn), np.int32); b = np.zeros((2, Pn), np.int32)
+    lib().g10o_geometry(C.c_int64(st.shape[0] - 1), C.c_int64(Pn), _p(st), _p(tb), _p(pt), _p(pu), _p(pv),
+                        C.c_uint64(host_bw), C.c_uint64(ssd_bw), _p(t), _p(a), _p(b))
+    return SimpleNamespace(transfer_ns=t, absent_first=a, absent_last=b)
+
+
+def timeline(trace):
+    """start, unplanned pressure, peak, peak slot of a Trace-like object."""
+    v = vitality(trace.kernel_ptr, trace.kernel_tensors, trace.N)
+    P, peak, slot = pressure(trace.K, trace.tensor_bytes, trace.tensor_global, v.first_use, v.last_use)
+    return slot_clock(trace.kernel_ns), P, peak, slot
+
+
+def plan(trace, gpu_capacity_bytes, host_bw=None, ssd_bw=None, host_capacity_bytes=None, max_iterations=0,
+         lazy=False):
+    host_bw = trace.host_bw if host_bw is None else host_bw
+    ssd_bw = trace.ssd_bw if ssd_bw is None else ssd_bw
+    hc = trace.host_capacity_bytes if host_capacity_bytes is None else host_capacity_bytes
+    ptr = _c(trace.kernel_ptr, np.int64); kt = _c(trace.kernel_tensors, np.int32)
+    tb = _c(trace.tensor_bytes, np.int64); dur = _c(trace.kernel_ns, np.int64)
+    tg = _c(trace.tensor_global, np.uint8) if trace.tensor_global is not None else None
+    K, N, E = trace.K, trace.N, trace.E
+    cap = max(E, 1)
+    out = np.zeros(cap, MIGRATION_DTYPE)
+    finalP = np.zeros(K, np.int64)
+    summary = np.zeros(8, np.int64)
+    wb = np.zeros(2 * cap, np.uint64); wc = np.zeros(cap, np.int64)
+    rc = lib().g10o_plan(C.c_int64(K), C.c_int64(N), _p(ptr), _p(kt), _p(tb), _p(dur), _p(tg),
+                         C.c_uint64(gpu_capacity_bytes), C.c_uint64(host_bw), C.c_uint64(ssd_bw), C.c_uint64(hc),
+                         C.c_int64(max_iterations), C.c_int32(1 if lazy else 0),
+                         _p(out), C.c_int64(cap), _p(finalP), _p(summary), _p(wb), _p(wc))
+    assert rc == 0
+    n = int(summary[0])
+    ben = [int(wb[2 * j]) | (int(wb[2 * j + 1]) << 64) for j in range(n)]
+    return SimpleNamespace(migrations=out[:n].copy(), final_pressure=finalP, summary=summary,
+                           status=STATUS[int(summary[2])], win_benefit=ben, win_cost=wc[:n].copy())
