@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the G10 planning path on B200.
+
+A step is one pass of the whole hot path -- slot clock, tensor vitality, pressure timeline, candidate
+geometry and the greedy eviction loop, i.e. one g10_plan_migrations call -- over the ResNet-152-shaped
+trace (config 1).  `value` = trace events planned per second with the trace resident in HBM; `plan_ms`
+is the same step as a latency.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-stress]
+
+With N > 1 (torchrun) every rank plans its own replica of the trace (the path does not shard: the greedy
+loop is a strict sequence); value is the aggregate over ranks, time the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2310_09443_b200 import traces  # noqa: E402
+
+WORKLOAD = "config1_resnet152_b256"
+L2_FLUSH_BYTES = 512 << 20
+KERNELS_PER_PLAN = 11      # slot clock, count, scan counts, scatter, heavy sort, emit, diff, pressure scan, geometry, loop, status
+KERNELS_PER_VITALITY = 6   # count, scan counts, scatter, heavy sort, emit, status
+KERNELS_PER_TIMELINE = 6   # slot clock, first/last events, decode, diff, pressure scan, status
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import g10_oracle as O
+    O.build()
+    tr = traces.config1_resnet152()
+    start, P0, peak, slot = O.timeline(tr)
+    cap = tr.capacity_from_peak(peak)
+    for _ in range(args.warmup):
+        O.plan(tr, cap)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        r = O.plan(tr, cap)
+    dt = time.perf_counter() - t0
+    value = tr.E * args.steps / dt
+    line = {
+        "impl": "reference", "metric": "trace_events_per_s", "value": value, "unit": "events/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "K": tr.K, "N": tr.N, "E": tr.E, "migrations": int(r.summary[0]),
+                   "status": r.status},
+        "cpu_baseline": {"value": value, "unit": "events/s", "cores": 1, "kind": "oracle",
+                         "sample": "whole config-1 plan (plain tier), %d repetitions" % args.steps},
+        "e2e": {"value": value, "unit": "events/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "plan_ms": dt / args.steps * 1e3,
+    }
+    print(json.dumps(line))
+
+
+def time_calls(torch, fn, steps, warmup, flush):
+    """CUDA-event time of `steps` calls of fn on the current stream, L2 flushed between calls.  Returns seconds."""
+    for _ in range(warmup):
+        flush.fill_(1)
+        fn()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        flush.fill_(1)
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return sum(a.elapsed_time(b) for a, b in evs) / 1e3
+
+
+def run_ours(args):
+    import torch
+    from paper_2310_09443_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the planner has no CPU path")
+    torch.cuda.set_device(local)
+    dev = "cuda:%d" % local
+    build.build()
+    binding.load_library()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    hbm_peak, peak_kind = measured_peaks()
+    tr = traces.config1_resnet152()
+    tb = binding.upload(tr, dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    cap = tr.capacity_from_peak(0)          # config 1 has an absolute capacity (16 GiB)
+    ws = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E), dtype=torch.uint8, device=dev)
+    plan = binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws)
+    torch.cuda.synchronize()
+    summary = plan.summary.cpu().numpy()
+    assert summary[7] == 0, "device status %x" % summary[7]
+
+    stage = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+    for e in stage:
+        e.record()
+    stage_ms = np.zeros(4)
+
+    def step():
+        binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws, out=plan, stage_events=stage)
+
+    # ---- device-resident throughput: W warm-up steps, then exactly K timed steps
+    for _ in range(args.warmup):
+        flush.fill_(1)
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    total_ms = 0.0
+    for a, b in evs:
+        flush.fill_(1)                      # L2 flush between timed iterations (outside the event pair)
+        a.record()
+        step()
+        b.record()
+        b.synchronize()
+        total_ms += a.elapsed_time(b)
+        stage_ms += np.array([stage[j].elapsed_time(stage[j + 1]) for j in range(4)])
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_s = float(t.item()) / 1e3
+    value = world * tr.E * args.steps / total_s
+    stage_ms /= args.steps
+
+    # ---- the two analysis passes on their own (same workload)
+    vit_s = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), args.steps, args.warmup, flush)
+    tl_s = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), args.steps, args.warmup, flush)
+
+    # ---- end to end through the host-pointer form of the call: H2D of the trace and D2H of the plan inside
+    tbh = binding.pin(tr)
+    wsh = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E, binding.MEM_HOST), dtype=torch.uint8, device=dev)
+    planh = binding.g10_plan_migrations(tbh, cap, tr.host_bw, tr.ssd_bw, ws=wsh, device=dev)
+    for _ in range(args.warmup):
+        binding.g10_plan_migrations(tbh, cap, tr.host_bw, tr.ssd_bw, ws=wsh, out=planh, device=dev)
+    barrier()
+    e2e_ms = 0.0
+    for _ in range(args.steps):
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        binding.g10_plan_migrations(tbh, cap, tr.host_bw, tr.ssd_bw, ws=wsh, out=planh, device=dev)   # synchronous
+        b.record()
+        b.synchronize()
+        e2e_ms += a.elapsed_time(b)
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * tr.E * args.steps / (float(t.item()) / 1e3)
+    n_mig = int(planh.summary[0])
+    h2d = tbh.nbytes()
+    d2h = 8 * 8 + 48 * n_mig + 8 * tr.K
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the greedy loop).  Algorithmic bytes per launch: every scoring round
+    # reads pressure and duration (16 B) of each slot of each live candidate's absent range, a commit rewrites the
+    # range (16 B per slot) and appends a 48-byte record; counted from the plan itself.
+    mig = binding.migrations_numpy(plan)
+    loop_bytes = plan_loop_algorithmic_bytes(tr, binding, tb, mig, int(summary[1]))
+    loop_s = stage_ms[3] / 1e3
+    roofline = {"kernel": "k_plan_loop", "bound": "hbm", "achieved": loop_bytes / loop_s / 1e9, "peak": hbm_peak,
+                "unit": "GB/s", "frac": loop_bytes / loop_s / 1e9 / hbm_peak, "traffic": None, "peak_kind": peak_kind,
+                "algorithmic_bytes": loop_bytes, "kernel_ms": stage_ms[3],
+                "note": "state is %d KB and stays in L2/L1: the loop is bound by %d grid-wide synchronisations, not by HBM"
+                        % ((tr.K * 48) // 1024, 2 * int(summary[1]))}
+
+    line = {
+        "metric": "trace_events_per_s", "value": value, "unit": "events/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_s / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "K": tr.K, "N": tr.N, "E": tr.E, "periods": int(plan_periods(binding, tb, ws)),
+                   "gpu_capacity_bytes": cap, "host_bw": tr.host_bw, "ssd_bw": tr.ssd_bw,
+                   "migrations": int(summary[0]), "scoring_rounds": int(summary[1]), "status": binding.STATUS[int(summary[2])],
+                   "l2": "flushed between timed iterations (%d MiB write)" % (L2_FLUSH_BYTES >> 20),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "plan_ms": total_s / args.steps * 1e3,
+        "stage_ms": {"clock_vitality": stage_ms[0], "pressure": stage_ms[1], "geometry": stage_ms[2], "greedy_loop": stage_ms[3]},
+        "passes": {"vitality_ms": vit_s / args.steps * 1e3, "timeline_ms": tl_s / args.steps * 1e3,
+                   "vitality_timeline_events_per_s": tr.E / ((vit_s + tl_s) / args.steps)},
+        "e2e": {"value": e2e_value, "unit": "events/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": float(t.item()) / args.steps},
+        "gpu_launches": args.steps * KERNELS_PER_PLAN,
+        "clocks": clocks,
+        "roofline": roofline,
+    }
+    if not args.no_stress and world == 1:
+        line["stress_passes"] = stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind)
+    line["cpu_baseline"] = cpu_baseline(tr)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def plan_periods(binding, tb, ws):
+    import torch
+    v = binding.g10_vitality(tb, ws=ws)
+    torch.cuda.synchronize()
+    return int(v.counts[1].item())
+
+
+def plan_loop_algorithmic_bytes(tr, binding, tb, mig, rounds):
+    """Bytes the greedy loop must touch, from the plan: per scoring round 16 B per slot of every live valid
+    candidate's absent range (upper bound: SSD range of all periods not yet committed), per commit 16 B per slot
+    of the winner's range plus the 48-byte record."""
+    import torch
+    v = binding.g10_vitality(tb)
+    tl = binding.g10_pressure_timeline(tb)
+    torch.cuda.synchronize()
+    pn = int(v.counts[1].item())
+    g = binding.g10_candidate_geometry(tr.K, tl.kernel_start_ns, tb.tensor_bytes, v.period_tensor[:pn].contiguous(),
+                                       v.period_prev_use[:pn].contiguous(), v.period_next_use[:pn].contiguous(),
+                                       tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    a = g.absent_first.cpu().numpy(); b = g.absent_last.cpu().numpy()
+    length = np.where(a[0] >= 0, b[0] - a[0] + 1, np.where(a[1] >= 0, b[1] - a[1] + 1, 0)).astype(np.int64)
+    total_len = int(length.sum())
+    committed = length[mig["period"]]
+    # live length before round r = total - sum of the lengths committed in rounds < r
+    live = total_len * rounds - int(np.cumsum(np.concatenate([[0], committed]))[:rounds].sum())
+    commit_slots = int((mig["absent_last"] - mig["absent_first"] + 1).sum())
+    return 16 * live + 16 * commit_slots + 48 * len(mig)
+
+
+def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind):
+    """Vitality and timeline passes on the 1M-kernel / 4M-tensor stress trace (config 4): the only workload whose
+    arrays are large enough for an HBM fraction to mean something.  Algorithmic bytes: vitality reads kernel_ptr
+    (8K) and kernel_tensors (4E) and writes first/last/num_uses (12N), use_ptr (8N), uses (4E'), period_ptr (8N)
+    and the periods (12 Pn); the timeline reads kernel_ns (8K), tensor_bytes (8N), first/last (8N), the global flag
+    (N) and writes start (8K) and pressure (8K)."""
+    tr = traces.config4_stress_dag()
+    tb = binding.upload(tr, dev)
+    ws = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E), dtype=torch.uint8, device=dev)
+    v = binding.g10_vitality(tb, ws=ws)
+    torch.cuda.synchronize()
+    e2, pn = int(v.counts[0].item()), int(v.counts[1].item())
+    K, N, E = tr.K, tr.N, tr.E
+    vit_bytes = 8 * K + 4 * E + 12 * N + 8 * N + 4 * e2 + 8 * N + 12 * pn
+    tl_bytes = 8 * K + 8 * N + 8 * N + N + 8 * K + 8 * K
+    steps, warm = 10, 3
+    vit_s = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), steps, warm, flush) / steps
+    tl_s = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), steps, warm, flush) / steps
+    out = {
+        "workload": "config4_stress_dag", "K": K, "N": N, "E": E, "uses": e2, "periods": pn,
+        "vitality_ms": vit_s * 1e3, "timeline_ms": tl_s * 1e3,
+        "events_per_s": E / (vit_s + tl_s),
+        "vitality_roofline": {"bound": "hbm", "achieved": vit_bytes / vit_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                              "frac": vit_bytes / vit_s / 1e9 / hbm_peak, "algorithmic_bytes": vit_bytes, "peak_kind": peak_kind},
+        "timeline_roofline": {"bound": "hbm", "achieved": tl_bytes / tl_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                              "frac": tl_bytes / tl_s / 1e9 / hbm_peak, "algorithmic_bytes": tl_bytes, "peak_kind": peak_kind},
+        "l2": "flushed between timed calls",
+    }
+    del tb, ws, v
+    torch.cuda.empty_cache()
+    return out
+
+
+def cpu_baseline(tr):
+    """The oracle (plain tier, one thread) on the same workload, bounded to roughly ten seconds."""
+    from oracle import g10_oracle as O
+    O.build()
+    start, P0, peak, slot = O.timeline(tr)
+    cap = tr.capacity_from_peak(peak)
+    O.plan(tr, cap)
+    reps, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < 10.0 and reps < 200:
+        O.plan(tr, cap)
+        reps += 1
+    dt = time.perf_counter() - t0
+    return {"value": tr.E * reps / dt, "unit": "events/s", "cores": 1, "kind": "oracle",
+            "sample": "whole config-1 plan (plain tier), %d repetitions in %.1f s" % (reps, dt),
+            "plan_ms": dt / reps * 1e3, "host_cores_available": os.cpu_count()}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-stress", action="store_true", help="skip the config-4 pass measurements")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,197 @@
+/*
+ * g10.h -- C ABI of the B200-native planner for G10's compile-time tensor-migration analysis
+ * (G10, MICRO '23: tensor vitality analysis, Section 4.2; GPU memory pressure and the smart tensor
+ * eviction loop, Section 4.3 and Algorithm 1; latest safe prefetch time, Section 4.4).
+ *
+ * Conventions
+ *   - All integers little-endian, all arrays contiguous.  Slots are kernels in trace order; slot k
+ *     occupies the time [start[k], start[k+1]) ns, start being the prefix sum of kernel_ns.
+ *   - Memory space: trace.mem says where EVERY array named by the trace and by the output struct of
+ *     the same call lives.  G10_MEM_DEVICE: device pointers, the call only enqueues work on `stream`
+ *     and returns; results are valid once the caller has synchronised the stream.  G10_MEM_HOST: host
+ *     pointers (pinned memory recommended); the library stages the inputs into the workspace with
+ *     cudaMemcpyAsync, runs the same kernels and copies the outputs back on the same stream; results
+ *     are valid once the stream has been synchronised.
+ *   - Ownership: the caller owns every buffer, the workspace and the stream.  The library allocates
+ *     no device memory, keeps no state between calls and frees nothing.  The workspace `ws` is ALWAYS
+ *     device memory, 256-byte aligned, of at least g10_workspace_bytes(...) bytes; its contents are
+ *     scratch.  Two calls may run concurrently only on different workspaces.
+ *   - Errors: the return value is 0 (enqueued) or a negative G10_ERR_* found on the host before any
+ *     launch.  Errors that depend on the data (tensor id out of range, non-monotone kernel_ptr,
+ *     sizes or durations outside their limits, an output array too small, a grid barrier that timed
+ *     out) are reported in a device status word (`counts[2]`, `summary[7]`, `*status`); outputs are
+ *     then unspecified but every access stays in bounds.  FIT / EXHAUSTED / ALREADY_FITS are results,
+ *     not errors.
+ *   - Limits: 0 <= K, N, E < 2^31 - 1; 1 <= tensor_bytes < 2^40; kernel_ns >= 1; sum(kernel_ns) < 2^44.
+ *     They make every benefit fit 84 bits and every benefit x cost product fit 128 bits.
+ */
+#ifndef G10_H_
+#define G10_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define G10_VERSION 1
+
+#define G10_MEM_DEVICE 0
+#define G10_MEM_HOST 1
+
+/* host-side return codes */
+#define G10_OK 0
+#define G10_ERR_ARG (-1)        /* NULL pointer, negative size, zero bandwidth, unknown enum       */
+#define G10_ERR_LIMIT (-2)      /* K, N or E beyond the limits above                               */
+#define G10_ERR_WORKSPACE (-3)  /* workspace NULL, misaligned or too small                         */
+#define G10_ERR_CUDA (-4)       /* a CUDA runtime call failed (launch, copy, attribute query)      */
+
+/* bits of the device status word (0 = no error) */
+#define G10_DEV_BAD_TENSOR_ID 0x1    /* kernel_tensors entry outside [0, N)                       */
+#define G10_DEV_BAD_KERNEL_PTR 0x2   /* kernel_ptr not nondecreasing from 0 to E                  */
+#define G10_DEV_BAD_BYTES 0x4        /* tensor_bytes outside [1, 2^40)                            */
+#define G10_DEV_BAD_DURATION 0x8     /* kernel_ns < 1 or sum >= 2^44                              */
+#define G10_DEV_USES_OVERFLOW 0x10   /* uses_cap too small (counts[0] holds the need)             */
+#define G10_DEV_PERIODS_OVERFLOW 0x20 /* periods_cap too small (counts[1] holds the need)         */
+#define G10_DEV_PLAN_OVERFLOW 0x40   /* migrations_cap too small (summary[0] holds the need)      */
+#define G10_DEV_TIMEOUT 0x80         /* an internal wait gave up; the kernel returned early       */
+
+/* exit status of the planner (summary[2]) */
+#define G10_ALREADY_FITS 0      /* unplanned peak pressure <= capacity, empty plan                 */
+#define G10_FIT 1               /* peak pressure brought down to <= capacity                       */
+#define G10_EXHAUSTED 2         /* no remaining inactive period relieves any pressure above capacity */
+#define G10_ITERATION_LIMIT 3   /* options.max_iterations reached first                            */
+
+#define G10_DEST_SSD 0
+#define G10_DEST_HOST 1
+
+/* The kernel execution trace (Section 4.2; the instrumented program of Figure 9 shows its shape:
+   an ordered list of kernels, each with its tensor arguments; a tensor may appear twice in one
+   kernel, as the in-place ReLU does). CSR: kernel k lists kernel_tensors[kernel_ptr[k] .. kernel_ptr[k+1]). */
+typedef struct g10_trace {
+    int64_t num_kernels;            /* K                                                            */
+    int64_t num_tensors;            /* N                                                            */
+    int64_t num_events;             /* E = kernel_ptr[K]                                            */
+    const int64_t *kernel_ptr;      /* [K+1]                                                        */
+    const int32_t *kernel_tensors;  /* [E]                                                          */
+    const int64_t *tensor_bytes;    /* [N]                                                          */
+    const int64_t *kernel_ns;       /* [K] profiled execution time of each kernel                   */
+    const uint8_t *tensor_global;   /* [N] 1 = global tensor (weights: allocated at program start,
+                                       never freed), 0 = intermediate; NULL = all intermediate      */
+    int32_t mem;                    /* G10_MEM_DEVICE or G10_MEM_HOST                               */
+} g10_trace;
+
+/* Tensor vitality (Section 4.2).  uses: per tensor the sorted distinct kernels that list it
+   (use_ptr CSR).  A tensor is born at its first use and dead after its last (-1 / -1 / 0 uses if the
+   trace never lists it).  One inactive period (tensor, prev_use u, next_use v) for every two
+   consecutive uses with v - u >= 2; periods are ordered by (tensor, u); period_ptr is the CSR by tensor. */
+typedef struct g10_vitality_out {
+    int32_t *first_use, *last_use, *num_uses;   /* [N]                                              */
+    int64_t *use_ptr;                           /* [N+1]                                            */
+    int32_t *uses;                              /* [uses_cap]   (E always suffices)                 */
+    int64_t uses_cap;
+    int64_t *period_ptr;                        /* [N+1]                                            */
+    int32_t *period_tensor, *period_prev_use, *period_next_use;   /* [periods_cap] (E always suffices) */
+    int64_t periods_cap;
+    int64_t *counts;                            /* [3]: number of uses E', number of periods Pn, device status word */
+} g10_vitality_out;
+
+/* Memory-pressure timeline (Section 4.3: pressure = total size of the tensors resident in GPU memory
+   at a time).  pressure[k] = bytes alive during slot k before any migration: an intermediate tensor
+   from first to last use, a global tensor in every slot if it is used at all. */
+typedef struct g10_timeline_out {
+    int64_t *kernel_start_ns;   /* [K+1] exclusive prefix sum of kernel_ns                          */
+    int64_t *pressure;          /* [K]                                                              */
+    int64_t *peak_bytes;        /* [1] max pressure (0 if K = 0)                                    */
+    int32_t *peak_slot;         /* [1] lowest slot attaining it (-1 if K = 0)                       */
+    int64_t *status;            /* [1] device status word                                           */
+} g10_timeline_out;
+
+/* Candidate geometry of a period for one destination (Algorithm 1: t = tensor_size / BW; Section 4.4:
+   prefetch at the latest safe prefetch time).  t = ceil(bytes * 1e9 / bw) ns (saturated at 2^62).
+   Eviction runs in [t_r, t_r + t), t_r = end of kernel u; prefetch in [t_end - t, t_end), t_end =
+   start of kernel v.  The tensor counts as absent in the slots lying wholly between the two windows,
+   absent_first .. absent_last.  A pair that cannot be used (2t > period length, or no whole slot
+   left) has absent_first = -1, absent_last = -2.  Index [X * Pn + p], X = G10_DEST_SSD / G10_DEST_HOST. */
+typedef struct g10_geometry_out {
+    int64_t *transfer_ns;       /* [2 * Pn]                                                         */
+    int32_t *absent_first;      /* [2 * Pn]                                                         */
+    int32_t *absent_last;       /* [2 * Pn]                                                         */
+} g10_geometry_out;
+
+/* One committed migration (Algorithm 1's "schedule pre-eviction(tensor, destination) at t_r"; the
+   matching prefetch is issued at prefetch_issue_ns).  Records appear in commit order. */
+typedef struct g10_migration {
+    int32_t period, tensor, dest;
+    int32_t absent_first, absent_last;
+    int32_t iteration;
+    int64_t evict_issue_ns, prefetch_issue_ns, transfer_ns;
+} g10_migration;                /* 48 bytes */
+
+typedef struct g10_plan_out {
+    g10_migration *migrations;  /* [migrations_cap] (the number of periods always suffices; E bounds it) */
+    int64_t migrations_cap;
+    int64_t *final_pressure;    /* [K] pressure after every committed migration                     */
+    int64_t *summary;           /* [8]: migrations, scoring rounds, exit status, final peak bytes,
+                                   final peak slot, bytes sent to SSD, bytes sent to host, device status word */
+} g10_plan_out;
+
+typedef struct g10_options {
+    uint64_t host_capacity_bytes;   /* host memory available for evicted tensors; 0 = unlimited      */
+    int64_t max_iterations;         /* 0 = as many as there are periods                              */
+    uint32_t flags;                 /* G10_FLAG_*                                                    */
+    void **stage_events;            /* optional: num_stage_events cudaEvent_t handles owned by the caller; the
+                                       planner records them on `stream` at its stage boundaries, in order:
+                                       start, after slot clock + vitality, after the pressure timeline,
+                                       after candidate geometry, after the greedy loop (extra handles unused) */
+    int32_t num_stage_events;
+} g10_options;
+
+#define G10_NUM_PLAN_STAGES 5
+
+#define G10_FLAG_RESCORE_ALL 0x1    /* rescore every live period every iteration (Algorithm 1 as
+                                       printed) instead of only those whose score can have changed;
+                                       the plan is identical, the run is slower                     */
+
+#define G10_WS_VITALITY 0
+#define G10_WS_TIMELINE 1
+#define G10_WS_PLAN 2
+#define G10_WS_GEOMETRY 3
+
+/* Section 4.2, tensor vitality analysis. */
+int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, size_t ws_bytes, void *stream);
+
+/* Section 4.3, GPU memory pressure over time (difference array of signed sizes + prefix scan). */
+int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, void *ws, size_t ws_bytes, void *stream);
+
+/* Algorithm 1 / Section 4.4: transfer times and absent-slot ranges of every period for both
+   destinations.  All pointers are DEVICE pointers; kernel_start_ns [K+1] and the period arrays come
+   from the two calls above.  Needs no workspace. */
+int32_t g10_candidate_geometry(int64_t num_kernels, int64_t num_periods, const int64_t *kernel_start_ns,
+                               const int64_t *tensor_bytes, const int32_t *period_tensor,
+                               const int32_t *period_prev_use, const int32_t *period_next_use,
+                               uint64_t host_bw, uint64_t ssd_bw, g10_geometry_out *out, void *stream);
+
+/* Algorithm 1, smart tensor eviction: vitality, pressure, geometry, then the greedy loop -- until the
+   peak pressure fits gpu_capacity_bytes or no period relieves pressure above it: score every live
+   period (destination SSD first, host when the SSD channel is booked or too slow; benefit = pressure
+   above capacity removed, in byte*ns; cost = eviction + prefetch time), take the best benefit/cost
+   ratio (exact comparison, ties to the lowest period index), commit it (pressure, channel time, host
+   occupancy) and erase the period.  Bandwidths in bytes per second. */
+int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
+                            const g10_options *options /* NULL = defaults */, g10_plan_out *out,
+                            void *ws, size_t ws_bytes, void *stream);
+
+/* Bytes of device workspace the call `which` (G10_WS_*) needs for a trace of K kernels, N tensors,
+   E events whose arrays live in `mem`. */
+int32_t g10_workspace_bytes(int32_t which, int64_t num_kernels, int64_t num_tensors, int64_t num_events,
+                            int32_t mem, size_t *out_bytes);
+
+const char *g10_strerror(int32_t code);
+int32_t g10_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* G10_H_ */

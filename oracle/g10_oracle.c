@@ -298,7 +298,7 @@ static void peak_of(const int64_t *P, int64_t K, int64_t *pk, int64_t *ps)
 }
 
 /* ---- a binary max-heap of (bound ratio, index) for the lazy tier --------------------------- */
-typedef struct { u128 ben; int64_t cost; int64_t idx; } hnode;
+typedef struct { u128 ben; int64_t cost; int64_t idx; int64_t ver; } hnode;
 static int hbeats(const hnode *x, const hnode *y) { return beats(x->ben, x->cost, x->idx, y->ben, y->cost, y->idx); }
 static void hpush(hnode *h, int64_t *n, hnode v)
 {
@@ -319,37 +319,22 @@ static hnode hpop(hnode *h, int64_t *n)
     return top;
 }
 
-/* Lazy tier.  For a fixed destination the absent range and the cost never change, pressure only
-   falls, and booked channel time / host occupancy only rise: each destination's ratio can only
-   fall and a destination once refused stays refused.  So the larger of the ratios of the
-   destinations still open to a period bounds every score the period can have later (it may fall
-   back from SSD to host, and a host transfer is cheaper).  lazy_eval computes, against the
-   current state, that bound and the period's true score (first admissible destination, SSD
-   before host).  Returns 0 when no destination is left or the bound has no benefit: the period
-   can be forgotten. */
-static int lazy_eval(const plan_state *S, int64_t p, char *open, hnode *bound, u128 *tb, int64_t *tc, int *tX)
-{
-    int have = 0;
-    *tX = -1; *tb = 0; *tc = 1;
-    for (int X = 0; X < 2; ++X) {
-        if (!open[2 * p + X]) continue;
-        if (!admissible(S, p, X)) { open[2 * p + X] = 0; continue; }
-        u128 b = benefit_of(S, p, X);
-        int64_t c = 2 * S->geo[X][p].t;
-        if (*tX < 0) { *tX = X; *tb = b; *tc = c; }
-        if (!have || beats(b, c, 0, bound->ben, bound->cost, 0)) { bound->ben = b; bound->cost = c; }
-        have = 1;
-    }
-    bound->idx = p;
-    return have && bound->ben > 0;
-}
+/* Lazy tier.  Pressure only falls and booked channel time / host occupancy only rise, so for a
+   fixed destination a period's ratio can only fall: the ratio computed earlier is an upper bound
+   of the current one, as long as the period's destination is still the one the rule picks.  The
+   destination is therefore kept exact: after every commit, each live period whose transfer
+   windows (or, with a finite host memory, whose whole period) share a slot with what the commit
+   booked on the same device is re-examined at once.  slots_meet tells whether two slot ranges
+   intersect. */
+static int slots_meet(int64_t a0, int64_t a1, int64_t b0, int64_t b1) { return a0 <= b1 && b0 <= a1 && a0 <= a1 && b0 <= b1; }
 
 /* ------------------------------------------------------------------------------------------
  * The planner (Algorithm 1).  Each iteration: stop if the peak fits; score every live period;
  * take the best benefit/cost ratio; book it; erase the period.  Stops EXHAUSTED when no live
  * period has a positive benefit ("no more beneficial eviction candidates").
  *   lazy = 0 : the definition (every live period is rescored every iteration).
- *   lazy = 1 : same result, periods rescored only when their stale bound is on top of a heap.
+ *   lazy = 1 : same result, periods rescored only when their earlier score (an upper bound) is on
+ *              top of a heap; destinations are kept exact after every commit.
  * win_benefit (optional, 2 words per record: low, high) and win_cost (optional) report the
  * winner's score for the invariant tests.
  * summary[8] = { migrations, scoring rounds, exit status, final peak, final peak slot,
@@ -399,15 +384,20 @@ int32_t g10o_plan(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t
     int fits_always = gpu_capacity_bytes >= ((uint64_t)1 << 63);
     S.cap = fits_always ? INT64_MAX : (int64_t)gpu_capacity_bytes;
 
-    hnode *heap = NULL, *popped = NULL; int64_t hn = 0; char *open = NULL;
+    hnode *heap = NULL, *popped = NULL; int64_t hn = 0;
+    int *dest = NULL; int64_t *ver = NULL;
     if (lazy) {
-        heap = (hnode *)malloc(sizeof(hnode) * nP);
-        open = (char *)malloc(2 * nP);
-        memset(open, 1, 2 * nP);
-        popped = (hnode *)malloc(sizeof(hnode) * nP);
+        /* every period enters the heap once, plus once per change of destination (at most two) */
+        heap = (hnode *)malloc(sizeof(hnode) * (3 * nP + 1));
+        popped = (hnode *)malloc(sizeof(hnode) * (3 * nP + 1));
+        dest = (int *)malloc(sizeof(int) * nP);
+        ver = (int64_t *)calloc(nP, sizeof(int64_t));
         for (int64_t p = 0; p < Pn; ++p) {
-            hnode nd; u128 tb; int64_t tc; int tX;
-            if (lazy_eval(&S, p, open, &nd, &tb, &tc, &tX)) hpush(heap, &hn, nd);
+            dest[p] = choose_destination(&S, p);
+            if (dest[p] < 0) { alive[p] = 0; continue; }
+            hnode nd; nd.idx = p; nd.ver = 0;
+            nd.ben = benefit_of(&S, p, dest[p]); nd.cost = 2 * S.geo[dest[p]][p].t;
+            if (nd.ben > 0) hpush(heap, &hn, nd);
         }
     }
 
@@ -429,18 +419,19 @@ int32_t g10o_plan(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t
                 if (best < 0 || beats(b, c, p, bestB, bestC, best)) { best = p; bestX = X; bestB = b; bestC = c; }
             }
         } else {
-            /* Pop while the top bound could still beat the best true score seen this iteration;
+            /* Pop while the top bound could still beat the best exact score seen this iteration;
                every popped period is rescored against the current state.  What stays in the heap
-               has bound <= best, hence true score <= best. */
+               has bound <= best, hence score <= best. */
             int64_t npop = 0;
             while (hn > 0 && (best < 0 || beats(heap[0].ben, heap[0].cost, heap[0].idx, bestB, bestC, best))) {
                 hnode top = hpop(heap, &hn);
-                hnode bd; u128 tb; int64_t tc; int tX;
-                if (!lazy_eval(&S, top.idx, open, &bd, &tb, &tc, &tX)) continue;
-                popped[npop++] = bd;
-                if (tb > 0 && (best < 0 || beats(tb, tc, top.idx, bestB, bestC, best))) {
-                    best = top.idx; bestX = tX; bestB = tb; bestC = tc;
-                }
+                int64_t p = top.idx;
+                if (!alive[p] || top.ver != ver[p]) continue;          /* superseded entry */
+                hnode nd; nd.idx = p; nd.ver = ver[p];
+                nd.ben = benefit_of(&S, p, dest[p]); nd.cost = 2 * S.geo[dest[p]][p].t;
+                if (nd.ben == 0) continue;            /* stays out until its destination changes */
+                popped[npop++] = nd;
+                if (best < 0 || beats(nd.ben, nd.cost, p, bestB, bestC, best)) { best = p; bestX = dest[p]; bestB = nd.ben; bestC = nd.cost; }
             }
             for (int64_t j = 0; j < npop; ++j) if (popped[j].idx != best) hpush(heap, &hn, popped[j]);
         }
@@ -456,6 +447,26 @@ int32_t g10o_plan(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t
         } else rc = -1;
         commit(&S, best, bestX);
         alive[best] = 0;
+        if (lazy) {
+            /* keep every destination exact: re-examine the periods the new bookings can affect */
+            const geo_t *gw = &S.geo[bestX][best];
+            int64_t aw = pu[best] + 1, bw = pv[best] - 1;
+            for (int64_t p = 0; p < Pn; ++p) {
+                if (!alive[p] || dest[p] != bestX) continue;
+                const geo_t *gp = &S.geo[bestX][p];
+                int64_t ap_ = pu[p] + 1, bp_ = pv[p] - 1;
+                int hit = slots_meet(ap_, gp->a_abs - 1, aw, gw->a_abs - 1) || slots_meet(gp->b_abs + 1, bp_, gw->b_abs + 1, bw);
+                if (!hit && bestX == DEST_HOST && S.host_capacity != 0) hit = slots_meet(ap_, bp_, aw, bw);
+                if (!hit) continue;
+                int nd_ = choose_destination(&S, p);
+                if (nd_ == dest[p]) continue;
+                dest[p] = nd_; ver[p] += 1;
+                if (nd_ < 0) { alive[p] = 0; continue; }
+                hnode nn; nn.idx = p; nn.ver = ver[p];
+                nn.ben = benefit_of(&S, p, nd_); nn.cost = 2 * S.geo[nd_][p].t;
+                if (nn.ben > 0) hpush(heap, &hn, nn);
+            }
+        }
         bytes_to[bestX] += tensor_bytes[pt[best]];
         n_mig += 1;
     }
@@ -467,6 +478,6 @@ int32_t g10o_plan(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t
     free(start); free(first); free(last); free(nuse); free(use_ptr); free(per_ptr); free(uses);
     free(pt); free(pu); free(pv); free(S.geo[0]); free(S.geo[1]);
     for (int c = 0; c < 4; ++c) free(S.busy[c]);
-    free(S.hocc); free(alive); free(heap); free(open); free(popped);
+    free(S.hocc); free(alive); free(heap); free(popped); free(dest); free(ver);
     return rc;
 }

@@ -1,0 +1,351 @@
+// The C ABI: argument checks, workspace layout, host-buffer staging and the launch sequence of each call.
+#include <cstring>
+
+#include "g10_internal.h"
+
+namespace g10 {
+namespace {
+
+struct Sizes {
+    int64_t K, N, E;
+    bool host;
+};
+
+// Lays the workspace out; with base == nullptr only measures it.
+struct Carver {
+    char *base;
+    size_t off = 0;
+    explicit Carver(void *b) : base((char *)b) {}
+    template <typename T>
+    T *take(size_t count)
+    {
+        off = align_up(off);
+        T *p = base ? (T *)(base + off) : nullptr;
+        off += sizeof(T) * (count ? count : 1);
+        return p;
+    }
+};
+
+void carve_scan(Carver &c, ScanSlot &s, int64_t tiles, int nv)
+{
+    s.ticket = c.take<unsigned>(1);
+    s.done = c.take<unsigned>(1);
+    s.flag = c.take<unsigned>((size_t)tiles);
+    s.agg = c.take<long long>((size_t)tiles * nv);
+    s.incl = c.take<long long>((size_t)tiles * nv);
+}
+
+size_t carve(void *base, const Sizes &z, Workspace &w)
+{
+    std::memset(&w, 0, sizeof(w));
+    Carver c(base);
+    const size_t K = (size_t)z.K, N = (size_t)z.N, E = (size_t)z.E;
+    const size_t heavy = E / (kHeavyThreshold + 1) + 1;
+    const int64_t ktiles = tiles_of(z.K, 2048), ntiles = tiles_of(z.N, 2048), etiles = tiles_of(z.N, 1024);
+    // zero-initialised region
+    w.zero_begin = c.base ? c.base : nullptr;
+    w.status = c.take<ull>(1);
+    w.heavy_count = c.take<unsigned>(1);
+    w.peak_key = c.take<int>(1);
+    w.barrier = c.take<unsigned>(4);
+    carve_scan(c, w.clock_scan, ktiles, 1);
+    carve_scan(c, w.count_scan, ntiles, 1);
+    carve_scan(c, w.emit_scan, etiles, 2);
+    carve_scan(c, w.pressure_scan, ktiles, 1);
+    w.cnt = c.take<int32_t>(N);
+    w.diff = c.take<int64_t>(K + 1);
+    w.busy = c.take<int64_t>(4 * K);
+    w.hocc = c.take<int64_t>(K);
+    w.dead = c.take<unsigned char>(E);
+    w.zero_bytes = align_up(c.off);
+    // scratch
+    w.raw_ptr = c.take<int32_t>(N + 1);
+    w.raw_uses = c.take<int32_t>(E);
+    w.heavy_list = c.take<int32_t>(heavy);
+    w.heavy_info = c.take<int32_t>(2 * heavy);
+    w.tile_max = c.take<int64_t>((size_t)ktiles);
+    w.tile_slot = c.take<int32_t>((size_t)ktiles);
+    w.first_use = c.take<int32_t>(N);
+    w.last_use = c.take<int32_t>(N);
+    w.num_uses = c.take<int32_t>(N);
+    w.use_ptr = c.take<int64_t>(N + 1);
+    w.period_ptr = c.take<int64_t>(N + 1);
+    w.uses = c.take<int32_t>(E);
+    w.period_tensor = c.take<int32_t>(E);
+    w.period_prev_use = c.take<int32_t>(E);
+    w.period_next_use = c.take<int32_t>(E);
+    w.counts = c.take<int64_t>(4);
+    w.start = c.take<int64_t>(K + 1);
+    w.pressure = c.take<int64_t>(K);
+    w.peak_bytes = c.take<int64_t>(1);
+    w.peak_slot = c.take<int32_t>(2);
+    w.geo_t = c.take<int64_t>(2 * E);
+    w.geo_a = c.take<int32_t>(2 * E);
+    w.geo_b = c.take<int32_t>(2 * E);
+    w.proposals = c.take<Proposal>(kMaxPlanBlocks);
+    w.peak_part = c.take<int64_t>(kMaxPlanBlocks);
+    w.summary = c.take<int64_t>(8);
+    if (z.host) {
+        w.migrations = c.take<g10_migration>(E);
+        w.s_kernel_ptr = c.take<int64_t>(K + 1);
+        w.s_kernel_tensors = c.take<int32_t>(E);
+        w.s_tensor_bytes = c.take<int64_t>(N);
+        w.s_kernel_ns = c.take<int64_t>(K);
+        w.s_tensor_global = c.take<uint8_t>(N);
+    }
+    return align_up(c.off);
+}
+
+int32_t check_trace(const g10_trace *t)
+{
+    if (!t) return G10_ERR_ARG;
+    if (t->num_kernels < 0 || t->num_tensors < 0 || t->num_events < 0) return G10_ERR_ARG;
+    if (t->mem != G10_MEM_DEVICE && t->mem != G10_MEM_HOST) return G10_ERR_ARG;
+    const int64_t lim = ((int64_t)1 << 31) - 1;
+    if (t->num_kernels >= lim || t->num_tensors >= lim || t->num_events >= lim) return G10_ERR_LIMIT;
+    if (!t->kernel_ptr) return G10_ERR_ARG;
+    if (t->num_events > 0 && !t->kernel_tensors) return G10_ERR_ARG;
+    if (t->num_tensors > 0 && !t->tensor_bytes) return G10_ERR_ARG;
+    if (t->num_kernels > 0 && !t->kernel_ns) return G10_ERR_ARG;
+    if (t->num_events > 0 && (t->num_kernels == 0 || t->num_tensors == 0)) return G10_ERR_ARG;
+    return G10_OK;
+}
+
+int32_t check_ws(int32_t which, const g10_trace *t, void *ws, size_t ws_bytes)
+{
+    size_t need = 0;
+    const int32_t rc = g10_workspace_bytes(which, t->num_kernels, t->num_tensors, t->num_events, t->mem, &need);
+    if (rc != G10_OK) return rc;
+    if (!ws || ((uintptr_t)ws % kAlign) != 0 || ws_bytes < need) return G10_ERR_WORKSPACE;
+    return G10_OK;
+}
+
+#define CU(x)                                   \
+    do {                                        \
+        if ((x) != cudaSuccess) return G10_ERR_CUDA; \
+    } while (0)
+
+// Prepares the workspace and returns the device view of the trace (staging it first in host mode).
+int32_t begin_call(const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, cudaStream_t s)
+{
+    Sizes z{t->num_kernels, t->num_tensors, t->num_events, t->mem == G10_MEM_HOST};
+    carve(ws, z, w);
+    CU(cudaMemsetAsync(w.zero_begin, 0, w.zero_bytes, s));
+    d.K = z.K; d.N = z.N; d.E = z.E;
+    if (!z.host) {
+        d.kernel_ptr = t->kernel_ptr; d.kernel_tensors = t->kernel_tensors; d.tensor_bytes = t->tensor_bytes;
+        d.kernel_ns = t->kernel_ns; d.tensor_global = t->tensor_global;
+    } else {
+        CU(cudaMemcpyAsync(w.s_kernel_ptr, t->kernel_ptr, sizeof(int64_t) * (size_t)(z.K + 1), cudaMemcpyHostToDevice, s));
+        if (z.E) CU(cudaMemcpyAsync(w.s_kernel_tensors, t->kernel_tensors, sizeof(int32_t) * (size_t)z.E, cudaMemcpyHostToDevice, s));
+        if (z.N) CU(cudaMemcpyAsync(w.s_tensor_bytes, t->tensor_bytes, sizeof(int64_t) * (size_t)z.N, cudaMemcpyHostToDevice, s));
+        if (z.K) CU(cudaMemcpyAsync(w.s_kernel_ns, t->kernel_ns, sizeof(int64_t) * (size_t)z.K, cudaMemcpyHostToDevice, s));
+        if (z.N && t->tensor_global)
+            CU(cudaMemcpyAsync(w.s_tensor_global, t->tensor_global, (size_t)z.N, cudaMemcpyHostToDevice, s));
+        d.kernel_ptr = w.s_kernel_ptr; d.kernel_tensors = w.s_kernel_tensors; d.tensor_bytes = w.s_tensor_bytes;
+        d.kernel_ns = w.s_kernel_ns; d.tensor_global = t->tensor_global ? w.s_tensor_global : nullptr;
+    }
+    return G10_OK;
+}
+
+template <typename T>
+cudaError_t d2h(T *dst, const T *src, size_t count, cudaStream_t s)
+{
+    if (count == 0 || dst == nullptr) return cudaSuccess;
+    return cudaMemcpyAsync(dst, src, sizeof(T) * count, cudaMemcpyDeviceToHost, s);
+}
+
+}  // namespace
+}  // namespace g10
+
+using namespace g10;
+
+extern "C" {
+
+int32_t g10_version(void) { return G10_VERSION; }
+
+const char *g10_strerror(int32_t code)
+{
+    switch (code) {
+        case G10_OK: return "ok";
+        case G10_ERR_ARG: return "invalid argument";
+        case G10_ERR_LIMIT: return "trace dimensions beyond the supported limits";
+        case G10_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case G10_ERR_CUDA: return "a CUDA runtime call failed";
+        default: return "unknown error code";
+    }
+}
+
+int32_t g10_workspace_bytes(int32_t which, int64_t K, int64_t N, int64_t E, int32_t mem, size_t *out_bytes)
+{
+    if (!out_bytes || K < 0 || N < 0 || E < 0) return G10_ERR_ARG;
+    if (which < G10_WS_VITALITY || which > G10_WS_GEOMETRY) return G10_ERR_ARG;
+    if (mem != G10_MEM_DEVICE && mem != G10_MEM_HOST) return G10_ERR_ARG;
+    const int64_t lim = ((int64_t)1 << 31) - 1;
+    if (K >= lim || N >= lim || E >= lim) return G10_ERR_LIMIT;
+    if (which == G10_WS_GEOMETRY) { *out_bytes = 0; return G10_OK; }
+    // one layout serves the three calls (the planner uses all of it; the others a prefix-independent subset)
+    Workspace w;
+    Sizes z{K, N, E, mem == G10_MEM_HOST};
+    *out_bytes = carve(nullptr, z, w);
+    return G10_OK;
+}
+
+int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, size_t ws_bytes, void *stream)
+{
+    int32_t rc = check_trace(trace);
+    if (rc != G10_OK) return rc;
+    if (!out || !out->first_use || !out->last_use || !out->num_uses || !out->use_ptr || !out->period_ptr || !out->counts)
+        return G10_ERR_ARG;
+    if (out->uses_cap < 0 || out->periods_cap < 0) return G10_ERR_ARG;
+    if ((out->uses_cap > 0 && !out->uses) ||
+        (out->periods_cap > 0 && (!out->period_tensor || !out->period_prev_use || !out->period_next_use)))
+        return G10_ERR_ARG;
+    rc = check_ws(G10_WS_VITALITY, trace, ws, ws_bytes);
+    if (rc != G10_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    Workspace w;
+    DeviceTrace d;
+    rc = begin_call(trace, ws, w, d, s);
+    if (rc != G10_OK) return rc;
+    const bool host = trace->mem == G10_MEM_HOST;
+    VitalityBuffers vb;
+    if (!host) {
+        vb = VitalityBuffers{out->first_use, out->last_use, out->num_uses, out->use_ptr, out->uses, out->uses_cap, out->period_ptr,
+                             out->period_tensor, out->period_prev_use, out->period_next_use, out->periods_cap, out->counts};
+    } else {
+        const int64_t ucap = out->uses_cap < d.E ? out->uses_cap : d.E, pcap = out->periods_cap < d.E ? out->periods_cap : d.E;
+        vb = VitalityBuffers{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, ucap, w.period_ptr,
+                             w.period_tensor, w.period_prev_use, w.period_next_use, pcap, w.counts};
+    }
+    CU(launch_vitality(d, w, vb, s));
+    CU(launch_publish_status(w, vb.counts + 2, s));
+    if (host) {
+        int64_t counts[3];
+        CU(cudaMemcpyAsync(counts, w.counts, sizeof(counts), cudaMemcpyDeviceToHost, s));
+        CU(cudaStreamSynchronize(s));
+        std::memcpy(out->counts, counts, sizeof(counts));
+        const size_t N = (size_t)d.N;
+        const size_t nu = (size_t)(counts[0] < vb.uses_cap ? counts[0] : vb.uses_cap);
+        const size_t np = (size_t)(counts[1] < vb.periods_cap ? counts[1] : vb.periods_cap);
+        CU(d2h(out->first_use, w.first_use, N, s));
+        CU(d2h(out->last_use, w.last_use, N, s));
+        CU(d2h(out->num_uses, w.num_uses, N, s));
+        CU(d2h(out->use_ptr, w.use_ptr, N + 1, s));
+        CU(d2h(out->period_ptr, w.period_ptr, N + 1, s));
+        CU(d2h(out->uses, w.uses, nu, s));
+        CU(d2h(out->period_tensor, w.period_tensor, np, s));
+        CU(d2h(out->period_prev_use, w.period_prev_use, np, s));
+        CU(d2h(out->period_next_use, w.period_next_use, np, s));
+        CU(cudaStreamSynchronize(s));
+    }
+    return G10_OK;
+}
+
+int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, void *ws, size_t ws_bytes, void *stream)
+{
+    int32_t rc = check_trace(trace);
+    if (rc != G10_OK) return rc;
+    if (!out || !out->kernel_start_ns || !out->peak_bytes || !out->peak_slot || !out->status) return G10_ERR_ARG;
+    if (trace->num_kernels > 0 && !out->pressure) return G10_ERR_ARG;
+    rc = check_ws(G10_WS_TIMELINE, trace, ws, ws_bytes);
+    if (rc != G10_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    Workspace w;
+    DeviceTrace d;
+    rc = begin_call(trace, ws, w, d, s);
+    if (rc != G10_OK) return rc;
+    const bool host = trace->mem == G10_MEM_HOST;
+    int64_t *start = host ? w.start : out->kernel_start_ns;
+    int64_t *P = host ? w.pressure : out->pressure;
+    int64_t *pk = host ? w.peak_bytes : out->peak_bytes;
+    int32_t *ps = host ? w.peak_slot : out->peak_slot;
+    int64_t *st = host ? w.counts + 2 : out->status;
+    CU(launch_slot_clock(d, w, start, s));
+    CU(launch_first_last(d, w, w.first_use, w.last_use, s));
+    CU(launch_pressure(d, w, w.first_use, w.last_use, P, pk, ps, s));
+    CU(launch_publish_status(w, st, s));
+    if (host) {
+        CU(d2h(out->kernel_start_ns, w.start, (size_t)d.K + 1, s));
+        CU(d2h(out->pressure, w.pressure, (size_t)d.K, s));
+        CU(d2h(out->peak_bytes, w.peak_bytes, 1, s));
+        CU(d2h(out->peak_slot, w.peak_slot, 1, s));
+        CU(d2h(out->status, w.counts + 2, 1, s));
+        CU(cudaStreamSynchronize(s));
+    }
+    return G10_OK;
+}
+
+int32_t g10_candidate_geometry(int64_t K, int64_t Pn, const int64_t *kernel_start_ns, const int64_t *tensor_bytes,
+                               const int32_t *period_tensor, const int32_t *period_prev_use, const int32_t *period_next_use,
+                               uint64_t host_bw, uint64_t ssd_bw, g10_geometry_out *out, void *stream)
+{
+    if (K < 0 || Pn < 0 || host_bw == 0 || ssd_bw == 0 || !out) return G10_ERR_ARG;
+    if (Pn == 0) return G10_OK;
+    if (!kernel_start_ns || !tensor_bytes || !period_tensor || !period_prev_use || !period_next_use) return G10_ERR_ARG;
+    if (!out->transfer_ns || !out->absent_first || !out->absent_last) return G10_ERR_ARG;
+    CU(launch_geometry(K, Pn, nullptr, kernel_start_ns, tensor_bytes, period_tensor, period_prev_use, period_next_use, host_bw, ssd_bw,
+                       Pn, out->transfer_ns, out->absent_first, out->absent_last, (cudaStream_t)stream));
+    return G10_OK;
+}
+
+int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
+                            const g10_options *options, g10_plan_out *out, void *ws, size_t ws_bytes, void *stream)
+{
+    int32_t rc = check_trace(trace);
+    if (rc != G10_OK) return rc;
+    if (host_bw == 0 || ssd_bw == 0 || !out || !out->summary) return G10_ERR_ARG;
+    if (out->migrations_cap < 0 || (out->migrations_cap > 0 && !out->migrations)) return G10_ERR_ARG;
+    if (trace->num_kernels > 0 && !out->final_pressure) return G10_ERR_ARG;
+    if (options && options->max_iterations < 0) return G10_ERR_ARG;
+    rc = check_ws(G10_WS_PLAN, trace, ws, ws_bytes);
+    if (rc != G10_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    Workspace w;
+    DeviceTrace d;
+    rc = begin_call(trace, ws, w, d, s);
+    if (rc != G10_OK) return rc;
+    const bool host = trace->mem == G10_MEM_HOST;
+    VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
+                       w.period_tensor, w.period_prev_use, w.period_next_use, d.E, w.counts};
+    PlanParams pp;
+    pp.gpu_capacity_bytes = gpu_capacity_bytes; pp.host_bw = host_bw; pp.ssd_bw = ssd_bw;
+    pp.host_capacity_bytes = options ? options->host_capacity_bytes : 0;
+    pp.max_iterations = options ? options->max_iterations : 0;
+    pp.flags = options ? options->flags : 0;
+    pp.migrations = host ? w.migrations : out->migrations;
+    pp.migrations_cap = host ? (out->migrations_cap < d.E ? out->migrations_cap : d.E) : out->migrations_cap;
+    pp.final_pressure = host ? w.pressure : out->final_pressure;
+    pp.summary = host ? w.summary : out->summary;
+    // optional caller-owned events at the stage boundaries
+    auto mark = [&](int stage) -> cudaError_t {
+        if (options && options->stage_events && stage < options->num_stage_events && options->stage_events[stage])
+            return cudaEventRecord((cudaEvent_t)options->stage_events[stage], s);
+        return cudaSuccess;
+    };
+    CU(mark(0));
+    CU(launch_slot_clock(d, w, w.start, s));
+    CU(launch_vitality(d, w, vb, s));
+    CU(mark(1));
+    CU(launch_pressure(d, w, w.first_use, w.last_use, pp.final_pressure, w.peak_bytes, w.peak_slot, s));
+    CU(mark(2));
+    CU(launch_geometry(d.K, d.E, w.counts + 1, w.start, d.tensor_bytes, w.period_tensor, w.period_prev_use, w.period_next_use,
+                       host_bw, ssd_bw, d.E > 0 ? d.E : 1, w.geo_t, w.geo_a, w.geo_b, s));
+    CU(mark(3));
+    CU(launch_plan_loop(d, w, pp, s));
+    CU(mark(4));
+    CU(launch_publish_status(w, pp.summary + 7, s));
+    if (host) {
+        int64_t summary[8];
+        CU(cudaMemcpyAsync(summary, w.summary, sizeof(summary), cudaMemcpyDeviceToHost, s));
+        CU(cudaStreamSynchronize(s));
+        std::memcpy(out->summary, summary, sizeof(summary));
+        const size_t nm = (size_t)(summary[0] < pp.migrations_cap ? summary[0] : pp.migrations_cap);
+        CU(d2h(out->migrations, w.migrations, nm, s));
+        CU(d2h(out->final_pressure, w.pressure, (size_t)d.K, s));
+        CU(cudaStreamSynchronize(s));
+    }
+    return G10_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,125 @@
+// Host-side declarations shared by the translation units of the library: workspace layout and the
+// launchers of each pass.  Everything here works on DEVICE pointers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "g10.h"
+
+namespace g10 {
+
+typedef unsigned long long ull;
+
+constexpr size_t kAlign = 256;
+constexpr int kHeavyThreshold = 32;      // tensors with more raw uses than this are sorted by a whole block
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline int64_t tiles_of(int64_t n, int64_t tile) { return n <= 0 ? 1 : (n + tile - 1) / tile; }
+
+// One scan's look-back state inside the zero-initialised part of the workspace.
+struct ScanSlot {
+    unsigned *ticket;
+    unsigned *done;
+    unsigned *flag;
+    long long *agg;
+    long long *incl;
+};
+
+struct Proposal {          // a block's best candidate of one scoring round (32 bytes)
+    ull ben_lo, ben_hi;
+    ull cost;
+    int idx;               // -1 = none
+    int dest;
+};
+
+// Device views of a trace and of the intermediate arrays; filled by carve() in g10_api.cu.
+struct Workspace {
+    // --- zero-initialised region (one memset per call) ---
+    char *zero_begin;
+    size_t zero_bytes;
+    ull *status;                 // device status word
+    unsigned *heavy_count;
+    int *peak_key;               // K - lowest peak slot (0 = none), reduced with atomicMax
+    void *barrier;               // GridBarrier
+    ScanSlot clock_scan, count_scan, emit_scan, pressure_scan;
+    int32_t *cnt;                // [N] raw use counts, then scatter cursor, then heavy slot index
+    int64_t *diff;               // [K+1] signed-size difference array
+    int64_t *busy;               // [4*K] booked channel time per slot
+    int64_t *hocc;               // [K] host-memory occupancy per slot
+    unsigned char *dead;         // [E] period erased
+    // --- uninitialised region ---
+    int32_t *raw_ptr;            // [N+1]
+    int32_t *raw_uses;           // [E]
+    int32_t *heavy_list;         // [E/33+1] tensor ids
+    int32_t *heavy_info;         // [2*(E/33+1)] distinct uses, periods
+    int64_t *tile_max;           // [tiles(K)]
+    int32_t *tile_slot;          // [tiles(K)]
+    // vitality / timeline outputs when the caller did not ask for them (planner) or passed host memory
+    int32_t *first_use, *last_use, *num_uses;
+    int64_t *use_ptr, *period_ptr;
+    int32_t *uses, *period_tensor, *period_prev_use, *period_next_use;
+    int64_t *counts;             // [3]
+    int64_t *start;              // [K+1]
+    int64_t *pressure;           // [K]
+    int64_t *peak_bytes;         // [1]
+    int32_t *peak_slot;          // [1]
+    int64_t *geo_t;              // [2*E]
+    int32_t *geo_a, *geo_b;      // [2*E]
+    Proposal *proposals;         // [max blocks]
+    int64_t *peak_part;          // [max blocks]
+    g10_migration *migrations;   // host mode only
+    int64_t *summary;            // [8]
+    // staged copies of the trace (host mode only)
+    int64_t *s_kernel_ptr, *s_tensor_bytes, *s_kernel_ns;
+    int32_t *s_kernel_tensors;
+    uint8_t *s_tensor_global;
+};
+
+struct DeviceTrace {
+    int64_t K, N, E;
+    const int64_t *kernel_ptr;
+    const int32_t *kernel_tensors;
+    const int64_t *tensor_bytes;
+    const int64_t *kernel_ns;
+    const uint8_t *tensor_global;
+};
+
+struct VitalityBuffers {
+    int32_t *first_use, *last_use, *num_uses;
+    int64_t *use_ptr;
+    int32_t *uses;
+    int64_t uses_cap;
+    int64_t *period_ptr;
+    int32_t *period_tensor, *period_prev_use, *period_next_use;
+    int64_t periods_cap;
+    int64_t *counts;   // [3]
+};
+
+struct PlanParams {
+    uint64_t gpu_capacity_bytes, host_bw, ssd_bw, host_capacity_bytes;
+    int64_t max_iterations;
+    uint32_t flags;
+    g10_migration *migrations;
+    int64_t migrations_cap;
+    int64_t *final_pressure;
+    int64_t *summary;
+};
+
+constexpr int kMaxPlanBlocks = 1024;
+
+// passes (g10_passes.cu)
+cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);
+cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
+cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s);
+cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use,
+                            int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);
+cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, const int64_t *start, const int64_t *tensor_bytes,
+                            const int32_t *per_t, const int32_t *per_u, const int32_t *per_v, uint64_t host_bw, uint64_t ssd_bw,
+                            int64_t stride, int64_t *geo_t, int32_t *geo_a, int32_t *geo_b, cudaStream_t s);
+// planner (g10_planner.cu)
+cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
+int plan_loop_max_blocks();
+cudaError_t launch_publish_status(const Workspace &w, int64_t *dst, cudaStream_t s);
+
+}  // namespace g10

@@ -1,0 +1,649 @@
+// The HBM-bound passes: slot clock (Section 4.2: kernel times measure the inactive periods), tensor
+// vitality (Section 4.2: born / dead / inactive periods), memory-pressure timeline (Section 4.3) and
+// candidate geometry (Algorithm 1's t = size / BW; Section 4.4's latest safe prefetch time).
+#include "g10_device.cuh"
+#include "g10_internal.h"
+
+namespace g10 {
+
+// =============================================================================================
+// Slot clock: start = exclusive prefix sum of kernel_ns, start[K] = total.  Also checks that
+// kernel_ptr runs from 0 to E without decreasing and that every duration is >= 1.
+// =============================================================================================
+__global__ void __launch_bounds__(kScanThreads) k_slot_clock(int64_t K, int64_t E, const int64_t *__restrict__ dur,
+                                                             const int64_t *__restrict__ kptr, int64_t *__restrict__ start,
+                                                             TileState<1> st, int tiles, ull *status)
+{
+    const int tile = next_tile(st.ticket);
+    if (tile >= tiles) return;
+    const int64_t base = (int64_t)tile * kScanTile + (int64_t)threadIdx.x * kScanItems;
+    long long v[kScanItems];
+    Sums<1> mine;
+    mine.v[0] = 0;
+    ull bad = 0;
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        const int64_t k = base + j;
+        v[j] = 0;
+        if (k < K) {
+            v[j] = dur[k];
+            if (v[j] < 1 || v[j] >= ((long long)1 << 44)) { bad |= G10_DEV_BAD_DURATION; v[j] = 1; }
+            const int64_t p0 = kptr[k], p1 = kptr[k + 1];
+            if (p0 > p1 || p0 < 0 || p1 > E || (k == 0 && p0 != 0) || (k == K - 1 && p1 != E)) bad |= G10_DEV_BAD_KERNEL_PTR;
+        }
+        mine.v[0] += v[j];
+    }
+    if (bad) raise_status(status, bad);
+    Sums<1> total;
+    Sums<1> ex = block_exclusive_with_lookback<1>(st, tile, mine, status, &total);
+    long long run = ex.v[0];
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        const int64_t k = base + j;
+        if (k < K) start[k] = run;
+        run += v[j];
+    }
+    if (tile == tiles - 1 && threadIdx.x == 0) {
+        start[K] = total.v[0];
+        if (total.v[0] >= ((long long)1 << 44)) raise_status(status, G10_DEV_BAD_DURATION);
+    }
+}
+
+cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s)
+{
+    const int tiles = (int)tiles_of(t.K, kScanTile);
+    TileState<1> st{w.clock_scan.ticket, w.clock_scan.flag, w.clock_scan.agg, w.clock_scan.incl};
+    k_slot_clock<<<tiles, kScanThreads, 0, s>>>(t.K, t.E, t.kernel_ns, t.kernel_ptr, start, st, tiles, w.status);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// Event passes.  An event is one (kernel, tensor) entry of the CSR.  Blocks take 2048 consecutive
+// events (128-bit loads); the kernel of an event is found by binary search in kernel_ptr, bracketed
+// once per block.
+// =============================================================================================
+constexpr int kEvThreads = 256;
+constexpr int kEvItems = 8;
+constexpr int kEvTile = kEvThreads * kEvItems;
+
+// last k in [lo, hi] with kptr[k] <= e  (kptr nondecreasing; lo is known to satisfy it)
+__device__ __forceinline__ int kernel_of_event(const int64_t *__restrict__ kptr, int lo, int hi, int64_t e)
+{
+    while (lo < hi) {
+        const int mid = lo + (hi - lo + 1) / 2;
+        if (kptr[mid] <= e) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// raw use count per tensor (a tensor listed twice by one kernel counts twice here; collapsed later)
+__global__ void __launch_bounds__(kEvThreads) k_count_events(int64_t E, int64_t N, const int32_t *__restrict__ kt,
+                                                             int32_t *__restrict__ cnt, ull *status)
+{
+    const int64_t base = (int64_t)blockIdx.x * kEvTile;
+    ull bad = 0;
+#pragma unroll
+    for (int j = 0; j < kEvItems; ++j) {
+        const int64_t e = base + (int64_t)j * kEvThreads + threadIdx.x;
+        if (e < E) {
+            const int32_t i = kt[e];
+            if (i < 0 || i >= N) bad = G10_DEV_BAD_TENSOR_ID;
+            else atomicAdd(&cnt[i], 1);
+        }
+    }
+    if (bad) raise_status(status, bad);
+}
+
+// raw_ptr = exclusive scan of the raw counts; tensors with more than kHeavyThreshold raw uses are
+// queued for the block-wide sort.
+__global__ void __launch_bounds__(kScanThreads) k_scan_counts(int64_t N, const int32_t *__restrict__ cnt, int32_t *__restrict__ raw_ptr,
+                                                              int32_t *__restrict__ heavy_list, unsigned *heavy_count,
+                                                              TileState<1> st, int tiles, ull *status)
+{
+    const int tile = next_tile(st.ticket);
+    if (tile >= tiles) return;
+    const int64_t base = (int64_t)tile * kScanTile + (int64_t)threadIdx.x * kScanItems;
+    int v[kScanItems];
+    Sums<1> mine;
+    mine.v[0] = 0;
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        const int64_t i = base + j;
+        v[j] = i < N ? cnt[i] : 0;
+        mine.v[0] += v[j];
+        if (v[j] > kHeavyThreshold) heavy_list[atomicAdd(heavy_count, 1u)] = (int32_t)i;
+    }
+    Sums<1> total;
+    Sums<1> ex = block_exclusive_with_lookback<1>(st, tile, mine, status, &total);
+    long long run = ex.v[0];
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        const int64_t i = base + j;
+        if (i < N) raw_ptr[i] = (int32_t)run;
+        run += v[j];
+    }
+    if (tile == tiles - 1 && threadIdx.x == 0) raw_ptr[N] = (int32_t)total.v[0];
+}
+
+// scatter every event's kernel index into its tensor's segment (order inside a segment is arbitrary)
+__global__ void __launch_bounds__(kEvThreads) k_scatter_events(int64_t E, int64_t N, int64_t K, const int64_t *__restrict__ kptr,
+                                                               const int32_t *__restrict__ kt, const int32_t *__restrict__ raw_ptr,
+                                                               int32_t *__restrict__ cursor, int32_t *__restrict__ raw_uses)
+{
+    __shared__ int s_lo, s_hi;
+    const int64_t base = (int64_t)blockIdx.x * kEvTile;
+    if (threadIdx.x == 0) {
+        const int64_t last = (base + kEvTile <= E ? base + kEvTile : E) - 1;
+        s_lo = kernel_of_event(kptr, 0, (int)K - 1, base);
+        s_hi = kernel_of_event(kptr, s_lo, (int)K - 1, last);
+    }
+    __syncthreads();
+    const int lo = s_lo, hi = s_hi;
+#pragma unroll
+    for (int j = 0; j < kEvItems; ++j) {
+        const int64_t e = base + (int64_t)j * kEvThreads + threadIdx.x;
+        if (e < E) {
+            const int32_t i = kt[e];
+            if (i >= 0 && i < N) {
+                const int k = kernel_of_event(kptr, lo, hi, e);
+                const int old = atomicSub(&cursor[i], 1);          // counts back down to zero
+                const int64_t pos = (int64_t)raw_ptr[i] + old - 1;
+                if (old >= 1 && pos < E) raw_uses[pos] = k;
+            }
+        }
+    }
+}
+
+// first / last use by atomic min / max (the timeline call alone does not need the sorted use lists)
+__global__ void __launch_bounds__(kEvThreads) k_first_last_events(int64_t E, int64_t N, int64_t K, const int64_t *__restrict__ kptr,
+                                                                  const int32_t *__restrict__ kt, int32_t *__restrict__ first_enc,
+                                                                  int32_t *__restrict__ last_enc, ull *status)
+{
+    // both arrays start at zero: first_enc holds max(K - k) (0 = unused), last_enc holds max(k + 1)
+    __shared__ int s_lo, s_hi;
+    const int64_t base = (int64_t)blockIdx.x * kEvTile;
+    if (threadIdx.x == 0) {
+        const int64_t last = (base + kEvTile <= E ? base + kEvTile : E) - 1;
+        s_lo = kernel_of_event(kptr, 0, (int)K - 1, base);
+        s_hi = kernel_of_event(kptr, s_lo, (int)K - 1, last);
+    }
+    __syncthreads();
+    const int lo = s_lo, hi = s_hi;
+    ull bad = 0;
+#pragma unroll
+    for (int j = 0; j < kEvItems; ++j) {
+        const int64_t e = base + (int64_t)j * kEvThreads + threadIdx.x;
+        if (e < E) {
+            const int32_t i = kt[e];
+            if (i < 0 || i >= N) bad = G10_DEV_BAD_TENSOR_ID;
+            else {
+                const int k = kernel_of_event(kptr, lo, hi, e);
+                atomicMax(&first_enc[i], (int)K - k);
+                atomicMax(&last_enc[i], k + 1);
+            }
+        }
+    }
+    if (bad) raise_status(status, bad);
+}
+
+__global__ void k_decode_first_last(int64_t N, int64_t K, int32_t *first, int32_t *last)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < N) {
+        const int f = first[i], l = last[i];
+        first[i] = f == 0 ? -1 : (int)K - f;
+        last[i] = l - 1;
+    }
+}
+
+cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s)
+{
+    if (t.N == 0) return cudaSuccess;
+    cudaError_t e = cudaMemsetAsync(first_use, 0, sizeof(int32_t) * (size_t)t.N, s);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(last_use, 0, sizeof(int32_t) * (size_t)t.N, s);
+    if (e != cudaSuccess) return e;
+    if (t.E > 0 && t.K > 0) {
+        const int blocks = (int)tiles_of(t.E, kEvTile);
+        k_first_last_events<<<blocks, kEvThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.status);
+    }
+    k_decode_first_last<<<(unsigned)((t.N + 255) / 256), 256, 0, s>>>(t.N, t.K, first_use, last_use);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// Heavy tensors: one block sorts the segment (bitonic network that only ever moves values up, so an
+// arbitrary length works by skipping partners beyond the end), removes repeats in place and counts
+// the periods.  cnt[tensor] receives the tensor's slot in heavy_info.
+// =============================================================================================
+constexpr int kHeavyThreads = 256;
+constexpr int kHeavySmem = 8192;   // ints sorted in shared memory; longer segments are sorted in global memory
+
+__device__ void block_bitonic_sort(int32_t *a, int n)
+{
+    int n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    for (int k = 2; k <= n2; k <<= 1) {
+        // first stage of each merge mirrors the upper half, the others are plain half-cleaners
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const bool mirror = (j == (k >> 1));
+            for (int t = threadIdx.x; t < n2 / 2; t += blockDim.x) {
+                const int blk = t / j, off = t % j;
+                const int i = blk * 2 * j + off;
+                const int p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
+                if (p < n) {
+                    const int32_t x = a[i], y = a[p];
+                    if (x > y) { a[i] = y; a[p] = x; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kHeavyThreads) k_sort_heavy(const unsigned *heavy_count, const int32_t *__restrict__ heavy_list,
+                                                              const int32_t *__restrict__ raw_ptr, int32_t *__restrict__ raw_uses,
+                                                              int32_t *__restrict__ cnt, int32_t *__restrict__ heavy_info)
+{
+    __shared__ int32_t s_buf[kHeavySmem];
+    __shared__ int s_wcount[kHeavyThreads / 32];
+    __shared__ int s_total, s_periods;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned nh = *heavy_count;
+    for (unsigned h = blockIdx.x; h < nh; h += gridDim.x) {
+        const int32_t i = heavy_list[h];
+        const int beg = raw_ptr[i], n = raw_ptr[i + 1] - beg;
+        int32_t *seg = raw_uses + beg;
+        int32_t *a = n <= kHeavySmem ? s_buf : seg;
+        if (n <= kHeavySmem) {
+            for (int t = threadIdx.x; t < n; t += blockDim.x) s_buf[t] = seg[t];
+        }
+        __syncthreads();
+        block_bitonic_sort(a, n);
+        // in-place compaction of the distinct values, chunk by chunk, in order (read chunk, sync, write)
+        if (threadIdx.x == 0) { s_total = 0; s_periods = 0; }
+        __syncthreads();
+        for (int c0 = 0; c0 < n; c0 += blockDim.x) {
+            const int t = c0 + threadIdx.x;
+            int32_t x = 0, prev = 0;
+            bool keep = false, per = false;
+            if (t < n) {
+                x = a[t];
+                if (t > 0) prev = a[t - 1];
+                keep = (t == 0) || (x != prev);
+                per = keep && t > 0 && (x - prev >= 2);
+            }
+            const unsigned mk = __ballot_sync(0xffffffffu, keep);
+            const unsigned mp = __ballot_sync(0xffffffffu, per);
+            if (lane == 0) s_wcount[warp] = __popc(mk);
+            __syncthreads();
+            int off = s_total;
+            for (int w = 0; w < warp; ++w) off += s_wcount[w];
+            off += __popc(mk & ((1u << lane) - 1u));
+            int chunk_total = 0;
+            for (int w = 0; w < kHeavyThreads / 32; ++w) chunk_total += s_wcount[w];
+            __syncthreads();                                   // every a[t], a[t-1] of this chunk has been read
+            if (keep) seg[off] = x;                            // off <= t: never overtakes an unread element
+            if (lane == 0 && mp) atomicAdd(&s_periods, __popc(mp));
+            if (threadIdx.x == 0) s_total += chunk_total;
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {
+            heavy_info[2 * h] = s_total;
+            heavy_info[2 * h + 1] = s_periods;
+            cnt[i] = (int32_t)h;
+        }
+        __syncthreads();
+    }
+}
+
+// =============================================================================================
+// Vitality emit: per tensor sort its (few) raw uses, drop repeats, count periods; one fused
+// two-sum look-back scan gives every tensor its offsets into `uses` and into the period arrays;
+// then first / last / count / CSR pointers / sorted uses / periods are written in a single pass.
+// =============================================================================================
+constexpr int kEmThreads = kScanThreads;
+constexpr int kEmItems = 4;
+constexpr int kEmTile = kEmThreads * kEmItems;
+
+__global__ void __launch_bounds__(kEmThreads) k_vitality_emit(int64_t N, const int32_t *__restrict__ raw_ptr, int32_t *__restrict__ raw_uses,
+                                                              const int32_t *__restrict__ cnt, const int32_t *__restrict__ heavy_info,
+                                                              VitalityBuffers out, TileState<2> st, int tiles, ull *status)
+{
+    __shared__ int s_heavy_n;
+    __shared__ int s_heavy_tensor[kEmTile];
+    __shared__ int s_wcount[kEmThreads / 32];
+    __shared__ int s_chunk_base;
+    const int tile = next_tile(st.ticket);
+    if (tile >= tiles) return;
+    if (threadIdx.x == 0) s_heavy_n = 0;
+    const int64_t base = (int64_t)tile * kEmTile + (int64_t)threadIdx.x * kEmItems;
+    int beg[kEmItems], d[kEmItems], pc[kEmItems];
+    bool heavy[kEmItems];
+    Sums<2> mine;
+    mine.v[0] = 0; mine.v[1] = 0;
+#pragma unroll
+    for (int j = 0; j < kEmItems; ++j) {
+        const int64_t i = base + j;
+        beg[j] = 0; d[j] = 0; pc[j] = 0; heavy[j] = false;
+        if (i < N) {
+            beg[j] = raw_ptr[i];
+            const int n = raw_ptr[i + 1] - beg[j];
+            if (n > kHeavyThreshold) {
+                const int h = cnt[i];
+                heavy[j] = true;
+                d[j] = heavy_info[2 * h];
+                pc[j] = heavy_info[2 * h + 1];
+            } else if (n > 0) {
+                int32_t *seg = raw_uses + beg[j];
+                for (int a = 1; a < n; ++a) {               // insertion sort, n <= 32
+                    const int32_t x = seg[a];
+                    int b = a - 1;
+                    while (b >= 0 && seg[b] > x) { seg[b + 1] = seg[b]; --b; }
+                    seg[b + 1] = x;
+                }
+                int32_t prev = seg[0];
+                int dd = 1, pp = 0;
+                for (int a = 1; a < n; ++a) {
+                    const int32_t x = seg[a];
+                    if (x != prev) { if (x - prev >= 2) ++pp; seg[dd++] = x; prev = x; }
+                }
+                d[j] = dd; pc[j] = pp;
+            }
+        }
+        mine.v[0] += d[j];
+        mine.v[1] += pc[j];
+    }
+    Sums<2> total;
+    Sums<2> ex = block_exclusive_with_lookback<2>(st, tile, mine, status, &total);
+    long long uoff = ex.v[0], poff = ex.v[1];
+    ull bad = 0;
+#pragma unroll
+    for (int j = 0; j < kEmItems; ++j) {
+        const int64_t i = base + j;
+        if (i < N) {
+            const int32_t *seg = raw_uses + beg[j];
+            out.num_uses[i] = d[j];
+            out.use_ptr[i] = uoff;
+            out.period_ptr[i] = poff;
+            out.first_use[i] = d[j] > 0 ? seg[0] : -1;
+            out.last_use[i] = d[j] > 0 ? seg[d[j] - 1] : -1;
+            if (uoff + d[j] > out.uses_cap) bad |= G10_DEV_USES_OVERFLOW;
+            if (poff + pc[j] > out.periods_cap) bad |= G10_DEV_PERIODS_OVERFLOW;
+            if (heavy[j]) {
+                s_heavy_tensor[atomicAdd(&s_heavy_n, 1)] = (int)i;
+            } else {
+                long long po = poff;
+                for (int a = 0; a < d[j]; ++a) {
+                    const int32_t x = seg[a];
+                    if (uoff + a < out.uses_cap) out.uses[uoff + a] = x;
+                    if (a > 0 && x - seg[a - 1] >= 2) {
+                        if (po < out.periods_cap) {
+                            out.period_tensor[po] = (int32_t)i;
+                            out.period_prev_use[po] = seg[a - 1];
+                            out.period_next_use[po] = x;
+                        }
+                        ++po;
+                    }
+                }
+            }
+        }
+        uoff += d[j];
+        poff += pc[j];
+    }
+    if (bad) raise_status(status, bad);
+    if (tile == tiles - 1 && threadIdx.x == 0) {
+        out.use_ptr[N] = total.v[0];
+        out.period_ptr[N] = total.v[1];
+        out.counts[0] = total.v[0];
+        out.counts[1] = total.v[1];
+    }
+    __syncthreads();
+    // heavy tensors of this tile, one after the other, with the whole block
+    const int nh = s_heavy_n;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int q = 0; q < nh; ++q) {
+        // offsets and counts were written to global memory by the owning thread before the barrier above
+        const int tensor = s_heavy_tensor[q];
+        const int32_t *seg = raw_uses + raw_ptr[tensor];
+        const int dd = out.num_uses[tensor];
+        const long long uo = out.use_ptr[tensor], po = out.period_ptr[tensor];
+        if (threadIdx.x == 0) s_chunk_base = 0;
+        __syncthreads();
+        for (int t = threadIdx.x; t < dd; t += blockDim.x)
+            if (uo + t < out.uses_cap) out.uses[uo + t] = seg[t];
+        for (int c0 = 1; c0 < dd; c0 += blockDim.x) {
+            const int t = c0 + threadIdx.x;
+            bool per = false;
+            int32_t x = 0, prev = 0;
+            if (t < dd) { x = seg[t]; prev = seg[t - 1]; per = (x - prev >= 2); }
+            const unsigned mp = __ballot_sync(0xffffffffu, per);
+            if (lane == 0) s_wcount[warp] = __popc(mp);
+            __syncthreads();
+            int off = s_chunk_base;
+            for (int w = 0; w < warp; ++w) off += s_wcount[w];
+            off += __popc(mp & ((1u << lane) - 1u));
+            if (per && po + off < out.periods_cap) {
+                out.period_tensor[po + off] = tensor;
+                out.period_prev_use[po + off] = prev;
+                out.period_next_use[po + off] = x;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) { int tot = 0; for (int w = 0; w < kEmThreads / 32; ++w) tot += s_wcount[w]; s_chunk_base += tot; }
+            __syncthreads();
+        }
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s)
+{
+    if (t.E > 0 && t.N > 0) {
+        k_count_events<<<(unsigned)tiles_of(t.E, kEvTile), kEvThreads, 0, s>>>(t.E, t.N, t.kernel_tensors, w.cnt, w.status);
+    }
+    {
+        const int tiles = (int)tiles_of(t.N, kScanTile);
+        TileState<1> st{w.count_scan.ticket, w.count_scan.flag, w.count_scan.agg, w.count_scan.incl};
+        k_scan_counts<<<tiles, kScanThreads, 0, s>>>(t.N, w.cnt, w.raw_ptr, w.heavy_list, w.heavy_count, st, tiles, w.status);
+    }
+    if (t.E > 0 && t.N > 0 && t.K > 0) {
+        k_scatter_events<<<(unsigned)tiles_of(t.E, kEvTile), kEvThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors,
+                                                                                 w.raw_ptr, w.cnt, w.raw_uses);
+        k_sort_heavy<<<64, kHeavyThreads, 0, s>>>(w.heavy_count, w.heavy_list, w.raw_ptr, w.raw_uses, w.cnt, w.heavy_info);
+    }
+    {
+        const int tiles = (int)tiles_of(t.N, kEmTile);
+        TileState<2> st{w.emit_scan.ticket, w.emit_scan.flag, w.emit_scan.agg, w.emit_scan.incl};
+        k_vitality_emit<<<tiles, kEmThreads, 0, s>>>(t.N, w.raw_ptr, w.raw_uses, w.cnt, w.heavy_info, out, st, tiles, w.status);
+    }
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// Pressure timeline: D[first] += size, D[last + 1] -= size (a global tensor that is used at all is
+// alive in every slot: its size goes to D[0] only), then P = inclusive scan of D, peak and its
+// lowest slot.
+// =============================================================================================
+__global__ void __launch_bounds__(256) k_diff_scatter(int64_t N, int64_t K, const int64_t *__restrict__ bytes, const uint8_t *__restrict__ glob,
+                                                      const int32_t *__restrict__ first, const int32_t *__restrict__ last,
+                                                      ull *__restrict__ diff, ull *status)
+{
+    __shared__ long long s_part[8];
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    long long gsum = 0;
+    if (i < N) {
+        const long long b = bytes[i];
+        if (b < 1 || b >= ((long long)1 << 40)) raise_status(status, G10_DEV_BAD_BYTES);
+        const int f = first[i];
+        if (f >= 0 && f < K) {
+            if (glob != nullptr && glob[i]) gsum = b;
+            else {
+                atomicAdd(&diff[f], (ull)b);
+                const int l = last[i];
+                if (l + 1 < K) atomicAdd(&diff[l + 1], (ull)(-b));
+            }
+        }
+    }
+    // global tensors all land on D[0]: one atomic per block instead of one per tensor
+    gsum = warp_sum_i64(gsum);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = gsum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long tot = 0;
+        for (int w = 0; w < 8; ++w) tot += s_part[w];
+        if (tot != 0) atomicAdd(&diff[0], (ull)tot);
+    }
+}
+
+__global__ void __launch_bounds__(kScanThreads) k_scan_pressure(int64_t K, const int64_t *__restrict__ diff, int64_t *__restrict__ P,
+                                                                TileState<1> st, unsigned *done, int64_t *__restrict__ tile_max,
+                                                                int32_t *__restrict__ tile_slot, int tiles, int64_t *peak_bytes,
+                                                                int32_t *peak_slot, ull *status)
+{
+    __shared__ long long s_mx[kScanThreads / 32];
+    __shared__ int s_sl[kScanThreads / 32];
+    __shared__ bool s_last;
+    const int tile = next_tile(st.ticket);
+    if (tile >= tiles) return;
+    const int64_t base = (int64_t)tile * kScanTile + (int64_t)threadIdx.x * kScanItems;
+    long long v[kScanItems];
+    Sums<1> mine;
+    mine.v[0] = 0;
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        const int64_t k = base + j;
+        v[j] = k < K ? diff[k] : 0;
+        mine.v[0] += v[j];
+    }
+    Sums<1> total;
+    Sums<1> ex = block_exclusive_with_lookback<1>(st, tile, mine, status, &total);
+    long long run = ex.v[0];
+    long long mx = 0;
+    int sl = -1;
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        const int64_t k = base + j;
+        run += v[j];
+        if (k < K) {
+            P[k] = run;
+            if (sl < 0 || run > mx) { mx = run; sl = (int)k; }
+        }
+    }
+    // block max, ties to the lowest slot
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long omx = __shfl_down_sync(0xffffffffu, mx, o);
+        const int osl = __shfl_down_sync(0xffffffffu, sl, o);
+        if (osl >= 0 && (sl < 0 || omx > mx || (omx == mx && osl < sl))) { mx = omx; sl = osl; }
+    }
+    if (lane == 0) { s_mx[warp] = mx; s_sl[warp] = sl; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kScanThreads / 32; ++w)
+            if (s_sl[w] >= 0 && (sl < 0 || s_mx[w] > mx || (s_mx[w] == mx && s_sl[w] < sl))) { mx = s_mx[w]; sl = s_sl[w]; }
+        tile_max[tile] = mx;
+        tile_slot[tile] = sl;
+        __threadfence();
+        s_last = (atomicAdd(done, 1u) == (unsigned)tiles - 1u);
+    }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        long long bm = 0;
+        int bs = -1;
+        for (int t = threadIdx.x; t < tiles; t += blockDim.x) {
+            const long long m = __ldcg(&tile_max[t]);
+            const int s2 = __ldcg(&tile_slot[t]);
+            if (s2 >= 0 && (bs < 0 || m > bm || (m == bm && s2 < bs))) { bm = m; bs = s2; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const long long omx = __shfl_down_sync(0xffffffffu, bm, o);
+            const int osl = __shfl_down_sync(0xffffffffu, bs, o);
+            if (osl >= 0 && (bs < 0 || omx > bm || (omx == bm && osl < bs))) { bm = omx; bs = osl; }
+        }
+        __syncthreads();
+        if (lane == 0) { s_mx[warp] = bm; s_sl[warp] = bs; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < kScanThreads / 32; ++w)
+                if (s_sl[w] >= 0 && (bs < 0 || s_mx[w] > bm || (s_mx[w] == bm && s_sl[w] < bs))) { bm = s_mx[w]; bs = s_sl[w]; }
+            *peak_bytes = bs < 0 ? 0 : bm;
+            *peak_slot = bs;
+        }
+    }
+}
+
+cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use,
+                            int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
+{
+    if (t.N > 0 && t.K > 0)
+        k_diff_scatter<<<(unsigned)((t.N + 255) / 256), 256, 0, s>>>(t.N, t.K, t.tensor_bytes, t.tensor_global, first_use, last_use,
+                                                                     (ull *)w.diff, w.status);
+    const int tiles = (int)tiles_of(t.K, kScanTile);
+    TileState<1> st{w.pressure_scan.ticket, w.pressure_scan.flag, w.pressure_scan.agg, w.pressure_scan.incl};
+    k_scan_pressure<<<tiles, kScanThreads, 0, s>>>(t.K, w.diff, pressure, st, w.pressure_scan.done, w.tile_max, w.tile_slot, tiles,
+                                                   peak_bytes, peak_slot, w.status);
+    return cudaGetLastError();
+}
+
+// =============================================================================================
+// Candidate geometry.
+// =============================================================================================
+__device__ __forceinline__ int64_t transfer_time_ns(int64_t bytes, uint64_t bw)
+{
+    const u128 num = (u128)(uint64_t)bytes * (u128)1000000000ull;
+    u128 q = num / (u128)bw;
+    if (q * (u128)bw != num) q += 1;
+    const u128 sat = (u128)1 << 62;
+    return (int64_t)(q > sat ? sat : q);
+}
+
+__global__ void __launch_bounds__(256) k_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, const int64_t *__restrict__ start,
+                                                  const int64_t *__restrict__ bytes, const int32_t *__restrict__ per_t,
+                                                  const int32_t *__restrict__ per_u, const int32_t *__restrict__ per_v,
+                                                  uint64_t host_bw, uint64_t ssd_bw, int64_t stride, int64_t *__restrict__ geo_t,
+                                                  int32_t *__restrict__ geo_a, int32_t *__restrict__ geo_b)
+{
+    const int64_t Pn = Pn_dev ? (*Pn_dev < Pn_bound ? *Pn_dev : Pn_bound) : Pn_bound;
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= Pn) return;
+    const int64_t s = bytes[per_t[p]];
+    const int u = per_u[p], v = per_v[p];
+    const int64_t t_r = start[u + 1], t_end = start[v], L = t_end - t_r;
+#pragma unroll
+    for (int X = 0; X < 2; ++X) {
+        const int64_t t = transfer_time_ns(s, X == G10_DEST_SSD ? ssd_bw : host_bw);
+        int a_abs = -1, b_abs = -2;
+        if (t <= L && 2 * t <= L) {
+            // first k in [u+1, v] with start[k] >= t_r + t   (start[v] = t_end > t_r + t - 1 always qualifies)
+            int lo = u + 1, hi = v;
+            const int64_t ev_end = t_r + t;
+            while (lo < hi) { const int mid = lo + (hi - lo) / 2; if (start[mid] >= ev_end) hi = mid; else lo = mid + 1; }
+            const int ap = lo;
+            // last j in [u+1, v] with start[j] <= t_end - t   (start[u+1] = t_r qualifies)
+            lo = u + 1; hi = v;
+            const int64_t pf_beg = t_end - t;
+            while (lo < hi) { const int mid = lo + (hi - lo + 1) / 2; if (start[mid] <= pf_beg) lo = mid; else hi = mid - 1; }
+            const int bp = lo - 1;
+            if (ap <= bp) { a_abs = ap; b_abs = bp; }
+        }
+        geo_t[X * stride + p] = t;
+        geo_a[X * stride + p] = a_abs;
+        geo_b[X * stride + p] = b_abs;
+    }
+    (void)K;
+}
+
+cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, const int64_t *start, const int64_t *tensor_bytes,
+                            const int32_t *per_t, const int32_t *per_u, const int32_t *per_v, uint64_t host_bw, uint64_t ssd_bw,
+                            int64_t stride, int64_t *geo_t, int32_t *geo_a, int32_t *geo_b, cudaStream_t s)
+{
+    if (Pn_bound <= 0) return cudaSuccess;
+    k_geometry<<<(unsigned)((Pn_bound + 255) / 256), 256, 0, s>>>(K, Pn_bound, Pn_dev, start, tensor_bytes, per_t, per_u, per_v,
+                                                                  host_bw, ssd_bw, stride, geo_t, geo_a, geo_b);
+    return cudaGetLastError();
+}
+
+}  // namespace g10

@@ -1,0 +1,242 @@
+"""Parity of the CUDA path with the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+import helpers
+from paper_2310_09443_b200 import traces
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    from paper_2310_09443_b200 import binding, build
+    build.build()
+    binding.load_library()
+    return binding
+
+
+def _np(t):
+    return t.cpu().numpy()
+
+
+def check_vitality(gpu, oracle, tr, tb):
+    import torch
+    v = gpu.g10_vitality(tb)
+    torch.cuda.synchronize()
+    ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+    counts = _np(v.counts)
+    assert counts[2] == 0, "device status %x" % counts[2]
+    assert counts[0] == len(ov.uses) and counts[1] == len(ov.period_tensor)
+    N = tr.N
+    assert np.array_equal(_np(v.first_use)[:N], ov.first_use) and np.array_equal(_np(v.last_use)[:N], ov.last_use)
+    assert np.array_equal(_np(v.num_uses)[:N], ov.num_uses)
+    assert np.array_equal(_np(v.use_ptr)[:N + 1], ov.use_ptr) and np.array_equal(_np(v.period_ptr)[:N + 1], ov.period_ptr)
+    e2, pn = int(counts[0]), int(counts[1])
+    assert np.array_equal(_np(v.uses)[:e2], ov.uses)
+    assert np.array_equal(_np(v.period_tensor)[:pn], ov.period_tensor)
+    assert np.array_equal(_np(v.period_prev_use)[:pn], ov.period_prev_use)
+    assert np.array_equal(_np(v.period_next_use)[:pn], ov.period_next_use)
+    return v, ov
+
+
+def check_timeline(gpu, oracle, tr, tb):
+    import torch
+    tl = gpu.g10_pressure_timeline(tb)
+    torch.cuda.synchronize()
+    start, P0, peak, slot = oracle.timeline(tr)
+    assert int(tl.status.item()) == 0
+    assert np.array_equal(_np(tl.kernel_start_ns)[:tr.K + 1], start)
+    assert np.array_equal(_np(tl.pressure)[:tr.K], P0)
+    assert int(tl.peak_bytes.item()) == peak and int(tl.peak_slot.item()) == slot
+    return tl, (start, P0, peak, slot)
+
+
+def check_geometry(gpu, oracle, tr, tb, v, ov, tl):
+    import torch
+    pn = len(ov.period_tensor)
+    g = gpu.g10_candidate_geometry(tr.K, tl.kernel_start_ns, tb.tensor_bytes, v.period_tensor[:pn].contiguous(),
+                                   v.period_prev_use[:pn].contiguous(), v.period_next_use[:pn].contiguous(),
+                                   tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    if pn == 0:
+        return
+    og = oracle.geometry(_np(tl.kernel_start_ns)[:tr.K + 1], tr.tensor_bytes, ov.period_tensor, ov.period_prev_use,
+                         ov.period_next_use, tr.host_bw, tr.ssd_bw)
+    assert np.array_equal(_np(g.transfer_ns), og.transfer_ns)
+    assert np.array_equal(_np(g.absent_first), og.absent_first) and np.array_equal(_np(g.absent_last), og.absent_last)
+
+
+def check_plan(gpu, tr, tb, cap, ref, host_capacity=0, max_iterations=0, flags=0):
+    import torch
+    plan = gpu.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, host_capacity_bytes=host_capacity,
+                                   max_iterations=max_iterations, flags=flags)
+    torch.cuda.synchronize()
+    summary = _np(plan.summary)
+    assert summary[7] == 0, "device status %x" % summary[7]
+    assert np.array_equal(summary[:7], ref.summary[:7]), (summary, ref.summary)
+    assert np.array_equal(gpu.migrations_numpy(plan), ref.migrations)
+    assert np.array_equal(_np(plan.final_pressure)[:tr.K], ref.final_pressure)
+    return plan
+
+
+def full_parity(gpu, oracle, tr, lazy_oracle=False, repeats=1, **plan_kw):
+    tb = gpu.upload(tr)
+    v, ov = check_vitality(gpu, oracle, tr, tb)
+    tl, (start, P0, peak, slot) = check_timeline(gpu, oracle, tr, tb)
+    check_geometry(gpu, oracle, tr, tb, v, ov, tl)
+    cap = tr.capacity_from_peak(int(tl.peak_bytes.item()))
+    ref = oracle.plan(tr, tr.capacity_from_peak(peak), lazy=lazy_oracle,
+                      host_capacity_bytes=plan_kw.get("host_capacity", 0), max_iterations=plan_kw.get("max_iterations", 0))
+    for _ in range(repeats):
+        check_plan(gpu, tr, tb, cap, ref, **plan_kw)
+    return ref
+
+
+def test_hand_worked_examples(gpu, oracle):
+    import json, os
+    ex_all = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_worked_examples.json")))["examples"]
+    for name, ex in ex_all.items():
+        tr = traces.from_lists(name, ex["kernel_lists"], ex["tensor_bytes"], ex["kernel_ns"], host_bw=ex["host_bw"],
+                               ssd_bw=ex["ssd_bw"], capacity_bytes=ex["capacity"])
+        ref = full_parity(gpu, oracle, tr)
+        assert ref.status == ex["status"] and ref.final_pressure.tolist() == ex["final_pressure"]
+
+
+def test_random_toy_traces(gpu, oracle):
+    """Empty kernels, repeats inside a kernel, unused tensors, globals; several capacities and a finite host memory."""
+    rng = np.random.default_rng(777)
+    for trial in range(60):
+        K = int(rng.integers(1, 40)); N = int(rng.integers(1, 30))
+        tr = traces.random_toy(rng, K, N, max_deg=5)
+        tr.capacity_frac = [(1, 2), (1, 5), (0, 1), (9, 10)][trial % 4]
+        hc = int(rng.integers(0, 3)) * int(rng.integers(1, 80))
+        full_parity(gpu, oracle, tr, host_capacity=hc)
+
+
+@pytest.mark.parametrize("cfg", [0, 1, 2, 3])
+def test_configs_bit_exact(gpu, oracle, cfg):
+    """Configs 0-3 at full size: every output of the three calls equals the oracle's; plan repeated 3 times."""
+    tr = traces.make_config(cfg)
+    ref = full_parity(gpu, oracle, tr, lazy_oracle=(cfg == 3), repeats=3)
+    assert len(ref.migrations) > 10
+
+
+def test_inplace_relu_variant(gpu, oracle):
+    tr = traces.config1_resnet152(inplace_relu=True)
+    full_parity(gpu, oracle, tr)
+
+
+def test_scaled_stress_dag(gpu, oracle):
+    """Several scan tiles and a ragged tail: K = 20 000, N = 80 000 (plain oracle still feasible)."""
+    tr = traces.config4_stress_dag(K=20000, N=80000)
+    ref = full_parity(gpu, oracle, tr, lazy_oracle=True)
+    assert len(ref.migrations) > 1000
+
+
+def test_iteration_limit_and_host_capacity(gpu, oracle):
+    tr = traces.config0_mlp_chain()
+    full_parity(gpu, oracle, tr, max_iterations=5)
+    full_parity(gpu, oracle, tr, host_capacity=200 << 20)
+    tr.capacity_frac = (1, 1)
+    ref = full_parity(gpu, oracle, tr)
+    assert ref.status == "ALREADY_FITS"
+    tr.capacity_frac = None; tr.capacity_bytes = 1 << 63
+    full_parity(gpu, oracle, tr)
+    tr.capacity_bytes = 0
+    full_parity(gpu, oracle, tr)
+
+
+def test_heavy_tensors(gpu, oracle):
+    """Tensors used by very many kernels take the block-wide sort (shared-memory and global-memory variants)."""
+    rng = np.random.default_rng(5)
+    K, N = 30000, 50
+    lists = []
+    for k in range(K):
+        lst = [int(x) for x in rng.integers(4, N, size=int(rng.integers(0, 3)))]
+        if k % 2 == 0: lst.append(0)                 # 15 000 uses: sorted in global memory
+        if k % 7 == 0: lst += [1, 1]                 # 4 286 uses, each listed twice: shared-memory sort + repeats
+        if k % 400 == 0: lst.append(2)               # 75 uses with long periods
+        if rng.random() < 0.002: lst.append(3)
+        lists.append(lst)
+    size = rng.integers(1 << 10, 1 << 24, size=N)
+    dur = rng.integers(1000, 100000, size=K)
+    tr = traces.from_lists("heavy", lists, size, dur, (rng.random(N) < 0.2).astype(np.uint8), capacity_frac=(1, 2))
+    tb = gpu.upload(tr)
+    v, ov = check_vitality(gpu, oracle, tr, tb)
+    tl, _ = check_timeline(gpu, oracle, tr, tb)
+    check_geometry(gpu, oracle, tr, tb, v, ov, tl)
+
+
+def test_empty_and_degenerate(gpu, oracle):
+    for lists, nb in (([], []), ([[], []], []), ([[], [], []], [5, 7]), ([[0], [0], [0]], [9]), ([[0, 0, 0]], [3])):
+        tr = traces.from_lists("e", lists, nb, [3] * len(lists), capacity_bytes=0)
+        full_parity(gpu, oracle, tr)
+
+
+def test_output_capacity_is_reported(gpu):
+    import torch
+    tr = traces.config0_mlp_chain()
+    tb = gpu.upload(tr)
+    v = gpu.g10_vitality(tb, uses_cap=10, periods_cap=5)
+    torch.cuda.synchronize()
+    c = _np(v.counts)
+    assert c[0] == 320 and c[1] == 93 and (c[2] & 0x10) and (c[2] & 0x20)
+    plan = gpu.g10_plan_migrations(tb, 1 << 20, tr.host_bw, tr.ssd_bw, migrations_cap=3)
+    torch.cuda.synchronize()
+    s = _np(plan.summary)
+    assert s[0] > 3 and (s[7] & 0x40)
+
+
+def test_bad_trace_sets_status_bits(gpu):
+    import torch
+    tr = traces.config0_mlp_chain()
+    tr.kernel_tensors = tr.kernel_tensors.copy(); tr.kernel_tensors[7] = 1000
+    tr.kernel_ns = tr.kernel_ns.copy(); tr.kernel_ns[3] = 0
+    tr.tensor_bytes = tr.tensor_bytes.copy(); tr.tensor_bytes[5] = 0
+    tb = gpu.upload(tr)
+    v = gpu.g10_vitality(tb)
+    tl = gpu.g10_pressure_timeline(tb)
+    torch.cuda.synchronize()
+    assert _np(v.counts)[2] & 0x1
+    st = int(tl.status.item())
+    assert (st & 0x1) and (st & 0x8) and (st & 0x4)
+
+
+def test_host_pointer_mode(gpu, oracle):
+    """The same calls with every array in (pinned) host memory: the library stages the copies itself."""
+    tr = traces.config1_resnet152()
+    tb = gpu.pin(tr)
+    v = gpu.g10_vitality(tb)
+    ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+    pn = int(v.counts[1])
+    assert int(v.counts[2]) == 0 and pn == len(ov.period_tensor)
+    assert np.array_equal(v.first_use.numpy(), ov.first_use) and np.array_equal(v.uses.numpy()[:int(v.counts[0])], ov.uses)
+    assert np.array_equal(v.period_next_use.numpy()[:pn], ov.period_next_use)
+    tl = gpu.g10_pressure_timeline(tb)
+    start, P0, peak, slot = oracle.timeline(tr)
+    assert np.array_equal(tl.pressure.numpy(), P0) and int(tl.peak_bytes) == peak and int(tl.peak_slot) == slot
+    assert np.array_equal(tl.kernel_start_ns.numpy(), start)
+    ref = oracle.plan(tr, tr.capacity_from_peak(peak))
+    plan = gpu.g10_plan_migrations(tb, tr.capacity_from_peak(int(tl.peak_bytes)), tr.host_bw, tr.ssd_bw)
+    assert np.array_equal(plan.summary.numpy()[:7], ref.summary[:7]) and int(plan.summary[7]) == 0
+    n = int(plan.summary[0])
+    assert np.array_equal(plan.migrations[:n * 48].numpy().view(gpu.MIGRATION_DTYPE), ref.migrations)
+    assert np.array_equal(plan.final_pressure.numpy(), ref.final_pressure)
+
+
+def test_full_size_stress_dag_passes(gpu, oracle):
+    """Config 4 at full size (K = 1e6, N = 4e6): vitality and timeline element by element; the plan's first
+    200 iterations bit for bit against the oracle's lazy tier, and the invariants of a valid plan on them."""
+    import torch
+    tr = traces.config4_stress_dag()
+    tb = gpu.upload(tr)
+    v, ov = check_vitality(gpu, oracle, tr, tb)
+    tl, (start, P0, peak, slot) = check_timeline(gpu, oracle, tr, tb)
+    cap = tr.capacity_from_peak(peak)
+    ref = oracle.plan(tr, cap, lazy=True, max_iterations=200)
+    plan = check_plan(gpu, tr, tb, cap, ref, max_iterations=200)
+    helpers.check_plan_invariants(tr, cap, start, P0, ov, gpu.migrations_numpy(plan), _np(plan.final_pressure),
+                                  gpu.STATUS[int(plan.summary[2].item())], tr.host_bw, tr.ssd_bw, check_area=False)

@@ -1,0 +1,58 @@
+"""CPU-side checks of the CUDA library: it loads, exports every symbol the header declares, and its
+host-side argument validation answers before anything is launched (no compute calls here)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2310_09443_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load_library()
+
+
+def test_exports_match_header(lib):
+    header = open(os.path.join(ROOT, "include", "g10.h")).read()
+    declared = set(re.findall(r"\b(g10_[a-z_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert lib.g10_version() == 1
+    assert lib.g10_strerror(-3).decode().startswith("workspace")
+
+
+def test_workspace_bytes_and_limits(lib):
+    a = binding.g10_workspace_bytes(binding.WS_PLAN, 96, 130, 320)
+    b = binding.g10_workspace_bytes(binding.WS_PLAN, 1000, 2000, 5000)
+    h = binding.g10_workspace_bytes(binding.WS_PLAN, 1000, 2000, 5000, binding.MEM_HOST)
+    assert 0 < a < b < h and a % 256 == 0
+    assert binding.g10_workspace_bytes(binding.WS_GEOMETRY, 10, 10, 10) == 0
+    out = C.c_size_t(0)
+    assert lib.g10_workspace_bytes(2, -1, 0, 0, 0, C.byref(out)) == -1
+    assert lib.g10_workspace_bytes(2, 1 << 31, 0, 0, 0, C.byref(out)) == -2
+    assert lib.g10_workspace_bytes(9, 1, 1, 1, 0, C.byref(out)) == -1
+
+
+def test_argument_errors_before_any_launch(lib):
+    tr = binding._Trace(4, 4, 4, None, None, None, None, None, 0)
+    vo = binding._VitalityOut()
+    assert lib.g10_vitality(C.byref(tr), C.byref(vo), None, 0, None) == -1        # NULL kernel_ptr
+    assert lib.g10_vitality(None, C.byref(vo), None, 0, None) == -1
+    tr2 = binding._Trace(-1, 4, 4, None, None, None, None, None, 0)
+    assert lib.g10_pressure_timeline(C.byref(tr2), None, None, 0, None) == -1
+    tr3 = binding._Trace(1 << 31, 4, 4, None, None, None, None, None, 0)
+    assert lib.g10_vitality(C.byref(tr3), C.byref(vo), None, 0, None) == -2
+    po = binding._PlanOut()
+    buf = (C.c_int64 * 8)()
+    tr4 = binding._Trace(0, 0, 0, C.cast(buf, C.c_void_p), None, None, None, None, 0)
+    assert lib.g10_plan_migrations(C.byref(tr4), 1, 0, 1, None, C.byref(po), None, 0, None) == -1      # zero bandwidth
+    po.summary = C.cast(buf, C.c_void_p)
+    assert lib.g10_plan_migrations(C.byref(tr4), 1, 1, 1, None, C.byref(po), None, 0, None) == -3      # no workspace
+    go = binding._GeometryOut()
+    assert lib.g10_candidate_geometry(1, 1, None, None, None, None, None, 1, 1, C.byref(go), None) == -1
