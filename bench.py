@@ -311,7 +311,7 @@ def plan_loop_algorithmic_bytes(tr, binding, tb, mig, rounds):
     return 16 * live + 16 * commit_slots + 48 * len(mig)
 
 
-def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind):
+def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=10):
     """Vitality and timeline passes on the 1M-kernel / 4M-tensor stress trace (config 4): the only workload whose
     arrays are large enough for an HBM fraction to mean something.  Algorithmic bytes: vitality reads kernel_ptr
     (8K) and kernel_tensors (4E) and writes first/last/num_uses (12N), use_ptr (8N), uses (4E'), period_ptr (8N)
@@ -326,7 +326,7 @@ def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind):
     K, N, E = tr.K, tr.N, tr.E
     vit_bytes = 8 * K + 4 * E + 12 * N + 8 * N + 4 * e2 + 8 * N + 12 * pn
     tl_bytes = 8 * K + 8 * N + 8 * N + N + 8 * K + 8 * K
-    steps, warm = 10, 3
+    steps, warm = reps, 3
     vit_s = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), steps, warm, flush) / steps
     tl_s = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), steps, warm, flush) / steps
     out = {
@@ -368,10 +368,21 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-stress", action="store_true", help="skip the config-4 pass measurements")
+    ap.add_argument("--stress-only", action="store_true",
+                    help="only time the vitality / timeline passes on config 4 (small profiling target)")
+    ap.add_argument("--stress-reps", type=int, default=10)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.stress_only:
+        import torch
+        from paper_2310_09443_b200 import binding, build
+        build.build()
+        torch.cuda.set_device(0)
+        flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda:0")
+        hbm_peak, peak_kind = measured_peaks()
+        print(json.dumps({"stress_passes": stress_passes(torch, binding, "cuda:0", flush, hbm_peak, peak_kind, args.stress_reps)}))
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
