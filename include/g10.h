@@ -183,6 +183,25 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
                             const g10_options *options /* NULL = defaults */, g10_plan_out *out,
                             void *ws, size_t ws_bytes, void *stream);
 
+/* The paper has no counterpart for this entry point: it is g10_pressure_timeline for callers that cannot
+   allocate device memory when they need a timeline (a host whose device memory is wholly owned by its own
+   pool, or a code path where cudaMalloc / cudaFree are ruled out because they may synchronise the device).
+   It takes no workspace: its scratch is a fixed 1.5 MiB array inside the library image, present on every GPU
+   that loads the library until the process exits.  Consequences the caller must know:
+     - device pointers only (trace->mem must be G10_MEM_DEVICE); same outputs, same device status word and the
+       same stream semantics as g10_pressure_timeline;
+     - traces up to G10_STATIC_MAX_KERNELS kernels and G10_STATIC_MAX_TENSORS tensors; anything larger is
+       refused with G10_ERR_LIMIT before any work is enqueued;
+     - the first call on each device looks the array's address up (cudaGetSymbolAddress, with that device
+       current); make that first call outside any stream capture;
+     - all calls on a device share the one array, which keeps the previous call's contents (the call clears
+       what it needs zeroed); two calls that overlap on the GPU -- different streams, or one stream per thread --
+       race on it and give wrong results, so serialise them;
+     - it never calls cudaMalloc, cudaFree or any allocating library routine. */
+#define G10_STATIC_MAX_KERNELS 32768
+#define G10_STATIC_MAX_TENSORS 131072
+int32_t g10_pressure_timeline_static(const g10_trace *trace, g10_timeline_out *out, void *stream);
+
 /* Bytes of device workspace the call `which` (G10_WS_*) needs for a trace of K kernels, N tensors,
    E events whose arrays live in `mem`. */
 int32_t g10_workspace_bytes(int32_t which, int64_t num_kernels, int64_t num_tensors, int64_t num_events,

@@ -22,7 +22,8 @@ DEST_SSD, DEST_HOST = 0, 1
 FLAG_RESCORE_ALL = 1
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
-           "g10_workspace_bytes", "g10_strerror", "g10_version")
+           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static")
+STATIC_MAX_KERNELS, STATIC_MAX_TENSORS = 32768, 131072
 
 MIGRATION_DTYPE = np.dtype([
     ("period", "<i4"), ("tensor", "<i4"), ("dest", "<i4"),
@@ -82,6 +83,8 @@ def load_library():
         lib.g10_vitality.argtypes = [C.POINTER(_Trace), C.POINTER(_VitalityOut), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.g10_pressure_timeline.restype = C.c_int32
         lib.g10_pressure_timeline.argtypes = [C.POINTER(_Trace), C.POINTER(_TimelineOut), C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.g10_pressure_timeline_static.restype = C.c_int32
+        lib.g10_pressure_timeline_static.argtypes = [C.POINTER(_Trace), C.POINTER(_TimelineOut), C.c_void_p]
         lib.g10_candidate_geometry.restype = C.c_int32
         lib.g10_candidate_geometry.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_uint64, C.c_uint64, C.POINTER(_GeometryOut), C.c_void_p]
@@ -214,6 +217,24 @@ def g10_pressure_timeline(tb: TraceBuffers, ws=None, stream=None, device=None):
     tr = tb.c_struct()
     _check(lib.g10_pressure_timeline(C.byref(tr), C.byref(out), _ptr(ws), ws_bytes, _stream(stream)))
     r.workspace = ws
+    return r
+
+
+def g10_pressure_timeline_static(tb: TraceBuffers, stream=None):
+    """g10_pressure_timeline for callers that cannot allocate: no workspace argument, the scratch is a fixed
+    array inside the library (traces up to STATIC_MAX_KERNELS kernels / STATIC_MAX_TENSORS tensors, device
+    memory only).  Calls on one device share that array, so do not let two of them overlap on the GPU.  The
+    output tensors are still the caller's; this wrapper creates them with torch for convenience."""
+    lib = load_library()
+    dev = tb.kernel_ptr.device
+    r = SimpleNamespace(
+        kernel_start_ns=torch.empty(tb.K + 1, dtype=torch.int64, device=dev),
+        pressure=torch.empty(max(tb.K, 1), dtype=torch.int64, device=dev),
+        peak_bytes=torch.empty(1, dtype=torch.int64, device=dev), peak_slot=torch.empty(1, dtype=torch.int32, device=dev),
+        status=torch.empty(1, dtype=torch.int64, device=dev))
+    out = _TimelineOut(_ptr(r.kernel_start_ns), _ptr(r.pressure), _ptr(r.peak_bytes), _ptr(r.peak_slot), _ptr(r.status))
+    tr = tb.c_struct()
+    _check(lib.g10_pressure_timeline_static(C.byref(tr), C.byref(out), _stream(stream)))
     return r
 
 
