@@ -154,6 +154,9 @@ typedef struct g10_options {
                                        printed) instead of only those whose score can have changed;
                                        the plan is identical, the run is slower                     */
 
+#define G10_FLAG_GLOBAL_STATE 0x2   /* keep the planner state in global memory even when the timeline would fit
+                                       in shared memory (the path large traces take); same plan              */
+
 #define G10_WS_VITALITY 0
 #define G10_WS_TIMELINE 1
 #define G10_WS_PLAN 2

@@ -20,6 +20,7 @@ MEM_DEVICE, MEM_HOST = 0, 1
 WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY = 0, 1, 2, 3
 DEST_SSD, DEST_HOST = 0, 1
 FLAG_RESCORE_ALL = 1
+FLAG_GLOBAL_STATE = 2
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
            "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static")

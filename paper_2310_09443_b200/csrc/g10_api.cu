@@ -57,6 +57,8 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.busy = c.take<int64_t>(4 * K);
     w.hocc = c.take<int64_t>(K);
     w.dead = c.take<unsigned char>(E);
+    w.wl_count = c.take<unsigned>(2);
+    w.xwords = c.take<ull>((2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16);
     w.zero_bytes = align_up(c.off);
     // scratch
     w.raw_ptr = c.take<int32_t>(N + 1);
@@ -83,6 +85,16 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.geo_a = c.take<int32_t>(2 * E);
     w.geo_b = c.take<int32_t>(2 * E);
     w.proposals = c.take<Proposal>(kMaxPlanBlocks);
+    w.prop_stale = c.take<Proposal>(kMaxPlanBlocks);
+    w.c_state = c.take<unsigned char>(E);
+    w.c_ben_lo = c.take<ull>(E);
+    w.c_ben_hi = c.take<ull>(E);
+    w.c_cost = c.take<ull>(E);
+    w.worklist = c.take<int>(2 * E);
+    if (z.K <= kSmallMaxSlots) {
+        w.busy_rep = c.take<int64_t>((size_t)kSmallMaxBlocks * 4 * K);
+        w.hocc_rep = c.take<int64_t>((size_t)kSmallMaxBlocks * K);
+    }
     w.peak_part = c.take<int64_t>(kMaxPlanBlocks);
     w.summary = c.take<int64_t>(8);
     if (z.host) {

@@ -48,6 +48,8 @@ struct Workspace {
     int64_t *busy;               // [4*K] booked channel time per slot
     int64_t *hocc;               // [K] host-memory occupancy per slot
     unsigned char *dead;         // [E] period erased
+    unsigned *wl_count;          // [2] lengths of the two DIRTY work lists
+    ull *xwords;                 // [2][kSmallMaxBlocks][16] tagged words of the proposal exchange
     // --- uninitialised region ---
     int32_t *raw_ptr;            // [N+1]
     int32_t *raw_uses;           // [E]
@@ -67,6 +69,11 @@ struct Workspace {
     int64_t *geo_t;              // [2*E]
     int32_t *geo_a, *geo_b;      // [2*E]
     Proposal *proposals;         // [max blocks]
+    Proposal *prop_stale;        // [max blocks]
+    unsigned char *c_state;      // [E] per-period state of the lazy planner
+    ull *c_ben_lo, *c_ben_hi, *c_cost;   // [E] cached benefit and cost
+    int *worklist;               // [2*E]
+    int64_t *busy_rep, *hocc_rep; // per-block copies of the channel bookings / host occupancy (small-trace planner)
     int64_t *peak_part;          // [max blocks]
     g10_migration *migrations;   // host mode only
     int64_t *summary;            // [8]
@@ -107,6 +114,8 @@ struct PlanParams {
 };
 
 constexpr int kMaxPlanBlocks = 1024;
+constexpr int kSmallMaxBlocks = 160;       // blocks of the small-trace planner (one per SM, at most)
+constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock fit in shared memory
 
 // passes (g10_passes.cu)
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);

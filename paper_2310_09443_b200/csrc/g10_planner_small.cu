@@ -1,0 +1,485 @@
+// Algorithm 1 for traces whose timeline fits in shared memory (a few thousand kernels: every DNN-shaped
+// configuration).  Each block keeps a private, identical copy of the planner state -- pressure and slot
+// clock in shared memory, channel bookings and host occupancy in a private slice of global memory -- and
+// owns a fixed share of the periods (period p belongs to block p mod G).  One iteration is then:
+//   1. every block rescores those of its periods whose score can have changed (state STALE / DIRTY, as in
+//      the large-trace planner), from shared memory;
+//   2. block-local argmax, published with an iteration tag; every block polls all G tagged slots and reduces
+//      them to the same global winner (this exchange is the only grid-wide synchronisation of the iteration);
+//   3. every block applies the winner to its own copy of the state and reclassifies its own periods.
+// Because all copies evolve identically no block ever reads another block's state, so no barrier separates
+// the commit from the next scoring round.
+#include <cstdio>
+
+#include "g10_planner.cuh"
+
+namespace g10 {
+
+enum { kFreshS = 1, kStaleS = 2, kDirtyS = 3 };
+
+// A block's proposal travels as kXWords 64-bit words, each holding 32 bits of payload and the 32-bit
+// iteration tag: a reader that finds the expected tag in a word knows the payload half next to it belongs
+// to this iteration (64-bit accesses are single-copy atomic), so no fence is needed on either side.
+constexpr int kXWords = 16;
+struct XPayload {                // 64 bytes = 16 payload halves
+    ull ben_lo, ben_hi;          // winner's benefit
+    long long t;                 // transfer time (cost = 2 t)
+    long long bytes;             // tensor size
+    int idx, dest;               // period, destination (-1 = no candidate)
+    int wa, wap, wbp, wb;        // evict slots [wa, wap-1], absent [wap, wbp], prefetch [wbp+1, wb]
+    int tensor, pad;
+};
+static_assert(sizeof(XPayload) == 4 * kXWords, "payload must fill the exchange words");
+
+struct SmallArgs {
+    int64_t *busy_rep;      // [G][4][K]
+    int64_t *hocc_rep;      // [G][K]
+    ull *xwords;            // [2][G][kXWords] tagged proposals, then [2][G][kXWords] winner records, one copy per block
+                            // (all start zeroed; tags start at 1)
+    int cand_cap;           // periods a block can own
+};
+
+// Static facts of an owned period, cached in shared memory for the whole run.
+struct PeriodInfo {
+    long long bytes;
+    long long t[2];
+    int a, b;                // inactive slots [a, b] = [u+1, v-1]
+    int ap[2], bp[2];        // absent range per destination (ap < 0: unusable)
+    int tensor, pad;
+};
+
+// busy + overlap <= dur over slots k0..k1 for the window [w0, w1), clock in shared memory; whole warp
+__device__ __forceinline__ bool window_free_s(const int64_t *sStart, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane)
+{
+    bool ok = true;
+    for (int k = k0 + lane; k <= k1; k += 32) {
+        const int64_t s0 = sStart[k], s1 = sStart[k + 1];
+        const int64_t lo = w0 > s0 ? w0 : s0, hi = w1 < s1 ? w1 : s1;
+        const int64_t ov = hi > lo ? hi - lo : 0;
+        if (busy[k] + ov > s1 - s0) ok = false;
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void st_volatile_u64(ull *p, ull v)
+{
+    asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Half-warp poll: lanes 0-15 (or 16-31) of a warp each read one word of a record, so that a poll is one
+// coalesced 128-byte request.  Returns when all 16 words carry `tag` (the payload word of every lane is then
+// in *word); gives up (false) when the grid-wide error flag is raised or after kBarrierTimeoutNs, raising
+// the flag itself.  `active` lanes must form complete half-warps; inactive lanes pass through.
+__device__ __forceinline__ bool poll_record_halfwarp(const ull *rec, bool active, ull tag, unsigned *word, unsigned *error_flag)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned half_mask = (lane < 16) ? 0x0000ffffu : 0xffff0000u;
+    const unsigned act = __ballot_sync(0xffffffffu, active);
+    unsigned polls = 0;
+    ull t0 = 0;
+    bool ok = true;
+    for (;;) {
+        bool mine_ok = true;
+        if (active) {
+            ull x;
+            asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(x) : "l"(rec + (lane & 15)) : "memory");
+            mine_ok = (x & 0xffffffff00000000ull) == tag;
+            *word = (unsigned)x;
+        }
+        const unsigned good = __ballot_sync(0xffffffffu, mine_ok);
+        // done when every active half-warp is complete
+        const bool lo_done = ((act & 0x0000ffffu) == 0u) || ((good & 0x0000ffffu) == 0x0000ffffu);
+        const bool hi_done = ((act & 0xffff0000u) == 0u) || ((good & 0xffff0000u) == 0xffff0000u);
+        (void)half_mask;
+        if (lo_done && hi_done) break;
+        if ((++polls & 255u) == 0u) {
+            if (t0 == 0) t0 = global_timer_ns();
+            const bool stop = ld_acquire_u32(error_flag) || global_timer_ns() - t0 > kBarrierTimeoutNs;
+            if (__any_sync(0xffffffffu, stop)) { ok = false; break; }
+        }
+    }
+    if (!ok && lane == 0) atomicExch(error_flag, 1u);
+    return ok;
+}
+
+#ifdef G10_PHASE_CLOCKS
+#define PHASE_CLOCK(var) var = clock64()
+#else
+#define PHASE_CLOCK(var)
+#endif
+
+__global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, SmallArgs S)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ Cand s_cand[kPlanWarps + 1];
+    __shared__ BestScratch s_best;
+    __shared__ XPayload s_pay;
+    __shared__ __align__(16) unsigned char s_recs[kSmallMaxBlocks * sizeof(XPayload)];
+    __shared__ int s_n_over;
+    __shared__ unsigned s_err;
+    const int G = gridDim.x, c = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int K = (int)A.K;
+    const int64_t Pn = *A.Pn_dev < A.geo_stride ? *A.Pn_dev : A.geo_stride;
+    const int64_t limit = (A.max_iterations <= 0 || A.max_iterations > Pn) ? Pn : A.max_iterations;
+    const int n_local = (int)((Pn - c + G - 1) / G > 0 ? (Pn - c + G - 1) / G : 0);     // periods c, c + G, ...
+
+    int64_t *sP = (int64_t *)smem_raw;
+    int64_t *sStart = sP + K;
+    ull *cben_lo = (ull *)(sStart + K + 1);
+    ull *cben_hi = cben_lo + S.cand_cap;
+    PeriodInfo *info = (PeriodInfo *)(cben_hi + S.cand_cap);
+    unsigned char *cstate = (unsigned char *)(info + S.cand_cap);
+    int64_t *busy = S.busy_rep + (size_t)c * 4 * K;
+    int64_t *hocc = S.hocc_rep + (size_t)c * K;
+#ifdef G10_PHASE_CLOCKS
+    long long c0 = 0, c1 = 0, c2 = 0, c3 = 0, c4 = 0, acc_eval = 0, acc_local = 0, acc_xchg = 0, acc_apply = 0;
+    long long d0 = 0, d1 = 0, d2 = 0, d3 = 0, acc_loop = 0, acc_bb = 0, acc_poll = 0, acc_bb2 = 0;
+#endif
+
+    if (threadIdx.x == 0) { s_n_over = 0; s_err = 0; }
+    __syncthreads();
+    {
+        int over = 0;
+        for (int k = threadIdx.x; k < K; k += kPlanThreads) {
+            const int64_t pv = A.P[k];
+            sP[k] = pv;
+            if (pv > A.cap) ++over;
+        }
+        for (int k = threadIdx.x; k <= K; k += kPlanThreads) sStart[k] = A.start[k];
+        for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
+            const int64_t p = (int64_t)li * G + c;
+            PeriodInfo I;
+            I.tensor = A.per_t[p];
+            I.bytes = A.bytes[I.tensor];
+            I.a = A.per_u[p] + 1; I.b = A.per_v[p] - 1;
+            for (int X = 0; X < 2; ++X) {
+                I.t[X] = A.geo_t[X * A.geo_stride + p];
+                I.ap[X] = A.geo_a[X * A.geo_stride + p];
+                I.bp[X] = A.geo_b[X * A.geo_stride + p];
+            }
+            I.pad = 0;
+            info[li] = I;
+            cstate[li] = (unsigned char)(kDirtyS << 2);
+        }
+        for (int k = threadIdx.x; k < 4 * K; k += kPlanThreads) busy[k] = 0;
+        if (A.host_capacity != 0) for (int k = threadIdx.x; k < K; k += kPlanThreads) hocc[k] = 0;
+        if (over) atomicAdd(&s_n_over, over);
+    }
+    __syncthreads();
+
+    int64_t n_mig = 0, rounds = 0, bytes_ssd = 0, bytes_host = 0;
+    int status = -1;
+    for (int64_t it = 0;; ++it) {
+        if (A.fits_always || s_n_over == 0) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
+        if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
+        rounds += 1;
+        PHASE_CLOCK(c0);
+        // ---------------- 1. bring this block's periods up to date (one warp per period)
+        for (int li = warp; li < n_local; li += kPlanWarps) {
+            const unsigned char st = cstate[li];
+            if (st == 0 || (st >> 2) == kFreshS) continue;
+            const int a = info[li].a, b = info[li].b;
+            const int64_t s = info[li].bytes;
+            int d = (st & 3) - 1;
+            if ((st >> 2) == kDirtyS) {
+                const int64_t t_r = sStart[a], t_end = sStart[b + 1];
+                d = -1;
+                for (int X = 0; X < 2 && d < 0; ++X) {
+                    const int ap = info[li].ap[X];
+                    if (ap < 0) continue;
+                    const int bp = info[li].bp[X];
+                    const int64_t t = info[li].t[X];
+                    if (!window_free_s(sStart, busy + (size_t)(2 * X) * K, t_r, t_r + t, a, ap - 1, lane)) continue;
+                    if (!window_free_s(sStart, busy + (size_t)(2 * X + 1) * K, t_end - t, t_end, bp + 1, b, lane)) continue;
+                    if (X == G10_DEST_HOST && A.host_capacity != 0) {
+                        bool ok = true;
+                        for (int k = a + lane; k <= b; k += 32)
+                            if ((uint64_t)hocc[k] + (uint64_t)s > A.host_capacity) ok = false;
+                        if (!__all_sync(0xffffffffu, ok)) continue;
+                    }
+                    d = X;
+                }
+                if (d < 0) { if (lane == 0) cstate[li] = 0; continue; }     // channels only fill up: gone for good
+            }
+            const int ap = info[li].ap[d], bp = info[li].bp[d];
+            u128 acc = 0;
+            for (int k = ap + lane; k <= bp; k += 32) {
+                int64_t ex = sP[k] - A.cap;
+                if (ex > 0) {
+                    if (ex > s) ex = s;
+                    acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
+                }
+            }
+            acc = warp_sum_u128(acc);
+            if (lane == 0) {
+                cben_lo[li] = (ull)acc; cben_hi[li] = (ull)(acc >> 64);
+                cstate[li] = (unsigned char)((d + 1) | (kFreshS << 2));
+            }
+        }
+        __syncthreads();
+        PHASE_CLOCK(c1);
+        // ---------------- 2. block-local argmax, published as tagged words
+        const int par = (int)(it & 1);
+        const ull tag = (ull)(unsigned)(it + 1) << 32;
+        if (n_local <= 64) {
+            // few periods: warp 0 alone finds the block's best (no block-wide barrier on this path)
+            if (warp == 0) {
+                Cand best;
+                best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
+                int bli = -1;
+                for (int li = lane; li < n_local; li += 32) {
+                    const unsigned char st = cstate[li];
+                    if (st == 0) continue;
+                    Cand x;
+                    x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li];
+                    if (x.ben == 0) continue;
+                    x.dest = (st & 3) - 1;
+                    x.cost = 2ull * (ull)info[li].t[x.dest]; x.idx = (int)((int64_t)li * G + c);
+                    if (cand_beats(x, best)) { best = x; bli = li; }
+                }
+                const double k = cand_key(best);
+                double m = k;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) { const double y = __shfl_xor_sync(0xffffffffu, m, o); if (y > m) m = y; }
+                const unsigned fin = __ballot_sync(0xffffffffu, k >= 0.0 && k >= m * (1.0 - 1e-10));
+                int src = -1;
+                if (__popc(fin) == 1) src = __ffs(fin) - 1;
+                else if (fin != 0u) {
+                    // several lanes within rounding of the maximum: settle it exactly
+                    Cand z = best;
+                    if (!((fin >> lane) & 1u)) z.idx = -1;
+#pragma unroll 1
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const Cand y = cand_shfl_xor(z, o);
+                        if (cand_beats(y, z)) z = y;
+                    }
+                    src = __ffs(__ballot_sync(0xffffffffu, best.idx >= 0 && best.idx == z.idx)) - 1;
+                }
+                if (src < 0) {
+                    if (lane == 0) { s_pay.idx = -1; s_pay.dest = -1; s_pay.ben_lo = 0; s_pay.ben_hi = 0; s_pay.t = 0; }
+                } else if (lane == src) {
+                    const PeriodInfo &I = info[bli];
+                    XPayload q;
+                    q.ben_lo = (ull)best.ben; q.ben_hi = (ull)(best.ben >> 64); q.idx = best.idx; q.dest = best.dest;
+                    q.t = I.t[best.dest]; q.bytes = I.bytes; q.wa = I.a; q.wb = I.b; q.wap = I.ap[best.dest]; q.wbp = I.bp[best.dest];
+                    q.tensor = I.tensor; q.pad = 0;
+                    s_pay = q;
+                }
+                __syncwarp();
+                if (lane < kXWords)
+                    st_volatile_u64(&S.xwords[((size_t)par * G + c) * kXWords + lane], tag | ((const unsigned *)&s_pay)[lane]);
+                __syncwarp();
+            }
+        } else {
+            Cand best;
+            best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
+            for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
+                const unsigned char st = cstate[li];
+                if (st == 0) continue;
+                Cand x;
+                x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li];
+                if (x.ben == 0) continue;
+                x.dest = (st & 3) - 1;
+                x.cost = 2ull * (ull)info[li].t[x.dest]; x.idx = (int)((int64_t)li * G + c);
+                if (cand_beats(x, best)) best = x;
+            }
+            best = block_best_fast(best, &s_best, s_cand);
+            if (threadIdx.x == 0) {
+                XPayload q;
+                q.ben_lo = (ull)best.ben; q.ben_hi = (ull)(best.ben >> 64); q.idx = best.idx; q.dest = best.dest;
+                q.t = 0; q.bytes = 0; q.wa = q.wap = q.wbp = q.wb = 0; q.tensor = 0; q.pad = 0;
+                if (best.idx >= 0) {
+                    const PeriodInfo &I = info[best.idx / G];
+                    q.t = I.t[best.dest]; q.bytes = I.bytes; q.wa = I.a; q.wb = I.b; q.wap = I.ap[best.dest]; q.wbp = I.bp[best.dest];
+                    q.tensor = I.tensor;
+                }
+                s_pay = q;
+            }
+            __syncthreads();
+            if (threadIdx.x < kXWords)
+                st_volatile_u64(&S.xwords[((size_t)par * G + c) * kXWords + threadIdx.x], tag | ((const unsigned *)&s_pay)[threadIdx.x]);
+            __syncthreads();                               // s_pay is reused for the winner's record below
+        }
+        PHASE_CLOCK(c2);
+        // ---------------- block 0 reads all G proposals (one half-warp per record), reduces them and writes one
+        // copy of the winner's record per block; every other block polls its own copy (no hot line)
+        ull *win_words = &S.xwords[((size_t)2 * G + (size_t)par * G) * kXWords];      // [G] copies for this parity
+        if (c == 0) {
+            XPayload *recs = (XPayload *)s_recs;
+            for (int j0 = 0; j0 < G; j0 += kPlanThreads / 16) {
+                const int j = j0 + (threadIdx.x >> 4);
+                unsigned word = 0;
+                const bool active = j < G;
+                if (!poll_record_halfwarp(&S.xwords[((size_t)par * G + (active ? j : 0)) * kXWords], active, tag, &word, &A.bar->error))
+                    s_err = 1u;
+                if (active) ((unsigned *)&recs[j])[threadIdx.x & 15] = word;
+            }
+            __syncthreads();
+            Cand x;
+            x.ben = 0; x.cost = 1; x.idx = -1; x.dest = -1;
+            for (int j = threadIdx.x; j < G; j += kPlanThreads) {
+                const XPayload &y = recs[j];
+                if (y.idx < 0) continue;
+                Cand cy;
+                cy.ben = ((u128)y.ben_hi << 64) | y.ben_lo; cy.cost = 2ull * (ull)y.t; cy.idx = y.idx; cy.dest = y.dest;
+                if (cand_beats(cy, x)) x = cy;
+            }
+            PHASE_CLOCK(d2);
+            const Cand gw = block_best_fast(x, &s_best, s_cand);         // (its barriers also publish s_err)
+            PHASE_CLOCK(d3);
+            if (threadIdx.x == 0) {
+                if (gw.idx < 0) { s_pay.idx = -1; s_pay.dest = -1; }
+                else s_pay = recs[gw.idx % G];             // period p was proposed by block p mod G
+            }
+            __syncthreads();
+            if (!s_err)
+                for (int w = threadIdx.x; w < G * kXWords; w += kPlanThreads)
+                    st_volatile_u64(&win_words[w], tag | ((const unsigned *)&s_pay)[w & (kXWords - 1)]);
+        } else {
+            if (warp == 0) {
+                unsigned word = 0;
+                const bool active = lane < 16;
+                if (!poll_record_halfwarp(&win_words[(size_t)c * kXWords], active, tag, &word, &A.bar->error)) s_err = 1u;
+                else if (active) ((unsigned *)&s_pay)[lane] = word;
+            }
+            __syncthreads();
+        }
+        if (s_err) { status = -2; break; }
+        const XPayload win = s_pay;
+        if (win.idx < 0) { status = G10_EXHAUSTED; break; }
+        PHASE_CLOCK(c3);
+        // ---------------- 3. apply the winner to this block's copy of the state
+        {
+            const int64_t p = win.idx;
+            const int X = win.dest;
+            const int wa = win.wa, wb = win.wb, wap = win.wap, wbp = win.wbp;
+            const int64_t s = win.bytes, t = win.t;
+            const int64_t t_r = sStart[wa], t_end = sStart[wb + 1];
+            int fell = 0;
+            for (int k = wap + threadIdx.x; k <= wbp; k += kPlanThreads) {
+                const int64_t before = sP[k], after = before - s;
+                sP[k] = after;
+                if (before > A.cap && after <= A.cap) ++fell;
+            }
+            if (fell) atomicSub(&s_n_over, fell);
+            int64_t *bo = busy + (size_t)(2 * X) * K, *bi = busy + (size_t)(2 * X + 1) * K;
+            for (int k = wa + threadIdx.x; k <= wap - 1; k += kPlanThreads) {
+                const int64_t s0 = sStart[k], s1 = sStart[k + 1];
+                const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
+                if (hi > lo) bo[k] += hi - lo;
+            }
+            for (int k = wbp + 1 + threadIdx.x; k <= wb; k += kPlanThreads) {
+                const int64_t s0 = sStart[k], s1 = sStart[k + 1];
+                const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
+                if (hi > lo) bi[k] += hi - lo;
+            }
+            if (X == G10_DEST_HOST && A.host_capacity != 0)
+                for (int k = wa + threadIdx.x; k <= wb; k += kPlanThreads) hocc[k] += s;
+            // reclassify this block's periods against the winner's slot ranges
+            for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
+                const unsigned char st = cstate[li];
+                if (st == 0) continue;
+                if ((int64_t)li * G + c == p) { cstate[li] = 0; continue; }
+                int state = st >> 2;
+                if (state == kDirtyS) continue;
+                const int d = (st & 3) - 1;
+                const int qa = info[li].a, qb = info[li].b;
+                if (!(qa <= wb && wa <= qb)) continue;
+                const int ap = info[li].ap[d], bp = info[li].bp[d];
+                bool hit = false;
+                if (d == X) {
+                    hit = (qa <= wap - 1 && wa <= ap - 1) || (bp + 1 <= wb && wbp + 1 <= qb);
+                    if (!hit && d == G10_DEST_HOST && A.host_capacity != 0) hit = true;
+                }
+                if (hit) state = kDirtyS;
+                else if (state == kFreshS && ap <= wbp && wap <= bp) state = kStaleS;
+                cstate[li] = (unsigned char)((st & 3) | (state << 2));
+            }
+            if (c == 0 && threadIdx.x == 0) {
+                if (n_mig < A.out_cap) {
+                    g10_migration m;
+                    m.period = (int32_t)p; m.tensor = win.tensor; m.dest = X; m.absent_first = wap; m.absent_last = wbp;
+                    m.iteration = (int32_t)it; m.evict_issue_ns = t_r; m.prefetch_issue_ns = t_end - t; m.transfer_ns = t;
+                    A.out[n_mig] = m;
+                } else raise_status(A.status, G10_DEV_PLAN_OVERFLOW);
+            }
+            n_mig += 1;
+            if (X == G10_DEST_SSD) bytes_ssd += s; else bytes_host += s;
+        }
+        __syncthreads();
+#ifdef G10_PHASE_CLOCKS
+        c4 = clock64();
+        acc_eval += c1 - c0; acc_local += c2 - c1; acc_xchg += c3 - c2; acc_apply += c4 - c3;
+        acc_loop += d0 - c1; acc_bb += d1 - d0; acc_poll += d2 - c2; acc_bb2 += d3 - d2;
+#endif
+    }
+    // ---------------- epilogue: block 0 writes the final pressure and the summary
+    if (c != 0) return;
+    __syncthreads();
+#ifdef G10_PHASE_CLOCKS
+    if (threadIdx.x == 0)
+        printf("k_plan_small clocks per iteration: eval %lld local %lld exchange %lld apply %lld (iterations %lld)\n",
+               acc_eval / (rounds ? rounds : 1), acc_local / (rounds ? rounds : 1), acc_xchg / (rounds ? rounds : 1),
+               acc_apply / (rounds ? rounds : 1), (long long)rounds);
+    if (threadIdx.x == 0)
+        printf("   local: loop %lld block_best %lld | exchange (leader): poll %lld block_best %lld\n", acc_loop / (rounds ? rounds : 1),
+               acc_bb / (rounds ? rounds : 1), acc_poll / (rounds ? rounds : 1), acc_bb2 / (rounds ? rounds : 1));
+#endif
+    long long pk = 0;
+    int ps = -1;
+    for (int k = threadIdx.x; k < K; k += kPlanThreads) {
+        const long long pv = sP[k];
+        A.P[k] = pv;
+        if (ps < 0 || pv > pk) { pk = pv; ps = k; }      // k ascending per thread: first maximum kept
+    }
+    __shared__ long long s_pk[kPlanThreads];
+    __shared__ int s_ps[kPlanThreads];
+    s_pk[threadIdx.x] = pk; s_ps[threadIdx.x] = ps;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int j = 1; j < kPlanThreads; ++j)
+            if (s_ps[j] >= 0 && (ps < 0 || s_pk[j] > pk || (s_pk[j] == pk && s_ps[j] < ps))) { pk = s_pk[j]; ps = s_ps[j]; }
+        if (status == -2) raise_status(A.status, G10_DEV_TIMEOUT);
+        A.summary[0] = n_mig; A.summary[1] = rounds; A.summary[2] = status == -2 ? -1 : status;
+        A.summary[3] = ps < 0 ? 0 : pk; A.summary[4] = ps;
+        A.summary[5] = bytes_ssd; A.summary[6] = bytes_host;
+    }
+}
+
+// Shared memory the small-trace planner needs for K slots and `cand_cap` periods per block.
+static size_t small_smem_bytes(int64_t K, int cand_cap)
+{
+    return (size_t)(2 * K + 1) * 8 + (size_t)cand_cap * (16 + sizeof(PeriodInfo) + 1) + 16;
+}
+
+bool plan_small_fits(int64_t K, int64_t E, int G, int *cand_cap_out, size_t *smem_out)
+{
+    if (G < 1) return false;
+    const int cand_cap = (int)((E + G - 1) / G) + 1;
+    const size_t smem = small_smem_bytes(K, cand_cap);
+    *cand_cap_out = cand_cap;
+    *smem_out = smem;
+    return smem <= 200 * 1024;
+}
+
+int plan_small_blocks()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return sms > kMaxPlanBlocks ? kMaxPlanBlocks : sms;
+}
+
+cudaError_t launch_plan_small(const PlanArgs &A_in, const Workspace &w, int G, int cand_cap, size_t smem, cudaStream_t s)
+{
+    PlanArgs A = A_in;
+    SmallArgs S;
+    S.busy_rep = w.busy_rep; S.hocc_rep = w.hocc_rep; S.xwords = w.xwords; S.cand_cap = cand_cap;
+    cudaError_t e = cudaFuncSetAttribute(k_plan_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    void *args[] = {&A, &S};
+    return cudaLaunchCooperativeKernel((const void *)k_plan_small, dim3(G), dim3(kPlanThreads), args, smem, s);
+}
+
+}  // namespace g10

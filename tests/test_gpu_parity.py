@@ -88,10 +88,14 @@ def full_parity(gpu, oracle, tr, lazy_oracle=False, repeats=1, **plan_kw):
     tl, (start, P0, peak, slot) = check_timeline(gpu, oracle, tr, tb)
     check_geometry(gpu, oracle, tr, tb, v, ov, tl)
     cap = tr.capacity_from_peak(int(tl.peak_bytes.item()))
+    also = plan_kw.pop("also_rescore_all", True)
     ref = oracle.plan(tr, tr.capacity_from_peak(peak), lazy=lazy_oracle,
                       host_capacity_bytes=plan_kw.get("host_capacity", 0), max_iterations=plan_kw.get("max_iterations", 0))
     for _ in range(repeats):
         check_plan(gpu, tr, tb, cap, ref, **plan_kw)
+    if also:
+        check_plan(gpu, tr, tb, cap, ref, flags=gpu.FLAG_RESCORE_ALL, **plan_kw)      # Algorithm 1 as printed
+        check_plan(gpu, tr, tb, cap, ref, flags=gpu.FLAG_GLOBAL_STATE, **plan_kw)     # the large-trace planner
     return ref
 
 
@@ -229,14 +233,14 @@ def test_host_pointer_mode(gpu, oracle):
 
 def test_full_size_stress_dag_passes(gpu, oracle):
     """Config 4 at full size (K = 1e6, N = 4e6): vitality and timeline element by element; the plan's first
-    200 iterations bit for bit against the oracle's lazy tier, and the invariants of a valid plan on them."""
+    1000 iterations bit for bit against the oracle's lazy tier, and the invariants of a valid plan on them."""
     import torch
     tr = traces.config4_stress_dag()
     tb = gpu.upload(tr)
     v, ov = check_vitality(gpu, oracle, tr, tb)
     tl, (start, P0, peak, slot) = check_timeline(gpu, oracle, tr, tb)
     cap = tr.capacity_from_peak(peak)
-    ref = oracle.plan(tr, cap, lazy=True, max_iterations=200)
-    plan = check_plan(gpu, tr, tb, cap, ref, max_iterations=200)
+    ref = oracle.plan(tr, cap, lazy=True, max_iterations=1000)
+    plan = check_plan(gpu, tr, tb, cap, ref, max_iterations=1000)
     helpers.check_plan_invariants(tr, cap, start, P0, ov, gpu.migrations_numpy(plan), _np(plan.final_pressure),
                                   gpu.STATUS[int(plan.summary[2].item())], tr.host_bw, tr.ssd_bw, check_area=False)
