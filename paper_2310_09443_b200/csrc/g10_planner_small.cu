@@ -52,11 +52,12 @@ struct PeriodInfo {
 __device__ __forceinline__ bool window_free_s(const int64_t *sStart, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane)
 {
     bool ok = true;
+#pragma unroll 1
     for (int k = k0 + lane; k <= k1; k += 32) {
         const int64_t s0 = sStart[k], s1 = sStart[k + 1];
         const int64_t lo = w0 > s0 ? w0 : s0, hi = w1 < s1 ? w1 : s1;
         const int64_t ov = hi > lo ? hi - lo : 0;
-        if (busy[k] + ov > s1 - s0) ok = false;
+        if (__ldcg(&busy[k]) + ov > s1 - s0) ok = false;      // bookings are reductions performed at L2
     }
     return __all_sync(0xffffffffu, ok);
 }
@@ -102,12 +103,17 @@ __device__ __forceinline__ bool poll_record_halfwarp(const ull *rec, bool active
     return ok;
 }
 
+// Developer aid (off in the library build): with -DG10_PHASE_CLOCKS thread 0 of blocks 0 and 1 accumulates
+// the cycles between the marked points of an iteration and prints the averages when the loop ends.
 #ifdef G10_PHASE_CLOCKS
-#define PHASE_CLOCK(var) var = clock64()
+#define PHASE_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
+                             ph_acc[i] += now_ - ph_last; ph_last = now_; asm volatile("" ::: "memory"); } } while (0)
 #else
-#define PHASE_CLOCK(var)
+#define PHASE_CLOCK(i)
 #endif
 
+// kFew: every block owns at most 256 periods (warp 0 alone finds the block's best candidate).
+template <bool kFew>
 __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, SmallArgs S)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -116,6 +122,8 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
     __shared__ XPayload s_pay;
     __shared__ __align__(16) unsigned char s_recs[kSmallMaxBlocks * sizeof(XPayload)];
     __shared__ int s_n_over;
+    __shared__ int s_todo;
+    __shared__ ull s_part[2 * kPlanWarps];
     __shared__ unsigned s_err;
     const int G = gridDim.x, c = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -126,33 +134,40 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
 
     int64_t *sP = (int64_t *)smem_raw;
     int64_t *sStart = sP + K;
-    ull *cben_lo = (ull *)(sStart + K + 1);
+    int64_t *sDur = sStart + K + 1;
+    ull *cben_lo = (ull *)(sDur + K);
     ull *cben_hi = cben_lo + S.cand_cap;
-    PeriodInfo *info = (PeriodInfo *)(cben_hi + S.cand_cap);
+    double *ckey = (double *)(cben_hi + S.cand_cap);        // rounded benefit/cost of the cached score
+    PeriodInfo *info = (PeriodInfo *)(ckey + S.cand_cap);
     unsigned char *cstate = (unsigned char *)(info + S.cand_cap);
     int64_t *busy = S.busy_rep + (size_t)c * 4 * K;
     int64_t *hocc = S.hocc_rep + (size_t)c * K;
 #ifdef G10_PHASE_CLOCKS
-    long long c0 = 0, c1 = 0, c2 = 0, c3 = 0, c4 = 0, acc_eval = 0, acc_local = 0, acc_xchg = 0, acc_apply = 0;
-    long long d0 = 0, d1 = 0, d2 = 0, d3 = 0, acc_loop = 0, acc_bb = 0, acc_poll = 0, acc_bb2 = 0;
+    long long ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
 #endif
 
     if (threadIdx.x == 0) { s_n_over = 0; s_err = 0; }
     __syncthreads();
     {
         int over = 0;
+#pragma unroll 1
         for (int k = threadIdx.x; k < K; k += kPlanThreads) {
             const int64_t pv = A.P[k];
             sP[k] = pv;
             if (pv > A.cap) ++over;
         }
+#pragma unroll 1
         for (int k = threadIdx.x; k <= K; k += kPlanThreads) sStart[k] = A.start[k];
+#pragma unroll 1
+        for (int k = threadIdx.x; k < K; k += kPlanThreads) sDur[k] = A.dur[k];
+#pragma unroll 1
         for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
             const int64_t p = (int64_t)li * G + c;
             PeriodInfo I;
             I.tensor = A.per_t[p];
             I.bytes = A.bytes[I.tensor];
             I.a = A.per_u[p] + 1; I.b = A.per_v[p] - 1;
+#pragma unroll 1
             for (int X = 0; X < 2; ++X) {
                 I.t[X] = A.geo_t[X * A.geo_stride + p];
                 I.ap[X] = A.geo_a[X * A.geo_stride + p];
@@ -162,6 +177,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             info[li] = I;
             cstate[li] = (unsigned char)(kDirtyS << 2);
         }
+#pragma unroll 1
         for (int k = threadIdx.x; k < 4 * K; k += kPlanThreads) busy[k] = 0;
         if (A.host_capacity != 0) for (int k = threadIdx.x; k < K; k += kPlanThreads) hocc[k] = 0;
         if (over) atomicAdd(&s_n_over, over);
@@ -170,21 +186,26 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
 
     int64_t n_mig = 0, rounds = 0, bytes_ssd = 0, bytes_host = 0;
     int status = -1;
+#pragma unroll 1
     for (int64_t it = 0;; ++it) {
         if (A.fits_always || s_n_over == 0) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
         if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
         rounds += 1;
-        PHASE_CLOCK(c0);
-        // ---------------- 1. bring this block's periods up to date (one warp per period)
+        PHASE_CLOCK(0);     // loop top (stop tests)
+        // ---------------- 1. bring this block's periods up to date (one warp per period).  With few periods per
+        // block only the DIRTY ones are done here (rare); STALE ones are rescored on demand in step 2.
+#pragma unroll 1
         for (int li = warp; li < n_local; li += kPlanWarps) {
             const unsigned char st = cstate[li];
             if (st == 0 || (st >> 2) == kFreshS) continue;
+            if (kFew && (st >> 2) == kStaleS) continue;
             const int a = info[li].a, b = info[li].b;
             const int64_t s = info[li].bytes;
             int d = (st & 3) - 1;
             if ((st >> 2) == kDirtyS) {
                 const int64_t t_r = sStart[a], t_end = sStart[b + 1];
                 d = -1;
+#pragma unroll 1
                 for (int X = 0; X < 2 && d < 0; ++X) {
                     const int ap = info[li].ap[X];
                     if (ap < 0) continue;
@@ -194,8 +215,9 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                     if (!window_free_s(sStart, busy + (size_t)(2 * X + 1) * K, t_end - t, t_end, bp + 1, b, lane)) continue;
                     if (X == G10_DEST_HOST && A.host_capacity != 0) {
                         bool ok = true;
+#pragma unroll 1
                         for (int k = a + lane; k <= b; k += 32)
-                            if ((uint64_t)hocc[k] + (uint64_t)s > A.host_capacity) ok = false;
+                            if ((uint64_t)__ldcg(&hocc[k]) + (uint64_t)s > A.host_capacity) ok = false;
                         if (!__all_sync(0xffffffffu, ok)) continue;
                     }
                     d = X;
@@ -204,76 +226,146 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             }
             const int ap = info[li].ap[d], bp = info[li].bp[d];
             u128 acc = 0;
+#pragma unroll 1
             for (int k = ap + lane; k <= bp; k += 32) {
                 int64_t ex = sP[k] - A.cap;
                 if (ex > 0) {
                     if (ex > s) ex = s;
-                    acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
+                    acc += (u128)(ull)ex * (u128)(ull)sDur[k];
                 }
             }
             acc = warp_sum_u128(acc);
             if (lane == 0) {
+                Cand cd;
+                cd.ben = acc; cd.cost = 2ull * (ull)info[li].t[d]; cd.idx = 0; cd.dest = d;
                 cben_lo[li] = (ull)acc; cben_hi[li] = (ull)(acc >> 64);
+                ckey[li] = acc == 0 ? 0.0 : cand_key(cd);
                 cstate[li] = (unsigned char)((d + 1) | (kFreshS << 2));
             }
         }
         __syncthreads();
-        PHASE_CLOCK(c1);
+        PHASE_CLOCK(1);     // evaluation + barrier
         // ---------------- 2. block-local argmax, published as tagged words
         const int par = (int)(it & 1);
         const ull tag = (ull)(unsigned)(it + 1) << 32;
-        if (n_local <= 64) {
-            // few periods: warp 0 alone finds the block's best (no block-wide barrier on this path)
-            if (warp == 0) {
-                Cand best;
-                best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
-                int bli = -1;
-                for (int li = lane; li < n_local; li += 32) {
-                    const unsigned char st = cstate[li];
-                    if (st == 0) continue;
-                    Cand x;
-                    x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li];
-                    if (x.ben == 0) continue;
-                    x.dest = (st & 3) - 1;
-                    x.cost = 2ull * (ull)info[li].t[x.dest]; x.idx = (int)((int64_t)li * G + c);
-                    if (cand_beats(x, best)) { best = x; bli = li; }
-                }
-                const double k = cand_key(best);
-                double m = k;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) { const double y = __shfl_xor_sync(0xffffffffu, m, o); if (y > m) m = y; }
-                const unsigned fin = __ballot_sync(0xffffffffu, k >= 0.0 && k >= m * (1.0 - 1e-10));
-                int src = -1;
-                if (__popc(fin) == 1) src = __ffs(fin) - 1;
-                else if (fin != 0u) {
-                    // several lanes within rounding of the maximum: settle it exactly
-                    Cand z = best;
-                    if (!((fin >> lane) & 1u)) z.idx = -1;
+        if (kFew) {
+            // Few periods per block.  A STALE period's cached score is an upper bound (pressure only falls), so
+            // only the STALE periods whose bound could still beat the best FRESH score are rescored, best bound
+            // first, by the whole block; the loop ends when the block's best is FRESH (exact).  Rounded ratios
+            // (ckey) steer the search; anything within 1e-10 of a decision is settled by exact comparison.
+#pragma unroll 1
+            for (;;) {
+                if (warp == 0) {
+                    double kf = -1.0, ks = -1.0;
+                    int lf = -1, ls = -1;
+#pragma unroll 1
+                    for (int li = lane; li < n_local; li += 32) {
+                        const unsigned char st = cstate[li];
+                        if (st == 0) continue;
+                        const double key = ckey[li];
+                        if (!(key > 0.0)) continue;                   // no benefit: never a winner
+                        if ((st >> 2) == kFreshS) {
+                            bool take = key > kf;
+                            if (lf >= 0 && key >= kf * (1.0 - 1e-10) && kf >= key * (1.0 - 1e-10)) {
+                                Cand x, y;                               // too close to call by rounding: exact
+                                x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)info[li].t[(st & 3) - 1];
+                                x.idx = (int)((int64_t)li * G + c); x.dest = 0;
+                                const unsigned char sf = cstate[lf];
+                                y.ben = ((u128)cben_hi[lf] << 64) | cben_lo[lf]; y.cost = 2ull * (ull)info[lf].t[(sf & 3) - 1];
+                                y.idx = (int)((int64_t)lf * G + c); y.dest = 0;
+                                take = cand_beats(x, y);
+                            }
+                            if (take) { kf = key; lf = li; }
+                        } else if (key > ks) { ks = key; ls = li; }
+                    }
+                    double mf = kf, ms = ks;
 #pragma unroll 1
                     for (int o = 16; o > 0; o >>= 1) {
-                        const Cand y = cand_shfl_xor(z, o);
-                        if (cand_beats(y, z)) z = y;
+                        const double yf = __shfl_xor_sync(0xffffffffu, mf, o), ys = __shfl_xor_sync(0xffffffffu, ms, o);
+                        if (yf > mf) mf = yf;
+                        if (ys > ms) ms = ys;
                     }
-                    src = __ffs(__ballot_sync(0xffffffffu, best.idx >= 0 && best.idx == z.idx)) - 1;
+                    int todo = -1;
+                    if (ms > 0.0 && ms >= mf * (1.0 - 1e-10)) {
+                        // the best STALE bound may beat (or tie) the best FRESH score: rescore it
+                        const unsigned who = __ballot_sync(0xffffffffu, ks == ms);
+                        todo = __shfl_sync(0xffffffffu, ls, __ffs(who) - 1);
+                    } else {
+                        // the block's best is FRESH: settle near-ties between lanes exactly, build the record
+                        const unsigned fin = __ballot_sync(0xffffffffu, lf >= 0 && kf >= mf * (1.0 - 1e-10));
+                        int src = -1;
+                        Cand best;
+                        best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
+                        if (lf >= 0) {
+                            const unsigned char sf = cstate[lf];
+                            best.ben = ((u128)cben_hi[lf] << 64) | cben_lo[lf]; best.dest = (sf & 3) - 1;
+                            best.cost = 2ull * (ull)info[lf].t[best.dest]; best.idx = (int)((int64_t)lf * G + c);
+                        }
+                        if (__popc(fin) == 1) src = __ffs(fin) - 1;
+                        else if (fin != 0u) {
+                            Cand z = best;
+                            if (!((fin >> lane) & 1u)) z.idx = -1;
+#pragma unroll 1
+                            for (int o = 16; o > 0; o >>= 1) {
+                                const Cand y = cand_shfl_xor(z, o);
+                                if (cand_beats(y, z)) z = y;
+                            }
+                            src = __ffs(__ballot_sync(0xffffffffu, best.idx >= 0 && best.idx == z.idx)) - 1;
+                        }
+                        if (src < 0) {
+                            if (lane == 0) { s_pay.idx = -1; s_pay.dest = -1; s_pay.ben_lo = 0; s_pay.ben_hi = 0; s_pay.t = 0; }
+                        } else if (lane == src) {
+                            const PeriodInfo &I = info[lf];
+                            XPayload q;
+                            q.ben_lo = (ull)best.ben; q.ben_hi = (ull)(best.ben >> 64); q.idx = best.idx; q.dest = best.dest;
+                            q.t = I.t[best.dest]; q.bytes = I.bytes; q.wa = I.a; q.wb = I.b; q.wap = I.ap[best.dest]; q.wbp = I.bp[best.dest];
+                            q.tensor = I.tensor; q.pad = 0;
+                            s_pay = q;
+                        }
+                        __syncwarp();
+                        if (lane < kXWords)
+                            st_volatile_u64(&S.xwords[((size_t)par * G + c) * kXWords + lane], tag | ((const unsigned *)&s_pay)[lane]);
+                    }
+                    if (lane == 0) s_todo = todo;
                 }
-                if (src < 0) {
-                    if (lane == 0) { s_pay.idx = -1; s_pay.dest = -1; s_pay.ben_lo = 0; s_pay.ben_hi = 0; s_pay.t = 0; }
-                } else if (lane == src) {
-                    const PeriodInfo &I = info[bli];
-                    XPayload q;
-                    q.ben_lo = (ull)best.ben; q.ben_hi = (ull)(best.ben >> 64); q.idx = best.idx; q.dest = best.dest;
-                    q.t = I.t[best.dest]; q.bytes = I.bytes; q.wa = I.a; q.wb = I.b; q.wap = I.ap[best.dest]; q.wbp = I.bp[best.dest];
-                    q.tensor = I.tensor; q.pad = 0;
-                    s_pay = q;
+                __syncthreads();
+                const int li = s_todo;
+                if (li < 0) break;
+                // the whole block rescores period li
+                {
+                    const unsigned char st = cstate[li];
+                    const int d = (st & 3) - 1;
+                    const int ap = info[li].ap[d], bp = info[li].bp[d];
+                    const int64_t s = info[li].bytes;
+                    u128 acc = 0;
+#pragma unroll 2
+                    for (int k = ap + (int)threadIdx.x; k <= bp; k += kPlanThreads) {
+                        int64_t ex = sP[k] - A.cap;
+                        if (ex > 0) {
+                            if (ex > s) ex = s;
+                            acc += (u128)(ull)ex * (u128)(ull)sDur[k];
+                        }
+                    }
+                    acc = warp_sum_u128(acc);
+                    if (lane == 0) { s_part[2 * warp] = (ull)acc; s_part[2 * warp + 1] = (ull)(acc >> 64); }
+                    __syncthreads();
+                    if (threadIdx.x == 0) {
+                        u128 tot = 0;
+#pragma unroll 1
+                        for (int w = 0; w < kPlanWarps; ++w) tot += ((u128)s_part[2 * w + 1] << 64) | s_part[2 * w];
+                        Cand cd;
+                        cd.ben = tot; cd.cost = 2ull * (ull)info[li].t[d]; cd.idx = 0; cd.dest = d;
+                        cben_lo[li] = (ull)tot; cben_hi[li] = (ull)(tot >> 64);
+                        ckey[li] = tot == 0 ? 0.0 : cand_key(cd);
+                        cstate[li] = (unsigned char)((d + 1) | (kFreshS << 2));
+                    }
+                    __syncthreads();
                 }
-                __syncwarp();
-                if (lane < kXWords)
-                    st_volatile_u64(&S.xwords[((size_t)par * G + c) * kXWords + lane], tag | ((const unsigned *)&s_pay)[lane]);
-                __syncwarp();
             }
         } else {
             Cand best;
             best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
+#pragma unroll 1
             for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
                 const unsigned char st = cstate[li];
                 if (st == 0) continue;
@@ -301,12 +393,13 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                 st_volatile_u64(&S.xwords[((size_t)par * G + c) * kXWords + threadIdx.x], tag | ((const unsigned *)&s_pay)[threadIdx.x]);
             __syncthreads();                               // s_pay is reused for the winner's record below
         }
-        PHASE_CLOCK(c2);
+        PHASE_CLOCK(2);     // local argmax + publish
         // ---------------- block 0 reads all G proposals (one half-warp per record), reduces them and writes one
         // copy of the winner's record per block; every other block polls its own copy (no hot line)
         ull *win_words = &S.xwords[((size_t)2 * G + (size_t)par * G) * kXWords];      // [G] copies for this parity
         if (c == 0) {
             XPayload *recs = (XPayload *)s_recs;
+#pragma unroll 1
             for (int j0 = 0; j0 < G; j0 += kPlanThreads / 16) {
                 const int j = j0 + (threadIdx.x >> 4);
                 unsigned word = 0;
@@ -318,6 +411,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             __syncthreads();
             Cand x;
             x.ben = 0; x.cost = 1; x.idx = -1; x.dest = -1;
+#pragma unroll 1
             for (int j = threadIdx.x; j < G; j += kPlanThreads) {
                 const XPayload &y = recs[j];
                 if (y.idx < 0) continue;
@@ -325,15 +419,16 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                 cy.ben = ((u128)y.ben_hi << 64) | y.ben_lo; cy.cost = 2ull * (ull)y.t; cy.idx = y.idx; cy.dest = y.dest;
                 if (cand_beats(cy, x)) x = cy;
             }
-            PHASE_CLOCK(d2);
+            PHASE_CLOCK(3);     // leader: all proposals arrived and compared per thread
             const Cand gw = block_best_fast(x, &s_best, s_cand);         // (its barriers also publish s_err)
-            PHASE_CLOCK(d3);
+            PHASE_CLOCK(4);     // leader: block argmax
             if (threadIdx.x == 0) {
                 if (gw.idx < 0) { s_pay.idx = -1; s_pay.dest = -1; }
                 else s_pay = recs[gw.idx % G];             // period p was proposed by block p mod G
             }
             __syncthreads();
             if (!s_err)
+#pragma unroll 1
                 for (int w = threadIdx.x; w < G * kXWords; w += kPlanThreads)
                     st_volatile_u64(&win_words[w], tag | ((const unsigned *)&s_pay)[w & (kXWords - 1)]);
         } else {
@@ -348,7 +443,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
         if (s_err) { status = -2; break; }
         const XPayload win = s_pay;
         if (win.idx < 0) { status = G10_EXHAUSTED; break; }
-        PHASE_CLOCK(c3);
+        PHASE_CLOCK(5);     // leader: copies written / follower: winner record arrived
         // ---------------- 3. apply the winner to this block's copy of the state
         {
             const int64_t p = win.idx;
@@ -357,6 +452,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             const int64_t s = win.bytes, t = win.t;
             const int64_t t_r = sStart[wa], t_end = sStart[wb + 1];
             int fell = 0;
+#pragma unroll 1
             for (int k = wap + threadIdx.x; k <= wbp; k += kPlanThreads) {
                 const int64_t before = sP[k], after = before - s;
                 sP[k] = after;
@@ -364,19 +460,23 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             }
             if (fell) atomicSub(&s_n_over, fell);
             int64_t *bo = busy + (size_t)(2 * X) * K, *bi = busy + (size_t)(2 * X + 1) * K;
+#pragma unroll 1
             for (int k = wa + threadIdx.x; k <= wap - 1; k += kPlanThreads) {
                 const int64_t s0 = sStart[k], s1 = sStart[k + 1];
                 const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
-                if (hi > lo) bo[k] += hi - lo;
+                if (hi > lo) atomicAdd((ull *)&bo[k], (ull)(hi - lo));
             }
+#pragma unroll 1
             for (int k = wbp + 1 + threadIdx.x; k <= wb; k += kPlanThreads) {
                 const int64_t s0 = sStart[k], s1 = sStart[k + 1];
                 const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
-                if (hi > lo) bi[k] += hi - lo;
+                if (hi > lo) atomicAdd((ull *)&bi[k], (ull)(hi - lo));
             }
             if (X == G10_DEST_HOST && A.host_capacity != 0)
-                for (int k = wa + threadIdx.x; k <= wb; k += kPlanThreads) hocc[k] += s;
+#pragma unroll 1
+                for (int k = wa + threadIdx.x; k <= wb; k += kPlanThreads) atomicAdd((ull *)&hocc[k], (ull)s);
             // reclassify this block's periods against the winner's slot ranges
+#pragma unroll 1
             for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
                 const unsigned char st = cstate[li];
                 if (st == 0) continue;
@@ -408,26 +508,22 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             if (X == G10_DEST_SSD) bytes_ssd += s; else bytes_host += s;
         }
         __syncthreads();
-#ifdef G10_PHASE_CLOCKS
-        c4 = clock64();
-        acc_eval += c1 - c0; acc_local += c2 - c1; acc_xchg += c3 - c2; acc_apply += c4 - c3;
-        acc_loop += d0 - c1; acc_bb += d1 - d0; acc_poll += d2 - c2; acc_bb2 += d3 - d2;
-#endif
+        PHASE_CLOCK(6);     // apply + barrier
     }
+#ifdef G10_PHASE_CLOCKS
+    if (threadIdx.x == 0 && c < 2) {
+        const long long r = rounds ? rounds : 1;
+        printf("block %d cycles/iteration: top %lld eval %lld local+publish %lld gather %lld argmax %lld winner %lld apply %lld [7: %lld] (n=%lld)\n", c,
+               ph_acc[0] / r, ph_acc[1] / r, ph_acc[2] / r, ph_acc[3] / r, ph_acc[4] / r, ph_acc[5] / r, ph_acc[6] / r, ph_acc[7] / r, (long long)rounds);
+    }
+#endif
     // ---------------- epilogue: block 0 writes the final pressure and the summary
     if (c != 0) return;
     __syncthreads();
-#ifdef G10_PHASE_CLOCKS
-    if (threadIdx.x == 0)
-        printf("k_plan_small clocks per iteration: eval %lld local %lld exchange %lld apply %lld (iterations %lld)\n",
-               acc_eval / (rounds ? rounds : 1), acc_local / (rounds ? rounds : 1), acc_xchg / (rounds ? rounds : 1),
-               acc_apply / (rounds ? rounds : 1), (long long)rounds);
-    if (threadIdx.x == 0)
-        printf("   local: loop %lld block_best %lld | exchange (leader): poll %lld block_best %lld\n", acc_loop / (rounds ? rounds : 1),
-               acc_bb / (rounds ? rounds : 1), acc_poll / (rounds ? rounds : 1), acc_bb2 / (rounds ? rounds : 1));
-#endif
+
     long long pk = 0;
     int ps = -1;
+#pragma unroll 1
     for (int k = threadIdx.x; k < K; k += kPlanThreads) {
         const long long pv = sP[k];
         A.P[k] = pv;
@@ -438,6 +534,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
     s_pk[threadIdx.x] = pk; s_ps[threadIdx.x] = ps;
     __syncthreads();
     if (threadIdx.x == 0) {
+#pragma unroll 1
         for (int j = 1; j < kPlanThreads; ++j)
             if (s_ps[j] >= 0 && (ps < 0 || s_pk[j] > pk || (s_pk[j] == pk && s_ps[j] < ps))) { pk = s_pk[j]; ps = s_ps[j]; }
         if (status == -2) raise_status(A.status, G10_DEV_TIMEOUT);
@@ -450,7 +547,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
 // Shared memory the small-trace planner needs for K slots and `cand_cap` periods per block.
 static size_t small_smem_bytes(int64_t K, int cand_cap)
 {
-    return (size_t)(2 * K + 1) * 8 + (size_t)cand_cap * (16 + sizeof(PeriodInfo) + 1) + 16;
+    return (size_t)(3 * K + 1) * 8 + (size_t)cand_cap * (24 + sizeof(PeriodInfo) + 1) + 16;
 }
 
 bool plan_small_fits(int64_t K, int64_t E, int G, int *cand_cap_out, size_t *smem_out)
@@ -476,10 +573,11 @@ cudaError_t launch_plan_small(const PlanArgs &A_in, const Workspace &w, int G, i
     PlanArgs A = A_in;
     SmallArgs S;
     S.busy_rep = w.busy_rep; S.hocc_rep = w.hocc_rep; S.xwords = w.xwords; S.cand_cap = cand_cap;
-    cudaError_t e = cudaFuncSetAttribute(k_plan_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const void *kernel = cand_cap <= 256 ? (const void *)k_plan_small<true> : (const void *)k_plan_small<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     void *args[] = {&A, &S};
-    return cudaLaunchCooperativeKernel((const void *)k_plan_small, dim3(G), dim3(kPlanThreads), args, smem, s);
+    return cudaLaunchCooperativeKernel(kernel, dim3(G), dim3(kPlanThreads), args, smem, s);
 }
 
 }  // namespace g10
