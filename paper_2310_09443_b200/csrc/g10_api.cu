@@ -52,14 +52,17 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     carve_scan(c, w.count_scan, ntiles, 1);
     carve_scan(c, w.emit_scan, etiles, 2);
     carve_scan(c, w.pressure_scan, ktiles, 1);
-    w.cnt = c.take<int32_t>(N);
-    w.diff = c.take<int64_t>(K + 1);
-    w.busy = c.take<int64_t>(4 * K);
-    w.hocc = c.take<int64_t>(K);
-    w.dead = c.take<unsigned char>(E);
     w.wl_count = c.take<unsigned>(2);
     w.xwords = c.take<ull>((2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16);
     w.zero_bytes = align_up(c.off);
+    // arrays that must start at zero, cleared only by the calls that use them
+    w.cnt = c.take<int32_t>(N);
+    w.diff = c.take<int64_t>(K + 1);
+    const size_t state_begin = align_up(c.off);
+    w.busy = c.take<int64_t>(4 * K);       // busy, hocc and dead are contiguous: one memset
+    w.hocc = c.take<int64_t>(K);
+    w.dead = c.take<unsigned char>(E);
+    w.state_bytes = align_up(c.off) - state_begin;
     // scratch
     w.raw_ptr = c.take<int32_t>(N + 1);
     w.raw_uses = c.take<int32_t>(E);
@@ -138,11 +141,16 @@ int32_t check_ws(int32_t which, const g10_trace *t, void *ws, size_t ws_bytes)
     } while (0)
 
 // Prepares the workspace and returns the device view of the trace (staging it first in host mode).
-int32_t begin_call(const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, cudaStream_t s)
+enum { kZeroCounts = 1, kZeroDiff = 2, kZeroState = 4 };
+
+int32_t begin_call(const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, cudaStream_t s, int zero_mask)
 {
     Sizes z{t->num_kernels, t->num_tensors, t->num_events, t->mem == G10_MEM_HOST};
     carve(ws, z, w);
     CU(cudaMemsetAsync(w.zero_begin, 0, w.zero_bytes, s));
+    if ((zero_mask & kZeroCounts) && z.N > 0) CU(cudaMemsetAsync(w.cnt, 0, sizeof(int32_t) * (size_t)z.N, s));
+    if (zero_mask & kZeroDiff) CU(cudaMemsetAsync(w.diff, 0, sizeof(int64_t) * (size_t)(z.K + 1), s));
+    if (zero_mask & kZeroState) CU(cudaMemsetAsync(w.busy, 0, w.state_bytes, s));
     d.K = z.K; d.N = z.N; d.E = z.E;
     if (!z.host) {
         d.kernel_ptr = t->kernel_ptr; d.kernel_tensors = t->kernel_tensors; d.tensor_bytes = t->tensor_bytes;
@@ -218,7 +226,7 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(trace, ws, w, d, s);
+    rc = begin_call(trace, ws, w, d, s, kZeroCounts);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     VitalityBuffers vb;
@@ -265,7 +273,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(trace, ws, w, d, s);
+    rc = begin_call(trace, ws, w, d, s, kZeroDiff);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     int64_t *start = host ? w.start : out->kernel_start_ns;
@@ -275,7 +283,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     int64_t *st = host ? w.counts + 2 : out->status;
     CU(launch_slot_clock(d, w, start, s));
     CU(launch_first_last(d, w, w.first_use, w.last_use, s));
-    CU(launch_pressure(d, w, w.first_use, w.last_use, P, pk, ps, s));
+    CU(launch_pressure(d, w, w.first_use, w.last_use, true, P, pk, ps, s));
     CU(launch_publish_status(w, st, s));
     if (host) {
         CU(d2h(out->kernel_start_ns, w.start, (size_t)d.K + 1, s));
@@ -315,7 +323,8 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(trace, ws, w, d, s);
+    const uint32_t flags = options ? options->flags : 0;
+    rc = begin_call(trace, ws, w, d, s, kZeroCounts | kZeroDiff | (plan_keeps_state_on_chip(trace->num_kernels, trace->num_events, flags) ? 0 : kZeroState));
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
@@ -339,7 +348,7 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
     CU(launch_slot_clock(d, w, w.start, s));
     CU(launch_vitality(d, w, vb, s));
     CU(mark(1));
-    CU(launch_pressure(d, w, w.first_use, w.last_use, pp.final_pressure, w.peak_bytes, w.peak_slot, s));
+    CU(launch_pressure(d, w, w.first_use, w.last_use, false, pp.final_pressure, w.peak_bytes, w.peak_slot, s));
     CU(mark(2));
     CU(launch_geometry(d.K, d.E, w.counts + 1, w.start, d.tensor_bytes, w.period_tensor, w.period_prev_use, w.period_next_use,
                        host_bw, ssd_bw, d.E > 0 ? d.E : 1, w.geo_t, w.geo_a, w.geo_b, s));

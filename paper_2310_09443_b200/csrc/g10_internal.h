@@ -38,6 +38,7 @@ struct Workspace {
     // --- zero-initialised region (one memset per call) ---
     char *zero_begin;
     size_t zero_bytes;
+    size_t state_bytes;          // bytes of busy + hocc + dead (contiguous)
     ull *status;                 // device status word
     unsigned *heavy_count;
     int *peak_key;               // K - lowest peak slot (0 = none), reduced with atomicMax
@@ -121,7 +122,7 @@ constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock f
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s);
-cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use,
+cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);
 cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, const int64_t *start, const int64_t *tensor_bytes,
                             const int32_t *per_t, const int32_t *per_u, const int32_t *per_v, uint64_t host_bw, uint64_t ssd_bw,
@@ -129,6 +130,7 @@ cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, 
 // planner (g10_planner.cu)
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
 int plan_loop_max_blocks();
+bool plan_keeps_state_on_chip(int64_t K, int64_t E, uint32_t flags);   // true: the small-trace planner will run
 cudaError_t launch_publish_status(const Workspace &w, int64_t *dst, cudaStream_t s);
 
 }  // namespace g10

@@ -7,6 +7,198 @@
 namespace g10 {
 
 // =============================================================================================
+// Segmented single-kernel scan for the two timeline-sized scans (slot clock, pressure).  A grid of a few
+// hundred blocks -- all resident at once, launched in one wave -- gives every block one contiguous
+// segment.  Pass 1 sums the segment and publishes the sum in one 64-bit word (2 state bits + 62 value
+// bits, so no fence is needed); every block then adds up the words of ALL its predecessors (a few
+// hundred loads spread over the block, no dependency chain between blocks) and pass 2 rescans the
+// segment, now L2-resident, with that prefix.  Segment numbers come from a ticket, so a predecessor
+// has always started.
+// =============================================================================================
+constexpr int kSegThreads = 512;
+constexpr int kSegItems = 4;
+constexpr int kSegChunk = kSegThreads * kSegItems;
+constexpr int kSegMaxBlocks = 512;
+
+__device__ __forceinline__ ull seg_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
+__device__ __forceinline__ long long seg_unpack(ull w) { return (long long)(w << 2) >> 2; }     // sign-extend 62 bits
+
+// kind 0: exclusive scan of kernel_ns into start[0..K] with validation of kernel_ns and kernel_ptr
+// kind 1: inclusive scan of the difference array into the pressure, plus peak and lowest peak slot
+template <int kind>
+__global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, const int64_t *__restrict__ in, const int64_t *__restrict__ kptr,
+                                                          int64_t *__restrict__ out, unsigned *ticket, unsigned *done, ull *words,
+                                                          int64_t *blk_max, int32_t *blk_slot, int64_t *peak_bytes, int32_t *peak_slot, ull *status)
+{
+    __shared__ long long s_w[kSegThreads / 32];
+    __shared__ int s_sl[kSegThreads / 32];
+    __shared__ long long s_bcast;
+    __shared__ bool s_last;
+    const int G = gridDim.x;
+    const int g = next_tile(ticket);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t seg = ((n + G - 1) / G + kSegChunk - 1) / kSegChunk * kSegChunk;
+    const int64_t lo = (int64_t)g * seg, hi = lo + seg < n ? lo + seg : n;
+    // ---- pass 1: segment sum
+    long long sum = 0;
+    ull bad = 0;
+    for (int64_t k0 = lo + threadIdx.x; k0 < hi; k0 += 8 * kSegThreads) {
+        long long v[8], p0[8], p1[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {                      // all loads of the batch in flight together
+            const int64_t k = k0 + (int64_t)j * kSegThreads;
+            v[j] = k < hi ? in[k] : (kind == 0 ? 1 : 0);
+            if (kind == 0) { p0[j] = k < hi ? kptr[k] : 0; p1[j] = k < hi ? kptr[k + 1] : 0; }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int64_t k = k0 + (int64_t)j * kSegThreads;
+            if (k < hi) {
+                if (kind == 0) {
+                    if (v[j] < 1 || v[j] >= ((long long)1 << 44)) { bad |= G10_DEV_BAD_DURATION; v[j] = 1; }
+                    if (p0[j] > p1[j] || p0[j] < 0 || p1[j] > E || (k == 0 && p0[j] != 0) || (k == n - 1 && p1[j] != E))
+                        bad |= G10_DEV_BAD_KERNEL_PTR;
+                }
+                sum += v[j];
+            }
+        }
+    }
+    if (bad) raise_status(status, bad);
+    sum = warp_sum_i64(sum);
+    if (lane == 0) s_w[warp] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long tot = 0;
+        for (int w = 0; w < kSegThreads / 32; ++w) tot += s_w[w];
+        asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&words[g]), "l"(seg_pack(tot)) : "memory");
+    }
+    // ---- prefix of the segment: all predecessors' sums
+    long long pre = 0;
+    for (int j = threadIdx.x; j < g; j += kSegThreads) {
+        ull w;
+        unsigned polls = 0;
+        for (;;) {
+            asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(w) : "l"(&words[j]) : "memory");
+            if (w >> 62) break;
+            if (++polls > kSpinLimit) { raise_status(status, G10_DEV_TIMEOUT); w = 0; break; }
+            __nanosleep(64);
+        }
+        pre += seg_unpack(w);
+    }
+    pre = warp_sum_i64(pre);
+    __syncthreads();
+    if (lane == 0) s_w[warp] = pre;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long tot = 0;
+        for (int w = 0; w < kSegThreads / 32; ++w) tot += s_w[w];
+        s_bcast = tot;
+    }
+    __syncthreads();
+    long long carry = s_bcast;
+    // ---- pass 2: scan the segment chunk by chunk (each thread kSegItems consecutive elements)
+    long long mx = 0;
+    int sl = -1;
+    for (int64_t c0 = lo; c0 < hi; c0 += kSegChunk) {
+        const int64_t base = c0 + (int64_t)threadIdx.x * kSegItems;
+        long long v[kSegItems];
+        long long tsum = 0;
+#pragma unroll
+        for (int j = 0; j < kSegItems; ++j) {
+            const int64_t k = base + j;
+            v[j] = k < hi ? in[k] : 0;
+            if (kind == 0 && k < hi && (v[j] < 1 || v[j] >= ((long long)1 << 44))) v[j] = 1;
+            tsum += v[j];
+        }
+        const long long incl = warp_inclusive_scan_i64(tsum, lane);
+        __syncthreads();
+        if (lane == 31) s_w[warp] = incl;
+        __syncthreads();
+        long long wpre = 0, ctot = 0;
+#pragma unroll
+        for (int w = 0; w < kSegThreads / 32; ++w) { const long long x = s_w[w]; if (w < warp) wpre += x; ctot += x; }
+        long long run = carry + wpre + incl - tsum;
+#pragma unroll
+        for (int j = 0; j < kSegItems; ++j) {
+            const int64_t k = base + j;
+            if (kind == 0) { if (k < hi) out[k] = run; run += v[j]; }
+            else {
+                run += v[j];
+                if (k < hi) { out[k] = run; if (sl < 0 || run > mx) { mx = run; sl = (int)k; } }
+            }
+        }
+        carry += ctot;
+    }
+    if (kind == 0) {
+        // after its own segment the last block's carry is the sum of everything
+        if (g == G - 1 && threadIdx.x == 0) {
+            out[n] = carry;
+            if (carry >= ((long long)1 << 44)) raise_status(status, G10_DEV_BAD_DURATION);
+        }
+        return;
+    }
+    // ---- kind 1: block maximum (ties to the lowest slot), then the last block reduces the per-block results
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long omx = __shfl_down_sync(0xffffffffu, mx, o);
+        const int osl = __shfl_down_sync(0xffffffffu, sl, o);
+        if (osl >= 0 && (sl < 0 || omx > mx || (omx == mx && osl < sl))) { mx = omx; sl = osl; }
+    }
+    __syncthreads();
+    if (lane == 0) { s_w[warp] = mx; s_sl[warp] = sl; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kSegThreads / 32; ++w)
+            if (s_sl[w] >= 0 && (sl < 0 || s_w[w] > mx || (s_w[w] == mx && s_sl[w] < sl))) { mx = s_w[w]; sl = s_sl[w]; }
+        blk_max[g] = mx;
+        blk_slot[g] = sl;
+        __threadfence();
+        s_last = (atomicAdd(done, 1u) == (unsigned)G - 1u);
+    }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        long long bm = 0;
+        int bs = -1;
+        for (int t = threadIdx.x; t < G; t += kSegThreads) {
+            const long long m = __ldcg(&blk_max[t]);
+            const int s2 = __ldcg(&blk_slot[t]);
+            if (s2 >= 0 && (bs < 0 || m > bm || (m == bm && s2 < bs))) { bm = m; bs = s2; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const long long omx = __shfl_down_sync(0xffffffffu, bm, o);
+            const int osl = __shfl_down_sync(0xffffffffu, bs, o);
+            if (osl >= 0 && (bs < 0 || omx > bm || (omx == bm && osl < bs))) { bm = omx; bs = osl; }
+        }
+        __syncthreads();
+        if (lane == 0) { s_w[warp] = bm; s_sl[warp] = bs; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < kSegThreads / 32; ++w)
+                if (s_sl[w] >= 0 && (bs < 0 || s_w[w] > bm || (s_w[w] == bm && s_sl[w] < bs))) { bm = s_w[w]; bs = s_sl[w]; }
+            *peak_bytes = bs < 0 ? 0 : bm;
+            *peak_slot = bs;
+        }
+    }
+}
+
+static int seg_scan_blocks(int64_t n)
+{
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;
+        if (sms <= 0) return 1;
+    }
+    int64_t g = 2 * (int64_t)sms;
+    const int64_t by_work = (n + kSegChunk - 1) / kSegChunk;        // no point in blocks without a full chunk
+    if (g > by_work) g = by_work;
+    if (g > kSegMaxBlocks) g = kSegMaxBlocks;
+    return g < 1 ? 1 : (int)g;
+}
+
+// =============================================================================================
 // Slot clock: start = exclusive prefix sum of kernel_ns, start[K] = total.  Also checks that
 // kernel_ptr runs from 0 to E without decreasing and that every duration is >= 1.
 // =============================================================================================
@@ -51,9 +243,9 @@ __global__ void __launch_bounds__(kScanThreads) k_slot_clock(int64_t K, int64_t 
 
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s)
 {
-    const int tiles = (int)tiles_of(t.K, kScanTile);
-    TileState<1> st{w.clock_scan.ticket, w.clock_scan.flag, w.clock_scan.agg, w.clock_scan.incl};
-    k_slot_clock<<<tiles, kScanThreads, 0, s>>>(t.K, t.E, t.kernel_ns, t.kernel_ptr, start, st, tiles, w.status);
+    const int G = seg_scan_blocks(t.K);
+    k_seg_scan<0><<<G, kSegThreads, 0, s>>>(t.K, t.E, t.kernel_ns, t.kernel_ptr, start, w.clock_scan.ticket, w.clock_scan.done,
+                                          (ull *)w.clock_scan.agg, nullptr, nullptr, nullptr, nullptr, w.status);
     return cudaGetLastError();
 }
 
@@ -67,13 +259,36 @@ constexpr int kEvItems = 8;
 constexpr int kEvTile = kEvThreads * kEvItems;
 
 // last k in [lo, hi] with kptr[k] <= e  (kptr nondecreasing; lo is known to satisfy it)
-__device__ __forceinline__ int kernel_of_event(const int64_t *__restrict__ kptr, int lo, int hi, int64_t e)
+__device__ __forceinline__ int kernel_of_event(const int64_t *kptr, int lo, int hi, int64_t e)
 {
     while (lo < hi) {
         const int mid = lo + (hi - lo + 1) / 2;
         if (kptr[mid] <= e) lo = mid; else hi = mid - 1;
     }
     return lo;
+}
+
+// Stages kernel_ptr[lo .. hi + 1] of the block's event tile in shared memory when it fits, so that the
+// per-event searches run on chip.  Returns the pointer to search in and rebases lo / hi accordingly.
+constexpr int kPtrStage = 3072;
+__device__ __forceinline__ const int64_t *stage_kernel_ptr(const int64_t *__restrict__ kptr, int64_t K, int64_t base, int64_t E,
+                                                           int64_t *s_ptr, int *s_lohi, int *lo_out, int *hi_out, int *shift_out)
+{
+    if (threadIdx.x == 0) {
+        const int64_t last = (base + kEvTile <= E ? base + kEvTile : E) - 1;
+        s_lohi[0] = kernel_of_event(kptr, 0, (int)K - 1, base);
+        s_lohi[1] = kernel_of_event(kptr, s_lohi[0], (int)K - 1, last);
+    }
+    __syncthreads();
+    const int lo = s_lohi[0], hi = s_lohi[1];
+    if (hi - lo + 2 <= kPtrStage) {
+        for (int j = threadIdx.x; j <= hi - lo + 1; j += blockDim.x) s_ptr[j] = kptr[lo + j];
+        __syncthreads();
+        *lo_out = 0; *hi_out = hi - lo; *shift_out = lo;
+        return s_ptr;
+    }
+    *lo_out = lo; *hi_out = hi; *shift_out = 0;
+    return kptr;
 }
 
 // raw use count per tensor (a tensor listed twice by one kernel counts twice here; collapsed later)
@@ -154,21 +369,18 @@ __global__ void __launch_bounds__(kEvThreads) k_scatter_events(int64_t E, int64_
     }
 }
 
-// first / last use by atomic min / max (the timeline call alone does not need the sorted use lists)
+// first / last use by atomic min / max (the timeline call alone does not need the sorted use lists);
+// the results stay encoded (see below) and are decoded by the difference-array pass
 __global__ void __launch_bounds__(kEvThreads) k_first_last_events(int64_t E, int64_t N, int64_t K, const int64_t *__restrict__ kptr,
                                                                   const int32_t *__restrict__ kt, int32_t *__restrict__ first_enc,
                                                                   int32_t *__restrict__ last_enc, ull *status)
 {
     // both arrays start at zero: first_enc holds max(K - k) (0 = unused), last_enc holds max(k + 1)
-    __shared__ int s_lo, s_hi;
+    __shared__ int64_t s_ptr[kPtrStage];
+    __shared__ int s_lohi[2];
     const int64_t base = (int64_t)blockIdx.x * kEvTile;
-    if (threadIdx.x == 0) {
-        const int64_t last = (base + kEvTile <= E ? base + kEvTile : E) - 1;
-        s_lo = kernel_of_event(kptr, 0, (int)K - 1, base);
-        s_hi = kernel_of_event(kptr, s_lo, (int)K - 1, last);
-    }
-    __syncthreads();
-    const int lo = s_lo, hi = s_hi;
+    int lo, hi, shift;
+    const int64_t *sp = stage_kernel_ptr(kptr, K, base, E, s_ptr, s_lohi, &lo, &hi, &shift);
     ull bad = 0;
 #pragma unroll
     for (int j = 0; j < kEvItems; ++j) {
@@ -177,23 +389,13 @@ __global__ void __launch_bounds__(kEvThreads) k_first_last_events(int64_t E, int
             const int32_t i = kt[e];
             if (i < 0 || i >= N) bad = G10_DEV_BAD_TENSOR_ID;
             else {
-                const int k = kernel_of_event(kptr, lo, hi, e);
+                const int k = kernel_of_event(sp, lo, hi, e) + shift;
                 atomicMax(&first_enc[i], (int)K - k);
                 atomicMax(&last_enc[i], k + 1);
             }
         }
     }
     if (bad) raise_status(status, bad);
-}
-
-__global__ void k_decode_first_last(int64_t N, int64_t K, int32_t *first, int32_t *last)
-{
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < N) {
-        const int f = first[i], l = last[i];
-        first[i] = f == 0 ? -1 : (int)K - f;
-        last[i] = l - 1;
-    }
 }
 
 cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s)
@@ -207,7 +409,6 @@ cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t 
         const int blocks = (int)tiles_of(t.E, kEvTile);
         k_first_last_events<<<blocks, kEvThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.status);
     }
-    k_decode_first_last<<<(unsigned)((t.N + 255) / 256), 256, 0, s>>>(t.N, t.K, first_use, last_use);
     return cudaGetLastError();
 }
 
@@ -464,6 +665,8 @@ cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const Vita
 // alive in every slot: its size goes to D[0] only), then P = inclusive scan of D, peak and its
 // lowest slot.
 // =============================================================================================
+// kEncoded: first / last come straight from k_first_last_events (first as K - k, 0 = unused; last as k + 1).
+template <bool kEncoded>
 __global__ void __launch_bounds__(256) k_diff_scatter(int64_t N, int64_t K, const int64_t *__restrict__ bytes, const uint8_t *__restrict__ glob,
                                                       const int32_t *__restrict__ first, const int32_t *__restrict__ last,
                                                       ull *__restrict__ diff, ull *status)
@@ -474,12 +677,13 @@ __global__ void __launch_bounds__(256) k_diff_scatter(int64_t N, int64_t K, cons
     if (i < N) {
         const long long b = bytes[i];
         if (b < 1 || b >= ((long long)1 << 40)) raise_status(status, G10_DEV_BAD_BYTES);
-        const int f = first[i];
+        int f = first[i];
+        if (kEncoded) f = f == 0 ? -1 : (int)K - f;
         if (f >= 0 && f < K) {
             if (glob != nullptr && glob[i]) gsum = b;
             else {
                 atomicAdd(&diff[f], (ull)b);
-                const int l = last[i];
+                const int l = kEncoded ? last[i] - 1 : last[i];
                 if (l + 1 < K) atomicAdd(&diff[l + 1], (ull)(-b));
             }
         }
@@ -575,16 +779,19 @@ __global__ void __launch_bounds__(kScanThreads) k_scan_pressure(int64_t K, const
     }
 }
 
-cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use,
+cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
 {
-    if (t.N > 0 && t.K > 0)
-        k_diff_scatter<<<(unsigned)((t.N + 255) / 256), 256, 0, s>>>(t.N, t.K, t.tensor_bytes, t.tensor_global, first_use, last_use,
-                                                                     (ull *)w.diff, w.status);
-    const int tiles = (int)tiles_of(t.K, kScanTile);
-    TileState<1> st{w.pressure_scan.ticket, w.pressure_scan.flag, w.pressure_scan.agg, w.pressure_scan.incl};
-    k_scan_pressure<<<tiles, kScanThreads, 0, s>>>(t.K, w.diff, pressure, st, w.pressure_scan.done, w.tile_max, w.tile_slot, tiles,
-                                                   peak_bytes, peak_slot, w.status);
+    if (t.N > 0 && t.K > 0) {
+        const unsigned blocks = (unsigned)((t.N + 255) / 256);
+        if (encoded)
+            k_diff_scatter<true><<<blocks, 256, 0, s>>>(t.N, t.K, t.tensor_bytes, t.tensor_global, first_use, last_use, (ull *)w.diff, w.status);
+        else
+            k_diff_scatter<false><<<blocks, 256, 0, s>>>(t.N, t.K, t.tensor_bytes, t.tensor_global, first_use, last_use, (ull *)w.diff, w.status);
+    }
+    const int G = seg_scan_blocks(t.K);
+    k_seg_scan<1><<<G, kSegThreads, 0, s>>>(t.K, 0, w.diff, nullptr, pressure, w.pressure_scan.ticket, w.pressure_scan.done,
+                                          (ull *)w.pressure_scan.agg, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
     return cudaGetLastError();
 }
 

@@ -120,6 +120,16 @@ cudaError_t launch_plan_small(const PlanArgs &A, const Workspace &w, int G, int 
 int plan_small_blocks();
 bool plan_small_fits(int64_t K, int64_t E, int G, int *cand_cap_out, size_t *smem_out);
 
+bool plan_keeps_state_on_chip(int64_t K, int64_t E, uint32_t flags)
+{
+    if ((flags & (G10_FLAG_RESCORE_ALL | G10_FLAG_GLOBAL_STATE)) || K > kSmallMaxSlots) return false;
+    int Gs = plan_small_blocks();
+    if (Gs > kSmallMaxBlocks) Gs = kSmallMaxBlocks;
+    int cand_cap = 0;
+    size_t smem = 0;
+    return Gs >= 1 && plan_small_fits(K, E, Gs, &cand_cap, &smem);
+}
+
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s)
 {
     PlanArgs A;
@@ -130,7 +140,7 @@ cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const Pla
         void *args[] = {&A};
         return cudaLaunchCooperativeKernel((const void *)k_plan_loop, dim3(G), dim3(kPlanThreads), args, 0, s);
     }
-    if (!(p.flags & G10_FLAG_GLOBAL_STATE) && t.K <= kSmallMaxSlots) {
+    if (plan_keeps_state_on_chip(t.K, t.E, p.flags)) {
         int Gs = plan_small_blocks();
         if (Gs > kSmallMaxBlocks) Gs = kSmallMaxBlocks;
         int cand_cap = 0;

@@ -106,7 +106,7 @@ extern "C" int32_t g10_pressure_timeline_static(const g10_trace *trace, g10_time
     DeviceTrace d{K, N, E, trace->kernel_ptr, trace->kernel_tensors, trace->tensor_bytes, trace->kernel_ns, trace->tensor_global};
     if (launch_slot_clock(d, w, out->kernel_start_ns, s) != cudaSuccess) return G10_ERR_CUDA;
     if (launch_first_last(d, w, w.first_use, w.last_use, s) != cudaSuccess) return G10_ERR_CUDA;
-    if (launch_pressure(d, w, w.first_use, w.last_use, out->pressure, out->peak_bytes, out->peak_slot, s) != cudaSuccess) return G10_ERR_CUDA;
+    if (launch_pressure(d, w, w.first_use, w.last_use, true, out->pressure, out->peak_bytes, out->peak_slot, s) != cudaSuccess) return G10_ERR_CUDA;
     if (launch_publish_status(w, out->status, s) != cudaSuccess) return G10_ERR_CUDA;
     return G10_OK;
 }
