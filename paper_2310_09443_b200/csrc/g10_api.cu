@@ -93,6 +93,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.c_ben_lo = c.take<ull>(E);
     w.c_ben_hi = c.take<ull>(E);
     w.c_cost = c.take<ull>(E);
+    w.c_key = c.take<double>(E);
     w.worklist = c.take<int>(2 * E);
     if (z.K <= kSmallMaxSlots) {
         w.busy_rep = c.take<int64_t>((size_t)kSmallMaxBlocks * 4 * K);

@@ -73,6 +73,7 @@ struct Workspace {
     Proposal *prop_stale;        // [max blocks]
     unsigned char *c_state;      // [E] per-period state of the lazy planner
     ull *c_ben_lo, *c_ben_hi, *c_cost;   // [E] cached benefit and cost
+    double *c_key;               // [E] rounded benefit / cost
     int *worklist;               // [2*E]
     int64_t *busy_rep, *hocc_rep; // per-block copies of the channel bookings / host occupancy (small-trace planner)
     int64_t *peak_part;          // [max blocks]

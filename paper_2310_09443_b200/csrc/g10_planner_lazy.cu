@@ -8,26 +8,27 @@
 //   STALE  a later commit lowered the pressure inside its absent range: the cached score is an upper bound;
 //   DIRTY  a later commit booked channel time (or host memory) inside one of its transfer windows: its
 //          destination has to be chosen again before anything can be said.
-// After a commit every block classifies its share of the periods against the winner's slot ranges (a few
-// integer comparisons each).  An iteration then alternates argmax rounds (best FRESH score; best STALE bound
-// per block) and evaluation rounds (all DIRTY periods, and the few best STALE periods whose bound still beats
-// the best FRESH score) until no DIRTY period is left and no STALE bound beats the best FRESH score: that
-// score is then the exact maximum over all live periods, ties included, and is committed.
+// After a commit every block classifies the periods it owns against the winner's slot ranges (a few integer
+// comparisons each).  DIRTY periods are rescored at once; a STALE period is rescored only while its bound may
+// still beat the best exact score known, so that when the iteration decides, the committed score is the exact
+// maximum over all live periods, ties included (see k_plan_lazy).
+#include <cstdio>
+
 #include "g10_planner.cuh"
 
 namespace g10 {
 
 constexpr int kLazyMaxBlocks = 256;
-constexpr int kStaleBatch = 8;           // STALE periods rescored per evaluation round, at most
 enum { kFresh = 1, kStale = 2, kDirty = 3 };
 
 struct LazyArgs {
     unsigned char *c_state;     // 0 = erased; else (dest + 1) | (state << 2)
     ull *c_ben_lo, *c_ben_hi;   // last computed benefit
     ull *c_cost;                // 2 t of the current destination
+    double *c_key;              // rounded benefit / cost of the cached score (steers the search; decisions are exact)
     int *worklist;              // [2][stride] DIRTY periods of the current round
     unsigned *wl_count;         // [2]
-    Proposal *prop_stale;       // [G] best STALE bound of each block
+    Proposal *prop_stale;       // [G] each block's exact best of step C (second proposal buffer)
     int64_t stride;
 };
 
@@ -49,6 +50,9 @@ __device__ __forceinline__ void store_score(const LazyArgs &L, int64_t p, int de
     L.c_ben_lo[p] = (ull)ben;
     L.c_ben_hi[p] = (ull)(ben >> 64);
     L.c_cost[p] = cost;
+    Cand cd;
+    cd.ben = ben; cd.cost = cost; cd.idx = 0; cd.dest = dest;
+    L.c_key[p] = ben == 0 ? 0.0 : cand_key(cd);
     L.c_state[p] = (unsigned char)((dest + 1) | (state << 2));
 }
 
@@ -137,12 +141,138 @@ __device__ __forceinline__ void store_proposal(Proposal *pr, const Cand &c)
     *pr = q;
 }
 
+// Best STALE bound of the block by rounded ratio (any of several equal ones): uniform result.
+__device__ __forceinline__ void block_max_key(double &k, int &idx, double *s_k /* [kPlanWarps] */, int *s_i /* [kPlanWarps] */)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double yk = __shfl_xor_sync(0xffffffffu, k, o);
+        const int yi = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (yk > k || (yk == k && yi > idx)) { k = yk; idx = yi; }
+    }
+    __syncthreads();
+    if (lane == 0) { s_k[warp] = k; s_i[warp] = idx; }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kPlanWarps; ++w) {
+        const double yk = s_k[w];
+        const int yi = s_i[w];
+        if (yk > k || (yk == k && yi > idx)) { k = yk; idx = yi; }
+    }
+}
+
+// One pass of a block over the periods it owns.  With `classify` the pending winner's slot ranges are applied
+// first (FRESH -> STALE where its absent range meets theirs, -> DIRTY where a booked window meets theirs) and
+// DIRTY periods are appended to the work list.  Returns the block's best FRESH candidate (exact) and its best
+// STALE bound (rounded ratio and period, approximate on purpose: it only says what to rescore next).
+struct ScanResult {
+    Cand bestF;
+    double keyS;
+    int idxS;
+};
+
+struct Winner {
+    int idx, dest, a, ap, bp, b;      // evict slots [a, ap-1], absent [ap, bp], prefetch [bp+1, b]
+};
+
+__device__ __forceinline__ ScanResult scan_owned(const PlanArgs &A, const LazyArgs &L, int64_t Pn, bool classify, const Winner &w,
+                                                 int par, BestScratch *sc, Cand *s_cand, double *s_k, int *s_i)
+{
+    const int G = gridDim.x, c = blockIdx.x, lane = threadIdx.x & 31;
+    double kf = -1.0, ks = -1.0;
+    int pf = -1, ps = -1;
+    for (int64_t p0 = (int64_t)c * kPlanThreads; p0 < Pn; p0 += (int64_t)G * kPlanThreads) {
+        const int64_t p = p0 + threadIdx.x;
+        bool dirty = false;
+        if (p < Pn) {
+            unsigned char st = L.c_state[p];
+            if (st != 0) {
+                int state = st >> 2;
+                const int d = (st & 3) - 1;
+                if (classify) {
+                    if (p == w.idx) { L.c_state[p] = 0; st = 0; }
+                    else if (state != kDirty) {
+                        const int u = A.per_u[p], v = A.per_v[p];
+                        if (u + 1 <= w.b && w.a <= v - 1) {          // the two periods share slots
+                            const int ap = A.geo_a[d * A.geo_stride + p], bp = A.geo_b[d * A.geo_stride + p];
+                            bool hit = false;
+                            if (d == w.dest) {
+                                hit = (u + 1 <= w.ap - 1 && w.a <= ap - 1) || (bp + 1 <= w.b && w.bp + 1 <= v - 1);
+                                if (!hit && d == G10_DEST_HOST && A.host_capacity != 0) hit = true;
+                            }
+                            if (hit) state = kDirty;
+                            else if (state == kFresh && ap <= w.bp && w.ap <= bp) state = kStale;
+                            if (state != (st >> 2)) { st = (unsigned char)((st & 3) | (state << 2)); L.c_state[p] = st; }
+                        }
+                    }
+                }
+                if (st != 0) {
+                    if (state == kDirty) dirty = true;
+                    else {
+                        const double key = L.c_key[p];
+                        if (key > 0.0) {
+                            if (state == kFresh) {
+                                bool take = key > kf;
+                                if (pf >= 0 && key >= kf * (1.0 - 1e-10) && kf >= key * (1.0 - 1e-10)) {
+                                    Cand x, y;                       // too close to call by rounding: exact
+                                    x.ben = ((u128)L.c_ben_hi[p] << 64) | L.c_ben_lo[p]; x.cost = L.c_cost[p]; x.idx = (int)p; x.dest = 0;
+                                    y.ben = ((u128)L.c_ben_hi[pf] << 64) | L.c_ben_lo[pf]; y.cost = L.c_cost[pf]; y.idx = pf; y.dest = 0;
+                                    take = cand_beats(x, y);
+                                }
+                                if (take) { kf = key; pf = (int)p; }
+                            } else if (key > ks) { ks = key; ps = (int)p; }
+                        }
+                    }
+                }
+            }
+        }
+        if (classify) {
+            // DIRTY periods go on the work list (one atomic per warp)
+            const unsigned md = __ballot_sync(0xffffffffu, dirty);
+            if (md) {
+                unsigned base = 0;
+                if (lane == 0) base = atomicAdd(&L.wl_count[par], (unsigned)__popc(md));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                if (dirty) L.worklist[(size_t)par * L.stride + base + __popc(md & ((1u << lane) - 1u))] = (int)p;
+            }
+        }
+    }
+    ScanResult r;
+    Cand x;
+    x.ben = 0; x.cost = 1; x.idx = -1; x.dest = -1;
+    if (pf >= 0) {
+        x.ben = ((u128)L.c_ben_hi[pf] << 64) | L.c_ben_lo[pf]; x.cost = L.c_cost[pf]; x.idx = pf;
+        x.dest = (L.c_state[pf] & 3) - 1;
+    }
+    r.bestF = block_best_fast(x, sc, s_cand);
+    block_max_key(ks, ps, s_k, s_i);
+    r.keyS = ks; r.idxS = ps;
+    return r;
+}
+
+// Could a STALE bound with rounded ratio `key` beat (or tie with) candidate t?  Conservative by 1e-10.
+__device__ __forceinline__ bool may_beat(double key, const Cand &t)
+{
+    if (!(key > 0.0)) return false;
+    if (t.idx < 0) return true;
+    return key >= cand_key(t) * (1.0 - 1e-10);
+}
+
+// Per iteration: (A) every block applies the previous commit to the slots it owns, classifies the periods it
+// owns and finds its best FRESH candidate and best STALE bound; (B) after the first grid barrier every block
+// knows the best FRESH score of the grid: DIRTY periods are rescored (shared out over the grid) and each block
+// rescores its own best STALE period if the bound may beat that score; (C) each block then makes its own best
+// exact -- it rescores its STALE periods, best bound first, while the bound may beat the better of the grid's
+// FRESH score and its own best; (D) after the last barrier the maximum of the blocks' exact bests is the exact
+// maximum over all live periods (every period left STALE has a bound below its block's best) and is committed.
 __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyArgs L)
 {
     __shared__ Cand s_cand[kPlanWarps + 1];
+    __shared__ BestScratch s_best;
     __shared__ long long s_max[kPlanWarps + 1];
-    __shared__ Cand s_stale[kLazyMaxBlocks];
-    __shared__ int s_sel[kStaleBatch];
+    __shared__ double s_k[kPlanWarps];
+    __shared__ int s_i[kPlanWarps];
     __shared__ int s_dest;
     __shared__ ull s_part[2 * kPlanWarps];
     const int G = gridDim.x, c = blockIdx.x;
@@ -153,11 +283,16 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     int64_t n_mig = 0, rounds = 0, bytes_ssd = 0, bytes_host = 0;
     int status = -1;
     long long peak = 0;
-    int par = 0;                               // which worklist buffer this round fills
+    int par = 0;                               // which worklist buffer this iteration fills
+#ifdef G10_PHASE_CLOCKS
+    long long dbg_dirty = 0, dbg_top = 0, dbg_local = 0;
+#endif
 
     // every period starts DIRTY: its first evaluation chooses the destination
-    for (int64_t p = (int64_t)c * kPlanThreads + threadIdx.x; p < Pn; p += (int64_t)G * kPlanThreads)
+    for (int64_t p = (int64_t)c * kPlanThreads + threadIdx.x; p < Pn; p += (int64_t)G * kPlanThreads) {
         L.c_state[p] = (unsigned char)(kDirty << 2);
+        L.c_key[p] = 0.0;
+    }
     {
         const long long m = own_slots_max(A, c, G, s_max);
         if (threadIdx.x == 0) A.peak_part[c] = m;
@@ -165,152 +300,109 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     if (!grid_barrier(A.bar, G, gen)) status = -2;
 
     bool pending = false;                      // a commit decided in the previous iteration, not yet applied
-    Cand win;
-    win.ben = 0; win.cost = 1; win.idx = -1; win.dest = -1;
-    int wa = 0, wap = 0, wbp = -1, wb = -1;    // winner's slot ranges: evict [wa, wap-1], absent [wap, wbp], prefetch [wbp+1, wb]
+    Winner win;
+    win.idx = -1; win.dest = -1; win.a = 0; win.ap = 0; win.bp = -1; win.b = -1;
 
     for (int64_t it = 0; status == -1; ++it) {
-        bool first_round = true;
-        bool decided = false;
-        while (!decided) {
-            // ---------------- apply the pending commit to what this block owns
-            if (pending) {
-                int64_t sz = 0;
-                const bool touched = commit_winner(A, win.idx, win.dest, it - 1, n_mig - 1, c, G, &sz);
-                if (touched) {
-                    const long long m = own_slots_max(A, c, G, s_max);
-                    if (threadIdx.x == 0) A.peak_part[c] = m;
-                }
+        // ---------------- apply the pending commit to what this block owns
+        if (pending) {
+            int64_t sz = 0;
+            const bool touched = commit_winner(A, win.idx, win.dest, it - 1, n_mig - 1, c, G, &sz);
+            if (touched) {
+                const long long m = own_slots_max(A, c, G, s_max);
+                if (threadIdx.x == 0) A.peak_part[c] = m;
             }
-            // ---------------- argmax round over this block's share of the periods
-            Cand bestF, bestS;
-            bestF.ben = 0; bestF.cost = 1; bestF.idx = -1; bestF.dest = -1;
-            bestS = bestF;
-            for (int64_t p0 = (int64_t)c * kPlanThreads; p0 < Pn; p0 += (int64_t)G * kPlanThreads) {
-                const int64_t p = p0 + threadIdx.x;
-                bool dirty = false;
-                if (p < Pn) {
-                    unsigned char st = L.c_state[p];
-                    if (st != 0) {
-                        int state = st >> 2;
-                        const int d = (st & 3) - 1;
-                        if (pending) {
-                            if (p == win.idx) { L.c_state[p] = 0; st = 0; }
-                            else if (state != kDirty) {
-                                const int u = A.per_u[p], v = A.per_v[p];
-                                if (u + 1 <= wb && wa <= v - 1) {          // the two periods share slots
-                                    const int ap = A.geo_a[d * A.geo_stride + p], bp = A.geo_b[d * A.geo_stride + p];
-                                    bool hit = false;
-                                    if (d == win.dest) {
-                                        hit = (u + 1 <= wap - 1 && wa <= ap - 1) || (bp + 1 <= wb && wbp + 1 <= v - 1);
-                                        if (!hit && d == G10_DEST_HOST && A.host_capacity != 0) hit = true;
-                                    }
-                                    if (hit) state = kDirty;
-                                    else if (state == kFresh && ap <= wbp && wap <= bp) state = kStale;
-                                    if (state != (st >> 2)) { st = (unsigned char)((st & 3) | (state << 2)); L.c_state[p] = st; }
-                                }
-                            }
-                        }
-                        if (st != 0) {
-                            if (state == kDirty) dirty = true;
-                            else {
-                                Cand x;
-                                x.ben = ((u128)L.c_ben_hi[p] << 64) | L.c_ben_lo[p];
-                                if (x.ben > 0) {
-                                    x.cost = L.c_cost[p]; x.idx = (int)p; x.dest = d;
-                                    if (state == kFresh) { if (cand_beats(x, bestF)) bestF = x; }
-                                    else if (cand_beats(x, bestS)) bestS = x;
-                                }
-                            }
-                        }
-                    }
-                }
-                // DIRTY periods go on the work list (one atomic per warp)
-                const unsigned md = __ballot_sync(0xffffffffu, dirty);
-                if (md) {
-                    unsigned base = 0;
-                    if (lane == 0) base = atomicAdd(&L.wl_count[par], (unsigned)__popc(md));
-                    base = __shfl_sync(0xffffffffu, base, 0);
-                    if (dirty) L.worklist[(size_t)par * L.stride + base + __popc(md & ((1u << lane) - 1u))] = (int)p;
-                }
-            }
-            bestF = block_best(bestF, s_cand);
-            bestS = block_best(bestS, s_cand);
-            if (threadIdx.x == 0) { store_proposal(&A.proposals[c], bestF); store_proposal(&L.prop_stale[c], bestS); }
-            pending = false;
-            if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
-
-            // ---------------- every block: best FRESH score, peak, work list length, STALE bounds that still compete
-            Cand gF;
-            gF.ben = 0; gF.cost = 1; gF.idx = -1; gF.dest = -1;
-            long long m = 0;
-            for (int j = threadIdx.x; j < G; j += kPlanThreads) {
-                const long long pm = __ldcg(&A.peak_part[j]);
-                if (pm > m) m = pm;
-                const Cand x = load_proposal(&A.proposals[j]);
-                if (cand_beats(x, gF)) gF = x;
-                s_stale[j] = load_proposal(&L.prop_stale[j]);
-            }
-            peak = block_max_i64(m, s_max);
-            gF = block_best(gF, s_cand);
-            const unsigned W = __ldcg(&L.wl_count[par]);
-            if (first_round) {
-                if (A.fits_always || peak <= A.cap) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
-                if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
-                rounds += 1;
-                first_round = false;
-            }
-            // rank the STALE proposals that beat the best FRESH score; the kStaleBatch best are rescored
-            bool qual = false;
-            int rank = 0;
-            if (threadIdx.x < G) {
-                const Cand me = s_stale[threadIdx.x];
-                qual = me.idx >= 0 && cand_beats(me, gF);
-                if (qual)
-                    for (int j = 0; j < G; ++j)
-                        if (j != (int)threadIdx.x && cand_beats(s_stale[j], me)) ++rank;
-                if (qual && rank < kStaleBatch) s_sel[rank] = me.idx;
-            }
-            int nS = __syncthreads_count(qual);
-            if (nS > kStaleBatch) nS = kStaleBatch;
-            if (W == 0 && nS == 0) {
-                // nothing can beat the best FRESH score: decide
-                if (gF.idx < 0) { status = G10_EXHAUSTED; break; }
-                win = gF;
-                {
-                    const int64_t p = win.idx;
-                    const int X = win.dest;
-                    wa = A.per_u[p] + 1; wb = A.per_v[p] - 1;
-                    wap = A.geo_a[X * A.geo_stride + p]; wbp = A.geo_b[X * A.geo_stride + p];
-                    const int64_t sz = A.bytes[A.per_t[p]];
-                    if (X == G10_DEST_SSD) bytes_ssd += sz; else bytes_host += sz;
-                }
-                n_mig += 1;
-                pending = true;
-                decided = true;
-                break;
-            }
-            // ---------------- evaluation round
-            const unsigned T = W + (unsigned)nS;
-            const int *wl = L.worklist + (size_t)par * L.stride;
-            if (T <= 2u * (unsigned)G) {
-                for (unsigned e = c; e < T; e += G) {
-                    const int64_t p = e < W ? wl[e] : s_sel[e - W];
-                    eval_block(A, L, p, &s_dest, s_part);
-                }
-            } else {
-                for (unsigned e = (unsigned)c * kPlanWarps + warp; e < T; e += (unsigned)G * kPlanWarps) {
-                    const int64_t p = e < W ? wl[e] : s_sel[e - W];
-                    eval_warp(A, L, p, lane);
-                }
-            }
-            if (c == 0 && threadIdx.x == 0) L.wl_count[par ^ 1] = 0;
-            par ^= 1;
-            if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
         }
+        // ---------------- A: classify the owned periods against the commit, collect DIRTY ones, local bests
+        // (on the first iteration `win` matches nothing and every period is DIRTY)
+        ScanResult sr = scan_owned(A, L, Pn, true, win, par, &s_best, s_cand, s_k, s_i);
+        if (threadIdx.x == 0) store_proposal(&A.proposals[c], sr.bestF);
+        pending = false;
+        if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+
+        // ---------------- B: global best FRESH score so far, peak, stop tests; rescore DIRTY periods (shared
+        // out over the grid) and this block's best STALE period if its bound may beat that score
+        Cand gF;
+        gF.ben = 0; gF.cost = 1; gF.idx = -1; gF.dest = -1;
+        long long m = 0;
+        for (int j = threadIdx.x; j < G; j += kPlanThreads) {
+            const long long pm = __ldcg(&A.peak_part[j]);
+            if (pm > m) m = pm;
+            const Cand x = load_proposal(&A.proposals[j]);
+            if (cand_beats(x, gF)) gF = x;
+        }
+        peak = block_max_i64(m, s_max);
+        gF = block_best_fast(gF, &s_best, s_cand);
+        const unsigned W = __ldcg(&L.wl_count[par]);
+        if (A.fits_always || peak <= A.cap) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
+        if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
+        rounds += 1;
+        const int *wl = L.worklist + (size_t)par * L.stride;
+        if (W <= 2u * (unsigned)G) {
+            for (unsigned e = c; e < W; e += G) eval_block(A, L, wl[e], &s_dest, s_part);
+        } else {
+            for (unsigned e = (unsigned)c * kPlanWarps + warp; e < W; e += (unsigned)G * kPlanWarps) eval_warp(A, L, wl[e], lane);
+        }
+        if (sr.idxS >= 0 && may_beat(sr.keyS, gF)) {
+            eval_block(A, L, sr.idxS, &s_dest, s_part);
+#ifdef G10_PHASE_CLOCKS
+            dbg_top += 1;
+#endif
+        }
+#ifdef G10_PHASE_CLOCKS
+        dbg_dirty += W;
+#endif
+        if (c == 0 && threadIdx.x == 0) L.wl_count[par ^ 1] = 0;
+        par ^= 1;
+        if (W > 0) {                               // DIRTY periods were rescored by other blocks than their owners
+            if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+        } else __syncthreads();
+
+        // ---------------- C: make this block's best exact
+        Cand localF;
+        for (;;) {
+            sr = scan_owned(A, L, Pn, false, win, par, &s_best, s_cand, s_k, s_i);
+            localF = sr.bestF;
+            const Cand &thr = cand_beats(localF, gF) ? localF : gF;
+            if (sr.idxS >= 0 && may_beat(sr.keyS, thr)) {
+                eval_block(A, L, sr.idxS, &s_dest, s_part);
+                __syncthreads();
+#ifdef G10_PHASE_CLOCKS
+                dbg_local += 1;
+#endif
+                continue;
+            }
+            break;
+        }
+        if (threadIdx.x == 0) store_proposal(&L.prop_stale[c], localF);      // second buffer: step A reuses the first
+        if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+
+        // ---------------- D: the exact global argmax; decide
+        Cand best;
+        best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
+        for (int j = threadIdx.x; j < G; j += kPlanThreads) {
+            const Cand x = load_proposal(&L.prop_stale[j]);
+            if (cand_beats(x, best)) best = x;
+        }
+        best = block_best_fast(best, &s_best, s_cand);
+        if (best.idx < 0) { status = G10_EXHAUSTED; break; }
+        {
+            const int64_t p = best.idx;
+            const int X = best.dest;
+            win.idx = best.idx; win.dest = X;
+            win.a = A.per_u[p] + 1; win.b = A.per_v[p] - 1;
+            win.ap = A.geo_a[X * A.geo_stride + p]; win.bp = A.geo_b[X * A.geo_stride + p];
+            const int64_t sz = A.bytes[A.per_t[p]];
+            if (X == G10_DEST_SSD) bytes_ssd += sz; else bytes_host += sz;
+        }
+        n_mig += 1;
+        pending = true;
     }
-    // a commit decided in the very last iteration is always applied above before the loop can end:
-    // the loop only ends at a first-round test or at an empty argmax, both of which follow the apply step.
+#ifdef G10_PHASE_CLOCKS
+    if (threadIdx.x == 0 && (c == 0 || c == 77))
+        printf("k_plan_lazy block %d: iterations %lld, DIRTY rescored (grid) %lld, own top STALE rescored %lld, further STALE rescored %lld\n",
+               c, (long long)rounds, dbg_dirty, dbg_top, dbg_local);
+#endif
     plan_epilogue(A, c, G, gen, status, peak, n_mig, rounds, bytes_ssd, bytes_host);
 }
 
@@ -328,7 +420,7 @@ cudaError_t launch_plan_lazy(const PlanArgs &A_in, const Workspace &w, int G, cu
 {
     PlanArgs A = A_in;
     LazyArgs L;
-    L.c_state = w.c_state; L.c_ben_lo = w.c_ben_lo; L.c_ben_hi = w.c_ben_hi; L.c_cost = w.c_cost;
+    L.c_state = w.c_state; L.c_ben_lo = w.c_ben_lo; L.c_ben_hi = w.c_ben_hi; L.c_cost = w.c_cost; L.c_key = w.c_key;
     L.worklist = w.worklist; L.wl_count = w.wl_count; L.prop_stale = w.prop_stale; L.stride = A.geo_stride;
     void *args[] = {&A, &L};
     return cudaLaunchCooperativeKernel((const void *)k_plan_lazy, dim3(G), dim3(kPlanThreads), args, 0, s);

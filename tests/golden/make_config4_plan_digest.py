@@ -1,0 +1,44 @@
+"""Writes tests/golden/config4_plan_digest.json: a digest of the CPU oracle's complete plan for the
+full-size stress trace (config 4: 1e6 kernels, 4e6 tensors).  The oracle's lazy tier needs about ten
+minutes for it, too long for a test, so the GPU parity test compares its own plan with this digest.
+Calls only the trace generator and the oracle.  Usage: python tests/golden/make_config4_plan_digest.py"""
+import hashlib
+import json
+import os
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, ROOT)
+
+from oracle import g10_oracle as O  # noqa: E402
+from paper_2310_09443_b200 import traces  # noqa: E402
+
+
+def digest(migrations, final_pressure, summary):
+    h = hashlib.sha256()
+    h.update(migrations.tobytes())
+    h.update(final_pressure.tobytes())
+    h.update(summary[:7].tobytes())
+    return h.hexdigest()
+
+
+def main():
+    tr = traces.config4_stress_dag()
+    start, P0, peak, slot = O.timeline(tr)
+    cap = tr.capacity_from_peak(peak)
+    r = O.plan(tr, cap, lazy=True)
+    out = {
+        "_source": "oracle/g10_oracle.c, lazy tier, on paper_2310_09443_b200.traces.config4_stress_dag() (seed 4)",
+        "trace_sha256": tr.sha256(), "peak_bytes": int(peak), "peak_slot": int(slot), "capacity_bytes": int(cap),
+        "summary": [int(x) for x in r.summary[:7]], "status": r.status,
+        "first_migrations": [[int(m[k]) for k in m.dtype.names] for m in r.migrations[:5]],
+        "plan_sha256": digest(r.migrations, r.final_pressure, r.summary),
+    }
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "config4_plan_digest.json")
+    with open(path, "w") as f:
+        json.dump(out, f, indent=1)
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()
