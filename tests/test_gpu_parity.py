@@ -244,3 +244,29 @@ def test_full_size_stress_dag_passes(gpu, oracle):
     plan = check_plan(gpu, tr, tb, cap, ref, max_iterations=1000)
     helpers.check_plan_invariants(tr, cap, start, P0, ov, gpu.migrations_numpy(plan), _np(plan.final_pressure),
                                   gpu.STATUS[int(plan.summary[2].item())], tr.host_bw, tr.ssd_bw, check_area=False)
+
+
+def test_full_size_stress_plan_digest(gpu):
+    """The complete plan of config 4 (13 505 migrations) against the digest of the CPU oracle's plan stored by
+    tests/golden/make_config4_plan_digest.py (the oracle needs about ten minutes for it)."""
+    import hashlib, json, os
+    import torch
+    path = os.path.join(os.path.dirname(__file__), "golden", "config4_plan_digest.json")
+    gold = json.load(open(path))
+    tr = traces.config4_stress_dag()
+    assert tr.sha256() == gold["trace_sha256"]
+    tb = gpu.upload(tr)
+    tl = gpu.g10_pressure_timeline(tb)
+    torch.cuda.synchronize()
+    assert int(tl.peak_bytes.item()) == gold["peak_bytes"] and int(tl.peak_slot.item()) == gold["peak_slot"]
+    cap = tr.capacity_from_peak(int(tl.peak_bytes.item()))
+    assert cap == gold["capacity_bytes"]
+    plan = gpu.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    summary = _np(plan.summary)
+    assert summary[7] == 0 and summary[:7].tolist() == gold["summary"]
+    mig = gpu.migrations_numpy(plan)
+    assert [[int(m[k]) for k in m.dtype.names] for m in mig[:5]] == gold["first_migrations"]
+    h = hashlib.sha256()
+    h.update(mig.tobytes()); h.update(_np(plan.final_pressure)[:tr.K].tobytes()); h.update(summary[:7].tobytes())
+    assert h.hexdigest() == gold["plan_sha256"]
