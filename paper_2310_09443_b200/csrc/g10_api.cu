@@ -53,6 +53,9 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     carve_scan(c, w.emit_scan, etiles, 2);
     carve_scan(c, w.pressure_scan, ktiles, 1);
     w.wl_count = c.take<unsigned>(2);
+    w.bk_count = c.take<unsigned>(4096);
+    w.bk_cursor = c.take<unsigned>(4096);
+    w.bk_words = c.take<ull>(2 * 4096);
     w.xwords = c.take<ull>((2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16);
     w.zero_bytes = align_up(c.off);
     // arrays that must start at zero, cleared only by the calls that use them
@@ -95,6 +98,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.c_cost = c.take<ull>(E);
     w.c_key = c.take<double>(E);
     w.worklist = c.take<int>(2 * E);
+    w.bk_pairs = c.take<ull>(E);
     if (z.K <= kSmallMaxSlots) {
         w.busy_rep = c.take<int64_t>((size_t)kSmallMaxBlocks * 4 * K);
         w.hocc_rep = c.take<int64_t>((size_t)kSmallMaxBlocks * K);
@@ -227,7 +231,8 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(trace, ws, w, d, s, kZeroCounts);
+    const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
+    rc = begin_call(trace, ws, w, d, s, buckets ? 0 : kZeroCounts);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     VitalityBuffers vb;
@@ -239,7 +244,7 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
         vb = VitalityBuffers{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, ucap, w.period_ptr,
                              w.period_tensor, w.period_prev_use, w.period_next_use, pcap, w.counts};
     }
-    CU(launch_vitality(d, w, vb, s));
+    CU(buckets ? launch_vitality_buckets(d, w, vb, s) : launch_vitality(d, w, vb, s));
     CU(launch_publish_status(w, vb.counts + 2, s));
     if (host) {
         int64_t counts[3];
@@ -325,7 +330,8 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
     Workspace w;
     DeviceTrace d;
     const uint32_t flags = options ? options->flags : 0;
-    rc = begin_call(trace, ws, w, d, s, kZeroCounts | kZeroDiff | (plan_keeps_state_on_chip(trace->num_kernels, trace->num_events, flags) ? 0 : kZeroState));
+    const bool buckets = !(flags & G10_FLAG_RESCORE_ALL) && vitality_buckets_supported(trace->num_tensors, trace->num_events);
+    rc = begin_call(trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff | (plan_keeps_state_on_chip(trace->num_kernels, trace->num_events, flags) ? 0 : kZeroState));
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
@@ -347,7 +353,7 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
     };
     CU(mark(0));
     CU(launch_slot_clock(d, w, w.start, s));
-    CU(launch_vitality(d, w, vb, s));
+    CU(buckets ? launch_vitality_buckets(d, w, vb, s) : launch_vitality(d, w, vb, s));
     CU(mark(1));
     CU(launch_pressure(d, w, w.first_use, w.last_use, false, pp.final_pressure, w.peak_bytes, w.peak_slot, s));
     CU(mark(2));

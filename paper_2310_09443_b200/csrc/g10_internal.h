@@ -50,6 +50,8 @@ struct Workspace {
     int64_t *hocc;               // [K] host-memory occupancy per slot
     unsigned char *dead;         // [E] period erased
     unsigned *wl_count;          // [2] lengths of the two DIRTY work lists
+    unsigned *bk_count, *bk_cursor;   // [4096] events per tensor bucket, scatter cursors
+    ull *bk_words;               // [2 * 4096] tagged per-bucket totals
     ull *xwords;                 // [2][kSmallMaxBlocks][16] tagged words of the proposal exchange
     // --- uninitialised region ---
     int32_t *raw_ptr;            // [N+1]
@@ -75,6 +77,7 @@ struct Workspace {
     ull *c_ben_lo, *c_ben_hi, *c_cost;   // [E] cached benefit and cost
     double *c_key;               // [E] rounded benefit / cost
     int *worklist;               // [2*E]
+    ull *bk_pairs;               // [E] events as (tensor in bucket, kernel) keys, bucket after bucket
     int64_t *busy_rep, *hocc_rep; // per-block copies of the channel bookings / host occupancy (small-trace planner)
     int64_t *peak_part;          // [max blocks]
     g10_migration *migrations;   // host mode only
@@ -122,6 +125,9 @@ constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock f
 // passes (g10_passes.cu)
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
+// bucketed formulation (g10_vitality_buckets.cu); supported for up to 4096 buckets of 4096 tensors
+bool vitality_buckets_supported(int64_t N, int64_t E);
+cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s);
 cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);
