@@ -4,15 +4,16 @@
 //   1. k_bk_hist     counts the events of every bucket (shared-memory histogram per block);
 //   2. k_bk_scatter  partitions the events by bucket: each event becomes one 64-bit key
 //                    (tensor id inside the bucket << 32 | kernel) written into its bucket's slice;
-//   3. k_bk_emit     takes one bucket at a time: sorts its keys in shared memory (bitonic network), after which
-//                    the sorted distinct kernels of every tensor are adjacent -- first / last use, the use lists
-//                    (repeats of a tensor inside one kernel collapse) and the inactive periods (consecutive
-//                    distinct uses at least two kernels apart) all follow from comparing neighbours and from
-//                    prefix counts; the offsets of a bucket in `uses` and in the period arrays are the sums of
-//                    the totals of all earlier buckets, exchanged through tagged 64-bit words.
+//   3. k_bk_emit     takes one bucket at a time, entirely in shared memory: counts the events of each tensor,
+//                    scans the counts, scatters the kernels into per-tensor segments, lets one thread sort and
+//                    de-duplicate each (short) segment -- a tensor listed by more than 32 kernels is sorted by the
+//                    whole block -- and counts the inactive periods (consecutive distinct uses at least two kernels
+//                    apart); the offsets of a bucket in `uses` and in the period arrays are the sums of the totals
+//                    of all earlier buckets, exchanged through tagged 64-bit words; then everything is written out
+//                    in coalesced runs.
 // Everything random happens in shared memory (atomics included); HBM sees the events twice, the keys once each
-// way and the outputs once, all in coalesced runs.  A bucket whose keys do not fit in shared memory (a tensor
-// listed by a great many kernels) is sorted in place in global memory by the same block: slower, same result.
+// way and the outputs once.  A bucket with more events than fit in shared memory (a tensor listed by a great many
+// kernels) keeps its segments in global memory instead: slower, same result.
 #include "g10_device.cuh"
 #include "g10_internal.h"
 
@@ -20,9 +21,10 @@ namespace g10 {
 
 constexpr int kBkThreads = 512;
 constexpr int kBkItems = 8;
-constexpr int kBkTile = kBkThreads * kBkItems;     // events per partition tile
-constexpr int kBkCap = 4096;                       // keys sorted in shared memory
-constexpr int kBkPtrStage = 2048;                  // kernel_ptr entries staged per tile
+constexpr int kBkTile = kBkThreads * kBkItems;     // events per partition tile (4096)
+constexpr int kBkCap = 12288;                      // events of a bucket kept in shared memory
+constexpr int kBkPtrStage = 3072;                  // kernel_ptr entries staged per tile
+constexpr int kBkHeavy = 32;                       // longer segments are sorted by the whole block
 
 struct BucketArgs {
     int64_t N, E, K;
@@ -33,6 +35,7 @@ struct BucketArgs {
     unsigned *bucket_cursor;   // [nb] scatter cursors (start at zero)
     ull *pairs;                // [E] keys, bucket after bucket
     ull *words;                // [2 * nb] tagged totals of each bucket: distinct uses, periods
+    int32_t *spill;            // [E] per-tensor segments of buckets too large for shared memory
     unsigned *ticket;
     ull *status;
 };
@@ -69,6 +72,27 @@ __device__ __forceinline__ int bk_kernel_of_event(const int64_t *kptr, int lo, i
         if (kptr[mid] <= e) lo = mid; else hi = mid - 1;
     }
     return lo;
+}
+
+// Same, by a whole warp: every round probes 32 evenly spaced kernels at once, so that a cold search over a
+// million kernels costs four dependent round trips instead of twenty.  Result in every lane.
+__device__ __forceinline__ int bk_kernel_of_event_warp(const int64_t *__restrict__ kptr, int lo, int hi, int64_t e, int lane)
+{
+    while (hi - lo > 31) {
+        const int step = (hi - lo) / 32 + 1;
+        const int probe = lo + lane * step;                   // lane 0 probes lo, which is known to qualify
+        const bool ok = probe <= hi && kptr[probe] <= e;
+        const unsigned m = __ballot_sync(0xffffffffu, ok);     // qualifying probes form a prefix of the lanes
+        const int last = 31 - __clz(m);
+        const int nlo = lo + last * step;
+        int nhi = nlo + step - 1;
+        if (nhi > hi) nhi = hi;
+        lo = nlo; hi = nhi;
+    }
+    const int probe = lo + lane;
+    const bool ok = probe <= hi && kptr[probe] <= e;
+    const unsigned m = __ballot_sync(0xffffffffu, ok);
+    return lo + (31 - __clz(m));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -108,9 +132,11 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int3
 __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
 {
     extern __shared__ int s_mem[];
-    int *s_base = s_mem;                          // [nb + 1] first key of each bucket
-    unsigned *s_cnt = (unsigned *)(s_base + B.nb + 1);   // [nb] events of this tile per bucket
-    unsigned *s_off = s_cnt + B.nb;               // [nb] where this tile's events start inside the bucket
+    int *s_base = s_mem;                                   // [nb + 1] first key of each bucket
+    int *s_cnt = s_base + B.nb + 1;                        // [nb + 1] events of this tile per bucket, then their scan
+    unsigned *s_off = (unsigned *)(s_cnt + B.nb + 1);      // [nb] where this tile's events start inside the bucket
+    ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkTile] keys of the tile in bucket order
+    unsigned short *s_bkt = (unsigned short *)(s_key + kBkTile);              // [kBkTile] their buckets
     __shared__ int s_warp[32];
     __shared__ int64_t s_ptr[kBkPtrStage];
     __shared__ int s_lohi[2];
@@ -118,11 +144,12 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
     const int64_t tiles = (B.E + kBkTile - 1) / kBkTile;
     for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         const int64_t base = tile * kBkTile;
-        for (int b = threadIdx.x; b < B.nb; b += kBkThreads) s_cnt[b] = 0;
-        if (threadIdx.x == 0) {
-            const int64_t last = (base + kBkTile <= B.E ? base + kBkTile : B.E) - 1;
-            s_lohi[0] = bk_kernel_of_event(kptr, 0, (int)B.K - 1, base);
-            s_lohi[1] = bk_kernel_of_event(kptr, s_lohi[0], (int)B.K - 1, last);
+        const int n_tile = (int)((B.E - base) < kBkTile ? (B.E - base) : kBkTile);
+        for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_cnt[b] = 0;
+        if (threadIdx.x < 32) {
+            const int klo = bk_kernel_of_event_warp(kptr, 0, (int)B.K - 1, base, (int)threadIdx.x);
+            const int khi = bk_kernel_of_event_warp(kptr, klo, (int)B.K - 1, base + n_tile - 1, (int)threadIdx.x);
+            if (threadIdx.x == 0) { s_lohi[0] = klo; s_lohi[1] = khi; }
         }
         __syncthreads();
         int lo = s_lohi[0], hi = s_lohi[1], shift_k = 0;
@@ -133,7 +160,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
         }
         __syncthreads();
         int bucket[kBkItems];
-        unsigned rank[kBkItems];
+        int rank[kBkItems];
         ull key[kBkItems];
 #pragma unroll
         for (int j = 0; j < kBkItems; ++j) {
@@ -145,40 +172,50 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
                     const int k = bk_kernel_of_event(sp, lo, hi, e) + shift_k;
                     bucket[j] = i >> B.shift;
                     key[j] = ((ull)(unsigned)(i & (B.bt - 1)) << 32) | (unsigned)k;
-                    rank[j] = atomicAdd(&s_cnt[bucket[j]], 1u);
+                    rank[j] = atomicAdd(&s_cnt[bucket[j]], 1);
                 }
             }
         }
         __syncthreads();
+        // reserve this tile's room in every bucket it touches, then turn the tile counts into tile offsets
         for (int b = threadIdx.x; b < B.nb; b += kBkThreads)
-            if (s_cnt[b]) s_off[b] = atomicAdd(&B.bucket_cursor[b], s_cnt[b]);
+            if (s_cnt[b]) s_off[b] = atomicAdd(&B.bucket_cursor[b], (unsigned)s_cnt[b]);
         __syncthreads();
+        block_scan_counts((const unsigned *)s_cnt, B.nb, s_cnt, s_warp);      // in place: s_cnt[b] = first slot of bucket b in the tile
 #pragma unroll
         for (int j = 0; j < kBkItems; ++j)
             if (bucket[j] >= 0) {
-                const int64_t pos = (int64_t)s_base[bucket[j]] + s_off[bucket[j]] + rank[j];
-                if (pos < B.E) B.pairs[pos] = key[j];
+                const int slot = s_cnt[bucket[j]] + rank[j];
+                s_key[slot] = key[j];
+                s_bkt[slot] = (unsigned short)bucket[j];
             }
+        __syncthreads();
+        const int n_valid = s_cnt[B.nb];
+        for (int slot = threadIdx.x; slot < n_valid; slot += kBkThreads) {
+            const int b = s_bkt[slot];
+            const int64_t pos = (int64_t)s_base[b] + s_off[b] + (slot - s_cnt[b]);
+            if (pos < B.E) B.pairs[pos] = s_key[slot];
+        }
         __syncthreads();
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// 3. one bucket at a time: sort, compare neighbours, count, emit
+// 3. one bucket at a time: count, scan, scatter, sort the short segments, count, emit
 // ---------------------------------------------------------------------------------------------
-__device__ void bk_bitonic_sort(ull *a, int n)          // arbitrary n: the network only ever moves values up
+__device__ void bk_bitonic_sort_i32(int32_t *a, int n)    // arbitrary n: the network only ever moves values up
 {
     int n2 = 1;
     while (n2 < n) n2 <<= 1;
     for (int k = 2; k <= n2; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int j = k >> 1, lj = 31 - __clz(k >> 1); j > 0; j >>= 1, --lj) {
             const bool mirror = (j == (k >> 1));
             for (int t = threadIdx.x; t < n2 / 2; t += blockDim.x) {
-                const int blk = t / j, off = t % j;
+                const int blk = t >> lj, off = t & (j - 1);
                 const int i = blk * 2 * j + off;
                 const int p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
                 if (p < n) {
-                    const ull x = a[i], y = a[p];
+                    const int32_t x = a[i], y = a[p];
                     if (x > y) { a[i] = y; a[p] = x; }
                 }
             }
@@ -187,131 +224,188 @@ __device__ void bk_bitonic_sort(ull *a, int n)          // arbitrary n: the netw
     }
 }
 
-struct BkFlags {
-    bool head, tail, dist, per;
-    int tl, k, kprev;
-};
-
-__device__ __forceinline__ BkFlags bk_flags(const ull *kp, int j, int n)
-{
-    BkFlags f;
-    const ull cur = kp[j];
-    f.tl = (int)(cur >> 32); f.k = (int)(unsigned)cur;
-    f.head = true; f.kprev = 0;
-    if (j > 0) {
-        const ull prev = kp[j - 1];
-        f.head = (int)(prev >> 32) != f.tl;
-        f.kprev = (int)(unsigned)prev;
-    }
-    f.dist = f.head || f.kprev != f.k;
-    f.per = f.dist && !f.head && (f.k - f.kprev >= 2);
-    f.tail = (j == n - 1) || ((int)(kp[j + 1] >> 32) != f.tl);
-    return f;
-}
-
 __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
+
+// in-place exclusive scan of two int arrays a[0..n), b[0..n); a[n], b[n] receive the totals; whole block
+__device__ __forceinline__ void bk_scan2(int *a, int *b, int n, int *s_wa, int *s_wb)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int ca = 0, cb = 0;
+    for (int base = 0; base < n; base += kBkThreads) {
+        const int t = base + threadIdx.x;
+        const int va = t < n ? a[t] : 0, vb = t < n ? b[t] : 0;
+        int ia = va, ib = vb;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int ya = __shfl_up_sync(0xffffffffu, ia, o), yb = __shfl_up_sync(0xffffffffu, ib, o);
+            if (lane >= o) { ia += ya; ib += yb; }
+        }
+        __syncthreads();
+        if (lane == 31) { s_wa[warp] = ia; s_wb[warp] = ib; }
+        __syncthreads();
+        int pa = 0, pb = 0, ta = 0, tb = 0;
+        for (int w = 0; w < kBkThreads / 32; ++w) {
+            if (w < warp) { pa += s_wa[w]; pb += s_wb[w]; }
+            ta += s_wa[w]; tb += s_wb[w];
+        }
+        if (t < n) { a[t] = ca + pa + ia - va; b[t] = cb + pb + ib - vb; }
+        ca += ta; cb += tb;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) { a[n] = ca; b[n] = cb; }
+    __syncthreads();
+}
 
 __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBuffers out)
 {
     extern __shared__ int s_mem[];
-    int *s_base = s_mem;                                   // [nb + 1]
-    int *t_first = s_base + B.nb + 1;                      // [bt] per-tensor results of the current bucket
-    int *t_last = t_first + B.bt;
-    int *t_nuse = t_last + B.bt;                           // counts, then exclusive offsets (bt + 1 entries)
-    int *t_nper = t_nuse + B.bt + 1;                       // counts, then exclusive offsets (bt + 1 entries)
-    ull *s_keys = (ull *)(((uintptr_t)(t_nper + B.bt + 1) + 7) & ~(uintptr_t)7);   // [kBkCap]
+    int *s_base = s_mem;                       // [nb + 1] first key of each bucket
+    int *t_off = s_base + B.nb + 1;            // [bt + 1] raw events per tensor, then segment offsets
+    int *t_d = t_off + B.bt + 1;               // [bt + 1] scatter cursor, then distinct uses, then their offsets
+    int *t_np = t_d + B.bt + 1;                // [bt + 1] periods per tensor, then their offsets
+    int32_t *s_ks = t_np + B.bt + 1;           // [kBkCap] kernels, tensor segment after tensor segment
     __shared__ int s_warp[32];
     __shared__ int s_wa[kBkThreads / 32], s_wb[kBkThreads / 32];
-    __shared__ int s_bucket;
+    __shared__ long long s_pu[kBkThreads / 32], s_pp[kBkThreads / 32];
+    __shared__ int s_bucket, s_nheavy, s_total, s_periods;
+    __shared__ int s_heavy[64];
     __shared__ long long s_pre[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     block_scan_counts(B.bucket_count, B.nb, s_base, s_warp);
     for (;;) {
         __syncthreads();
-        if (threadIdx.x == 0) s_bucket = (int)atomicAdd(B.ticket, 1u);
+        if (threadIdx.x == 0) { s_bucket = (int)atomicAdd(B.ticket, 1u); s_nheavy = 0; }
         __syncthreads();
         const int b = s_bucket;
         if (b >= B.nb) break;
         const int n = s_base[b + 1] - s_base[b];
         const int64_t t0 = (int64_t)b * B.bt;
         const int bt_eff = (int)((B.N - t0) < B.bt ? (B.N - t0) : B.bt);
-        ull *gk = B.pairs + s_base[b];
-        const ull *kp;
-        // ---- sort the bucket's keys
-        if (n <= kBkCap) {
-            for (int j = threadIdx.x; j < n; j += kBkThreads) s_keys[j] = gk[j];
-            __syncthreads();
-            bk_bitonic_sort(s_keys, n);
-            kp = s_keys;
-        } else {
-            __syncthreads();
-            bk_bitonic_sort(gk, n);
-            __threadfence_block();
-            kp = gk;
-        }
-        for (int tl = threadIdx.x; tl <= bt_eff; tl += kBkThreads) {
-            if (tl < bt_eff) { t_first[tl] = -1; t_last[tl] = -1; }
-            t_nuse[tl] = 0; t_nper[tl] = 0;
-        }
+        const ull *gk = B.pairs + s_base[b];
+        int32_t *ks = n <= kBkCap ? s_ks : B.spill + s_base[b];
+        for (int tl = threadIdx.x; tl <= bt_eff; tl += kBkThreads) { t_off[tl] = 0; t_d[tl] = 0; t_np[tl] = 0; }
         __syncthreads();
-        // ---- pass A: per-tensor first / last / counts
-        for (int j = threadIdx.x; j < n; j += kBkThreads) {
-            const BkFlags f = bk_flags(kp, j, n);
-            if (f.head) t_first[f.tl] = f.k;
-            if (f.tail) t_last[f.tl] = f.k;
-            if (f.dist) atomicAdd(&t_nuse[f.tl], 1);
-            if (f.per) atomicAdd(&t_nper[f.tl], 1);
-        }
-        __syncthreads();
-        // in-place exclusive scans over the tensors of the bucket: [bt_eff] becomes the bucket total
-        {
-            int ca = 0, cb = 0;
-            for (int base = 0; base < bt_eff; base += kBkThreads) {
-                const int tl = base + threadIdx.x;
-                const int va = tl < bt_eff ? t_nuse[tl] : 0, vb = tl < bt_eff ? t_nper[tl] : 0;
-                int ia = va, ib = vb;
+        // ---- raw events per tensor, segment offsets, scatter (the keys of a usual bucket stay in registers)
+        constexpr int kRegKeys = 12;
+        ull rk[kRegKeys];
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int ya = __shfl_up_sync(0xffffffffu, ia, o), yb = __shfl_up_sync(0xffffffffu, ib, o);
-                    if (lane >= o) { ia += ya; ib += yb; }
-                }
-                __syncthreads();
-                if (lane == 31) { s_wa[warp] = ia; s_wb[warp] = ib; }
-                __syncthreads();
-                int pa = 0, pb = 0, ta = 0, tb = 0;
-                for (int w = 0; w < kBkThreads / 32; ++w) {
-                    if (w < warp) { pa += s_wa[w]; pb += s_wb[w]; }
-                    ta += s_wa[w]; tb += s_wb[w];
-                }
-                if (tl < bt_eff) { t_nuse[tl] = ca + pa + ia - va; t_nper[tl] = cb + pb + ib - vb; }
-                ca += ta; cb += tb;
+        for (int q = 0; q < kRegKeys; ++q) {
+            const int j = q * kBkThreads + threadIdx.x;
+            rk[q] = j < n ? gk[j] : ~0ull;
+        }
+#pragma unroll
+        for (int q = 0; q < kRegKeys; ++q)
+            if (rk[q] != ~0ull) atomicAdd(&t_off[(int)(rk[q] >> 32)], 1);
+        for (int j = kRegKeys * kBkThreads + threadIdx.x; j < n; j += kBkThreads) atomicAdd(&t_off[(int)(gk[j] >> 32)], 1);
+        __syncthreads();
+        bk_scan2(t_off, t_np, bt_eff, s_wa, s_wb);          // (t_np is all zero here and stays zero)
+#pragma unroll
+        for (int q = 0; q < kRegKeys; ++q)
+            if (rk[q] != ~0ull) {
+                const int tl = (int)(rk[q] >> 32);
+                ks[t_off[tl] + atomicAdd(&t_d[tl], 1)] = (int32_t)(unsigned)rk[q];
             }
+        for (int j = kRegKeys * kBkThreads + threadIdx.x; j < n; j += kBkThreads) {
+            const ull key = gk[j];
+            const int tl = (int)(key >> 32);
+            ks[t_off[tl] + atomicAdd(&t_d[tl], 1)] = (int32_t)(unsigned)key;
+        }
+        __syncthreads();
+        // ---- short segments: one thread sorts, removes repeats (in place) and counts the periods
+        for (int tl = threadIdx.x; tl < bt_eff; tl += kBkThreads) {
+            const int m = t_off[tl + 1] - t_off[tl];
+            int dd = 0, pp = 0;
+            if (m > kBkHeavy) {
+                const int q = atomicAdd(&s_nheavy, 1);
+                if (q < 64) s_heavy[q] = tl;
+            } else if (m > 0) {
+                int32_t *seg = ks + t_off[tl];
+                for (int a = 1; a < m; ++a) {
+                    const int32_t x = seg[a];
+                    int c = a - 1;
+                    while (c >= 0 && seg[c] > x) { seg[c + 1] = seg[c]; --c; }
+                    seg[c + 1] = x;
+                }
+                int32_t prev = seg[0];
+                dd = 1;
+                for (int a = 1; a < m; ++a) {
+                    const int32_t x = seg[a];
+                    if (x != prev) { if (x - prev >= 2) ++pp; seg[dd++] = x; prev = x; }
+                }
+            }
+            t_d[tl] = dd; t_np[tl] = pp;
+        }
+        __syncthreads();
+        // ---- long segments: the whole block sorts, compacts and counts, one tensor after the other
+        const int nheavy = s_nheavy;
+        for (int hq = 0; hq < (nheavy <= 64 ? nheavy : bt_eff); ++hq) {
+            const int tl = nheavy <= 64 ? s_heavy[hq] : hq;
+            const int m = t_off[tl + 1] - t_off[tl];
+            if (m <= kBkHeavy) continue;                       // (only when the list overflowed: uniform test)
+            int32_t *seg = ks + t_off[tl];
+            bk_bitonic_sort_i32(seg, m);
+            if (threadIdx.x == 0) { s_total = 0; s_periods = 0; }
             __syncthreads();
-            if (threadIdx.x == 0) { t_nuse[bt_eff] = ca; t_nper[bt_eff] = cb; }
+            for (int c0 = 0; c0 < m; c0 += kBkThreads) {
+                const int t = c0 + threadIdx.x;
+                int32_t x = 0, prev = 0;
+                bool keep = false, per = false;
+                if (t < m) {
+                    x = seg[t];
+                    if (t > 0) prev = seg[t - 1];
+                    keep = (t == 0) || (x != prev);
+                    per = keep && t > 0 && (x - prev >= 2);
+                }
+                const unsigned mk = __ballot_sync(0xffffffffu, keep), mp = __ballot_sync(0xffffffffu, per);
+                if (lane == 0) s_wa[warp] = __popc(mk);
+                __syncthreads();
+                int off = s_total, chunk_total = 0;
+                for (int w = 0; w < kBkThreads / 32; ++w) { if (w < warp) off += s_wa[w]; chunk_total += s_wa[w]; }
+                off += __popc(mk & ((1u << lane) - 1u));
+                __syncthreads();                               // every seg[t], seg[t-1] of this chunk has been read
+                if (keep) seg[off] = x;                        // off <= t: never overtakes an unread element
+                if (lane == 0 && mp) atomicAdd(&s_periods, __popc(mp));
+                if (threadIdx.x == 0) s_total += chunk_total;
+                __syncthreads();
+            }
+            if (threadIdx.x == 0) { t_d[tl] = s_total; t_np[tl] = s_periods; }
             __syncthreads();
         }
-        const long long D = t_nuse[bt_eff], PC = t_nper[bt_eff];
+        // ---- offsets of every tensor's distinct uses and periods inside the bucket; bucket totals
+        bk_scan2(t_d, t_np, bt_eff, s_wa, s_wb);
+        const long long D = t_d[bt_eff], PC = t_np[bt_eff];
         // ---- offsets of this bucket in the global arrays: totals of all earlier buckets
         if (threadIdx.x == 0) {
             asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&B.words[2 * b]), "l"(bk_pack(D)) : "memory");
             asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&B.words[2 * b + 1]), "l"(bk_pack(PC)) : "memory");
         }
-        long long pu = 0, pp = 0;
-        for (int j = threadIdx.x; j < 2 * b; j += kBkThreads) {
-            ull w;
+        long long pu = 0, pq = 0;
+        for (int j0 = threadIdx.x; j0 < 2 * b; j0 += 4 * kBkThreads) {
+            ull w[4];
+            bool pending = true;
             unsigned polls = 0;
-            for (;;) {
-                asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(w) : "l"(&B.words[j]) : "memory");
-                if (w >> 62) break;
-                if (++polls > kSpinLimit) { raise_status(B.status, G10_DEV_TIMEOUT); w = 0; break; }
-                __nanosleep(64);
+            while (pending) {                                  // up to four words per thread in flight
+                pending = false;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int j = j0 + q * kBkThreads;
+                    w[q] = 1ull << 62;
+                    if (j < 2 * b) asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(w[q]) : "l"(&B.words[j]) : "memory");
+                    if (!(w[q] >> 62)) pending = true;
+                }
+                if (pending) {
+                    if (++polls > kSpinLimit) { raise_status(B.status, G10_DEV_TIMEOUT); break; }
+                    __nanosleep(100);
+                }
             }
-            const long long v = (long long)(w & ((1ull << 62) - 1));
-            if (j & 1) pp += v; else pu += v;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int j = j0 + q * kBkThreads;
+                if (j < 2 * b) { const long long v = (long long)(w[q] & ((1ull << 62) - 1)); if (j & 1) pq += v; else pu += v; }
+            }
         }
-        pu = warp_sum_i64(pu); pp = warp_sum_i64(pp);
-        __shared__ long long s_pu[kBkThreads / 32], s_pp[kBkThreads / 32];
-        if (lane == 0) { s_pu[warp] = pu; s_pp[warp] = pp; }
+        pu = warp_sum_i64(pu); pq = warp_sum_i64(pq);
+        if (lane == 0) { s_pu[warp] = pu; s_pp[warp] = pq; }
         __syncthreads();
         if (threadIdx.x == 0) {
             long long a = 0, c2 = 0;
@@ -324,51 +418,33 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         if (U + D > out.uses_cap) bad |= G10_DEV_USES_OVERFLOW;
         if (PB + PC > out.periods_cap) bad |= G10_DEV_PERIODS_OVERFLOW;
         if (bad && threadIdx.x == 0) raise_status(B.status, bad);
-        // ---- per-tensor outputs, coalesced
+        // ---- outputs
         for (int tl = threadIdx.x; tl < bt_eff; tl += kBkThreads) {
             const int64_t t = t0 + tl;
-            out.first_use[t] = t_first[tl];
-            out.last_use[t] = t_last[tl];
-            out.num_uses[t] = t_nuse[tl + 1] - t_nuse[tl];
-            out.use_ptr[t] = U + t_nuse[tl];
-            out.period_ptr[t] = PB + t_nper[tl];
+            const int dd = t_d[tl + 1] - t_d[tl];
+            const int32_t *seg = ks + t_off[tl];
+            out.first_use[t] = dd > 0 ? seg[0] : -1;
+            out.last_use[t] = dd > 0 ? seg[dd - 1] : -1;
+            out.num_uses[t] = dd;
+            out.use_ptr[t] = U + t_d[tl];
+            out.period_ptr[t] = PB + t_np[tl];
+            long long uo = U + t_d[tl], po = PB + t_np[tl];
+            for (int a = 0; a < dd; ++a) {
+                const int32_t x = seg[a];
+                if (uo + a < out.uses_cap) out.uses[uo + a] = x;
+                if (a > 0 && x - seg[a - 1] >= 2) {
+                    if (po < out.periods_cap) {
+                        out.period_tensor[po] = (int32_t)t;
+                        out.period_prev_use[po] = seg[a - 1];
+                        out.period_next_use[po] = x;
+                    }
+                    ++po;
+                }
+            }
         }
         if (b == B.nb - 1 && threadIdx.x == 0) {
             out.use_ptr[B.N] = U + D; out.period_ptr[B.N] = PB + PC;
             out.counts[0] = U + D; out.counts[1] = PB + PC;
-        }
-        // ---- pass B: sorted distinct uses and periods; positions are prefix counts of the flags
-        {
-            int ca = 0, cb = 0;
-            for (int base = 0; base < n; base += kBkThreads) {
-                const int j = base + threadIdx.x;
-                BkFlags f;
-                f.dist = false; f.per = false; f.tl = 0; f.k = 0; f.kprev = 0;
-                if (j < n) f = bk_flags(kp, j, n);
-                const unsigned md = __ballot_sync(0xffffffffu, f.dist), mp = __ballot_sync(0xffffffffu, f.per);
-                __syncthreads();
-                if (lane == 0) { s_wa[warp] = __popc(md); s_wb[warp] = __popc(mp); }
-                __syncthreads();
-                int pa = 0, pb = 0, ta = 0, tb = 0;
-                for (int w = 0; w < kBkThreads / 32; ++w) {
-                    if (w < warp) { pa += s_wa[w]; pb += s_wb[w]; }
-                    ta += s_wa[w]; tb += s_wb[w];
-                }
-                const unsigned below = (1u << lane) - 1u;
-                if (f.dist) {
-                    const long long pos = U + ca + pa + __popc(md & below);
-                    if (pos < out.uses_cap) out.uses[pos] = f.k;
-                }
-                if (f.per) {
-                    const long long pos = PB + cb + pb + __popc(mp & below);
-                    if (pos < out.periods_cap) {
-                        out.period_tensor[pos] = (int32_t)(t0 + f.tl);
-                        out.period_prev_use[pos] = f.kprev;
-                        out.period_next_use[pos] = f.k;
-                    }
-                }
-                ca += ta; cb += tb;
-            }
         }
     }
 }
@@ -377,7 +453,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
 static bool choose_buckets(int64_t N, int64_t E, int *shift, int *bt, int *nb)
 {
     if (N <= 0) return false;
-    int64_t want = E > 0 ? (2500 * N) / E : 4096;        // tensors per bucket for about 2500 events
+    int64_t want = E > 0 ? (6000 * N) / E : 4096;        // tensors per bucket for about 4000-6000 events
     int s = 6;
     while (s < 12 && ((int64_t)1 << (s + 1)) <= want) ++s;
     while (s < 12 && ((N + ((int64_t)1 << s) - 1) >> s) > 4096) ++s;
@@ -399,7 +475,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     B.N = t.N; B.E = t.E; B.K = t.K;
     if (!choose_buckets(t.N, t.E, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
     B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
-    B.ticket = w.emit_scan.ticket; B.status = w.status;
+    B.ticket = w.emit_scan.ticket; B.status = w.status; B.spill = w.raw_uses;
     static int sms = 0;
     if (sms == 0) {
         int dev = 0;
@@ -412,12 +488,12 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
         k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_tensors);
-        const size_t sm2 = sizeof(int) * (size_t)(3 * B.nb + 1);
+        const size_t sm2 = sizeof(int) * (size_t)(3 * B.nb + 2) + 8 + (sizeof(ull) + sizeof(unsigned short)) * kBkTile;
         cudaError_t e = cudaFuncSetAttribute(k_bk_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
         if (e != cudaSuccess) return e;
         k_bk_scatter<<<g, kBkThreads, sm2, s>>>(B, t.kernel_ptr, t.kernel_tensors);
     }
-    const size_t sm3 = sizeof(int) * (size_t)(B.nb + 1 + 4 * B.bt + 2) + 8 + sizeof(ull) * kBkCap;
+    const size_t sm3 = sizeof(int) * (size_t)(B.nb + 1 + 3 * (B.bt + 1) + kBkCap);
     cudaError_t e = cudaFuncSetAttribute(k_bk_emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
     const int g3 = B.nb < 2 * sms ? B.nb : 2 * sms;
