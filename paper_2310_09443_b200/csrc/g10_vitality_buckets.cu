@@ -14,6 +14,8 @@
 // Everything random happens in shared memory (atomics included); HBM sees the events twice, the keys once each
 // way and the outputs once.  A bucket with more events than fit in shared memory (a tensor listed by a great many
 // kernels) keeps its segments in global memory instead: slower, same result.
+#include <cstdio>
+
 #include "g10_device.cuh"
 #include "g10_internal.h"
 
@@ -40,28 +42,59 @@ struct BucketArgs {
     ull *status;
 };
 
-// exclusive scan of cnt[0..n) into out[0..n] (out[n] = total), n <= kBkMaxBuckets, whole block
-__device__ __forceinline__ void block_scan_counts(const unsigned *cnt, int n, int *out, int *s_warp /* [32] */)
+// Block-wide exclusive scans over at most kBkThreads * 8 = 4096 entries, eight consecutive entries per thread.
+// in[0..n) -> out[0..n), out[n] = total (in == out allowed).  NA = 1 or 2 arrays scanned together.
+template <int NA>
+__device__ __forceinline__ void bk_block_scan(const int *in0, int *out0, const int *in1, int *out1, int n, int *s_w /* [NA][kBkThreads/32 + 1] */)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    int carry = 0;
-    for (int base = 0; base < n; base += blockDim.x) {
-        const int j = base + threadIdx.x;
-        const int v = j < n ? (int)cnt[j] : 0;
-        int incl = v;
+    constexpr int W = kBkThreads / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int base = threadIdx.x * 8;
+    int v[NA][8], tot[NA];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
-        __syncthreads();
-        if (lane == 31) s_warp[warp] = incl;
-        __syncthreads();
-        int wpre = 0, tot = 0;
-        for (int w = 0; w < nw; ++w) { const int x = s_warp[w]; if (w < warp) wpre += x; tot += x; }
-        if (j < n) out[j] = carry + wpre + incl - v;
-        carry += tot;
+    for (int a = 0; a < NA; ++a) {
+        const int *in = a == 0 ? in0 : in1;
+        tot[a] = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { v[a][j] = base + j < n ? in[base + j] : 0; tot[a] += v[a][j]; }
+    }
+    int incl[NA];
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+        incl[a] = tot[a];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl[a], o); if (lane >= o) incl[a] += y; }
+    }
+    __syncthreads();                                      // all inputs read (in == out), scratch free
+#pragma unroll
+    for (int a = 0; a < NA; ++a) if (lane == 31) s_w[a * (W + 1) + warp] = incl[a];
+    __syncthreads();
+    if (warp == 0) {
+#pragma unroll
+        for (int a = 0; a < NA; ++a) {
+            const int x = lane < W ? s_w[a * (W + 1) + lane] : 0;
+            int xi = x;
+#pragma unroll
+            for (int o = 1; o < W; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, xi, o); if (lane >= o) xi += y; }
+            if (lane < W) s_w[a * (W + 1) + lane] = xi - x;
+            if (lane == W - 1) s_w[a * (W + 1) + W] = xi;
+        }
     }
     __syncthreads();
-    if (threadIdx.x == 0) out[n] = carry;
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+        int *out = a == 0 ? out0 : out1;
+        int run = s_w[a * (W + 1) + warp] + incl[a] - tot[a];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { if (base + j < n) out[base + j] = run; run += v[a][j]; }
+        if (threadIdx.x == 0) out[n] = s_w[a * (W + 1) + W];
+    }
     __syncthreads();
+}
+
+__device__ __forceinline__ void block_scan_counts(const unsigned *cnt, int n, int *out, int *s_w)
+{
+    bk_block_scan<1>((const int *)cnt, out, nullptr, nullptr, n, s_w);
 }
 
 // last k in [lo, hi] with kptr[k] <= e
@@ -137,7 +170,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
     unsigned *s_off = (unsigned *)(s_cnt + B.nb + 1);      // [nb] where this tile's events start inside the bucket
     ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkTile] keys of the tile in bucket order
     unsigned short *s_bkt = (unsigned short *)(s_key + kBkTile);              // [kBkTile] their buckets
-    __shared__ int s_warp[32];
+    __shared__ int s_warp[2 * (kBkThreads / 32 + 1)];
     __shared__ int64_t s_ptr[kBkPtrStage];
     __shared__ int s_lohi[2];
     block_scan_counts(B.bucket_count, B.nb, s_base, s_warp);
@@ -226,64 +259,49 @@ __device__ void bk_bitonic_sort_i32(int32_t *a, int n)    // arbitrary n: the ne
 
 __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
 
-// in-place exclusive scan of two int arrays a[0..n), b[0..n); a[n], b[n] receive the totals; whole block
-__device__ __forceinline__ void bk_scan2(int *a, int *b, int n, int *s_wa, int *s_wb)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int ca = 0, cb = 0;
-    for (int base = 0; base < n; base += kBkThreads) {
-        const int t = base + threadIdx.x;
-        const int va = t < n ? a[t] : 0, vb = t < n ? b[t] : 0;
-        int ia = va, ib = vb;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int ya = __shfl_up_sync(0xffffffffu, ia, o), yb = __shfl_up_sync(0xffffffffu, ib, o);
-            if (lane >= o) { ia += ya; ib += yb; }
-        }
-        __syncthreads();
-        if (lane == 31) { s_wa[warp] = ia; s_wb[warp] = ib; }
-        __syncthreads();
-        int pa = 0, pb = 0, ta = 0, tb = 0;
-        for (int w = 0; w < kBkThreads / 32; ++w) {
-            if (w < warp) { pa += s_wa[w]; pb += s_wb[w]; }
-            ta += s_wa[w]; tb += s_wb[w];
-        }
-        if (t < n) { a[t] = ca + pa + ia - va; b[t] = cb + pb + ib - vb; }
-        ca += ta; cb += tb;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) { a[n] = ca; b[n] = cb; }
-    __syncthreads();
-}
+#ifdef G10_PHASE_CLOCKS
+#define BK_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
+                         ph_acc[i] += now_ - ph_last; ph_last = now_; asm volatile("" ::: "memory"); } } while (0)
+#else
+#define BK_CLOCK(i)
+#endif
 
 __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBuffers out)
 {
+#ifdef G10_PHASE_CLOCKS
+    long long ph_acc[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
+    int ph_n = 0;
+#endif
     extern __shared__ int s_mem[];
     int *s_base = s_mem;                       // [nb + 1] first key of each bucket
     int *t_off = s_base + B.nb + 1;            // [bt + 1] raw events per tensor, then segment offsets
     int *t_d = t_off + B.bt + 1;               // [bt + 1] scatter cursor, then distinct uses, then their offsets
     int *t_np = t_d + B.bt + 1;                // [bt + 1] periods per tensor, then their offsets
     int32_t *s_ks = t_np + B.bt + 1;           // [kBkCap] kernels, tensor segment after tensor segment
-    __shared__ int s_warp[32];
-    __shared__ int s_wa[kBkThreads / 32], s_wb[kBkThreads / 32];
+    __shared__ int s_scan[2 * (kBkThreads / 32 + 1)];
+    __shared__ int s_wa[kBkThreads / 32];
     __shared__ long long s_pu[kBkThreads / 32], s_pp[kBkThreads / 32];
     __shared__ int s_bucket, s_nheavy, s_total, s_periods;
     __shared__ int s_heavy[64];
     __shared__ long long s_pre[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    block_scan_counts(B.bucket_count, B.nb, s_base, s_warp);
+    block_scan_counts(B.bucket_count, B.nb, s_base, s_scan);
     for (;;) {
         __syncthreads();
         if (threadIdx.x == 0) { s_bucket = (int)atomicAdd(B.ticket, 1u); s_nheavy = 0; }
         __syncthreads();
         const int b = s_bucket;
         if (b >= B.nb) break;
+        BK_CLOCK(0);
+#ifdef G10_PHASE_CLOCKS
+        ph_n += 1;
+#endif
         const int n = s_base[b + 1] - s_base[b];
         const int64_t t0 = (int64_t)b * B.bt;
         const int bt_eff = (int)((B.N - t0) < B.bt ? (B.N - t0) : B.bt);
         const ull *gk = B.pairs + s_base[b];
         int32_t *ks = n <= kBkCap ? s_ks : B.spill + s_base[b];
-        for (int tl = threadIdx.x; tl <= bt_eff; tl += kBkThreads) { t_off[tl] = 0; t_d[tl] = 0; t_np[tl] = 0; }
+        for (int tl = threadIdx.x; tl <= bt_eff; tl += kBkThreads) { t_off[tl] = 0; t_d[tl] = 0; }
         __syncthreads();
         // ---- raw events per tensor, segment offsets, scatter (the keys of a usual bucket stay in registers)
         constexpr int kRegKeys = 12;
@@ -298,7 +316,9 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             if (rk[q] != ~0ull) atomicAdd(&t_off[(int)(rk[q] >> 32)], 1);
         for (int j = kRegKeys * kBkThreads + threadIdx.x; j < n; j += kBkThreads) atomicAdd(&t_off[(int)(gk[j] >> 32)], 1);
         __syncthreads();
-        bk_scan2(t_off, t_np, bt_eff, s_wa, s_wb);          // (t_np is all zero here and stays zero)
+        BK_CLOCK(1);
+        bk_block_scan<1>(t_off, t_off, nullptr, nullptr, bt_eff, s_scan);
+        BK_CLOCK(2);
 #pragma unroll
         for (int q = 0; q < kRegKeys; ++q)
             if (rk[q] != ~0ull) {
@@ -311,6 +331,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             ks[t_off[tl] + atomicAdd(&t_d[tl], 1)] = (int32_t)(unsigned)key;
         }
         __syncthreads();
+        BK_CLOCK(3);
         // ---- short segments: one thread sorts, removes repeats (in place) and counts the periods
         for (int tl = threadIdx.x; tl < bt_eff; tl += kBkThreads) {
             const int m = t_off[tl + 1] - t_off[tl];
@@ -336,6 +357,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             t_d[tl] = dd; t_np[tl] = pp;
         }
         __syncthreads();
+        BK_CLOCK(4);
         // ---- long segments: the whole block sorts, compacts and counts, one tensor after the other
         const int nheavy = s_nheavy;
         for (int hq = 0; hq < (nheavy <= 64 ? nheavy : bt_eff); ++hq) {
@@ -372,7 +394,9 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             __syncthreads();
         }
         // ---- offsets of every tensor's distinct uses and periods inside the bucket; bucket totals
-        bk_scan2(t_d, t_np, bt_eff, s_wa, s_wb);
+        BK_CLOCK(5);
+        bk_block_scan<2>(t_d, t_d, t_np, t_np, bt_eff, s_scan);
+        BK_CLOCK(6);
         const long long D = t_d[bt_eff], PC = t_np[bt_eff];
         // ---- offsets of this bucket in the global arrays: totals of all earlier buckets
         if (threadIdx.x == 0) {
@@ -414,6 +438,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         }
         __syncthreads();
         const long long U = s_pre[0], PB = s_pre[1];
+        BK_CLOCK(7);
         ull bad = 0;
         if (U + D > out.uses_cap) bad |= G10_DEV_USES_OVERFLOW;
         if (PB + PC > out.periods_cap) bad |= G10_DEV_PERIODS_OVERFLOW;
@@ -446,7 +471,14 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             out.use_ptr[B.N] = U + D; out.period_ptr[B.N] = PB + PC;
             out.counts[0] = U + D; out.counts[1] = PB + PC;
         }
+        BK_CLOCK(8);
     }
+#ifdef G10_PHASE_CLOCKS
+    if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 100) && ph_n > 0)
+        printf("k_bk_emit block %d (%d buckets) cycles/bucket: ticket %lld load+count %lld scan %lld scatter %lld short %lld heavy %lld scan2 %lld prefix %lld outputs %lld\n",
+               blockIdx.x, ph_n, ph_acc[0] / ph_n, ph_acc[1] / ph_n, ph_acc[2] / ph_n, ph_acc[3] / ph_n, ph_acc[4] / ph_n, ph_acc[5] / ph_n,
+               ph_acc[6] / ph_n, ph_acc[7] / ph_n, ph_acc[8] / ph_n);
+#endif
 }
 
 // Picks the bucket width for a trace; false if the trace is outside what the bucket path handles.
