@@ -481,3 +481,47 @@ int32_t g10o_plan(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t
     free(S.hocc); free(alive); free(heap); free(popped); free(dest); free(ver);
     return rc;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Smart tensor prefetching (Section 4.4).  The eviction loop above assumes every prefetch at its
+ * latest safe prefetch time.  Afterwards the evicted periods are sorted by that time and visited in
+ * order; for each one the search goes backward from the latest safe prefetch time to the earliest
+ * time at which the GPU can hold the whole tensor with the space that is left, the prefetch is
+ * rescheduled there and the pressure curve in between is updated.
+ * Readings: (1) whole-slot granularity as in the eviction loop -- the tensor becomes resident again
+ * in whole slots, so the search walks slot by slot from absent_last downwards while pressure + size
+ * stays within capacity, never past absent_first; (2) ties in the sort go to the earlier plan
+ * record; (3) only memory is examined, as the section says -- channel bookings are not revisited;
+ * (4) a prefetch that moves is issued at the start of the first slot in which the tensor is resident
+ * again; one that cannot move keeps its time.
+ * order[i] = plan record visited i-th; new_absent_last / new_issue_ns are indexed by plan record.
+ * summary[4] = { prefetches moved, slots regained in total, peak pressure after, its lowest slot }.
+ * ---------------------------------------------------------------------------------------- */
+void g10o_schedule_prefetch(int64_t K, int64_t n, const g10o_migration *mig, const int64_t *start,
+                            const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes, int64_t *pressure /* [K] in/out */,
+                            int32_t *order, int32_t *new_absent_last, int64_t *new_issue_ns, int64_t *summary)
+{
+    int64_t cap = gpu_capacity_bytes >= ((uint64_t)1 << 63) ? INT64_MAX : (int64_t)gpu_capacity_bytes;
+    for (int64_t i = 0; i < n; ++i) order[i] = (int32_t)i;
+    /* insertion sort by (latest safe prefetch time, record): plain and stable */
+    for (int64_t i = 1; i < n; ++i) {
+        int32_t x = order[i];
+        int64_t j = i - 1;
+        while (j >= 0 && (mig[order[j]].prefetch_issue_ns > mig[x].prefetch_issue_ns)) { order[j + 1] = order[j]; --j; }
+        order[j + 1] = x;
+    }
+    int64_t moved = 0, regained = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        const g10o_migration *m = &mig[order[i]];
+        int64_t s = tensor_bytes[m->tensor];
+        int64_t j = m->absent_last;
+        while (j >= m->absent_first && pressure[j] <= cap - s) --j;      /* pressure + s <= cap, without overflow */
+        for (int64_t k = j + 1; k <= m->absent_last; ++k) pressure[k] += s;
+        new_absent_last[order[i]] = (int32_t)j;
+        new_issue_ns[order[i]] = j < m->absent_last ? start[j + 1] : m->prefetch_issue_ns;
+        if (j < m->absent_last) { moved += 1; regained += m->absent_last - j; }
+    }
+    int64_t pk, ps;
+    peak_of(pressure, K, &pk, &ps);
+    summary[0] = moved; summary[1] = regained; summary[2] = pk; summary[3] = ps;
+}

@@ -128,3 +128,18 @@ def plan(trace, gpu_capacity_bytes, host_bw=None, ssd_bw=None, host_capacity_byt
     ben = [int(wb[2 * j]) | (int(wb[2 * j + 1]) << 64) for j in range(n)]
     return SimpleNamespace(migrations=out[:n].copy(), final_pressure=finalP, summary=summary,
                            status=STATUS[int(summary[2])], win_benefit=ben, win_cost=wc[:n].copy())
+
+
+def schedule_prefetch(K, migrations, start, tensor_bytes, gpu_capacity_bytes, pressure):
+    """Section 4.4 eager prefetch pass over a finished eviction plan.  Returns new pressure and per-record results."""
+    mig = np.ascontiguousarray(migrations)
+    assert mig.dtype == MIGRATION_DTYPE
+    n = mig.shape[0]
+    st = _c(start, np.int64); tb = _c(tensor_bytes, np.int64)
+    P = _c(pressure, np.int64).copy()
+    order = np.zeros(max(n, 1), np.int32); nal = np.zeros(max(n, 1), np.int32); nis = np.zeros(max(n, 1), np.int64)
+    summary = np.zeros(4, np.int64)
+    lib().g10o_schedule_prefetch(C.c_int64(K), C.c_int64(n), _p(mig), _p(st), _p(tb), C.c_uint64(gpu_capacity_bytes),
+                                 _p(P), _p(order), _p(nal), _p(nis), _p(summary))
+    return SimpleNamespace(pressure=P, order=order[:n].copy(), new_absent_last=nal[:n].copy(),
+                           new_prefetch_issue_ns=nis[:n].copy(), summary=summary)

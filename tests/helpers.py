@@ -235,3 +235,26 @@ def check_plan_invariants(tr, cap, start, P0, vit, migrations, final_pressure, s
     if status in ("EXHAUSTED", "ITERATION_LIMIT"):
         assert (P.max() if K else 0) > cap
     return P, busy, hocc
+
+
+# ------------------------------------------------------------------------------------------------
+# Eager prefetch pass (Section 4.4), dense restatement
+# ------------------------------------------------------------------------------------------------
+def brute_prefetch(plan, pressure, start, tensor_bytes, cap):
+    """plan: list of dicts as returned by brute_plan; returns (order, new_absent_last, new_issue, new pressure)."""
+    P = list(pressure)
+    order = sorted(range(len(plan)), key=lambda i: (plan[i]["prefetch_issue_ns"], i))
+    new_last = [None] * len(plan)
+    new_issue = [None] * len(plan)
+    for i in order:
+        m = plan[i]
+        s = int(tensor_bytes[m["tensor"]])
+        # earliest slot j such that the tensor fits in every slot j .. absent_last
+        j = m["absent_last"] + 1
+        while j - 1 >= m["absent_first"] and P[j - 1] + s <= cap:
+            j -= 1
+        for k in range(j, m["absent_last"] + 1):
+            P[k] += s
+        new_last[i] = j - 1
+        new_issue[i] = start[j] if j <= m["absent_last"] else m["prefetch_issue_ns"]
+    return order, new_last, new_issue, P
