@@ -150,9 +150,9 @@ typedef struct g10_options {
 
 #define G10_NUM_PLAN_STAGES 5
 
-#define G10_FLAG_RESCORE_ALL 0x1    /* rescore every live period every iteration (Algorithm 1 as
-                                       printed) instead of only those whose score can have changed;
-                                       the plan is identical, the run is slower                     */
+#define G10_FLAG_RESCORE_ALL 0x1    /* the plain formulation of every stage: every live period rescored every
+                                       iteration (Algorithm 1 as printed), use lists built with global atomics
+                                       instead of shared-memory buckets; identical results, slower           */
 
 #define G10_FLAG_GLOBAL_STATE 0x2   /* keep the planner state in global memory even when the timeline would fit
                                        in shared memory (the path large traces take); same plan              */
@@ -185,6 +185,26 @@ int32_t g10_candidate_geometry(int64_t num_kernels, int64_t num_periods, const i
 int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
                             const g10_options *options /* NULL = defaults */, g10_plan_out *out,
                             void *ws, size_t ws_bytes, void *stream);
+
+/* Section 4.4, smart tensor prefetching: visits the committed migrations in the order of their latest safe
+   prefetch time (ties: the earlier plan record) and moves each prefetch back to the earliest slot from which
+   pressure + size stays within gpu_capacity_bytes up to the old prefetch slot (never past absent_first), adding
+   the tensor's size to the slots it becomes resident in again.  Only memory is examined (the section says nothing
+   of bandwidth); a prefetch that moves is issued at the start of its first newly resident slot.
+   All pointers are DEVICE pointers.  `pressure` [K] is the final pressure of the eviction plan on entry and the
+   pressure after the pass on return; order [n] receives the visiting order; new_absent_last [n] and
+   new_prefetch_issue_ns [n] are indexed by plan record; summary [4] = prefetches moved, slots regained, new peak,
+   its lowest slot.  Needs no workspace; one block does the (strictly sequential) pass. */
+typedef struct g10_prefetch_out {
+    int64_t *pressure;
+    int32_t *order;
+    int32_t *new_absent_last;
+    int64_t *new_prefetch_issue_ns;
+    int64_t *summary;
+} g10_prefetch_out;
+int32_t g10_schedule_prefetch(int64_t num_kernels, int64_t num_migrations, const g10_migration *migrations,
+                              const int64_t *kernel_start_ns, const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes,
+                              g10_prefetch_out *out, void *stream);
 
 /* The paper has no counterpart for this entry point: it is g10_pressure_timeline for callers that cannot
    allocate device memory when they need a timeline (a host whose device memory is wholly owned by its own

@@ -23,7 +23,7 @@ FLAG_RESCORE_ALL = 1
 FLAG_GLOBAL_STATE = 2
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
-           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static")
+           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch")
 STATIC_MAX_KERNELS, STATIC_MAX_TENSORS = 32768, 131072
 
 MIGRATION_DTYPE = np.dtype([
@@ -60,6 +60,11 @@ class _PlanOut(C.Structure):
                 ("summary", C.c_void_p)]
 
 
+class _PrefetchOut(C.Structure):
+    _fields_ = [("pressure", C.c_void_p), ("order", C.c_void_p), ("new_absent_last", C.c_void_p),
+                ("new_prefetch_issue_ns", C.c_void_p), ("summary", C.c_void_p)]
+
+
 class _Options(C.Structure):
     _fields_ = [("host_capacity_bytes", C.c_uint64), ("max_iterations", C.c_int64), ("flags", C.c_uint32),
                 ("stage_events", C.POINTER(C.c_void_p)), ("num_stage_events", C.c_int32)]
@@ -89,6 +94,9 @@ def load_library():
         lib.g10_candidate_geometry.restype = C.c_int32
         lib.g10_candidate_geometry.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_uint64, C.c_uint64, C.POINTER(_GeometryOut), C.c_void_p]
+        lib.g10_schedule_prefetch.restype = C.c_int32
+        lib.g10_schedule_prefetch.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
+                                              C.POINTER(_PrefetchOut), C.c_void_p]
         lib.g10_plan_migrations.restype = C.c_int32
         lib.g10_plan_migrations.argtypes = [C.POINTER(_Trace), C.c_uint64, C.c_uint64, C.c_uint64, C.POINTER(_Options),
                                             C.POINTER(_PlanOut), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -278,6 +286,23 @@ def g10_plan_migrations(tb: TraceBuffers, gpu_capacity_bytes, host_bw, ssd_bw, h
                                    ws_bytes, _stream(stream)))
     out.workspace = ws
     return out
+
+
+def g10_schedule_prefetch(K, num_migrations, migrations, kernel_start_ns, tensor_bytes, gpu_capacity_bytes, pressure,
+                          stream=None):
+    """Section 4.4 eager prefetch pass.  `migrations` is the uint8 record tensor of a finished plan, `pressure` its
+    final pressure (updated in place).  Device tensors only."""
+    lib = load_library()
+    dev = kernel_start_ns.device
+    n = int(num_migrations)
+    r = SimpleNamespace(pressure=pressure, order=torch.empty(max(n, 1), dtype=torch.int32, device=dev),
+                        new_absent_last=torch.empty(max(n, 1), dtype=torch.int32, device=dev),
+                        new_prefetch_issue_ns=torch.empty(max(n, 1), dtype=torch.int64, device=dev),
+                        summary=torch.empty(4, dtype=torch.int64, device=dev))
+    out = _PrefetchOut(_ptr(r.pressure), _ptr(r.order), _ptr(r.new_absent_last), _ptr(r.new_prefetch_issue_ns), _ptr(r.summary))
+    _check(lib.g10_schedule_prefetch(K, n, _ptr(migrations), _ptr(kernel_start_ns), _ptr(tensor_bytes), gpu_capacity_bytes,
+                                     C.byref(out), _stream(stream)))
+    return r
 
 
 def migrations_numpy(plan) -> np.ndarray:

@@ -315,6 +315,19 @@ int32_t g10_candidate_geometry(int64_t K, int64_t Pn, const int64_t *kernel_star
     return G10_OK;
 }
 
+int32_t g10_schedule_prefetch(int64_t K, int64_t n, const g10_migration *migrations, const int64_t *kernel_start_ns,
+                              const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes, g10_prefetch_out *out, void *stream)
+{
+    if (K < 0 || n < 0 || !out || !out->summary) return G10_ERR_ARG;
+    if (K >= (((int64_t)1 << 31) - 1) || n >= (((int64_t)1 << 31) - 1)) return G10_ERR_LIMIT;
+    if (K > 0 && !out->pressure) return G10_ERR_ARG;
+    if (n > 0 && (!migrations || !kernel_start_ns || !tensor_bytes || !out->order || !out->new_absent_last || !out->new_prefetch_issue_ns))
+        return G10_ERR_ARG;
+    CU(launch_schedule_prefetch(K, n, migrations, kernel_start_ns, tensor_bytes, gpu_capacity_bytes, out->pressure, out->order,
+                                out->new_absent_last, out->new_prefetch_issue_ns, out->summary, (cudaStream_t)stream));
+    return G10_OK;
+}
+
 int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
                             const g10_options *options, g10_plan_out *out, void *ws, size_t ws_bytes, void *stream)
 {

@@ -134,6 +134,10 @@ cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int3
 cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, const int64_t *start, const int64_t *tensor_bytes,
                             const int32_t *per_t, const int32_t *per_u, const int32_t *per_v, uint64_t host_bw, uint64_t ssd_bw,
                             int64_t stride, int64_t *geo_t, int32_t *geo_a, int32_t *geo_b, cudaStream_t s);
+// eager prefetch pass (g10_prefetch.cu)
+cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *mig, const int64_t *start, const int64_t *bytes,
+                                     uint64_t gpu_capacity_bytes, int64_t *P, int32_t *order, int32_t *new_last, int64_t *new_issue,
+                                     int64_t *summary, cudaStream_t s);
 // planner (g10_planner.cu)
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
 int plan_loop_max_blocks();

@@ -27,12 +27,17 @@ def main():
     start, P0, peak, slot = O.timeline(tr)
     cap = tr.capacity_from_peak(peak)
     r = O.plan(tr, cap, lazy=True)
+    pf = O.schedule_prefetch(tr.K, r.migrations, start, tr.tensor_bytes, cap, r.final_pressure)
+    hp = hashlib.sha256()
+    for a in (pf.order, pf.new_absent_last, pf.new_prefetch_issue_ns, pf.pressure, pf.summary):
+        hp.update(a.tobytes())
     out = {
         "_source": "oracle/g10_oracle.c, lazy tier, on paper_2310_09443_b200.traces.config4_stress_dag() (seed 4)",
         "trace_sha256": tr.sha256(), "peak_bytes": int(peak), "peak_slot": int(slot), "capacity_bytes": int(cap),
         "summary": [int(x) for x in r.summary[:7]], "status": r.status,
         "first_migrations": [[int(m[k]) for k in m.dtype.names] for m in r.migrations[:5]],
         "plan_sha256": digest(r.migrations, r.final_pressure, r.summary),
+        "prefetch_summary": [int(x) for x in pf.summary], "prefetch_sha256": hp.hexdigest(),
     }
     path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "config4_plan_digest.json")
     with open(path, "w") as f:

@@ -270,3 +270,59 @@ def test_full_size_stress_plan_digest(gpu):
     h = hashlib.sha256()
     h.update(mig.tobytes()); h.update(_np(plan.final_pressure)[:tr.K].tobytes()); h.update(summary[:7].tobytes())
     assert h.hexdigest() == gold["plan_sha256"]
+    # the eager prefetch pass over the same plan
+    n = int(summary[0])
+    pf = gpu.g10_schedule_prefetch(tr.K, n, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap, plan.final_pressure)
+    torch.cuda.synchronize()
+    assert _np(pf.summary).tolist() == gold["prefetch_summary"]
+    hp = hashlib.sha256()
+    for a in (_np(pf.order)[:n], _np(pf.new_absent_last)[:n], _np(pf.new_prefetch_issue_ns)[:n], _np(pf.pressure)[:tr.K], _np(pf.summary)):
+        hp.update(np.ascontiguousarray(a).tobytes())
+    assert hp.hexdigest() == gold["prefetch_sha256"]
+
+
+def check_prefetch(gpu, oracle, tr, cap):
+    """Eviction plan then the eager prefetch pass (Section 4.4), both sides from their own plan."""
+    import torch
+    tb = gpu.upload(tr)
+    tl = gpu.g10_pressure_timeline(tb)
+    plan = gpu.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    n = int(plan.summary[0].item())
+    pf = gpu.g10_schedule_prefetch(tr.K, n, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap, plan.final_pressure)
+    torch.cuda.synchronize()
+    start = oracle.slot_clock(tr.kernel_ns)
+    ref = oracle.plan(tr, cap, lazy=True)
+    opf = oracle.schedule_prefetch(tr.K, ref.migrations, start, tr.tensor_bytes, cap, ref.final_pressure)
+    assert n == len(ref.migrations)
+    assert np.array_equal(_np(pf.order)[:n], opf.order)
+    assert np.array_equal(_np(pf.new_absent_last)[:n], opf.new_absent_last)
+    assert np.array_equal(_np(pf.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
+    assert np.array_equal(_np(pf.pressure)[:tr.K], opf.pressure)
+    assert np.array_equal(_np(pf.summary), opf.summary)
+    return opf
+
+
+def test_prefetch_pass(gpu, oracle):
+    import json, os
+    ex = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_worked_examples.json")))["examples"]["prefetch"]
+    tr = traces.from_lists("p", ex["kernel_lists"], ex["tensor_bytes"], ex["kernel_ns"], host_bw=ex["host_bw"], ssd_bw=ex["ssd_bw"])
+    opf = check_prefetch(gpu, oracle, tr, ex["capacity"])
+    assert opf.pressure.tolist() == ex["prefetch_pass"]["pressure"]
+    rng = np.random.default_rng(99)
+    for trial in range(40):
+        toy = traces.random_toy(rng, int(rng.integers(4, 40)), int(rng.integers(1, 30)), max_deg=5)
+        start, P0, peak, slot = oracle.timeline(toy)
+        check_prefetch(gpu, oracle, toy, peak * int(rng.integers(1, 10)) // 10)
+    moved = 0
+    for cfg in (0, 1, 2, 3):
+        tr = traces.make_config(cfg)
+        start, P0, peak, slot = oracle.timeline(tr)
+        moved += int(check_prefetch(gpu, oracle, tr, tr.capacity_from_peak(peak)).summary[0])
+        if cfg == 0:
+            moved += int(check_prefetch(gpu, oracle, tr, peak * 9 // 10).summary[0])      # ends FIT: room to move
+    assert moved > 0
+    tr = traces.config4_stress_dag(K=20000, N=80000)
+    start, P0, peak, slot = oracle.timeline(tr)
+    check_prefetch(gpu, oracle, tr, tr.capacity_from_peak(peak))
+    check_prefetch(gpu, oracle, tr, peak * 8 // 10)
