@@ -161,6 +161,7 @@ typedef struct g10_options {
 #define G10_WS_TIMELINE 1
 #define G10_WS_PLAN 2
 #define G10_WS_GEOMETRY 3
+#define G10_WS_EMIT 4
 
 /* Section 4.2, tensor vitality analysis. */
 int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, size_t ws_bytes, void *stream);
@@ -205,6 +206,37 @@ typedef struct g10_prefetch_out {
 int32_t g10_schedule_prefetch(int64_t num_kernels, int64_t num_migrations, const g10_migration *migrations,
                               const int64_t *kernel_start_ns, const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes,
                               g10_prefetch_out *out, void *stream);
+
+/* Section 4.4, code instrumentation (the instrumented program of Figure 9): the g10_alloc / g10_free /
+   g10_pre_evict / g10_prefetch calls to insert between the kernels.  Boundary b (0 <= b <= K) is the gap before
+   kernel b (b = K: after the last kernel).  ALLOC sits before the first kernel using the tensor (boundary 0 for a
+   global tensor), FREE right after the last kernel using an intermediate tensor (global tensors are never freed),
+   PRE_EVICT at the boundary whose time is the period start t_r, PREFETCH at the last boundary at or before its
+   issue time.  Inside a boundary: FREE, PRE_EVICT, ALLOC, PREFETCH (as in Figure 9), then by tensor id.
+   inst_ptr [K + 2] is the CSR by boundary; counts [2] = number of instructions, device status word
+   (G10_DEV_PLAN_OVERFLOW if instructions_cap is too small).  new_prefetch_issue_ns (optional) are the times from
+   g10_schedule_prefetch.  All pointers are DEVICE pointers; `ws` as for the other calls (G10_WS_EMIT, with the
+   number of migrations in place of E).  Limits: K + 1 <= 4096 * 4096 boundaries. */
+#define G10_OP_FREE 0
+#define G10_OP_PRE_EVICT 1
+#define G10_OP_ALLOC 2
+#define G10_OP_PREFETCH 3
+typedef struct g10_instruction {
+    int32_t opcode, tensor;
+    int32_t target;                 /* destination of a pre-eviction (G10_DEST_*), else -1 */
+    int32_t record;                 /* plan record of a pre-eviction / prefetch, else -1   */
+    int64_t bytes, time_ns;
+} g10_instruction;                  /* 32 bytes */
+typedef struct g10_emit_out {
+    int64_t *inst_ptr;
+    g10_instruction *instructions;
+    int64_t instructions_cap;       /* 2 * N + 2 * num_migrations always suffices */
+    int64_t *counts;
+} g10_emit_out;
+int32_t g10_emit_instructions(int64_t num_kernels, int64_t num_tensors, const int32_t *first_use, const int32_t *last_use,
+                              const int64_t *tensor_bytes, const uint8_t *tensor_global, const int64_t *kernel_start_ns,
+                              int64_t num_migrations, const g10_migration *migrations, const int64_t *new_prefetch_issue_ns,
+                              g10_emit_out *out, void *ws, size_t ws_bytes, void *stream);
 
 /* The paper has no counterpart for this entry point: it is g10_pressure_timeline for callers that cannot
    allocate device memory when they need a timeline (a host whose device memory is wholly owned by its own

@@ -525,3 +525,82 @@ void g10o_schedule_prefetch(int64_t K, int64_t n, const g10o_migration *mig, con
     peak_of(pressure, K, &pk, &ps);
     summary[0] = moved; summary[1] = regained; summary[2] = pk; summary[3] = ps;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Code instrumentation (Section 4.4; the instrumented program of Figure 9): the list of
+ * g10_alloc / g10_free / g10_pre_evict / g10_prefetch calls inserted between the kernels.
+ * Boundary b (0 <= b <= K) is the gap before kernel b (b = K: after the last kernel).
+ *   ALLOC     before the first kernel that uses the tensor; a global tensor (weights) is allocated
+ *             at the beginning of the program: boundary 0.  (Figure 9: g10_alloc before Kernel 3.)
+ *   FREE      right after the last kernel that uses an intermediate tensor: boundary last + 1;
+ *             global tensors are never freed.  (Figure 9: g10_free right after Kernel 4.)
+ *   PRE_EVICT at the start of the inactive period, t_r: the boundary whose time is t_r.
+ *   PREFETCH  at its issue time; an instruction can only sit between kernels, so it goes to the
+ *             last boundary at or before that time (earlier is safe, later is not).
+ * Within one boundary the order is FREE, PRE_EVICT (tidy up after the previous kernel), ALLOC,
+ * PREFETCH (get ready for the next), as in Figure 9; then by tensor id.  A tensor never has two
+ * instructions of the same kind at one boundary, so the order is total.
+ * new_issue_ns (optional): prefetch times from the eager prefetch pass, indexed by plan record.
+ * Returns the number of instructions (records beyond out_cap are not written).
+ * ---------------------------------------------------------------------------------------- */
+enum { OP_FREE = 0, OP_PRE_EVICT = 1, OP_ALLOC = 2, OP_PREFETCH = 3 };
+
+typedef struct {
+    int32_t opcode, tensor, target, record;     /* target: destination of a pre-eviction, else -1; record: plan record, else -1 */
+    int64_t bytes, time_ns;
+} g10o_instruction;
+
+typedef struct { int64_t boundary; g10o_instruction ins; } keyed_ins;
+
+static int cmp_keyed(const void *x, const void *y)
+{
+    const keyed_ins *a = (const keyed_ins *)x, *b = (const keyed_ins *)y;
+    if (a->boundary != b->boundary) return a->boundary < b->boundary ? -1 : 1;
+    if (a->ins.opcode != b->ins.opcode) return a->ins.opcode < b->ins.opcode ? -1 : 1;
+    if (a->ins.tensor != b->ins.tensor) return a->ins.tensor < b->ins.tensor ? -1 : 1;
+    return 0;
+}
+
+int64_t g10o_emit_instructions(int64_t K, int64_t N, const int32_t *first_use, const int32_t *last_use,
+                               const int64_t *tensor_bytes, const uint8_t *tensor_global, const int64_t *start,
+                               int64_t n, const g10o_migration *mig, const int64_t *new_issue_ns,
+                               int64_t *inst_ptr /* [K+2] */, g10o_instruction *out, int64_t out_cap)
+{
+    keyed_ins *list = (keyed_ins *)malloc(sizeof(keyed_ins) * (size_t)(2 * N + 2 * n + 1));
+    int64_t m = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        if (first_use[i] < 0) continue;
+        int glob = tensor_global && tensor_global[i];
+        keyed_ins a; a.boundary = glob ? 0 : first_use[i];
+        a.ins.opcode = OP_ALLOC; a.ins.tensor = (int32_t)i; a.ins.target = -1; a.ins.record = -1;
+        a.ins.bytes = tensor_bytes[i]; a.ins.time_ns = start[a.boundary];
+        list[m++] = a;
+        if (!glob) {
+            keyed_ins f = a; f.boundary = (int64_t)last_use[i] + 1; f.ins.opcode = OP_FREE; f.ins.time_ns = start[f.boundary];
+            list[m++] = f;
+        }
+    }
+    for (int64_t r = 0; r < n; ++r) {
+        keyed_ins e;
+        int64_t b = 0;
+        while (start[b] < mig[r].evict_issue_ns) ++b;            /* the boundary whose time is t_r */
+        e.boundary = b; e.ins.opcode = OP_PRE_EVICT; e.ins.tensor = mig[r].tensor; e.ins.target = mig[r].dest;
+        e.ins.record = (int32_t)r; e.ins.bytes = tensor_bytes[mig[r].tensor]; e.ins.time_ns = mig[r].evict_issue_ns;
+        list[m++] = e;
+        keyed_ins p = e;
+        int64_t t = new_issue_ns ? new_issue_ns[r] : mig[r].prefetch_issue_ns;
+        b = K;
+        while (start[b] > t) --b;                                /* last boundary at or before the issue time */
+        p.boundary = b; p.ins.opcode = OP_PREFETCH; p.ins.target = -1; p.ins.time_ns = t;
+        list[m++] = p;
+    }
+    qsort(list, (size_t)m, sizeof(keyed_ins), cmp_keyed);
+    int64_t j = 0;
+    for (int64_t b = 0; b <= K; ++b) {
+        inst_ptr[b] = j;
+        while (j < m && list[j].boundary == b) { if (j < out_cap) out[j] = list[j].ins; ++j; }
+    }
+    inst_ptr[K + 1] = m;
+    free(list);
+    return m;
+}

@@ -24,6 +24,11 @@ MIGRATION_DTYPE = np.dtype([
 ])
 assert MIGRATION_DTYPE.itemsize == 48
 
+INSTRUCTION_DTYPE = np.dtype([("opcode", "<i4"), ("tensor", "<i4"), ("target", "<i4"), ("record", "<i4"),
+                              ("bytes", "<i8"), ("time_ns", "<i8")])
+assert INSTRUCTION_DTYPE.itemsize == 32
+OPCODES = {0: "g10_free", 1: "g10_pre_evict", 2: "g10_alloc", 3: "g10_prefetch"}
+
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 
 
@@ -143,3 +148,19 @@ def schedule_prefetch(K, migrations, start, tensor_bytes, gpu_capacity_bytes, pr
                                  _p(P), _p(order), _p(nal), _p(nis), _p(summary))
     return SimpleNamespace(pressure=P, order=order[:n].copy(), new_absent_last=nal[:n].copy(),
                            new_prefetch_issue_ns=nis[:n].copy(), summary=summary)
+
+
+def emit_instructions(K, first_use, last_use, tensor_bytes, tensor_global, start, migrations, new_issue_ns=None):
+    """Section 4.4 code instrumentation: the alloc / free / pre-evict / prefetch stream by kernel boundary."""
+    f = _c(first_use, np.int32); l = _c(last_use, np.int32); tb = _c(tensor_bytes, np.int64)
+    tg = _c(tensor_global, np.uint8) if tensor_global is not None else None
+    st = _c(start, np.int64); mig = np.ascontiguousarray(migrations)
+    ni = _c(new_issue_ns, np.int64) if new_issue_ns is not None else None
+    N, n = f.shape[0], mig.shape[0]
+    cap = 2 * N + 2 * n + 1
+    out = np.zeros(cap, INSTRUCTION_DTYPE)
+    ptr = np.zeros(K + 2, np.int64)
+    lib().g10o_emit_instructions.restype = C.c_int64
+    m = lib().g10o_emit_instructions(C.c_int64(K), C.c_int64(N), _p(f), _p(l), _p(tb), _p(tg), _p(st), C.c_int64(n), _p(mig),
+                                     _p(ni), _p(ptr), _p(out), C.c_int64(cap))
+    return SimpleNamespace(inst_ptr=ptr, instructions=out[:int(m)].copy())

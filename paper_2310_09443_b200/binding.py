@@ -17,14 +17,18 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libg10.so")
 
 MEM_DEVICE, MEM_HOST = 0, 1
-WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY = 0, 1, 2, 3
+WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT = 0, 1, 2, 3, 4
 DEST_SSD, DEST_HOST = 0, 1
 FLAG_RESCORE_ALL = 1
 FLAG_GLOBAL_STATE = 2
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
-           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch")
+           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions")
 STATIC_MAX_KERNELS, STATIC_MAX_TENSORS = 32768, 131072
+
+INSTRUCTION_DTYPE = np.dtype([("opcode", "<i4"), ("tensor", "<i4"), ("target", "<i4"), ("record", "<i4"),
+                              ("bytes", "<i8"), ("time_ns", "<i8")])
+OPCODES = {0: "g10_free", 1: "g10_pre_evict", 2: "g10_alloc", 3: "g10_prefetch"}
 
 MIGRATION_DTYPE = np.dtype([
     ("period", "<i4"), ("tensor", "<i4"), ("dest", "<i4"),
@@ -65,6 +69,10 @@ class _PrefetchOut(C.Structure):
                 ("new_prefetch_issue_ns", C.c_void_p), ("summary", C.c_void_p)]
 
 
+class _EmitOut(C.Structure):
+    _fields_ = [("inst_ptr", C.c_void_p), ("instructions", C.c_void_p), ("instructions_cap", C.c_int64), ("counts", C.c_void_p)]
+
+
 class _Options(C.Structure):
     _fields_ = [("host_capacity_bytes", C.c_uint64), ("max_iterations", C.c_int64), ("flags", C.c_uint32),
                 ("stage_events", C.POINTER(C.c_void_p)), ("num_stage_events", C.c_int32)]
@@ -97,6 +105,10 @@ def load_library():
         lib.g10_schedule_prefetch.restype = C.c_int32
         lib.g10_schedule_prefetch.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
                                               C.POINTER(_PrefetchOut), C.c_void_p]
+        lib.g10_emit_instructions.restype = C.c_int32
+        lib.g10_emit_instructions.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                              C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(_EmitOut), C.c_void_p, C.c_size_t,
+                                              C.c_void_p]
         lib.g10_plan_migrations.restype = C.c_int32
         lib.g10_plan_migrations.argtypes = [C.POINTER(_Trace), C.c_uint64, C.c_uint64, C.c_uint64, C.POINTER(_Options),
                                             C.POINTER(_PlanOut), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -303,6 +315,33 @@ def g10_schedule_prefetch(K, num_migrations, migrations, kernel_start_ns, tensor
     _check(lib.g10_schedule_prefetch(K, n, _ptr(migrations), _ptr(kernel_start_ns), _ptr(tensor_bytes), gpu_capacity_bytes,
                                      C.byref(out), _stream(stream)))
     return r
+
+
+def g10_emit_instructions(K, N, first_use, last_use, tensor_bytes, tensor_global, kernel_start_ns, num_migrations, migrations,
+                          new_prefetch_issue_ns=None, ws=None, stream=None):
+    """Section 4.4 code instrumentation: the alloc / free / pre-evict / prefetch stream by kernel boundary (device tensors).
+    `instructions` is a uint8 tensor of 32-byte records (INSTRUCTION_DTYPE); counts = [number of instructions, status]."""
+    lib = load_library()
+    dev = kernel_start_ns.device
+    n = int(num_migrations)
+    cap = 2 * N + 2 * n
+    r = SimpleNamespace(inst_ptr=torch.empty(K + 2, dtype=torch.int64, device=dev),
+                        instructions=torch.empty(max(cap, 1) * 32, dtype=torch.uint8, device=dev),
+                        counts=torch.empty(2, dtype=torch.int64, device=dev))
+    need = g10_workspace_bytes(WS_EMIT, K, N, n)
+    if ws is None:
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    out = _EmitOut(_ptr(r.inst_ptr), _ptr(r.instructions), cap, _ptr(r.counts))
+    _check(lib.g10_emit_instructions(K, N, _ptr(first_use), _ptr(last_use), _ptr(tensor_bytes), _ptr(tensor_global),
+                                     _ptr(kernel_start_ns), n, _ptr(migrations), _ptr(new_prefetch_issue_ns), C.byref(out),
+                                     _ptr(ws), ws.numel(), _stream(stream)))
+    r.workspace = ws
+    return r
+
+
+def instructions_numpy(em) -> np.ndarray:
+    n = int(em.counts[0].item())
+    return em.instructions[: n * 32].cpu().numpy().view(INSTRUCTION_DTYPE).copy()
 
 
 def migrations_numpy(plan) -> np.ndarray:

@@ -180,6 +180,21 @@ cudaError_t d2h(T *dst, const T *src, size_t count, cudaStream_t s)
     return cudaMemcpyAsync(dst, src, sizeof(T) * count, cudaMemcpyDeviceToHost, s);
 }
 
+size_t carve_emit(void *base, int64_t N, int64_t n, EmitLaunch &L, char **zero_begin, size_t *zero_bytes)
+{
+    Carver c(base);
+    const size_t total = (size_t)(2 * N + 2 * n) + 1;
+    *zero_begin = c.base;
+    L.status = c.take<ull>(1);
+    L.ticket = c.take<unsigned>(1);
+    L.bucket_count = c.take<unsigned>(4096);
+    L.bucket_cursor = c.take<unsigned>(4096);
+    *zero_bytes = align_up(c.off);
+    L.keys = c.take<ull>(total);
+    L.payload = c.take<int32_t>(total);
+    return align_up(c.off);
+}
+
 }  // namespace
 }  // namespace g10
 
@@ -204,11 +219,18 @@ const char *g10_strerror(int32_t code)
 int32_t g10_workspace_bytes(int32_t which, int64_t K, int64_t N, int64_t E, int32_t mem, size_t *out_bytes)
 {
     if (!out_bytes || K < 0 || N < 0 || E < 0) return G10_ERR_ARG;
-    if (which < G10_WS_VITALITY || which > G10_WS_GEOMETRY) return G10_ERR_ARG;
+    if (which < G10_WS_VITALITY || which > G10_WS_EMIT) return G10_ERR_ARG;
     if (mem != G10_MEM_DEVICE && mem != G10_MEM_HOST) return G10_ERR_ARG;
     const int64_t lim = ((int64_t)1 << 31) - 1;
     if (K >= lim || N >= lim || E >= lim) return G10_ERR_LIMIT;
     if (which == G10_WS_GEOMETRY) { *out_bytes = 0; return G10_OK; }
+    if (which == G10_WS_EMIT) {                    // E stands for the number of migrations here
+        EmitLaunch L;
+        char *zb = nullptr;
+        size_t zbytes = 0;
+        *out_bytes = carve_emit(nullptr, N, E, L, &zb, &zbytes);
+        return G10_OK;
+    }
     // one layout serves the three calls (the planner uses all of it; the others a prefix-independent subset)
     Workspace w;
     Sizes z{K, N, E, mem == G10_MEM_HOST};
@@ -312,6 +334,37 @@ int32_t g10_candidate_geometry(int64_t K, int64_t Pn, const int64_t *kernel_star
     if (!out->transfer_ns || !out->absent_first || !out->absent_last) return G10_ERR_ARG;
     CU(launch_geometry(K, Pn, nullptr, kernel_start_ns, tensor_bytes, period_tensor, period_prev_use, period_next_use, host_bw, ssd_bw,
                        Pn, out->transfer_ns, out->absent_first, out->absent_last, (cudaStream_t)stream));
+    return G10_OK;
+}
+
+int32_t g10_emit_instructions(int64_t K, int64_t N, const int32_t *first_use, const int32_t *last_use, const int64_t *tensor_bytes,
+                              const uint8_t *tensor_global, const int64_t *kernel_start_ns, int64_t n, const g10_migration *migrations,
+                              const int64_t *new_prefetch_issue_ns, g10_emit_out *out, void *ws, size_t ws_bytes, void *stream)
+{
+    if (K < 0 || N < 0 || n < 0 || !out || !out->inst_ptr || !out->counts || !kernel_start_ns) return G10_ERR_ARG;
+    const int64_t lim = ((int64_t)1 << 31) - 1;
+    if (K >= lim || N >= lim || n >= lim) return G10_ERR_LIMIT;
+    if (N > 0 && (!first_use || !last_use || !tensor_bytes)) return G10_ERR_ARG;
+    if (n > 0 && !migrations) return G10_ERR_ARG;
+    if (out->instructions_cap < 0 || (out->instructions_cap > 0 && !out->instructions)) return G10_ERR_ARG;
+    int shift = 0, nb = 0;
+    if (!emit_choose_buckets(K, 2 * N + 2 * n, &shift, &nb)) return G10_ERR_LIMIT;
+    EmitLaunch L;
+    char *zb = nullptr;
+    size_t zbytes = 0;
+    const size_t need = carve_emit(nullptr, N, n, L, &zb, &zbytes);
+    if (!ws || ((uintptr_t)ws % kAlign) != 0 || ws_bytes < need) return G10_ERR_WORKSPACE;
+    carve_emit(ws, N, n, L, &zb, &zbytes);
+    cudaStream_t s = (cudaStream_t)stream;
+    CU(cudaMemsetAsync(zb, 0, zbytes, s));
+    L.K = K; L.N = N; L.n = n; L.first_use = first_use; L.last_use = last_use; L.bytes = tensor_bytes; L.glob = tensor_global;
+    L.start = kernel_start_ns; L.mig = migrations; L.new_issue = new_prefetch_issue_ns;
+    L.inst_ptr = out->inst_ptr; L.inst = out->instructions; L.inst_cap = out->instructions_cap; L.counts = out->counts;
+    CU(launch_emit(L, s));
+    Workspace w;
+    std::memset(&w, 0, sizeof(w));
+    w.status = L.status;
+    CU(launch_publish_status(w, out->counts + 1, s));
     return G10_OK;
 }
 

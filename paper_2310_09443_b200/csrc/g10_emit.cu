@@ -1,0 +1,270 @@
+// Code instrumentation (Section 4.4, Figure 9): the stream of g10_alloc / g10_free / g10_pre_evict /
+// g10_prefetch calls, ordered by kernel boundary, then FREE < PRE_EVICT < ALLOC < PREFETCH, then tensor id.
+//
+// Every instruction is one 64-bit key (boundary << 33 | opcode << 31 | tensor; unique) plus the plan record it
+// came from.  The keys are sorted with the same shape as the vitality pass: boundaries are cut into buckets of
+// consecutive boundaries holding a couple of thousand instructions, a histogram sizes the buckets, the keys are
+// scattered into their bucket's slice, and one block per bucket sorts its slice in shared memory (bitonic
+// network), counts the instructions of every boundary for the CSR pointers and writes the records out in order.
+// A bucket too large for shared memory (very many tensors allocated at one boundary) is sorted in global memory.
+#include "g10_device.cuh"
+#include "g10_internal.h"
+
+namespace g10 {
+
+constexpr int kEmitThreads = 512;
+constexpr int kEmitCap = 4096;            // instructions of a bucket sorted in shared memory
+enum { kOpFree = 0, kOpPreEvict = 1, kOpAlloc = 2, kOpPrefetch = 3 };
+
+struct EmitArgs {
+    int64_t K, N, n;
+    const int32_t *first_use, *last_use;
+    const int64_t *bytes;
+    const uint8_t *glob;
+    const int64_t *start;
+    const g10_migration *mig;
+    const int64_t *new_issue;
+    int shift, nb;                        // boundaries per bucket = 1 << shift
+    unsigned *bucket_count, *bucket_cursor;
+    ull *keys;
+    int32_t *payload;
+    unsigned *ticket;
+    ull *status;
+};
+
+// item -> (boundary, opcode, tensor, record); false if the item does not exist
+__device__ __forceinline__ bool emit_item(const EmitArgs &A, int64_t item, int64_t *boundary, int *opcode, int *tensor, int *record)
+{
+    *record = -1;
+    if (item < 2 * A.N) {
+        const int64_t i = item < A.N ? item : item - A.N;
+        const int f = A.first_use[i];
+        if (f < 0) return false;
+        const bool g = A.glob != nullptr && A.glob[i] != 0;
+        *tensor = (int)i;
+        if (item < A.N) { *opcode = kOpAlloc; *boundary = g ? 0 : f; return true; }
+        if (g) return false;
+        *opcode = kOpFree; *boundary = (int64_t)A.last_use[i] + 1;
+        return true;
+    }
+    const int64_t r = item - 2 * A.N < A.n ? item - 2 * A.N : item - 2 * A.N - A.n;
+    const bool evict = item - 2 * A.N < A.n;
+    *record = (int)r; *tensor = A.mig[r].tensor;
+    const int64_t t = evict ? A.mig[r].evict_issue_ns : (A.new_issue ? A.new_issue[r] : A.mig[r].prefetch_issue_ns);
+    // last boundary b in [0, K] with start[b] <= t (for a pre-eviction start[b] == t_r exactly)
+    int lo = 0, hi = (int)A.K;
+    while (lo < hi) { const int mid = lo + (hi - lo + 1) / 2; if (A.start[mid] <= t) lo = mid; else hi = mid - 1; }
+    *boundary = lo; *opcode = evict ? kOpPreEvict : kOpPrefetch;
+    return true;
+}
+
+__device__ __forceinline__ ull emit_key(int64_t boundary, int opcode, int tensor)
+{
+    return ((ull)boundary << 33) | ((ull)opcode << 31) | (ull)(unsigned)tensor;
+}
+
+__global__ void __launch_bounds__(kEmitThreads) k_emit_hist(EmitArgs A)
+{
+    extern __shared__ unsigned s_hist[];
+    for (int b = threadIdx.x; b < A.nb; b += kEmitThreads) s_hist[b] = 0;
+    __syncthreads();
+    const int64_t total = 2 * A.N + 2 * A.n;
+    for (int64_t item = (int64_t)blockIdx.x * kEmitThreads + threadIdx.x; item < total; item += (int64_t)gridDim.x * kEmitThreads) {
+        int64_t bd; int op, tn, rc;
+        if (emit_item(A, item, &bd, &op, &tn, &rc)) atomicAdd(&s_hist[bd >> A.shift], 1u);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < A.nb; b += kEmitThreads)
+        if (s_hist[b]) atomicAdd(&A.bucket_count[b], s_hist[b]);
+}
+
+// exclusive scan of the bucket counts (nb <= 4096) into s_base[0..nb]
+__device__ __forceinline__ void emit_scan_buckets(const unsigned *cnt, int nb, long long *s_base, long long *s_w)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    long long carry = 0;
+    for (int base = 0; base < nb; base += kEmitThreads) {
+        const int j = base + threadIdx.x;
+        const long long v = j < nb ? (long long)cnt[j] : 0;
+        const long long incl = warp_inclusive_scan_i64(v, lane);
+        __syncthreads();
+        if (lane == 31) s_w[warp] = incl;
+        __syncthreads();
+        long long wpre = 0, tot = 0;
+        for (int w = 0; w < kEmitThreads / 32; ++w) { const long long x = s_w[w]; if (w < warp) wpre += x; tot += x; }
+        if (j < nb) s_base[j] = carry + wpre + incl - v;
+        carry += tot;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) s_base[nb] = carry;
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kEmitThreads) k_emit_scatter(EmitArgs A)
+{
+    extern __shared__ long long s_base[];            // [nb + 1]
+    __shared__ long long s_w[kEmitThreads / 32];
+    emit_scan_buckets(A.bucket_count, A.nb, s_base, s_w);
+    const int64_t total = 2 * A.N + 2 * A.n;
+    for (int64_t item = (int64_t)blockIdx.x * kEmitThreads + threadIdx.x; item < total; item += (int64_t)gridDim.x * kEmitThreads) {
+        int64_t bd; int op, tn, rc;
+        if (emit_item(A, item, &bd, &op, &tn, &rc)) {
+            const int b = (int)(bd >> A.shift);
+            const long long pos = s_base[b] + atomicAdd(&A.bucket_cursor[b], 1u);
+            A.keys[pos] = emit_key(bd, op, tn);
+            A.payload[pos] = rc;
+        }
+    }
+}
+
+// bitonic network over (key, payload) pairs; arbitrary n (values only ever move up)
+__device__ void emit_bitonic(ull *k, int32_t *p, int n)
+{
+    int n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    for (int kk = 2; kk <= n2; kk <<= 1) {
+        for (int j = kk >> 1, lj = 31 - __clz(kk >> 1); j > 0; j >>= 1, --lj) {
+            const bool mirror = (j == (kk >> 1));
+            for (int t = threadIdx.x; t < n2 / 2; t += blockDim.x) {
+                const int blk = t >> lj, off = t & (j - 1);
+                const int i = blk * 2 * j + off;
+                const int q = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
+                if (q < n) {
+                    const ull x = k[i], y = k[q];
+                    if (x > y) { k[i] = y; k[q] = x; const int32_t px = p[i]; p[i] = p[q]; p[q] = px; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kEmitThreads) k_emit_write(EmitArgs A, int64_t *inst_ptr, g10_instruction *inst, int64_t inst_cap, int64_t *counts)
+{
+    extern __shared__ long long s_dyn[];
+    long long *s_base = s_dyn;                                   // [nb + 1]
+    int *s_cnt = (int *)(s_base + A.nb + 1);                     // [bw + 1] instructions per boundary of the bucket
+    ull *s_keys = (ull *)(((uintptr_t)(s_cnt + (1 << A.shift) + 1) + 7) & ~(uintptr_t)7);   // [kEmitCap]
+    int32_t *s_pay = (int32_t *)(s_keys + kEmitCap);              // [kEmitCap]
+    __shared__ long long s_w[kEmitThreads / 32];
+    __shared__ int s_bucket;
+    const int bw = 1 << A.shift;
+    emit_scan_buckets(A.bucket_count, A.nb, s_base, s_w);
+    for (;;) {
+        __syncthreads();
+        if (threadIdx.x == 0) s_bucket = (int)atomicAdd(A.ticket, 1u);
+        __syncthreads();
+        const int b = s_bucket;
+        if (b >= A.nb) break;
+        const long long base = s_base[b];
+        const int n = (int)(s_base[b + 1] - base);
+        ull *gk = A.keys + base;
+        int32_t *gp = A.payload + base;
+        const ull *kp; const int32_t *pp;
+        if (n <= kEmitCap) {
+            for (int j = threadIdx.x; j < n; j += kEmitThreads) { s_keys[j] = gk[j]; s_pay[j] = gp[j]; }
+            __syncthreads();
+            emit_bitonic(s_keys, s_pay, n);
+            kp = s_keys; pp = s_pay;
+        } else {
+            __syncthreads();
+            emit_bitonic(gk, gp, n);
+            kp = gk; pp = gp;
+        }
+        // instructions per boundary -> CSR pointers of the bucket's boundaries
+        const int64_t b0 = (int64_t)b << A.shift;
+        const int bw_eff = (int)((A.K + 1 - b0) < bw ? (A.K + 1 - b0) : bw);
+        for (int j = threadIdx.x; j <= bw_eff; j += kEmitThreads) s_cnt[j] = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < n; j += kEmitThreads) atomicAdd(&s_cnt[(int)((kp[j] >> 33) - b0)], 1);
+        __syncthreads();
+        {   // in-place exclusive scan of s_cnt[0..bw_eff)
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            int carry = 0;
+            for (int c0 = 0; c0 < bw_eff; c0 += kEmitThreads) {
+                const int j = c0 + threadIdx.x;
+                const int v = j < bw_eff ? s_cnt[j] : 0;
+                int incl = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+                __syncthreads();
+                if (lane == 31) s_w[warp] = incl;
+                __syncthreads();
+                int wpre = 0, tot = 0;
+                for (int w = 0; w < kEmitThreads / 32; ++w) { const int x = (int)s_w[w]; if (w < warp) wpre += x; tot += x; }
+                if (j < bw_eff) s_cnt[j] = carry + wpre + incl - v;
+                carry += tot;
+            }
+            __syncthreads();
+        }
+        for (int j = threadIdx.x; j < bw_eff; j += kEmitThreads) inst_ptr[b0 + j] = base + s_cnt[j];
+        if (b == A.nb - 1 && threadIdx.x == 0) {
+            inst_ptr[A.K + 1] = s_base[A.nb];
+            counts[0] = s_base[A.nb];
+            if (s_base[A.nb] > inst_cap) raise_status(A.status, G10_DEV_PLAN_OVERFLOW);
+        }
+        // the records, in order
+        for (int j = threadIdx.x; j < n; j += kEmitThreads) {
+            const long long pos = base + j;
+            if (pos >= inst_cap) continue;
+            const ull key = kp[j];
+            const int64_t boundary = (int64_t)(key >> 33);
+            g10_instruction ins;
+            ins.opcode = (int)((key >> 31) & 3u); ins.tensor = (int)(key & 0x7fffffffu); ins.record = pp[j]; ins.target = -1;
+            ins.bytes = A.bytes[ins.tensor];
+            ins.time_ns = A.start[boundary];
+            if (ins.opcode == kOpPreEvict) { ins.target = A.mig[ins.record].dest; ins.time_ns = A.mig[ins.record].evict_issue_ns; }
+            if (ins.opcode == kOpPrefetch)
+                ins.time_ns = A.new_issue ? A.new_issue[ins.record] : A.mig[ins.record].prefetch_issue_ns;
+            inst[pos] = ins;
+        }
+    }
+}
+
+bool emit_choose_buckets(int64_t K, int64_t total_items, int *shift, int *nb)
+{
+    // boundaries per bucket so that a bucket holds about 2000 instructions; at most 4096 buckets of 4096 boundaries
+    const int64_t B = K + 1;
+    int64_t want = total_items > 0 ? (2000 * B) / total_items : 4096;
+    int s = 0;
+    while (s < 12 && ((int64_t)1 << (s + 1)) <= want) ++s;
+    while (s < 12 && ((B + ((int64_t)1 << s) - 1) >> s) > 4096) ++s;
+    const int64_t buckets = (B + ((int64_t)1 << s) - 1) >> s;
+    if (buckets > 4096) return false;
+    *shift = s; *nb = (int)buckets;
+    return true;
+}
+
+cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s)
+{
+    EmitArgs A;
+    A.K = L.K; A.N = L.N; A.n = L.n;
+    A.first_use = L.first_use; A.last_use = L.last_use; A.bytes = L.bytes; A.glob = L.glob; A.start = L.start;
+    A.mig = L.mig; A.new_issue = L.new_issue;
+    if (!emit_choose_buckets(L.K, 2 * L.N + 2 * L.n, &A.shift, &A.nb)) return cudaErrorInvalidValue;
+    A.bucket_count = L.bucket_count; A.bucket_cursor = L.bucket_cursor; A.keys = L.keys; A.payload = L.payload;
+    A.ticket = L.ticket; A.status = L.status;
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+            sms = 0;
+            return cudaErrorInvalidDevice;
+        }
+    }
+    const int64_t total = 2 * L.N + 2 * L.n;
+    int64_t g = (total + kEmitThreads - 1) / kEmitThreads;
+    if (g > 4 * (int64_t)sms) g = 4 * (int64_t)sms;
+    if (g < 1) g = 1;
+    k_emit_hist<<<(int)g, kEmitThreads, sizeof(unsigned) * (size_t)A.nb, s>>>(A);
+    k_emit_scatter<<<(int)g, kEmitThreads, sizeof(long long) * (size_t)(A.nb + 1), s>>>(A);
+    const size_t sm3 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(int) * (size_t)((1 << A.shift) + 2) + 8 +
+                       (sizeof(ull) + sizeof(int32_t)) * kEmitCap;
+    cudaError_t e = cudaFuncSetAttribute(k_emit_write, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
+    if (e != cudaSuccess) return e;
+    const int g3 = A.nb < 2 * sms ? A.nb : 2 * sms;
+    k_emit_write<<<g3, kEmitThreads, sm3, s>>>(A, L.inst_ptr, L.inst, L.inst_cap, L.counts);
+    return cudaGetLastError();
+}
+
+}  // namespace g10

@@ -138,6 +138,26 @@ cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, 
 cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *mig, const int64_t *start, const int64_t *bytes,
                                      uint64_t gpu_capacity_bytes, int64_t *P, int32_t *order, int32_t *new_last, int64_t *new_issue,
                                      int64_t *summary, cudaStream_t s);
+// instruction-stream emission (g10_emit.cu)
+struct EmitLaunch {
+    int64_t K, N, n;
+    const int32_t *first_use, *last_use;
+    const int64_t *bytes;
+    const uint8_t *glob;
+    const int64_t *start;
+    const g10_migration *mig;
+    const int64_t *new_issue;
+    unsigned *bucket_count, *bucket_cursor, *ticket;
+    ull *keys;
+    int32_t *payload;
+    ull *status;
+    int64_t *inst_ptr;
+    g10_instruction *inst;
+    int64_t inst_cap;
+    int64_t *counts;
+};
+bool emit_choose_buckets(int64_t K, int64_t total_items, int *shift, int *nb);
+cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s);
 // planner (g10_planner.cu)
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
 int plan_loop_max_blocks();

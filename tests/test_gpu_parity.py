@@ -326,3 +326,58 @@ def test_prefetch_pass(gpu, oracle):
     start, P0, peak, slot = oracle.timeline(tr)
     check_prefetch(gpu, oracle, tr, tr.capacity_from_peak(peak))
     check_prefetch(gpu, oracle, tr, peak * 8 // 10)
+
+
+def check_emit(gpu, oracle, tr, cap, eager):
+    """Instruction stream (Section 4.4, Figure 9) from the GPU's own vitality + plan (+ eager prefetch pass)."""
+    import torch
+    tb = gpu.upload(tr)
+    v = gpu.g10_vitality(tb)
+    tl = gpu.g10_pressure_timeline(tb)
+    plan = gpu.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    n = int(plan.summary[0].item())
+    ni = None
+    if eager:
+        pf = gpu.g10_schedule_prefetch(tr.K, n, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap, plan.final_pressure)
+        ni = pf.new_prefetch_issue_ns
+    em = gpu.g10_emit_instructions(tr.K, tr.N, v.first_use, v.last_use, tb.tensor_bytes, tb.tensor_global, tl.kernel_start_ns,
+                                   n, plan.migrations, ni)
+    torch.cuda.synchronize()
+    assert int(em.counts[1].item()) == 0
+    ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+    start = oracle.slot_clock(tr.kernel_ns)
+    ref = oracle.plan(tr, cap, lazy=True)
+    oni = None
+    if eager:
+        oni = oracle.schedule_prefetch(tr.K, ref.migrations, start, tr.tensor_bytes, cap, ref.final_pressure).new_prefetch_issue_ns
+    oe = oracle.emit_instructions(tr.K, ov.first_use, ov.last_use, tr.tensor_bytes, tr.tensor_global, start, ref.migrations, oni)
+    assert int(em.counts[0].item()) == len(oe.instructions)
+    assert np.array_equal(_np(em.inst_ptr), oe.inst_ptr)
+    got = gpu.instructions_numpy(em)
+    for name in oe.instructions.dtype.names:
+        assert np.array_equal(got[name], oe.instructions[name]), name
+    return len(oe.instructions)
+
+
+def test_instruction_stream(gpu, oracle):
+    import json, os
+    ex = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_worked_examples.json")))["examples"]["A"]
+    tr = traces.from_lists("A", ex["kernel_lists"], ex["tensor_bytes"], ex["kernel_ns"], host_bw=ex["host_bw"], ssd_bw=ex["ssd_bw"])
+    assert check_emit(gpu, oracle, tr, ex["capacity"], False) == len(ex["instruction_stream"]["instructions"])
+    rng = np.random.default_rng(2024)
+    for trial in range(40):
+        toy = traces.random_toy(rng, int(rng.integers(1, 40)), int(rng.integers(1, 30)), max_deg=5)
+        start, P0, peak, slot = oracle.timeline(toy)
+        check_emit(gpu, oracle, toy, peak * int(rng.integers(1, 10)) // 10, bool(trial % 2))
+    for cfg in (0, 1, 2, 3):
+        tr = traces.make_config(cfg)
+        start, P0, peak, slot = oracle.timeline(tr)
+        check_emit(gpu, oracle, tr, tr.capacity_from_peak(peak), cfg % 2 == 0)
+    tr = traces.config4_stress_dag(K=20000, N=80000)
+    start, P0, peak, slot = oracle.timeline(tr)
+    assert check_emit(gpu, oracle, tr, tr.capacity_from_peak(peak), True) > 100000
+    # very many tensors allocated at one boundary: the bucket is sorted in global memory
+    lists = [list(range(6000))] + [[i] for i in range(0, 6000, 7)]
+    big = traces.from_lists("wide", lists, [64] * 6000, [100] * len(lists), [1] * 3000 + [0] * 3000, capacity_bytes=10**9)
+    check_emit(gpu, oracle, big, 10**9, False)
