@@ -604,3 +604,41 @@ int64_t g10o_emit_instructions(int64_t K, int64_t N, const int32_t *first_use, c
     free(list);
     return m;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Workload characterisation (Section 3): the statistics behind the paper's Figures 2-4, on a trace.
+ *   active_bytes[k]   memory of the tensors kernel k uses (inputs and outputs, each once): the "active
+ *                     tensors" of Figure 2; also the working set that must fit while kernel k runs.
+ *   len_hist[b]       number of inactive periods whose length L = start[v] - start[u+1] (ns) has
+ *                     floor(log2 L) = b: the distribution of Figure 3.
+ *   size_len_hist     [41][45] periods by floor(log2 size) x floor(log2 L): the scatter of Figure 4.
+ *   hide[2]           periods long enough to swap the tensor out and back in, 2 t <= L, over the SSD
+ *                     and over the host link (Section 3: most periods can hide the swap latency).
+ * ---------------------------------------------------------------------------------------- */
+static int floor_log2_i64(int64_t x) { int b = 0; while (x > 1) { x >>= 1; ++b; } return b; }
+
+void g10o_characterize(int64_t K, int64_t N, const int64_t *use_ptr, const int32_t *uses, const int64_t *tensor_bytes,
+                       const int64_t *start, int64_t Pn, const int32_t *period_tensor, const int32_t *period_prev_use,
+                       const int32_t *period_next_use, uint64_t host_bw, uint64_t ssd_bw,
+                       int64_t *active_bytes /* [K] */, int64_t *len_hist /* [64] */, int64_t *size_len_hist /* [41*45] */,
+                       int64_t *hide /* [2] */, int64_t *summary /* [2]: max active bytes, its lowest kernel */)
+{
+    for (int64_t k = 0; k < K; ++k) active_bytes[k] = 0;
+    for (int64_t i = 0; i < N; ++i)
+        for (int64_t j = use_ptr[i]; j < use_ptr[i + 1]; ++j) active_bytes[uses[j]] += tensor_bytes[i];
+    for (int b = 0; b < 64; ++b) len_hist[b] = 0;
+    for (int b = 0; b < 41 * 45; ++b) size_len_hist[b] = 0;
+    hide[0] = hide[1] = 0;
+    for (int64_t p = 0; p < Pn; ++p) {
+        int64_t L = start[period_next_use[p]] - start[period_prev_use[p] + 1];
+        int64_t s = tensor_bytes[period_tensor[p]];
+        int bl = floor_log2_i64(L), bs = floor_log2_i64(s);
+        len_hist[bl] += 1;
+        size_len_hist[(bs > 40 ? 40 : bs) * 45 + (bl > 44 ? 44 : bl)] += 1;
+        if (2 * transfer_ns(s, ssd_bw) <= L) hide[0] += 1;
+        if (2 * transfer_ns(s, host_bw) <= L) hide[1] += 1;
+    }
+    int64_t mx = 0, arg = -1;
+    for (int64_t k = 0; k < K; ++k) if (arg < 0 || active_bytes[k] > mx) { mx = active_bytes[k]; arg = k; }
+    summary[0] = mx; summary[1] = arg;
+}

@@ -164,3 +164,15 @@ def emit_instructions(K, first_use, last_use, tensor_bytes, tensor_global, start
     m = lib().g10o_emit_instructions(C.c_int64(K), C.c_int64(N), _p(f), _p(l), _p(tb), _p(tg), _p(st), C.c_int64(n), _p(mig),
                                      _p(ni), _p(ptr), _p(out), C.c_int64(cap))
     return SimpleNamespace(inst_ptr=ptr, instructions=out[:int(m)].copy())
+
+
+def characterize(K, vit, tensor_bytes, start, host_bw, ssd_bw):
+    """Section 3 statistics (Figures 2-4) of a trace from its vitality results."""
+    up = _c(vit.use_ptr, np.int64); us = _c(vit.uses, np.int32); tb = _c(tensor_bytes, np.int64); st = _c(start, np.int64)
+    pt = _c(vit.period_tensor, np.int32); pu = _c(vit.period_prev_use, np.int32); pv = _c(vit.period_next_use, np.int32)
+    active = np.zeros(K, np.int64); lh = np.zeros(64, np.int64); slh = np.zeros(41 * 45, np.int64)
+    hide = np.zeros(2, np.int64); summary = np.zeros(2, np.int64)
+    lib().g10o_characterize(C.c_int64(K), C.c_int64(tb.shape[0]), _p(up), _p(us), _p(tb), _p(st), C.c_int64(pt.shape[0]),
+                            _p(pt), _p(pu), _p(pv), C.c_uint64(host_bw), C.c_uint64(ssd_bw), _p(active), _p(lh), _p(slh),
+                            _p(hide), _p(summary))
+    return SimpleNamespace(active_bytes=active, len_hist=lh, size_len_hist=slh.reshape(41, 45), hide=hide, summary=summary)
