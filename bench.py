@@ -353,6 +353,15 @@ def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=10):
     # the whole plan of the stress trace (capacity = 3/10 of the unplanned peak), once
     tl = binding.g10_pressure_timeline(tb, ws=ws)
     torch.cuda.synchronize()
+    # characterisation statistics (Section 3): reads use_ptr (8N), uses (4E'), tensor_bytes (8N), the periods (12 Pn)
+    # and two clock entries per period (16 Pn), one 8-byte atomic per use (8E') into active_bytes (8K)
+    st_bytes = 8 * N + 4 * e2 + 8 * N + 12 * pn + 16 * pn + 8 * e2 + 8 * K
+    st_s = time_calls(torch, lambda: binding.g10_characterize(K, N, v.use_ptr, v.uses, tb.tensor_bytes, tl.kernel_start_ns, pn,
+                                                              v.period_tensor, v.period_prev_use, v.period_next_use,
+                                                              tr.host_bw, tr.ssd_bw), steps, warm, flush) / steps
+    out["characterize_ms"] = st_s * 1e3
+    out["characterize_roofline"] = {"bound": "hbm", "achieved": st_bytes / st_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                                    "frac": st_bytes / st_s / 1e9 / hbm_peak, "algorithmic_bytes": st_bytes, "peak_kind": peak_kind}
     cap = tr.capacity_from_peak(int(tl.peak_bytes.item()))
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()

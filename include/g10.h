@@ -238,6 +238,28 @@ int32_t g10_emit_instructions(int64_t num_kernels, int64_t num_tensors, const in
                               int64_t num_migrations, const g10_migration *migrations, const int64_t *new_prefetch_issue_ns,
                               g10_emit_out *out, void *ws, size_t ws_bytes, void *stream);
 
+/* Section 3, workload characterisation (the statistics of Figures 2-4) from the results of g10_vitality and the
+   slot clock of g10_pressure_timeline.  active_bytes [K]: bytes of the tensors kernel k uses, each once (the
+   working set that has to fit while k runs).  len_hist [64]: inactive periods by floor(log2 L), L = the period's
+   length in ns.  size_len_hist [41 * 45], row-major: periods by min(floor(log2 size), 40) x min(floor(log2 L), 44).
+   hide [2]: periods with 2 * transfer time <= L for the SSD and for the host link (indexed by G10_DEST_*).
+   summary [2]: max of active_bytes and its lowest kernel (0, -1 for K = 0).  All pointers are DEVICE pointers;
+   use_ptr [N + 1] / uses are the CSR of distinct uses; the call zeroes its outputs itself.  Needs no workspace. */
+#define G10_STATS_LEN_BINS 64
+#define G10_STATS_SIZE_BINS 41
+#define G10_STATS_LEN2_BINS 45
+typedef struct g10_stats_out {
+    int64_t *active_bytes;
+    int64_t *len_hist;
+    int64_t *size_len_hist;
+    int64_t *hide;
+    int64_t *summary;
+} g10_stats_out;
+int32_t g10_characterize(int64_t num_kernels, int64_t num_tensors, const int64_t *use_ptr, const int32_t *uses,
+                         const int64_t *tensor_bytes, const int64_t *kernel_start_ns, int64_t num_periods,
+                         const int32_t *period_tensor, const int32_t *period_prev_use, const int32_t *period_next_use,
+                         uint64_t host_bw, uint64_t ssd_bw, g10_stats_out *out, void *stream);
+
 /* The paper has no counterpart for this entry point: it is g10_pressure_timeline for callers that cannot
    allocate device memory when they need a timeline (a host whose device memory is wholly owned by its own
    pool, or a code path where cudaMalloc / cudaFree are ruled out because they may synchronise the device).

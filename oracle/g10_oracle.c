@@ -635,8 +635,8 @@ void g10o_characterize(int64_t K, int64_t N, const int64_t *use_ptr, const int32
         int bl = floor_log2_i64(L), bs = floor_log2_i64(s);
         len_hist[bl] += 1;
         size_len_hist[(bs > 40 ? 40 : bs) * 45 + (bl > 44 ? 44 : bl)] += 1;
-        if (2 * transfer_ns(s, ssd_bw) <= L) hide[0] += 1;
-        if (2 * transfer_ns(s, host_bw) <= L) hide[1] += 1;
+        if (transfer_ns(s, ssd_bw) <= L / 2) hide[0] += 1;     /* 2 t <= L without overflow */
+        if (transfer_ns(s, host_bw) <= L / 2) hide[1] += 1;
     }
     int64_t mx = 0, arg = -1;
     for (int64_t k = 0; k < K; ++k) if (arg < 0 || active_bytes[k] > mx) { mx = active_bytes[k]; arg = k; }

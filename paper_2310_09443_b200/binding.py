@@ -23,7 +23,7 @@ FLAG_RESCORE_ALL = 1
 FLAG_GLOBAL_STATE = 2
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
-           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions")
+           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize")
 STATIC_MAX_KERNELS, STATIC_MAX_TENSORS = 32768, 131072
 
 INSTRUCTION_DTYPE = np.dtype([("opcode", "<i4"), ("tensor", "<i4"), ("target", "<i4"), ("record", "<i4"),
@@ -69,6 +69,11 @@ class _PrefetchOut(C.Structure):
                 ("new_prefetch_issue_ns", C.c_void_p), ("summary", C.c_void_p)]
 
 
+class _StatsOut(C.Structure):
+    _fields_ = [("active_bytes", C.c_void_p), ("len_hist", C.c_void_p), ("size_len_hist", C.c_void_p), ("hide", C.c_void_p),
+                ("summary", C.c_void_p)]
+
+
 class _EmitOut(C.Structure):
     _fields_ = [("inst_ptr", C.c_void_p), ("instructions", C.c_void_p), ("instructions_cap", C.c_int64), ("counts", C.c_void_p)]
 
@@ -109,6 +114,9 @@ def load_library():
         lib.g10_emit_instructions.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                               C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(_EmitOut), C.c_void_p, C.c_size_t,
                                               C.c_void_p]
+        lib.g10_characterize.restype = C.c_int32
+        lib.g10_characterize.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.POINTER(_StatsOut), C.c_void_p]
         lib.g10_plan_migrations.restype = C.c_int32
         lib.g10_plan_migrations.argtypes = [C.POINTER(_Trace), C.c_uint64, C.c_uint64, C.c_uint64, C.POINTER(_Options),
                                             C.POINTER(_PlanOut), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -336,6 +344,22 @@ def g10_emit_instructions(K, N, first_use, last_use, tensor_bytes, tensor_global
                                      _ptr(kernel_start_ns), n, _ptr(migrations), _ptr(new_prefetch_issue_ns), C.byref(out),
                                      _ptr(ws), ws.numel(), _stream(stream)))
     r.workspace = ws
+    return r
+
+
+def g10_characterize(K, N, use_ptr, uses, tensor_bytes, kernel_start_ns, num_periods, period_tensor, period_prev_use,
+                     period_next_use, host_bw, ssd_bw, stream=None):
+    """Section 3 statistics (Figures 2-4) from the vitality results and the slot clock (device tensors)."""
+    lib = load_library()
+    dev = kernel_start_ns.device
+    r = SimpleNamespace(active_bytes=torch.empty(max(K, 1), dtype=torch.int64, device=dev),
+                        len_hist=torch.empty(64, dtype=torch.int64, device=dev),
+                        size_len_hist=torch.empty(41 * 45, dtype=torch.int64, device=dev),
+                        hide=torch.empty(2, dtype=torch.int64, device=dev), summary=torch.empty(2, dtype=torch.int64, device=dev))
+    out = _StatsOut(_ptr(r.active_bytes), _ptr(r.len_hist), _ptr(r.size_len_hist), _ptr(r.hide), _ptr(r.summary))
+    _check(lib.g10_characterize(K, N, _ptr(use_ptr), _ptr(uses), _ptr(tensor_bytes), _ptr(kernel_start_ns), int(num_periods),
+                                _ptr(period_tensor), _ptr(period_prev_use), _ptr(period_next_use), host_bw, ssd_bw, C.byref(out),
+                                _stream(stream)))
     return r
 
 

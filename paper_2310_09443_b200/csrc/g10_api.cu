@@ -368,6 +368,22 @@ int32_t g10_emit_instructions(int64_t K, int64_t N, const int32_t *first_use, co
     return G10_OK;
 }
 
+int32_t g10_characterize(int64_t K, int64_t N, const int64_t *use_ptr, const int32_t *uses, const int64_t *tensor_bytes,
+                         const int64_t *kernel_start_ns, int64_t Pn, const int32_t *period_tensor, const int32_t *period_prev_use,
+                         const int32_t *period_next_use, uint64_t host_bw, uint64_t ssd_bw, g10_stats_out *out, void *stream)
+{
+    if (K < 0 || N < 0 || Pn < 0 || host_bw == 0 || ssd_bw == 0 || !out) return G10_ERR_ARG;
+    const int64_t lim = ((int64_t)1 << 31) - 1;
+    if (K >= lim || N >= lim || Pn >= lim) return G10_ERR_LIMIT;
+    if (!out->len_hist || !out->size_len_hist || !out->hide || !out->summary || (K > 0 && !out->active_bytes)) return G10_ERR_ARG;
+    if (N > 0 && (!use_ptr || !tensor_bytes)) return G10_ERR_ARG;
+    if (Pn > 0 && (!kernel_start_ns || !tensor_bytes || !period_tensor || !period_prev_use || !period_next_use)) return G10_ERR_ARG;
+    CU(launch_characterize(K, N, use_ptr, uses, tensor_bytes, kernel_start_ns, Pn, period_tensor, period_prev_use, period_next_use,
+                           host_bw, ssd_bw, out->active_bytes, out->len_hist, out->size_len_hist, out->hide, out->summary,
+                           (cudaStream_t)stream));
+    return G10_OK;
+}
+
 int32_t g10_schedule_prefetch(int64_t K, int64_t n, const g10_migration *migrations, const int64_t *kernel_start_ns,
                               const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes, g10_prefetch_out *out, void *stream)
 {

@@ -158,6 +158,9 @@ struct EmitLaunch {
 };
 bool emit_choose_buckets(int64_t K, int64_t total_items, int *shift, int *nb);
 cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s);
+cudaError_t launch_characterize(int64_t K, int64_t N, const int64_t *use_ptr, const int32_t *uses, const int64_t *bytes, const int64_t *start,
+                                int64_t Pn, const int32_t *per_t, const int32_t *per_u, const int32_t *per_v, uint64_t host_bw, uint64_t ssd_bw,
+                                int64_t *active, int64_t *len_hist, int64_t *size_len_hist, int64_t *hide, int64_t *summary, cudaStream_t s);
 // planner (g10_planner.cu)
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
 int plan_loop_max_blocks();

@@ -381,3 +381,41 @@ def test_instruction_stream(gpu, oracle):
     lists = [list(range(6000))] + [[i] for i in range(0, 6000, 7)]
     big = traces.from_lists("wide", lists, [64] * 6000, [100] * len(lists), [1] * 3000 + [0] * 3000, capacity_bytes=10**9)
     check_emit(gpu, oracle, big, 10**9, False)
+
+
+def check_stats(gpu, oracle, tr):
+    """Characterisation statistics (Section 3, Figures 2-4) from the GPU's own vitality + slot clock."""
+    import torch
+    tb = gpu.upload(tr)
+    v = gpu.g10_vitality(tb)
+    tl = gpu.g10_pressure_timeline(tb)
+    torch.cuda.synchronize()
+    Pn = int(v.counts[1].item())
+    st = gpu.g10_characterize(tr.K, tr.N, v.use_ptr, v.uses, tb.tensor_bytes, tl.kernel_start_ns, Pn, v.period_tensor,
+                              v.period_prev_use, v.period_next_use, tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+    oc = oracle.characterize(tr.K, ov, tr.tensor_bytes, oracle.slot_clock(tr.kernel_ns), tr.host_bw, tr.ssd_bw)
+    assert np.array_equal(_np(st.active_bytes)[:tr.K], oc.active_bytes)
+    assert np.array_equal(_np(st.len_hist), oc.len_hist)
+    assert np.array_equal(_np(st.size_len_hist).reshape(41, 45), oc.size_len_hist)
+    assert np.array_equal(_np(st.hide), oc.hide)
+    assert np.array_equal(_np(st.summary), oc.summary)
+    return int(oc.len_hist.sum())
+
+
+@pytest.mark.gpu
+def test_characterisation_statistics(gpu, oracle):
+    rng = np.random.default_rng(77)
+    for trial in range(40):
+        check_stats(gpu, oracle, traces.random_toy(rng, int(rng.integers(1, 40)), int(rng.integers(1, 30)), max_deg=5))
+    for cfg in (0, 1, 2, 3):
+        check_stats(gpu, oracle, traces.make_config(cfg))
+    assert check_stats(gpu, oracle, traces.config4_stress_dag(K=200000, N=800000)) > 100000
+    # one tensor used by thousands of kernels (the warp shares its use list); sizes and lengths at the histogram edges
+    lists = [[0, 1 + (k % 5)] for k in range(5000)]
+    tr = traces.from_lists("hot", lists, [1 << 44, 1, 2, 3, 1 << 41, 1 << 40], [((1 << 44) - 1) if k % 3 else 1 for k in range(5000)],
+                           [1, 0, 0, 0, 0, 0], capacity_bytes=1 << 50)
+    check_stats(gpu, oracle, tr)
+    # empty trace
+    check_stats(gpu, oracle, traces.from_lists("empty", [], [], [], [], capacity_bytes=1))
