@@ -157,6 +157,9 @@ typedef struct g10_options {
 #define G10_FLAG_GLOBAL_STATE 0x2   /* keep the planner state in global memory even when the timeline would fit
                                        in shared memory (the path large traces take); same plan              */
 
+#define G10_FLAG_MULTI_BLOCK 0x4    /* never let a single block run the greedy loop out of its shared memory (the path
+                                       the smallest traces take); same plan                                  */
+
 #define G10_WS_VITALITY 0
 #define G10_WS_TIMELINE 1
 #define G10_WS_PLAN 2

@@ -21,6 +21,7 @@ WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT = 0, 1, 2, 3, 4
 DEST_SSD, DEST_HOST = 0, 1
 FLAG_RESCORE_ALL = 1
 FLAG_GLOBAL_STATE = 2
+FLAG_MULTI_BLOCK = 4
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
            "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize")

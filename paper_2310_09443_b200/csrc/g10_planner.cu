@@ -119,6 +119,8 @@ int plan_lazy_blocks();
 cudaError_t launch_plan_small(const PlanArgs &A, const Workspace &w, int G, int cand_cap, size_t smem, cudaStream_t s);
 int plan_small_blocks();
 bool plan_small_fits(int64_t K, int64_t E, int G, int *cand_cap_out, size_t *smem_out);
+bool plan_one_possible(int64_t K, int64_t E, bool host_cap);
+cudaError_t launch_plan_one(const PlanArgs &A, const Workspace &w, cudaStream_t s);
 
 bool plan_keeps_state_on_chip(int64_t K, int64_t E, uint32_t flags)
 {
@@ -145,7 +147,15 @@ cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const Pla
         if (Gs > kSmallMaxBlocks) Gs = kSmallMaxBlocks;
         int cand_cap = 0;
         size_t smem = 0;
-        if (Gs >= 1 && plan_small_fits(t.K, t.E, Gs, &cand_cap, &smem)) return launch_plan_small(A, w, Gs, cand_cap, smem, s);
+        if (Gs >= 1 && plan_small_fits(t.K, t.E, Gs, &cand_cap, &smem)) {
+            // one block does the whole loop when the device finds that everything fits its shared memory; the
+            // multi-block planner queued behind it returns at once in that case and does the work otherwise
+            if (!(p.flags & G10_FLAG_MULTI_BLOCK) && plan_one_possible(t.K, t.E, p.host_capacity_bytes != 0)) {
+                const cudaError_t e = launch_plan_one(A, w, s);
+                if (e != cudaSuccess) return e;
+            }
+            return launch_plan_small(A, w, Gs, cand_cap, smem, s);
+        }
     }
     const int G = plan_lazy_blocks();
     if (G < 1) return cudaErrorLaunchFailure;

@@ -1,0 +1,563 @@
+// Algorithm 1 for traces small enough for ONE block to hold everything in shared memory: pressure, slot clock,
+// channel bookings (and host occupancy), and per period its cached score, exact benefit, size, transfer time,
+// slot ranges and state.  With the whole state on one SM an iteration needs no exchange between SMs; what is
+// left is the lazy evaluation itself, arranged so that few warps have to issue instructions at any time:
+//   - the rounded scores (positive doubles, compared as 64-bit integers) sit under a two-level maximum: one
+//     entry per group of 32 periods, refreshed only when a score of the group changed, and a scan of the group
+//     entries by one warp;
+//   - the top entry is the winner if its score is FRESH (exact for the current state); a STALE score is an
+//     upper bound (pressure only falls), so a stale top is rescored by the whole block and the search repeats;
+//   - scores within 1e-10 of a fresh top are settled exactly (128-bit cross products, lowest index on ties),
+//     after any stale one among them has been rescored;
+//   - the winner is applied: pressure range, channel bookings, and every live period is reclassified against
+//     the winner's slot ranges (STALE if the absent ranges meet, DIRTY if transfer windows on the same device
+//     meet); DIRTY periods have their destination re-examined before the next search, one warp per period,
+//     and are rescored only if the destination changed.
+// The kernel decides by itself, from the number of periods found on the device, whether the trace fits; if it
+// does not, it leaves `done` at zero and the multi-block planner launched right behind it does the work.
+#include <cstdio>
+
+#include "g10_planner.cuh"
+
+namespace g10 {
+
+#ifndef G10_ONE_THREADS
+#define G10_ONE_THREADS 512
+#endif
+constexpr int kOneThreads = G10_ONE_THREADS;
+constexpr int kOneWarps = kOneThreads / 32;
+constexpr int kOneMaxFin = 64;
+constexpr int kOneDirtyCap = 256;            // DIRTY periods of one commit that are listed (more: full sweep)
+enum { kFreshO = 1 << 2, kStaleO = 2 << 2, kStateMaskO = 3 << 2, kDirtyO = 0x10 };
+
+struct OneArgs {
+    unsigned *done;          // set to 1 when this kernel produced the plan
+    int smem_bytes;          // dynamic shared memory the launch provides
+};
+
+struct __align__(8) OneRanges { unsigned short a, b, ap, bp; };   // inactive slots [a, b], absent [ap, bp] (current destination)
+
+// A DIRTY period with the geometry of both destinations, fetched from global memory by the thread that found it
+struct __align__(16) OneDirty {
+    int li;
+    int ap[2], bp[2];
+    int pad[3];
+    long long t[2];
+};
+
+__device__ __forceinline__ bool window_free_one(const int64_t *sStart, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane)
+{
+    bool ok = true;
+#pragma unroll 1
+    for (int k = k0 + lane; k <= k1; k += 32) {
+        const int64_t s0 = sStart[k], s1 = sStart[k + 1];
+        const int64_t lo = w0 > s0 ? w0 : s0, hi = w1 < s1 ? w1 : s1;
+        const int64_t ov = hi > lo ? hi - lo : 0;
+        if (busy[k] + ov > s1 - s0) ok = false;
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
+// A window [w0, w1) over slots wk0..wk1 was just booked on a channel (`busy` already includes it).  Can another
+// window [q0, q1) over slots qk0..qk1, admissible before, still be booked on it?  Only slots of both windows matter.
+// A slot strictly inside the new booking is full (it took the slot's whole duration), and every slot of q's range
+// needs time; so q survives only if the ranges meet in the booking's first / last slot alone and the sums still fit.
+__device__ __forceinline__ bool window_conflict(const int64_t *sStart, const int64_t *busy, int wk0, int wk1, int64_t q0, int64_t q1,
+                                                int qk0, int qk1)
+{
+    const int i0 = qk0 > wk0 ? qk0 : wk0, i1 = qk1 < wk1 ? qk1 : wk1;
+    if (i0 > i1) return false;
+    if ((i0 > wk0 + 1 ? i0 : wk0 + 1) <= (i1 < wk1 - 1 ? i1 : wk1 - 1)) return true;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int k = e == 0 ? i0 : i1;
+        if (e == 1 && i1 == i0) break;
+        const int64_t s0 = sStart[k], s1 = sStart[k + 1];
+        const int64_t lo = q0 > s0 ? q0 : s0, hi = q1 < s1 ? q1 : s1;
+        const int64_t ov = hi > lo ? hi - lo : 0;
+        if (busy[k] + ov > s1 - s0) return true;
+    }
+    return false;
+}
+
+__host__ __device__ inline size_t one_smem_need(int64_t K, int64_t Pn, bool host_cap)
+{
+    const int64_t groups = (Pn + 31) / 32;
+    return (size_t)(2 * K + 1) * 8 + (size_t)4 * K * 8 + (host_cap ? (size_t)K * 8 : 0) + (size_t)groups * 32 * 8 + (size_t)Pn * 41 +
+           (size_t)groups * 13 + 128;
+}
+
+// Warp-wide maximum of 64-bit keys with the lowest index among equal keys; same result in every lane.
+__device__ __forceinline__ void warp_argmax_u64(ull k, int idx, ull *mk, int *mi)
+{
+    const unsigned hi = (unsigned)(k >> 32);
+    const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
+    const unsigned lo = hi == mh ? (unsigned)k : 0u;
+    const unsigned ml = __reduce_max_sync(0xffffffffu, lo);
+    const bool top = hi == mh && (unsigned)k == ml;
+    *mk = ((ull)mh << 32) | ml;
+    *mi = (int)__reduce_min_sync(0xffffffffu, top ? (unsigned)idx : 0x7fffffffu);
+}
+
+// Developer aid (off in the library build): with -DG10_PHASE_CLOCKS thread 0 accumulates the cycles between the
+// marked points of an iteration and prints the averages when the loop ends.
+#ifdef G10_PHASE_CLOCKS
+#define ONE_COUNT(i) do { if ((threadIdx.x & 31) == 0) atomicAdd(&s_dbg[i], 1); } while (0)
+#define ONE_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
+                           ph_acc[i] += now_ - ph_last; ph_last = now_; ph_cnt[i] += 1; asm volatile("" ::: "memory"); } } while (0)
+#else
+#define ONE_CLOCK(i)
+#define ONE_COUNT(i)
+#endif
+
+__global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs O)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ ull s_part[2 * kOneWarps];
+    __shared__ int s_fin[kOneMaxFin];
+#ifdef G10_PHASE_CLOCKS
+    __shared__ int s_dbg[4];
+    if (threadIdx.x < 4) s_dbg[threadIdx.x] = 0;
+#endif
+    __shared__ OneDirty s_dirty[kOneDirtyCap];
+    __shared__ int s_n_over, s_ndirty, s_nlist, s_nfin, s_force, s_win, s_top, s_flagged;
+    __shared__ ull s_topkey;
+    __shared__ long long s_pk[kOneWarps];
+    __shared__ int s_ps[kOneWarps];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = (int)A.K;
+    const int64_t Pn64 = *A.Pn_dev < A.geo_stride ? *A.Pn_dev : A.geo_stride;
+    const bool host_cap = A.host_capacity != 0;
+    if (A.K > 65000 || Pn64 > 0x7fffffff || one_smem_need(A.K, Pn64, host_cap) > (size_t)O.smem_bytes) return;
+    const int Pn = (int)Pn64;
+    const int G1 = (Pn + 31) / 32;
+    const int64_t limit = (A.max_iterations <= 0 || A.max_iterations > Pn64) ? Pn64 : A.max_iterations;
+
+    int64_t *sP = (int64_t *)smem_raw;
+    int64_t *sStart = sP + K;
+    int64_t *sBusy = sStart + K + 1;                    // [4][K]
+    int64_t *sHocc = sBusy + (size_t)4 * K;             // [K] if host_cap
+    ull *ckey = (ull *)(sHocc + (host_cap ? K : 0));    // [G1 * 32] bits of the rounded score (0 = none)
+    ull *gkey = ckey + (size_t)G1 * 32;                 // [G1] maximum of each group
+    int64_t *cbytes = (int64_t *)(gkey + G1);
+    int64_t *ct = cbytes + Pn;                          // transfer time of the current destination
+    ull *cben_lo = (ull *)(ct + Pn);
+    ull *cben_hi = cben_lo + Pn;
+    OneRanges *crng = (OneRanges *)(cben_hi + Pn);
+    int *garg = (int *)(crng + Pn);                     // [G1] period holding the group's maximum
+    unsigned char *cstate = (unsigned char *)(garg + G1);   // 0 = erased, else (destination + 1) | state | dirty flag
+    unsigned char *gflag = cstate + Pn;                 // [G1] a score of the group changed
+
+    if (tid == 0) { s_n_over = 0; s_ndirty = Pn; s_nlist = kOneDirtyCap + 1; s_nfin = 0; s_force = 0x7fffffff; s_win = -1; s_flagged = 1; }
+    __syncthreads();
+    {
+        int over = 0;
+#pragma unroll 1
+        for (int k = tid; k < K; k += kOneThreads) {
+            const int64_t pv = A.P[k];
+            sP[k] = pv;
+            if (pv > A.cap) ++over;
+        }
+#pragma unroll 1
+        for (int k = tid; k <= K; k += kOneThreads) sStart[k] = A.start[k];
+#pragma unroll 1
+        for (int k = tid; k < (host_cap ? 5 : 4) * K; k += kOneThreads) sBusy[k] = 0;
+#pragma unroll 1
+        for (int li = tid; li < G1 * 32; li += kOneThreads) ckey[li] = 0;
+#pragma unroll 1
+        for (int g = tid; g < G1; g += kOneThreads) { gkey[g] = 0; garg[g] = g * 32; gflag[g] = 0; }
+#pragma unroll 1
+        for (int li = tid; li < Pn; li += kOneThreads) {
+            OneRanges r;
+            r.a = (unsigned short)(A.per_u[li] + 1); r.b = (unsigned short)(A.per_v[li] - 1); r.ap = 0; r.bp = 0;
+            crng[li] = r;
+            cbytes[li] = A.bytes[A.per_t[li]];
+            ct[li] = 0; cben_lo[li] = 0; cben_hi[li] = 0;
+            cstate[li] = (unsigned char)kDirtyO;
+        }
+        over = __reduce_add_sync(0xffffffffu, over);
+        if (lane == 0 && over) atomicAdd(&s_n_over, over);
+    }
+    __syncthreads();
+
+    int64_t n_mig = 0, rounds = 0, bytes_ssd = 0, bytes_host = 0;
+    int status = -1;
+#ifdef G10_PHASE_CLOCKS
+    long long ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_cnt[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
+#endif
+#pragma unroll 1
+    for (int64_t it = 0;; ++it) {
+        if (A.fits_always || s_n_over == 0) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
+        if (it >= limit) { status = limit < Pn64 ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
+        rounds += 1;
+        ONE_CLOCK(0);
+        // ---------------- 1. DIRTY periods: destination (SSD first, then host), one warp per period; a new score
+        // only if the destination changed
+        if (s_ndirty > 0) {
+            const int nlist = s_nlist;
+            const bool listed = nlist <= kOneDirtyCap;            // else: sweep all periods for the flag
+            // listed periods go round the warps one by one; a sweep hands each warp 32 consecutive periods at a time
+            const int n_items = listed ? nlist : (Pn + 31) / 32 * 32;
+            const int step = listed ? kOneWarps : kOneThreads;
+#pragma unroll 1
+            for (int base = listed ? warp : warp * 32; base < n_items; base += step) {
+                unsigned m = 1u;
+                if (!listed) { const int mine = base + lane; m = __ballot_sync(0xffffffffu, mine < Pn && (cstate[mine] & kDirtyO) != 0); }
+#pragma unroll 1
+                while (m) {
+                    const int j = base + __ffs(m) - 1;
+                    m &= m - 1;
+                    const int li = listed ? s_dirty[j].li : j;
+                    ONE_COUNT(0);
+                    const unsigned char st = cstate[li];
+                    const OneRanges r = crng[li];
+                    const int a = r.a, b = r.b;
+                    const int64_t s = cbytes[li];
+                    const int64_t t_r = sStart[a], t_end = sStart[b + 1];
+                    int d = -1, ap = 0, bp = -1;
+                    int64_t t = 0;
+#pragma unroll 1
+                    for (int X = 0; X < 2 && d < 0; ++X) {
+                        if (listed) { ap = s_dirty[j].ap[X]; bp = s_dirty[j].bp[X]; t = s_dirty[j].t[X]; }
+                        else {
+                            ap = __ldg(&A.geo_a[X * A.geo_stride + li]);
+                            bp = __ldg(&A.geo_b[X * A.geo_stride + li]);
+                            t = __ldg(&A.geo_t[X * A.geo_stride + li]);
+                        }
+                        if (ap < 0) continue;
+                        if (!window_free_one(sStart, sBusy + (size_t)(2 * X) * K, t_r, t_r + t, a, ap - 1, lane)) continue;
+                        if (!window_free_one(sStart, sBusy + (size_t)(2 * X + 1) * K, t_end - t, t_end, bp + 1, b, lane)) continue;
+                        if (X == G10_DEST_HOST && host_cap) {
+                            bool ok = true;
+#pragma unroll 1
+                            for (int k = a + lane; k <= b; k += 32)
+                                if ((uint64_t)sHocc[k] + (uint64_t)s > A.host_capacity) ok = false;
+                            if (!__all_sync(0xffffffffu, ok)) continue;
+                        }
+                        d = X;
+                    }
+                    if (d < 0) {                                  // channels only fill up: gone for good
+                        ONE_COUNT(2);
+                        if (lane == 0) { cstate[li] = 0; ckey[li] = 0; gflag[li >> 5] = 1; s_flagged = 1; }
+                        continue;
+                    }
+                    if (d == (int)(st & 3) - 1) {                 // same destination: score and state stand
+                        if (lane == 0) cstate[li] = (unsigned char)(st & ~kDirtyO);
+                        continue;
+                    }
+                    ONE_COUNT(1);
+                    u128 acc = 0;
+#pragma unroll 1
+                    for (int k = ap + lane; k <= bp; k += 32) {
+                        int64_t ex = sP[k] - A.cap;
+                        if (ex > 0) {
+                            if (ex > s) ex = s;
+                            acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
+                        }
+                    }
+                    acc = warp_sum_u128(acc);
+                    if (lane == 0) {
+                        Cand cd;
+                        cd.ben = acc; cd.cost = 2ull * (ull)t; cd.idx = 0; cd.dest = d;
+                        OneRanges w = r;
+                        w.ap = (unsigned short)ap; w.bp = (unsigned short)bp;
+                        crng[li] = w; ct[li] = t;
+                        cben_lo[li] = (ull)acc; cben_hi[li] = (ull)(acc >> 64);
+                        ckey[li] = acc == 0 ? 0ull : (ull)__double_as_longlong(cand_key(cd));
+                        cstate[li] = (unsigned char)((d + 1) | kFreshO);
+                        gflag[li >> 5] = 1; s_flagged = 1;
+                    }
+                }
+            }
+            __syncthreads();
+            if (tid == 0) { s_ndirty = 0; s_nlist = 0; }
+            ONE_CLOCK(1);
+        }
+        // ---------------- 2. search: refresh the group maxima that changed, take the top, rescore it while it is stale
+        int win = -1;
+        bool exhausted = false;
+#pragma unroll 1
+        for (;;) {
+            if (warp == 0) {
+                if (s_flagged) {
+                __syncwarp();
+                if (lane == 0) s_flagged = 0;
+#pragma unroll 1
+                for (int g0 = 0; g0 < G1; g0 += 32) {
+                    unsigned m = __ballot_sync(0xffffffffu, g0 + lane < G1 && gflag[g0 + lane] != 0);
+#pragma unroll 1
+                    while (m) {
+                        const int g = g0 + __ffs(m) - 1;
+                        m &= m - 1;
+                        ull mk; int mi;
+                        warp_argmax_u64(ckey[g * 32 + lane], g * 32 + lane, &mk, &mi);
+                        if (lane == 0) { gkey[g] = mk; garg[g] = mi; gflag[g] = 0; }
+                    }
+                }
+                }
+                __syncwarp();
+                ull bk = 0; int bi = 0x7fffffff;
+#pragma unroll 4
+                for (int g = lane; g < G1; g += 32) {
+                    const ull k = gkey[g];
+                    if (k > bk) { bk = k; bi = garg[g]; }         // g ascending: the lowest index stays on ties
+                }
+                ull mk; int mi;
+                warp_argmax_u64(bk, bi, &mk, &mi);
+                if (lane == 0) { s_topkey = mk; s_top = mi; }
+            }
+            __syncthreads();
+            ONE_CLOCK(2);
+            const ull topkey = s_topkey;
+            const int top = s_top;
+            if (topkey == 0) { exhausted = true; break; }
+            int target = -1;
+            if ((cstate[top] & kStateMaskO) == kStaleO) target = top;
+            else {
+                // a fresh top: can anything else within 1e-10 of it beat it exactly?  (A stale entry competes with
+                // its bound: if even the bound loses, the period cannot win this iteration.)
+                const double thr = __longlong_as_double((long long)topkey) * (1.0 - 1e-10);
+                const ull thr_bits = (ull)__double_as_longlong(thr);
+                bool other = false;
+#pragma unroll 4
+                for (int g = warp; g < G1; g += kOneWarps) {
+                    if (gkey[g] < thr_bits) continue;
+                    const int li = g * 32 + lane;
+                    if (ckey[li] < thr_bits || li == top) continue;
+                    Cand x, y;
+                    x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
+                    y.ben = ((u128)cben_hi[top] << 64) | cben_lo[top]; y.cost = 2ull * (ull)ct[top]; y.idx = top; y.dest = 0;
+                    if (!cand_beats(x, y)) continue;
+                    other = true;
+                    if ((cstate[li] & kStateMaskO) == kStaleO) atomicMin(&s_force, li);
+                    else { const int pos = atomicAdd(&s_nfin, 1); if (pos < kOneMaxFin) s_fin[pos] = li; }
+                }
+                if (!__syncthreads_or(other)) { win = top; break; }
+                if (s_force != 0x7fffffff) target = s_force;
+                else {
+                    if (tid == 0) {
+                        Cand w;
+                        w.ben = ((u128)cben_hi[top] << 64) | cben_lo[top]; w.cost = 2ull * (ull)ct[top]; w.idx = top; w.dest = 0;
+                        const int n = s_nfin;
+                        if (n <= kOneMaxFin) {
+                            for (int i = 0; i < n; ++i) {
+                                const int li = s_fin[i];
+                                Cand x;
+                                x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
+                                if (cand_beats(x, w)) w = x;
+                            }
+                        } else {
+                            for (int li = 0; li < Pn; ++li) {      // very many close scores: plain sweep
+                                if (ckey[li] < thr_bits || (cstate[li] & kStateMaskO) != kFreshO) continue;
+                                Cand x;
+                                x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
+                                if (cand_beats(x, w)) w = x;
+                            }
+                        }
+                        s_win = w.idx; s_nfin = 0;
+                    }
+                    __syncthreads();
+                    win = s_win;
+                    break;
+                }
+            }
+            ONE_CLOCK(3);
+            // the whole block rescores period `target`
+            {
+                const OneRanges r = crng[target];
+                const int64_t s = cbytes[target];
+                u128 acc = 0;
+#pragma unroll 1
+                for (int k = r.ap + tid; k <= r.bp; k += kOneThreads) {
+                    int64_t ex = sP[k] - A.cap;
+                    if (ex > 0) {
+                        if (ex > s) ex = s;
+                        acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
+                    }
+                }
+                acc = warp_sum_u128(acc);
+                if (lane == 0) { s_part[2 * warp] = (ull)acc; s_part[2 * warp + 1] = (ull)(acc >> 64); }
+                __syncthreads();
+                if (tid == 0) {
+                    u128 tot = 0;
+#pragma unroll
+                    for (int w = 0; w < kOneWarps; ++w) tot += ((u128)s_part[2 * w + 1] << 64) | s_part[2 * w];
+                    Cand cd;
+                    cd.ben = tot; cd.cost = 2ull * (ull)ct[target]; cd.idx = 0; cd.dest = 0;
+                    cben_lo[target] = (ull)tot; cben_hi[target] = (ull)(tot >> 64);
+                    ckey[target] = tot == 0 ? 0ull : (ull)__double_as_longlong(cand_key(cd));
+                    cstate[target] = (unsigned char)((cstate[target] & 3) | kFreshO);
+                    gflag[target >> 5] = 1; s_flagged = 1;
+                    s_force = 0x7fffffff; s_nfin = 0;
+                }
+                __syncwarp();                   // warp 0 goes straight on to the refresh; the others wait at the barrier above
+            }
+            ONE_CLOCK(4);
+        }
+        if (exhausted) { status = G10_EXHAUSTED; break; }
+        ONE_CLOCK(5);
+        // ---------------- 3. apply the winner
+        {
+            const OneRanges r = crng[win];
+            const int X = (cstate[win] & 3) - 1;
+            const int wa = r.a, wb = r.b, wap = r.ap, wbp = r.bp;
+            const int64_t s = cbytes[win], t = ct[win];
+            const int64_t t_r = sStart[wa], t_end = sStart[wb + 1];
+            int win_tensor = 0;
+            if (tid == 0) win_tensor = A.per_t[win];              // needed only for the record written at the end
+            __syncthreads();                       // everyone has read the winner's entry before it is erased
+            int fell = 0;
+#pragma unroll 1
+            for (int k = wap + tid; k <= wbp; k += kOneThreads) {
+                const int64_t before = sP[k], after = before - s;
+                sP[k] = after;
+                if (before > A.cap && after <= A.cap) ++fell;
+            }
+            if (fell) atomicSub(&s_n_over, fell);
+            int64_t *bo = sBusy + (size_t)(2 * X) * K, *bi = sBusy + (size_t)(2 * X + 1) * K;
+#pragma unroll 1
+            for (int k = wa + tid; k <= wap - 1; k += kOneThreads) {
+                const int64_t s0 = sStart[k], s1 = sStart[k + 1];
+                const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
+                if (hi > lo) bo[k] += hi - lo;
+            }
+#pragma unroll 1
+            for (int k = wbp + 1 + tid; k <= wb; k += kOneThreads) {
+                const int64_t s0 = sStart[k], s1 = sStart[k + 1];
+                const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
+                if (hi > lo) bi[k] += hi - lo;
+            }
+            if (X == G10_DEST_HOST && host_cap)
+#pragma unroll 1
+                for (int k = wa + tid; k <= wb; k += kOneThreads) sHocc[k] += s;
+            __syncthreads();                       // the bookings are in place for the conflict tests below
+            int newly_dirty = 0;
+#pragma unroll 2
+            for (int li = tid; li < Pn; li += kOneThreads) {
+                const unsigned char st = cstate[li];
+                if (st == 0) continue;
+                if (li == win) { cstate[li] = 0; ckey[li] = 0; gflag[li >> 5] = 1; s_flagged = 1; continue; }
+                if (st & kDirtyO) continue;
+                const int d = (st & 3) - 1;
+                const OneRanges q = crng[li];
+                if (!((int)q.a <= wb && wa <= (int)q.b)) continue;
+                unsigned char ns = st;
+                if ((st & kStateMaskO) == kFreshO && (int)q.ap <= wbp && wap <= (int)q.bp) ns = (unsigned char)((st & 3) | kStaleO);
+                if (d == X) {
+                    // same device: is one of its transfer windows no longer free?  (host occupancy: looked at in full)
+                    const bool meet_out = (int)q.a <= wap - 1 && wa <= (int)q.ap - 1;
+                    const bool meet_in = (int)q.bp + 1 <= wb && wbp + 1 <= (int)q.b;
+                    bool hit = false;
+                    if (meet_out || meet_in) {
+                        const int64_t tq = ct[li];
+                        const int64_t q_r = sStart[q.a], q_end = sStart[(int)q.b + 1];
+                        hit = (meet_out && window_conflict(sStart, bo, wa, wap - 1, q_r, q_r + tq, q.a, (int)q.ap - 1)) ||
+                              (meet_in && window_conflict(sStart, bi, wbp + 1, wb, q_end - tq, q_end, (int)q.bp + 1, q.b));
+                    }
+                    if (!hit && d == G10_DEST_HOST && host_cap) hit = true;
+                    if (hit) {
+                        ns |= kDirtyO; ++newly_dirty;
+                        const int pos = atomicAdd(&s_nlist, 1);
+                        if (pos < kOneDirtyCap) {                  // fetch both geometries now: the latency hides behind the rest
+                            OneDirty e;
+                            e.li = li;
+#pragma unroll
+                            for (int Y = 0; Y < 2; ++Y) {
+                                e.ap[Y] = __ldg(&A.geo_a[Y * A.geo_stride + li]);
+                                e.bp[Y] = __ldg(&A.geo_b[Y * A.geo_stride + li]);
+                                e.t[Y] = __ldg(&A.geo_t[Y * A.geo_stride + li]);
+                            }
+                            e.pad[0] = e.pad[1] = e.pad[2] = 0;
+                            s_dirty[pos] = e;
+                        }
+                    }
+                }
+                if (ns != st) cstate[li] = ns;
+            }
+            if (newly_dirty) atomicAdd(&s_ndirty, newly_dirty);
+            if (tid == 0) {
+                if (n_mig < A.out_cap) {
+                    g10_migration m;
+                    m.period = (int32_t)win; m.tensor = win_tensor; m.dest = X; m.absent_first = wap; m.absent_last = wbp;
+                    m.iteration = (int32_t)it; m.evict_issue_ns = t_r; m.prefetch_issue_ns = t_end - t; m.transfer_ns = t;
+                    A.out[n_mig] = m;
+                } else raise_status(A.status, G10_DEV_PLAN_OVERFLOW);
+            }
+            n_mig += 1;
+            if (X == G10_DEST_SSD) bytes_ssd += s; else bytes_host += s;
+        }
+        __syncthreads();
+        ONE_CLOCK(6);
+    }
+#ifdef G10_PHASE_CLOCKS
+    if (threadIdx.x == 0) {
+        const long long r = rounds ? rounds : 1;
+        printf("one-block cycles/iteration: top %lld dirty %lld (x%lld) topscan %lld (x%lld) tiescan %lld (x%lld) rescore %lld (x%lld) winner %lld apply %lld (n=%lld)\n",
+               ph_acc[0] / r, ph_acc[1] / r, ph_cnt[1], ph_acc[2] / r, ph_cnt[2], ph_acc[3] / r, ph_cnt[3], ph_acc[4] / r, ph_cnt[4], ph_acc[5] / r,
+               ph_acc[6] / r, (long long)rounds);
+        printf("dirty periods examined %d, rescored %d, erased %d\n", s_dbg[0], s_dbg[1], s_dbg[2]);
+    }
+#endif
+    // ---------------- epilogue: final pressure, peak and its lowest slot, summary
+    __syncthreads();
+    long long pk = 0;
+    int ps = -1;
+#pragma unroll 1
+    for (int k = tid; k < K; k += kOneThreads) {
+        const long long pv = sP[k];
+        A.P[k] = pv;
+        if (ps < 0 || pv > pk) { pk = pv; ps = k; }      // k ascending per thread: first maximum kept
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long yk = __shfl_xor_sync(0xffffffffu, pk, o);
+        const int ys = __shfl_xor_sync(0xffffffffu, ps, o);
+        if (ys >= 0 && (ps < 0 || yk > pk || (yk == pk && ys < ps))) { pk = yk; ps = ys; }
+    }
+    if (lane == 0) { s_pk[warp] = pk; s_ps[warp] = ps; }
+    __syncthreads();
+    if (tid == 0) {
+#pragma unroll 1
+        for (int j = 1; j < kOneWarps; ++j)
+            if (s_ps[j] >= 0 && (ps < 0 || s_pk[j] > pk || (s_pk[j] == pk && s_ps[j] < ps))) { pk = s_pk[j]; ps = s_ps[j]; }
+        A.summary[0] = n_mig; A.summary[1] = rounds; A.summary[2] = status;
+        A.summary[3] = ps < 0 ? 0 : pk; A.summary[4] = ps;
+        A.summary[5] = bytes_ssd; A.summary[6] = bytes_host;
+        *O.done = 1u;
+    }
+}
+
+// Shared memory a launch can offer (opt-in maximum minus the kernel's static part); 0 if the device query fails.
+static int one_smem_budget()
+{
+    int dev = 0, optin = 0;
+    cudaFuncAttributes fa;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return 0;
+    if (cudaFuncGetAttributes(&fa, (const void *)k_plan_one) != cudaSuccess) return 0;
+    const int room = optin - (int)fa.sharedSizeBytes;
+    return room > 0 ? room : 0;
+}
+
+// Worth launching: the fixed part of the state (pressure, clock, bookings) leaves room for at least a few
+// hundred periods.  Whether the periods fit too is only known on the device.
+bool plan_one_possible(int64_t K, int64_t E, bool host_cap)
+{
+    if (K > 65000 || E < 1) return false;
+    const int budget = one_smem_budget();
+    return budget > 0 && one_smem_need(K, E < 512 ? E : 512, host_cap) <= (size_t)budget;
+}
+
+cudaError_t launch_plan_one(const PlanArgs &A_in, const Workspace &w, cudaStream_t s)
+{
+    PlanArgs A = A_in;
+    OneArgs O;
+    O.done = w.one_done;
+    O.smem_bytes = one_smem_budget();
+    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
+    if (e != cudaSuccess) return e;
+    k_plan_one<<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O);
+    return cudaGetLastError();
+}
+
+}  // namespace g10

@@ -37,6 +37,7 @@ struct SmallArgs {
     ull *xwords;            // [2][G][kXWords] tagged proposals, then [2][G][kXWords] winner records, one copy per block
                             // (all start zeroed; tags start at 1)
     int cand_cap;           // periods a block can own
+    const unsigned *done;   // non-zero: the single-block planner already produced the plan
 };
 
 // Static facts of an owned period, cached in shared memory for the whole run.
@@ -125,6 +126,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
     __shared__ int s_todo;
     __shared__ ull s_part[2 * kPlanWarps];
     __shared__ unsigned s_err;
+    if (*S.done) return;                  // same answer in every thread of the grid: written by an earlier launch
     const int G = gridDim.x, c = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int K = (int)A.K;
@@ -572,7 +574,7 @@ cudaError_t launch_plan_small(const PlanArgs &A_in, const Workspace &w, int G, i
 {
     PlanArgs A = A_in;
     SmallArgs S;
-    S.busy_rep = w.busy_rep; S.hocc_rep = w.hocc_rep; S.xwords = w.xwords; S.cand_cap = cand_cap;
+    S.busy_rep = w.busy_rep; S.hocc_rep = w.hocc_rep; S.xwords = w.xwords; S.cand_cap = cand_cap; S.done = w.one_done;
     const void *kernel = cand_cap <= 256 ? (const void *)k_plan_small<true> : (const void *)k_plan_small<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

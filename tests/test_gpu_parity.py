@@ -96,6 +96,7 @@ def full_parity(gpu, oracle, tr, lazy_oracle=False, repeats=1, **plan_kw):
     if also:
         check_plan(gpu, tr, tb, cap, ref, flags=gpu.FLAG_RESCORE_ALL, **plan_kw)      # Algorithm 1 as printed
         check_plan(gpu, tr, tb, cap, ref, flags=gpu.FLAG_GLOBAL_STATE, **plan_kw)     # the large-trace planner
+        check_plan(gpu, tr, tb, cap, ref, flags=gpu.FLAG_MULTI_BLOCK, **plan_kw)      # never the single-block planner
     return ref
 
 
