@@ -176,3 +176,26 @@ def characterize(K, vit, tensor_bytes, start, host_bw, ssd_bw):
                             _p(pt), _p(pu), _p(pv), C.c_uint64(host_bw), C.c_uint64(ssd_bw), _p(active), _p(lh), _p(slh),
                             _p(hide), _p(summary))
     return SimpleNamespace(active_bytes=active, len_hist=lh, size_len_hist=slh.reshape(41, 45), hide=hide, summary=summary)
+
+
+def plan_batch(trace, variants, max_iterations=0, lazy=True):
+    """Re-planning under changed conditions (Section 5's sensitivity studies seen from the planner): every variant is a
+    whole plan of the same trace with its own kernel durations (profiling error), bandwidths, capacities.  A variant is
+    a dict with any of kernel_ns, gpu_capacity_bytes, host_bw, ssd_bw, host_capacity_bytes; gpu_capacity_bytes is
+    required.  Plan stability of variant v against variant 0 is reported as the pair (|M_v & M_0|, |M_v | M_0|) over
+    the sets of migrated periods (their quotient is the Jaccard index)."""
+    import copy
+    plans, stability = [], []
+    base = None
+    for v in variants:
+        tr = copy.copy(trace)
+        if v.get("kernel_ns") is not None:
+            tr.kernel_ns = _c(v["kernel_ns"], np.int64)
+        r = plan(tr, int(v["gpu_capacity_bytes"]), host_bw=v.get("host_bw"), ssd_bw=v.get("ssd_bw"),
+                 host_capacity_bytes=v.get("host_capacity_bytes", 0), max_iterations=max_iterations, lazy=lazy)
+        mine = set(int(p) for p in r.migrations["period"])
+        if base is None:
+            base = mine
+        stability.append((len(mine & base), len(mine | base)))
+        plans.append(r)
+    return SimpleNamespace(plans=plans, stability=np.asarray(stability, dtype=np.int64).reshape(-1, 2))
