@@ -56,6 +56,7 @@ extern "C" {
 #define G10_DEV_PERIODS_OVERFLOW 0x20 /* periods_cap too small (counts[1] holds the need)         */
 #define G10_DEV_PLAN_OVERFLOW 0x40   /* migrations_cap too small (summary[0] holds the need)      */
 #define G10_DEV_TIMEOUT 0x80         /* an internal wait gave up; the kernel returned early       */
+#define G10_DEV_BATCH_UNFIT 0x100    /* g10_plan_batch: the trace does not fit one SM (no plan)   */
 
 /* exit status of the planner (summary[2]) */
 #define G10_ALREADY_FITS 0      /* unplanned peak pressure <= capacity, empty plan                 */
@@ -165,6 +166,7 @@ typedef struct g10_options {
 #define G10_WS_PLAN 2
 #define G10_WS_GEOMETRY 3
 #define G10_WS_EMIT 4
+#define G10_WS_BATCH 5
 
 /* Section 4.2, tensor vitality analysis. */
 int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, size_t ws_bytes, void *stream);
@@ -240,6 +242,34 @@ int32_t g10_emit_instructions(int64_t num_kernels, int64_t num_tensors, const in
                               const int64_t *tensor_bytes, const uint8_t *tensor_global, const int64_t *kernel_start_ns,
                               int64_t num_migrations, const g10_migration *migrations, const int64_t *new_prefetch_issue_ns,
                               g10_emit_out *out, void *ws, size_t ws_bytes, void *stream);
+
+/* Section 5's sensitivity studies seen from the planner: the same trace planned under V variants at once -- other
+   kernel durations (profiling error), SSD / host bandwidths, GPU capacity, host capacity -- one thread block per
+   variant, all variants running concurrently.  Every variant's result is exactly what g10_plan_migrations gives for
+   the trace with that variant's durations and parameters.  `variants` is a HOST array (copied before the call
+   returns); its kernel_ns pointers are DEVICE pointers.  Outputs are DEVICE pointers: migrations [V][migrations_cap],
+   final_pressure [V][K], summary [V][8] (as in g10_plan_out; summary[8 v + 7] holds the status bits of variant v),
+   stability [V][2] = (|M_v & M_0|, |M_v | M_0|) over the sets of migrated periods of variant v and variant 0 (their
+   quotient is the Jaccard index; (-1, -1) when a plan is missing).
+   Limits: the trace has to be device resident (G10_MEM_DEVICE); 1 <= V <= 1024; pressure, clock, bookings and the
+   periods of the trace must fit the shared memory of one SM (the DNN-shaped traces of a few thousand kernels do),
+   else every variant reports G10_DEV_BATCH_UNFIT and summary[2] = -1: plan such traces one by one.
+   Workspace: G10_WS_BATCH. */
+typedef struct g10_variant {
+    const int64_t *kernel_ns;       /* [K] device pointer, or NULL: the trace's own durations */
+    uint64_t gpu_capacity_bytes;
+    uint64_t host_bw, ssd_bw;       /* bytes per second */
+    uint64_t host_capacity_bytes;   /* 0 = unlimited */
+} g10_variant;
+typedef struct g10_batch_out {
+    g10_migration *migrations;
+    int64_t migrations_cap;         /* records per variant */
+    int64_t *final_pressure;
+    int64_t *summary;
+    int64_t *stability;
+} g10_batch_out;
+int32_t g10_plan_batch(const g10_trace *trace, int32_t num_variants, const g10_variant *variants, int64_t max_iterations,
+                       g10_batch_out *out, void *ws, size_t ws_bytes, void *stream);
 
 /* Section 3, workload characterisation (the statistics of Figures 2-4) from the results of g10_vitality and the
    slot clock of g10_pressure_timeline.  active_bytes [K]: bytes of the tensors kernel k uses, each once (the

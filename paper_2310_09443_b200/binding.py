@@ -17,14 +17,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libg10.so")
 
 MEM_DEVICE, MEM_HOST = 0, 1
-WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT = 0, 1, 2, 3, 4
+WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT, WS_BATCH = 0, 1, 2, 3, 4, 5
 DEST_SSD, DEST_HOST = 0, 1
 FLAG_RESCORE_ALL = 1
 FLAG_GLOBAL_STATE = 2
 FLAG_MULTI_BLOCK = 4
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
-           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize")
+           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize", "g10_plan_batch")
 STATIC_MAX_KERNELS, STATIC_MAX_TENSORS = 32768, 131072
 
 INSTRUCTION_DTYPE = np.dtype([("opcode", "<i4"), ("tensor", "<i4"), ("target", "<i4"), ("record", "<i4"),
@@ -63,6 +63,16 @@ class _GeometryOut(C.Structure):
 class _PlanOut(C.Structure):
     _fields_ = [("migrations", C.c_void_p), ("migrations_cap", C.c_int64), ("final_pressure", C.c_void_p),
                 ("summary", C.c_void_p)]
+
+
+class _Variant(C.Structure):
+    _fields_ = [("kernel_ns", C.c_void_p), ("gpu_capacity_bytes", C.c_uint64), ("host_bw", C.c_uint64), ("ssd_bw", C.c_uint64),
+                ("host_capacity_bytes", C.c_uint64)]
+
+
+class _BatchOut(C.Structure):
+    _fields_ = [("migrations", C.c_void_p), ("migrations_cap", C.c_int64), ("final_pressure", C.c_void_p),
+                ("summary", C.c_void_p), ("stability", C.c_void_p)]
 
 
 class _PrefetchOut(C.Structure):
@@ -118,6 +128,9 @@ def load_library():
         lib.g10_characterize.restype = C.c_int32
         lib.g10_characterize.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.POINTER(_StatsOut), C.c_void_p]
+        lib.g10_plan_batch.restype = C.c_int32
+        lib.g10_plan_batch.argtypes = [C.POINTER(_Trace), C.c_int32, C.POINTER(_Variant), C.c_int64, C.POINTER(_BatchOut),
+                                       C.c_void_p, C.c_size_t, C.c_void_p]
         lib.g10_plan_migrations.restype = C.c_int32
         lib.g10_plan_migrations.argtypes = [C.POINTER(_Trace), C.c_uint64, C.c_uint64, C.c_uint64, C.POINTER(_Options),
                                             C.POINTER(_PlanOut), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -307,6 +320,42 @@ def g10_plan_migrations(tb: TraceBuffers, gpu_capacity_bytes, host_bw, ssd_bw, h
                                    ws_bytes, _stream(stream)))
     out.workspace = ws
     return out
+
+
+def g10_plan_batch(tb: TraceBuffers, variants, max_iterations=0, migrations_cap=None, ws=None, stream=None):
+    """Plans the device-resident trace under every variant at once (one thread block each).  A variant is a dict with
+    gpu_capacity_bytes, host_bw, ssd_bw and optionally kernel_ns (int64 device tensor [K]) and host_capacity_bytes.
+    Returns migrations [V, migrations_cap * 48] (uint8), final_pressure [V, K], summary [V, 8], stability [V, 2]."""
+    lib = load_library()
+    V = len(variants)
+    dev = tb.kernel_ptr.device
+    mcap = tb.E if migrations_cap is None else migrations_cap
+    out = SimpleNamespace(migrations=torch.empty((max(V, 1), max(mcap, 1) * 48), dtype=torch.uint8, device=dev),
+                          final_pressure=torch.empty((max(V, 1), max(tb.K, 1)), dtype=torch.int64, device=dev),
+                          summary=torch.empty((max(V, 1), 8), dtype=torch.int64, device=dev),
+                          stability=torch.empty((max(V, 1), 2), dtype=torch.int64, device=dev), migrations_cap=mcap)
+    arr = (_Variant * max(V, 1))()
+    keep = []
+    for j, v in enumerate(variants):
+        kn = v.get("kernel_ns")
+        if kn is not None:
+            assert kn.dtype == torch.int64 and kn.is_contiguous() and kn.numel() >= tb.K
+            keep.append(kn)
+        arr[j] = _Variant(_ptr(kn) if kn is not None else None, int(v["gpu_capacity_bytes"]), int(v["host_bw"]), int(v["ssd_bw"]),
+                          int(v.get("host_capacity_bytes", 0)))
+    ws, ws_bytes = _workspace(tb, WS_BATCH, ws, None)
+    bo = _BatchOut(_ptr(out.migrations), mcap, _ptr(out.final_pressure), _ptr(out.summary), _ptr(out.stability))
+    tr = tb.c_struct()
+    _check(lib.g10_plan_batch(C.byref(tr), V, arr, max_iterations, C.byref(bo), _ptr(ws), ws_bytes, _stream(stream)))
+    out.workspace = ws
+    out.keep = keep
+    return out
+
+
+def batch_migrations_numpy(batch, v) -> np.ndarray:
+    """Committed migration records of variant v of a finished batch (synchronises)."""
+    n = min(int(batch.summary[v, 0].item()), batch.migrations_cap)
+    return batch.migrations[v, : n * 48].cpu().numpy().view(MIGRATION_DTYPE).copy()
 
 
 def g10_schedule_prefetch(K, num_migrations, migrations, kernel_start_ns, tensor_bytes, gpu_capacity_bytes, pressure,

@@ -1,5 +1,6 @@
 // The C ABI: argument checks, workspace layout, host-buffer staging and the launch sequence of each call.
 #include <cstring>
+#include <vector>
 
 #include "g10_internal.h"
 
@@ -106,6 +107,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     }
     w.peak_part = c.take<int64_t>(kMaxPlanBlocks);
     w.summary = c.take<int64_t>(8);
+    w.batch_variants = c.take<BatchVariant>(kMaxVariants);
     if (z.host) {
         w.migrations = c.take<g10_migration>(E);
         w.s_kernel_ptr = c.take<int64_t>(K + 1);
@@ -220,7 +222,7 @@ const char *g10_strerror(int32_t code)
 int32_t g10_workspace_bytes(int32_t which, int64_t K, int64_t N, int64_t E, int32_t mem, size_t *out_bytes)
 {
     if (!out_bytes || K < 0 || N < 0 || E < 0) return G10_ERR_ARG;
-    if (which < G10_WS_VITALITY || which > G10_WS_EMIT) return G10_ERR_ARG;
+    if (which < G10_WS_VITALITY || which > G10_WS_BATCH) return G10_ERR_ARG;
     if (mem != G10_MEM_DEVICE && mem != G10_MEM_HOST) return G10_ERR_ARG;
     const int64_t lim = ((int64_t)1 << 31) - 1;
     if (K >= lim || N >= lim || E >= lim) return G10_ERR_LIMIT;
@@ -395,6 +397,45 @@ int32_t g10_schedule_prefetch(int64_t K, int64_t n, const g10_migration *migrati
         return G10_ERR_ARG;
     CU(launch_schedule_prefetch(K, n, migrations, kernel_start_ns, tensor_bytes, gpu_capacity_bytes, out->pressure, out->order,
                                 out->new_absent_last, out->new_prefetch_issue_ns, out->summary, (cudaStream_t)stream));
+    return G10_OK;
+}
+
+int32_t g10_plan_batch(const g10_trace *trace, int32_t V, const g10_variant *variants, int64_t max_iterations, g10_batch_out *out,
+                       void *ws, size_t ws_bytes, void *stream)
+{
+    int32_t rc = check_trace(trace);
+    if (rc != G10_OK) return rc;
+    if (trace->mem != G10_MEM_DEVICE || !variants || !out || !out->summary || !out->stability || max_iterations < 0) return G10_ERR_ARG;
+    if (V < 1 || V > kMaxVariants) return G10_ERR_LIMIT;
+    if (out->migrations_cap < 0 || (out->migrations_cap > 0 && !out->migrations)) return G10_ERR_ARG;
+    if (trace->num_kernels > 0 && !out->final_pressure) return G10_ERR_ARG;
+    std::vector<BatchVariant> bv((size_t)V);
+    for (int32_t v = 0; v < V; ++v) {
+        if (variants[v].host_bw == 0 || variants[v].ssd_bw == 0) return G10_ERR_ARG;
+        bv[v].kernel_ns = variants[v].kernel_ns ? variants[v].kernel_ns : trace->kernel_ns;
+        bv[v].cap = variants[v].gpu_capacity_bytes; bv[v].host_bw = variants[v].host_bw; bv[v].ssd_bw = variants[v].ssd_bw;
+        bv[v].host_capacity = variants[v].host_capacity_bytes;
+    }
+    rc = check_ws(G10_WS_BATCH, trace, ws, ws_bytes);
+    if (rc != G10_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    Workspace w;
+    DeviceTrace d;
+    const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
+    rc = begin_call(trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff);
+    if (rc != G10_OK) return rc;
+    CU(cudaMemcpyAsync(w.batch_variants, bv.data(), sizeof(BatchVariant) * (size_t)V, cudaMemcpyHostToDevice, s));
+    VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
+                       w.period_tensor, w.period_prev_use, w.period_next_use, d.E, w.counts};
+    PlanParams pp;
+    pp.gpu_capacity_bytes = 0; pp.host_bw = 1; pp.ssd_bw = 1; pp.host_capacity_bytes = 0;      // per variant, on the device
+    pp.max_iterations = max_iterations; pp.flags = 0;
+    pp.migrations = out->migrations; pp.migrations_cap = out->migrations_cap;
+    pp.final_pressure = out->final_pressure; pp.summary = out->summary;
+    CU(launch_slot_clock(d, w, w.start, s));                    // validates kernel_ptr and the trace's own durations
+    CU(buckets ? launch_vitality_buckets(d, w, vb, s) : launch_vitality(d, w, vb, s));
+    CU(launch_pressure(d, w, w.first_use, w.last_use, false, w.pressure, w.peak_bytes, w.peak_slot, s));
+    CU(launch_plan_variants(d, w, pp, V, out->stability, s));
     return G10_OK;
 }
 

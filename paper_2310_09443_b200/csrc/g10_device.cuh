@@ -187,6 +187,44 @@ __device__ __forceinline__ int next_tile(unsigned *ticket)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Candidate geometry of one inactive period (Algorithm 1 / Section 4.4) for one destination.
+// ---------------------------------------------------------------------------------------------
+// Time to move `bytes` at `bw` bytes per second, in ns, rounded up; saturates at 2^62.
+__device__ __forceinline__ int64_t transfer_time_ns(int64_t bytes, uint64_t bw)
+{
+    const u128 num = (u128)(uint64_t)bytes * (u128)1000000000ull;
+    u128 q = num / (u128)bw;
+    if (q * (u128)bw != num) q += 1;
+    const u128 sat = (u128)1 << 62;
+    return (int64_t)(q > sat ? sat : q);
+}
+
+// Period between uses u and v of a tensor of s bytes; `start` is the slot clock (global or shared memory).
+// The eviction occupies [t_r, t_r + t) from the period's start, the prefetch [t_end - t, t_end) up to its end;
+// the tensor is absent in the slots that lie wholly between the two.  (-1, -2) when they leave no such slot.
+__device__ __forceinline__ void period_geometry(const int64_t *start, int u, int v, int64_t s, uint64_t bw, int64_t *t_out,
+                                                int *a_abs_out, int *b_abs_out)
+{
+    const int64_t t_r = start[u + 1], t_end = start[v], L = t_end - t_r;
+    const int64_t t = transfer_time_ns(s, bw);
+    int a_abs = -1, b_abs = -2;
+    if (t <= L && 2 * t <= L) {
+        // first k in [u+1, v] with start[k] >= t_r + t   (start[v] = t_end > t_r + t - 1 always qualifies)
+        int lo = u + 1, hi = v;
+        const int64_t ev_end = t_r + t;
+        while (lo < hi) { const int mid = lo + (hi - lo) / 2; if (start[mid] >= ev_end) hi = mid; else lo = mid + 1; }
+        const int ap = lo;
+        // last j in [u+1, v] with start[j] <= t_end - t   (start[u+1] = t_r qualifies)
+        lo = u + 1; hi = v;
+        const int64_t pf_beg = t_end - t;
+        while (lo < hi) { const int mid = lo + (hi - lo + 1) / 2; if (start[mid] <= pf_beg) lo = mid; else hi = mid - 1; }
+        const int bp = lo - 1;
+        if (ap <= bp) { a_abs = ap; b_abs = bp; }
+    }
+    *t_out = t; *a_abs_out = a_abs; *b_abs_out = b_abs;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Grid barrier for the persistent planner kernel (launched cooperatively, so all blocks are
 // resident).  Sense comes from a generation counter.  A wait that lasts longer than
 // kBarrierTimeoutNs sets `error`; from then on every barrier returns false at once and the

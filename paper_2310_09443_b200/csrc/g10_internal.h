@@ -33,6 +33,18 @@ struct Proposal {          // a block's best candidate of one scoring round (32 
     int dest;
 };
 
+// One variant of a batched re-planning call (device copy of g10_variant with the defaults filled in).
+struct BatchVariant {
+    const int64_t *kernel_ns;
+    uint64_t cap, host_bw, ssd_bw, host_capacity;
+};
+struct BatchArgs {
+    const BatchVariant *variants;     // [V]
+    const int64_t *P0;                // [K] unplanned pressure, shared by all variants
+    int64_t *P_out;                   // [V][K]
+};
+constexpr int kMaxVariants = 1024;
+
 // Device views of a trace and of the intermediate arrays; filled by carve() in g10_api.cu.
 struct Workspace {
     // --- zero-initialised region (one memset per call) ---
@@ -83,6 +95,7 @@ struct Workspace {
     int64_t *peak_part;          // [max blocks]
     g10_migration *migrations;   // host mode only
     int64_t *summary;            // [8]
+    BatchVariant *batch_variants; // [kMaxVariants]
     // staged copies of the trace (host mode only)
     int64_t *s_kernel_ptr, *s_tensor_bytes, *s_kernel_ns;
     int32_t *s_kernel_tensors;
@@ -164,6 +177,7 @@ cudaError_t launch_characterize(int64_t K, int64_t N, const int64_t *use_ptr, co
                                 int64_t *active, int64_t *len_hist, int64_t *size_len_hist, int64_t *hide, int64_t *summary, cudaStream_t s);
 // planner (g10_planner.cu)
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
+cudaError_t launch_plan_variants(const DeviceTrace &t, const Workspace &w, const PlanParams &p, int V, int64_t *stability, cudaStream_t s);
 int plan_loop_max_blocks();
 bool plan_keeps_state_on_chip(int64_t K, int64_t E, uint32_t flags);   // true: the small-trace planner will run
 cudaError_t launch_publish_status(const Workspace &w, int64_t *dst, cudaStream_t s);

@@ -798,15 +798,6 @@ cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int3
 // =============================================================================================
 // Candidate geometry.
 // =============================================================================================
-__device__ __forceinline__ int64_t transfer_time_ns(int64_t bytes, uint64_t bw)
-{
-    const u128 num = (u128)(uint64_t)bytes * (u128)1000000000ull;
-    u128 q = num / (u128)bw;
-    if (q * (u128)bw != num) q += 1;
-    const u128 sat = (u128)1 << 62;
-    return (int64_t)(q > sat ? sat : q);
-}
-
 __global__ void __launch_bounds__(256) k_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, const int64_t *__restrict__ start,
                                                   const int64_t *__restrict__ bytes, const int32_t *__restrict__ per_t,
                                                   const int32_t *__restrict__ per_u, const int32_t *__restrict__ per_v,
@@ -818,24 +809,11 @@ __global__ void __launch_bounds__(256) k_geometry(int64_t K, int64_t Pn_bound, c
     if (p >= Pn) return;
     const int64_t s = bytes[per_t[p]];
     const int u = per_u[p], v = per_v[p];
-    const int64_t t_r = start[u + 1], t_end = start[v], L = t_end - t_r;
 #pragma unroll
     for (int X = 0; X < 2; ++X) {
-        const int64_t t = transfer_time_ns(s, X == G10_DEST_SSD ? ssd_bw : host_bw);
-        int a_abs = -1, b_abs = -2;
-        if (t <= L && 2 * t <= L) {
-            // first k in [u+1, v] with start[k] >= t_r + t   (start[v] = t_end > t_r + t - 1 always qualifies)
-            int lo = u + 1, hi = v;
-            const int64_t ev_end = t_r + t;
-            while (lo < hi) { const int mid = lo + (hi - lo) / 2; if (start[mid] >= ev_end) hi = mid; else lo = mid + 1; }
-            const int ap = lo;
-            // last j in [u+1, v] with start[j] <= t_end - t   (start[u+1] = t_r qualifies)
-            lo = u + 1; hi = v;
-            const int64_t pf_beg = t_end - t;
-            while (lo < hi) { const int mid = lo + (hi - lo + 1) / 2; if (start[mid] <= pf_beg) lo = mid; else hi = mid - 1; }
-            const int bp = lo - 1;
-            if (ap <= bp) { a_abs = ap; b_abs = bp; }
-        }
+        int64_t t;
+        int a_abs, b_abs;
+        period_geometry(start, u, v, s, X == G10_DEST_SSD ? ssd_bw : host_bw, &t, &a_abs, &b_abs);
         geo_t[X * stride + p] = t;
         geo_a[X * stride + p] = a_abs;
         geo_b[X * stride + p] = b_abs;

@@ -132,6 +132,17 @@ bool plan_keeps_state_on_chip(int64_t K, int64_t E, uint32_t flags)
     return Gs >= 1 && plan_small_fits(K, E, Gs, &cand_cap, &smem);
 }
 
+cudaError_t launch_plan_batch(const PlanArgs &A, const Workspace &w, int V, const BatchArgs &B, int64_t *stability, cudaStream_t s);
+
+cudaError_t launch_plan_variants(const DeviceTrace &t, const Workspace &w, const PlanParams &p, int V, int64_t *stability, cudaStream_t s)
+{
+    PlanArgs A;
+    fill_plan_args(t, w, p, A);
+    BatchArgs B;
+    B.variants = w.batch_variants; B.P0 = w.pressure; B.P_out = p.final_pressure;
+    return launch_plan_batch(A, w, V, B, stability, s);
+}
+
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s)
 {
     PlanArgs A;

@@ -15,6 +15,11 @@
 //     and are rescored only if the destination changed.
 // The kernel decides by itself, from the number of periods found on the device, whether the trace fits; if it
 // does not, it leaves `done` at zero and the multi-block planner launched right behind it does the work.
+//
+// Batch mode (kBatch): one block per VARIANT of the same trace -- its own kernel durations, bandwidths and
+// capacities -- each running the whole loop independently of the others (re-planning under profiling error,
+// other SSD bandwidths or host capacities).  A variant's block builds its own slot clock (block-wide scan of its
+// durations) and derives the geometry of a period when it needs it, from that clock in shared memory.
 #include <cstdio>
 
 #include "g10_planner.cuh"
@@ -26,7 +31,7 @@ namespace g10 {
 #endif
 constexpr int kOneThreads = G10_ONE_THREADS;
 constexpr int kOneWarps = kOneThreads / 32;
-constexpr int kOneMaxFin = 64;
+constexpr int kOneMaxFin = 64;                // (at least kOneWarps: the list doubles as scratch at the end)
 constexpr int kOneDirtyCap = 256;            // DIRTY periods of one commit that are listed (more: full sweep)
 enum { kFreshO = 1 << 2, kStaleO = 2 << 2, kStateMaskO = 3 << 2, kDirtyO = 0x10 };
 
@@ -42,7 +47,7 @@ struct __align__(16) OneDirty {
     int li;
     int ap[2], bp[2];
     int pad[3];
-    long long t[2];
+    int64_t t[2];
 };
 
 __device__ __forceinline__ bool window_free_one(const int64_t *sStart, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane)
@@ -110,7 +115,8 @@ __device__ __forceinline__ void warp_argmax_u64(ull k, int idx, ull *mk, int *mi
 #define ONE_COUNT(i)
 #endif
 
-__global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs O)
+template <bool kBatch>
+__global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs O, BatchArgs B)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ ull s_part[2 * kOneWarps];
@@ -127,8 +133,30 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K = (int)A.K;
     const int64_t Pn64 = *A.Pn_dev < A.geo_stride ? *A.Pn_dev : A.geo_stride;
+    const int64_t *P_src = A.P;
+    uint64_t bw[2] = {0, 0};
+    const int64_t *var_dur = nullptr;
+    if (kBatch) {
+        const BatchVariant var = B.variants[blockIdx.x];
+        A.fits_always = var.cap >= ((uint64_t)1 << 63) ? 1 : 0;
+        A.cap = A.fits_always ? INT64_MAX : (int64_t)var.cap;
+        A.host_capacity = var.host_capacity;
+        A.out += (size_t)blockIdx.x * A.out_cap;
+        A.summary += (size_t)blockIdx.x * 8;
+        P_src = B.P0;
+        A.P = B.P_out + (size_t)blockIdx.x * K;
+        bw[G10_DEST_SSD] = var.ssd_bw; bw[G10_DEST_HOST] = var.host_bw;
+        var_dur = var.kernel_ns;
+    }
     const bool host_cap = A.host_capacity != 0;
-    if (A.K > 65000 || Pn64 > 0x7fffffff || one_smem_need(A.K, Pn64, host_cap) > (size_t)O.smem_bytes) return;
+    unsigned dev_bits = 0;                              // device status bits of this block's plan
+    if (A.K > 65000 || Pn64 > 0x7fffffff || one_smem_need(A.K, Pn64, host_cap) > (size_t)O.smem_bytes) {
+        if (kBatch && threadIdx.x == 0) {
+            for (int j = 0; j < 7; ++j) A.summary[j] = j == 2 || j == 4 ? -1 : 0;
+            A.summary[7] = G10_DEV_BATCH_UNFIT;
+        }
+        return;
+    }
     const int Pn = (int)Pn64;
     const int G1 = (Pn + 31) / 32;
     const int64_t limit = (A.max_iterations <= 0 || A.max_iterations > Pn64) ? Pn64 : A.max_iterations;
@@ -154,12 +182,40 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
         int over = 0;
 #pragma unroll 1
         for (int k = tid; k < K; k += kOneThreads) {
-            const int64_t pv = A.P[k];
+            const int64_t pv = P_src[k];
             sP[k] = pv;
             if (pv > A.cap) ++over;
         }
+        if (!kBatch) {
 #pragma unroll 1
-        for (int k = tid; k <= K; k += kOneThreads) sStart[k] = A.start[k];
+            for (int k = tid; k <= K; k += kOneThreads) sStart[k] = A.start[k];
+        } else {
+            // slot clock of this variant: exclusive scan of its durations (each thread a run of consecutive kernels);
+            // a duration outside [1, 2^44) counts as 1 and raises the status bit, as in the trace-level pass
+            const int chunk = (K + kOneThreads - 1) / kOneThreads;
+            const int k0 = tid * chunk < K ? tid * chunk : K, k1 = k0 + chunk < K ? k0 + chunk : K;
+            long long sum = 0;
+#pragma unroll 1
+            for (int k = k0; k < k1; ++k) {
+                long long d = var_dur[k];
+                if (d < 1 || d >= ((long long)1 << 44)) { d = 1; dev_bits |= G10_DEV_BAD_DURATION; }
+                sum += d;
+            }
+            const long long incl = warp_inclusive_scan_i64(sum, lane);
+            if (lane == 31) s_pk[warp] = incl;
+            __syncthreads();
+            long long run = incl - sum;
+#pragma unroll 1
+            for (int w = 0; w < warp; ++w) run += s_pk[w];
+#pragma unroll 1
+            for (int k = k0; k < k1; ++k) {
+                long long d = var_dur[k];
+                if (d < 1 || d >= ((long long)1 << 44)) d = 1;
+                sStart[k] = run;
+                run += d;
+            }
+            if (k1 == K) sStart[K] = run;              // every thread at or past the end holds the total
+        }
 #pragma unroll 1
         for (int k = tid; k < (host_cap ? 5 : 4) * K; k += kOneThreads) sBusy[k] = 0;
 #pragma unroll 1
@@ -219,6 +275,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
 #pragma unroll 1
                     for (int X = 0; X < 2 && d < 0; ++X) {
                         if (listed) { ap = s_dirty[j].ap[X]; bp = s_dirty[j].bp[X]; t = s_dirty[j].t[X]; }
+                        else if (kBatch) period_geometry(sStart, a - 1, b + 1, s, bw[X], &t, &ap, &bp);
                         else {
                             ap = __ldg(&A.geo_a[X * A.geo_stride + li]);
                             bp = __ldg(&A.geo_b[X * A.geo_stride + li]);
@@ -463,9 +520,12 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                             e.li = li;
 #pragma unroll
                             for (int Y = 0; Y < 2; ++Y) {
-                                e.ap[Y] = __ldg(&A.geo_a[Y * A.geo_stride + li]);
-                                e.bp[Y] = __ldg(&A.geo_b[Y * A.geo_stride + li]);
-                                e.t[Y] = __ldg(&A.geo_t[Y * A.geo_stride + li]);
+                                if (kBatch) period_geometry(sStart, (int)q.a - 1, (int)q.b + 1, cbytes[li], bw[Y], &e.t[Y], &e.ap[Y], &e.bp[Y]);
+                                else {
+                                    e.ap[Y] = __ldg(&A.geo_a[Y * A.geo_stride + li]);
+                                    e.bp[Y] = __ldg(&A.geo_b[Y * A.geo_stride + li]);
+                                    e.t[Y] = __ldg(&A.geo_t[Y * A.geo_stride + li]);
+                                }
                             }
                             e.pad[0] = e.pad[1] = e.pad[2] = 0;
                             s_dirty[pos] = e;
@@ -481,7 +541,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                     m.period = (int32_t)win; m.tensor = win_tensor; m.dest = X; m.absent_first = wap; m.absent_last = wbp;
                     m.iteration = (int32_t)it; m.evict_issue_ns = t_r; m.prefetch_issue_ns = t_end - t; m.transfer_ns = t;
                     A.out[n_mig] = m;
-                } else raise_status(A.status, G10_DEV_PLAN_OVERFLOW);
+                } else dev_bits |= G10_DEV_PLAN_OVERFLOW;
             }
             n_mig += 1;
             if (X == G10_DEST_SSD) bytes_ssd += s; else bytes_host += s;
@@ -523,18 +583,30 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
         A.summary[0] = n_mig; A.summary[1] = rounds; A.summary[2] = status;
         A.summary[3] = ps < 0 ? 0 : pk; A.summary[4] = ps;
         A.summary[5] = bytes_ssd; A.summary[6] = bytes_host;
-        *O.done = 1u;
+        if (!kBatch) *O.done = 1u;
+    }
+    // status bits found by this block: the batch keeps them per variant, a single plan in the call's status word
+    dev_bits = __reduce_or_sync(0xffffffffu, dev_bits);
+    if (lane == 0) s_fin[warp] = (int)dev_bits;           // (the finalist list is no longer in use)
+    __syncthreads();
+    if (tid == 0) {
+        unsigned bits = 0;
+#pragma unroll 1
+        for (int j = 0; j < kOneWarps; ++j) bits |= (unsigned)s_fin[j];
+        if (kBatch) A.summary[7] = bits;
+        else if (bits) raise_status(A.status, bits);
     }
 }
 
 // Shared memory a launch can offer (opt-in maximum minus the kernel's static part); 0 if the device query fails.
+template <bool kBatch>
 static int one_smem_budget()
 {
     int dev = 0, optin = 0;
     cudaFuncAttributes fa;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
     if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return 0;
-    if (cudaFuncGetAttributes(&fa, (const void *)k_plan_one) != cudaSuccess) return 0;
+    if (cudaFuncGetAttributes(&fa, (const void *)k_plan_one<kBatch>) != cudaSuccess) return 0;
     const int room = optin - (int)fa.sharedSizeBytes;
     return room > 0 ? room : 0;
 }
@@ -544,7 +616,7 @@ static int one_smem_budget()
 bool plan_one_possible(int64_t K, int64_t E, bool host_cap)
 {
     if (K > 65000 || E < 1) return false;
-    const int budget = one_smem_budget();
+    const int budget = one_smem_budget<false>();
     return budget > 0 && one_smem_need(K, E < 512 ? E : 512, host_cap) <= (size_t)budget;
 }
 
@@ -552,11 +624,68 @@ cudaError_t launch_plan_one(const PlanArgs &A_in, const Workspace &w, cudaStream
 {
     PlanArgs A = A_in;
     OneArgs O;
+    BatchArgs B;
+    B.variants = nullptr; B.P0 = nullptr; B.P_out = nullptr;
     O.done = w.one_done;
-    O.smem_bytes = one_smem_budget();
-    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
+    O.smem_bytes = one_smem_budget<false>();
+    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
     if (e != cudaSuccess) return e;
-    k_plan_one<<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O);
+    k_plan_one<false><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Batch: one block per variant, then one block per variant again for the stability pairs.
+// ---------------------------------------------------------------------------------------------
+// stability[v] = (|M_v & M_0|, |M_v | M_0|) over the migrated periods of variant v and of variant 0; (-1, -1) if
+// either plan is missing.  Also folds the call-wide status word (trace validation) into every variant's summary[7].
+__global__ void __launch_bounds__(256) k_batch_finish(int64_t Pn_bound, const int64_t *Pn_dev, const g10_migration *out, int64_t out_cap,
+                                                      int64_t *summary, int64_t *stability, const ull *status)
+{
+    extern __shared__ unsigned s_bits[];
+    __shared__ int s_inter;
+    const int v = blockIdx.x;
+    const int64_t Pn = *Pn_dev < Pn_bound ? *Pn_dev : Pn_bound;
+    const int words = (int)((Pn + 31) / 32);
+    const int64_t n0 = summary[0] < out_cap ? summary[0] : out_cap, nv = summary[v * 8] < out_cap ? summary[v * 8] : out_cap;
+    const bool ok = summary[2] >= 0 && summary[v * 8 + 2] >= 0;
+    if (threadIdx.x == 0) s_inter = 0;
+    for (int j = threadIdx.x; j < words; j += blockDim.x) s_bits[j] = 0;
+    __syncthreads();
+    if (ok) {
+        for (int64_t j = threadIdx.x; j < n0; j += blockDim.x) { const int p = out[j].period; atomicOr(&s_bits[p >> 5], 1u << (p & 31)); }
+        __syncthreads();
+        int mine = 0;
+        const g10_migration *mv = out + (size_t)v * out_cap;
+        for (int64_t j = threadIdx.x; j < nv; j += blockDim.x) { const int p = mv[j].period; mine += (s_bits[p >> 5] >> (p & 31)) & 1u; }
+        mine = __reduce_add_sync(0xffffffffu, mine);
+        if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&s_inter, mine);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        stability[2 * v] = ok ? s_inter : -1;
+        stability[2 * v + 1] = ok ? n0 + nv - s_inter : -1;
+        summary[v * 8 + 7] |= (int64_t)*status;
+    }
+}
+
+int batch_max_periods()          // periods whose bitmap fits the finishing kernel's shared memory
+{
+    return 40 * 1024 * 8;
+}
+
+cudaError_t launch_plan_batch(const PlanArgs &A_in, const Workspace &w, int V, const BatchArgs &B, int64_t *stability, cudaStream_t s)
+{
+    PlanArgs A = A_in;
+    OneArgs O;
+    O.done = w.one_done;
+    O.smem_bytes = one_smem_budget<true>();
+    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
+    if (e != cudaSuccess) return e;
+    k_plan_one<true><<<V, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const int64_t bound = A.geo_stride < batch_max_periods() ? A.geo_stride : batch_max_periods();
+    k_batch_finish<<<V, 256, (size_t)((bound + 31) / 32) * 4, s>>>(bound, A.Pn_dev, A.out, A.out_cap, A.summary, stability, A.status);
     return cudaGetLastError();
 }
 

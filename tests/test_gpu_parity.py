@@ -420,3 +420,62 @@ def test_characterisation_statistics(gpu, oracle):
     check_stats(gpu, oracle, tr)
     # empty trace
     check_stats(gpu, oracle, traces.from_lists("empty", [], [], [], [], capacity_bytes=1))
+
+
+def check_batch(gpu, oracle, tr, variants, max_iterations=0):
+    """Batched re-planning: every variant equals the oracle's plan of the perturbed trace; stability pairs equal."""
+    import torch
+    tb = gpu.upload(tr)
+    dev_variants = []
+    for v in variants:
+        d = dict(v)
+        if v.get("kernel_ns") is not None:
+            d["kernel_ns"] = torch.from_numpy(np.ascontiguousarray(v["kernel_ns"], dtype=np.int64)).cuda()
+        dev_variants.append(d)
+    got = gpu.g10_plan_batch(tb, dev_variants, max_iterations=max_iterations)
+    torch.cuda.synchronize()
+    ref = oracle.plan_batch(tr, variants, max_iterations=max_iterations)
+    summary = _np(got.summary)
+    for j, r in enumerate(ref.plans):
+        assert summary[j, 7] == 0, "variant %d device status %x" % (j, summary[j, 7])
+        assert np.array_equal(summary[j, :7], r.summary[:7]), (j, summary[j], r.summary)
+        assert np.array_equal(gpu.batch_migrations_numpy(got, j), r.migrations), j
+        assert np.array_equal(_np(got.final_pressure)[j, :tr.K], r.final_pressure), j
+    assert np.array_equal(_np(got.stability)[:len(variants)], ref.stability)
+    return ref
+
+
+def _jitter(rng, dur, pct):
+    f = rng.uniform(1.0 - pct / 100.0, 1.0 + pct / 100.0, size=len(dur))
+    return np.maximum(1, np.rint(np.asarray(dur, dtype=np.float64) * f)).astype(np.int64)
+
+
+@pytest.mark.gpu
+def test_batched_replanning(gpu, oracle):
+    rng = np.random.default_rng(4242)
+    for trial in range(12):
+        tr = traces.random_toy(rng, int(rng.integers(1, 40)), int(rng.integers(1, 30)), max_deg=5)
+        start, P0, peak, slot = oracle.timeline(tr)
+        cap = peak * int(rng.integers(1, 10)) // 10
+        base = dict(gpu_capacity_bytes=cap, host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)
+        variants = [base, dict(base, kernel_ns=_jitter(rng, tr.kernel_ns, 25)), dict(base, ssd_bw=tr.ssd_bw * 3),
+                    dict(base, host_capacity_bytes=int(rng.integers(1, 200))), dict(base, gpu_capacity_bytes=cap // 2)]
+        check_batch(gpu, oracle, tr, variants, max_iterations=int(rng.integers(0, 3)) * 2)
+    for cfg in (0, 1, 2):
+        tr = traces.make_config(cfg)
+        start, P0, peak, slot = oracle.timeline(tr)
+        cap = tr.capacity_from_peak(peak)
+        base = dict(gpu_capacity_bytes=cap, host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)
+        variants = [base] + [dict(base, kernel_ns=_jitter(rng, tr.kernel_ns, pct)) for pct in (5, 10, 15, 20, 25)]
+        variants += [dict(base, ssd_bw=bw) for bw in (12_800_000_000, 19_200_000_000, 32_000_000_000)]
+        variants += [dict(base, host_capacity_bytes=hc << 30) for hc in (1, 32, 256)]
+        ref = check_batch(gpu, oracle, tr, variants)
+        assert ref.stability[0, 0] == ref.stability[0, 1] == len(ref.plans[0].migrations)
+    # a trace too large for one SM: every variant says so, nothing else is written
+    import torch
+    tr = traces.make_config(3)
+    tb = gpu.upload(tr)
+    got = gpu.g10_plan_batch(tb, [dict(gpu_capacity_bytes=1 << 30, host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)] * 2)
+    torch.cuda.synchronize()
+    s = _np(got.summary)
+    assert (s[:, 7] & 0x100).all() and (s[:, 2] == -1).all() and (_np(got.stability) == -1).all()
