@@ -92,6 +92,35 @@ __device__ __forceinline__ bool window_free(const PlanArgs &A, const int64_t *bu
     return __all_sync(0xffffffffu, ok);
 }
 
+// A window [w0, w1) over slots wk0..wk1 is booked on a channel.  Can another window [q0, q1) over slots qk0..qk1,
+// admissible before, still be booked on it?  Only slots of both windows matter.  A slot strictly inside the booking is
+// full (it takes the slot's whole duration) and every slot of q's range needs time; so q survives only if the ranges
+// meet in the booking's first / last slot alone and the sums still fit there.
+// kBooked: `busy` already includes the booking (else its share of the slot is added here).  kL2: read busy at L2.
+template <bool kBooked, bool kL2>
+__device__ __forceinline__ bool window_conflict(const int64_t *start, const int64_t *busy, int wk0, int wk1, int64_t w0, int64_t w1,
+                                                int64_t q0, int64_t q1, int qk0, int qk1)
+{
+    const int i0 = qk0 > wk0 ? qk0 : wk0, i1 = qk1 < wk1 ? qk1 : wk1;
+    if (i0 > i1) return false;
+    if ((i0 > wk0 + 1 ? i0 : wk0 + 1) <= (i1 < wk1 - 1 ? i1 : wk1 - 1)) return true;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int k = e == 0 ? i0 : i1;
+        if (e == 1 && i1 == i0) break;
+        const int64_t s0 = start[k], s1 = start[k + 1];
+        const int64_t lo = q0 > s0 ? q0 : s0, hi = q1 < s1 ? q1 : s1;
+        int64_t need = hi > lo ? hi - lo : 0;
+        if (!kBooked) {
+            const int64_t wl = w0 > s0 ? w0 : s0, wh = w1 < s1 ? w1 : s1;
+            need += wh > wl ? wh - wl : 0;
+        }
+        const int64_t booked = kL2 ? __ldcg(&busy[k]) : busy[k];
+        if (booked + need > s1 - s0) return true;
+    }
+    return false;
+}
+
 // Scores period p against the current state: destination (SSD first, then host) and benefit.
 // Whole warp; result valid in lane 0.  Returns false if no destination is admissible (permanent).
 __device__ __forceinline__ bool score_period(const PlanArgs &A, int64_t p, int lane, Cand *out)

@@ -63,28 +63,6 @@ __device__ __forceinline__ bool window_free_one(const int64_t *sStart, const int
     return __all_sync(0xffffffffu, ok);
 }
 
-// A window [w0, w1) over slots wk0..wk1 was just booked on a channel (`busy` already includes it).  Can another
-// window [q0, q1) over slots qk0..qk1, admissible before, still be booked on it?  Only slots of both windows matter.
-// A slot strictly inside the new booking is full (it took the slot's whole duration), and every slot of q's range
-// needs time; so q survives only if the ranges meet in the booking's first / last slot alone and the sums still fit.
-__device__ __forceinline__ bool window_conflict(const int64_t *sStart, const int64_t *busy, int wk0, int wk1, int64_t q0, int64_t q1,
-                                                int qk0, int qk1)
-{
-    const int i0 = qk0 > wk0 ? qk0 : wk0, i1 = qk1 < wk1 ? qk1 : wk1;
-    if (i0 > i1) return false;
-    if ((i0 > wk0 + 1 ? i0 : wk0 + 1) <= (i1 < wk1 - 1 ? i1 : wk1 - 1)) return true;
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-        const int k = e == 0 ? i0 : i1;
-        if (e == 1 && i1 == i0) break;
-        const int64_t s0 = sStart[k], s1 = sStart[k + 1];
-        const int64_t lo = q0 > s0 ? q0 : s0, hi = q1 < s1 ? q1 : s1;
-        const int64_t ov = hi > lo ? hi - lo : 0;
-        if (busy[k] + ov > s1 - s0) return true;
-    }
-    return false;
-}
-
 __host__ __device__ inline size_t one_smem_need(int64_t K, int64_t Pn, bool host_cap)
 {
     const int64_t groups = (Pn + 31) / 32;
@@ -508,8 +486,8 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                     if (meet_out || meet_in) {
                         const int64_t tq = ct[li];
                         const int64_t q_r = sStart[q.a], q_end = sStart[(int)q.b + 1];
-                        hit = (meet_out && window_conflict(sStart, bo, wa, wap - 1, q_r, q_r + tq, q.a, (int)q.ap - 1)) ||
-                              (meet_in && window_conflict(sStart, bi, wbp + 1, wb, q_end - tq, q_end, (int)q.bp + 1, q.b));
+                        hit = (meet_out && window_conflict<true, false>(sStart, bo, wa, wap - 1, 0, 0, q_r, q_r + tq, q.a, (int)q.ap - 1)) ||
+                              (meet_in && window_conflict<true, false>(sStart, bi, wbp + 1, wb, 0, 0, q_end - tq, q_end, (int)q.bp + 1, q.b));
                     }
                     if (!hit && d == G10_DEST_HOST && host_cap) hit = true;
                     if (hit) {

@@ -453,6 +453,36 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             const int wa = win.wa, wb = win.wb, wap = win.wap, wbp = win.wbp;
             const int64_t s = win.bytes, t = win.t;
             const int64_t t_r = sStart[wa], t_end = sStart[wb + 1];
+            int64_t *bo = busy + (size_t)(2 * X) * K, *bi = busy + (size_t)(2 * X + 1) * K;
+            // reclassify this block's periods against the winner's slot ranges; the bookings are not in `busy` yet
+            // (the sums of the two shared boundary slots are formed here), so this runs before they are added
+#pragma unroll 1
+            for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
+                const unsigned char st = cstate[li];
+                if (st == 0) continue;
+                if ((int64_t)li * G + c == p) { cstate[li] = 0; continue; }
+                int state = st >> 2;
+                if (state == kDirtyS) continue;
+                const int d = (st & 3) - 1;
+                const int qa = info[li].a, qb = info[li].b;
+                if (!(qa <= wb && wa <= qb)) continue;
+                const int ap = info[li].ap[d], bp = info[li].bp[d];
+                bool hit = false;
+                if (d == X) {
+                    const bool meet_out = qa <= wap - 1 && wa <= ap - 1, meet_in = bp + 1 <= wb && wbp + 1 <= qb;
+                    if (meet_out || meet_in) {
+                        const int64_t tq = info[li].t[d];
+                        const int64_t q_r = sStart[qa], q_end = sStart[qb + 1];
+                        hit = (meet_out && window_conflict<false, true>(sStart, bo, wa, wap - 1, t_r, t_r + t, q_r, q_r + tq, qa, ap - 1)) ||
+                              (meet_in && window_conflict<false, true>(sStart, bi, wbp + 1, wb, t_end - t, t_end, q_end - tq, q_end, bp + 1, qb));
+                    }
+                    if (!hit && d == G10_DEST_HOST && A.host_capacity != 0) hit = true;
+                }
+                if (hit) state = kDirtyS;
+                else if (state == kFreshS && ap <= wbp && wap <= bp) state = kStaleS;
+                cstate[li] = (unsigned char)((st & 3) | (state << 2));
+            }
+            __syncthreads();
             int fell = 0;
 #pragma unroll 1
             for (int k = wap + threadIdx.x; k <= wbp; k += kPlanThreads) {
@@ -461,7 +491,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                 if (before > A.cap && after <= A.cap) ++fell;
             }
             if (fell) atomicSub(&s_n_over, fell);
-            int64_t *bo = busy + (size_t)(2 * X) * K, *bi = busy + (size_t)(2 * X + 1) * K;
 #pragma unroll 1
             for (int k = wa + threadIdx.x; k <= wap - 1; k += kPlanThreads) {
                 const int64_t s0 = sStart[k], s1 = sStart[k + 1];
@@ -477,27 +506,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             if (X == G10_DEST_HOST && A.host_capacity != 0)
 #pragma unroll 1
                 for (int k = wa + threadIdx.x; k <= wb; k += kPlanThreads) atomicAdd((ull *)&hocc[k], (ull)s);
-            // reclassify this block's periods against the winner's slot ranges
-#pragma unroll 1
-            for (int li = threadIdx.x; li < n_local; li += kPlanThreads) {
-                const unsigned char st = cstate[li];
-                if (st == 0) continue;
-                if ((int64_t)li * G + c == p) { cstate[li] = 0; continue; }
-                int state = st >> 2;
-                if (state == kDirtyS) continue;
-                const int d = (st & 3) - 1;
-                const int qa = info[li].a, qb = info[li].b;
-                if (!(qa <= wb && wa <= qb)) continue;
-                const int ap = info[li].ap[d], bp = info[li].bp[d];
-                bool hit = false;
-                if (d == X) {
-                    hit = (qa <= wap - 1 && wa <= ap - 1) || (bp + 1 <= wb && wbp + 1 <= qb);
-                    if (!hit && d == G10_DEST_HOST && A.host_capacity != 0) hit = true;
-                }
-                if (hit) state = kDirtyS;
-                else if (state == kFreshS && ap <= wbp && wap <= bp) state = kStaleS;
-                cstate[li] = (unsigned char)((st & 3) | (state << 2));
-            }
             if (c == 0 && threadIdx.x == 0) {
                 if (n_mig < A.out_cap) {
                     g10_migration m;
