@@ -94,6 +94,10 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.geo_b = c.take<int32_t>(2 * E);
     w.proposals = c.take<Proposal>(kMaxPlanBlocks);
     w.prop_stale = c.take<Proposal>(kMaxPlanBlocks);
+    w.lazy_props = c.take<LazyProp>(2 * kLazyMaxBlocks);
+    w.lazy_partials = c.take<ull>((size_t)2 * kRoundM * kLazyMaxBlocks * 2);
+    w.lazy_tmin = c.take<int64_t>((size_t)tiles_of(z.K, 1024));
+    w.lazy_tmax = c.take<int64_t>((size_t)tiles_of(z.K, 1024));
     w.c_state = c.take<unsigned char>(E);
     w.c_ben_lo = c.take<ull>(E);
     w.c_ben_hi = c.take<ull>(E);

@@ -33,6 +33,20 @@ struct Proposal {          // a block's best candidate of one scoring round (32 
     int dest;
 };
 
+// Large-trace planner: what a block publishes after a pass over its periods (best FRESH candidate, best STALE
+// bounds) and the sizes of its joint rescoring rounds.
+constexpr int kLazyMaxBlocks = 256;
+constexpr int kTopT = 4;
+constexpr int kRoundM = 256;      // periods rescored together in one round, at most
+constexpr int kDirtyPool = 256;   // DIRTY periods of one commit that join a round (more: rescored at once, shared out)
+constexpr int kFirstM = 8;        // ... in the first round of an iteration (best bounds first)
+struct __align__(16) LazyProp {
+    ull ben_lo, ben_hi, cost;
+    int idx, dest;
+    double skey[kTopT];
+    int sidx[kTopT];
+};
+
 // One variant of a batched re-planning call (device copy of g10_variant with the defaults filled in).
 struct BatchVariant {
     const int64_t *kernel_ns;
@@ -86,6 +100,9 @@ struct Workspace {
     int32_t *geo_a, *geo_b;      // [2*E]
     Proposal *proposals;         // [max blocks]
     Proposal *prop_stale;        // [max blocks]
+    LazyProp *lazy_props;        // [2][kLazyMaxBlocks]
+    ull *lazy_partials;          // [2][kRoundM][kLazyMaxBlocks][2]
+    int64_t *lazy_tmin, *lazy_tmax; // [tiles of 1024 slots]
     unsigned char *c_state;      // [E] per-period state of the lazy planner
     ull *c_ben_lo, *c_ben_hi, *c_cost;   // [E] cached benefit and cost
     double *c_key;               // [E] rounded benefit / cost

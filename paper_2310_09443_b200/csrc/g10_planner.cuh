@@ -272,7 +272,7 @@ __device__ __forceinline__ long long own_slots_max(const PlanArgs &A, int c, int
 // owns, channel bookings, the plan record and the erase flag by block 0.  Returns true if this block's
 // pressure slots changed.
 __device__ __forceinline__ bool commit_winner(const PlanArgs &A, int64_t p, int X, int64_t it, int64_t n_mig, int c, int G,
-                                              int64_t *bytes_out)
+                                              int64_t *bytes_out, bool with_bookings = true)
 {
     const int64_t K = A.K;
     const int i = A.per_t[p], u = A.per_u[p], v = A.per_v[p];
@@ -298,16 +298,18 @@ __device__ __forceinline__ bool commit_winner(const PlanArgs &A, int64_t p, int 
         }
     }
     if (c == 0) {
-        int64_t *bo = A.busy + (size_t)(2 * X) * K, *bi = A.busy + (size_t)(2 * X + 1) * K;
-        for (int k = a + threadIdx.x; k <= ap - 1; k += kPlanThreads) {
-            const int64_t s0 = A.start[k], s1 = A.start[k + 1];
-            const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
-            if (hi > lo) bo[k] += hi - lo;
-        }
-        for (int k = bp + 1 + threadIdx.x; k <= b; k += kPlanThreads) {
-            const int64_t s0 = A.start[k], s1 = A.start[k + 1];
-            const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
-            if (hi > lo) bi[k] += hi - lo;
+        if (with_bookings) {
+            int64_t *bo = A.busy + (size_t)(2 * X) * K, *bi = A.busy + (size_t)(2 * X + 1) * K;
+            for (int k = a + threadIdx.x; k <= ap - 1; k += kPlanThreads) {
+                const int64_t s0 = A.start[k], s1 = A.start[k + 1];
+                const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
+                if (hi > lo) bo[k] += hi - lo;
+            }
+            for (int k = bp + 1 + threadIdx.x; k <= b; k += kPlanThreads) {
+                const int64_t s0 = A.start[k], s1 = A.start[k + 1];
+                const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
+                if (hi > lo) bi[k] += hi - lo;
+            }
         }
         if (threadIdx.x == 0) {
             A.dead[p] = 1;
@@ -321,6 +323,28 @@ __device__ __forceinline__ bool commit_winner(const PlanArgs &A, int64_t p, int 
     }
     *bytes_out = s;
     return touched;
+}
+
+// The channel bookings of a committed period (one block adds them, all its threads).
+__device__ __forceinline__ void book_winner(const PlanArgs &A, int64_t p, int X)
+{
+    const int64_t K = A.K;
+    const int u = A.per_u[p], v = A.per_v[p];
+    const int a = u + 1, b = v - 1;
+    const int ap = A.geo_a[X * A.geo_stride + p], bp = A.geo_b[X * A.geo_stride + p];
+    const int64_t t = A.geo_t[X * A.geo_stride + p];
+    const int64_t t_r = A.start[a], t_end = A.start[v];
+    int64_t *bo = A.busy + (size_t)(2 * X) * K, *bi = A.busy + (size_t)(2 * X + 1) * K;
+    for (int k = a + threadIdx.x; k <= ap - 1; k += kPlanThreads) {
+        const int64_t s0 = A.start[k], s1 = A.start[k + 1];
+        const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
+        if (hi > lo) bo[k] += hi - lo;
+    }
+    for (int k = bp + 1 + threadIdx.x; k <= b; k += kPlanThreads) {
+        const int64_t s0 = A.start[k], s1 = A.start[k + 1];
+        const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
+        if (hi > lo) bi[k] += hi - lo;
+    }
 }
 
 // Final peak slot (lowest slot holding the peak) and the summary words.  Every block calls it.

@@ -9,17 +9,19 @@
 //   DIRTY  a later commit booked channel time (or host memory) inside one of its transfer windows: its
 //          destination has to be chosen again before anything can be said.
 // After a commit every block classifies the periods it owns against the winner's slot ranges (a few integer
-// comparisons each).  DIRTY periods are rescored at once; a STALE period is rescored only while its bound may
-// still beat the best exact score known, so that when the iteration decides, the committed score is the exact
-// maximum over all live periods, ties included (see k_plan_lazy).
+// comparisons each; whether a booked window still leaves another window of the same channel free is decided in
+// constant time).  DIRTY periods are rescored at once; a STALE period is rescored only while its bound may still
+// beat the best exact score known to the whole grid, and then by the whole grid together (absent ranges of the
+// best candidates span a large part of a long timeline), so that when the iteration decides, the committed score
+// is the exact maximum over all live periods, ties included (see k_plan_lazy).
 #include <cstdio>
 
 #include "g10_planner.cuh"
 
 namespace g10 {
 
-constexpr int kLazyMaxBlocks = 256;
 enum { kFresh = 1, kStale = 2, kDirty = 3 };
+constexpr int kMixCap = 1024;            // tiles of one round that a block reads slot by slot, listed
 
 struct LazyArgs {
     unsigned char *c_state;     // 0 = erased; else (dest + 1) | (state << 2)
@@ -28,7 +30,9 @@ struct LazyArgs {
     double *c_key;              // rounded benefit / cost of the cached score (steers the search; decisions are exact)
     int *worklist;              // [2][stride] DIRTY periods of the current round
     unsigned *wl_count;         // [2]
-    Proposal *prop_stale;       // [G] each block's exact best of step C (second proposal buffer)
+    LazyProp *props;            // [2][kLazyMaxBlocks] each block's best FRESH candidate and best STALE bounds
+    ull *partials;              // [2][kRoundM][kLazyMaxBlocks][2] slices of the benefits rescored together
+    int64_t *tmin, *tmax;       // [tiles of kSlotTile slots] smallest / largest pressure of each tile
     int64_t stride;
 };
 
@@ -40,6 +44,31 @@ __device__ __forceinline__ u128 benefit_partial(const PlanArgs &A, int ap, int b
         if (ex > 0) {
             if (ex > s) ex = s;
             acc += (u128)(ull)ex * (u128)(ull)A.dur[k];
+        }
+    }
+    return acc;
+}
+
+// The same sum for one tile read by one warp: eight slots per lane in flight (the tile comes from L2).
+__device__ __forceinline__ u128 benefit_tile_warp(const PlanArgs &A, int k_lo, int k_hi, int64_t s, int lane)
+{
+    u128 acc = 0;
+#pragma unroll 1
+    for (int k0 = k_lo + lane; k0 <= k_hi; k0 += 8 * 32) {
+        int64_t ex[8], du[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int k = k0 + 32 * j;
+            ex[j] = k <= k_hi ? A.P[k] : 0;
+            du[j] = k <= k_hi ? A.dur[k] : 0;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            int64_t e = ex[j] - A.cap;
+            if (k0 + 32 * j <= k_hi && e > 0) {
+                if (e > s) e = s;
+                acc += (u128)(ull)e * (u128)(ull)du[j];
+            }
         }
     }
     return acc;
@@ -72,6 +101,42 @@ __device__ __forceinline__ void eval_warp(const PlanArgs &A, const LazyArgs &L, 
     const int64_t s = A.bytes[A.per_t[p]];
     u128 acc = warp_sum_u128(benefit_partial(A, ap, bp, s, lane, 32));
     if (lane == 0) store_score(L, p, d, kFresh, acc, 2ull * (ull)A.geo_t[d * A.geo_stride + p]);
+}
+
+// One warp re-chooses the destination of DIRTY period p (SSD first, then host).  The period is erased if no
+// destination is left; otherwise it becomes STALE with an unbounded score, so that it is rescored with the others.
+__device__ __forceinline__ void dest_warp(const PlanArgs &A, const LazyArgs &L, int64_t p, int lane)
+{
+    if (L.c_state[p] == 0) return;
+    const int u = A.per_u[p], v = A.per_v[p];
+    const int a = u + 1, b = v - 1;
+    const int64_t s = A.bytes[A.per_t[p]];
+    const int64_t t_r = A.start[a], t_end = A.start[v];
+    int dest = -1;
+    int64_t t = 0;
+    for (int X = 0; X < 2 && dest < 0; ++X) {
+        const int ap = A.geo_a[X * A.geo_stride + p];
+        if (ap < 0) continue;
+        const int bp = A.geo_b[X * A.geo_stride + p];
+        t = A.geo_t[X * A.geo_stride + p];
+        if (!window_free(A, A.busy + (size_t)(2 * X) * A.K, t_r, t_r + t, a, ap - 1, lane)) continue;
+        if (!window_free(A, A.busy + (size_t)(2 * X + 1) * A.K, t_end - t, t_end, bp + 1, b, lane)) continue;
+        if (X == G10_DEST_HOST && A.host_capacity != 0) {
+            bool ok = true;
+            for (int k = a + lane; k <= b; k += 32)
+                if ((uint64_t)A.hocc[k] + (uint64_t)s > A.host_capacity) ok = false;
+            if (!__all_sync(0xffffffffu, ok)) continue;
+        }
+        dest = X;
+    }
+    if (lane == 0) {
+        if (dest < 0) L.c_state[p] = 0;
+        else {
+            L.c_ben_lo[p] = 0; L.c_ben_hi[p] = 0; L.c_cost[p] = 2ull * (ull)t;
+            L.c_key[p] = __longlong_as_double(0x7ff0000000000000ll);      // +infinity: rescored before anything is decided
+            L.c_state[p] = (unsigned char)((dest + 1) | (kStale << 2));
+        }
+    }
 }
 
 // The whole block brings period p up to date (long absent ranges).
@@ -124,24 +189,124 @@ __device__ __forceinline__ void eval_block(const PlanArgs &A, const LazyArgs &L,
     }
 }
 
-__device__ __forceinline__ Cand load_proposal(const Proposal *pr)
+// Smallest and largest pressure of slot tile tl, recomputed by the whole block (the tile's owner).
+__device__ __forceinline__ void tile_minmax(const PlanArgs &A, const LazyArgs &L, int tl, long long *s_red /* [2 * kPlanWarps] */)
 {
-    Cand x;
-    const ull lo = __ldcg(&pr->ben_lo), hi = __ldcg(&pr->ben_hi);
-    x.ben = ((u128)hi << 64) | lo;
-    x.cost = __ldcg(&pr->cost);
-    x.idx = __ldcg(&pr->idx);
-    x.dest = __ldcg(&pr->dest);
-    return x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t k0 = (int64_t)tl * kSlotTile;
+    long long mn = 0x7fffffffffffffffll, mx = -0x7fffffffffffffffll - 1;
+    for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < A.K; k += kPlanThreads) {
+        const long long pv = A.P[k];
+        if (pv < mn) mn = pv;
+        if (pv > mx) mx = pv;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long a = __shfl_xor_sync(0xffffffffu, mn, o), b = __shfl_xor_sync(0xffffffffu, mx, o);
+        if (a < mn) mn = a;
+        if (b > mx) mx = b;
+    }
+    __syncthreads();
+    if (lane == 0) { s_red[2 * warp] = mn; s_red[2 * warp + 1] = mx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kPlanWarps; ++w) { if (s_red[2 * w] < mn) mn = s_red[2 * w]; if (s_red[2 * w + 1] > mx) mx = s_red[2 * w + 1]; }
+        L.tmin[tl] = mn; L.tmax[tl] = mx;
+    }
 }
-__device__ __forceinline__ void store_proposal(Proposal *pr, const Cand &c)
+
+// Largest pressure over the tiles this block owns (tiles c, c + G, ...), from the tile maxima.
+__device__ __forceinline__ long long own_tiles_max(const PlanArgs &A, const LazyArgs &L, int c, int G, long long *s_tmp)
 {
-    Proposal q;
+    const int n_slot_tiles = (int)((A.K + kSlotTile - 1) / kSlotTile);
+    long long m = 0;
+    for (int tl = c + (int)threadIdx.x * G; tl < n_slot_tiles; tl += kPlanThreads * G) {
+        const long long x = L.tmax[tl];
+        if (x > m) m = x;
+    }
+    return block_max_i64(m, s_tmp);
+}
+
+// Commits period p with destination X on what this block owns: the pressure slots of its tiles (with their new
+// minima / maxima) and host occupancy; block 0 also writes the plan record and the erase flag.  The channel
+// bookings are added later (book_winner).  Returns true if a tile of this block changed.
+__device__ __forceinline__ bool commit_lazy(const PlanArgs &A, const LazyArgs &L, int64_t p, int X, int64_t it, int64_t n_mig, int c, int G,
+                                            long long *s_red)
+{
+    const int64_t K = A.K;
+    const int i = A.per_t[p], u = A.per_u[p], v = A.per_v[p];
+    const int a = u + 1, b = v - 1;
+    const int64_t s = A.bytes[i];
+    const int ap = A.geo_a[X * A.geo_stride + p], bp = A.geo_b[X * A.geo_stride + p];
+    const int64_t t = A.geo_t[X * A.geo_stride + p];
+    bool touched = false;
+    {
+        const int ta = ap / kSlotTile, tb = bp / kSlotTile;
+        int tl = ta + ((c - ta % G) % G + G) % G;            // first tile >= ta that this block owns
+        for (; tl <= tb; tl += G) {
+            touched = true;
+            const int64_t k0 = (int64_t)tl * kSlotTile;
+            for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < K; k += kPlanThreads)
+                if (k >= ap && k <= bp) A.P[k] -= s;
+            __syncthreads();
+            tile_minmax(A, L, tl, s_red);
+        }
+    }
+    if (X == G10_DEST_HOST && A.host_capacity != 0) {
+        const int ta = a / kSlotTile, tb = b / kSlotTile;
+        int tl = ta + ((c - ta % G) % G + G) % G;
+        for (; tl <= tb; tl += G) {
+            const int64_t k0 = (int64_t)tl * kSlotTile;
+            for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < K; k += kPlanThreads)
+                if (k >= a && k <= b) A.hocc[k] += s;
+        }
+    }
+    if (c == 0 && threadIdx.x == 0) {
+        A.dead[p] = 1;
+        if (n_mig < A.out_cap) {
+            g10_migration m;
+            m.period = (int32_t)p; m.tensor = i; m.dest = X; m.absent_first = ap; m.absent_last = bp;
+            m.iteration = (int32_t)it; m.evict_issue_ns = A.start[a]; m.prefetch_issue_ns = A.start[v] - t; m.transfer_ns = t;
+            A.out[n_mig] = m;
+        } else raise_status(A.status, G10_DEV_PLAN_OVERFLOW);
+    }
+    return touched;
+}
+
+// This block's share of the benefit of absent range [ap, bp] for a tensor of s bytes: tiles ta + c, ta + c + G, ...
+// of the range, one warp.  A tile whose smallest pressure is at least capacity + s counts s for its whole time,
+// one whose largest pressure is within capacity counts nothing; only the others are read slot by slot.
+__device__ __forceinline__ u128 benefit_tiles(const PlanArgs &A, const LazyArgs &L, int ap, int bp, int64_t s, int c, int G, int lane)
+{
+    u128 acc = 0;
+    const int ta = ap / kSlotTile, tb = bp / kSlotTile;
+    for (int tl = ta + c; tl <= tb; tl += G) {
+        const int64_t t0 = (int64_t)tl * kSlotTile, t1 = t0 + kSlotTile - 1;
+        const int k_lo = (int)(t0 > ap ? t0 : ap), k_hi = (int)(t1 < bp ? t1 : bp);
+        const long long mn = L.tmin[tl], mx = L.tmax[tl];
+        if (mx <= A.cap) continue;
+        if (mn >= A.cap && mn - A.cap >= s) {
+            if (lane == 0) acc += (u128)(ull)s * (u128)(ull)(A.start[k_hi + 1] - A.start[k_lo]);
+            continue;
+        }
+        acc += benefit_partial(A, k_lo, k_hi, s, lane, 32);
+    }
+    return acc;
+}
+
+// What a block tells the grid after a pass over its periods: its best FRESH candidate (exact) and its kTopT best
+// STALE bounds (rounded ratio and period, descending; idx < 0 = none).  Any STALE period it did not list has a
+// bound no larger than the last one listed.
+__device__ __forceinline__ void store_prop(LazyProp *pr, const Cand &c, const double *tk, const int *ti)
+{
+    LazyProp q;
     q.ben_lo = (ull)c.ben; q.ben_hi = (ull)(c.ben >> 64); q.cost = c.cost; q.idx = c.idx; q.dest = c.dest;
+#pragma unroll
+    for (int j = 0; j < kTopT; ++j) { q.skey[j] = tk[j]; q.sidx[j] = ti[j]; }
     *pr = q;
 }
 
-// Best STALE bound of the block by rounded ratio (any of several equal ones): uniform result.
+// Block-wide maximum of (key, idx), larger idx on equal keys: uniform result.
 __device__ __forceinline__ void block_max_key(double &k, int &idx, double *s_k /* [kPlanWarps] */, int *s_i /* [kPlanWarps] */)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -162,43 +327,70 @@ __device__ __forceinline__ void block_max_key(double &k, int &idx, double *s_k /
     }
 }
 
-// One pass of a block over the periods it owns.  With `classify` the pending winner's slot ranges are applied
-// first (FRESH -> STALE where its absent range meets theirs, -> DIRTY where a booked window meets theirs) and
-// DIRTY periods are appended to the work list.  Returns the block's best FRESH candidate (exact) and its best
-// STALE bound (rounded ratio and period, approximate on purpose: it only says what to rescore next).
-struct ScanResult {
-    Cand bestF;
-    double keyS;
-    int idxS;
-};
+// Can STALE period p, whose cached score (rounded ratio `key`) bounds its current one, still beat candidate t
+// (rounded ratio t_key)?  Clear cases by the rounded ratios, anything within 1e-10 by the exact comparison of the
+// cached benefit and cost (a tie goes to the lower period index, as in the final decision).
+__device__ __forceinline__ bool bound_may_beat(const LazyArgs &L, int p, double key, double t_key, const Cand *t)
+{
+    if (!(key > 0.0)) return false;
+    if (!t || t->idx < 0) return true;
+    if (key > t_key * (1.0 + 1e-10)) return true;
+    if (key < t_key * (1.0 - 1e-10)) return false;
+    Cand x;
+    x.ben = ((u128)__ldcg(&L.c_ben_hi[p]) << 64) | __ldcg(&L.c_ben_lo[p]); x.cost = __ldcg(&L.c_cost[p]); x.idx = p; x.dest = 0;
+    return cand_beats(x, *t);
+}
 
 struct Winner {
     int idx, dest, a, ap, bp, b;      // evict slots [a, ap-1], absent [ap, bp], prefetch [bp+1, b]
+    int64_t t, t_r, t_end;            // transfer time, start of the eviction, end of the prefetch
 };
 
-__device__ __forceinline__ ScanResult scan_owned(const PlanArgs &A, const LazyArgs &L, int64_t Pn, bool classify, const Winner &w,
-                                                 int par, BestScratch *sc, Cand *s_cand, double *s_k, int *s_i)
+// One pass of a block over the periods it owns (period p belongs to block (p / kPlanThreads) mod G).  With
+// `classify` the pending winner's slot ranges are applied first (FRESH -> STALE where its absent range meets
+// theirs, -> DIRTY where its booking leaves one of their transfer windows no room; the bookings are not in
+// A.busy yet) and DIRTY periods are appended to the work list.  Returns the block's best FRESH candidate (exact)
+// and leaves its kTopT best STALE bounds in s_tk / s_ti (uniform).
+__device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L, int64_t Pn, bool classify, const Winner &w,
+                                           int par, BestScratch *sc, Cand *s_cand, double *s_k, int *s_i, double *s_tk, int *s_ti,
+                                           const Cand *floor = nullptr)
 {
+    // with a floor (the best exact score known to the grid) only the STALE bounds that can beat it are listed
+    const double floor_key = floor && floor->idx >= 0 ? cand_key(*floor) : -1.0;
     const int G = gridDim.x, c = blockIdx.x, lane = threadIdx.x & 31;
-    double kf = -1.0, ks = -1.0;
-    int pf = -1, ps = -1;
+    double kf = -1.0;
+    int pf = -1;
+    double tk[kTopT];
+    int ti[kTopT];
+#pragma unroll
+    for (int j = 0; j < kTopT; ++j) { tk[j] = -1.0; ti[j] = -1; }
+    const int64_t *bo = A.busy + (size_t)(2 * (w.dest < 0 ? 0 : w.dest)) * A.K, *bi = bo + A.K;
     for (int64_t p0 = (int64_t)c * kPlanThreads; p0 < Pn; p0 += (int64_t)G * kPlanThreads) {
         const int64_t p = p0 + threadIdx.x;
         bool dirty = false;
         if (p < Pn) {
             unsigned char st = L.c_state[p];
+            // (independent loads issued together: the pass is a chain of L2 latencies otherwise)
+            const double key_ld = L.c_key[p];
+            int u = 0, v = 0;
+            if (classify) { u = A.per_u[p]; v = A.per_v[p]; }
             if (st != 0) {
                 int state = st >> 2;
                 const int d = (st & 3) - 1;
                 if (classify) {
                     if (p == w.idx) { L.c_state[p] = 0; st = 0; }
                     else if (state != kDirty) {
-                        const int u = A.per_u[p], v = A.per_v[p];
                         if (u + 1 <= w.b && w.a <= v - 1) {          // the two periods share slots
                             const int ap = A.geo_a[d * A.geo_stride + p], bp = A.geo_b[d * A.geo_stride + p];
                             bool hit = false;
                             if (d == w.dest) {
-                                hit = (u + 1 <= w.ap - 1 && w.a <= ap - 1) || (bp + 1 <= w.b && w.bp + 1 <= v - 1);
+                                const bool meet_out = u + 1 <= w.ap - 1 && w.a <= ap - 1, meet_in = bp + 1 <= w.b && w.bp + 1 <= v - 1;
+                                if (meet_out || meet_in) {
+                                    const int64_t tq = A.geo_t[d * A.geo_stride + p];
+                                    const int64_t q_r = A.start[u + 1], q_end = A.start[v];
+                                    hit = (meet_out && window_conflict<false, true>(A.start, bo, w.a, w.ap - 1, w.t_r, w.t_r + w.t, q_r, q_r + tq, u + 1, ap - 1)) ||
+                                          (meet_in && window_conflict<false, true>(A.start, bi, w.bp + 1, w.b, w.t_end - w.t, w.t_end, q_end - tq, q_end, bp + 1, v - 1));
+                                }
                                 if (!hit && d == G10_DEST_HOST && A.host_capacity != 0) hit = true;
                             }
                             if (hit) state = kDirty;
@@ -210,7 +402,7 @@ __device__ __forceinline__ ScanResult scan_owned(const PlanArgs &A, const LazyAr
                 if (st != 0) {
                     if (state == kDirty) dirty = true;
                     else {
-                        const double key = L.c_key[p];
+                        const double key = key_ld;
                         if (key > 0.0) {
                             if (state == kFresh) {
                                 bool take = key > kf;
@@ -221,7 +413,14 @@ __device__ __forceinline__ ScanResult scan_owned(const PlanArgs &A, const LazyAr
                                     take = cand_beats(x, y);
                                 }
                                 if (take) { kf = key; pf = (int)p; }
-                            } else if (key > ks) { ks = key; ps = (int)p; }
+                            } else if (key > tk[kTopT - 1] && bound_may_beat(L, (int)p, key, floor_key, floor)) {
+                                // insertion into this thread's sorted best STALE bounds
+                                int j = kTopT - 1;
+#pragma unroll
+                                for (int q = kTopT - 1; q > 0; --q)
+                                    if (j == q && key > tk[q - 1]) { tk[q] = tk[q - 1]; ti[q] = ti[q - 1]; j = q - 1; }
+                                tk[j] = key; ti[j] = (int)p;
+                            }
                         }
                     }
                 }
@@ -238,17 +437,28 @@ __device__ __forceinline__ ScanResult scan_owned(const PlanArgs &A, const LazyAr
             }
         }
     }
-    ScanResult r;
     Cand x;
     x.ben = 0; x.cost = 1; x.idx = -1; x.dest = -1;
     if (pf >= 0) {
         x.ben = ((u128)L.c_ben_hi[pf] << 64) | L.c_ben_lo[pf]; x.cost = L.c_cost[pf]; x.idx = pf;
         x.dest = (L.c_state[pf] & 3) - 1;
     }
-    r.bestF = block_best_fast(x, sc, s_cand);
-    block_max_key(ks, ps, s_k, s_i);
-    r.keyS = ks; r.idxS = ps;
-    return r;
+    const Cand bestF = block_best_fast(x, sc, s_cand);
+    // the block's kTopT best bounds: kTopT rounds of block-wide maximum over the threads' current heads
+#pragma unroll 1
+    for (int r = 0; r < kTopT; ++r) {
+        double k = tk[0];
+        int idx = ti[0];
+        block_max_key(k, idx, s_k, s_i);
+        if (idx >= 0 && idx == ti[0]) {                 // this thread's head was taken: next one moves up
+#pragma unroll
+            for (int q = 0; q < kTopT - 1; ++q) { tk[q] = tk[q + 1]; ti[q] = ti[q + 1]; }
+            tk[kTopT - 1] = -1.0; ti[kTopT - 1] = -1;
+        }
+        if (threadIdx.x == 0) { s_tk[r] = idx >= 0 ? k : -1.0; s_ti[r] = idx; }
+    }
+    __syncthreads();
+    return bestF;
 }
 
 // Could a STALE bound with rounded ratio `key` beat (or tie with) candidate t?  Conservative by 1e-10.
@@ -259,22 +469,47 @@ __device__ __forceinline__ bool may_beat(double key, const Cand &t)
     return key >= cand_key(t) * (1.0 - 1e-10);
 }
 
-// Per iteration: (A) every block applies the previous commit to the slots it owns, classifies the periods it
-// owns and finds its best FRESH candidate and best STALE bound; (B) after the first grid barrier every block
-// knows the best FRESH score of the grid: DIRTY periods are rescored (shared out over the grid) and each block
-// rescores its own best STALE period if the bound may beat that score; (C) each block then makes its own best
-// exact -- it rescores its STALE periods, best bound first, while the bound may beat the better of the grid's
-// FRESH score and its own best; (D) after the last barrier the maximum of the blocks' exact bests is the exact
-// maximum over all live periods (every period left STALE has a bound below its block's best) and is committed.
+// Per iteration:
+//  A  every block applies the previous commit to the pressure slots it owns, classifies the periods it owns
+//     and publishes its best FRESH candidate and its kTopT best STALE bounds; grid barrier;
+//  B  every block reads all publications: the best FRESH score of the grid, the peak, the stop tests; block 0
+//     adds the previous commit's bookings; DIRTY periods, if any, are rescored (shared out over the grid) and
+//     everything is published again;
+//  R  rounds: the (at most kRoundM) best published bounds that may still beat the best exact score are rescored
+//     by the whole grid together -- every block sums its slice of each absent range, a barrier, every block adds
+//     up the slices -- and the best exact score is updated; a block whose published bounds are used up while the
+//     last of them may still beat the best score looks again and publishes more;
+//  D  no bound left that may beat it: the best exact score is the exact maximum over all live periods; commit.
+// All decisions are taken from data every block has, so the control flow is the same in every block.
 __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyArgs L)
 {
     __shared__ Cand s_cand[kPlanWarps + 1];
     __shared__ BestScratch s_best;
-    __shared__ long long s_max[kPlanWarps + 1];
+    __shared__ long long s_max[2 * kPlanWarps + 1];
     __shared__ double s_k[kPlanWarps];
     __shared__ int s_i[kPlanWarps];
     __shared__ int s_dest;
     __shared__ ull s_part[2 * kPlanWarps];
+    __shared__ double s_tk[kTopT];
+    __shared__ int s_ti[kTopT];
+    __shared__ double s_pkey[kLazyMaxBlocks * kTopT];      // published bounds of all blocks
+    __shared__ int s_pidx[kLazyMaxBlocks * kTopT];
+    __shared__ unsigned char s_pdone[kLazyMaxBlocks * kTopT];
+    __shared__ int s_sel[kRoundM];
+    __shared__ Cand s_new[kRoundM];
+    __shared__ int s_wcnt[kPlanWarps];
+    __shared__ int s_it_d[kRoundM], s_it_ap[kRoundM], s_it_bp[kRoundM];
+    __shared__ long long s_it_s[kRoundM];
+    __shared__ ull s_it_cost[kRoundM];
+    __shared__ ull s_acc[2 * kRoundM];
+    __shared__ int s_mix[kMixCap];
+    __shared__ int s_nmix;
+    __shared__ int s_flag;
+#ifdef G10_PHASE_CLOCKS
+    __shared__ ull s_dbg_slots, s_dbg_mixed, s_dbg_tiles, s_dbg_over;
+    if (threadIdx.x == 0) { s_dbg_slots = 0; s_dbg_mixed = 0; s_dbg_tiles = 0; s_dbg_over = 0; }
+#endif
+    __shared__ unsigned char s_refresh[kLazyMaxBlocks];
     const int G = gridDim.x, c = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t Pn = *A.Pn_dev < A.geo_stride ? *A.Pn_dev : A.geo_stride;
@@ -284,8 +519,14 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     int status = -1;
     long long peak = 0;
     int par = 0;                               // which worklist buffer this iteration fills
+    int pbuf = 0;                              // which publication buffer is written next
+    int pp = 0;                                // which slice buffer is written next
 #ifdef G10_PHASE_CLOCKS
-    long long dbg_dirty = 0, dbg_top = 0, dbg_local = 0;
+    long long dbg_dirty = 0, dbg_coop = 0, dbg_rounds = 0, dbg_refresh = 0;
+    long long pc_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, pc_last = clock64();
+#define LAZY_CLOCK(i) do { if (threadIdx.x == 0) { const long long now_ = clock64(); pc_acc[i] += now_ - pc_last; pc_last = now_; } } while (0)
+#else
+#define LAZY_CLOCK(i)
 #endif
 
     // every period starts DIRTY: its first evaluation chooses the destination
@@ -294,114 +535,359 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         L.c_key[p] = 0.0;
     }
     {
-        const long long m = own_slots_max(A, c, G, s_max);
+        const int n_slot_tiles = (int)((A.K + kSlotTile - 1) / kSlotTile);
+        for (int tl = c; tl < n_slot_tiles; tl += G) tile_minmax(A, L, tl, s_max);
+        __syncthreads();
+        const long long m = own_tiles_max(A, L, c, G, s_max);
         if (threadIdx.x == 0) A.peak_part[c] = m;
     }
     if (!grid_barrier(A.bar, G, gen)) status = -2;
 
     bool pending = false;                      // a commit decided in the previous iteration, not yet applied
     Winner win;
-    win.idx = -1; win.dest = -1; win.a = 0; win.ap = 0; win.bp = -1; win.b = -1;
+    win.idx = -1; win.dest = -1; win.a = 0; win.ap = 0; win.bp = -1; win.b = -1; win.t = 0; win.t_r = 0; win.t_end = 0;
+    Cand gBest;
+
+    // reads the published bounds from buffer `buf` into shared memory, unused; with only_flagged just those of
+    // the blocks that published again (s_refresh)
+    auto load_bounds = [&](int buf, bool only_flagged) {
+        for (int e = threadIdx.x; e < G * kTopT; e += kPlanThreads) {
+            const int j = e / kTopT, q = e % kTopT;
+            if (only_flagged && !s_refresh[j]) continue;
+            const LazyProp *pr = &L.props[(size_t)buf * kLazyMaxBlocks + j];
+            s_pkey[e] = __ldcg(&pr->skey[q]);
+            s_pidx[e] = __ldcg(&pr->sidx[q]);
+            s_pdone[e] = 0;
+        }
+        __syncthreads();
+    };
+    auto load_best = [&](int buf) -> Cand {
+        Cand x;
+        x.ben = 0; x.cost = 1; x.idx = -1; x.dest = -1;
+        for (int j = threadIdx.x; j < G; j += kPlanThreads) {
+            const LazyProp *pr = &L.props[(size_t)buf * kLazyMaxBlocks + j];
+            Cand y;
+            const ull lo = __ldcg(&pr->ben_lo), hi = __ldcg(&pr->ben_hi);
+            y.ben = ((u128)hi << 64) | lo; y.cost = __ldcg(&pr->cost); y.idx = __ldcg(&pr->idx); y.dest = __ldcg(&pr->dest);
+            if (cand_beats(y, x)) x = y;
+        }
+        return block_best_fast(x, &s_best, s_cand);
+    };
 
     for (int64_t it = 0; status == -1; ++it) {
-        // ---------------- apply the pending commit to what this block owns
+        bool barrier_since_booking = true;
+        // ---------------- A: apply the pending commit to the slots this block owns (bookings: after the barrier)
         if (pending) {
-            int64_t sz = 0;
-            const bool touched = commit_winner(A, win.idx, win.dest, it - 1, n_mig - 1, c, G, &sz);
+            const bool touched = commit_lazy(A, L, win.idx, win.dest, it - 1, n_mig - 1, c, G, s_max);
+            LAZY_CLOCK(10);
             if (touched) {
-                const long long m = own_slots_max(A, c, G, s_max);
+                __syncthreads();
+                const long long m = own_tiles_max(A, L, c, G, s_max);
                 if (threadIdx.x == 0) A.peak_part[c] = m;
             }
+            LAZY_CLOCK(11);
         }
-        // ---------------- A: classify the owned periods against the commit, collect DIRTY ones, local bests
+        // classify the owned periods against the commit, collect DIRTY ones, local bests
         // (on the first iteration `win` matches nothing and every period is DIRTY)
-        ScanResult sr = scan_owned(A, L, Pn, true, win, par, &s_best, s_cand, s_k, s_i);
-        if (threadIdx.x == 0) store_proposal(&A.proposals[c], sr.bestF);
-        pending = false;
+        {
+            const Cand bestF = scan_owned(A, L, Pn, true, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti);
+            if (threadIdx.x == 0) store_prop(&L.props[(size_t)pbuf * kLazyMaxBlocks + c], bestF, s_tk, s_ti);
+        }
+        LAZY_CLOCK(0);
         if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+        LAZY_CLOCK(1);
+        int rbuf = pbuf;
+        pbuf ^= 1;
 
-        // ---------------- B: global best FRESH score so far, peak, stop tests; rescore DIRTY periods (shared
-        // out over the grid) and this block's best STALE period if its bound may beat that score
-        Cand gF;
-        gF.ben = 0; gF.cost = 1; gF.idx = -1; gF.dest = -1;
+        // ---------------- B: best FRESH score of the grid, peak, stop tests
         long long m = 0;
         for (int j = threadIdx.x; j < G; j += kPlanThreads) {
             const long long pm = __ldcg(&A.peak_part[j]);
             if (pm > m) m = pm;
-            const Cand x = load_proposal(&A.proposals[j]);
-            if (cand_beats(x, gF)) gF = x;
         }
         peak = block_max_i64(m, s_max);
-        gF = block_best_fast(gF, &s_best, s_cand);
+        gBest = load_best(rbuf);
         const unsigned W = __ldcg(&L.wl_count[par]);
         if (A.fits_always || peak <= A.cap) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
         if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
         rounds += 1;
+        if (pending && c == 0) { book_winner(A, win.idx, win.dest); barrier_since_booking = false; }
+        if (pending) barrier_since_booking = false;
+        pending = false;
         const int *wl = L.worklist + (size_t)par * L.stride;
-        if (W <= 2u * (unsigned)G) {
-            for (unsigned e = c; e < W; e += G) eval_block(A, L, wl[e], &s_dest, s_part);
-        } else {
-            for (unsigned e = (unsigned)c * kPlanWarps + warp; e < W; e += (unsigned)G * kPlanWarps) eval_warp(A, L, wl[e], lane);
-        }
-        if (sr.idxS >= 0 && may_beat(sr.keyS, gF)) {
-            eval_block(A, L, sr.idxS, &s_dest, s_part);
-#ifdef G10_PHASE_CLOCKS
-            dbg_top += 1;
-#endif
-        }
-#ifdef G10_PHASE_CLOCKS
-        dbg_dirty += W;
-#endif
         if (c == 0 && threadIdx.x == 0) L.wl_count[par ^ 1] = 0;
         par ^= 1;
-        if (W > 0) {                               // DIRTY periods were rescored by other blocks than their owners
+        const bool few_dirty = W > 0 && W <= (unsigned)kDirtyPool && G * kTopT + kDirtyPool <= kLazyMaxBlocks * kTopT;
+        LAZY_CLOCK(2);
+        if (few_dirty) {
+            // DIRTY periods need the bookings in place: barrier; one warp re-chooses each one's destination; barrier.
+            // They join the published bounds below with an unbounded score and are rescored with the others.
             if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
-        } else __syncthreads();
-
-        // ---------------- C: make this block's best exact
-        Cand localF;
-        for (;;) {
-            sr = scan_owned(A, L, Pn, false, win, par, &s_best, s_cand, s_k, s_i);
-            localF = sr.bestF;
-            const Cand &thr = cand_beats(localF, gF) ? localF : gF;
-            if (sr.idxS >= 0 && may_beat(sr.keyS, thr)) {
-                eval_block(A, L, sr.idxS, &s_dest, s_part);
-                __syncthreads();
+            barrier_since_booking = true;
+            for (unsigned e = (unsigned)c * kPlanWarps + warp; e < W; e += (unsigned)G * kPlanWarps) dest_warp(A, L, wl[e], lane);
 #ifdef G10_PHASE_CLOCKS
-                dbg_local += 1;
+            dbg_dirty += W;
 #endif
+            if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+        } else if (W > 0) {
+            // very many DIRTY periods (the first iteration): rescore them at once, shared out, and look again
+            if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+            barrier_since_booking = true;
+            for (unsigned e = (unsigned)c * kPlanWarps + warp; e < W; e += (unsigned)G * kPlanWarps) eval_warp(A, L, wl[e], lane);
+#ifdef G10_PHASE_CLOCKS
+            dbg_dirty += W;
+#endif
+            if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+            {
+                const Cand bestF = scan_owned(A, L, Pn, false, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti);
+                if (threadIdx.x == 0) store_prop(&L.props[(size_t)pbuf * kLazyMaxBlocks + c], bestF, s_tk, s_ti);
+            }
+            if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+            rbuf = pbuf;
+            pbuf ^= 1;
+            gBest = load_best(rbuf);
+        }
+        load_bounds(rbuf, false);
+        int n_pool = G * kTopT;
+        if (few_dirty) {
+            for (unsigned e = threadIdx.x; e < W; e += kPlanThreads) {
+                const int p = wl[e];
+                const bool live = __ldcg(&L.c_state[p]) != 0;
+                s_pkey[n_pool + e] = __longlong_as_double(0x7ff0000000000000ll);
+                s_pidx[n_pool + e] = live ? p : -1;
+                s_pdone[n_pool + e] = 0;
+            }
+            n_pool += (int)W;
+            __syncthreads();
+        }
+        LAZY_CLOCK(3);
+
+        // ---------------- R: rounds of joint rescoring
+        bool failed = false;
+        int round_no = 0;
+#pragma unroll 1
+        for (;;) {
+            const double gkey = gBest.idx >= 0 ? cand_key(gBest) : -1.0;
+            int msel = 0;
+            {
+                // which published bounds are rescored this round (same choice in every block, in publication order):
+                // every unused one that may beat the best exact score -- in the first round of an iteration only those
+                // within 10 % of the best bound (the winner is usually among them, and a strong exact score spares the
+                // rest).  Bounds that cannot beat the best exact score are set aside for good.
+                double floor0 = -1.0;
+                if (round_no == 0) {
+                    double k = -1.0;
+                    int e_best = -1;
+                    for (int e = threadIdx.x; e < n_pool; e += kPlanThreads)
+                        if (!s_pdone[e] && s_pidx[e] >= 0 && s_pkey[e] > k && s_pkey[e] < 1e300) { k = s_pkey[e]; e_best = e; }
+                    block_max_key(k, e_best, s_k, s_i);
+                    floor0 = 0.9 * k;
+                }
+                int base = 0;
+#pragma unroll 1
+                for (int e0 = 0; e0 < n_pool; e0 += kPlanThreads) {
+                    const int e = e0 + threadIdx.x;
+                    bool take = false;
+                    if (e < n_pool && !s_pdone[e] && s_pidx[e] >= 0 && s_pkey[e] >= floor0) {
+                        take = bound_may_beat(L, s_pidx[e], s_pkey[e], gkey, &gBest);
+                        if (!take) s_pdone[e] = 4;
+                    }
+                    const unsigned mk = __ballot_sync(0xffffffffu, take);
+                    if (lane == 0) s_wcnt[warp] = __popc(mk);
+                    __syncthreads();
+                    int before = base, total = base;
+                    for (int w2 = 0; w2 < kPlanWarps; ++w2) { if (w2 < warp) before += s_wcnt[w2]; total += s_wcnt[w2]; }
+                    const int pos = before + __popc(mk & ((1u << lane) - 1u));
+                    if (take && pos < kRoundM) { s_sel[pos] = e; s_pdone[e] = 1; }     // beyond the cap: next round
+                    base = total;
+                    __syncthreads();
+                }
+                msel = base < kRoundM ? base : kRoundM;
+                // what the rescoring needs to know of each chosen period, fetched once, all of them together
+                for (int r = threadIdx.x; r < msel; r += kPlanThreads) {
+                    const int p = s_pidx[s_sel[r]];
+                    const int d = (__ldcg(&L.c_state[p]) & 3) - 1;
+                    s_it_d[r] = d;
+                    s_it_ap[r] = A.geo_a[d * A.geo_stride + p]; s_it_bp[r] = A.geo_b[d * A.geo_stride + p];
+                    s_it_s[r] = A.bytes[A.per_t[p]];
+                    s_it_cost[r] = 2ull * (ull)A.geo_t[d * A.geo_stride + p];
+                }
+            }
+            __syncthreads();
+            LAZY_CLOCK(4);
+            if (msel == 0) {
+                if (round_no == 0) { round_no = 1; continue; }      // (the first round only looks at the best bounds)
+                // nothing published may beat the best score.  A block that has used all its bounds may hold more.
+                if (threadIdx.x == 0) s_flag = 0;
+                __syncthreads();
+                for (int j = threadIdx.x; j < G; j += kPlanThreads) {
+                    bool all = true;
+                    for (int q = 0; q < kTopT; ++q) if (s_pidx[j * kTopT + q] < 0 || !s_pdone[j * kTopT + q]) all = false;
+                    const double lastk = s_pkey[j * kTopT + kTopT - 1];
+                    const bool again = all && lastk > 0.0 && (gBest.idx < 0 || lastk >= gkey * (1.0 - 1e-10));
+                    s_refresh[j] = again ? 1 : 0;
+                    if (again) s_flag = 1;
+                }
+                __syncthreads();
+                if (!s_flag) break;
+#ifdef G10_PHASE_CLOCKS
+                dbg_refresh += 1;
+#endif
+                if (s_refresh[c]) {
+                    const Cand bestF = scan_owned(A, L, Pn, false, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti, &gBest);
+                    if (threadIdx.x == 0) store_prop(&L.props[(size_t)pbuf * kLazyMaxBlocks + c], bestF, s_tk, s_ti);
+                }
+                if (!grid_barrier(A.bar, G, gen)) { failed = true; break; }
+                barrier_since_booking = true;
+                load_bounds(pbuf, true);
+                pbuf ^= 1;
+                LAZY_CLOCK(8);
                 continue;
             }
-            break;
+            round_no += 1;
+#ifdef G10_PHASE_CLOCKS
+            dbg_rounds += 1; dbg_coop += msel;
+#endif
+            // every block sums its share of each chosen period's absent range: tiles ta + c, ta + c + G, ... of the
+            // range.  One thread per period classifies its tiles from their pressure minima / maxima (a tile wholly
+            // at least s above capacity counts s for its whole time, one wholly within capacity nothing); the few
+            // tiles in between are read slot by slot, one warp each.
+            for (int r = threadIdx.x; r < msel; r += kPlanThreads) { s_acc[2 * r] = 0; s_acc[2 * r + 1] = 0; }
+            if (threadIdx.x == 0) s_nmix = 0;
+            __syncthreads();
+            {
+                int nsub = 1;                                    // threads per period (a power of two)
+                while (nsub < 8 && 2 * nsub * msel <= kPlanThreads) nsub *= 2;
+                const int r = (int)threadIdx.x / nsub, sub = (int)threadIdx.x % nsub;
+                if (r < msel) {
+                    const int ap = s_it_ap[r], bp = s_it_bp[r];
+                    const int64_t sz = s_it_s[r];
+#ifdef G10_PHASE_CLOCKS
+                    if (sub == 0) atomicAdd((ull *)&s_dbg_slots, (ull)(bp - ap + 1));
+#endif
+                    u128 acc = 0;
+                    const int ta = ap / kSlotTile, tb = bp / kSlotTile;
+                    for (int tl = ta + c + sub * G; tl <= tb; tl += nsub * G) {
+                        const int64_t t0 = (int64_t)tl * kSlotTile, t1 = t0 + kSlotTile - 1;
+                        const int k_lo = (int)(t0 > ap ? t0 : ap), k_hi = (int)(t1 < bp ? t1 : bp);
+                        const long long mn = L.tmin[tl], mx = L.tmax[tl];
+#ifdef G10_PHASE_CLOCKS
+                        atomicAdd((ull *)&s_dbg_tiles, 1ull);
+#endif
+                        if (mx <= A.cap) continue;
+                        if (mn >= A.cap && mn - A.cap >= sz) { acc += (u128)(ull)sz * (u128)(ull)(A.start[k_hi + 1] - A.start[k_lo]); continue; }
+#ifdef G10_PHASE_CLOCKS
+                        atomicAdd((ull *)&s_dbg_mixed, 1ull);
+#endif
+                        const int pos = atomicAdd(&s_nmix, 1);
+                        if (pos < kMixCap) s_mix[pos] = (r << 22) | tl;
+                        else acc += benefit_partial(A, k_lo, k_hi, sz, 0, 1);          // list full: this thread reads the tile itself
+                    }
+                    if (acc != 0) {
+                        const ull lo = (ull)acc;
+                        const ull old = atomicAdd(&s_acc[2 * r], lo);
+                        atomicAdd(&s_acc[2 * r + 1], (ull)(acc >> 64) + (old + lo < old ? 1ull : 0ull));
+                    }
+                }
+            }
+            __syncthreads();
+            {
+                const int nmix = s_nmix < kMixCap ? s_nmix : kMixCap;
+#ifdef G10_PHASE_CLOCKS
+                if (threadIdx.x == 0 && s_nmix > kMixCap) s_dbg_over += s_nmix - kMixCap;
+                LAZY_CLOCK(10);
+#endif
+#pragma unroll 1
+                for (int m = warp; m < nmix; m += kPlanWarps) {
+                    const int r = s_mix[m] >> 22, tl = s_mix[m] & ((1 << 22) - 1);
+                    const int ap = s_it_ap[r], bp = s_it_bp[r];
+                    const int64_t t0 = (int64_t)tl * kSlotTile, t1 = t0 + kSlotTile - 1;
+                    const int k_lo = (int)(t0 > ap ? t0 : ap), k_hi = (int)(t1 < bp ? t1 : bp);
+                    const u128 acc = warp_sum_u128(benefit_tile_warp(A, k_lo, k_hi, s_it_s[r], lane));
+                    if (lane == 0) {
+                        const ull lo = (ull)acc;
+                        const ull old = atomicAdd(&s_acc[2 * r], lo);
+                        atomicAdd(&s_acc[2 * r + 1], (ull)(acc >> 64) + (old + lo < old ? 1ull : 0ull));
+                    }
+                }
+            }
+            __syncthreads();
+            for (int r = threadIdx.x; r < msel; r += kPlanThreads) {
+                ull *dst = L.partials + (((size_t)pp * kRoundM + r) * kLazyMaxBlocks + c) * 2;
+                dst[0] = s_acc[2 * r]; dst[1] = s_acc[2 * r + 1];
+            }
+            LAZY_CLOCK(5);
+            if (!grid_barrier(A.bar, G, gen)) { failed = true; break; }
+            barrier_since_booking = true;
+            LAZY_CLOCK(6);
+            // every block adds up the slices (one warp per period at a time); the owner stores the new score
+#pragma unroll 2
+            for (int r = warp; r < msel; r += kPlanWarps) {
+                const int p = s_pidx[s_sel[r]];
+                const int d = s_it_d[r];
+                u128 tot = 0;
+                {
+                    const ulonglong2 *src = (const ulonglong2 *)(L.partials + ((size_t)pp * kRoundM + r) * kLazyMaxBlocks * 2);
+                    ulonglong2 vals[kLazyMaxBlocks / 32];
+#pragma unroll
+                    for (int q = 0; q < kLazyMaxBlocks / 32; ++q) {          // all loads first
+                        const int j = lane + 32 * q;
+                        vals[q] = j < G ? __ldcg(&src[j]) : make_ulonglong2(0ull, 0ull);
+                    }
+#pragma unroll
+                    for (int q = 0; q < kLazyMaxBlocks / 32; ++q) tot += ((u128)vals[q].y << 64) | vals[q].x;
+                }
+                tot = warp_sum_u128(tot);
+                if (lane == 0) {
+                    Cand x;
+                    x.ben = tot; x.cost = s_it_cost[r]; x.idx = tot == 0 ? -1 : p; x.dest = d;
+                    s_new[r] = x;
+                    if ((int)((p / kPlanThreads) % G) == c) store_score(L, p, d, kFresh, tot, x.cost);
+                }
+            }
+            __syncthreads();
+            {
+                Cand x;
+                x.ben = 0; x.cost = 1; x.idx = -1; x.dest = -1;
+                if ((int)threadIdx.x < msel) x = s_new[threadIdx.x];
+                const Cand b = block_best_fast(x, &s_best, s_cand);
+                if (cand_beats(b, gBest)) gBest = b;
+            }
+            pp ^= 1;
+            __syncthreads();
+            LAZY_CLOCK(7);
         }
-        if (threadIdx.x == 0) store_proposal(&L.prop_stale[c], localF);      // second buffer: step A reuses the first
-        if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
+        if (failed) { status = -2; break; }
+        if (!barrier_since_booking) { if (!grid_barrier(A.bar, G, gen)) { status = -2; break; } }
 
-        // ---------------- D: the exact global argmax; decide
-        Cand best;
-        best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
-        for (int j = threadIdx.x; j < G; j += kPlanThreads) {
-            const Cand x = load_proposal(&L.prop_stale[j]);
-            if (cand_beats(x, best)) best = x;
-        }
-        best = block_best_fast(best, &s_best, s_cand);
-        if (best.idx < 0) { status = G10_EXHAUSTED; break; }
+        // ---------------- D: decide
+        if (gBest.idx < 0) { status = G10_EXHAUSTED; break; }
         {
-            const int64_t p = best.idx;
-            const int X = best.dest;
-            win.idx = best.idx; win.dest = X;
+            const int64_t p = gBest.idx;
+            const int X = gBest.dest;
+            win.idx = gBest.idx; win.dest = X;
             win.a = A.per_u[p] + 1; win.b = A.per_v[p] - 1;
             win.ap = A.geo_a[X * A.geo_stride + p]; win.bp = A.geo_b[X * A.geo_stride + p];
+            win.t = A.geo_t[X * A.geo_stride + p];
+            win.t_r = A.start[win.a]; win.t_end = A.start[win.b + 1];
             const int64_t sz = A.bytes[A.per_t[p]];
             if (X == G10_DEST_SSD) bytes_ssd += sz; else bytes_host += sz;
         }
         n_mig += 1;
         pending = true;
+        LAZY_CLOCK(9);
     }
 #ifdef G10_PHASE_CLOCKS
+    if (threadIdx.x == 0 && c == 0) {
+        const long long r_ = rounds ? rounds : 1;
+        printf("k_plan_lazy cycles/iteration: A %lld bar1 %lld B %lld dirty %lld select %lld slices %lld bar %lld combine %lld refresh %lld decide %lld\n",
+               pc_acc[0] / r_, pc_acc[1] / r_, pc_acc[2] / r_, pc_acc[3] / r_, pc_acc[4] / r_, pc_acc[5] / r_, pc_acc[6] / r_, pc_acc[7] / r_, pc_acc[8] / r_, pc_acc[9] / r_);
+        printf("  within A: commit %lld own-slots max %lld\n", pc_acc[10] / r_, pc_acc[11] / r_);
+    }
+    if (threadIdx.x == 0 && c == 0) printf("slots of jointly rescored ranges: %llu; tiles looked at by block 0: %llu, read slot by slot %llu, beyond the list %llu\n", s_dbg_slots, s_dbg_tiles, s_dbg_mixed, s_dbg_over);
     if (threadIdx.x == 0 && (c == 0 || c == 77))
-        printf("k_plan_lazy block %d: iterations %lld, DIRTY rescored (grid) %lld, own top STALE rescored %lld, further STALE rescored %lld\n",
-               c, (long long)rounds, dbg_dirty, dbg_top, dbg_local);
+        printf("k_plan_lazy block %d: iterations %lld, DIRTY rescored (grid) %lld, rounds %lld, periods rescored jointly %lld, refreshes %lld\n",
+               c, (long long)rounds, dbg_dirty, dbg_rounds, dbg_coop, dbg_refresh);
 #endif
     plan_epilogue(A, c, G, gen, status, peak, n_mig, rounds, bytes_ssd, bytes_host);
 }
@@ -421,7 +907,8 @@ cudaError_t launch_plan_lazy(const PlanArgs &A_in, const Workspace &w, int G, cu
     PlanArgs A = A_in;
     LazyArgs L;
     L.c_state = w.c_state; L.c_ben_lo = w.c_ben_lo; L.c_ben_hi = w.c_ben_hi; L.c_cost = w.c_cost; L.c_key = w.c_key;
-    L.worklist = w.worklist; L.wl_count = w.wl_count; L.prop_stale = w.prop_stale; L.stride = A.geo_stride;
+    L.worklist = w.worklist; L.wl_count = w.wl_count; L.props = w.lazy_props; L.partials = w.lazy_partials; L.stride = A.geo_stride;
+    L.tmin = w.lazy_tmin; L.tmax = w.lazy_tmax;
     void *args[] = {&A, &L};
     return cudaLaunchCooperativeKernel((const void *)k_plan_lazy, dim3(G), dim3(kPlanThreads), args, 0, s);
 }
