@@ -31,6 +31,7 @@ from paper_2310_09443_b200 import traces  # noqa: E402
 
 WORKLOAD = "config1_resnet152_b256"
 L2_FLUSH_BYTES = 512 << 20
+PLAN_ONE_DRAM_BYTES = 211456    # dram__bytes_read.sum + dram__bytes_write.sum of one k_plan_one launch on config 1 (ncu --set full capture)
 KERNELS_PER_PLAN = 10      # slot clock, bucket histogram, bucket scatter, bucket emit, diff, pressure scan, geometry,
                            # single-block loop, multi-block loop (returns at once when the former did the work), status
 KERNELS_PER_VITALITY = 4   # bucket histogram, bucket scatter, bucket emit, status
@@ -298,7 +299,7 @@ def run_ours(args):
     loop_bytes = plan_loop_algorithmic_bytes(mig)
     loop_s = stage_ms[3] / 1e3
     roofline = {"kernel": "k_plan_one", "bound": "hbm", "achieved": loop_bytes / loop_s / 1e9, "peak": hbm_peak,
-                "unit": "GB/s", "frac": loop_bytes / loop_s / 1e9 / hbm_peak, "traffic": None, "peak_kind": peak_kind,
+                "unit": "GB/s", "frac": loop_bytes / loop_s / 1e9 / hbm_peak, "traffic": PLAN_ONE_DRAM_BYTES, "peak_kind": peak_kind,
                 "algorithmic_bytes": loop_bytes, "kernel_ms": stage_ms[3], "us_per_iteration": stage_ms[3] * 1e3 / max(int(summary[1]), 1),
                 "note": "the whole planner state of this workload (pressure, clock, bookings, %d periods) lives in the shared "
                         "memory of one SM: the kernel is a chain of %d dependent iterations (search, rescore, commit), bound by "
