@@ -21,6 +21,14 @@
  *       residency at every use).  The paper prints no numeric example of Algorithm 1 (its figures
  *       did not survive), so agreement with the paper's own numbers is "parity unpinned".
  *   g10o_plan (lazy tier) : must equal the plain tier bit for bit.
+ *   g10o_schedule_prefetch : a hand-worked example, a dense slot-by-slot restatement on toy plans, invariants
+ *       (capacity never exceeded by the pass, bytes added = size x slots regained, issue times only earlier).
+ *   g10o_emit_instructions : the stream of hand-worked example A, a dense restatement on toy traces, structural
+ *       invariants (one ALLOC per used tensor, one FREE per intermediate tensor, order inside a boundary).
+ *   g10o_characterize : dense restatement on toy traces, closed forms on the MLP chain, conservation identities
+ *       (sum of active bytes = sum of size x uses, active <= pressure, hidden-latency counts against the geometry).
+ *   batched re-planning (g10_oracle.py, plan_batch: a loop of g10o_plan plus set arithmetic) : every variant against
+ *       the dense brute force, the set identities of the stability pairs.
  */
 #include <stdint.h>
 #include <stdlib.h>
