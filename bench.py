@@ -329,7 +329,7 @@ def run_ours(args):
         "roofline": roofline,
     }
     if not args.no_stress and world == 1:
-        line["stress_passes"] = stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind)
+        line["stress_passes"] = stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, args.stress_reps)
     line["cpu_baseline"] = cpu_baseline(tr)
     print(json.dumps(line))
     if world > 1:
@@ -351,7 +351,7 @@ def plan_loop_algorithmic_bytes(mig):
     return 32 * slots + 48 * len(mig)
 
 
-def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=10):
+def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=20):
     """Vitality and timeline passes on the 1M-kernel / 4M-tensor stress trace (config 4): the only workload whose
     arrays are large enough for an HBM fraction to mean something.  Algorithmic bytes: vitality reads kernel_ptr
     (8K) and kernel_tensors (4E) and writes first/last/num_uses (12N), use_ptr (8N), uses (4E'), period_ptr (8N)
@@ -369,15 +369,19 @@ def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=10):
     steps, warm = reps, 3
     vit_s = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), steps, warm, flush) / steps
     tl_s = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), steps, warm, flush) / steps
+    no_flush = torch.empty(1, dtype=torch.uint8, device=dev)      # warm-L2 numbers: nothing written between the calls
+    vit_w = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), steps, warm, no_flush) / steps
+    tl_w = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), steps, warm, no_flush) / steps
     out = {
         "workload": "config4_stress_dag", "K": K, "N": N, "E": E, "uses": e2, "periods": pn,
-        "vitality_ms": vit_s * 1e3, "timeline_ms": tl_s * 1e3,
+        "vitality_ms": vit_s * 1e3, "timeline_ms": tl_s * 1e3, "repetitions": steps,
+        "vitality_ms_warm_l2": vit_w * 1e3, "timeline_ms_warm_l2": tl_w * 1e3,
         "events_per_s": E / (vit_s + tl_s),
         "vitality_roofline": {"bound": "hbm", "achieved": vit_bytes / vit_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
                               "frac": vit_bytes / vit_s / 1e9 / hbm_peak, "algorithmic_bytes": vit_bytes, "peak_kind": peak_kind},
         "timeline_roofline": {"bound": "hbm", "achieved": tl_bytes / tl_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
                               "frac": tl_bytes / tl_s / 1e9 / hbm_peak, "algorithmic_bytes": tl_bytes, "peak_kind": peak_kind},
-        "l2": "flushed between timed calls",
+        "l2": "flushed between timed calls (the *_warm_l2 figures: not flushed)",
     }
     # the whole plan of the stress trace (capacity = 3/10 of the unplanned peak), once
     tl = binding.g10_pressure_timeline(tb, ws=ws)
@@ -417,7 +421,15 @@ def cpu_baseline(tr):
         O.plan(tr, cap)
         reps += 1
     dt = time.perf_counter() - t0
+    # the analysis passes alone (slot clock, vitality, pressure), median of three
+    ts = []
+    for _ in range(3):
+        t1 = time.perf_counter()
+        O.timeline(tr)
+        ts.append(time.perf_counter() - t1)
+    passes_s = sorted(ts)[1]
     return {"value": tr.E * reps / dt, "unit": "events/s", "cores": 1, "kind": "oracle",
+            "vitality_timeline_events_per_s": tr.E / passes_s,
             "sample": "whole config-1 plan (plain tier), %d repetitions in %.1f s" % (reps, dt),
             "plan_ms": dt / reps * 1e3, "host_cores_available": os.cpu_count()}
 
@@ -431,7 +443,7 @@ def main():
     ap.add_argument("--no-stress", action="store_true", help="skip the config-4 pass measurements")
     ap.add_argument("--stress-only", action="store_true",
                     help="only time the vitality / timeline passes on config 4 (small profiling target)")
-    ap.add_argument("--stress-reps", type=int, default=10)
+    ap.add_argument("--stress-reps", type=int, default=20)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
