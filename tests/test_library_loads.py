@@ -56,3 +56,33 @@ def test_argument_errors_before_any_launch(lib):
     assert lib.g10_plan_migrations(C.byref(tr4), 1, 1, 1, None, C.byref(po), None, 0, None) == -3      # no workspace
     go = binding._GeometryOut()
     assert lib.g10_candidate_geometry(1, 1, None, None, None, None, None, 1, 1, C.byref(go), None) == -1
+
+
+def test_argument_errors_of_the_later_entry_points(lib):
+    buf = (C.c_int64 * 8)()
+    ptr = C.cast(buf, C.c_void_p)
+    # statistics: zero bandwidth, missing outputs, oversize
+    so = binding._StatsOut()
+    assert lib.g10_characterize(1, 1, None, None, None, None, 0, None, None, None, 0, 1, C.byref(so), None) == -1
+    assert lib.g10_characterize(1, 1, ptr, ptr, ptr, ptr, 0, None, None, None, 1, 1, C.byref(so), None) == -1
+    assert lib.g10_characterize(1 << 31, 1, ptr, ptr, ptr, ptr, 0, None, None, None, 1, 1, C.byref(so), None) == -2
+    # batch: host traces refused, variant count, zero bandwidth, workspace
+    bo = binding._BatchOut()
+    bo.summary = ptr; bo.stability = ptr
+    var = (binding._Variant * 1)(binding._Variant(None, 1, 1, 1, 0))
+    tr_host = binding._Trace(0, 0, 0, ptr, None, None, None, None, binding.MEM_HOST)
+    assert lib.g10_plan_batch(C.byref(tr_host), 1, var, 0, C.byref(bo), None, 0, None) == -1
+    tr_dev = binding._Trace(0, 0, 0, ptr, None, None, None, None, binding.MEM_DEVICE)
+    assert lib.g10_plan_batch(C.byref(tr_dev), 0, var, 0, C.byref(bo), None, 0, None) == -2
+    assert lib.g10_plan_batch(C.byref(tr_dev), 2000, var, 0, C.byref(bo), None, 0, None) == -2
+    bad = (binding._Variant * 1)(binding._Variant(None, 1, 0, 1, 0))
+    assert lib.g10_plan_batch(C.byref(tr_dev), 1, bad, 0, C.byref(bo), None, 0, None) == -1
+    assert lib.g10_plan_batch(C.byref(tr_dev), 1, var, -1, C.byref(bo), None, 0, None) == -1
+    assert lib.g10_plan_batch(C.byref(tr_dev), 1, var, 0, C.byref(bo), None, 0, None) == -3
+    # prefetch pass and instruction stream
+    pf = binding._PrefetchOut()
+    assert lib.g10_schedule_prefetch(1, 1, None, None, None, 1, C.byref(pf), None) == -1
+    eo = binding._EmitOut()
+    assert lib.g10_emit_instructions(1, 1, None, None, None, None, None, 0, None, None, C.byref(eo), None, 0, None) == -1
+    # the workspace of the batch call is the planner's
+    assert binding.g10_workspace_bytes(binding.WS_BATCH, 96, 130, 320) == binding.g10_workspace_bytes(binding.WS_PLAN, 96, 130, 320)
