@@ -491,6 +491,167 @@ int32_t g10o_plan(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Steady-state (cyclic) planning.  Section 4.2 notes that the inactive period of a global tensor (a
+ * weight) may span two consecutive training iterations.  Readings taken here:
+ *   (1) the traced iteration repeats unchanged, so the timeline is a cycle of K slots of length T =
+ *       sum of the durations; slot k of the next iteration is slot k again.  Unrolled index k + K
+ *       names slot k one iteration later, unrolled time start[k] + T;
+ *   (2) every global tensor that is used has, besides its periods inside the iteration, one more
+ *       inactive period from its last use to its first use in the next iteration, (i, last, first + K),
+ *       provided at least one slot lies in between (first + K - last >= 2).  These wrap-around periods
+ *       are numbered after the ordinary ones, by tensor id;
+ *   (3) geometry, admissibility, benefit and commit are those of the ordinary planner on the unrolled
+ *       clock; pressure, channel bookings and host occupancy belong to the physical slot k mod K (a
+ *       wrap-around period covers at most K - 1 slots, so no slot is met twice);
+ *   (4) records carry unrolled slot indices and times (absent_last and the prefetch time of a
+ *       wrap-around period may lie in the next iteration).
+ * Plain tier only (every live period rescored every iteration).  periods_out (optional, 3 * (E + N)
+ * ints) receives the period list used: tensor, prev use, next use (unrolled).
+ * ---------------------------------------------------------------------------------------- */
+typedef struct {
+    int64_t K, Pn;
+    const int64_t *start2;          /* [2K + 1] unrolled clock */
+    const int64_t *dur, *bytes;
+    const int32_t *per_tensor, *per_u, *per_v;
+    geo_t *geo[2];
+    int64_t *P, *busy[4], *hocc;
+    int64_t cap;
+    uint64_t host_capacity;
+} cyc_state;
+
+static int64_t cyc_overlap(const cyc_state *S, int64_t w0, int64_t w1, int64_t k)      /* k unrolled */
+{
+    int64_t lo = w0 > S->start2[k] ? w0 : S->start2[k];
+    int64_t hi = w1 < S->start2[k + 1] ? w1 : S->start2[k + 1];
+    return hi > lo ? hi - lo : 0;
+}
+
+static int cyc_channel_free(const cyc_state *S, int ch, int64_t w0, int64_t w1, int64_t k0, int64_t k1)
+{
+    for (int64_t k = k0; k <= k1; ++k)
+        if (S->busy[ch][k % S->K] + cyc_overlap(S, w0, w1, k) > S->dur[k % S->K]) return 0;
+    return 1;
+}
+
+static int cyc_admissible(const cyc_state *S, int64_t p, int X)
+{
+    const geo_t *g = &S->geo[X][p];
+    if (!g->valid) return 0;
+    int64_t a = S->per_u[p] + 1, b = S->per_v[p] - 1;
+    int64_t t_r = S->start2[a], t_end = S->start2[b + 1];
+    int out = X == DEST_SSD ? CH_SSD_OUT : CH_HOST_OUT, in = X == DEST_SSD ? CH_SSD_IN : CH_HOST_IN;
+    if (!cyc_channel_free(S, out, t_r, t_r + g->t, a, g->a_abs - 1)) return 0;
+    if (!cyc_channel_free(S, in, t_end - g->t, t_end, g->b_abs + 1, b)) return 0;
+    if (X == DEST_HOST && S->host_capacity != 0) {
+        uint64_t s = (uint64_t)S->bytes[S->per_tensor[p]];
+        for (int64_t k = a; k <= b; ++k)
+            if ((uint64_t)S->hocc[k % S->K] + s > S->host_capacity) return 0;
+    }
+    return 1;
+}
+
+int32_t g10o_plan_cyclic(int64_t K, int64_t N, const int64_t *kernel_ptr, const int32_t *kernel_tensors,
+                         const int64_t *tensor_bytes, const int64_t *kernel_ns, const uint8_t *tensor_global,
+                         uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
+                         uint64_t host_capacity_bytes, int64_t max_iterations,
+                         g10o_migration *out, int64_t out_cap, int64_t *final_pressure /* [K] */,
+                         int64_t *summary /* [8] */, int32_t *periods_out, int64_t *num_periods_out)
+{
+    int64_t E = K > 0 ? kernel_ptr[K] : 0;
+    size_t nN = (size_t)(N > 0 ? N : 1), nK = (size_t)(K > 0 ? K : 1), nE = (size_t)(E + N > 0 ? E + N : 1);
+    int64_t *start = (int64_t *)malloc(8 * (nK + 1)), *start2 = (int64_t *)malloc(8 * (2 * nK + 1));
+    int32_t *first = (int32_t *)malloc(4 * nN), *last = (int32_t *)malloc(4 * nN), *nuse = (int32_t *)malloc(4 * nN);
+    int64_t *use_ptr = (int64_t *)malloc(8 * (nN + 1)), *per_ptr = (int64_t *)malloc(8 * (nN + 1));
+    int32_t *uses = (int32_t *)malloc(4 * nE);
+    int32_t *pt = (int32_t *)malloc(4 * nE), *pu = (int32_t *)malloc(4 * nE), *pv = (int32_t *)malloc(4 * nE);
+    int64_t counts[2];
+    g10o_slot_clock(K, kernel_ns, start);
+    for (int64_t k = 0; k <= 2 * K; ++k) start2[k] = k <= K ? start[k] : start[k - K] + start[K];
+    g10o_vitality(K, N, kernel_ptr, kernel_tensors, first, last, nuse, use_ptr, uses, E, per_ptr, pt, pu, pv, E, counts);
+    int64_t Pn = counts[1];
+    for (int64_t i = 0; i < N; ++i)                      /* the wrap-around periods of the global tensors */
+        if (tensor_global && tensor_global[i] && first[i] >= 0 && first[i] + K - last[i] >= 2) {
+            pt[Pn] = (int32_t)i; pu[Pn] = last[i]; pv[Pn] = (int32_t)(first[i] + K); Pn += 1;
+        }
+    int64_t pk; int32_t ps32;
+    g10o_pressure(K, N, tensor_bytes, tensor_global, first, last, final_pressure, &pk, &ps32);
+
+    cyc_state S;
+    S.K = K; S.Pn = Pn; S.start2 = start2; S.dur = kernel_ns; S.bytes = tensor_bytes;
+    S.per_tensor = pt; S.per_u = pu; S.per_v = pv; S.P = final_pressure; S.host_capacity = host_capacity_bytes;
+    size_t nP = (size_t)(Pn > 0 ? Pn : 1);
+    for (int X = 0; X < 2; ++X) {
+        S.geo[X] = (geo_t *)malloc(sizeof(geo_t) * nP);
+        for (int64_t p = 0; p < Pn; ++p)
+            S.geo[X][p] = geometry_one(2 * K, start2, tensor_bytes[pt[p]], pu[p], pv[p], X == DEST_SSD ? ssd_bw : host_bw);
+    }
+    for (int c = 0; c < 4; ++c) S.busy[c] = (int64_t *)calloc(nK, 8);
+    S.hocc = (int64_t *)calloc(nK, 8);
+    unsigned char *alive = (unsigned char *)malloc(nP);
+    for (int64_t p = 0; p < Pn; ++p) alive[p] = 1;
+    int fits_always = gpu_capacity_bytes >= ((uint64_t)1 << 63);
+    S.cap = fits_always ? INT64_MAX : (int64_t)gpu_capacity_bytes;
+    int64_t limit = (max_iterations <= 0 || max_iterations > Pn) ? Pn : max_iterations;
+    int64_t n_mig = 0, n_rounds = 0, status = -1, bytes_to[2] = {0, 0};
+    int32_t rc = 0;
+    for (int64_t it = 0;; ++it) {
+        int64_t cur_peak, cur_slot;
+        peak_of(S.P, K, &cur_peak, &cur_slot);
+        if (fits_always || cur_peak <= S.cap) { status = n_mig == 0 ? ST_ALREADY_FITS : ST_FIT; break; }
+        if (it >= limit) { status = limit < Pn ? ST_ITERATION_LIMIT : ST_EXHAUSTED; break; }
+        n_rounds += 1;
+        int64_t best = -1; int bestX = -1; u128 bestB = 0; int64_t bestC = 1;
+        for (int64_t p = 0; p < Pn; ++p) {
+            if (!alive[p]) continue;
+            int X = cyc_admissible(&S, p, DEST_SSD) ? DEST_SSD : (cyc_admissible(&S, p, DEST_HOST) ? DEST_HOST : -1);
+            if (X < 0) continue;
+            const geo_t *g = &S.geo[X][p];
+            int64_t s = tensor_bytes[pt[p]];
+            u128 b = 0;
+            for (int64_t k = g->a_abs; k <= g->b_abs; ++k) {
+                int64_t ex = S.P[k % K] - S.cap;
+                if (ex <= 0) continue;
+                if (ex > s) ex = s;
+                b += (u128)(uint64_t)ex * (u128)(uint64_t)kernel_ns[k % K];
+            }
+            if (b == 0) continue;
+            int64_t c = 2 * g->t;
+            if (best < 0 || beats(b, c, p, bestB, bestC, best)) { best = p; bestX = X; bestB = b; bestC = c; }
+        }
+        if (best < 0) { status = ST_EXHAUSTED; break; }
+        const geo_t *g = &S.geo[bestX][best];
+        int64_t s = tensor_bytes[pt[best]];
+        int64_t a = pu[best] + 1, b = pv[best] - 1;
+        int64_t t_r = start2[a], t_end = start2[b + 1];
+        if (n_mig < out_cap) {
+            g10o_migration *m = &out[n_mig];
+            m->period = (int32_t)best; m->tensor = pt[best]; m->dest = bestX;
+            m->absent_first = g->a_abs; m->absent_last = g->b_abs; m->iteration = (int32_t)it;
+            m->evict_issue_ns = t_r; m->prefetch_issue_ns = t_end - g->t; m->transfer_ns = g->t;
+        } else rc = -1;
+        int outc = bestX == DEST_SSD ? CH_SSD_OUT : CH_HOST_OUT, inc = bestX == DEST_SSD ? CH_SSD_IN : CH_HOST_IN;
+        for (int64_t k = g->a_abs; k <= g->b_abs; ++k) S.P[k % K] -= s;
+        for (int64_t k = a; k <= g->a_abs - 1; ++k) S.busy[outc][k % K] += cyc_overlap(&S, t_r, t_r + g->t, k);
+        for (int64_t k = g->b_abs + 1; k <= b; ++k) S.busy[inc][k % K] += cyc_overlap(&S, t_end - g->t, t_end, k);
+        if (bestX == DEST_HOST) for (int64_t k = a; k <= b; ++k) S.hocc[k % K] += s;
+        alive[best] = 0;
+        bytes_to[bestX] += s;
+        n_mig += 1;
+    }
+    int64_t fpk, fps;
+    peak_of(S.P, K, &fpk, &fps);
+    summary[0] = n_mig; summary[1] = n_rounds; summary[2] = status; summary[3] = fpk; summary[4] = fps;
+    summary[5] = bytes_to[DEST_SSD]; summary[6] = bytes_to[DEST_HOST]; summary[7] = 0;
+    if (periods_out) for (int64_t p = 0; p < Pn; ++p) { periods_out[3 * p] = pt[p]; periods_out[3 * p + 1] = pu[p]; periods_out[3 * p + 2] = pv[p]; }
+    if (num_periods_out) *num_periods_out = Pn;
+    free(start); free(start2); free(first); free(last); free(nuse); free(use_ptr); free(per_ptr); free(uses);
+    free(pt); free(pu); free(pv); free(S.geo[0]); free(S.geo[1]);
+    for (int c = 0; c < 4; ++c) free(S.busy[c]);
+    free(S.hocc); free(alive);
+    return rc;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Smart tensor prefetching (Section 4.4).  The eviction loop above assumes every prefetch at its
  * latest safe prefetch time.  Afterwards the evicted periods are sorted by that time and visited in
  * order; for each one the search goes backward from the latest safe prefetch time to the earliest

@@ -199,3 +199,28 @@ def plan_batch(trace, variants, max_iterations=0, lazy=True):
         stability.append((len(mine & base), len(mine | base)))
         plans.append(r)
     return SimpleNamespace(plans=plans, stability=np.asarray(stability, dtype=np.int64).reshape(-1, 2))
+
+
+def plan_cyclic(trace, gpu_capacity_bytes, host_bw=None, ssd_bw=None, host_capacity_bytes=None, max_iterations=0):
+    """Steady-state planning on the cyclic timeline (wrap-around periods of global tensors; plain tier)."""
+    host_bw = trace.host_bw if host_bw is None else host_bw
+    ssd_bw = trace.ssd_bw if ssd_bw is None else ssd_bw
+    hc = trace.host_capacity_bytes if host_capacity_bytes is None else host_capacity_bytes
+    ptr = _c(trace.kernel_ptr, np.int64); kt = _c(trace.kernel_tensors, np.int32)
+    tb = _c(trace.tensor_bytes, np.int64); dur = _c(trace.kernel_ns, np.int64)
+    tg = _c(trace.tensor_global, np.uint8) if trace.tensor_global is not None else None
+    K, N, E = trace.K, trace.N, trace.E
+    cap = max(E + N, 1)
+    out = np.zeros(cap, MIGRATION_DTYPE)
+    finalP = np.zeros(K, np.int64)
+    summary = np.zeros(8, np.int64)
+    periods = np.zeros(3 * cap, np.int32)
+    npd = C.c_int64(0)
+    rc = lib().g10o_plan_cyclic(C.c_int64(K), C.c_int64(N), _p(ptr), _p(kt), _p(tb), _p(dur), _p(tg),
+                                C.c_uint64(gpu_capacity_bytes), C.c_uint64(host_bw), C.c_uint64(ssd_bw), C.c_uint64(hc),
+                                C.c_int64(max_iterations), _p(out), C.c_int64(cap), _p(finalP), _p(summary), _p(periods),
+                                C.byref(npd))
+    assert rc == 0
+    n = int(summary[0])
+    return SimpleNamespace(migrations=out[:n].copy(), final_pressure=finalP, summary=summary, status=STATUS[int(summary[2])],
+                           periods=periods[:3 * npd.value].reshape(-1, 3).copy())

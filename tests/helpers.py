@@ -258,3 +258,114 @@ def brute_prefetch(plan, pressure, start, tensor_bytes, cap):
         new_last[i] = j - 1
         new_issue[i] = start[j] if j <= m["absent_last"] else m["prefetch_issue_ns"]
     return order, new_last, new_issue, P
+
+
+# ------------------------------------------------------------------------------------------------
+# Steady-state (cyclic) planning, dense restatement for toy traces: the iteration repeats unchanged, a used global
+# tensor has one more period from its last use to its first use one iteration later; every nanosecond of a transfer
+# window is charged to the physical slot it falls in.
+# ------------------------------------------------------------------------------------------------
+def brute_plan_cyclic(tr, cap, host_bw, ssd_bw, host_capacity=0, max_iterations=0):
+    uses, first, last, periods = brute_vitality(tr)
+    K = tr.K
+    periods = list(periods)
+    for i in range(tr.N):
+        if tr.tensor_global[i] and uses[i] and first[i] + K - last[i] >= 2:
+            periods.append((i, last[i], first[i] + K))
+    start = brute_start(tr)
+    T = start[K] if K else 0
+    dur = [int(d) for d in tr.kernel_ns]
+    P = brute_pressure(tr, uses)
+
+    def when(k):                                  # unrolled start time of unrolled slot k (k <= 2K)
+        return start[k] if k <= K else start[k - K] + T
+
+    def slot_at(ns):                              # unrolled slot holding unrolled nanosecond ns
+        it, r = divmod(ns, T)
+        for k in range(K):
+            if start[k] <= r < start[k + 1]:
+                return k + it * K
+        raise AssertionError
+
+    def geometry(period, bw):
+        i, u, v = period
+        s = int(tr.tensor_bytes[i])
+        t = -((-s * 10 ** 9) // bw)
+        t_r, t_end = when(u + 1), when(v)
+        if 2 * t > t_end - t_r:
+            return dict(t=t, valid=False)
+        ev, pf = {}, {}
+        for ns in range(t_r, t_r + t):
+            ev[slot_at(ns)] = ev.get(slot_at(ns), 0) + 1
+        for ns in range(t_end - t, t_end):
+            pf[slot_at(ns)] = pf.get(slot_at(ns), 0) + 1
+        absent = [k for k in range(u + 1, v) if k > max(ev) and k < min(pf)]
+        if not absent:
+            return dict(t=t, valid=False)
+        return dict(t=t, valid=True, a_abs=absent[0], b_abs=absent[-1], ev=ev, pf=pf)
+
+    geo = [[geometry(p, ssd_bw) for p in periods], [geometry(p, host_bw) for p in periods]]
+    booked = {(X, d): [0] * K for X in (SSD, HOST) for d in ("out", "in")}
+    hocc = [0] * K
+    alive = [True] * len(periods)
+    plan = []
+    limit = len(periods) if max_iterations <= 0 else min(max_iterations, len(periods))
+    it = rounds = 0
+    while True:
+        if max(P, default=0) <= cap:
+            status = "ALREADY_FITS" if not plan else "FIT"
+            break
+        if it >= limit:
+            status = "ITERATION_LIMIT" if limit < len(periods) else "EXHAUSTED"
+            break
+        rounds += 1
+        best = None
+        for p, (i, u, v) in enumerate(periods):
+            if not alive[p]:
+                continue
+            s = int(tr.tensor_bytes[i])
+            dest = None
+            for X in (SSD, HOST):
+                g = geo[X][p]
+                if not g["valid"]:
+                    continue
+                if any(booked[(X, "out")][k % K] + n > dur[k % K] for k, n in g["ev"].items()):
+                    continue
+                if any(booked[(X, "in")][k % K] + n > dur[k % K] for k, n in g["pf"].items()):
+                    continue
+                if X == HOST and host_capacity and any(hocc[k % K] + s > host_capacity for k in range(u + 1, v)):
+                    continue
+                dest = X
+                break
+            if dest is None:
+                continue
+            g = geo[dest][p]
+            benefit = sum(min(s, max(0, P[k % K] - cap)) * dur[k % K] for k in range(g["a_abs"], g["b_abs"] + 1))
+            if benefit <= 0:
+                continue
+            ratio = Fraction(benefit, 2 * g["t"])
+            if best is None or ratio > best[0]:
+                best = (ratio, p, dest)
+        if best is None:
+            status = "EXHAUSTED"
+            break
+        _, p, dest = best
+        i, u, v = periods[p]
+        g = geo[dest][p]
+        s = int(tr.tensor_bytes[i])
+        for k in range(g["a_abs"], g["b_abs"] + 1):
+            P[k % K] -= s
+        for k, n in g["ev"].items():
+            booked[(dest, "out")][k % K] += n
+        for k, n in g["pf"].items():
+            booked[(dest, "in")][k % K] += n
+        if dest == HOST:
+            for k in range(u + 1, v):
+                hocc[k % K] += s
+        alive[p] = False
+        plan.append(dict(period=p, tensor=i, dest=dest, absent_first=g["a_abs"], absent_last=g["b_abs"], iteration=it,
+                         evict_issue_ns=when(u + 1), prefetch_issue_ns=when(v) - g["t"], transfer_ns=g["t"]))
+        it += 1
+    pk = max(P, default=0)
+    return dict(plan=plan, final_pressure=P, status=status, rounds=rounds, periods=periods,
+                final_peak=(pk, P.index(pk) if P else -1))
