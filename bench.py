@@ -264,6 +264,18 @@ def run_ours(args):
                  "note": "same planning path, one thread block per variant, all variants concurrently (binding allocates outputs inside the timed call)"}
         del wsb, bo, variants
 
+    # ---- steady-state (cyclic) plan of the same trace: the weights' wrap-around periods become candidates
+    cyclic = None
+    if rank == 0:
+        csteps = max(3, args.steps // 4)
+        c_s = time_calls(torch, lambda: binding.g10_plan_cyclic(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws), csteps, 3, flush) / csteps
+        cp = binding.g10_plan_cyclic(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws)
+        torch.cuda.synchronize()
+        cs = cp.summary.cpu().numpy()
+        cyclic = {"plan_ms": c_s * 1e3, "migrations": int(cs[0]), "status": binding.STATUS.get(int(cs[2]), "?"),
+                  "final_peak_bytes": int(cs[3]), "final_peak_bytes_acyclic": int(summary[3]), "device_status": int(cs[7])}
+        del cp
+
     # ---- end to end through the host-pointer form of the call: H2D of the trace and D2H of the plan inside
     tbh = binding.pin(tr)
     wsh = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E, binding.MEM_HOST), dtype=torch.uint8, device=dev)
@@ -324,6 +336,7 @@ def run_ours(args):
         "prefetch_pass": {"ms": prefetch_ms, "moved": int(pf_summary[0]), "slots_regained": int(pf_summary[1]),
                           "peak_after": int(pf_summary[2]), "note": "plan + pass timed together, plan time subtracted"},
         "batch_replan": batch,
+        "cyclic_plan": cyclic,
         "gpu_launches": args.steps * KERNELS_PER_PLAN,
         "clocks": clocks,
         "roofline": roofline,

@@ -56,7 +56,7 @@ extern "C" {
 #define G10_DEV_PERIODS_OVERFLOW 0x20 /* periods_cap too small (counts[1] holds the need)         */
 #define G10_DEV_PLAN_OVERFLOW 0x40   /* migrations_cap too small (summary[0] holds the need)      */
 #define G10_DEV_TIMEOUT 0x80         /* an internal wait gave up; the kernel returned early       */
-#define G10_DEV_BATCH_UNFIT 0x100    /* g10_plan_batch: the trace does not fit one SM (no plan)   */
+#define G10_DEV_BATCH_UNFIT 0x100    /* g10_plan_batch / g10_plan_cyclic: the trace does not fit one SM (no plan) */
 
 /* exit status of the planner (summary[2]) */
 #define G10_ALREADY_FITS 0      /* unplanned peak pressure <= capacity, empty plan                 */
@@ -242,6 +242,22 @@ int32_t g10_emit_instructions(int64_t num_kernels, int64_t num_tensors, const in
                               const int64_t *tensor_bytes, const uint8_t *tensor_global, const int64_t *kernel_start_ns,
                               int64_t num_migrations, const g10_migration *migrations, const int64_t *new_prefetch_issue_ns,
                               g10_emit_out *out, void *ws, size_t ws_bytes, void *stream);
+
+/* Steady-state planning on the cyclic timeline.  Section 4.2 notes that the inactive period of a global tensor (a
+   weight) may span two consecutive training iterations.  Here the traced iteration is taken to repeat unchanged:
+   the timeline is a cycle of K slots, unrolled slot k + K is slot k one iteration later (unrolled time + the length
+   of the iteration).  Besides the ordinary periods, every used global tensor has one wrap-around period from its
+   last use to its first use of the next iteration, (tensor, last, first + K), if at least one slot lies in between;
+   these are numbered after the ordinary periods, by tensor id.  Geometry, scoring and commits are those of
+   g10_plan_migrations on the unrolled clock, while pressure, channel bookings and host occupancy belong to the
+   physical slot k mod K.  Records carry unrolled slots and times (absent_last may be >= K, the prefetch time may lie
+   in the next iteration).  Same arguments, outputs and workspace (G10_WS_PLAN) as g10_plan_migrations; of the
+   options only host_capacity_bytes and max_iterations are used.
+   Limits: device-resident traces (G10_MEM_DEVICE); one thread block plans, so pressure, clock, bookings and periods
+   must fit the shared memory of one SM (K <= 32000), else summary[2] = -1 and summary[7] has G10_DEV_BATCH_UNFIT. */
+int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
+                        const g10_options *options /* NULL = defaults */, g10_plan_out *out,
+                        void *ws, size_t ws_bytes, void *stream);
 
 /* Section 5's sensitivity studies seen from the planner: the same trace planned under V variants at once -- other
    kernel durations (profiling error), SSD / host bandwidths, GPU capacity, host capacity -- one thread block per

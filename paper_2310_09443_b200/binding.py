@@ -24,7 +24,7 @@ FLAG_GLOBAL_STATE = 2
 FLAG_MULTI_BLOCK = 4
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
-           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize", "g10_plan_batch")
+           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize", "g10_plan_batch", "g10_plan_cyclic")
 STATIC_MAX_KERNELS, STATIC_MAX_TENSORS = 32768, 131072
 
 INSTRUCTION_DTYPE = np.dtype([("opcode", "<i4"), ("tensor", "<i4"), ("target", "<i4"), ("record", "<i4"),
@@ -128,6 +128,9 @@ def load_library():
         lib.g10_characterize.restype = C.c_int32
         lib.g10_characterize.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.POINTER(_StatsOut), C.c_void_p]
+        lib.g10_plan_cyclic.restype = C.c_int32
+        lib.g10_plan_cyclic.argtypes = [C.POINTER(_Trace), C.c_uint64, C.c_uint64, C.c_uint64, C.POINTER(_Options),
+                                        C.POINTER(_PlanOut), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.g10_plan_batch.restype = C.c_int32
         lib.g10_plan_batch.argtypes = [C.POINTER(_Trace), C.c_int32, C.POINTER(_Variant), C.c_int64, C.POINTER(_BatchOut),
                                        C.c_void_p, C.c_size_t, C.c_void_p]
@@ -318,6 +321,26 @@ def g10_plan_migrations(tb: TraceBuffers, gpu_capacity_bytes, host_bw, ssd_bw, h
     tr = tb.c_struct()
     _check(lib.g10_plan_migrations(C.byref(tr), gpu_capacity_bytes, host_bw, ssd_bw, C.byref(opt), C.byref(po), _ptr(ws),
                                    ws_bytes, _stream(stream)))
+    out.workspace = ws
+    return out
+
+
+def g10_plan_cyclic(tb: TraceBuffers, gpu_capacity_bytes, host_bw, ssd_bw, host_capacity_bytes=0, max_iterations=0, ws=None,
+                    stream=None, migrations_cap=None):
+    """Steady-state plan on the cyclic timeline (wrap-around periods of global tensors).  Device traces only; records as in
+    g10_plan_migrations with unrolled slots and times."""
+    lib = load_library()
+    mcap = tb.E if migrations_cap is None else migrations_cap
+    dev = tb.kernel_ptr.device
+    out = SimpleNamespace(migrations=torch.empty(max(mcap, 1) * 48, dtype=torch.uint8, device=dev),
+                          final_pressure=torch.empty(max(tb.K, 1), dtype=torch.int64, device=dev),
+                          summary=torch.empty(8, dtype=torch.int64, device=dev))
+    ws, ws_bytes = _workspace(tb, WS_PLAN, ws, None)
+    po = _PlanOut(_ptr(out.migrations), mcap, _ptr(out.final_pressure), _ptr(out.summary))
+    opt = _Options(host_capacity_bytes, max_iterations, 0, None, 0)
+    tr = tb.c_struct()
+    _check(lib.g10_plan_cyclic(C.byref(tr), gpu_capacity_bytes, host_bw, ssd_bw, C.byref(opt), C.byref(po), _ptr(ws), ws_bytes,
+                               _stream(stream)))
     out.workspace = ws
     return out
 

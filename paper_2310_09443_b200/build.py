@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libg10.so")
-SOURCES = ["g10_api.cu", "g10_passes.cu", "g10_planner.cu", "g10_planner_lazy.cu", "g10_planner_small.cu", "g10_planner_one.cu", "g10_vitality_buckets.cu", "g10_prefetch.cu", "g10_emit.cu", "g10_stats.cu", "g10_static.cu"]
+SOURCES = ["g10_api.cu", "g10_passes.cu", "g10_planner.cu", "g10_planner_lazy.cu", "g10_planner_small.cu", "g10_planner_one.cu", "g10_vitality_buckets.cu", "g10_prefetch.cu", "g10_emit.cu", "g10_stats.cu", "g10_cyclic.cu", "g10_static.cu"]
 HEADERS = ["g10_device.cuh", "g10_internal.h", "g10_planner.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]

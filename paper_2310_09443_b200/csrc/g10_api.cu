@@ -86,6 +86,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.period_next_use = c.take<int32_t>(E);
     w.counts = c.take<int64_t>(4);
     w.start = c.take<int64_t>(K + 1);
+    w.start2 = c.take<int64_t>(2 * K + 1);
     w.pressure = c.take<int64_t>(K);
     w.peak_bytes = c.take<int64_t>(1);
     w.peak_slot = c.take<int32_t>(2);
@@ -401,6 +402,43 @@ int32_t g10_schedule_prefetch(int64_t K, int64_t n, const g10_migration *migrati
         return G10_ERR_ARG;
     CU(launch_schedule_prefetch(K, n, migrations, kernel_start_ns, tensor_bytes, gpu_capacity_bytes, out->pressure, out->order,
                                 out->new_absent_last, out->new_prefetch_issue_ns, out->summary, (cudaStream_t)stream));
+    return G10_OK;
+}
+
+int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
+                        const g10_options *options, g10_plan_out *out, void *ws, size_t ws_bytes, void *stream)
+{
+    int32_t rc = check_trace(trace);
+    if (rc != G10_OK) return rc;
+    if (trace->mem != G10_MEM_DEVICE || host_bw == 0 || ssd_bw == 0 || !out || !out->summary) return G10_ERR_ARG;
+    if (out->migrations_cap < 0 || (out->migrations_cap > 0 && !out->migrations)) return G10_ERR_ARG;
+    if (trace->num_kernels > 0 && !out->final_pressure) return G10_ERR_ARG;
+    if (options && options->max_iterations < 0) return G10_ERR_ARG;
+    rc = check_ws(G10_WS_PLAN, trace, ws, ws_bytes);
+    if (rc != G10_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    Workspace w;
+    DeviceTrace d;
+    const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
+    rc = begin_call(trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff);
+    if (rc != G10_OK) return rc;
+    VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
+                       w.period_tensor, w.period_prev_use, w.period_next_use, d.E, w.counts};
+    PlanParams pp;
+    pp.gpu_capacity_bytes = gpu_capacity_bytes; pp.host_bw = host_bw; pp.ssd_bw = ssd_bw;
+    pp.host_capacity_bytes = options ? options->host_capacity_bytes : 0;
+    pp.max_iterations = options ? options->max_iterations : 0;
+    pp.flags = 0;
+    pp.migrations = out->migrations; pp.migrations_cap = out->migrations_cap;
+    pp.final_pressure = out->final_pressure; pp.summary = out->summary;
+    CU(launch_slot_clock(d, w, w.start, s));
+    CU(buckets ? launch_vitality_buckets(d, w, vb, s) : launch_vitality(d, w, vb, s));
+    CU(launch_pressure(d, w, w.first_use, w.last_use, false, pp.final_pressure, w.peak_bytes, w.peak_slot, s));
+    CU(launch_cyclic_prepare(d, w, s));
+    CU(launch_geometry(2 * d.K, d.E, w.counts + 1, w.start2, d.tensor_bytes, w.period_tensor, w.period_prev_use, w.period_next_use,
+                       host_bw, ssd_bw, d.E > 0 ? d.E : 1, w.geo_t, w.geo_a, w.geo_b, s));
+    CU(launch_plan_cyclic(d, w, pp, s));
+    CU(launch_publish_status_or(w, pp.summary + 7, s));
     return G10_OK;
 }
 

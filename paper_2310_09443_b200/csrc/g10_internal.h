@@ -93,6 +93,7 @@ struct Workspace {
     int32_t *uses, *period_tensor, *period_prev_use, *period_next_use;
     int64_t *counts;             // [3]
     int64_t *start;              // [K+1]
+    int64_t *start2;             // [2K+1] unrolled clock (cyclic planning)
     int64_t *pressure;           // [K]
     int64_t *peak_bytes;         // [1]
     int32_t *peak_slot;          // [1]
@@ -194,9 +195,12 @@ cudaError_t launch_characterize(int64_t K, int64_t N, const int64_t *use_ptr, co
                                 int64_t *active, int64_t *len_hist, int64_t *size_len_hist, int64_t *hide, int64_t *summary, cudaStream_t s);
 // planner (g10_planner.cu)
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
+cudaError_t launch_cyclic_prepare(const DeviceTrace &t, const Workspace &w, cudaStream_t s);
+cudaError_t launch_plan_cyclic(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
 cudaError_t launch_plan_variants(const DeviceTrace &t, const Workspace &w, const PlanParams &p, int V, int64_t *stability, cudaStream_t s);
 int plan_loop_max_blocks();
 bool plan_keeps_state_on_chip(int64_t K, int64_t E, uint32_t flags);   // true: the small-trace planner will run
 cudaError_t launch_publish_status(const Workspace &w, int64_t *dst, cudaStream_t s);
+cudaError_t launch_publish_status_or(const Workspace &w, int64_t *dst, cudaStream_t s);
 
 }  // namespace g10

@@ -143,6 +143,25 @@ cudaError_t launch_plan_variants(const DeviceTrace &t, const Workspace &w, const
     return launch_plan_batch(A, w, V, B, stability, s);
 }
 
+cudaError_t launch_plan_one_cyclic(const PlanArgs &A, const Workspace &w, cudaStream_t s);
+
+cudaError_t launch_plan_cyclic(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s)
+{
+    PlanArgs A;
+    fill_plan_args(t, w, p, A);
+    A.start = w.start2;
+    return launch_plan_one_cyclic(A, w, s);
+}
+
+// ORs the call's status word into *dst (which the planner may already have written)
+__global__ void k_publish_status_or(const ull *status, int64_t *dst) { *dst |= (int64_t)*status; }
+
+cudaError_t launch_publish_status_or(const Workspace &w, int64_t *dst, cudaStream_t s)
+{
+    k_publish_status_or<<<1, 1, 0, s>>>(w.status, dst);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s)
 {
     PlanArgs A;

@@ -99,7 +99,7 @@ __device__ __forceinline__ bool window_free(const PlanArgs &A, const int64_t *bu
 // kBooked: `busy` already includes the booking (else its share of the slot is added here).  kL2: read busy at L2.
 template <bool kBooked, bool kL2>
 __device__ __forceinline__ bool window_conflict(const int64_t *start, const int64_t *busy, int wk0, int wk1, int64_t w0, int64_t w1,
-                                                int64_t q0, int64_t q1, int qk0, int qk1)
+                                                int64_t q0, int64_t q1, int qk0, int qk1, int Kc = 0 /* physical slots, if the indices are unrolled */)
 {
     const int i0 = qk0 > wk0 ? qk0 : wk0, i1 = qk1 < wk1 ? qk1 : wk1;
     if (i0 > i1) return false;
@@ -115,7 +115,8 @@ __device__ __forceinline__ bool window_conflict(const int64_t *start, const int6
             const int64_t wl = w0 > s0 ? w0 : s0, wh = w1 < s1 ? w1 : s1;
             need += wh > wl ? wh - wl : 0;
         }
-        const int64_t booked = kL2 ? __ldcg(&busy[k]) : busy[k];
+        const int kp = Kc && k >= Kc ? k - Kc : k;
+        const int64_t booked = kL2 ? __ldcg(&busy[kp]) : busy[kp];
         if (booked + need > s1 - s0) return true;
     }
     return false;

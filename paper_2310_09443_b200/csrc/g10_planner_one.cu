@@ -50,7 +50,20 @@ struct __align__(16) OneDirty {
     int64_t t[2];
 };
 
-__device__ __forceinline__ bool window_free_one(const int64_t *sStart, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane)
+// Kc: number of physical slots when the slot indices are unrolled (cyclic mode), else 0
+__device__ __forceinline__ int phys_slot(int k, int Kc) { return Kc && k >= Kc ? k - Kc : k; }
+
+// Do the unrolled slot ranges [a1, b1] and [a2, b2] share a slot?  On the cycle also when one of them, taken one
+// iteration earlier or later, meets the other.
+__device__ __forceinline__ bool ranges_meet(int a1, int b1, int a2, int b2, int Kc)
+{
+    if (a1 <= b2 && a2 <= b1) return true;
+    if (!Kc) return false;
+    return (a1 <= b2 + Kc && a2 + Kc <= b1) || (a1 <= b2 - Kc && a2 - Kc <= b1);
+}
+
+__device__ __forceinline__ bool window_free_one(const int64_t *sStart, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane,
+                                                int Kc)
 {
     bool ok = true;
 #pragma unroll 1
@@ -58,15 +71,26 @@ __device__ __forceinline__ bool window_free_one(const int64_t *sStart, const int
         const int64_t s0 = sStart[k], s1 = sStart[k + 1];
         const int64_t lo = w0 > s0 ? w0 : s0, hi = w1 < s1 ? w1 : s1;
         const int64_t ov = hi > lo ? hi - lo : 0;
-        if (busy[k] + ov > s1 - s0) ok = false;
+        if (busy[phys_slot(k, Kc)] + ov > s1 - s0) ok = false;
     }
     return __all_sync(0xffffffffu, ok);
 }
 
-__host__ __device__ inline size_t one_smem_need(int64_t K, int64_t Pn, bool host_cap)
+// window_conflict on the cycle: the other window may meet the booking as it is, or one iteration earlier / later
+// (T = length of the iteration).  Only slots of the booking's own range are read.
+__device__ __forceinline__ bool window_conflict_cyc(const int64_t *sStart, const int64_t *busy, int wk0, int wk1, int64_t q0, int64_t q1,
+                                                    int qk0, int qk1, int Kc, int64_t T)
+{
+    if (window_conflict<true, false>(sStart, busy, wk0, wk1, 0, 0, q0, q1, qk0, qk1, Kc)) return true;
+    if (!Kc) return false;
+    return window_conflict<true, false>(sStart, busy, wk0, wk1, 0, 0, q0 + T, q1 + T, qk0 + Kc, qk1 + Kc, Kc) ||
+           window_conflict<true, false>(sStart, busy, wk0, wk1, 0, 0, q0 - T, q1 - T, qk0 - Kc, qk1 - Kc, Kc);
+}
+
+__host__ __device__ inline size_t one_smem_need(int64_t K, int64_t Pn, bool host_cap, bool cyclic = false)
 {
     const int64_t groups = (Pn + 31) / 32;
-    return (size_t)(2 * K + 1) * 8 + (size_t)4 * K * 8 + (host_cap ? (size_t)K * 8 : 0) + (size_t)groups * 32 * 8 + (size_t)Pn * 41 +
+    return (size_t)(2 * K + 1) * 8 + (cyclic ? (size_t)K * 8 : 0) + (size_t)4 * K * 8 + (host_cap ? (size_t)K * 8 : 0) + (size_t)groups * 32 * 8 + (size_t)Pn * 41 +
            (size_t)groups * 13 + 128;
 }
 
@@ -93,7 +117,7 @@ __device__ __forceinline__ void warp_argmax_u64(ull k, int idx, ull *mk, int *mi
 #define ONE_COUNT(i)
 #endif
 
-template <bool kBatch>
+template <bool kBatch, bool kCyclic>
 __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs O, BatchArgs B)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -128,8 +152,9 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
     }
     const bool host_cap = A.host_capacity != 0;
     unsigned dev_bits = 0;                              // device status bits of this block's plan
-    if (A.K > 65000 || Pn64 > 0x7fffffff || one_smem_need(A.K, Pn64, host_cap) > (size_t)O.smem_bytes) {
-        if (kBatch && threadIdx.x == 0) {
+    const int Kc = kCyclic ? (int)A.K : 0;             // physical slots when the indices are unrolled
+    if (A.K > (kCyclic ? 32000 : 65000) || Pn64 > 0x7fffffff || one_smem_need(A.K, Pn64, host_cap, kCyclic) > (size_t)O.smem_bytes) {
+        if ((kBatch || kCyclic) && threadIdx.x == 0) {
             for (int j = 0; j < 7; ++j) A.summary[j] = j == 2 || j == 4 ? -1 : 0;
             A.summary[7] = G10_DEV_BATCH_UNFIT;
         }
@@ -141,7 +166,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
 
     int64_t *sP = (int64_t *)smem_raw;
     int64_t *sStart = sP + K;
-    int64_t *sBusy = sStart + K + 1;                    // [4][K]
+    int64_t *sBusy = sStart + (kCyclic ? 2 * K : K) + 1; // [4][K]  (the clock has 2K + 1 entries in cyclic mode)
     int64_t *sHocc = sBusy + (size_t)4 * K;             // [K] if host_cap
     ull *ckey = (ull *)(sHocc + (host_cap ? K : 0));    // [G1 * 32] bits of the rounded score (0 = none)
     ull *gkey = ckey + (size_t)G1 * 32;                 // [G1] maximum of each group
@@ -166,7 +191,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
         }
         if (!kBatch) {
 #pragma unroll 1
-            for (int k = tid; k <= K; k += kOneThreads) sStart[k] = A.start[k];
+            for (int k = tid; k <= (kCyclic ? 2 * K : K); k += kOneThreads) sStart[k] = A.start[k];
         } else {
             // slot clock of this variant: exclusive scan of its durations (each thread a run of consecutive kernels);
             // a duration outside [1, 2^44) counts as 1 and raises the status bit, as in the trace-level pass
@@ -260,13 +285,13 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                             t = __ldg(&A.geo_t[X * A.geo_stride + li]);
                         }
                         if (ap < 0) continue;
-                        if (!window_free_one(sStart, sBusy + (size_t)(2 * X) * K, t_r, t_r + t, a, ap - 1, lane)) continue;
-                        if (!window_free_one(sStart, sBusy + (size_t)(2 * X + 1) * K, t_end - t, t_end, bp + 1, b, lane)) continue;
+                        if (!window_free_one(sStart, sBusy + (size_t)(2 * X) * K, t_r, t_r + t, a, ap - 1, lane, Kc)) continue;
+                        if (!window_free_one(sStart, sBusy + (size_t)(2 * X + 1) * K, t_end - t, t_end, bp + 1, b, lane, Kc)) continue;
                         if (X == G10_DEST_HOST && host_cap) {
                             bool ok = true;
 #pragma unroll 1
                             for (int k = a + lane; k <= b; k += 32)
-                                if ((uint64_t)sHocc[k] + (uint64_t)s > A.host_capacity) ok = false;
+                                if ((uint64_t)sHocc[phys_slot(k, Kc)] + (uint64_t)s > A.host_capacity) ok = false;
                             if (!__all_sync(0xffffffffu, ok)) continue;
                         }
                         d = X;
@@ -284,7 +309,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                     u128 acc = 0;
 #pragma unroll 1
                     for (int k = ap + lane; k <= bp; k += 32) {
-                        int64_t ex = sP[k] - A.cap;
+                        int64_t ex = sP[phys_slot(k, Kc)] - A.cap;
                         if (ex > 0) {
                             if (ex > s) ex = s;
                             acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
@@ -404,7 +429,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                 u128 acc = 0;
 #pragma unroll 1
                 for (int k = r.ap + tid; k <= r.bp; k += kOneThreads) {
-                    int64_t ex = sP[k] - A.cap;
+                    int64_t ex = sP[phys_slot(k, Kc)] - A.cap;
                     if (ex > 0) {
                         if (ex > s) ex = s;
                         acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
@@ -444,8 +469,9 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             int fell = 0;
 #pragma unroll 1
             for (int k = wap + tid; k <= wbp; k += kOneThreads) {
-                const int64_t before = sP[k], after = before - s;
-                sP[k] = after;
+                const int kp = phys_slot(k, Kc);
+                const int64_t before = sP[kp], after = before - s;
+                sP[kp] = after;
                 if (before > A.cap && after <= A.cap) ++fell;
             }
             if (fell) atomicSub(&s_n_over, fell);
@@ -454,17 +480,17 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             for (int k = wa + tid; k <= wap - 1; k += kOneThreads) {
                 const int64_t s0 = sStart[k], s1 = sStart[k + 1];
                 const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
-                if (hi > lo) bo[k] += hi - lo;
+                if (hi > lo) bo[phys_slot(k, Kc)] += hi - lo;
             }
 #pragma unroll 1
             for (int k = wbp + 1 + tid; k <= wb; k += kOneThreads) {
                 const int64_t s0 = sStart[k], s1 = sStart[k + 1];
                 const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
-                if (hi > lo) bi[k] += hi - lo;
+                if (hi > lo) bi[phys_slot(k, Kc)] += hi - lo;
             }
             if (X == G10_DEST_HOST && host_cap)
 #pragma unroll 1
-                for (int k = wa + tid; k <= wb; k += kOneThreads) sHocc[k] += s;
+                for (int k = wa + tid; k <= wb; k += kOneThreads) sHocc[phys_slot(k, Kc)] += s;
             __syncthreads();                       // the bookings are in place for the conflict tests below
             int newly_dirty = 0;
 #pragma unroll 2
@@ -475,19 +501,20 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                 if (st & kDirtyO) continue;
                 const int d = (st & 3) - 1;
                 const OneRanges q = crng[li];
-                if (!((int)q.a <= wb && wa <= (int)q.b)) continue;
+                if (!ranges_meet(q.a, q.b, wa, wb, Kc)) continue;
                 unsigned char ns = st;
-                if ((st & kStateMaskO) == kFreshO && (int)q.ap <= wbp && wap <= (int)q.bp) ns = (unsigned char)((st & 3) | kStaleO);
+                if ((st & kStateMaskO) == kFreshO && ranges_meet(q.ap, q.bp, wap, wbp, Kc)) ns = (unsigned char)((st & 3) | kStaleO);
                 if (d == X) {
                     // same device: is one of its transfer windows no longer free?  (host occupancy: looked at in full)
-                    const bool meet_out = (int)q.a <= wap - 1 && wa <= (int)q.ap - 1;
-                    const bool meet_in = (int)q.bp + 1 <= wb && wbp + 1 <= (int)q.b;
+                    const bool meet_out = ranges_meet(q.a, (int)q.ap - 1, wa, wap - 1, Kc);
+                    const bool meet_in = ranges_meet((int)q.bp + 1, q.b, wbp + 1, wb, Kc);
                     bool hit = false;
                     if (meet_out || meet_in) {
                         const int64_t tq = ct[li];
                         const int64_t q_r = sStart[q.a], q_end = sStart[(int)q.b + 1];
-                        hit = (meet_out && window_conflict<true, false>(sStart, bo, wa, wap - 1, 0, 0, q_r, q_r + tq, q.a, (int)q.ap - 1)) ||
-                              (meet_in && window_conflict<true, false>(sStart, bi, wbp + 1, wb, 0, 0, q_end - tq, q_end, (int)q.bp + 1, q.b));
+                        const int64_t T = kCyclic ? sStart[K] : 0;
+                        hit = (meet_out && window_conflict_cyc(sStart, bo, wa, wap - 1, q_r, q_r + tq, q.a, (int)q.ap - 1, Kc, T)) ||
+                              (meet_in && window_conflict_cyc(sStart, bi, wbp + 1, wb, q_end - tq, q_end, (int)q.bp + 1, q.b, Kc, T));
                     }
                     if (!hit && d == G10_DEST_HOST && host_cap) hit = true;
                     if (hit) {
@@ -571,20 +598,20 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
         unsigned bits = 0;
 #pragma unroll 1
         for (int j = 0; j < kOneWarps; ++j) bits |= (unsigned)s_fin[j];
-        if (kBatch) A.summary[7] = bits;
+        if (kBatch || kCyclic) A.summary[7] = bits;          // (the call-wide status word is folded in afterwards)
         else if (bits) raise_status(A.status, bits);
     }
 }
 
 // Shared memory a launch can offer (opt-in maximum minus the kernel's static part); 0 if the device query fails.
-template <bool kBatch>
+template <bool kBatch, bool kCyclic>
 static int one_smem_budget()
 {
     int dev = 0, optin = 0;
     cudaFuncAttributes fa;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
     if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return 0;
-    if (cudaFuncGetAttributes(&fa, (const void *)k_plan_one<kBatch>) != cudaSuccess) return 0;
+    if (cudaFuncGetAttributes(&fa, (const void *)k_plan_one<kBatch, kCyclic>) != cudaSuccess) return 0;
     const int room = optin - (int)fa.sharedSizeBytes;
     return room > 0 ? room : 0;
 }
@@ -594,7 +621,7 @@ static int one_smem_budget()
 bool plan_one_possible(int64_t K, int64_t E, bool host_cap)
 {
     if (K > 65000 || E < 1) return false;
-    const int budget = one_smem_budget<false>();
+    const int budget = one_smem_budget<false, false>();
     return budget > 0 && one_smem_need(K, E < 512 ? E : 512, host_cap) <= (size_t)budget;
 }
 
@@ -605,10 +632,25 @@ cudaError_t launch_plan_one(const PlanArgs &A_in, const Workspace &w, cudaStream
     BatchArgs B;
     B.variants = nullptr; B.P0 = nullptr; B.P_out = nullptr;
     O.done = w.one_done;
-    O.smem_bytes = one_smem_budget<false>();
-    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
+    O.smem_bytes = one_smem_budget<false, false>();
+    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
     if (e != cudaSuccess) return e;
-    k_plan_one<false><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    k_plan_one<false, false><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    return cudaGetLastError();
+}
+
+// Steady-state planning: A.start is the unrolled clock [2K + 1], the period and geometry arrays hold unrolled slots.
+cudaError_t launch_plan_one_cyclic(const PlanArgs &A_in, const Workspace &w, cudaStream_t s)
+{
+    PlanArgs A = A_in;
+    OneArgs O;
+    BatchArgs B;
+    B.variants = nullptr; B.P0 = nullptr; B.P_out = nullptr;
+    O.done = w.one_done;
+    O.smem_bytes = one_smem_budget<false, true>();
+    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
+    if (e != cudaSuccess) return e;
+    k_plan_one<false, true><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
     return cudaGetLastError();
 }
 
@@ -657,10 +699,10 @@ cudaError_t launch_plan_batch(const PlanArgs &A_in, const Workspace &w, int V, c
     PlanArgs A = A_in;
     OneArgs O;
     O.done = w.one_done;
-    O.smem_bytes = one_smem_budget<true>();
-    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
+    O.smem_bytes = one_smem_budget<true, false>();
+    cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
     if (e != cudaSuccess) return e;
-    k_plan_one<true><<<V, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    k_plan_one<true, false><<<V, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const int64_t bound = A.geo_stride < batch_max_periods() ? A.geo_stride : batch_max_periods();
     k_batch_finish<<<V, 256, (size_t)((bound + 31) / 32) * 4, s>>>(bound, A.Pn_dev, A.out, A.out_cap, A.summary, stability, A.status);

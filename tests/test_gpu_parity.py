@@ -479,3 +479,55 @@ def test_batched_replanning(gpu, oracle):
     torch.cuda.synchronize()
     s = _np(got.summary)
     assert (s[:, 7] & 0x100).all() and (s[:, 2] == -1).all() and (_np(got.stability) == -1).all()
+
+
+def check_cyclic(gpu, oracle, tr, cap, host_capacity=0, max_iterations=0):
+    """Steady-state plan on the cyclic timeline against the oracle's (plain tier)."""
+    import torch
+    tb = gpu.upload(tr)
+    plan = gpu.g10_plan_cyclic(tb, cap, tr.host_bw, tr.ssd_bw, host_capacity_bytes=host_capacity, max_iterations=max_iterations)
+    torch.cuda.synchronize()
+    ref = oracle.plan_cyclic(tr, cap, host_capacity_bytes=host_capacity, max_iterations=max_iterations)
+    summary = _np(plan.summary)
+    assert summary[7] == 0, "device status %x" % summary[7]
+    assert np.array_equal(summary[:7], ref.summary[:7]), (summary, ref.summary)
+    assert np.array_equal(gpu.migrations_numpy(plan), ref.migrations)
+    assert np.array_equal(_np(plan.final_pressure)[:tr.K], ref.final_pressure)
+    return ref
+
+
+@pytest.mark.gpu
+def test_cyclic_planning(gpu, oracle):
+    import json, os, torch
+    ex = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "cyclic_example.json")))
+    tr = traces.from_lists("cyc", ex["kernel_lists"], ex["tensor_bytes"], ex["kernel_ns"], ex["tensor_global"],
+                           host_bw=ex["host_bw"], ssd_bw=ex["ssd_bw"], capacity_bytes=ex["capacity"])
+    ref = check_cyclic(gpu, oracle, tr, ex["capacity"])
+    assert ref.final_pressure.tolist() == ex["final_pressure"]
+    rng = np.random.default_rng(1618)
+    wrapped = 0
+    for trial in range(60):
+        toy = traces.random_toy(rng, int(rng.integers(1, 40)), int(rng.integers(1, 30)), max_deg=5)
+        if trial % 3 == 0:
+            toy.tensor_global = np.ones(toy.N, np.uint8)
+        start, P0, peak, slot = oracle.timeline(toy)
+        hc = int(rng.integers(0, 3)) * int(rng.integers(1, 80))
+        ref = check_cyclic(gpu, oracle, toy, peak * int(rng.integers(0, 10)) // 10, host_capacity=hc, max_iterations=int(rng.integers(0, 2)) * 3)
+        wrapped += int((ref.migrations["absent_last"] >= toy.K).sum())
+    assert wrapped > 10
+    for cfg in (0, 1, 2):
+        tr = traces.make_config(cfg)
+        start, P0, peak, slot = oracle.timeline(tr)
+        ref = check_cyclic(gpu, oracle, tr, tr.capacity_from_peak(peak))
+        plain = oracle.plan(tr, tr.capacity_from_peak(peak), lazy=True)
+        assert ref.summary[3] <= plain.summary[3]            # the weights' wrap-around periods only add options here
+    for lists, nb in (([], []), ([[], []], []), ([[0], [0], [0]], [9])):
+        tr = traces.from_lists("e", lists, nb, [3] * len(lists), [1] * len(nb), capacity_bytes=0)
+        check_cyclic(gpu, oracle, tr, 0)
+    # too large for one SM: reported, no plan
+    tr = traces.make_config(3)
+    tb = gpu.upload(tr)
+    plan = gpu.g10_plan_cyclic(tb, 1 << 30, tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    s = _np(plan.summary)
+    assert s[2] == -1 and (s[7] & 0x100)
