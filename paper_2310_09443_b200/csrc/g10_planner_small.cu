@@ -142,6 +142,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
     double *ckey = (double *)(cben_hi + S.cand_cap);        // rounded benefit/cost of the cached score
     PeriodInfo *info = (PeriodInfo *)(ckey + S.cand_cap);
     unsigned char *cstate = (unsigned char *)(info + S.cand_cap);
+    unsigned char *cskip = cstate + S.cand_cap;             // STALE period that cannot be this block's proposal in this iteration
     int64_t *busy = S.busy_rep + (size_t)c * 4 * K;
     int64_t *hocc = S.hocc_rep + (size_t)c * K;
 #ifdef G10_PHASE_CLOCKS
@@ -194,6 +195,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
         if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
         rounds += 1;
         PHASE_CLOCK(0);     // loop top (stop tests)
+        if (kFew) for (int li = threadIdx.x; li < n_local; li += kPlanThreads) cskip[li] = 0;
         // ---------------- 1. bring this block's periods up to date (one warp per period).  With few periods per
         // block only the DIRTY ones are done here (rare); STALE ones are rescored on demand in step 2.
 #pragma unroll 1
@@ -278,7 +280,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                                 take = cand_beats(x, y);
                             }
                             if (take) { kf = key; lf = li; }
-                        } else if (key > ks) { ks = key; ls = li; }
+                        } else if (!cskip[li] && key > ks) { ks = key; ls = li; }
                     }
                     double mf = kf, ms = ks;
 #pragma unroll 1
@@ -287,17 +289,20 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                         if (yf > mf) mf = yf;
                         if (ys > ms) ms = ys;
                     }
-                    int todo = -1;
-                    if (ms > 0.0 && ms >= mf * (1.0 - 1e-10)) {
-                        // the best STALE bound may beat (or tie) the best FRESH score: rescore it
-                        const unsigned who = __ballot_sync(0xffffffffu, ks == ms);
-                        todo = __shfl_sync(0xffffffffu, ls, __ffs(who) - 1);
-                    } else {
-                        // the block's best is FRESH: settle near-ties between lanes exactly, build the record
+                    // A STALE bound clearly above the best FRESH score has to be rescored; one within 1e-10 of it only
+                    // if the bound can win exactly (benefit and cost of the cached score, ties to the lower index):
+                    // otherwise the period cannot be this block's proposal in this iteration and is set aside.
+                    const bool above = ls >= 0 && ks > 0.0 && (!(mf > 0.0) || ks > mf * (1.0 + 1e-10));
+                    const bool near = ls >= 0 && ks > 0.0 && mf > 0.0 && !above && ks >= mf * (1.0 - 1e-10);
+                    // the block's exact best FRESH period (near-ties between lanes settled exactly): needed to judge a
+                    // near-tie and to publish, not when a bound is clearly above and gets rescored anyway
+                    const bool any_near = __any_sync(0xffffffffu, near);
+                    const bool need_best = any_near || !__any_sync(0xffffffffu, above);
+                    int src = -1;
+                    Cand best;
+                    best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
+                    if (need_best) {
                         const unsigned fin = __ballot_sync(0xffffffffu, lf >= 0 && kf >= mf * (1.0 - 1e-10));
-                        int src = -1;
-                        Cand best;
-                        best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
                         if (lf >= 0) {
                             const unsigned char sf = cstate[lf];
                             best.ben = ((u128)cben_hi[lf] << 64) | cben_lo[lf]; best.dest = (sf & 3) - 1;
@@ -314,6 +319,36 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                             }
                             src = __ffs(__ballot_sync(0xffffffffu, best.idx >= 0 && best.idx == z.idx)) - 1;
                         }
+                    }
+                    Cand zbest = best;
+                    bool can = above, set_aside = false;
+                    if (any_near) {
+                        // (every lane needs the exact best: broadcast it from its lane)
+                        const int from = src < 0 ? 0 : src;
+                        zbest.ben = ((u128)__shfl_sync(0xffffffffu, (ull)(best.ben >> 64), from) << 64) | __shfl_sync(0xffffffffu, (ull)best.ben, from);
+                        zbest.cost = __shfl_sync(0xffffffffu, best.cost, from);
+                        zbest.idx = __shfl_sync(0xffffffffu, best.idx, from);
+                        if (near) {
+                            Cand x;
+                            const unsigned char ss = cstate[ls];
+                            x.ben = ((u128)cben_hi[ls] << 64) | cben_lo[ls]; x.cost = 2ull * (ull)info[ls].t[(ss & 3) - 1];
+                            x.idx = (int)((int64_t)ls * G + c); x.dest = 0;
+                            can = src < 0 || cand_beats(x, zbest);
+                            if (!can) { cskip[ls] = 1; set_aside = true; }
+                        }
+                    }
+                    int todo = -1;
+                    const unsigned want = __ballot_sync(0xffffffffu, can);
+                    if (want) {
+                        double m2 = can ? ks : -1.0;
+#pragma unroll 1
+                        for (int o = 16; o > 0; o >>= 1) { const double y = __shfl_xor_sync(0xffffffffu, m2, o); if (y > m2) m2 = y; }
+                        const unsigned who = __ballot_sync(0xffffffffu, can && ks == m2);
+                        todo = __shfl_sync(0xffffffffu, ls, __ffs(who) - 1);
+                    } else if (__any_sync(0xffffffffu, set_aside)) {
+                        todo = -2;                                 // look again: a lane may hold further STALE periods
+                    } else {
+                        // the block's best is FRESH: build the record
                         if (src < 0) {
                             if (lane == 0) { s_pay.idx = -1; s_pay.dest = -1; s_pay.ben_lo = 0; s_pay.ben_hi = 0; s_pay.t = 0; }
                         } else if (lane == src) {
@@ -332,7 +367,8 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                 }
                 __syncthreads();
                 const int li = s_todo;
-                if (li < 0) break;
+                if (li == -1) break;
+                if (li == -2) continue;
                 // the whole block rescores period li
                 {
                     const unsigned char st = cstate[li];
@@ -557,7 +593,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
 // Shared memory the small-trace planner needs for K slots and `cand_cap` periods per block.
 static size_t small_smem_bytes(int64_t K, int cand_cap)
 {
-    return (size_t)(3 * K + 1) * 8 + (size_t)cand_cap * (24 + sizeof(PeriodInfo) + 1) + 16;
+    return (size_t)(3 * K + 1) * 8 + (size_t)cand_cap * (24 + sizeof(PeriodInfo) + 2) + 16;
 }
 
 bool plan_small_fits(int64_t K, int64_t E, int G, int *cand_cap_out, size_t *smem_out)
