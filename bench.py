@@ -32,6 +32,11 @@ from paper_2310_09443_b200 import traces  # noqa: E402
 WORKLOAD = "config1_resnet152_b256"
 L2_FLUSH_BYTES = 512 << 20
 PLAN_ONE_DRAM_BYTES = 211456    # dram__bytes_read.sum + dram__bytes_write.sum of one k_plan_one launch on config 1 (ncu --set full capture)
+# DRAM bytes per call on the stress trace, from an ncu capture of `bench.py --stress-only --stress-reps 1` (dram__bytes_read.sum +
+# dram__bytes_write.sum summed over the call's kernels): k_bk_hist 19.9 + k_bk_scatter 28.1 + k_bk_emit 135.5 MB; k_seg_scan<0> 16.0 +
+# k_first_last_events 59.9 + k_diff_scatter 76.1 + k_seg_scan<1> 8.0 MB
+STRESS_VITALITY_DRAM_BYTES = 183_500_000
+STRESS_TIMELINE_DRAM_BYTES = 160_000_000
 KERNELS_PER_PLAN = 10      # slot clock, bucket histogram, bucket scatter, bucket emit, diff, pressure scan, geometry,
                            # single-block loop, multi-block loop (returns at once when the former did the work), status
 KERNELS_PER_VITALITY = 4   # bucket histogram, bucket scatter, bucket emit, status
@@ -391,9 +396,11 @@ def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=20):
         "vitality_ms_warm_l2": vit_w * 1e3, "timeline_ms_warm_l2": tl_w * 1e3,
         "events_per_s": E / (vit_s + tl_s),
         "vitality_roofline": {"bound": "hbm", "achieved": vit_bytes / vit_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                              "frac": vit_bytes / vit_s / 1e9 / hbm_peak, "algorithmic_bytes": vit_bytes, "peak_kind": peak_kind},
+                              "frac": vit_bytes / vit_s / 1e9 / hbm_peak, "algorithmic_bytes": vit_bytes, "traffic": STRESS_VITALITY_DRAM_BYTES,
+                              "peak_kind": peak_kind},
         "timeline_roofline": {"bound": "hbm", "achieved": tl_bytes / tl_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                              "frac": tl_bytes / tl_s / 1e9 / hbm_peak, "algorithmic_bytes": tl_bytes, "peak_kind": peak_kind},
+                              "frac": tl_bytes / tl_s / 1e9 / hbm_peak, "algorithmic_bytes": tl_bytes, "traffic": STRESS_TIMELINE_DRAM_BYTES,
+                              "peak_kind": peak_kind},
         "l2": "flushed between timed calls (the *_warm_l2 figures: not flushed)",
     }
     # the whole plan of the stress trace (capacity = 3/10 of the unplanned peak), once

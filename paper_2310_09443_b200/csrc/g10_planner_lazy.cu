@@ -670,7 +670,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
             const double gkey = gBest.idx >= 0 ? cand_key(gBest) : -1.0;
             int msel = 0;
             {
-                // which published bounds are rescored this round (same choice in every block, in publication order):
+                // which published bounds are rescored now (same choice in every block, in publication order):
                 // every unused one that may beat the best exact score -- in the first round of an iteration only those
                 // within 10 % of the best bound (the winner is usually among them, and a strong exact score spares the
                 // rest).  Bounds that cannot beat the best exact score are set aside for good.

@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                     // otherwise the period cannot be this block's proposal in this iteration and is set aside.
                     const bool above = ls >= 0 && ks > 0.0 && (!(mf > 0.0) || ks > mf * (1.0 + 1e-10));
                     const bool near = ls >= 0 && ks > 0.0 && mf > 0.0 && !above && ks >= mf * (1.0 - 1e-10);
-                    // the block's exact best FRESH period (near-ties between lanes settled exactly): needed to judge a
+                    // the block's exact best FRESH period (near-ties between lanes settled exactly): needed to decide a
                     // near-tie and to publish, not when a bound is clearly above and gets rescored anyway
                     const bool any_near = __any_sync(0xffffffffu, near);
                     const bool need_best = any_near || !__any_sync(0xffffffffu, above);
