@@ -11,7 +11,10 @@
 
 namespace g10 {
 
-constexpr int kPfThreads = 1024;
+#ifndef G10_PF_THREADS
+#define G10_PF_THREADS 256
+#endif
+constexpr int kPfThreads = G10_PF_THREADS;       // a block-wide barrier per search chunk and per record: few warps keep it cheap
 
 __device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y)
 {
@@ -22,60 +25,118 @@ __device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y
 __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int64_t n, const g10_migration *__restrict__ mig,
                                                                   const int64_t *__restrict__ start, const int64_t *__restrict__ bytes,
                                                                   int64_t cap, int64_t *P, int32_t *order, int32_t *new_last,
-                                                                  int64_t *new_issue, int64_t *summary)
+                                                                  int64_t *new_issue, int64_t *summary, int p_in_smem, int sort_in_smem)
 {
-    __shared__ int s_stop;                 // highest slot of the current chunk that cannot take the tensor (-1: none)
+    extern __shared__ long long s_dyn[];   // the pressure curve, when the launch gave it room
+    __shared__ int s_wstop[2][kPfThreads / 32];   // per warp: highest slot of the current chunk that cannot take the tensor (-1: none);
+                                                  // two copies used in turn, so that one barrier per chunk is enough
+    __shared__ int s_ra[kPfThreads], s_rb[kPfThreads], s_rj[kPfThreads];
+    __shared__ long long s_rs[kPfThreads];
+    long long *Pw = (long long *)P;
+    if (p_in_smem) {
+        Pw = s_dyn;
+        for (int64_t k = threadIdx.x; k < K; k += kPfThreads) Pw[k] = P[k];
+    }
     __shared__ long long s_mx[kPfThreads / 32];
     __shared__ int s_sl[kPfThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // ---- order the records by (latest safe prefetch time, record index)
-    for (int64_t i = threadIdx.x; i < n; i += kPfThreads) order[i] = (int32_t)i;
-    __syncthreads();
     int64_t n2 = 1;
     while (n2 < n) n2 <<= 1;
-    for (int64_t k = 2; k <= n2; k <<= 1) {
-        for (int64_t j = k >> 1; j > 0; j >>= 1) {
-            const bool mirror = (j == (k >> 1));
-            for (int64_t t = threadIdx.x; t < n2 / 2; t += kPfThreads) {
-                const int64_t blk = t / j, off = t % j;
-                const int64_t i = blk * 2 * j + off;
-                const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
-                if (p < n) {
-                    const int32_t x = order[i], y = order[p];
-                    if (pf_before(mig, y, x)) { order[i] = y; order[p] = x; }
-                }
-            }
-            __syncthreads();
+    if (sort_in_smem) {
+        // (time, record) pairs sorted in shared memory: the network's comparisons would otherwise each cost two
+        // dependent global loads
+        long long *s_key = s_dyn + (p_in_smem ? K : 0);
+        int *s_idx = (int *)(s_key + n2);
+        for (int64_t i = threadIdx.x; i < n2; i += kPfThreads) {
+            s_key[i] = i < n ? mig[i].prefetch_issue_ns : 0x7fffffffffffffffll;
+            s_idx[i] = i < n ? (int)i : 0x7fffffff;
         }
-    }
-    // ---- visit the records in that order
-    long long moved = 0, regained = 0;
-    for (int64_t q = 0; q < n; ++q) {
-        const int r = order[q];
-        const int a_abs = mig[r].absent_first, b_abs = mig[r].absent_last;
-        const int64_t s = bytes[mig[r].tensor];
-        int hi = b_abs;                     // slots (j, b_abs] are known to take the tensor
-        int j = a_abs - 1;                  // result: last slot that stays absent
-        while (hi >= a_abs) {
-            const int lo = hi - kPfThreads + 1 > a_abs ? hi - kPfThreads + 1 : a_abs;
-            if (threadIdx.x == 0) s_stop = -1;
-            __syncthreads();
-            const int k = hi - (int)threadIdx.x;
-            if (k >= lo && P[k] > cap - s) atomicMax(&s_stop, k);
-            __syncthreads();
-            const int stop = s_stop;
-            __syncthreads();
-            if (stop >= 0) { j = stop; break; }
-            hi = lo - 1;
-        }
-        for (int k = j + 1 + (int)threadIdx.x; k <= b_abs; k += kPfThreads) P[k] += s;
-        if (threadIdx.x == 0) {
-            new_last[r] = j;
-            new_issue[r] = j < b_abs ? start[j + 1] : mig[r].prefetch_issue_ns;
-        }
-        if (j < b_abs) { moved += 1; regained += b_abs - j; }
         __syncthreads();
+        for (int64_t k = 2; k <= n2; k <<= 1) {
+            for (int64_t j = k >> 1; j > 0; j >>= 1) {
+                const bool mirror = (j == (k >> 1));
+                for (int64_t t = threadIdx.x; t < n2 / 2; t += kPfThreads) {
+                    const int64_t blk = t / j, off = t % j;
+                    const int64_t i = blk * 2 * j + off;
+                    const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
+                    const long long kx = s_key[i], ky = s_key[p];
+                    const int ix = s_idx[i], iy = s_idx[p];
+                    if (ky < kx || (ky == kx && iy < ix)) { s_key[i] = ky; s_key[p] = kx; s_idx[i] = iy; s_idx[p] = ix; }
+                }
+                __syncthreads();
+            }
+        }
+        for (int64_t i = threadIdx.x; i < n; i += kPfThreads) order[i] = s_idx[i];
+        __syncthreads();
+    } else {
+        for (int64_t i = threadIdx.x; i < n; i += kPfThreads) order[i] = (int32_t)i;
+        __syncthreads();
+        for (int64_t k = 2; k <= n2; k <<= 1) {
+            for (int64_t j = k >> 1; j > 0; j >>= 1) {
+                const bool mirror = (j == (k >> 1));
+                for (int64_t t = threadIdx.x; t < n2 / 2; t += kPfThreads) {
+                    const int64_t blk = t / j, off = t % j;
+                    const int64_t i = blk * 2 * j + off;
+                    const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
+                    if (p < n) {
+                        const int32_t x = order[i], y = order[p];
+                        if (pf_before(mig, y, x)) { order[i] = y; order[p] = x; }
+                    }
+                }
+                __syncthreads();
+            }
+        }
     }
+    // ---- visit the records in that order, a batch of kPfThreads at a time: the batch's fields are fetched together
+    // (one thread per record), the visits read them from shared memory; the pressure curve sits in shared memory
+    // too when it fits (Pw), else in global memory
+    long long moved = 0, regained = 0;
+    int turn = 0;
+    for (int64_t q0 = 0; q0 < n; q0 += kPfThreads) {
+        const int nb = (int)(n - q0 < kPfThreads ? n - q0 : kPfThreads);
+        __syncthreads();
+        if ((int)threadIdx.x < nb) {
+            const int r = order[q0 + threadIdx.x];
+            s_ra[threadIdx.x] = mig[r].absent_first; s_rb[threadIdx.x] = mig[r].absent_last;
+            s_rs[threadIdx.x] = bytes[mig[r].tensor];
+        }
+        __syncthreads();
+        for (int q = 0; q < nb; ++q) {
+            const int a_abs = s_ra[q], b_abs = s_rb[q];
+            const int64_t s = s_rs[q];
+            int hi = b_abs;                     // slots (j, b_abs] are known to take the tensor
+            int j = a_abs - 1;                  // result: last slot that stays absent
+            while (hi >= a_abs) {
+                const int lo = hi - kPfThreads + 1 > a_abs ? hi - kPfThreads + 1 : a_abs;
+                // threads look at slots hi, hi - 1, ...: the first failing lane of the first failing warp is the highest slot
+                const int k = hi - (int)threadIdx.x;
+                const unsigned fail = __ballot_sync(0xffffffffu, k >= lo && Pw[k] > cap - s);
+                if (lane == 0) s_wstop[turn][warp] = fail ? hi - (warp * 32 + __ffs(fail) - 1) : -1;
+                __syncthreads();
+                int stop = -1;
+                const int mine = lane < kPfThreads / 32 ? s_wstop[turn][lane] : -1;      // one warp result per lane
+                const unsigned any = __ballot_sync(0xffffffffu, mine >= 0);
+                if (any) stop = __shfl_sync(0xffffffffu, mine, __ffs(any) - 1);
+                turn ^= 1;                                                   // (the other copy was last read two barriers ago)
+                if (stop >= 0) { j = stop; break; }
+                hi = lo - 1;
+            }
+            for (int k = j + 1 + (int)threadIdx.x; k <= b_abs; k += kPfThreads) Pw[k] += s;
+            if (threadIdx.x == 0) s_rj[q] = j;
+            if (j < b_abs) { moved += 1; regained += b_abs - j; }
+            __syncthreads();
+        }
+        if ((int)threadIdx.x < nb) {
+            const int r = order[q0 + threadIdx.x];
+            const int j = s_rj[threadIdx.x];
+            new_last[r] = j;
+            new_issue[r] = j < s_rb[threadIdx.x] ? start[j + 1] : mig[r].prefetch_issue_ns;
+        }
+    }
+    __syncthreads();
+    if (p_in_smem) for (int64_t k = threadIdx.x; k < K; k += kPfThreads) P[k] = Pw[k];
+    __syncthreads();
     // ---- new peak and its lowest slot
     long long mx = 0;
     int sl = -1;
@@ -103,7 +164,20 @@ cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *
                                      int64_t *summary, cudaStream_t s)
 {
     const int64_t cap = gpu_capacity_bytes >= ((uint64_t)1 << 63) ? INT64_MAX : (int64_t)gpu_capacity_bytes;
-    k_schedule_prefetch<<<1, kPfThreads, 0, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary);
+    // the pressure curve in shared memory if it fits beside the kernel's own arrays
+    static_assert(kPfThreads / 32 <= 32, "one warp result per lane");
+    size_t dyn = 0;
+    int in_smem = 0;
+    if (K > 0 && (size_t)K * 8 <= 120 * 1024) { dyn = (size_t)K * 8; in_smem = 1; }
+    int64_t n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    int sort_smem = 0;
+    if (n > 0 && (size_t)n2 * 12 <= 64 * 1024) { dyn += (size_t)n2 * 12; sort_smem = 1; }
+    if (dyn > 0) {
+        const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+        if (e != cudaSuccess) return e;
+    }
+    k_schedule_prefetch<<<1, kPfThreads, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem);
     return cudaGetLastError();
 }
 
