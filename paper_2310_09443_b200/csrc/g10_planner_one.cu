@@ -87,11 +87,75 @@ __device__ __forceinline__ bool window_conflict_cyc(const int64_t *sStart, const
            window_conflict<true, false>(sStart, busy, wk0, wk1, 0, 0, q0 - T, q1 - T, qk0 - Kc, qk1 - Kc, Kc);
 }
 
+
+// Pressure tiles: 32 consecutive slots with their smallest and largest pressure.  A tile wholly at least s above the
+// capacity counts s for its whole time in a benefit, one wholly within capacity nothing; only the others are read.
+constexpr int kTileO = 32;
+
+// smallest / largest pressure of tile t, by one warp (pressures are never negative: compared as unsigned halves)
+__device__ __forceinline__ void tile_refresh_warp(const int64_t *sP, int K, int t, int64_t *tmin, int64_t *tmax, int lane)
+{
+    const int k = t * kTileO + lane;
+    const bool in = k < K;
+    const ull v = in ? (ull)sP[k] : 0ull;
+    const unsigned hi = (unsigned)(v >> 32), lo = (unsigned)v;
+    const unsigned xh = __reduce_max_sync(0xffffffffu, in ? hi : 0u);
+    const unsigned xl = __reduce_max_sync(0xffffffffu, in && hi == xh ? lo : 0u);
+    const unsigned nh = __reduce_min_sync(0xffffffffu, in ? hi : 0xffffffffu);
+    const unsigned nl = __reduce_min_sync(0xffffffffu, in && hi == nh ? lo : 0xffffffffu);
+    if (lane == 0) { tmax[t] = (int64_t)(((ull)xh << 32) | xl); tmin[t] = (int64_t)(((ull)nh << 32) | nl); }
+}
+
+// Benefit of physical slots [lo, hi] for a tensor of s bytes, by one warp: every lane's share (sum them afterwards).
+__device__ __forceinline__ u128 benefit_tiles_warp(const int64_t *sP, const int64_t *sStart, const int64_t *tmin, const int64_t *tmax,
+                                                   int64_t cap, int64_t s, int lo, int hi, int lane)
+{
+    u128 acc = 0;
+    const int ta = lo / kTileO, tb = hi / kTileO;
+#pragma unroll 1
+    for (int t0 = ta; t0 <= tb; t0 += 32) {
+        const int t = t0 + lane;
+        bool mixed = false;
+        if (t <= tb) {
+            const int k_lo = t * kTileO > lo ? t * kTileO : lo, k_hi = t * kTileO + kTileO - 1 < hi ? t * kTileO + kTileO - 1 : hi;
+            const int64_t mn = tmin[t], mx = tmax[t];
+            if (mx > cap) {
+                if (mn >= cap && mn - cap >= s) acc += (u128)(ull)s * (u128)(ull)(sStart[k_hi + 1] - sStart[k_lo]);
+                else mixed = true;
+            }
+        }
+        unsigned m = __ballot_sync(0xffffffffu, mixed);
+#pragma unroll 1
+        while (m) {
+            const int tt = t0 + __ffs(m) - 1;
+            m &= m - 1;
+            const int k = tt * kTileO + lane;
+            if (k >= lo && k <= hi) {
+                int64_t ex = sP[k] - cap;
+                if (ex > 0) {
+                    if (ex > s) ex = s;
+                    acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
+                }
+            }
+        }
+    }
+    return acc;
+}
+
+// The same for an unrolled slot range [a, b] (at most Kc slots long when Kc != 0): its one or two physical pieces.
+__device__ __forceinline__ u128 benefit_range_warp(const int64_t *sP, const int64_t *sStart, const int64_t *tmin, const int64_t *tmax,
+                                                   int64_t cap, int64_t s, int a, int b, int Kc, int lane)
+{
+    if (!Kc || b < Kc) return benefit_tiles_warp(sP, sStart, tmin, tmax, cap, s, a, b, lane);
+    if (a >= Kc) return benefit_tiles_warp(sP, sStart, tmin, tmax, cap, s, a - Kc, b - Kc, lane);
+    return benefit_tiles_warp(sP, sStart, tmin, tmax, cap, s, a, Kc - 1, lane) + benefit_tiles_warp(sP, sStart, tmin, tmax, cap, s, 0, b - Kc, lane);
+}
+
 __host__ __device__ inline size_t one_smem_need(int64_t K, int64_t Pn, bool host_cap, bool cyclic = false)
 {
     const int64_t groups = (Pn + 31) / 32;
     return (size_t)(2 * K + 1) * 8 + (cyclic ? (size_t)K * 8 : 0) + (size_t)4 * K * 8 + (host_cap ? (size_t)K * 8 : 0) + (size_t)groups * 32 * 8 + (size_t)Pn * 41 +
-           (size_t)groups * 13 + 128;
+           (size_t)groups * 13 + (size_t)((K + 31) / 32) * 16 + 128;
 }
 
 // Warp-wide maximum of 64-bit keys with the lowest index among equal keys; same result in every lane.
@@ -168,7 +232,10 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
     int64_t *sStart = sP + K;
     int64_t *sBusy = sStart + (kCyclic ? 2 * K : K) + 1; // [4][K]  (the clock has 2K + 1 entries in cyclic mode)
     int64_t *sHocc = sBusy + (size_t)4 * K;             // [K] if host_cap
-    ull *ckey = (ull *)(sHocc + (host_cap ? K : 0));    // [G1 * 32] bits of the rounded score (0 = none)
+    const int NT = (K + kTileO - 1) / kTileO;
+    int64_t *tmin = sHocc + (host_cap ? K : 0);         // [NT] smallest pressure of each tile of 32 slots
+    int64_t *tmax = tmin + NT;                          // [NT] largest
+    ull *ckey = (ull *)(tmax + NT);                     // [G1 * 32] bits of the rounded score (0 = none)
     ull *gkey = ckey + (size_t)G1 * 32;                 // [G1] maximum of each group
     int64_t *cbytes = (int64_t *)(gkey + G1);
     int64_t *ct = cbytes + Pn;                          // transfer time of the current destination
@@ -238,6 +305,8 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
         if (lane == 0 && over) atomicAdd(&s_n_over, over);
     }
     __syncthreads();
+    for (int t = warp; t < NT; t += kOneWarps) tile_refresh_warp(sP, K, t, tmin, tmax, lane);
+    __syncthreads();
 
     int64_t n_mig = 0, rounds = 0, bytes_ssd = 0, bytes_host = 0;
     int status = -1;
@@ -306,16 +375,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                         continue;
                     }
                     ONE_COUNT(1);
-                    u128 acc = 0;
-#pragma unroll 1
-                    for (int k = ap + lane; k <= bp; k += 32) {
-                        int64_t ex = sP[phys_slot(k, Kc)] - A.cap;
-                        if (ex > 0) {
-                            if (ex > s) ex = s;
-                            acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
-                        }
-                    }
-                    acc = warp_sum_u128(acc);
+                    const u128 acc = warp_sum_u128(benefit_range_warp(sP, sStart, tmin, tmax, A.cap, s, ap, bp, Kc, lane));
                     if (lane == 0) {
                         Cand cd;
                         cd.ben = acc; cd.cost = 2ull * (ull)t; cd.idx = 0; cd.dest = d;
@@ -333,126 +393,122 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             if (tid == 0) { s_ndirty = 0; s_nlist = 0; }
             ONE_CLOCK(1);
         }
-        // ---------------- 2. search: refresh the group maxima that changed, take the top, rescore it while it is stale
+        // ---------------- 2. search: warp 0 refreshes the group maxima that changed, takes the top and, while the top is
+        // STALE, rescores it (from the pressure tiles) and looks again; the other warps wait at the barrier
         int win = -1;
         bool exhausted = false;
+        // rescoring of one period by warp 0 (uniform arguments)
+        auto rescore_warp0 = [&](int target) {
+            const OneRanges r = crng[target];
+            const u128 tot = warp_sum_u128(benefit_range_warp(sP, sStart, tmin, tmax, A.cap, cbytes[target], r.ap, r.bp, Kc, lane));
+            if (lane == 0) {
+                Cand cd;
+                cd.ben = tot; cd.cost = 2ull * (ull)ct[target]; cd.idx = 0; cd.dest = 0;
+                cben_lo[target] = (ull)tot; cben_hi[target] = (ull)(tot >> 64);
+                ckey[target] = tot == 0 ? 0ull : (ull)__double_as_longlong(cand_key(cd));
+                cstate[target] = (unsigned char)((cstate[target] & 3) | kFreshO);
+                gflag[target >> 5] = 1; s_flagged = 1;
+            }
+            __syncwarp();
+        };
 #pragma unroll 1
         for (;;) {
             if (warp == 0) {
-                if (s_flagged) {
-                __syncwarp();
-                if (lane == 0) s_flagged = 0;
 #pragma unroll 1
-                for (int g0 = 0; g0 < G1; g0 += 32) {
-                    unsigned m = __ballot_sync(0xffffffffu, g0 + lane < G1 && gflag[g0 + lane] != 0);
+                for (;;) {
+                    if (s_flagged) {
+                        __syncwarp();
+                        if (lane == 0) s_flagged = 0;
 #pragma unroll 1
-                    while (m) {
-                        const int g = g0 + __ffs(m) - 1;
-                        m &= m - 1;
-                        ull mk; int mi;
-                        warp_argmax_u64(ckey[g * 32 + lane], g * 32 + lane, &mk, &mi);
-                        if (lane == 0) { gkey[g] = mk; garg[g] = mi; gflag[g] = 0; }
+                        for (int g0 = 0; g0 < G1; g0 += 32) {
+                            unsigned m = __ballot_sync(0xffffffffu, g0 + lane < G1 && gflag[g0 + lane] != 0);
+#pragma unroll 1
+                            while (m) {
+                                const int g = g0 + __ffs(m) - 1;
+                                m &= m - 1;
+                                ull mk; int mi;
+                                warp_argmax_u64(ckey[g * 32 + lane], g * 32 + lane, &mk, &mi);
+                                if (lane == 0) { gkey[g] = mk; garg[g] = mi; gflag[g] = 0; }
+                            }
+                        }
                     }
-                }
-                }
-                __syncwarp();
-                ull bk = 0; int bi = 0x7fffffff;
+                    __syncwarp();
+                    ull bk = 0; int bi = 0x7fffffff;
 #pragma unroll 4
-                for (int g = lane; g < G1; g += 32) {
-                    const ull k = gkey[g];
-                    if (k > bk) { bk = k; bi = garg[g]; }         // g ascending: the lowest index stays on ties
+                    for (int g = lane; g < G1; g += 32) {
+                        const ull k = gkey[g];
+                        if (k > bk) { bk = k; bi = garg[g]; }         // g ascending: the lowest index stays on ties
+                    }
+                    ull mk; int mi;
+                    warp_argmax_u64(bk, bi, &mk, &mi);
+                    if (mk == 0 || (cstate[mi] & kStateMaskO) != kStaleO) {
+                        if (lane == 0) { s_topkey = mk; s_top = mi; }
+                        break;
+                    }
+                    ONE_COUNT(3);
+                    rescore_warp0(mi);
                 }
-                ull mk; int mi;
-                warp_argmax_u64(bk, bi, &mk, &mi);
-                if (lane == 0) { s_topkey = mk; s_top = mi; }
             }
             __syncthreads();
             ONE_CLOCK(2);
             const ull topkey = s_topkey;
             const int top = s_top;
             if (topkey == 0) { exhausted = true; break; }
-            int target = -1;
-            if ((cstate[top] & kStateMaskO) == kStaleO) target = top;
-            else {
-                // a fresh top: can anything else within 1e-10 of it beat it exactly?  (A stale entry competes with
-                // its bound: if even the bound loses, the period cannot win this iteration.)
-                const double thr = __longlong_as_double((long long)topkey) * (1.0 - 1e-10);
-                const ull thr_bits = (ull)__double_as_longlong(thr);
-                bool other = false;
+            // a fresh top: can anything else within 1e-10 of it beat it exactly?  (A stale entry competes with its
+            // bound: if even the bound loses, the period cannot win this iteration.)
+            const double thr = __longlong_as_double((long long)topkey) * (1.0 - 1e-10);
+            const ull thr_bits = (ull)__double_as_longlong(thr);
+            bool other = false;
 #pragma unroll 4
-                for (int g = warp; g < G1; g += kOneWarps) {
-                    if (gkey[g] < thr_bits) continue;
-                    const int li = g * 32 + lane;
-                    if (ckey[li] < thr_bits || li == top) continue;
-                    Cand x, y;
-                    x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
-                    y.ben = ((u128)cben_hi[top] << 64) | cben_lo[top]; y.cost = 2ull * (ull)ct[top]; y.idx = top; y.dest = 0;
-                    if (!cand_beats(x, y)) continue;
-                    other = true;
-                    if ((cstate[li] & kStateMaskO) == kStaleO) atomicMin(&s_force, li);
-                    else { const int pos = atomicAdd(&s_nfin, 1); if (pos < kOneMaxFin) s_fin[pos] = li; }
-                }
-                if (!__syncthreads_or(other)) { win = top; break; }
-                if (s_force != 0x7fffffff) target = s_force;
-                else {
-                    if (tid == 0) {
-                        Cand w;
-                        w.ben = ((u128)cben_hi[top] << 64) | cben_lo[top]; w.cost = 2ull * (ull)ct[top]; w.idx = top; w.dest = 0;
-                        const int n = s_nfin;
-                        if (n <= kOneMaxFin) {
-                            for (int i = 0; i < n; ++i) {
-                                const int li = s_fin[i];
-                                Cand x;
-                                x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
-                                if (cand_beats(x, w)) w = x;
-                            }
-                        } else {
-                            for (int li = 0; li < Pn; ++li) {      // very many close scores: plain sweep
-                                if (ckey[li] < thr_bits || (cstate[li] & kStateMaskO) != kFreshO) continue;
-                                Cand x;
-                                x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
-                                if (cand_beats(x, w)) w = x;
-                            }
-                        }
-                        s_win = w.idx; s_nfin = 0;
-                    }
-                    __syncthreads();
-                    win = s_win;
-                    break;
-                }
+            for (int g = warp; g < G1; g += kOneWarps) {
+                if (gkey[g] < thr_bits) continue;
+                const int li = g * 32 + lane;
+                if (ckey[li] < thr_bits || li == top) continue;
+                Cand x, y;
+                x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
+                y.ben = ((u128)cben_hi[top] << 64) | cben_lo[top]; y.cost = 2ull * (ull)ct[top]; y.idx = top; y.dest = 0;
+                if (!cand_beats(x, y)) continue;
+                other = true;
+                if ((cstate[li] & kStateMaskO) == kStaleO) atomicMin(&s_force, li);
+                else { const int pos = atomicAdd(&s_nfin, 1); if (pos < kOneMaxFin) s_fin[pos] = li; }
             }
-            ONE_CLOCK(3);
-            // the whole block rescores period `target`
-            {
-                const OneRanges r = crng[target];
-                const int64_t s = cbytes[target];
-                u128 acc = 0;
-#pragma unroll 1
-                for (int k = r.ap + tid; k <= r.bp; k += kOneThreads) {
-                    int64_t ex = sP[phys_slot(k, Kc)] - A.cap;
-                    if (ex > 0) {
-                        if (ex > s) ex = s;
-                        acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
+            if (!__syncthreads_or(other)) { win = top; break; }
+            const int forced = s_force;
+            if (forced != 0x7fffffff) {
+                // a stale period whose bound beats the top exactly: rescore it, then search again
+                __syncthreads();                   // everyone has read s_force
+                if (warp == 0) {
+                    rescore_warp0(forced);
+                    if (lane == 0) { s_force = 0x7fffffff; s_nfin = 0; }
+                    __syncwarp();
+                }
+                ONE_CLOCK(4);
+                continue;
+            }
+            if (tid == 0) {
+                Cand w;
+                w.ben = ((u128)cben_hi[top] << 64) | cben_lo[top]; w.cost = 2ull * (ull)ct[top]; w.idx = top; w.dest = 0;
+                const int n = s_nfin;
+                if (n <= kOneMaxFin) {
+                    for (int i = 0; i < n; ++i) {
+                        const int li = s_fin[i];
+                        Cand x;
+                        x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
+                        if (cand_beats(x, w)) w = x;
+                    }
+                } else {
+                    for (int li = 0; li < Pn; ++li) {      // very many close scores: plain sweep
+                        if (ckey[li] < thr_bits || (cstate[li] & kStateMaskO) != kFreshO) continue;
+                        Cand x;
+                        x.ben = ((u128)cben_hi[li] << 64) | cben_lo[li]; x.cost = 2ull * (ull)ct[li]; x.idx = li; x.dest = 0;
+                        if (cand_beats(x, w)) w = x;
                     }
                 }
-                acc = warp_sum_u128(acc);
-                if (lane == 0) { s_part[2 * warp] = (ull)acc; s_part[2 * warp + 1] = (ull)(acc >> 64); }
-                __syncthreads();
-                if (tid == 0) {
-                    u128 tot = 0;
-#pragma unroll
-                    for (int w = 0; w < kOneWarps; ++w) tot += ((u128)s_part[2 * w + 1] << 64) | s_part[2 * w];
-                    Cand cd;
-                    cd.ben = tot; cd.cost = 2ull * (ull)ct[target]; cd.idx = 0; cd.dest = 0;
-                    cben_lo[target] = (ull)tot; cben_hi[target] = (ull)(tot >> 64);
-                    ckey[target] = tot == 0 ? 0ull : (ull)__double_as_longlong(cand_key(cd));
-                    cstate[target] = (unsigned char)((cstate[target] & 3) | kFreshO);
-                    gflag[target >> 5] = 1; s_flagged = 1;
-                    s_force = 0x7fffffff; s_nfin = 0;
-                }
-                __syncwarp();                   // warp 0 goes straight on to the refresh; the others wait at the barrier above
+                s_win = w.idx; s_nfin = 0;
             }
-            ONE_CLOCK(4);
+            __syncthreads();
+            win = s_win;
+            break;
         }
         if (exhausted) { status = G10_EXHAUSTED; break; }
         ONE_CLOCK(5);
@@ -492,6 +548,13 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
 #pragma unroll 1
                 for (int k = wa + tid; k <= wb; k += kOneThreads) sHocc[phys_slot(k, Kc)] += s;
             __syncthreads();                       // the bookings are in place for the conflict tests below
+            // the pressure tiles the commit touched (one or two physical pieces of the absent range), one warp per tile
+            {
+                const int lo0 = phys_slot(wap, Kc), hi0 = (Kc && wap < Kc && wbp >= Kc) ? Kc - 1 : phys_slot(wbp, Kc);
+                for (int t = lo0 / kTileO + warp; t <= hi0 / kTileO; t += kOneWarps) tile_refresh_warp(sP, K, t, tmin, tmax, lane);
+                if (Kc && wap < Kc && wbp >= Kc)
+                    for (int t = warp; t <= (wbp - Kc) / kTileO; t += kOneWarps) tile_refresh_warp(sP, K, t, tmin, tmax, lane);
+            }
             int newly_dirty = 0;
 #pragma unroll 2
             for (int li = tid; li < Pn; li += kOneThreads) {
