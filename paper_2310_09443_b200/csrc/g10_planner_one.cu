@@ -88,60 +88,6 @@ __device__ __forceinline__ bool window_conflict_cyc(const int64_t *sStart, const
 }
 
 
-// Pressure tiles: 32 consecutive slots with their smallest and largest pressure.  A tile wholly at least s above the
-// capacity counts s for its whole time in a benefit, one wholly within capacity nothing; only the others are read.
-constexpr int kTileO = 32;
-
-// smallest / largest pressure of tile t, by one warp (pressures are never negative: compared as unsigned halves)
-__device__ __forceinline__ void tile_refresh_warp(const int64_t *sP, int K, int t, int64_t *tmin, int64_t *tmax, int lane)
-{
-    const int k = t * kTileO + lane;
-    const bool in = k < K;
-    const ull v = in ? (ull)sP[k] : 0ull;
-    const unsigned hi = (unsigned)(v >> 32), lo = (unsigned)v;
-    const unsigned xh = __reduce_max_sync(0xffffffffu, in ? hi : 0u);
-    const unsigned xl = __reduce_max_sync(0xffffffffu, in && hi == xh ? lo : 0u);
-    const unsigned nh = __reduce_min_sync(0xffffffffu, in ? hi : 0xffffffffu);
-    const unsigned nl = __reduce_min_sync(0xffffffffu, in && hi == nh ? lo : 0xffffffffu);
-    if (lane == 0) { tmax[t] = (int64_t)(((ull)xh << 32) | xl); tmin[t] = (int64_t)(((ull)nh << 32) | nl); }
-}
-
-// Benefit of physical slots [lo, hi] for a tensor of s bytes, by one warp: every lane's share (sum them afterwards).
-__device__ __forceinline__ u128 benefit_tiles_warp(const int64_t *sP, const int64_t *sStart, const int64_t *tmin, const int64_t *tmax,
-                                                   int64_t cap, int64_t s, int lo, int hi, int lane)
-{
-    u128 acc = 0;
-    const int ta = lo / kTileO, tb = hi / kTileO;
-#pragma unroll 1
-    for (int t0 = ta; t0 <= tb; t0 += 32) {
-        const int t = t0 + lane;
-        bool mixed = false;
-        if (t <= tb) {
-            const int k_lo = t * kTileO > lo ? t * kTileO : lo, k_hi = t * kTileO + kTileO - 1 < hi ? t * kTileO + kTileO - 1 : hi;
-            const int64_t mn = tmin[t], mx = tmax[t];
-            if (mx > cap) {
-                if (mn >= cap && mn - cap >= s) acc += (u128)(ull)s * (u128)(ull)(sStart[k_hi + 1] - sStart[k_lo]);
-                else mixed = true;
-            }
-        }
-        unsigned m = __ballot_sync(0xffffffffu, mixed);
-#pragma unroll 1
-        while (m) {
-            const int tt = t0 + __ffs(m) - 1;
-            m &= m - 1;
-            const int k = tt * kTileO + lane;
-            if (k >= lo && k <= hi) {
-                int64_t ex = sP[k] - cap;
-                if (ex > 0) {
-                    if (ex > s) ex = s;
-                    acc += (u128)(ull)ex * (u128)(ull)(sStart[k + 1] - sStart[k]);
-                }
-            }
-        }
-    }
-    return acc;
-}
-
 // The same for an unrolled slot range [a, b] (at most Kc slots long when Kc != 0): its one or two physical pieces.
 __device__ __forceinline__ u128 benefit_range_warp(const int64_t *sP, const int64_t *sStart, const int64_t *tmin, const int64_t *tmax,
                                                    int64_t cap, int64_t s, int a, int b, int Kc, int lane)

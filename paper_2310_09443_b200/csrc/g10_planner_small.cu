@@ -143,6 +143,9 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
     PeriodInfo *info = (PeriodInfo *)(ckey + S.cand_cap);
     unsigned char *cstate = (unsigned char *)(info + S.cand_cap);
     unsigned char *cskip = cstate + S.cand_cap;             // STALE period that cannot be this block's proposal in this iteration
+    const int NT = (K + kTileO - 1) / kTileO;
+    int64_t *tmin = (int64_t *)(((uintptr_t)(cskip + S.cand_cap) + 7) & ~(uintptr_t)7);   // [NT] smallest pressure per tile of 32 slots
+    int64_t *tmax = tmin + NT;                                                             // [NT] largest
     int64_t *busy = S.busy_rep + (size_t)c * 4 * K;
     int64_t *hocc = S.hocc_rep + (size_t)c * K;
 #ifdef G10_PHASE_CLOCKS
@@ -185,6 +188,8 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
         if (A.host_capacity != 0) for (int k = threadIdx.x; k < K; k += kPlanThreads) hocc[k] = 0;
         if (over) atomicAdd(&s_n_over, over);
     }
+    __syncthreads();
+    for (int t = warp; t < NT; t += kPlanWarps) tile_refresh_warp(sP, K, t, tmin, tmax, lane);
     __syncthreads();
 
     int64_t n_mig = 0, rounds = 0, bytes_ssd = 0, bytes_host = 0;
@@ -255,11 +260,11 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
         if (kFew) {
             // Few periods per block.  A STALE period's cached score is an upper bound (pressure only falls), so
             // only the STALE periods whose bound could still beat the best FRESH score are rescored, best bound
-            // first, by the whole block; the loop ends when the block's best is FRESH (exact).  Rounded ratios
+            // first, by warp 0 from the pressure tiles; the loop ends when the block's best is FRESH (exact).  Rounded ratios
             // (ckey) steer the search; anything within 1e-10 of a decision is settled by exact comparison.
+            if (warp == 0) {
 #pragma unroll 1
-            for (;;) {
-                if (warp == 0) {
+                for (;;) {
                     double kf = -1.0, ks = -1.0;
                     int lf = -1, ls = -1;
 #pragma unroll 1
@@ -363,43 +368,26 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                         if (lane < kXWords)
                             st_volatile_u64(&S.xwords[((size_t)par * G + c) * kXWords + lane], tag | ((const unsigned *)&s_pay)[lane]);
                     }
-                    if (lane == 0) s_todo = todo;
-                }
-                __syncthreads();
-                const int li = s_todo;
-                if (li == -1) break;
-                if (li == -2) continue;
-                // the whole block rescores period li
-                {
-                    const unsigned char st = cstate[li];
-                    const int d = (st & 3) - 1;
-                    const int ap = info[li].ap[d], bp = info[li].bp[d];
-                    const int64_t s = info[li].bytes;
-                    u128 acc = 0;
-#pragma unroll 2
-                    for (int k = ap + (int)threadIdx.x; k <= bp; k += kPlanThreads) {
-                        int64_t ex = sP[k] - A.cap;
-                        if (ex > 0) {
-                            if (ex > s) ex = s;
-                            acc += (u128)(ull)ex * (u128)(ull)sDur[k];
+                    if (todo == -1) break;                     // published
+                    if (todo == -2) { __syncwarp(); continue; }
+                    // warp 0 rescores period `todo` from the pressure tiles and looks again
+                    {
+                        const int li = todo;
+                        const unsigned char st = cstate[li];
+                        const int d = (st & 3) - 1;
+                        const u128 tot = warp_sum_u128(benefit_tiles_warp(sP, sStart, tmin, tmax, A.cap, info[li].bytes, info[li].ap[d], info[li].bp[d], lane));
+                        if (lane == 0) {
+                            Cand cd;
+                            cd.ben = tot; cd.cost = 2ull * (ull)info[li].t[d]; cd.idx = 0; cd.dest = d;
+                            cben_lo[li] = (ull)tot; cben_hi[li] = (ull)(tot >> 64);
+                            ckey[li] = tot == 0 ? 0.0 : cand_key(cd);
+                            cstate[li] = (unsigned char)((d + 1) | (kFreshS << 2));
                         }
+                        __syncwarp();
                     }
-                    acc = warp_sum_u128(acc);
-                    if (lane == 0) { s_part[2 * warp] = (ull)acc; s_part[2 * warp + 1] = (ull)(acc >> 64); }
-                    __syncthreads();
-                    if (threadIdx.x == 0) {
-                        u128 tot = 0;
-#pragma unroll 1
-                        for (int w = 0; w < kPlanWarps; ++w) tot += ((u128)s_part[2 * w + 1] << 64) | s_part[2 * w];
-                        Cand cd;
-                        cd.ben = tot; cd.cost = 2ull * (ull)info[li].t[d]; cd.idx = 0; cd.dest = d;
-                        cben_lo[li] = (ull)tot; cben_hi[li] = (ull)(tot >> 64);
-                        ckey[li] = tot == 0 ? 0.0 : cand_key(cd);
-                        cstate[li] = (unsigned char)((d + 1) | (kFreshS << 2));
-                    }
-                    __syncthreads();
                 }
             }
+            __syncthreads();
         } else {
             Cand best;
             best.ben = 0; best.cost = 1; best.idx = -1; best.dest = -1;
@@ -552,6 +540,8 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             }
             n_mig += 1;
             if (X == G10_DEST_SSD) bytes_ssd += s; else bytes_host += s;
+            __syncthreads();                               // the pressure is updated: refresh the tiles the commit touched
+            for (int tl = wap / kTileO + warp; tl <= wbp / kTileO; tl += kPlanWarps) tile_refresh_warp(sP, K, tl, tmin, tmax, lane);
         }
         __syncthreads();
         PHASE_CLOCK(6);     // apply + barrier
@@ -593,7 +583,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
 // Shared memory the small-trace planner needs for K slots and `cand_cap` periods per block.
 static size_t small_smem_bytes(int64_t K, int cand_cap)
 {
-    return (size_t)(3 * K + 1) * 8 + (size_t)cand_cap * (24 + sizeof(PeriodInfo) + 2) + 16;
+    return (size_t)(3 * K + 1) * 8 + (size_t)cand_cap * (24 + sizeof(PeriodInfo) + 2) + 16 + 8 + (size_t)((K + 31) / 32) * 16;
 }
 
 bool plan_small_fits(int64_t K, int64_t E, int G, int *cand_cap_out, size_t *smem_out)
