@@ -315,6 +315,17 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                         }
                         if (__popc(fin) == 1) src = __ffs(fin) - 1;
                         else if (fin != 0u) {
+                            // usual case of a tie: identical benefit and cost (repeated layers): the lowest index wins
+                            const int f0 = __ffs(fin) - 1;
+                            // (every lane takes part in the shuffles: no short-circuit around them)
+                            const ull b0 = __shfl_sync(0xffffffffu, (ull)best.ben, f0);
+                            const ull b1 = __shfl_sync(0xffffffffu, (ull)(best.ben >> 64), f0);
+                            const ull c0 = __shfl_sync(0xffffffffu, best.cost, f0);
+                            const bool same = !((fin >> lane) & 1u) || ((ull)best.ben == b0 && (ull)(best.ben >> 64) == b1 && best.cost == c0);
+                            if (__all_sync(0xffffffffu, same)) {
+                                const unsigned lowest = __reduce_min_sync(0xffffffffu, ((fin >> lane) & 1u) ? (unsigned)best.idx : 0xffffffffu);
+                                src = __ffs(__ballot_sync(0xffffffffu, ((fin >> lane) & 1u) && (unsigned)best.idx == lowest)) - 1;
+                            } else {
                             Cand z = best;
                             if (!((fin >> lane) & 1u)) z.idx = -1;
 #pragma unroll 1
@@ -323,6 +334,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                                 if (cand_beats(y, z)) z = y;
                             }
                             src = __ffs(__ballot_sync(0xffffffffu, best.idx >= 0 && best.idx == z.idx)) - 1;
+                            }
                         }
                     }
                     Cand zbest = best;
