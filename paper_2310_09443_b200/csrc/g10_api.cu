@@ -317,8 +317,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     int64_t *pk = host ? w.peak_bytes : out->peak_bytes;
     int32_t *ps = host ? w.peak_slot : out->peak_slot;
     int64_t *st = host ? w.counts + 2 : out->status;
-    CU(launch_slot_clock(d, w, start, s));
-    CU(launch_first_last(d, w, w.first_use, w.last_use, s));
+    CU(launch_clock_and_first_last(d, w, start, w.first_use, w.last_use, s));
     CU(launch_pressure(d, w, w.first_use, w.last_use, true, P, pk, ps, s));
     CU(launch_publish_status(w, st, s));
     if (host) {

@@ -156,6 +156,8 @@ constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock f
 
 // passes (g10_passes.cu)
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);
+cudaError_t launch_clock_and_first_last(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *first_use, int32_t *last_use,
+                                        cudaStream_t s);
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 // bucketed formulation (g10_vitality_buckets.cu); supported for up to 4096 buckets of 4096 tensors
 bool vitality_buckets_supported(int64_t N, int64_t E);

@@ -35,6 +35,9 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
     __shared__ long long s_bcast;
     __shared__ bool s_last;
     const int G = gridDim.x;
+    // Nothing later in a call reads the slot clock, so a kernel launched behind this one with programmatic stream
+    // serialisation may start as soon as every block of this grid is running (no effect on ordinary launches).
+    if (kind == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int g = next_tile(ticket);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t seg = ((n + G - 1) / G + kSegChunk - 1) / kSegChunk * kSegChunk;
@@ -274,10 +277,11 @@ constexpr int kPtrStage = 3072;
 __device__ __forceinline__ const int64_t *stage_kernel_ptr(const int64_t *__restrict__ kptr, int64_t K, int64_t base, int64_t E,
                                                            int64_t *s_ptr, int *s_lohi, int *lo_out, int *hi_out, int *shift_out)
 {
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < 32) {                      // (32-ary search by warp 0: four dependent round trips for a million kernels)
         const int64_t last = (base + kEvTile <= E ? base + kEvTile : E) - 1;
-        s_lohi[0] = kernel_of_event(kptr, 0, (int)K - 1, base);
-        s_lohi[1] = kernel_of_event(kptr, s_lohi[0], (int)K - 1, last);
+        const int klo = kernel_of_event_warp(kptr, 0, (int)K - 1, base, (int)threadIdx.x);
+        const int khi = kernel_of_event_warp(kptr, klo, (int)K - 1, last, (int)threadIdx.x);
+        if (threadIdx.x == 0) { s_lohi[0] = klo; s_lohi[1] = khi; }
     }
     __syncthreads();
     const int lo = s_lohi[0], hi = s_lohi[1];
@@ -408,6 +412,34 @@ cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t 
     if (t.E > 0 && t.K > 0) {
         const int blocks = (int)tiles_of(t.E, kEvTile);
         k_first_last_events<<<blocks, kEvThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.status);
+    }
+    return cudaGetLastError();
+}
+
+// Slot clock and first / last use for the timeline call: the two are independent, so the event kernel is launched
+// with programmatic stream serialisation and runs beside the clock scan (it never reads what the scan writes).
+cudaError_t launch_clock_and_first_last(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *first_use, int32_t *last_use,
+                                        cudaStream_t s)
+{
+    cudaError_t e;
+    if (t.N > 0) {
+        if ((e = cudaMemsetAsync(first_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
+        if ((e = cudaMemsetAsync(last_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
+    }
+    if ((e = launch_slot_clock(t, w, start, s)) != cudaSuccess) return e;
+    if (t.N > 0 && t.E > 0 && t.K > 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)tiles_of(t.E, kEvTile));
+        cfg.blockDim = dim3(kEvThreads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, k_first_last_events, t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.status);
+        if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
 }

@@ -107,27 +107,6 @@ __device__ __forceinline__ int bk_kernel_of_event(const int64_t *kptr, int lo, i
     return lo;
 }
 
-// Same, by a whole warp: every round probes 32 evenly spaced kernels at once, so that a cold search over a
-// million kernels costs four dependent round trips instead of twenty.  Result in every lane.
-__device__ __forceinline__ int bk_kernel_of_event_warp(const int64_t *__restrict__ kptr, int lo, int hi, int64_t e, int lane)
-{
-    while (hi - lo > 31) {
-        const int step = (hi - lo) / 32 + 1;
-        const int probe = lo + lane * step;                   // lane 0 probes lo, which is known to qualify
-        const bool ok = probe <= hi && kptr[probe] <= e;
-        const unsigned m = __ballot_sync(0xffffffffu, ok);     // qualifying probes form a prefix of the lanes
-        const int last = 31 - __clz(m);
-        const int nlo = lo + last * step;
-        int nhi = nlo + step - 1;
-        if (nhi > hi) nhi = hi;
-        lo = nlo; hi = nhi;
-    }
-    const int probe = lo + lane;
-    const bool ok = probe <= hi && kptr[probe] <= e;
-    const unsigned m = __ballot_sync(0xffffffffu, ok);
-    return lo + (31 - __clz(m));
-}
-
 // ---------------------------------------------------------------------------------------------
 // 1. events per bucket
 // ---------------------------------------------------------------------------------------------
@@ -180,8 +159,8 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
         const int n_tile = (int)((B.E - base) < kBkTile ? (B.E - base) : kBkTile);
         for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_cnt[b] = 0;
         if (threadIdx.x < 32) {
-            const int klo = bk_kernel_of_event_warp(kptr, 0, (int)B.K - 1, base, (int)threadIdx.x);
-            const int khi = bk_kernel_of_event_warp(kptr, klo, (int)B.K - 1, base + n_tile - 1, (int)threadIdx.x);
+            const int klo = kernel_of_event_warp(kptr, 0, (int)B.K - 1, base, (int)threadIdx.x);
+            const int khi = kernel_of_event_warp(kptr, klo, (int)B.K - 1, base + n_tile - 1, (int)threadIdx.x);
             if (threadIdx.x == 0) { s_lohi[0] = klo; s_lohi[1] = khi; }
         }
         __syncthreads();
