@@ -258,7 +258,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
     int *t_np = t_d + B.bt + 1;                // [bt + 1] periods per tensor, then their offsets
     int32_t *s_ks = t_np + B.bt + 1;           // [kBkCap] kernels, tensor segment after tensor segment
     __shared__ int s_scan[2 * (kBkThreads / 32 + 1)];
-    __shared__ int s_wa[kBkThreads / 32];
+    __shared__ int s_wa[kBkThreads / 32], s_wb[kBkThreads / 32];
     __shared__ long long s_pu[kBkThreads / 32], s_pp[kBkThreads / 32];
     __shared__ int s_bucket, s_nheavy, s_total, s_periods;
     __shared__ int s_heavy[64];
@@ -312,6 +312,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         __syncthreads();
         BK_CLOCK(3);
         // ---- short segments: one thread sorts, removes repeats (in place) and counts the periods
+        int my_d = 0, my_p = 0;                 // this thread's share of the bucket totals
         for (int tl = threadIdx.x; tl < bt_eff; tl += kBkThreads) {
             const int m = t_off[tl + 1] - t_off[tl];
             int dd = 0, pp = 0;
@@ -334,6 +335,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
                 }
             }
             t_d[tl] = dd; t_np[tl] = pp;
+            my_d += dd; my_p += pp;
         }
         __syncthreads();
         BK_CLOCK(4);
@@ -369,19 +371,26 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
                 if (threadIdx.x == 0) s_total += chunk_total;
                 __syncthreads();
             }
-            if (threadIdx.x == 0) { t_d[tl] = s_total; t_np[tl] = s_periods; }
+            if (threadIdx.x == 0) { t_d[tl] = s_total; t_np[tl] = s_periods; my_d += s_total; my_p += s_periods; }
             __syncthreads();
         }
-        // ---- offsets of every tensor's distinct uses and periods inside the bucket; bucket totals
+        // ---- the bucket's totals go out first (later buckets wait for them), then the offsets of every tensor's
+        // distinct uses and periods inside the bucket
         BK_CLOCK(5);
+        {
+            const int wd = __reduce_add_sync(0xffffffffu, my_d), wp = __reduce_add_sync(0xffffffffu, my_p);
+            if (lane == 0) { s_wa[warp] = wd; s_wb[warp] = wp; }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                long long td = 0, tp = 0;
+                for (int w = 0; w < kBkThreads / 32; ++w) { td += s_wa[w]; tp += s_wb[w]; }
+                asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&B.words[2 * b]), "l"(bk_pack(td)) : "memory");
+                asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&B.words[2 * b + 1]), "l"(bk_pack(tp)) : "memory");
+            }
+        }
         bk_block_scan<2>(t_d, t_d, t_np, t_np, bt_eff, s_scan);
         BK_CLOCK(6);
         const long long D = t_d[bt_eff], PC = t_np[bt_eff];
-        // ---- offsets of this bucket in the global arrays: totals of all earlier buckets
-        if (threadIdx.x == 0) {
-            asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&B.words[2 * b]), "l"(bk_pack(D)) : "memory");
-            asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&B.words[2 * b + 1]), "l"(bk_pack(PC)) : "memory");
-        }
         long long pu = 0, pq = 0;
         for (int j0 = threadIdx.x; j0 < 2 * b; j0 += 4 * kBkThreads) {
             ull w[4];
