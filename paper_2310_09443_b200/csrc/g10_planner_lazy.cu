@@ -31,7 +31,7 @@ struct LazyArgs {
     int *worklist;              // [2][stride] DIRTY periods of the current round
     unsigned *wl_count;         // [2]
     LazyProp *props;            // [2][kLazyMaxBlocks] each block's best FRESH candidate and best STALE bounds
-    ull *partials;              // [2][kRoundM][kLazyMaxBlocks][2] slices of the benefits rescored together
+    ull *partials;              // [3][kRoundM][2] 128-bit sums of the benefits rescored together (three buffers in turn)
     int64_t *tmin, *tmax;       // [tiles of kSlotTile slots] smallest / largest pressure of each tile
     int64_t stride;
 };
@@ -529,6 +529,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
 #define LAZY_CLOCK(i)
 #endif
 
+    if (c == 0) for (int j = threadIdx.x; j < 3 * kRoundM * 2; j += kPlanThreads) L.partials[j] = 0;
     // every period starts DIRTY: its first evaluation chooses the destination
     for (int64_t p = (int64_t)c * kPlanThreads + threadIdx.x; p < Pn; p += (int64_t)G * kPlanThreads) {
         L.c_state[p] = (unsigned char)(kDirty << 2);
@@ -812,38 +813,33 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                 }
             }
             __syncthreads();
+            // this block's shares go into the grid-wide 128-bit sums (low word first; its carry goes with the high word)
             for (int r = threadIdx.x; r < msel; r += kPlanThreads) {
-                ull *dst = L.partials + (((size_t)pp * kRoundM + r) * kLazyMaxBlocks + c) * 2;
-                dst[0] = s_acc[2 * r]; dst[1] = s_acc[2 * r + 1];
+                const ull lo = s_acc[2 * r], hi = s_acc[2 * r + 1];
+                if (lo | hi) {
+                    ull *dst = L.partials + ((size_t)pp * kRoundM + r) * 2;
+                    const ull old = atomicAdd(&dst[0], lo);
+                    const ull up = hi + (old + lo < old ? 1ull : 0ull);
+                    if (up) atomicAdd(&dst[1], up);
+                }
             }
             LAZY_CLOCK(5);
             if (!grid_barrier(A.bar, G, gen)) { failed = true; break; }
             barrier_since_booking = true;
             LAZY_CLOCK(6);
-            // every block adds up the slices (one warp per period at a time); the owner stores the new score
-#pragma unroll 2
-            for (int r = warp; r < msel; r += kPlanWarps) {
+            // the buffer used two rounds from now was last read one round ago: block 0 clears it
+            if (c == 0)
+                for (int j = threadIdx.x; j < kRoundM * 2; j += kPlanThreads) L.partials[(size_t)((pp + 2) % 3) * kRoundM * 2 + j] = 0;
+            // every block reads the sums; the owner of a period stores its new score
+            for (int r = threadIdx.x; r < msel; r += kPlanThreads) {
                 const int p = s_pidx[s_sel[r]];
                 const int d = s_it_d[r];
-                u128 tot = 0;
-                {
-                    const ulonglong2 *src = (const ulonglong2 *)(L.partials + ((size_t)pp * kRoundM + r) * kLazyMaxBlocks * 2);
-                    ulonglong2 vals[kLazyMaxBlocks / 32];
-#pragma unroll
-                    for (int q = 0; q < kLazyMaxBlocks / 32; ++q) {          // all loads first
-                        const int j = lane + 32 * q;
-                        vals[q] = j < G ? __ldcg(&src[j]) : make_ulonglong2(0ull, 0ull);
-                    }
-#pragma unroll
-                    for (int q = 0; q < kLazyMaxBlocks / 32; ++q) tot += ((u128)vals[q].y << 64) | vals[q].x;
-                }
-                tot = warp_sum_u128(tot);
-                if (lane == 0) {
-                    Cand x;
-                    x.ben = tot; x.cost = s_it_cost[r]; x.idx = tot == 0 ? -1 : p; x.dest = d;
-                    s_new[r] = x;
-                    if ((int)((p / kPlanThreads) % G) == c) store_score(L, p, d, kFresh, tot, x.cost);
-                }
+                const ull *src = L.partials + ((size_t)pp * kRoundM + r) * 2;
+                const u128 tot = ((u128)__ldcg(&src[1]) << 64) | __ldcg(&src[0]);
+                Cand x;
+                x.ben = tot; x.cost = s_it_cost[r]; x.idx = tot == 0 ? -1 : p; x.dest = d;
+                s_new[r] = x;
+                if ((int)((p / kPlanThreads) % G) == c) store_score(L, p, d, kFresh, tot, x.cost);
             }
             __syncthreads();
             {
@@ -853,7 +849,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                 const Cand b = block_best_fast(x, &s_best, s_cand);
                 if (cand_beats(b, gBest)) gBest = b;
             }
-            pp ^= 1;
+            pp = (pp + 1) % 3;
             __syncthreads();
             LAZY_CLOCK(7);
         }
