@@ -365,15 +365,26 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
 #pragma unroll
     for (int j = 0; j < kTopT; ++j) { tk[j] = -1.0; ti[j] = -1; }
     const int64_t *bo = A.busy + (size_t)(2 * (w.dest < 0 ? 0 : w.dest)) * A.K, *bi = bo + A.K;
+    // The pass is a chain of L2 latencies: the loads of the next period of this thread are issued before the
+    // current one is worked on.
+    unsigned char st_nx = 0;
+    double key_nx = 0.0;
+    int u_nx = 0, v_nx = 0;
+    {
+        const int64_t p = (int64_t)c * kPlanThreads + threadIdx.x;
+        if (p < Pn) { st_nx = L.c_state[p]; key_nx = L.c_key[p]; if (classify) { u_nx = A.per_u[p]; v_nx = A.per_v[p]; } }
+    }
     for (int64_t p0 = (int64_t)c * kPlanThreads; p0 < Pn; p0 += (int64_t)G * kPlanThreads) {
         const int64_t p = p0 + threadIdx.x;
         bool dirty = false;
+        unsigned char st = st_nx;
+        const double key_ld = key_nx;
+        const int u = u_nx, v = v_nx;
+        {
+            const int64_t pn = p + (int64_t)G * kPlanThreads;
+            if (pn < Pn) { st_nx = L.c_state[pn]; key_nx = L.c_key[pn]; if (classify) { u_nx = A.per_u[pn]; v_nx = A.per_v[pn]; } }
+        }
         if (p < Pn) {
-            unsigned char st = L.c_state[p];
-            // (independent loads issued together: the pass is a chain of L2 latencies otherwise)
-            const double key_ld = L.c_key[p];
-            int u = 0, v = 0;
-            if (classify) { u = A.per_u[p]; v = A.per_v[p]; }
             if (st != 0) {
                 int state = st >> 2;
                 const int d = (st & 3) - 1;
