@@ -201,49 +201,6 @@ static int seg_scan_blocks(int64_t n)
     return g < 1 ? 1 : (int)g;
 }
 
-// =============================================================================================
-// Slot clock: start = exclusive prefix sum of kernel_ns, start[K] = total.  Also checks that
-// kernel_ptr runs from 0 to E without decreasing and that every duration is >= 1.
-// =============================================================================================
-__global__ void __launch_bounds__(kScanThreads) k_slot_clock(int64_t K, int64_t E, const int64_t *__restrict__ dur,
-                                                             const int64_t *__restrict__ kptr, int64_t *__restrict__ start,
-                                                             TileState<1> st, int tiles, ull *status)
-{
-    const int tile = next_tile(st.ticket);
-    if (tile >= tiles) return;
-    const int64_t base = (int64_t)tile * kScanTile + (int64_t)threadIdx.x * kScanItems;
-    long long v[kScanItems];
-    Sums<1> mine;
-    mine.v[0] = 0;
-    ull bad = 0;
-#pragma unroll
-    for (int j = 0; j < kScanItems; ++j) {
-        const int64_t k = base + j;
-        v[j] = 0;
-        if (k < K) {
-            v[j] = dur[k];
-            if (v[j] < 1 || v[j] >= ((long long)1 << 44)) { bad |= G10_DEV_BAD_DURATION; v[j] = 1; }
-            const int64_t p0 = kptr[k], p1 = kptr[k + 1];
-            if (p0 > p1 || p0 < 0 || p1 > E || (k == 0 && p0 != 0) || (k == K - 1 && p1 != E)) bad |= G10_DEV_BAD_KERNEL_PTR;
-        }
-        mine.v[0] += v[j];
-    }
-    if (bad) raise_status(status, bad);
-    Sums<1> total;
-    Sums<1> ex = block_exclusive_with_lookback<1>(st, tile, mine, status, &total);
-    long long run = ex.v[0];
-#pragma unroll
-    for (int j = 0; j < kScanItems; ++j) {
-        const int64_t k = base + j;
-        if (k < K) start[k] = run;
-        run += v[j];
-    }
-    if (tile == tiles - 1 && threadIdx.x == 0) {
-        start[K] = total.v[0];
-        if (total.v[0] >= ((long long)1 << 44)) raise_status(status, G10_DEV_BAD_DURATION);
-    }
-}
-
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s)
 {
     const int G = seg_scan_blocks(t.K);
@@ -730,87 +687,6 @@ __global__ void __launch_bounds__(256) k_diff_scatter(int64_t N, int64_t K, cons
         if (tot != 0) atomicAdd(&diff[0], (ull)tot);
     }
 }
-
-__global__ void __launch_bounds__(kScanThreads) k_scan_pressure(int64_t K, const int64_t *__restrict__ diff, int64_t *__restrict__ P,
-                                                                TileState<1> st, unsigned *done, int64_t *__restrict__ tile_max,
-                                                                int32_t *__restrict__ tile_slot, int tiles, int64_t *peak_bytes,
-                                                                int32_t *peak_slot, ull *status)
-{
-    __shared__ long long s_mx[kScanThreads / 32];
-    __shared__ int s_sl[kScanThreads / 32];
-    __shared__ bool s_last;
-    const int tile = next_tile(st.ticket);
-    if (tile >= tiles) return;
-    const int64_t base = (int64_t)tile * kScanTile + (int64_t)threadIdx.x * kScanItems;
-    long long v[kScanItems];
-    Sums<1> mine;
-    mine.v[0] = 0;
-#pragma unroll
-    for (int j = 0; j < kScanItems; ++j) {
-        const int64_t k = base + j;
-        v[j] = k < K ? diff[k] : 0;
-        mine.v[0] += v[j];
-    }
-    Sums<1> total;
-    Sums<1> ex = block_exclusive_with_lookback<1>(st, tile, mine, status, &total);
-    long long run = ex.v[0];
-    long long mx = 0;
-    int sl = -1;
-#pragma unroll
-    for (int j = 0; j < kScanItems; ++j) {
-        const int64_t k = base + j;
-        run += v[j];
-        if (k < K) {
-            P[k] = run;
-            if (sl < 0 || run > mx) { mx = run; sl = (int)k; }
-        }
-    }
-    // block max, ties to the lowest slot
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const long long omx = __shfl_down_sync(0xffffffffu, mx, o);
-        const int osl = __shfl_down_sync(0xffffffffu, sl, o);
-        if (osl >= 0 && (sl < 0 || omx > mx || (omx == mx && osl < sl))) { mx = omx; sl = osl; }
-    }
-    if (lane == 0) { s_mx[warp] = mx; s_sl[warp] = sl; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < kScanThreads / 32; ++w)
-            if (s_sl[w] >= 0 && (sl < 0 || s_mx[w] > mx || (s_mx[w] == mx && s_sl[w] < sl))) { mx = s_mx[w]; sl = s_sl[w]; }
-        tile_max[tile] = mx;
-        tile_slot[tile] = sl;
-        __threadfence();
-        s_last = (atomicAdd(done, 1u) == (unsigned)tiles - 1u);
-    }
-    __syncthreads();
-    if (s_last) {
-        __threadfence();
-        long long bm = 0;
-        int bs = -1;
-        for (int t = threadIdx.x; t < tiles; t += blockDim.x) {
-            const long long m = __ldcg(&tile_max[t]);
-            const int s2 = __ldcg(&tile_slot[t]);
-            if (s2 >= 0 && (bs < 0 || m > bm || (m == bm && s2 < bs))) { bm = m; bs = s2; }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const long long omx = __shfl_down_sync(0xffffffffu, bm, o);
-            const int osl = __shfl_down_sync(0xffffffffu, bs, o);
-            if (osl >= 0 && (bs < 0 || omx > bm || (omx == bm && osl < bs))) { bm = omx; bs = osl; }
-        }
-        __syncthreads();
-        if (lane == 0) { s_mx[warp] = bm; s_sl[warp] = bs; }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            for (int w = 1; w < kScanThreads / 32; ++w)
-                if (s_sl[w] >= 0 && (bs < 0 || s_mx[w] > bm || (s_mx[w] == bm && s_sl[w] < bs))) { bm = s_mx[w]; bs = s_sl[w]; }
-            *peak_bytes = bs < 0 ? 0 : bm;
-            *peak_slot = bs;
-        }
-    }
-}
-
 cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
 {

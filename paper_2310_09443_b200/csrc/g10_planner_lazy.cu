@@ -139,55 +139,6 @@ __device__ __forceinline__ void dest_warp(const PlanArgs &A, const LazyArgs &L, 
     }
 }
 
-// The whole block brings period p up to date (long absent ranges).
-__device__ __forceinline__ void eval_block(const PlanArgs &A, const LazyArgs &L, int64_t p, int *s_dest, ull *s_part /* [2*kPlanWarps] */)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const unsigned char st = L.c_state[p];
-    if (st == 0) return;                       // uniform across the block
-    int d = (st & 3) - 1;
-    if ((st >> 2) == kDirty) {
-        __syncthreads();
-        if (warp == 0) {
-            // destination rule: SSD first, then host; the windows are short, one warp checks them
-            const int u = A.per_u[p], v = A.per_v[p];
-            const int a = u + 1, b = v - 1;
-            const int64_t s = A.bytes[A.per_t[p]];
-            const int64_t t_r = A.start[a], t_end = A.start[v];
-            int dest = -1;
-            for (int X = 0; X < 2 && dest < 0; ++X) {
-                const int ap = A.geo_a[X * A.geo_stride + p];
-                if (ap < 0) continue;
-                const int bp = A.geo_b[X * A.geo_stride + p];
-                const int64_t t = A.geo_t[X * A.geo_stride + p];
-                if (!window_free(A, A.busy + (size_t)(2 * X) * A.K, t_r, t_r + t, a, ap - 1, lane)) continue;
-                if (!window_free(A, A.busy + (size_t)(2 * X + 1) * A.K, t_end - t, t_end, bp + 1, b, lane)) continue;
-                if (X == G10_DEST_HOST && A.host_capacity != 0) {
-                    bool ok = true;
-                    for (int k = a + lane; k <= b; k += 32)
-                        if ((uint64_t)A.hocc[k] + (uint64_t)s > A.host_capacity) ok = false;
-                    if (!__all_sync(0xffffffffu, ok)) continue;
-                }
-                dest = X;
-            }
-            if (lane == 0) *s_dest = dest;
-        }
-        __syncthreads();
-        d = *s_dest;
-        if (d < 0) { if (threadIdx.x == 0) L.c_state[p] = 0; return; }
-    }
-    const int ap = A.geo_a[d * A.geo_stride + p], bp = A.geo_b[d * A.geo_stride + p];
-    const int64_t s = A.bytes[A.per_t[p]];
-    u128 acc = warp_sum_u128(benefit_partial(A, ap, bp, s, threadIdx.x, kPlanThreads));
-    __syncthreads();
-    if (lane == 0) { s_part[2 * warp] = (ull)acc; s_part[2 * warp + 1] = (ull)(acc >> 64); }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        u128 tot = 0;
-        for (int w = 0; w < kPlanWarps; ++w) tot += ((u128)s_part[2 * w + 1] << 64) | s_part[2 * w];
-        store_score(L, p, d, kFresh, tot, 2ull * (ull)A.geo_t[d * A.geo_stride + p]);
-    }
-}
 
 // Smallest and largest pressure of slot tile tl, recomputed by the whole block (the tile's owner).
 __device__ __forceinline__ void tile_minmax(const PlanArgs &A, const LazyArgs &L, int tl, long long *s_red /* [2 * kPlanWarps] */)
@@ -499,8 +450,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     __shared__ long long s_max[2 * kPlanWarps + 1];
     __shared__ double s_k[kPlanWarps];
     __shared__ int s_i[kPlanWarps];
-    __shared__ int s_dest;
-    __shared__ ull s_part[2 * kPlanWarps];
     __shared__ double s_tk[kTopT];
     __shared__ int s_ti[kTopT];
     __shared__ double s_pkey[kLazyMaxBlocks * kTopT];      // published bounds of all blocks

@@ -131,7 +131,6 @@ template <bool kBatch, bool kCyclic>
 __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs O, BatchArgs B)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ ull s_part[2 * kOneWarps];
     __shared__ int s_fin[kOneMaxFin];
 #ifdef G10_PHASE_CLOCKS
     __shared__ int s_dbg[4];

@@ -123,8 +123,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
     __shared__ XPayload s_pay;
     __shared__ __align__(16) unsigned char s_recs[kSmallMaxBlocks * sizeof(XPayload)];
     __shared__ int s_n_over;
-    __shared__ int s_todo;
-    __shared__ ull s_part[2 * kPlanWarps];
     __shared__ unsigned s_err;
     if (*S.done) return;                  // same answer in every thread of the grid: written by an earlier launch
     const int G = gridDim.x, c = blockIdx.x;
