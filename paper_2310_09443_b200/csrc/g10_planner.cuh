@@ -48,6 +48,7 @@ __device__ __forceinline__ bool cand_beats(const Cand &a, const Cand &b)
 {
     if (a.idx < 0) return false;
     if (b.idx < 0) return true;
+    if (a.ben == b.ben && a.cost == b.cost) return a.idx < b.idx;      // (repeated layers: identical scores are common)
     const u128 l = a.ben * (u128)b.cost, r = b.ben * (u128)a.cost;
     if (l != r) return l > r;
     return a.idx < b.idx;
