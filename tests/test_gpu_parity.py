@@ -531,3 +531,26 @@ def test_cyclic_planning(gpu, oracle):
     torch.cuda.synchronize()
     s = _np(plan.summary)
     assert s[2] == -1 and (s[7] & 0x100)
+
+
+@pytest.mark.gpu
+def test_crowded_ties_and_conflicts(gpu, oracle):
+    """Thousands of identical periods: every commit makes all the others stale with equal bounds and blocks their
+    transfer windows, so the planners' rarely used paths run (rounds beyond their size limits, lists used up and
+    published again, very many destinations re-chosen at once).  All planners against the oracle."""
+    K = 60
+    for n, size, dur in ((1500, 1 << 20, 1000000), (700, 3 << 20, 2000000)):
+        lists = [[] for _ in range(K)]
+        for i in range(n):
+            lists[i % 20].append(i)                      # twenty groups of identical periods, all overlapping in the middle
+            lists[K - 1 - (i % 7)].append(i)
+        sizes = [size + (i % 4) for i in range(n)]       # a few distinct sizes: near-ties next to exact ties
+        tr = traces.from_lists("crowd", lists, sizes, [dur] * K, capacity_frac=(1, 3))
+        tb = gpu.upload(tr)
+        start, P0, peak, slot = oracle.timeline(tr)
+        cap = tr.capacity_from_peak(peak)
+        ref = oracle.plan(tr, cap, lazy=True)
+        assert np.array_equal(ref.migrations, oracle.plan(tr, cap).migrations) and len(ref.migrations) > 100
+        for flags in (0, gpu.FLAG_GLOBAL_STATE, gpu.FLAG_MULTI_BLOCK, gpu.FLAG_RESCORE_ALL):
+            check_plan(gpu, tr, tb, cap, ref, flags=flags)
+        check_cyclic(gpu, oracle, tr, cap)
