@@ -119,12 +119,14 @@ __device__ __forceinline__ void warp_argmax_u64(ull k, int idx, ull *mk, int *mi
 // Developer aid (off in the library build): with -DG10_PHASE_CLOCKS thread 0 accumulates the cycles between the
 // marked points of an iteration and prints the averages when the loop ends.
 #ifdef G10_PHASE_CLOCKS
+#define W0_CLOCK(i) do { if (threadIdx.x == 0) { const long long now_ = clock64(); w0_acc[i] += now_ - w0_last; w0_last = now_; } } while (0)
 #define ONE_COUNT(i) do { if ((threadIdx.x & 31) == 0) atomicAdd(&s_dbg[i], 1); } while (0)
 #define ONE_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
                            ph_acc[i] += now_ - ph_last; ph_last = now_; ph_cnt[i] += 1; asm volatile("" ::: "memory"); } } while (0)
 #else
 #define ONE_CLOCK(i)
 #define ONE_COUNT(i)
+#define W0_CLOCK(i)
 #endif
 
 template <bool kBatch, bool kCyclic>
@@ -257,6 +259,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
     int status = -1;
 #ifdef G10_PHASE_CLOCKS
     long long ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_cnt[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
+    long long w0_acc[4] = {0, 0, 0, 0}, w0_last = clock64();
 #endif
 #pragma unroll 1
     for (int64_t it = 0;; ++it) {
@@ -361,6 +364,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             if (warp == 0) {
 #pragma unroll 1
                 for (;;) {
+                    W0_CLOCK(0);
                     if (s_flagged) {
                         __syncwarp();
                         if (lane == 0) s_flagged = 0;
@@ -378,6 +382,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                         }
                     }
                     __syncwarp();
+                    W0_CLOCK(1);
                     ull bk = 0; int bi = 0x7fffffff;
 #pragma unroll 4
                     for (int g = lane; g < G1; g += 32) {
@@ -386,12 +391,14 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                     }
                     ull mk; int mi;
                     warp_argmax_u64(bk, bi, &mk, &mi);
+                    W0_CLOCK(2);
                     if (mk == 0 || (cstate[mi] & kStateMaskO) != kStaleO) {
                         if (lane == 0) { s_topkey = mk; s_top = mi; }
                         break;
                     }
                     ONE_COUNT(3);
                     rescore_warp0(mi);
+                    W0_CLOCK(3);
                 }
             }
             __syncthreads();
@@ -568,7 +575,8 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
         printf("one-block cycles/iteration: top %lld dirty %lld (x%lld) topscan %lld (x%lld) tiescan %lld (x%lld) rescore %lld (x%lld) winner %lld apply %lld (n=%lld)\n",
                ph_acc[0] / r, ph_acc[1] / r, ph_cnt[1], ph_acc[2] / r, ph_cnt[2], ph_acc[3] / r, ph_cnt[3], ph_acc[4] / r, ph_cnt[4], ph_acc[5] / r,
                ph_acc[6] / r, (long long)rounds);
-        printf("dirty periods examined %d, rescored %d, erased %d\n", s_dbg[0], s_dbg[1], s_dbg[2]);
+        printf("dirty periods examined %d, rescored %d, erased %d; search-loop rescorings %d\n", s_dbg[0], s_dbg[1], s_dbg[2], s_dbg[3]);
+        printf("warp 0 search loop cycles/iteration: other %lld flag refresh %lld top scan %lld rescore %lld\n", w0_acc[0] / r, w0_acc[1] / r, w0_acc[2] / r, w0_acc[3] / r);
     }
 #endif
     // ---------------- epilogue: final pressure, peak and its lowest slot, summary
