@@ -471,8 +471,18 @@ def test_batched_replanning(gpu, oracle):
         variants += [dict(base, host_capacity_bytes=hc << 30) for hc in (1, 32, 256)]
         ref = check_batch(gpu, oracle, tr, variants)
         assert ref.stability[0, 0] == ref.stability[0, 1] == len(ref.plans[0].migrations)
-    # a trace too large for one SM: every variant says so, nothing else is written
+    # a variant with an invalid duration reports it in its own status word, the others stay clean
     import torch
+    tr = traces.config0_mlp_chain()
+    tb = gpu.upload(tr)
+    start, P0, peak, slot = oracle.timeline(tr)
+    base = dict(gpu_capacity_bytes=tr.capacity_from_peak(peak), host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)
+    bad = tr.kernel_ns.copy(); bad[5] = 0
+    got = gpu.g10_plan_batch(tb, [base, dict(base, kernel_ns=torch.from_numpy(bad).cuda()), base])
+    torch.cuda.synchronize()
+    s7 = _np(got.summary)[:, 7]
+    assert s7[0] == 0 and (s7[1] & 0x8) and s7[2] == 0
+    # a trace too large for one SM: every variant says so, nothing else is written
     tr = traces.make_config(3)
     tb = gpu.upload(tr)
     got = gpu.g10_plan_batch(tb, [dict(gpu_capacity_bytes=1 << 30, host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)] * 2)
