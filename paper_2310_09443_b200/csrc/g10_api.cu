@@ -60,9 +60,10 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.bk_words = c.take<ull>(2 * 4096);
     w.xwords = c.take<ull>((2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16);
     w.zero_bytes = align_up(c.off);
-    // arrays that must start at zero, cleared only by the calls that use them
-    w.cnt = c.take<int32_t>(N);
+    // arrays that must start at zero, cleared only by the calls that use them (the difference array sits right behind
+    // the zero-initialised region, so that one memset covers both)
     w.diff = c.take<int64_t>(K + 1);
+    w.cnt = c.take<int32_t>(N);
     const size_t state_begin = align_up(c.off);
     w.busy = c.take<int64_t>(4 * K);       // busy, hocc and dead are contiguous: one memset
     w.hocc = c.take<int64_t>(K);
@@ -160,9 +161,12 @@ int32_t begin_call(const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, c
 {
     Sizes z{t->num_kernels, t->num_tensors, t->num_events, t->mem == G10_MEM_HOST};
     carve(ws, z, w);
-    CU(cudaMemsetAsync(w.zero_begin, 0, w.zero_bytes, s));
+    {
+        size_t head = w.zero_bytes;
+        if (zero_mask & kZeroDiff) head = (size_t)((char *)(w.diff + z.K + 1) - w.zero_begin);
+        CU(cudaMemsetAsync(w.zero_begin, 0, head, s));
+    }
     if ((zero_mask & kZeroCounts) && z.N > 0) CU(cudaMemsetAsync(w.cnt, 0, sizeof(int32_t) * (size_t)z.N, s));
-    if (zero_mask & kZeroDiff) CU(cudaMemsetAsync(w.diff, 0, sizeof(int64_t) * (size_t)(z.K + 1), s));
     if (zero_mask & kZeroState) CU(cudaMemsetAsync(w.busy, 0, w.state_bytes, s));
     d.K = z.K; d.N = z.N; d.E = z.E;
     if (!z.host) {

@@ -380,8 +380,13 @@ cudaError_t launch_clock_and_first_last(const DeviceTrace &t, const Workspace &w
 {
     cudaError_t e;
     if (t.N > 0) {
-        if ((e = cudaMemsetAsync(first_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
-        if ((e = cudaMemsetAsync(last_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
+        const ptrdiff_t gap = (const char *)last_use - (const char *)(first_use + t.N);
+        if (gap >= 0 && gap < 4096) {                 // the two arrays follow each other in the workspace: one memset
+            if ((e = cudaMemsetAsync(first_use, 0, (size_t)((const char *)(last_use + t.N) - (const char *)first_use), s)) != cudaSuccess) return e;
+        } else {
+            if ((e = cudaMemsetAsync(first_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
+            if ((e = cudaMemsetAsync(last_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
+        }
     }
     if ((e = launch_slot_clock(t, w, start, s)) != cudaSuccess) return e;
     if (t.N > 0 && t.E > 0 && t.K > 0) {
