@@ -244,14 +244,8 @@ cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s)
     if (!emit_choose_buckets(L.K, 2 * L.N + 2 * L.n, &A.shift, &A.nb)) return cudaErrorInvalidValue;
     A.bucket_count = L.bucket_count; A.bucket_cursor = L.bucket_cursor; A.keys = L.keys; A.payload = L.payload;
     A.ticket = L.ticket; A.status = L.status;
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
-            sms = 0;
-            return cudaErrorInvalidDevice;
-        }
-    }
+    const int sms = current_sm_count();
+    if (sms <= 0) return cudaErrorInvalidDevice;
     const int64_t total = 2 * L.N + 2 * L.n;
     int64_t g = (total + kEmitThreads - 1) / kEmitThreads;
     if (g > 4 * (int64_t)sms) g = 4 * (int64_t)sms;

@@ -14,6 +14,14 @@ typedef unsigned long long ull;
 constexpr size_t kAlign = 256;
 constexpr int kHeavyThreshold = 32;      // tensors with more raw uses than this are sorted by a whole block
 
+// Multiprocessors of the current device (0 if the query fails).  Asked every time: a process may use several devices.
+inline int current_sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return sms > 0 ? sms : 0;
+}
+
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t tiles_of(int64_t n, int64_t tile) { return n <= 0 ? 1 : (n + tile - 1) / tile; }
 

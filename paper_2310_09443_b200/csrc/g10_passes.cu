@@ -188,12 +188,8 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
 
 static int seg_scan_blocks(int64_t n)
 {
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;
-        if (sms <= 0) return 1;
-    }
+    const int sms = current_sm_count();
+    if (sms <= 0) return 1;
     int64_t g = 2 * (int64_t)sms;
     const int64_t by_work = (n + kSegChunk - 1) / kSegChunk;        // no point in blocks without a full chunk
     if (g > by_work) g = by_work;

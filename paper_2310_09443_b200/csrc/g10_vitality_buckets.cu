@@ -496,14 +496,8 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     if (!choose_buckets(t.N, t.E, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
     B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
     B.ticket = w.emit_scan.ticket; B.status = w.status; B.spill = w.raw_uses;
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
-            sms = 0;
-            return cudaErrorInvalidDevice;
-        }
-    }
+    const int sms = current_sm_count();
+    if (sms <= 0) return cudaErrorInvalidDevice;
     const int64_t tiles = (t.E + kBkTile - 1) / kBkTile;
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
