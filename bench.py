@@ -121,8 +121,8 @@ def run_reference(args):
         "impl": "reference", "metric": "trace_events_per_s", "value": value, "unit": "events/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "K": tr.K, "N": tr.N, "E": tr.E, "migrations": int(r.summary[0]),
-                   "status": r.status},
+        "config": {"workload": WORKLOAD, "trace_sha256": tr.sha256(), "K": tr.K, "N": tr.N, "E": tr.E,
+                   "migrations": int(r.summary[0]), "status": r.status},
         "cpu_baseline": {"value": value, "unit": "events/s", "cores": 1, "kind": "oracle",
                          "sample": "whole config-1 plan (plain tier), %d repetitions" % args.steps},
         "e2e": {"value": value, "unit": "events/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -327,7 +327,8 @@ def run_ours(args):
         "metric": "trace_events_per_s", "value": value, "unit": "events/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_s / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "K": tr.K, "N": tr.N, "E": tr.E, "periods": int(plan_periods(binding, tb, ws)),
+        "config": {"workload": WORKLOAD, "trace_sha256": tr.sha256(), "K": tr.K, "N": tr.N, "E": tr.E,
+                   "periods": int(plan_periods(binding, tb, ws)),
                    "gpu_capacity_bytes": cap, "host_bw": tr.host_bw, "ssd_bw": tr.ssd_bw,
                    "migrations": int(summary[0]), "scoring_rounds": int(summary[1]), "status": binding.STATUS[int(summary[2])],
                    "l2": "flushed between timed iterations (%d MiB write)" % (L2_FLUSH_BYTES >> 20),

@@ -68,6 +68,31 @@ class Trace:
             h.update(np.ascontiguousarray(a).tobytes())
         return h.hexdigest()
 
+    def save(self, path: str) -> str:
+        """Write the trace to an .npz file (arrays plus scalars) and return its digest."""
+        cap = -1 if self.capacity_bytes is None else int(self.capacity_bytes)
+        frac = (0, 0) if self.capacity_frac is None else tuple(int(x) for x in self.capacity_frac)
+        np.savez(path, name=np.array(self.name), kernel_ptr=self.kernel_ptr, kernel_tensors=self.kernel_tensors,
+                 tensor_bytes=self.tensor_bytes, kernel_ns=self.kernel_ns, tensor_global=self.tensor_global,
+                 scalars=np.array([cap, frac[0], frac[1], self.host_bw, self.ssd_bw, self.host_capacity_bytes],
+                                  dtype=np.int64))
+        return self.sha256()
+
+    @staticmethod
+    def load(path: str) -> "Trace":
+        """Read back a trace written by :meth:`save`."""
+        with np.load(path, allow_pickle=False) as z:
+            cap, fnum, fden, host_bw, ssd_bw, host_cap = (int(x) for x in z["scalars"])
+            tr = Trace(name=str(z["name"]), kernel_ptr=z["kernel_ptr"].astype(np.int64),
+                       kernel_tensors=z["kernel_tensors"].astype(np.int32),
+                       tensor_bytes=z["tensor_bytes"].astype(np.int64), kernel_ns=z["kernel_ns"].astype(np.int64),
+                       tensor_global=z["tensor_global"].astype(np.uint8),
+                       capacity_bytes=None if cap < 0 else cap,
+                       capacity_frac=None if fden == 0 else (fnum, fden),
+                       host_bw=host_bw, ssd_bw=ssd_bw, host_capacity_bytes=host_cap)
+        tr.validate()
+        return tr
+
     def validate(self) -> None:
         assert self.kernel_ptr.dtype == np.int64 and self.kernel_ptr.shape == (self.K + 1,)
         assert self.kernel_tensors.dtype == np.int32
