@@ -129,6 +129,25 @@ def test_configs_bit_exact(gpu, oracle, cfg):
     assert len(ref.migrations) > 10
 
 
+def test_bandwidth_and_capacity_sweep(gpu, oracle):
+    """The planner-side half of the paper's sensitivity studies (SSD bandwidth, host memory): configs 1 and 2 with
+    SSD bandwidths from one SSD to sixteen times the default, a sixteen times faster host link, two GPU capacities
+    and a finite host memory.  Faster links make more periods usable and the greedy loop longer."""
+    import dataclasses
+    GiB = 1 << 30
+    n = 0
+    for cfg, caps in ((1, (12, 16)), (2, (20,))):
+        base = traces.make_config(cfg)
+        for ssd in (3_200_000_000, 12_800_000_000, 102_400_000_000):
+            for host in (32_000_000_000, 512_000_000_000):
+                for capg in caps:
+                    for hc in (0, 8 * GiB):
+                        tr = dataclasses.replace(base, ssd_bw=ssd, host_bw=host, capacity_bytes=capg * GiB)
+                        ref = full_parity(gpu, oracle, tr, lazy_oracle=True, host_capacity=hc, also_rescore_all=(n % 9 == 0))
+                        assert len(ref.migrations) > 300
+                        n += 1
+
+
 def test_inplace_relu_variant(gpu, oracle):
     tr = traces.config1_resnet152(inplace_relu=True)
     full_parity(gpu, oracle, tr)
