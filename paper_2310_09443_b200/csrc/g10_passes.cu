@@ -132,14 +132,13 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
         }
         carry += ctot;
     }
-    if (kind == 0) {
+    if constexpr (kind == 0) {
         // after its own segment the last block's carry is the sum of everything
         if (g == G - 1 && threadIdx.x == 0) {
             out[n] = carry;
             if (carry >= ((long long)1 << 44)) raise_status(status, G10_DEV_BAD_DURATION);
         }
-        return;
-    }
+    } else {
     // ---- kind 1: block maximum (ties to the lowest slot), then the last block reduces the per-block results
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -183,6 +182,7 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
             *peak_bytes = bs < 0 ? 0 : bm;
             *peak_slot = bs;
         }
+    }
     }
 }
 
