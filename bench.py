@@ -124,7 +124,7 @@ def run_reference(args):
         "config": {"workload": WORKLOAD, "trace_sha256": tr.sha256(), "K": tr.K, "N": tr.N, "E": tr.E,
                    "migrations": int(r.summary[0]), "status": r.status},
         "cpu_baseline": {"value": value, "unit": "events/s", "cores": 1, "kind": "oracle",
-                         "sample": "whole config-1 plan (plain tier), %d repetitions" % args.steps},
+                         "sample": "whole config-1 plan (plain tier), %d repetitions" % args.steps, "cpu_model": cpu_model()},
         "e2e": {"value": value, "unit": "events/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "plan_ms": dt / args.steps * 1e3,
     }
@@ -433,6 +433,17 @@ def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=20):
     return out
 
 
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for ln in f:
+                if ln.lower().startswith("model name"):
+                    return ln.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def cpu_baseline(tr):
     """The oracle (plain tier, one thread) on the same workload, bounded to roughly ten seconds."""
     from oracle import g10_oracle as O
@@ -462,7 +473,7 @@ def cpu_baseline(tr):
     return {"value": tr.E * reps / dt, "unit": "events/s", "cores": 1, "kind": "oracle", "lazy_tier_plan_ms": lazy_s * 1e3,
             "vitality_timeline_events_per_s": tr.E / passes_s,
             "sample": "whole config-1 plan (plain tier), %d repetitions in %.1f s" % (reps, dt),
-            "plan_ms": dt / reps * 1e3, "host_cores_available": os.cpu_count()}
+            "plan_ms": dt / reps * 1e3, "host_cores_available": os.cpu_count(), "cpu_model": cpu_model()}
 
 
 def main():
