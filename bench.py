@@ -171,11 +171,14 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the planner has no CPU path")
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
-    build.build()
-    binding.load_library()
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl")
+        if local == 0:
+            build.build()                   # one build per node; the others wait for it
+        dist.barrier()
+    build.build()
+    binding.load_library()
 
     def barrier():
         if world > 1:

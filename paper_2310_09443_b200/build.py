@@ -26,9 +26,15 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "nvcc")
+        tmp = "%s.%d.tmp" % (LIB, os.getpid())       # several processes may build at once: each renames a finished file
         cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-              ["-I" + os.path.join(ROOT, "include"), "-o", LIB] + [os.path.join(CSRC, f) for f in SOURCES]
-        subprocess.check_call(cmd)
+              ["-I" + os.path.join(ROOT, "include"), "-o", tmp] + [os.path.join(CSRC, f) for f in SOURCES]
+        try:
+            subprocess.check_call(cmd)
+            os.replace(tmp, LIB)
+        finally:
+            if os.path.exists(tmp):
+                os.remove(tmp)
     return LIB
 
 
