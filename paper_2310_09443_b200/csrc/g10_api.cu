@@ -55,6 +55,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     carve_scan(c, w.pressure_scan, ktiles, 1);
     w.wl_count = c.take<unsigned>(2);
     w.one_done = c.take<unsigned>(1);
+    w.event_budget = c.take<ull>(1);
     w.bk_count = c.take<unsigned>(4096);
     w.bk_cursor = c.take<unsigned>(4096);
     w.bk_words = c.take<ull>(2 * 4096);

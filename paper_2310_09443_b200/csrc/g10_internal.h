@@ -85,6 +85,7 @@ struct Workspace {
     unsigned char *dead;         // [E] period erased
     unsigned *wl_count;          // [2] lengths of the two DIRTY work lists
     unsigned *one_done;          // [1] the single-block planner produced the plan
+    ull *event_budget;           // [1] events booked by the blocks of the first / last pass (at most E for a valid trace)
     unsigned *bk_count, *bk_cursor;   // [4096] events per tensor bucket, scatter cursors
     ull *bk_words;               // [2 * 4096] tagged per-bucket totals
     ull *xwords;                 // [2][kSmallMaxBlocks][16] tagged words of the proposal exchange

@@ -326,29 +326,60 @@ __global__ void __launch_bounds__(kEvThreads) k_scatter_events(int64_t E, int64_
     }
 }
 
-// first / last use by atomic min / max (the timeline call alone does not need the sorted use lists);
-// the results stay encoded (see below) and are decoded by the difference-array pass
-__global__ void __launch_bounds__(kEvThreads) k_first_last_events(int64_t E, int64_t N, int64_t K, const int64_t *__restrict__ kptr,
+// first / last use by atomic maxima (the timeline call alone does not need the sorted use lists); the results stay
+// encoded (see below) and are decoded by the difference-array pass.
+// One thread per kernel, a warp per 32 consecutive kernels: the warp walks the events of its kernels 32 at a time
+// and finds the kernel of an event by a search over the lanes' kernel_ptr values (five shuffles), so nothing is
+// searched in memory.  The kernel may run beside the pass that validates kernel_ptr, so it bounds its own work:
+// a block books the events between its first and last kernel_ptr entry against a call-wide budget of E events
+// (a valid kernel_ptr hands every event to exactly one block) and its warps stay inside that range.
+constexpr int kFlThreads = 256;
+__global__ void __launch_bounds__(kFlThreads) k_first_last_events(int64_t E, int64_t N, int64_t K, const int64_t *__restrict__ kptr,
                                                                   const int32_t *__restrict__ kt, int32_t *__restrict__ first_enc,
-                                                                  int32_t *__restrict__ last_enc, ull *status)
+                                                                  int32_t *__restrict__ last_enc, ull *budget, ull *status)
 {
     // both arrays start at zero: first_enc holds max(K - k) (0 = unused), last_enc holds max(k + 1)
-    __shared__ int64_t s_ptr[kPtrStage];
-    __shared__ int s_lohi[2];
-    const int64_t base = (int64_t)blockIdx.x * kEvTile;
-    int lo, hi, shift;
-    const int64_t *sp = stage_kernel_ptr(kptr, K, base, E, s_ptr, s_lohi, &lo, &hi, &shift);
+    __shared__ int64_t s_span[2];
+    const int lane = threadIdx.x & 31;
+    const int64_t kb0 = (int64_t)blockIdx.x * kFlThreads;
+    if (threadIdx.x == 0) {
+        const int64_t kb1 = kb0 + kFlThreads < K ? kb0 + kFlThreads : K;
+        int64_t b0 = kptr[kb0], b1 = kptr[kb1];
+        b0 = b0 < 0 ? 0 : (b0 > E ? E : b0);
+        b1 = b1 < 0 ? 0 : (b1 > E ? E : b1);
+        if (b1 < b0) b1 = b0;
+        if (b1 > b0 && atomicAdd(budget, (ull)(b1 - b0)) + (ull)(b1 - b0) > (ull)E) {
+            raise_status(status, G10_DEV_BAD_KERNEL_PTR);
+            b1 = b0;
+        }
+        s_span[0] = b0; s_span[1] = b1;
+    }
+    __syncthreads();
+    const int64_t b0 = s_span[0], b1 = s_span[1];
+    const int64_t k = kb0 + threadIdx.x, k0 = k - lane;
+    if (k0 >= K || b1 == b0) return;
+    int64_t mine = kptr[k < K ? k : K];                          // lanes past the last kernel hold kernel_ptr[K]
+    int64_t span1 = kptr[k0 + 32 < K ? k0 + 32 : K];
+    mine = mine < b0 ? b0 : (mine > b1 ? b1 : mine);
+    span1 = span1 < b0 ? b0 : (span1 > b1 ? b1 : span1);
+    const int64_t span0 = __shfl_sync(0xffffffffu, mine, 0);
     ull bad = 0;
+#pragma unroll 1
+    for (int64_t base = span0; base < span1; base += 32) {
+        const int64_t e = base + lane;
+        int lo = 0;                                              // last lane whose kernel starts at or before e
 #pragma unroll
-    for (int j = 0; j < kEvItems; ++j) {
-        const int64_t e = base + (int64_t)j * kEvThreads + threadIdx.x;
-        if (e < E) {
+        for (int st = 16; st > 0; st >>= 1) {
+            const int64_t p = __shfl_sync(0xffffffffu, mine, (lo + st) & 31);
+            if (p <= e) lo += st;
+        }
+        if (e < span1) {
             const int32_t i = kt[e];
             if (i < 0 || i >= N) bad = G10_DEV_BAD_TENSOR_ID;
             else {
-                const int k = kernel_of_event(sp, lo, hi, e) + shift;
-                atomicMax(&first_enc[i], (int)K - k);
-                atomicMax(&last_enc[i], k + 1);
+                const int kq = (int)(k0 + lo);
+                atomicMax(&first_enc[i], (int)K - kq);
+                atomicMax(&last_enc[i], kq + 1);
             }
         }
     }
@@ -363,8 +394,8 @@ cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t 
     e = cudaMemsetAsync(last_use, 0, sizeof(int32_t) * (size_t)t.N, s);
     if (e != cudaSuccess) return e;
     if (t.E > 0 && t.K > 0) {
-        const int blocks = (int)tiles_of(t.E, kEvTile);
-        k_first_last_events<<<blocks, kEvThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.status);
+        const int blocks = (int)tiles_of(t.K, kFlThreads);
+        k_first_last_events<<<blocks, kFlThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.event_budget, w.status);
     }
     return cudaGetLastError();
 }
@@ -387,8 +418,8 @@ cudaError_t launch_clock_and_first_last(const DeviceTrace &t, const Workspace &w
     if ((e = launch_slot_clock(t, w, start, s)) != cudaSuccess) return e;
     if (t.N > 0 && t.E > 0 && t.K > 0) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)tiles_of(t.E, kEvTile));
-        cfg.blockDim = dim3(kEvThreads);
+        cfg.gridDim = dim3((unsigned)tiles_of(t.K, kFlThreads));
+        cfg.blockDim = dim3(kFlThreads);
         cfg.dynamicSmemBytes = 0;
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
@@ -396,7 +427,7 @@ cudaError_t launch_clock_and_first_last(const DeviceTrace &t, const Workspace &w
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, k_first_last_events, t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.status);
+        e = cudaLaunchKernelEx(&cfg, k_first_last_events, t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.event_budget, w.status);
         if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();

@@ -90,6 +90,7 @@ extern "C" int32_t g10_pressure_timeline_static(const g10_trace *trace, g10_time
     const size_t ktiles = (size_t)tiles_of(K, 2048);
     w.zero_begin = (char *)base;
     w.status = b.take<ull>(1);
+    w.event_budget = b.take<ull>(1);
     take_scan(b, w.clock_scan, ktiles);
     take_scan(b, w.pressure_scan, ktiles);
     w.diff = b.take<int64_t>((size_t)K + 1);

@@ -3,7 +3,8 @@
 // bucket holds a few thousand trace events):
 //   1. k_bk_hist     counts the events of every bucket (shared-memory histogram per block);
 //   2. k_bk_scatter  partitions the events by bucket: each event becomes one 64-bit key
-//                    (tensor id inside the bucket << 32 | kernel) written into its bucket's slice;
+//                    (tensor id inside the bucket << 32 | kernel) written into its bucket's slice; the events are
+//                    walked kernel by kernel, one lane per kernel, so no event has to look its kernel up;
 //   3. k_bk_emit     takes one bucket at a time, entirely in shared memory: counts the events of each tensor,
 //                    scans the counts, scatters the kernels into per-tensor segments, lets one thread sort and
 //                    de-duplicate each (short) segment -- a tensor listed by more than 32 kernels is sorted by the
@@ -25,7 +26,8 @@ constexpr int kBkThreads = 512;
 constexpr int kBkItems = 8;
 constexpr int kBkTile = kBkThreads * kBkItems;     // events per partition tile (4096)
 constexpr int kBkCap = 12288;                      // events of a bucket kept in shared memory
-constexpr int kBkPtrStage = 3072;                  // kernel_ptr entries staged per tile
+constexpr int kBkWide = 64;                        // a kernel with more events is walked by its whole warp in the partition
+constexpr int kBkKeyCap = 6144;                    // keys of one partition tile staged in shared memory
 constexpr int kBkHeavy = 32;                       // longer segments are sorted by the whole block
 
 struct BucketArgs {
@@ -33,6 +35,7 @@ struct BucketArgs {
     int shift;                 // log2(bt)
     int bt;                    // tensors per bucket
     int nb;                    // number of buckets
+    int tile_kernels;          // kernels per partition tile (a multiple of kBkThreads)
     unsigned *bucket_count;    // [nb] events per bucket
     unsigned *bucket_cursor;   // [nb] scatter cursors (start at zero)
     ull *pairs;                // [E] keys, bucket after bucket
@@ -97,25 +100,29 @@ __device__ __forceinline__ void block_scan_counts(const unsigned *cnt, int n, in
     bk_block_scan<1>((const int *)cnt, out, nullptr, nullptr, n, s_w);
 }
 
-// last k in [lo, hi] with kptr[k] <= e
-__device__ __forceinline__ int bk_kernel_of_event(const int64_t *kptr, int lo, int hi, int64_t e)
-{
-    while (lo < hi) {
-        const int mid = lo + (hi - lo + 1) / 2;
-        if (kptr[mid] <= e) lo = mid; else hi = mid - 1;
-    }
-    return lo;
-}
+// Developer aid (off in the library build): with -DG10_PHASE_CLOCKS thread 0 of two blocks adds up the cycles
+// between the marked points and prints the averages at the end.
+#ifdef G10_PHASE_CLOCKS
+#define BK_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
+                         ph_acc[i] += now_ - ph_last; ph_last = now_; asm volatile("" ::: "memory"); } } while (0)
+#else
+#define BK_CLOCK(i)
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // 1. events per bucket
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int32_t *__restrict__ kt)
+__global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
 {
     extern __shared__ unsigned s_hist[];
     for (int b = threadIdx.x; b < B.nb; b += kBkThreads) s_hist[b] = 0;
     __syncthreads();
     ull bad = 0;
+    // the partition walks the events kernel by kernel: kernel_ptr has to be a monotone map onto [0, E]
+    for (int64_t k = (int64_t)blockIdx.x * kBkThreads + threadIdx.x; k < B.K; k += (int64_t)gridDim.x * kBkThreads) {
+        const int64_t p0 = kptr[k], p1 = kptr[k + 1];
+        if (p0 > p1 || p0 < 0 || p1 > B.E || (k == 0 && p0 != 0) || (k == B.K - 1 && p1 != B.E)) bad |= G10_DEV_BAD_KERNEL_PTR;
+    }
     const int64_t tiles = (B.E + kBkTile - 1) / kBkTile;
     for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         const int64_t base = tile * kBkTile;
@@ -128,7 +135,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int3
 #pragma unroll
         for (int j = 0; j < kBkItems; ++j) {
             if (id[j] == -2) continue;
-            if (id[j] < 0 || id[j] >= B.N) bad = G10_DEV_BAD_TENSOR_ID;
+            if (id[j] < 0 || id[j] >= B.N) bad |= G10_DEV_BAD_TENSOR_ID;
             else atomicAdd(&s_hist[id[j] >> B.shift], 1u);
         }
     }
@@ -141,75 +148,120 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int3
 // ---------------------------------------------------------------------------------------------
 // 2. partition the events by bucket
 // ---------------------------------------------------------------------------------------------
+// One sweep of a tile's kernels over the events [eb, ee): a warp takes 32 consecutive kernels, every lane walks the
+// events of its own kernel (so the kernel of an event is known without a search); a kernel with more than
+// kBkWide events is walked by the whole warp instead.
+// kPlace false: count the events of every bucket.  true: s_cnt[b] is the next free slot of bucket b in the tile's
+// staging area; the key and its bucket go there.
+template <bool kPlace>
+__device__ __forceinline__ void bk_take(const BucketArgs &B, int32_t i, int64_t k, int *s_cnt, ull *s_key, unsigned short *s_bkt)
+{
+    if (i < 0 || i >= B.N) return;
+    const int b = i >> B.shift;
+    if (!kPlace) atomicAdd(&s_cnt[b], 1);
+    else {
+        const int slot = atomicAdd(&s_cnt[b], 1);
+        if (slot < kBkKeyCap) {
+            s_key[slot] = ((ull)(unsigned)(i & (B.bt - 1)) << 32) | (unsigned)k;
+            s_bkt[slot] = (unsigned short)b;
+        }
+    }
+}
+
+template <bool kPlace>
+__device__ __forceinline__ void bk_walk(const BucketArgs &B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt, int64_t tk0,
+                                        int64_t tk1, int64_t eb, int64_t ee, int *s_cnt, ull *s_key, unsigned short *s_bkt)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll 1
+    for (int64_t k0 = tk0 + warp * 32; k0 < tk1; k0 += kBkThreads) {
+        const int64_t k = k0 + lane;
+        int64_t a = kptr[k < B.K ? k : B.K];                       // lanes past the last kernel hold kernel_ptr[K] = E: no events
+        int64_t b = kptr[k + 1 < B.K ? k + 1 : B.K];
+        a = a > eb ? a : eb;
+        b = b < ee ? b : ee;
+        const bool wide = b - a > kBkWide;
+        if (!wide) {
+#pragma unroll 1
+            for (int64_t e = a; e < b; e += 4) {                   // four events of this lane's kernel at a time
+                int32_t id[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) id[u] = e + u < b ? kt[e + u] : -1;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) bk_take<kPlace>(B, id[u], k, s_cnt, s_key, s_bkt);
+            }
+        }
+        unsigned m = __ballot_sync(0xffffffffu, wide);
+#pragma unroll 1
+        while (m) {
+            const int src = __ffs(m) - 1;
+            m &= m - 1;
+            const int64_t wa = __shfl_sync(0xffffffffu, a, src), wb = __shfl_sync(0xffffffffu, b, src);
+#pragma unroll 1
+            for (int64_t e = wa + lane; e < wb; e += 32) bk_take<kPlace>(B, kt[e], k0 + src, s_cnt, s_key, s_bkt);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
 {
     extern __shared__ int s_mem[];
     int *s_base = s_mem;                                   // [nb + 1] first key of each bucket
-    int *s_cnt = s_base + B.nb + 1;                        // [nb + 1] events of this tile per bucket, then their scan
-    unsigned *s_off = (unsigned *)(s_cnt + B.nb + 1);      // [nb] where this tile's events start inside the bucket
-    ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkTile] keys of the tile in bucket order
-    unsigned short *s_bkt = (unsigned short *)(s_key + kBkTile);              // [kBkTile] their buckets
+    int *s_cnt = s_base + B.nb + 1;                        // [nb + 1] events of this tile per bucket, then their scan, then fill cursors
+    int *s_off = s_cnt + B.nb + 1;                         // [nb] global position of the tile's first key of the bucket minus its slot
+    ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkKeyCap] keys of the tile in bucket order
+    unsigned short *s_bkt = (unsigned short *)(s_key + kBkKeyCap);           // [kBkKeyCap] their buckets
     __shared__ int s_warp[2 * (kBkThreads / 32 + 1)];
-    __shared__ int64_t s_ptr[kBkPtrStage];
-    __shared__ int s_lohi[2];
+    if (*(volatile ull *)B.status & G10_DEV_BAD_KERNEL_PTR) return;          // (found by k_bk_hist: nothing is partitioned)
+#ifdef G10_PHASE_CLOCKS
+    long long ph_acc[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
+    int ph_n = 0;
+#endif
     block_scan_counts(B.bucket_count, B.nb, s_base, s_warp);
-    const int64_t tiles = (B.E + kBkTile - 1) / kBkTile;
+    BK_CLOCK(0);
+    const int64_t TK = B.tile_kernels;
+    const int64_t tiles = (B.K + TK - 1) / TK;
+#pragma unroll 1
     for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        const int64_t base = tile * kBkTile;
-        const int n_tile = (int)((B.E - base) < kBkTile ? (B.E - base) : kBkTile);
-        for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_cnt[b] = 0;
-        if (threadIdx.x < 32) {
-            const int klo = kernel_of_event_warp(kptr, 0, (int)B.K - 1, base, (int)threadIdx.x);
-            const int khi = kernel_of_event_warp(kptr, klo, (int)B.K - 1, base + n_tile - 1, (int)threadIdx.x);
-            if (threadIdx.x == 0) { s_lohi[0] = klo; s_lohi[1] = khi; }
-        }
-        __syncthreads();
-        int lo = s_lohi[0], hi = s_lohi[1], shift_k = 0;
-        const int64_t *sp = kptr;
-        if (hi - lo + 2 <= kBkPtrStage) {
-            for (int j = threadIdx.x; j <= hi - lo + 1; j += kBkThreads) s_ptr[j] = kptr[lo + j];
-            shift_k = lo; hi -= lo; lo = 0; sp = s_ptr;
-        }
-        __syncthreads();
-        int bucket[kBkItems];
-        int rank[kBkItems];
-        ull key[kBkItems];
-#pragma unroll
-        for (int j = 0; j < kBkItems; ++j) {
-            const int64_t e = base + (int64_t)j * kBkThreads + threadIdx.x;
-            bucket[j] = -1;
-            if (e < B.E) {
-                const int32_t i = kt[e];
-                if (i >= 0 && i < B.N) {
-                    const int k = bk_kernel_of_event(sp, lo, hi, e) + shift_k;
-                    bucket[j] = i >> B.shift;
-                    key[j] = ((ull)(unsigned)(i & (B.bt - 1)) << 32) | (unsigned)k;
-                    rank[j] = atomicAdd(&s_cnt[bucket[j]], 1);
-                }
+        const int64_t tk0 = tile * TK, tk1 = tk0 + TK < B.K ? tk0 + TK : B.K;
+        const int64_t T0 = kptr[tk0], T1 = kptr[tk1];
+        // (a tile with more events than the staging area holds goes through it in several rounds)
+#pragma unroll 1
+        for (int64_t eb = T0; eb < T1; eb += kBkKeyCap) {
+#ifdef G10_PHASE_CLOCKS
+            ++ph_n;
+#endif
+            const int64_t ee = eb + kBkKeyCap < T1 ? eb + kBkKeyCap : T1;
+            for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_cnt[b] = 0;
+            __syncthreads();
+            BK_CLOCK(1);
+            bk_walk<false>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key, s_bkt);
+            __syncthreads();
+            BK_CLOCK(2);
+            // reserve this tile's room in every bucket it touches, then turn the tile counts into tile offsets
+            for (int b = threadIdx.x; b < B.nb; b += kBkThreads)
+                s_off[b] = s_cnt[b] ? (int)atomicAdd(&B.bucket_cursor[b], (unsigned)s_cnt[b]) : 0;
+            block_scan_counts((const unsigned *)s_cnt, B.nb, s_cnt, s_warp);      // in place: s_cnt[b] = first slot of bucket b in the tile
+            BK_CLOCK(3);
+            for (int b = threadIdx.x; b < B.nb; b += kBkThreads) s_off[b] += s_base[b] - s_cnt[b];
+            __syncthreads();
+            bk_walk<true>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key, s_bkt);
+            __syncthreads();
+            BK_CLOCK(4);
+            const int n_valid = s_cnt[B.nb] < kBkKeyCap ? s_cnt[B.nb] : kBkKeyCap;
+            for (int slot = threadIdx.x; slot < n_valid; slot += kBkThreads) {
+                const int64_t pos = (int64_t)s_off[s_bkt[slot]] + slot;
+                if (pos >= 0 && pos < B.E) B.pairs[pos] = s_key[slot];
             }
+            __syncthreads();
+            BK_CLOCK(5);
         }
-        __syncthreads();
-        // reserve this tile's room in every bucket it touches, then turn the tile counts into tile offsets
-        for (int b = threadIdx.x; b < B.nb; b += kBkThreads)
-            if (s_cnt[b]) s_off[b] = atomicAdd(&B.bucket_cursor[b], (unsigned)s_cnt[b]);
-        __syncthreads();
-        block_scan_counts((const unsigned *)s_cnt, B.nb, s_cnt, s_warp);      // in place: s_cnt[b] = first slot of bucket b in the tile
-#pragma unroll
-        for (int j = 0; j < kBkItems; ++j)
-            if (bucket[j] >= 0) {
-                const int slot = s_cnt[bucket[j]] + rank[j];
-                s_key[slot] = key[j];
-                s_bkt[slot] = (unsigned short)bucket[j];
-            }
-        __syncthreads();
-        const int n_valid = s_cnt[B.nb];
-        for (int slot = threadIdx.x; slot < n_valid; slot += kBkThreads) {
-            const int b = s_bkt[slot];
-            const int64_t pos = (int64_t)s_base[b] + s_off[b] + (slot - s_cnt[b]);
-            if (pos < B.E) B.pairs[pos] = s_key[slot];
-        }
-        __syncthreads();
     }
+#ifdef G10_PHASE_CLOCKS
+    if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 100) && ph_n > 0)
+        printf("k_bk_scatter block %d (%d rounds): setup %lld; cycles/round: zero %lld count %lld cursors+scan %lld place %lld write %lld\n",
+               blockIdx.x, ph_n, ph_acc[0], ph_acc[1] / ph_n, ph_acc[2] / ph_n, ph_acc[3] / ph_n, ph_acc[4] / ph_n, ph_acc[5] / ph_n);
+#endif
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -238,12 +290,6 @@ __device__ void bk_bitonic_sort_i32(int32_t *a, int n)    // arbitrary n: the ne
 
 __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
 
-#ifdef G10_PHASE_CLOCKS
-#define BK_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
-                         ph_acc[i] += now_ - ph_last; ph_last = now_; asm volatile("" ::: "memory"); } } while (0)
-#else
-#define BK_CLOCK(i)
-#endif
 
 __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBuffers out)
 {
@@ -265,6 +311,10 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
     __shared__ long long s_pre[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     block_scan_counts(B.bucket_count, B.nb, s_base, s_scan);
+    if (*(volatile ull *)B.status & G10_DEV_BAD_KERNEL_PTR) {      // nothing was partitioned: every tensor comes out unused
+        for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_base[b] = 0;
+        __syncthreads();
+    }
     for (;;) {
         __syncthreads();
         if (threadIdx.x == 0) { s_bucket = (int)atomicAdd(B.ticket, 1u); s_nheavy = 0; }
@@ -492,7 +542,7 @@ bool vitality_buckets_supported(int64_t N, int64_t E)
 cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s)
 {
     BucketArgs B;
-    B.N = t.N; B.E = t.E; B.K = t.K;
+    B.N = t.N; B.E = t.E; B.K = t.K; B.tile_kernels = kBkThreads;
     if (!choose_buckets(t.N, t.E, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
     B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
     B.ticket = w.emit_scan.ticket; B.status = w.status; B.spill = w.raw_uses;
@@ -501,11 +551,17 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     const int64_t tiles = (t.E + kBkTile - 1) / kBkTile;
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
-        k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_tensors);
-        const size_t sm2 = sizeof(int) * (size_t)(3 * B.nb + 2) + 8 + (sizeof(ull) + sizeof(unsigned short)) * kBkTile;
+        k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
+        // kernels per partition tile: as many as fill the staging area on average, in steps of one sweep of the block
+        int64_t sweeps = ((int64_t)kBkKeyCap * t.K) / (t.E * kBkThreads);
+        sweeps = sweeps < 1 ? 1 : (sweeps > 8 ? 8 : sweeps);
+        B.tile_kernels = (int)(sweeps * kBkThreads);
+        const int64_t ktiles = (t.K + B.tile_kernels - 1) / B.tile_kernels;
+        const int g2 = (int)(ktiles < 3 * (int64_t)sms ? ktiles : 3 * (int64_t)sms);
+        const size_t sm2 = sizeof(int) * (size_t)(3 * B.nb + 2) + 8 + (sizeof(ull) + sizeof(unsigned short)) * kBkKeyCap;
         cudaError_t e = cudaFuncSetAttribute(k_bk_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
         if (e != cudaSuccess) return e;
-        k_bk_scatter<<<g, kBkThreads, sm2, s>>>(B, t.kernel_ptr, t.kernel_tensors);
+        k_bk_scatter<<<g2, kBkThreads, sm2, s>>>(B, t.kernel_ptr, t.kernel_tensors);
     }
     const size_t sm3 = sizeof(int) * (size_t)(B.nb + 1 + 3 * (B.bt + 1) + kBkCap);
     cudaError_t e = cudaFuncSetAttribute(k_bk_emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);

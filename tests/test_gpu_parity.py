@@ -148,6 +148,25 @@ def test_bandwidth_and_capacity_sweep(gpu, oracle):
                         n += 1
 
 
+def test_wide_kernels(gpu, oracle):
+    """Kernels that list hundreds or thousands of tensors (an optimizer step over everything): more events in one
+    kernel than a warp row, and more in one partition tile than its staging area holds."""
+    rng = np.random.default_rng(99)
+    N = 15000
+    lists = []
+    for k in range(48):
+        if k in (3, 40):
+            lists.append(list(range(N)) if k == 3 else list(range(0, N, 2)))      # 15 000 and 7 500 tensors
+        elif k in (7, 8):
+            lists.append(rng.integers(0, N, size=300 if k == 7 else 65).tolist()) # repeats inside the list allowed
+        else:
+            lists.append(rng.integers(0, N, size=int(rng.integers(0, 6))).tolist())
+    tr = traces.from_lists("wide", lists, rng.integers(1, 1 << 20, size=N).tolist(), rng.integers(1000, 50000, size=48).tolist(),
+                           capacity_frac=(1, 2))
+    ref = full_parity(gpu, oracle, tr)
+    assert len(ref.migrations) > 0
+
+
 def test_inplace_relu_variant(gpu, oracle):
     tr = traces.config1_resnet152(inplace_relu=True)
     full_parity(gpu, oracle, tr)
