@@ -239,11 +239,20 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
             __syncthreads();
             BK_CLOCK(2);
             // reserve this tile's room in every bucket it touches, then turn the tile counts into tile offsets
-            for (int b = threadIdx.x; b < B.nb; b += kBkThreads)
-                s_off[b] = s_cnt[b] ? (int)atomicAdd(&B.bucket_cursor[b], (unsigned)s_cnt[b]) : 0;
+            // (the global cursors answer while the block scans: their results stay in registers until after the scan)
+            int cur[8];                                            // nb <= 4096 = 8 * kBkThreads
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int b = j * kBkThreads + threadIdx.x;
+                cur[j] = (b < B.nb && s_cnt[b]) ? (int)atomicAdd(&B.bucket_cursor[b], (unsigned)s_cnt[b]) : 0;
+            }
             block_scan_counts((const unsigned *)s_cnt, B.nb, s_cnt, s_warp);      // in place: s_cnt[b] = first slot of bucket b in the tile
             BK_CLOCK(3);
-            for (int b = threadIdx.x; b < B.nb; b += kBkThreads) s_off[b] += s_base[b] - s_cnt[b];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int b = j * kBkThreads + threadIdx.x;
+                if (b < B.nb) s_off[b] = cur[j] + s_base[b] - s_cnt[b];
+            }
             __syncthreads();
             bk_walk<true>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key, s_bkt);
             __syncthreads();
