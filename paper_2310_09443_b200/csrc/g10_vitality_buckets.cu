@@ -50,6 +50,10 @@ struct BucketArgs {
 template <int NA>
 __device__ __forceinline__ void bk_block_scan(const int *in0, int *out0, const int *in1, int *out1, int n, int *s_w /* [NA][kBkThreads/32 + 1] */)
 {
+    // The arrays start on 16-byte boundaries and are padded to a multiple of four entries (bk_pad), so a thread's
+    // eight entries move as two 128-bit accesses (eight 32-bit ones at a stride of eight words would meet in the
+    // same banks eight at a time).  Entries at or past n are read (they lie inside the padding or the next array)
+    // but never used or written.
     constexpr int W = kBkThreads / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int base = threadIdx.x * 8;
@@ -57,9 +61,13 @@ __device__ __forceinline__ void bk_block_scan(const int *in0, int *out0, const i
 #pragma unroll
     for (int a = 0; a < NA; ++a) {
         const int *in = a == 0 ? in0 : in1;
+        int4 x = make_int4(0, 0, 0, 0), y = make_int4(0, 0, 0, 0);
+        if (base < n) x = *reinterpret_cast<const int4 *>(in + base);
+        if (base + 4 < n) y = *reinterpret_cast<const int4 *>(in + base + 4);
+        v[a][0] = x.x; v[a][1] = x.y; v[a][2] = x.z; v[a][3] = x.w; v[a][4] = y.x; v[a][5] = y.y; v[a][6] = y.z; v[a][7] = y.w;
         tot[a] = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { v[a][j] = base + j < n ? in[base + j] : 0; tot[a] += v[a][j]; }
+        for (int j = 0; j < 8; ++j) { if (base + j >= n) v[a][j] = 0; tot[a] += v[a][j]; }
     }
     int incl[NA];
 #pragma unroll
@@ -88,12 +96,23 @@ __device__ __forceinline__ void bk_block_scan(const int *in0, int *out0, const i
     for (int a = 0; a < NA; ++a) {
         int *out = a == 0 ? out0 : out1;
         int run = s_w[a * (W + 1) + warp] + incl[a] - tot[a];
+        int r[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { if (base + j < n) out[base + j] = run; run += v[a][j]; }
+        for (int j = 0; j < 8; ++j) { r[j] = run; run += v[a][j]; }
+        if (base + 8 <= n) {
+            *reinterpret_cast<int4 *>(out + base) = make_int4(r[0], r[1], r[2], r[3]);
+            *reinterpret_cast<int4 *>(out + base + 4) = make_int4(r[4], r[5], r[6], r[7]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) if (base + j < n) out[base + j] = r[j];
+        }
         if (threadIdx.x == 0) out[n] = s_w[a * (W + 1) + W];
     }
     __syncthreads();
 }
+
+// entries of a shared-memory array of n + 1 ints, padded so that the next array starts on a 16-byte boundary
+__host__ __device__ inline int bk_pad(int n) { return (n + 1 + 3) & ~3; }
 
 __device__ __forceinline__ void block_scan_counts(const unsigned *cnt, int n, int *out, int *s_w)
 {
@@ -205,10 +224,10 @@ __device__ __forceinline__ void bk_walk(const BucketArgs &B, const int64_t *__re
 
 __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
 {
-    extern __shared__ int s_mem[];
+    extern __shared__ __align__(16) int s_mem[];
     int *s_base = s_mem;                                   // [nb + 1] first key of each bucket
-    int *s_cnt = s_base + B.nb + 1;                        // [nb + 1] events of this tile per bucket, then their scan, then fill cursors
-    int *s_off = s_cnt + B.nb + 1;                         // [nb] global position of the tile's first key of the bucket minus its slot
+    int *s_cnt = s_base + bk_pad(B.nb);                      // [nb + 1] events of this tile per bucket, then their scan, then fill cursors
+    int *s_off = s_cnt + bk_pad(B.nb);                      // [nb] global position of the tile's first key of the bucket minus its slot
     ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkKeyCap] keys of the tile in bucket order
     unsigned short *s_bkt = (unsigned short *)(s_key + kBkKeyCap);           // [kBkKeyCap] their buckets
     __shared__ int s_warp[2 * (kBkThreads / 32 + 1)];
@@ -306,12 +325,12 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
     long long ph_acc[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
     int ph_n = 0;
 #endif
-    extern __shared__ int s_mem[];
+    extern __shared__ __align__(16) int s_mem[];
     int *s_base = s_mem;                       // [nb + 1] first key of each bucket
-    int *t_off = s_base + B.nb + 1;            // [bt + 1] raw events per tensor, then segment offsets
-    int *t_d = t_off + B.bt + 1;               // [bt + 1] scatter cursor, then distinct uses, then their offsets
-    int *t_np = t_d + B.bt + 1;                // [bt + 1] periods per tensor, then their offsets
-    int32_t *s_ks = t_np + B.bt + 1;           // [kBkCap] kernels, tensor segment after tensor segment
+    int *t_off = s_base + bk_pad(B.nb);          // [bt + 1] raw events per tensor, then segment offsets
+    int *t_d = t_off + bk_pad(B.bt);             // [bt + 1] scatter cursor, then distinct uses, then their offsets
+    int *t_np = t_d + bk_pad(B.bt);             // [bt + 1] periods per tensor, then their offsets
+    int32_t *s_ks = t_np + bk_pad(B.bt);         // [kBkCap] kernels, tensor segment after tensor segment
     __shared__ int s_scan[2 * (kBkThreads / 32 + 1)];
     __shared__ int s_wa[kBkThreads / 32], s_wb[kBkThreads / 32];
     __shared__ long long s_pu[kBkThreads / 32], s_pp[kBkThreads / 32];
@@ -567,12 +586,12 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         B.tile_kernels = (int)(sweeps * kBkThreads);
         const int64_t ktiles = (t.K + B.tile_kernels - 1) / B.tile_kernels;
         const int g2 = (int)(ktiles < 3 * (int64_t)sms ? ktiles : 3 * (int64_t)sms);
-        const size_t sm2 = sizeof(int) * (size_t)(3 * B.nb + 2) + 8 + (sizeof(ull) + sizeof(unsigned short)) * kBkKeyCap;
+        const size_t sm2 = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8 + (sizeof(ull) + sizeof(unsigned short)) * kBkKeyCap;
         cudaError_t e = cudaFuncSetAttribute(k_bk_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
         if (e != cudaSuccess) return e;
         k_bk_scatter<<<g2, kBkThreads, sm2, s>>>(B, t.kernel_ptr, t.kernel_tensors);
     }
-    const size_t sm3 = sizeof(int) * (size_t)(B.nb + 1 + 3 * (B.bt + 1) + kBkCap);
+    const size_t sm3 = sizeof(int) * (size_t)(bk_pad(B.nb) + 3 * bk_pad(B.bt) + kBkCap);
     cudaError_t e = cudaFuncSetAttribute(k_bk_emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
     const int g3 = B.nb < 2 * sms ? B.nb : 2 * sms;
