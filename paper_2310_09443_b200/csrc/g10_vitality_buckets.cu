@@ -331,10 +331,11 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
     int *t_d = t_off + bk_pad(B.bt);             // [bt + 1] scatter cursor, then distinct uses, then their offsets
     int *t_np = t_d + bk_pad(B.bt);             // [bt + 1] periods per tensor, then their offsets
     int32_t *s_ks = t_np + bk_pad(B.bt);         // [kBkCap] kernels, tensor segment after tensor segment
+    unsigned short *s_mid = (unsigned short *)(s_ks + kBkCap);   // [bt] tensors of the bucket with three to kBkHeavy raw uses
     __shared__ int s_scan[2 * (kBkThreads / 32 + 1)];
     __shared__ int s_wa[kBkThreads / 32], s_wb[kBkThreads / 32];
     __shared__ long long s_pu[kBkThreads / 32], s_pp[kBkThreads / 32];
-    __shared__ int s_bucket, s_nheavy, s_total, s_periods;
+    __shared__ int s_bucket, s_nheavy, s_nmid, s_total, s_periods;
     __shared__ int s_heavy[64];
     __shared__ long long s_pre[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -345,7 +346,9 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
     }
     for (;;) {
         __syncthreads();
-        if (threadIdx.x == 0) { s_bucket = (int)atomicAdd(B.ticket, 1u); s_nheavy = 0; }
+        // (the number is taken when the work starts, not earlier: a later bucket waits for the totals of all earlier
+        // ones, which are then certain to be under way)
+        if (threadIdx.x == 0) { s_bucket = (int)atomicAdd(B.ticket, 1u); s_nheavy = 0; s_nmid = 0; }
         __syncthreads();
         const int b = s_bucket;
         if (b >= B.nb) break;
@@ -389,28 +392,42 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         }
         __syncthreads();
         BK_CLOCK(3);
-        // ---- short segments: one thread sorts, removes repeats (in place) and counts the periods
+        // ---- short segments: one or two raw uses are settled on the spot; three to kBkHeavy go to a list that the
+        // threads then take one tensor each from (one thread sorts, removes repeats in place and counts the periods),
+        // so that a warp is not held up eight times over by its longest segment
         int my_d = 0, my_p = 0;                 // this thread's share of the bucket totals
         for (int tl = threadIdx.x; tl < bt_eff; tl += kBkThreads) {
-            const int m = t_off[tl + 1] - t_off[tl];
+            const int o = t_off[tl], m = t_off[tl + 1] - o;
             int dd = 0, pp = 0;
-            if (m > kBkHeavy) {
+            if (m == 1) dd = 1;
+            else if (m == 2) {
+                const int32_t x = ks[o], y = ks[o + 1];
+                const int32_t lo = x < y ? x : y, hi = x < y ? y : x;
+                if (lo == hi) dd = 1;
+                else { ks[o] = lo; ks[o + 1] = hi; dd = 2; pp = hi - lo >= 2 ? 1 : 0; }
+            } else if (m > kBkHeavy) {
                 const int q = atomicAdd(&s_nheavy, 1);
                 if (q < 64) s_heavy[q] = tl;
-            } else if (m > 0) {
-                int32_t *seg = ks + t_off[tl];
-                for (int a = 1; a < m; ++a) {
-                    const int32_t x = seg[a];
-                    int c = a - 1;
-                    while (c >= 0 && seg[c] > x) { seg[c + 1] = seg[c]; --c; }
-                    seg[c + 1] = x;
-                }
-                int32_t prev = seg[0];
-                dd = 1;
-                for (int a = 1; a < m; ++a) {
-                    const int32_t x = seg[a];
-                    if (x != prev) { if (x - prev >= 2) ++pp; seg[dd++] = x; prev = x; }
-                }
+            } else if (m > 2) s_mid[atomicAdd(&s_nmid, 1)] = (unsigned short)tl;
+            t_d[tl] = dd; t_np[tl] = pp;
+            my_d += dd; my_p += pp;
+        }
+        __syncthreads();
+        for (int q = threadIdx.x; q < s_nmid; q += kBkThreads) {
+            const int tl = s_mid[q];
+            const int m = t_off[tl + 1] - t_off[tl];
+            int32_t *seg = ks + t_off[tl];
+            for (int a = 1; a < m; ++a) {
+                const int32_t x = seg[a];
+                int c = a - 1;
+                while (c >= 0 && seg[c] > x) { seg[c + 1] = seg[c]; --c; }
+                seg[c + 1] = x;
+            }
+            int32_t prev = seg[0];
+            int dd = 1, pp = 0;
+            for (int a = 1; a < m; ++a) {
+                const int32_t x = seg[a];
+                if (x != prev) { if (x - prev >= 2) ++pp; seg[dd++] = x; prev = x; }
             }
             t_d[tl] = dd; t_np[tl] = pp;
             my_d += dd; my_p += pp;
@@ -591,7 +608,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         if (e != cudaSuccess) return e;
         k_bk_scatter<<<g2, kBkThreads, sm2, s>>>(B, t.kernel_ptr, t.kernel_tensors);
     }
-    const size_t sm3 = sizeof(int) * (size_t)(bk_pad(B.nb) + 3 * bk_pad(B.bt) + kBkCap);
+    const size_t sm3 = sizeof(int) * (size_t)(bk_pad(B.nb) + 3 * bk_pad(B.bt) + kBkCap) + sizeof(unsigned short) * (size_t)B.bt;
     cudaError_t e = cudaFuncSetAttribute(k_bk_emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
     const int g3 = B.nb < 2 * sms ? B.nb : 2 * sms;
