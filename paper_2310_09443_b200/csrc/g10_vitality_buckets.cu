@@ -25,7 +25,7 @@ namespace g10 {
 constexpr int kBkThreads = 512;
 constexpr int kBkItems = 8;
 constexpr int kBkTile = kBkThreads * kBkItems;     // events per partition tile (4096)
-constexpr int kBkCap = 12288;                      // events of a bucket kept in shared memory
+constexpr int kBkCap = 10240;                      // events of a bucket kept in shared memory
 constexpr int kBkWide = 64;                        // a kernel with more events is walked by its whole warp in the partition
 constexpr int kBkKeyCap = 6144;                    // keys of one partition tile staged in shared memory
 constexpr int kBkHeavy = 32;                       // longer segments are sorted by the whole block
@@ -526,7 +526,12 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         if (U + D > out.uses_cap) bad |= G10_DEV_USES_OVERFLOW;
         if (PB + PC > out.periods_cap) bad |= G10_DEV_PERIODS_OVERFLOW;
         if (bad && threadIdx.x == 0) raise_status(B.status, bad);
-        // ---- outputs
+        // ---- outputs.  Without repeats anywhere in the bucket (the usual case) the segments are already the use
+        // lists, back to back in tensor order: they go out as one coalesced copy.
+        const bool dense = D == n;
+        if (dense)
+            for (int j = threadIdx.x; j < n; j += kBkThreads)
+                if (U + j < out.uses_cap) out.uses[U + j] = ks[j];
         for (int tl = threadIdx.x; tl < bt_eff; tl += kBkThreads) {
             const int64_t t = t0 + tl;
             const int dd = t_d[tl + 1] - t_d[tl];
@@ -537,9 +542,9 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             out.use_ptr[t] = U + t_d[tl];
             out.period_ptr[t] = PB + t_np[tl];
             long long uo = U + t_d[tl], po = PB + t_np[tl];
-            for (int a = 0; a < dd; ++a) {
+            for (int a = dense ? 1 : 0; a < dd; ++a) {
                 const int32_t x = seg[a];
-                if (uo + a < out.uses_cap) out.uses[uo + a] = x;
+                if (!dense && uo + a < out.uses_cap) out.uses[uo + a] = x;
                 if (a > 0 && x - seg[a - 1] >= 2) {
                     if (po < out.periods_cap) {
                         out.period_tensor[po] = (int32_t)t;
