@@ -33,9 +33,9 @@ WORKLOAD = "config1_resnet152_b256"
 L2_FLUSH_BYTES = 512 << 20
 PLAN_ONE_DRAM_BYTES = 211456    # dram__bytes_read.sum + dram__bytes_write.sum of one k_plan_one launch on config 1 (ncu --set full capture)
 # DRAM bytes per call on the stress trace, from an ncu capture of `bench.py --stress-only --stress-reps 1` (dram__bytes_read.sum +
-# dram__bytes_write.sum summed over the call's kernels): k_bk_hist 19.9 + k_bk_scatter 28.1 + k_bk_emit 135.5 MB; k_seg_scan<0> 16.0 +
+# dram__bytes_write.sum summed over the call's kernels): k_bk_hist 28.0 + k_bk_scatter 28.2 + k_bk_emit 138.0 MB; k_seg_scan<0> 16.0 +
 # k_first_last_events 59.9 + k_diff_scatter 76.1 + k_seg_scan<1> 8.0 MB
-STRESS_VITALITY_DRAM_BYTES = 183_500_000
+STRESS_VITALITY_DRAM_BYTES = 194_200_000
 STRESS_TIMELINE_DRAM_BYTES = 160_000_000
 KERNELS_PER_PLAN = 10      # slot clock, bucket histogram, bucket scatter, bucket emit, diff, pressure scan, geometry,
                            # single-block loop, multi-block loop (returns at once when the former did the work), status

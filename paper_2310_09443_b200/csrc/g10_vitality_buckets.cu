@@ -123,7 +123,7 @@ __device__ __forceinline__ void block_scan_counts(const unsigned *cnt, int n, in
 // between the marked points and prints the averages at the end.
 #ifdef G10_PHASE_CLOCKS
 #define BK_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
-                         ph_acc[i] += now_ - ph_last; ph_last = now_; asm volatile("" ::: "memory"); } } while (0)
+                         ph_acc[i] += now_ - ph_acc[15]; ph_acc[15] = now_; asm volatile("" ::: "memory"); } } while (0)
 #else
 #define BK_CLOCK(i)
 #endif
@@ -233,7 +233,8 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
     __shared__ int s_warp[2 * (kBkThreads / 32 + 1)];
     if (*(volatile ull *)B.status & G10_DEV_BAD_KERNEL_PTR) return;          // (found by k_bk_hist: nothing is partitioned)
 #ifdef G10_PHASE_CLOCKS
-    long long ph_acc[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
+    __shared__ long long ph_acc[16];                     // (in shared memory: the register count stays that of the library build)
+    if (threadIdx.x == 0) { for (int i = 0; i < 15; ++i) ph_acc[i] = 0; ph_acc[15] = clock64(); }
     int ph_n = 0;
 #endif
     block_scan_counts(B.bucket_count, B.nb, s_base, s_warp);
@@ -322,7 +323,8 @@ __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ul
 __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBuffers out)
 {
 #ifdef G10_PHASE_CLOCKS
-    long long ph_acc[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
+    __shared__ long long ph_acc[16];                     // (in shared memory: the register count stays that of the library build)
+    if (threadIdx.x == 0) { for (int i = 0; i < 15; ++i) ph_acc[i] = 0; ph_acc[15] = clock64(); }
     int ph_n = 0;
 #endif
     extern __shared__ __align__(16) int s_mem[];

@@ -248,6 +248,29 @@ def test_bad_trace_sets_status_bits(gpu):
     assert (st & 0x1) and (st & 0x8) and (st & 0x4)
 
 
+def test_bad_kernel_ptr_is_flagged(gpu):
+    """A kernel_ptr that is not a monotone map onto [0, E]: both calls finish, stay in bounds and say so."""
+    import torch
+    base = traces.config0_mlp_chain()
+    for kind in ("swapped", "beyond", "short"):
+        tr = traces.config0_mlp_chain()
+        ptr = base.kernel_ptr.copy()
+        if kind == "swapped":
+            ptr[10], ptr[20] = base.kernel_ptr[20], base.kernel_ptr[10]
+        elif kind == "beyond":
+            ptr[50:60] = base.E + 1000
+        else:
+            ptr[-1] = base.E - 7
+        tr.kernel_ptr = ptr
+        tb = gpu.upload(tr)
+        v = gpu.g10_vitality(tb)
+        tl = gpu.g10_pressure_timeline(tb)
+        torch.cuda.synchronize()
+        assert _np(v.counts)[2] & 0x2, kind
+        assert int(tl.status.item()) & 0x2, kind
+        assert _np(v.counts)[0] == 0 and (_np(v.num_uses) == 0).all()       # nothing is partitioned
+
+
 def test_host_pointer_mode(gpu, oracle):
     """The same calls with every array in (pinned) host memory: the library stages the copies itself."""
     tr = traces.config1_resnet152()
