@@ -168,7 +168,8 @@ typedef struct g10_options {
 #define G10_WS_EMIT 4
 #define G10_WS_BATCH 5
 
-/* Section 4.2, tensor vitality analysis. */
+/* Section 4.2, tensor vitality analysis.  Device-found errors land in counts[2]; with G10_DEV_BAD_KERNEL_PTR every
+   tensor is reported unused (no uses, no periods), with G10_DEV_BAD_TENSOR_ID the offending entries are skipped. */
 int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, size_t ws_bytes, void *stream);
 
 /* Section 4.3, GPU memory pressure over time (difference array of signed sizes + prefix scan). */
