@@ -16,23 +16,38 @@ namespace g10 {
 // has always started.
 // =============================================================================================
 constexpr int kSegThreads = 512;
-constexpr int kSegItems = 4;
+constexpr int kSegWarps = kSegThreads / 32;
+constexpr int kSegItems = 8;
 constexpr int kSegChunk = kSegThreads * kSegItems;
 constexpr int kSegMaxBlocks = 512;
 
 __device__ __forceinline__ ull seg_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
 __device__ __forceinline__ long long seg_unpack(ull w) { return (long long)(w << 2) >> 2; }     // sign-extend 62 bits
 
+// Sum of one value per warp (s_w[kSegWarps], written by the lanes 0 before a barrier): every warp adds them up
+// for itself with shuffles.  Also returns the sum over the warps before this one.
+__device__ __forceinline__ long long seg_warp_totals(const long long *s_w, int lane, int warp, long long *before)
+{
+    const long long x = lane < kSegWarps ? s_w[lane] : 0;
+    long long incl = x;
+#pragma unroll
+    for (int o = 1; o < kSegWarps; o <<= 1) {
+        const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    *before = __shfl_sync(0xffffffffu, incl - x, warp);
+    return __shfl_sync(0xffffffffu, incl, kSegWarps - 1);
+}
+
 // kind 0: exclusive scan of kernel_ns into start[0..K] with validation of kernel_ns and kernel_ptr
 // kind 1: inclusive scan of the difference array into the pressure, plus peak and lowest peak slot
 template <int kind>
-__global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, const int64_t *__restrict__ in, const int64_t *__restrict__ kptr,
-                                                          int64_t *__restrict__ out, unsigned *ticket, unsigned *done, ull *words,
-                                                          int64_t *blk_max, int32_t *blk_slot, int64_t *peak_bytes, int32_t *peak_slot, ull *status)
+__global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t E, const int64_t *__restrict__ in, const int64_t *__restrict__ kptr,
+                                                             int64_t *__restrict__ out, unsigned *ticket, unsigned *done, ull *words,
+                                                             int64_t *blk_max, int32_t *blk_slot, int64_t *peak_bytes, int32_t *peak_slot, ull *status)
 {
-    __shared__ long long s_w[kSegThreads / 32];
-    __shared__ int s_sl[kSegThreads / 32];
-    __shared__ long long s_bcast;
+    __shared__ long long s_w[kSegWarps];
+    __shared__ int s_sl[kSegWarps];
     __shared__ bool s_last;
     const int G = gridDim.x;
     // Nothing later in a call reads the slot clock, so a kernel launched behind this one with programmatic stream
@@ -45,16 +60,16 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
     // ---- pass 1: segment sum
     long long sum = 0;
     ull bad = 0;
-    for (int64_t k0 = lo + threadIdx.x; k0 < hi; k0 += 8 * kSegThreads) {
-        long long v[8], p0[8], p1[8];
+    for (int64_t k0 = lo + threadIdx.x; k0 < hi; k0 += 4 * kSegThreads) {
+        long long v[4], p0[4], p1[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {                      // all loads of the batch in flight together
+        for (int j = 0; j < 4; ++j) {                      // all loads of the batch in flight together
             const int64_t k = k0 + (int64_t)j * kSegThreads;
             v[j] = k < hi ? in[k] : (kind == 0 ? 1 : 0);
             if (kind == 0) { p0[j] = k < hi ? kptr[k] : 0; p1[j] = k < hi ? kptr[k + 1] : 0; }
         }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < 4; ++j) {
             const int64_t k = k0 + (int64_t)j * kSegThreads;
             if (k < hi) {
                 if (kind == 0) {
@@ -70,11 +85,10 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
     sum = warp_sum_i64(sum);
     if (lane == 0) s_w[warp] = sum;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        long long tot = 0;
-        for (int w = 0; w < kSegThreads / 32; ++w) tot += s_w[w];
-        asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&words[g]), "l"(seg_pack(tot)) : "memory");
-    }
+    long long unused;
+    const long long seg_total = seg_warp_totals(s_w, lane, warp, &unused);
+    if (threadIdx.x == 0)
+        asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&words[g]), "l"(seg_pack(seg_total)) : "memory");
     // ---- prefix of the segment: all predecessors' sums
     long long pre = 0;
     for (int j = threadIdx.x; j < g; j += kSegThreads) {
@@ -89,16 +103,10 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
         pre += seg_unpack(w);
     }
     pre = warp_sum_i64(pre);
-    __syncthreads();
+    __syncthreads();                                       // s_w has been read by every warp
     if (lane == 0) s_w[warp] = pre;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        long long tot = 0;
-        for (int w = 0; w < kSegThreads / 32; ++w) tot += s_w[w];
-        s_bcast = tot;
-    }
-    __syncthreads();
-    long long carry = s_bcast;
+    long long carry = seg_warp_totals(s_w, lane, warp, &unused);
     // ---- pass 2: scan the segment chunk by chunk (each thread kSegItems consecutive elements)
     long long mx = 0;
     int sl = -1;
@@ -114,12 +122,11 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
             tsum += v[j];
         }
         const long long incl = warp_inclusive_scan_i64(tsum, lane);
-        __syncthreads();
+        __syncthreads();                                   // s_w has been read by every warp
         if (lane == 31) s_w[warp] = incl;
         __syncthreads();
-        long long wpre = 0, ctot = 0;
-#pragma unroll
-        for (int w = 0; w < kSegThreads / 32; ++w) { const long long x = s_w[w]; if (w < warp) wpre += x; ctot += x; }
+        long long wpre;
+        const long long ctot = seg_warp_totals(s_w, lane, warp, &wpre);
         long long run = carry + wpre + incl - tsum;
 #pragma unroll
         for (int j = 0; j < kSegItems; ++j) {
@@ -150,7 +157,7 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
     if (lane == 0) { s_w[warp] = mx; s_sl[warp] = sl; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int w = 1; w < kSegThreads / 32; ++w)
+        for (int w = 1; w < kSegWarps; ++w)
             if (s_sl[w] >= 0 && (sl < 0 || s_w[w] > mx || (s_w[w] == mx && s_sl[w] < sl))) { mx = s_w[w]; sl = s_sl[w]; }
         blk_max[g] = mx;
         blk_slot[g] = sl;
@@ -177,7 +184,7 @@ __global__ void __launch_bounds__(kSegThreads) k_seg_scan(int64_t n, int64_t E, 
         if (lane == 0) { s_w[warp] = bm; s_sl[warp] = bs; }
         __syncthreads();
         if (threadIdx.x == 0) {
-            for (int w = 1; w < kSegThreads / 32; ++w)
+            for (int w = 1; w < kSegWarps; ++w)
                 if (s_sl[w] >= 0 && (bs < 0 || s_w[w] > bm || (s_w[w] == bm && s_sl[w] < bs))) { bm = s_w[w]; bs = s_sl[w]; }
             *peak_bytes = bs < 0 ? 0 : bm;
             *peak_slot = bs;
