@@ -171,9 +171,9 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
 // events of its own kernel (so the kernel of an event is known without a search); a kernel with more than
 // kBkWide events is walked by the whole warp instead.
 // kPlace false: count the events of every bucket.  true: s_cnt[b] is the next free slot of bucket b in the tile's
-// staging area; the key and its bucket go there.
+// staging area; the key goes there with its bucket in the spare upper bits.
 template <bool kPlace>
-__device__ __forceinline__ void bk_take(const BucketArgs &B, int32_t i, int64_t k, int *s_cnt, ull *s_key, unsigned short *s_bkt)
+__device__ __forceinline__ void bk_take(const BucketArgs &B, int32_t i, int64_t k, int *s_cnt, ull *s_key)
 {
     if (i < 0 || i >= B.N) return;
     const int b = i >> B.shift;
@@ -181,15 +181,14 @@ __device__ __forceinline__ void bk_take(const BucketArgs &B, int32_t i, int64_t 
     else {
         const int slot = atomicAdd(&s_cnt[b], 1);
         if (slot < kBkKeyCap) {
-            s_key[slot] = ((ull)(unsigned)(i & (B.bt - 1)) << 32) | (unsigned)k;
-            s_bkt[slot] = (unsigned short)b;
+            s_key[slot] = ((ull)(unsigned)b << 48) | ((ull)(unsigned)(i & (B.bt - 1)) << 32) | (unsigned)k;
         }
     }
 }
 
 template <bool kPlace>
 __device__ __forceinline__ void bk_walk(const BucketArgs &B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt, int64_t tk0,
-                                        int64_t tk1, int64_t eb, int64_t ee, int *s_cnt, ull *s_key, unsigned short *s_bkt)
+                                        int64_t tk1, int64_t eb, int64_t ee, int *s_cnt, ull *s_key)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll 1
@@ -207,7 +206,7 @@ __device__ __forceinline__ void bk_walk(const BucketArgs &B, const int64_t *__re
 #pragma unroll
                 for (int u = 0; u < 4; ++u) id[u] = e + u < b ? kt[e + u] : -1;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) bk_take<kPlace>(B, id[u], k, s_cnt, s_key, s_bkt);
+                for (int u = 0; u < 4; ++u) bk_take<kPlace>(B, id[u], k, s_cnt, s_key);
             }
         }
         unsigned m = __ballot_sync(0xffffffffu, wide);
@@ -217,7 +216,7 @@ __device__ __forceinline__ void bk_walk(const BucketArgs &B, const int64_t *__re
             m &= m - 1;
             const int64_t wa = __shfl_sync(0xffffffffu, a, src), wb = __shfl_sync(0xffffffffu, b, src);
 #pragma unroll 1
-            for (int64_t e = wa + lane; e < wb; e += 32) bk_take<kPlace>(B, kt[e], k0 + src, s_cnt, s_key, s_bkt);
+            for (int64_t e = wa + lane; e < wb; e += 32) bk_take<kPlace>(B, kt[e], k0 + src, s_cnt, s_key);
         }
     }
 }
@@ -228,8 +227,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
     int *s_base = s_mem;                                   // [nb + 1] first key of each bucket
     int *s_cnt = s_base + bk_pad(B.nb);                      // [nb + 1] events of this tile per bucket, then their scan, then fill cursors
     int *s_off = s_cnt + bk_pad(B.nb);                      // [nb] global position of the tile's first key of the bucket minus its slot
-    ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkKeyCap] keys of the tile in bucket order
-    unsigned short *s_bkt = (unsigned short *)(s_key + kBkKeyCap);           // [kBkKeyCap] their buckets
+    ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkKeyCap] keys of the tile in bucket order, the bucket in bits 48..59
     __shared__ int s_warp[2 * (kBkThreads / 32 + 1)];
     if (*(volatile ull *)B.status & G10_DEV_BAD_KERNEL_PTR) return;          // (found by k_bk_hist: nothing is partitioned)
 #ifdef G10_PHASE_CLOCKS
@@ -255,7 +253,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
             for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_cnt[b] = 0;
             __syncthreads();
             BK_CLOCK(1);
-            bk_walk<false>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key, s_bkt);
+            bk_walk<false>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key);
             __syncthreads();
             BK_CLOCK(2);
             // reserve this tile's room in every bucket it touches, then turn the tile counts into tile offsets
@@ -274,13 +272,14 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
                 if (b < B.nb) s_off[b] = cur[j] + s_base[b] - s_cnt[b];
             }
             __syncthreads();
-            bk_walk<true>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key, s_bkt);
+            bk_walk<true>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key);
             __syncthreads();
             BK_CLOCK(4);
             const int n_valid = s_cnt[B.nb] < kBkKeyCap ? s_cnt[B.nb] : kBkKeyCap;
             for (int slot = threadIdx.x; slot < n_valid; slot += kBkThreads) {
-                const int64_t pos = (int64_t)s_off[s_bkt[slot]] + slot;
-                if (pos >= 0 && pos < B.E) B.pairs[pos] = s_key[slot];
+                const ull key = s_key[slot];                       // bits 48..59: the bucket (staging only)
+                const int64_t pos = (int64_t)s_off[(int)(key >> 48)] + slot;
+                if (pos >= 0 && pos < B.E) B.pairs[pos] = key & 0x0000ffffffffffffull;
             }
             __syncthreads();
             BK_CLOCK(5);
@@ -610,7 +609,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         B.tile_kernels = (int)(sweeps * kBkThreads);
         const int64_t ktiles = (t.K + B.tile_kernels - 1) / B.tile_kernels;
         const int g2 = (int)(ktiles < 3 * (int64_t)sms ? ktiles : 3 * (int64_t)sms);
-        const size_t sm2 = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8 + (sizeof(ull) + sizeof(unsigned short)) * kBkKeyCap;
+        const size_t sm2 = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8 + sizeof(ull) * kBkKeyCap;
         cudaError_t e = cudaFuncSetAttribute(k_bk_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
         if (e != cudaSuccess) return e;
         k_bk_scatter<<<g2, kBkThreads, sm2, s>>>(B, t.kernel_ptr, t.kernel_tensors);
