@@ -167,6 +167,42 @@ def test_wide_kernels(gpu, oracle):
     assert len(ref.migrations) > 0
 
 
+def _csr_trace(name, rng, K, N, degrees):
+    """A trace from per-kernel degrees (tensor ids uniform, repeats allowed), sizes and durations random."""
+    ptr = np.zeros(K + 1, dtype=np.int64)
+    ptr[1:] = np.cumsum(degrees)
+    E = int(ptr[-1])
+    return traces.Trace(name=name, kernel_ptr=ptr, kernel_tensors=rng.integers(0, N, size=E).astype(np.int32),
+                        tensor_bytes=rng.integers(1, 1 << 24, size=N).astype(np.int64),
+                        kernel_ns=rng.integers(1, 100000, size=K).astype(np.int64),
+                        tensor_global=(rng.random(N) < 0.01).astype(np.uint8), capacity_frac=(1, 2))
+
+
+@pytest.mark.parametrize("shape", ["one_event_per_kernel", "mostly_empty_kernels", "few_tensors_many_uses", "every_kernel_wide", "many_tensors"])
+def test_pass_shapes(gpu, oracle, shape):
+    """Vitality and timeline on traces whose shape drives the partition differently: the widest and the narrowest tiles,
+    empty kernels, buckets that overflow shared memory, kernels all wider than a warp row, thousands of buckets."""
+    rng = np.random.default_rng(1000 + len(shape))
+    if shape == "one_event_per_kernel":
+        K, N = 200_000, 50_000
+        tr = _csr_trace(shape, rng, K, N, np.ones(K, dtype=np.int64))
+    elif shape == "mostly_empty_kernels":
+        K, N = 100_000, 30_000
+        tr = _csr_trace(shape, rng, K, N, (rng.random(K) < 0.1) * rng.integers(1, 12, size=K))
+    elif shape == "few_tensors_many_uses":
+        K, N = 20_000, 300
+        tr = _csr_trace(shape, rng, K, N, rng.integers(0, 11, size=K))
+    elif shape == "every_kernel_wide":
+        K, N = 600, 40_000
+        tr = _csr_trace(shape, rng, K, N, rng.integers(65, 400, size=K))
+    else:
+        K, N = 50_000, 3_000_000
+        tr = _csr_trace(shape, rng, K, N, rng.integers(0, 9, size=K))
+    tb = gpu.upload(tr)
+    check_vitality(gpu, oracle, tr, tb)
+    check_timeline(gpu, oracle, tr, tb)
+
+
 def test_inplace_relu_variant(gpu, oracle):
     tr = traces.config1_resnet152(inplace_relu=True)
     full_parity(gpu, oracle, tr)
