@@ -186,26 +186,6 @@ __device__ __forceinline__ int next_tile(unsigned *ticket)
     return s_tile;
 }
 
-// The kernel of trace event e (last k in [lo, hi] with kptr[k] <= e; lo is known to qualify), by a whole warp: every round probes 32 evenly spaced kernels at once, so that a cold search over a
-// million kernels costs four dependent round trips instead of twenty.  Result in every lane.
-__device__ __forceinline__ int kernel_of_event_warp(const int64_t *__restrict__ kptr, int lo, int hi, int64_t e, int lane)
-{
-    while (hi - lo > 31) {
-        const int step = (hi - lo) / 32 + 1;
-        const int probe = lo + lane * step;                   // lane 0 probes lo, which is known to qualify
-        const bool ok = probe <= hi && kptr[probe] <= e;
-        const unsigned m = __ballot_sync(0xffffffffu, ok);     // qualifying probes form a prefix of the lanes
-        const int last = 31 - __clz(m);
-        const int nlo = lo + last * step;
-        int nhi = nlo + step - 1;
-        if (nhi > hi) nhi = hi;
-        lo = nlo; hi = nhi;
-    }
-    const int probe = lo + lane;
-    const bool ok = probe <= hi && kptr[probe] <= e;
-    const unsigned m = __ballot_sync(0xffffffffu, ok);
-    return lo + (31 - __clz(m));
-}
 
 // ---------------------------------------------------------------------------------------------
 // Candidate geometry of one inactive period (Algorithm 1 / Section 4.4) for one destination.

@@ -213,9 +213,9 @@ cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t 
 }
 
 // =============================================================================================
-// Event passes.  An event is one (kernel, tensor) entry of the CSR.  Blocks take 2048 consecutive
-// events (128-bit loads); the kernel of an event is found by binary search in kernel_ptr, bracketed
-// once per block.
+// Event passes.  An event is one (kernel, tensor) entry of the CSR.  In the plain vitality kernels a
+// block takes 2048 consecutive events and finds the kernel of an event by binary search in kernel_ptr,
+// bracketed once per block; the first / last pass of the timeline call walks the events kernel by kernel.
 // =============================================================================================
 constexpr int kEvThreads = 256;
 constexpr int kEvItems = 8;
@@ -229,30 +229,6 @@ __device__ __forceinline__ int kernel_of_event(const int64_t *kptr, int lo, int 
         if (kptr[mid] <= e) lo = mid; else hi = mid - 1;
     }
     return lo;
-}
-
-// Stages kernel_ptr[lo .. hi + 1] of the block's event tile in shared memory when it fits, so that the
-// per-event searches run on chip.  Returns the pointer to search in and rebases lo / hi accordingly.
-constexpr int kPtrStage = 3072;
-__device__ __forceinline__ const int64_t *stage_kernel_ptr(const int64_t *__restrict__ kptr, int64_t K, int64_t base, int64_t E,
-                                                           int64_t *s_ptr, int *s_lohi, int *lo_out, int *hi_out, int *shift_out)
-{
-    if (threadIdx.x < 32) {                      // (32-ary search by warp 0: four dependent round trips for a million kernels)
-        const int64_t last = (base + kEvTile <= E ? base + kEvTile : E) - 1;
-        const int klo = kernel_of_event_warp(kptr, 0, (int)K - 1, base, (int)threadIdx.x);
-        const int khi = kernel_of_event_warp(kptr, klo, (int)K - 1, last, (int)threadIdx.x);
-        if (threadIdx.x == 0) { s_lohi[0] = klo; s_lohi[1] = khi; }
-    }
-    __syncthreads();
-    const int lo = s_lohi[0], hi = s_lohi[1];
-    if (hi - lo + 2 <= kPtrStage) {
-        for (int j = threadIdx.x; j <= hi - lo + 1; j += blockDim.x) s_ptr[j] = kptr[lo + j];
-        __syncthreads();
-        *lo_out = 0; *hi_out = hi - lo; *shift_out = lo;
-        return s_ptr;
-    }
-    *lo_out = lo; *hi_out = hi; *shift_out = 0;
-    return kptr;
 }
 
 // raw use count per tensor (a tensor listed twice by one kernel counts twice here; collapsed later)
