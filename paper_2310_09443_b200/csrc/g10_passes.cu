@@ -53,6 +53,7 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
     // Nothing later in a call reads the slot clock, so a kernel launched behind this one with programmatic stream
     // serialisation may start as soon as every block of this grid is running (no effect on ordinary launches).
     if (kind == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    else asm volatile("griddepcontrol.wait;" ::: "memory");   // (the difference array is complete; see k_diff_scatter)
     const int g = next_tile(ticket);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t seg = ((n + G - 1) / G + kSegChunk - 1) / kSegChunk * kSegChunk;
@@ -676,6 +677,9 @@ __global__ void __launch_bounds__(256) k_diff_scatter(int64_t N, int64_t K, cons
                                                       ull *__restrict__ diff, ull *status)
 {
     __shared__ long long s_part[8];
+    // (launched with programmatic stream serialisation: its blocks may be placed while the kernel before it drains;
+    // nothing is read before that kernel has finished and its writes are visible.  No effect on an ordinary launch.)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     long long gsum = 0;
     if (i < N) {
@@ -705,16 +709,32 @@ __global__ void __launch_bounds__(256) k_diff_scatter(int64_t N, int64_t K, cons
 cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
 {
+    // Both kernels are launched with programmatic stream serialisation and wait for their predecessor themselves
+    // (griddepcontrol.wait at their start): the launch and the placement of their blocks overlap its tail.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
     if (t.N > 0 && t.K > 0) {
-        const unsigned blocks = (unsigned)((t.N + 255) / 256);
-        if (encoded)
-            k_diff_scatter<true><<<blocks, 256, 0, s>>>(t.N, t.K, t.tensor_bytes, t.tensor_global, first_use, last_use, (ull *)w.diff, w.status);
-        else
-            k_diff_scatter<false><<<blocks, 256, 0, s>>>(t.N, t.K, t.tensor_bytes, t.tensor_global, first_use, last_use, (ull *)w.diff, w.status);
+        cfg.gridDim = dim3((unsigned)((t.N + 255) / 256));
+        cfg.blockDim = dim3(256);
+        const int64_t *bytes = t.tensor_bytes;
+        const uint8_t *glob = t.tensor_global;
+        ull *diff = (ull *)w.diff;
+        if (encoded) e = cudaLaunchKernelEx(&cfg, k_diff_scatter<true>, t.N, t.K, bytes, glob, first_use, last_use, diff, w.status);
+        else e = cudaLaunchKernelEx(&cfg, k_diff_scatter<false>, t.N, t.K, bytes, glob, first_use, last_use, diff, w.status);
+        if (e != cudaSuccess) return e;
     }
-    const int G = seg_scan_blocks(t.K);
-    k_seg_scan<1><<<G, kSegThreads, 0, s>>>(t.K, 0, w.diff, nullptr, pressure, w.pressure_scan.ticket, w.pressure_scan.done,
-                                          (ull *)w.pressure_scan.agg, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
+    cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
+    cfg.blockDim = dim3(kSegThreads);
+    e = cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)nullptr, pressure, w.pressure_scan.ticket,
+                           w.pressure_scan.done, (ull *)w.pressure_scan.agg, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 

@@ -229,6 +229,9 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
     int *s_off = s_cnt + bk_pad(B.nb);                      // [nb] global position of the tile's first key of the bucket minus its slot
     ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkKeyCap] keys of the tile in bucket order, the bucket in bits 48..59
     __shared__ int s_warp[2 * (kBkThreads / 32 + 1)];
+    // (launched with programmatic stream serialisation: the blocks are placed while k_bk_hist drains and wait here
+    // until it has finished and its counts are visible; no effect on an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (*(volatile ull *)B.status & G10_DEV_BAD_KERNEL_PTR) return;          // (found by k_bk_hist: nothing is partitioned)
 #ifdef G10_PHASE_CLOCKS
     __shared__ long long ph_acc[16];                     // (in shared memory: the register count stays that of the library build)
@@ -340,6 +343,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
     __shared__ int s_heavy[64];
     __shared__ long long s_pre[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.wait;" ::: "memory");             // (as in k_bk_scatter: the partition is complete)
     block_scan_counts(B.bucket_count, B.nb, s_base, s_scan);
     if (*(volatile ull *)B.status & G10_DEV_BAD_KERNEL_PTR) {      // nothing was partitioned: every tensor comes out unused
         for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_base[b] = 0;
@@ -600,6 +604,16 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     const int sms = current_sm_count();
     if (sms <= 0) return cudaErrorInvalidDevice;
     const int64_t tiles = (t.E + kBkTile - 1) / kBkTile;
+    // the second and third kernel are launched with programmatic stream serialisation (they wait for their
+    // predecessor themselves): launch and block placement overlap its tail
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kBkThreads);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
         k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
@@ -612,13 +626,19 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         const size_t sm2 = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8 + sizeof(ull) * kBkKeyCap;
         cudaError_t e = cudaFuncSetAttribute(k_bk_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
         if (e != cudaSuccess) return e;
-        k_bk_scatter<<<g2, kBkThreads, sm2, s>>>(B, t.kernel_ptr, t.kernel_tensors);
+        cfg.gridDim = dim3((unsigned)g2);
+        cfg.dynamicSmemBytes = sm2;
+        const int64_t *kp = t.kernel_ptr;
+        const int32_t *kt = t.kernel_tensors;
+        if ((e = cudaLaunchKernelEx(&cfg, k_bk_scatter, B, kp, kt)) != cudaSuccess) return e;
     }
     const size_t sm3 = sizeof(int) * (size_t)(bk_pad(B.nb) + 3 * bk_pad(B.bt) + kBkCap) + sizeof(unsigned short) * (size_t)B.bt;
     cudaError_t e = cudaFuncSetAttribute(k_bk_emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
     const int g3 = B.nb < 2 * sms ? B.nb : 2 * sms;
-    k_bk_emit<<<g3, kBkThreads, sm3, s>>>(B, out);
+    cfg.gridDim = dim3((unsigned)g3);
+    cfg.dynamicSmemBytes = sm3;
+    if ((e = cudaLaunchKernelEx(&cfg, k_bk_emit, B, out)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
