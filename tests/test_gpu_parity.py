@@ -342,11 +342,22 @@ def test_full_size_stress_dag_passes(gpu, oracle):
     plan = check_plan(gpu, tr, tb, cap, ref, max_iterations=1000)
     helpers.check_plan_invariants(tr, cap, start, P0, ov, gpu.migrations_numpy(plan), _np(plan.final_pressure),
                                   gpu.STATUS[int(plan.summary[2].item())], tr.host_bw, tr.ssd_bw, check_area=False)
+    # the characterisation statistics (Section 3) at the same size, from the vitality just checked
+    pn = int(v.counts[1].item())
+    st = gpu.g10_characterize(tr.K, tr.N, v.use_ptr, v.uses, tb.tensor_bytes, tl.kernel_start_ns, pn, v.period_tensor,
+                              v.period_prev_use, v.period_next_use, tr.host_bw, tr.ssd_bw)
+    torch.cuda.synchronize()
+    oc = oracle.characterize(tr.K, ov, tr.tensor_bytes, start, tr.host_bw, tr.ssd_bw)
+    assert np.array_equal(_np(st.active_bytes)[:tr.K], oc.active_bytes)
+    assert np.array_equal(_np(st.len_hist), oc.len_hist)
+    assert np.array_equal(_np(st.size_len_hist).reshape(41, 45), oc.size_len_hist)
+    assert np.array_equal(_np(st.hide), oc.hide) and np.array_equal(_np(st.summary), oc.summary)
 
 
 def test_full_size_stress_plan_digest(gpu):
-    """The complete plan of config 4 (13 505 migrations) against the digest of the CPU oracle's plan stored by
-    tests/golden/make_config4_plan_digest.py (the oracle needs about ten minutes for it)."""
+    """The complete plan of config 4 (13 505 migrations), the eager prefetch pass over it and the instruction stream
+    emitted from both, against the digests of the CPU oracle's results stored by
+    tests/golden/make_config4_plan_digest.py (the oracle needs about ten minutes for the plan)."""
     import hashlib, json, os
     import torch
     path = os.path.join(os.path.dirname(__file__), "golden", "config4_plan_digest.json")
@@ -377,6 +388,18 @@ def test_full_size_stress_plan_digest(gpu):
     for a in (_np(pf.order)[:n], _np(pf.new_absent_last)[:n], _np(pf.new_prefetch_issue_ns)[:n], _np(pf.pressure)[:tr.K], _np(pf.summary)):
         hp.update(np.ascontiguousarray(a).tobytes())
     assert hp.hexdigest() == gold["prefetch_sha256"]
+    # the instruction stream of that plan with the eager prefetch times (8 M records), field by field
+    v = gpu.g10_vitality(tb)
+    em = gpu.g10_emit_instructions(tr.K, tr.N, v.first_use, v.last_use, tb.tensor_bytes, tb.tensor_global, tl.kernel_start_ns,
+                                   n, plan.migrations, pf.new_prefetch_issue_ns)
+    torch.cuda.synchronize()
+    assert int(em.counts[1].item()) == 0 and int(em.counts[0].item()) == gold["num_instructions"]
+    got = gpu.instructions_numpy(em)
+    he = hashlib.sha256()
+    he.update(np.ascontiguousarray(_np(em.inst_ptr)).tobytes())
+    for name in gold["instruction_fields"]:
+        he.update(np.ascontiguousarray(got[name]).tobytes())
+    assert he.hexdigest() == gold["instructions_sha256"]
 
 
 def check_prefetch(gpu, oracle, tr, cap):
