@@ -4,8 +4,9 @@
 // Every instruction is one 64-bit key (boundary << 33 | opcode << 31 | tensor; unique) plus the plan record it
 // came from.  The keys are sorted with the same shape as the vitality pass: boundaries are cut into buckets of
 // consecutive boundaries holding a couple of thousand instructions, a histogram sizes the buckets, the keys are
-// scattered into their bucket's slice, and one block per bucket sorts its slice in shared memory (bitonic
-// network), counts the instructions of every boundary for the CSR pointers and writes the records out in order.
+// scattered into their bucket's slice, and one block per bucket sorts its slice in shared memory (counting sort by
+// boundary, then the few instructions of every boundary in key order by one thread; a boundary with more than 32
+// by a bitonic network), which also gives the CSR pointers, and writes the records out in order.
 // A bucket too large for shared memory (very many tensors allocated at one boundary) is sorted in global memory.
 #include "g10_device.cuh"
 #include "g10_internal.h"
@@ -139,20 +140,25 @@ __device__ void emit_bitonic(ull *k, int32_t *p, int n)
     }
 }
 
-__global__ void __launch_bounds__(kEmitThreads) k_emit_write(EmitArgs A, int64_t *inst_ptr, g10_instruction *inst, int64_t inst_cap, int64_t *counts)
+constexpr int kEmitRegs = kEmitCap / kEmitThreads;   // keys a thread keeps in registers between the two passes
+constexpr int kEmitWide = 32;                        // a boundary with more instructions is sorted by the whole block
+
+__global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int64_t *inst_ptr, g10_instruction *inst, int64_t inst_cap, int64_t *counts)
 {
     extern __shared__ long long s_dyn[];
     long long *s_base = s_dyn;                                   // [nb + 1]
-    int *s_cnt = (int *)(s_base + A.nb + 1);                     // [bw + 1] instructions per boundary of the bucket
-    ull *s_keys = (ull *)(((uintptr_t)(s_cnt + (1 << A.shift) + 1) + 7) & ~(uintptr_t)7);   // [kEmitCap]
+    int *s_cnt = (int *)(s_base + A.nb + 1);                     // [bw + 1] instructions per boundary of the bucket, then their offsets
+    int *s_cur = s_cnt + (1 << A.shift) + 1;                     // [bw] fill cursors
+    ull *s_keys = (ull *)(((uintptr_t)(s_cur + (1 << A.shift)) + 7) & ~(uintptr_t)7);   // [kEmitCap]
     int32_t *s_pay = (int32_t *)(s_keys + kEmitCap);              // [kEmitCap]
     __shared__ long long s_w[kEmitThreads / 32];
-    __shared__ int s_bucket;
+    __shared__ int s_bucket, s_nwide;
+    __shared__ int s_wide[64];
     const int bw = 1 << A.shift;
     emit_scan_buckets(A.bucket_count, A.nb, s_base, s_w);
     for (;;) {
         __syncthreads();
-        if (threadIdx.x == 0) s_bucket = (int)atomicAdd(A.ticket, 1u);
+        if (threadIdx.x == 0) { s_bucket = (int)atomicAdd(A.ticket, 1u); s_nwide = 0; }
         __syncthreads();
         const int b = s_bucket;
         if (b >= A.nb) break;
@@ -160,43 +166,104 @@ __global__ void __launch_bounds__(kEmitThreads) k_emit_write(EmitArgs A, int64_t
         const int n = (int)(s_base[b + 1] - base);
         ull *gk = A.keys + base;
         int32_t *gp = A.payload + base;
-        const ull *kp; const int32_t *pp;
-        if (n <= kEmitCap) {
-            for (int j = threadIdx.x; j < n; j += kEmitThreads) { s_keys[j] = gk[j]; s_pay[j] = gp[j]; }
-            __syncthreads();
-            emit_bitonic(s_keys, s_pay, n);
-            kp = s_keys; pp = s_pay;
-        } else {
-            __syncthreads();
-            emit_bitonic(gk, gp, n);
-            kp = gk; pp = gp;
-        }
-        // instructions per boundary -> CSR pointers of the bucket's boundaries
         const int64_t b0 = (int64_t)b << A.shift;
         const int bw_eff = (int)((A.K + 1 - b0) < bw ? (A.K + 1 - b0) : bw);
-        for (int j = threadIdx.x; j <= bw_eff; j += kEmitThreads) s_cnt[j] = 0;
+        for (int j = threadIdx.x; j <= bw_eff; j += kEmitThreads) { s_cnt[j] = 0; if (j < bw_eff) s_cur[j] = 0; }
         __syncthreads();
-        for (int j = threadIdx.x; j < n; j += kEmitThreads) atomicAdd(&s_cnt[(int)((kp[j] >> 33) - b0)], 1);
-        __syncthreads();
-        {   // in-place exclusive scan of s_cnt[0..bw_eff)
-            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-            int carry = 0;
-            for (int c0 = 0; c0 < bw_eff; c0 += kEmitThreads) {
-                const int j = c0 + threadIdx.x;
-                const int v = j < bw_eff ? s_cnt[j] : 0;
-                int incl = v;
+        const ull *kp; const int32_t *pp;
+        if (n <= kEmitCap) {
+            // Counting sort by boundary in shared memory (the keys stay in registers between the two passes), then
+            // every boundary's few instructions are put in key order by one thread; the keys are unique, so this is
+            // the order a sort of the whole bucket would give.
+            ull rk[kEmitRegs];
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+            for (int q = 0; q < kEmitRegs; ++q) {
+                const int j = q * kEmitThreads + threadIdx.x;
+                rk[q] = j < n ? gk[j] : ~0ull;
+            }
+#pragma unroll
+            for (int q = 0; q < kEmitRegs; ++q)
+                if (rk[q] != ~0ull) atomicAdd(&s_cnt[(int)((rk[q] >> 33) - b0)], 1);
+            __syncthreads();
+            {   // in-place exclusive scan of s_cnt[0..bw_eff), total in s_cnt[bw_eff]
+                const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+                int carry = 0;
+                for (int c0 = 0; c0 < bw_eff; c0 += kEmitThreads) {
+                    const int j = c0 + threadIdx.x;
+                    const int v = j < bw_eff ? s_cnt[j] : 0;
+                    int incl = v;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+                    __syncthreads();
+                    if (lane == 31) s_w[warp] = incl;
+                    __syncthreads();
+                    int wpre = 0, tot = 0;
+                    for (int w = 0; w < kEmitThreads / 32; ++w) { const int x = (int)s_w[w]; if (w < warp) wpre += x; tot += x; }
+                    if (j < bw_eff) s_cnt[j] = carry + wpre + incl - v;
+                    carry += tot;
+                }
                 __syncthreads();
-                if (lane == 31) s_w[warp] = incl;
+                if (threadIdx.x == 0) s_cnt[bw_eff] = carry;
                 __syncthreads();
-                int wpre = 0, tot = 0;
-                for (int w = 0; w < kEmitThreads / 32; ++w) { const int x = (int)s_w[w]; if (w < warp) wpre += x; tot += x; }
-                if (j < bw_eff) s_cnt[j] = carry + wpre + incl - v;
-                carry += tot;
+            }
+#pragma unroll
+            for (int q = 0; q < kEmitRegs; ++q)
+                if (rk[q] != ~0ull) {
+                    const int j = q * kEmitThreads + threadIdx.x;
+                    const int bd = (int)((rk[q] >> 33) - b0);
+                    const int slot = s_cnt[bd] + atomicAdd(&s_cur[bd], 1);
+                    s_keys[slot] = rk[q];
+                    s_pay[slot] = gp[j];
+                }
+            __syncthreads();
+            for (int bd = threadIdx.x; bd < bw_eff; bd += kEmitThreads) {
+                const int o = s_cnt[bd], m = s_cnt[bd + 1] - o;
+                if (m > kEmitWide) { const int q = atomicAdd(&s_nwide, 1); if (q < 64) s_wide[q] = bd; }
+                else {
+                    for (int a = 1; a < m; ++a) {
+                        const ull x = s_keys[o + a];
+                        const int32_t px = s_pay[o + a];
+                        int c = a - 1;
+                        while (c >= 0 && s_keys[o + c] > x) { s_keys[o + c + 1] = s_keys[o + c]; s_pay[o + c + 1] = s_pay[o + c]; --c; }
+                        s_keys[o + c + 1] = x; s_pay[o + c + 1] = px;
+                    }
+                }
             }
             __syncthreads();
+            const int nwide = s_nwide;
+            for (int hq = 0; hq < (nwide <= 64 ? nwide : bw_eff); ++hq) {
+                const int bd = nwide <= 64 ? s_wide[hq] : hq;
+                const int o = s_cnt[bd], m = s_cnt[bd + 1] - o;
+                if (m <= kEmitWide) continue;                      // (only when the list overflowed: uniform test)
+                emit_bitonic(s_keys + o, s_pay + o, m);
+            }
+            kp = s_keys; pp = s_pay;
+        } else {
+            emit_bitonic(gk, gp, n);
+            for (int j = threadIdx.x; j < n; j += kEmitThreads) atomicAdd(&s_cnt[(int)((gk[j] >> 33) - b0)], 1);
+            __syncthreads();
+            {   // in-place exclusive scan of s_cnt[0..bw_eff)
+                const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+                int carry = 0;
+                for (int c0 = 0; c0 < bw_eff; c0 += kEmitThreads) {
+                    const int j = c0 + threadIdx.x;
+                    const int v = j < bw_eff ? s_cnt[j] : 0;
+                    int incl = v;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+                    __syncthreads();
+                    if (lane == 31) s_w[warp] = incl;
+                    __syncthreads();
+                    int wpre = 0, tot = 0;
+                    for (int w = 0; w < kEmitThreads / 32; ++w) { const int x = (int)s_w[w]; if (w < warp) wpre += x; tot += x; }
+                    if (j < bw_eff) s_cnt[j] = carry + wpre + incl - v;
+                    carry += tot;
+                }
+                __syncthreads();
+            }
+            kp = gk; pp = gp;
         }
+        // CSR pointers of the bucket's boundaries
         for (int j = threadIdx.x; j < bw_eff; j += kEmitThreads) inst_ptr[b0 + j] = base + s_cnt[j];
         if (b == A.nb - 1 && threadIdx.x == 0) {
             inst_ptr[A.K + 1] = s_base[A.nb];
@@ -252,7 +319,7 @@ cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s)
     if (g < 1) g = 1;
     k_emit_hist<<<(int)g, kEmitThreads, sizeof(unsigned) * (size_t)A.nb, s>>>(A);
     k_emit_scatter<<<(int)g, kEmitThreads, sizeof(long long) * (size_t)(A.nb + 1), s>>>(A);
-    const size_t sm3 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(int) * (size_t)((1 << A.shift) + 2) + 8 +
+    const size_t sm3 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(int) * (size_t)(2 * (1 << A.shift) + 2) + 8 +
                        (sizeof(ull) + sizeof(int32_t)) * kEmitCap;
     cudaError_t e = cudaFuncSetAttribute(k_emit_write, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
