@@ -4,8 +4,8 @@
 //
 // The pass is a strict sequence over the plan records (each move changes the pressure the next search sees), so
 // one block does it: the records are ordered by a bitonic network over their indices, then, record by record, the
-// block searches backward in chunks of its own width (a chunk stops the search as soon as one of its slots cannot
-// take the tensor) and adds the tensor's size to the slots it regained.  Parallelism is inside each search.
+// block searches backward in chunks of eight times its own width (a chunk stops the search as soon as one of its
+// slots cannot take the tensor) and adds the tensor's size to the slots it regained.  Parallelism is inside each search.
 #include "g10_device.cuh"
 #include "g10_internal.h"
 
@@ -15,6 +15,7 @@ namespace g10 {
 #define G10_PF_THREADS 256
 #endif
 constexpr int kPfThreads = G10_PF_THREADS;       // a block-wide barrier per search chunk and per record: few warps keep it cheap
+constexpr int kPfRows = 8;                       // slots a thread looks at per search chunk
 
 __device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y)
 {
@@ -28,7 +29,7 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
                                                                   int64_t *new_issue, int64_t *summary, int p_in_smem, int sort_in_smem)
 {
     extern __shared__ long long s_dyn[];   // the pressure curve, when the launch gave it room
-    __shared__ int s_wstop[2][kPfThreads / 32];   // per warp: highest slot of the current chunk that cannot take the tensor (-1: none);
+    __shared__ int s_wstop[2][kPfThreads / 32];   // per warp: smallest offset below hi of a slot of the current chunk that cannot take the tensor;
                                                   // two copies used in turn, so that one barrier per chunk is enough
     __shared__ int s_ra[kPfThreads], s_rb[kPfThreads], s_rj[kPfThreads];
     __shared__ long long s_rs[kPfThreads];
@@ -108,21 +109,42 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
             int hi = b_abs;                     // slots (j, b_abs] are known to take the tensor
             int j = a_abs - 1;                  // result: last slot that stays absent
             while (hi >= a_abs) {
-                const int lo = hi - kPfThreads + 1 > a_abs ? hi - kPfThreads + 1 : a_abs;
-                // threads look at slots hi, hi - 1, ...: the first failing lane of the first failing warp is the highest slot
-                const int k = hi - (int)threadIdx.x;
-                const unsigned fail = __ballot_sync(0xffffffffu, k >= lo && Pw[k] > cap - s);
-                if (lane == 0) s_wstop[turn][warp] = fail ? hi - (warp * 32 + __ffs(fail) - 1) : -1;
+                // a chunk of kPfRows rows of kPfThreads slots, from hi downwards: row r, thread t looks at slot
+                // hi - (r * kPfThreads + t); all loads of a thread are in flight together.  The highest slot that
+                // cannot take the tensor is the failing one with the smallest offset r * kPfThreads + t.
+                const int span = hi - a_abs + 1;                     // slots still to look at
+                int first = 0x7fffffff;                             // this warp's smallest failing offset
+                long long pv[kPfRows];
+#pragma unroll
+                for (int r = 0; r < kPfRows; ++r) {
+                    const int off = r * kPfThreads + (int)threadIdx.x;
+                    pv[r] = off < span ? Pw[hi - off] : 0;
+                }
+#pragma unroll
+                for (int r = 0; r < kPfRows; ++r) {
+                    const int off = r * kPfThreads + (int)threadIdx.x;
+                    const unsigned fail = __ballot_sync(0xffffffffu, off < span && pv[r] > cap - s);
+                    if (fail && first == 0x7fffffff) first = r * kPfThreads + warp * 32 + __ffs(fail) - 1;
+                }
+                if (lane == 0) s_wstop[turn][warp] = first;
                 __syncthreads();
-                int stop = -1;
-                const int mine = lane < kPfThreads / 32 ? s_wstop[turn][lane] : -1;      // one warp result per lane
-                const unsigned any = __ballot_sync(0xffffffffu, mine >= 0);
-                if (any) stop = __shfl_sync(0xffffffffu, mine, __ffs(any) - 1);
+                const int mine = lane < kPfThreads / 32 ? s_wstop[turn][lane] : 0x7fffffff;      // one warp result per lane
+                const int best = (int)__reduce_min_sync(0xffffffffu, (unsigned)mine);
                 turn ^= 1;                                                   // (the other copy was last read two barriers ago)
-                if (stop >= 0) { j = stop; break; }
-                hi = lo - 1;
+                if (best != 0x7fffffff) { j = hi - best; break; }
+                hi -= kPfRows * kPfThreads;
             }
-            for (int k = j + 1 + (int)threadIdx.x; k <= b_abs; k += kPfThreads) Pw[k] += s;
+            {   // the regained slots take the tensor back: read-modify-write, eight per thread in flight
+                const int k0 = j + 1 + (int)threadIdx.x;
+#pragma unroll 1
+                for (int k = k0; k <= b_abs; k += 8 * kPfThreads) {
+                    long long v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = k + u * kPfThreads <= b_abs ? Pw[k + u * kPfThreads] : 0;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) if (k + u * kPfThreads <= b_abs) Pw[k + u * kPfThreads] = v[u] + s;
+                }
+            }
             if (threadIdx.x == 0) s_rj[q] = j;
             if (j < b_abs) { moved += 1; regained += b_abs - j; }
             __syncthreads();
