@@ -11,10 +11,8 @@
 
 namespace g10 {
 
-#ifndef G10_PF_THREADS
-#define G10_PF_THREADS 256
-#endif
-constexpr int kPfThreads = G10_PF_THREADS;       // a block-wide barrier per search chunk and per record: few warps keep it cheap
+// kPfThreads (template parameter): 256 for a timeline that fits shared memory (a block-wide barrier per search chunk
+// and per record: few warps keep it cheap), 1024 for a long one in global memory (its ranges are long: width pays)
 constexpr int kPfRows = 8;                       // slots a thread looks at per search chunk
 
 __device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y)
@@ -23,6 +21,7 @@ __device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y
     return kx < ky || (kx == ky && x < y);
 }
 
+template <int kPfThreads>
 __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int64_t n, const g10_migration *__restrict__ mig,
                                                                   const int64_t *__restrict__ start, const int64_t *__restrict__ bytes,
                                                                   int64_t cap, int64_t *P, int32_t *order, int32_t *new_last,
@@ -187,7 +186,6 @@ cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *
 {
     const int64_t cap = gpu_capacity_bytes >= ((uint64_t)1 << 63) ? INT64_MAX : (int64_t)gpu_capacity_bytes;
     // the pressure curve in shared memory if it fits beside the kernel's own arrays
-    static_assert(kPfThreads / 32 <= 32, "one warp result per lane");
     size_t dyn = 0;
     int in_smem = 0;
     if (K > 0 && (size_t)K * 8 <= 120 * 1024) { dyn = (size_t)K * 8; in_smem = 1; }
@@ -195,11 +193,19 @@ cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *
     while (n2 < n) n2 <<= 1;
     int sort_smem = 0;
     if (n > 0 && (size_t)n2 * 12 <= 64 * 1024) { dyn += (size_t)n2 * 12; sort_smem = 1; }
-    if (dyn > 0) {
-        const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
-        if (e != cudaSuccess) return e;
+    if (in_smem) {
+        if (dyn > 0) {
+            const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+            if (e != cudaSuccess) return e;
+        }
+        k_schedule_prefetch<256><<<1, 256, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem);
+    } else {
+        if (dyn > 0) {
+            const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+            if (e != cudaSuccess) return e;
+        }
+        k_schedule_prefetch<1024><<<1, 1024, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem);
     }
-    k_schedule_prefetch<<<1, kPfThreads, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem);
     return cudaGetLastError();
 }
 
