@@ -243,26 +243,26 @@ __device__ __forceinline__ bool grid_barrier(GridBarrier *b, unsigned nblocks, u
     __shared__ unsigned s_ok;
     __syncthreads();
     if (threadIdx.x == 0) {
+        // (no look at the error word before arriving: a block that arrives after another one gave up finds the word
+        // set at its next check while polling, which costs one round trip less on every barrier that succeeds)
         unsigned ok = 1u;
-        if (ld_acquire_u32(&b->error)) ok = 0u;
-        else {
-            __threadfence();
-            unsigned arrived = atomicAdd(&b->count, 1u);
-            if (arrived == nblocks - 1u) {
-                b->count = 0u;
-                __threadfence();
-                st_release_u32(&b->gen, my_gen + 1u);
-            } else {
-                ull t0 = global_timer_ns();
-                unsigned polls = 0;
-                while (ld_acquire_u32(&b->gen) == my_gen) {
-                    if ((++polls & 1023u) == 0u) {
-                        if (ld_acquire_u32(&b->error)) { ok = 0u; break; }
-                        if (global_timer_ns() - t0 > kBarrierTimeoutNs) { atomicExch(&b->error, 1u); ok = 0u; break; }
-                    }
+        // arrival is an acquire-release add (it publishes this block's writes, ordered before it by the block barrier
+        // above, and the last arrival has acquired everyone's); the generation is stored with release and polled with
+        // acquire: no separate fences
+        unsigned arrived;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(&b->count) : "memory");
+        if (arrived == nblocks - 1u) {
+            b->count = 0u;
+            st_release_u32(&b->gen, my_gen + 1u);
+        } else {
+            ull t0 = global_timer_ns();
+            unsigned polls = 0;
+            while (ld_acquire_u32(&b->gen) == my_gen) {
+                if ((++polls & 1023u) == 0u) {
+                    if (ld_acquire_u32(&b->error)) { ok = 0u; break; }
+                    if (global_timer_ns() - t0 > kBarrierTimeoutNs) { atomicExch(&b->error, 1u); ok = 0u; break; }
                 }
             }
-            __threadfence();
         }
         s_ok = ok;
     }
