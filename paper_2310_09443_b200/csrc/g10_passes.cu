@@ -162,12 +162,13 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
             if (s_sl[w] >= 0 && (sl < 0 || s_w[w] > mx || (s_w[w] == mx && s_sl[w] < sl))) { mx = s_w[w]; sl = s_sl[w]; }
         blk_max[g] = mx;
         blk_slot[g] = sl;
-        __threadfence();
-        s_last = (atomicAdd(done, 1u) == (unsigned)G - 1u);
+        // (acquire-release add: publishes this block's result; the last block to arrive has acquired everyone's)
+        unsigned arrived;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(done) : "memory");
+        s_last = (arrived == (unsigned)G - 1u);
     }
     __syncthreads();
     if (s_last) {
-        __threadfence();
         long long bm = 0;
         int bs = -1;
         for (int t = threadIdx.x; t < G; t += kSegThreads) {
