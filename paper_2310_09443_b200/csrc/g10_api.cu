@@ -60,6 +60,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.bk_cursor = c.take<unsigned>(4096);
     w.bk_words = c.take<ull>(2 * 4096);
     w.xwords = c.take<ull>((2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16);
+    w.tl_words = c.take<ull>(2 * kTlMaxBlocks);
     w.zero_bytes = align_up(c.off);
     // arrays that must start at zero, cleared only by the calls that use them (the difference array sits right behind
     // the zero-initialised region, so that one memset covers both)
@@ -77,6 +78,9 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.heavy_info = c.take<int32_t>(2 * heavy);
     w.tile_max = c.take<int64_t>((size_t)ktiles);
     w.tile_slot = c.take<int32_t>((size_t)ktiles);
+    w.tl_pair = c.take<int>(2 * N);
+    w.tl_blk_max = c.take<int64_t>(kTlMaxBlocks);
+    w.tl_blk_slot = c.take<int32_t>(kTlMaxBlocks);
     w.first_use = c.take<int32_t>(N);
     w.last_use = c.take<int32_t>(N);
     w.num_uses = c.take<int32_t>(N);
@@ -314,7 +318,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(trace, ws, w, d, s, kZeroDiff);
+    rc = begin_call(trace, ws, w, d, s, 0);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     int64_t *start = host ? w.start : out->kernel_start_ns;
@@ -322,8 +326,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     int64_t *pk = host ? w.peak_bytes : out->peak_bytes;
     int32_t *ps = host ? w.peak_slot : out->peak_slot;
     int64_t *st = host ? w.counts + 2 : out->status;
-    CU(launch_clock_and_first_last(d, w, start, w.first_use, w.last_use, s));
-    CU(launch_pressure(d, w, w.first_use, w.last_use, true, P, pk, ps, s));
+    CU(launch_timeline(d, w, start, P, pk, ps, s));
     CU(launch_publish_status(w, st, s));
     if (host) {
         CU(d2h(out->kernel_start_ns, w.start, (size_t)d.K + 1, s));

@@ -27,7 +27,6 @@ constexpr int kBkItems = 8;
 constexpr int kBkTile = kBkThreads * kBkItems;     // events per partition tile (4096)
 constexpr int kBkCap = 10240;                      // events of a bucket kept in shared memory
 constexpr int kBkWide = 64;                        // a kernel with more events is walked by its whole warp in the partition
-constexpr int kBkKeyCap = 6144;                    // keys of one partition tile staged in shared memory
 constexpr int kBkHeavy = 32;                       // longer segments are sorted by the whole block
 
 struct BucketArgs {
@@ -35,7 +34,8 @@ struct BucketArgs {
     int shift;                 // log2(bt)
     int bt;                    // tensors per bucket
     int nb;                    // number of buckets
-    int tile_kernels;          // kernels per partition tile (a multiple of kBkThreads)
+    int tile_kernels;          // kernels per partition tile (at most 32768)
+    int tile_cap;              // events of a tile that go through shared memory in one round (a multiple of kBkThreads)
     unsigned *bucket_count;    // [nb] events per bucket
     unsigned *bucket_cursor;   // [nb] scatter cursors (start at zero)
     ull *pairs;                // [E] keys, bucket after bucket
@@ -167,99 +167,81 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
 // ---------------------------------------------------------------------------------------------
 // 2. partition the events by bucket
 // ---------------------------------------------------------------------------------------------
-// One sweep of a tile's kernels over the events [eb, ee): a warp takes 32 consecutive kernels, every lane walks the
-// events of its own kernel (so the kernel of an event is known without a search); a kernel with more than
-// kBkWide events is walked by the whole warp instead.
-// kPlace false: count the events of every bucket.  true: s_cnt[b] is the next free slot of bucket b in the tile's
-// staging area; the key goes there with its bucket in the spare upper bits.
-template <bool kPlace>
-__device__ __forceinline__ void bk_take(const BucketArgs &B, int32_t i, int64_t k, int *s_cnt, ull *s_key)
-{
-    if (i < 0 || i >= B.N) return;
-    const int b = i >> B.shift;
-    if (!kPlace) atomicAdd(&s_cnt[b], 1);
-    else {
-        const int slot = atomicAdd(&s_cnt[b], 1);
-        if (slot < kBkKeyCap) {
-            s_key[slot] = ((ull)(unsigned)b << 48) | ((ull)(unsigned)(i & (B.bt - 1)) << 32) | (unsigned)k;
-        }
-    }
-}
+// A tile is a run of consecutive kernels; its events [T0, T1) go through the block in rounds of at most B.tile_cap.
+// Per round: (a) the kernels of the tile write their number (relative to the tile) over the positions of their
+// events in shared memory -- a lane per kernel, a whole warp for a kernel with more than kBkWide events; stores
+// only, nothing is loaded inside the walk; (b) the events are read coalesced, each looks its kernel up at its own
+// position and takes its rank inside (round, bucket) from a shared-memory counter; ids and ranks stay in
+// registers; (c) the counters are scanned and the round's room in every bucket it touches is reserved with one
+// global atomic per bucket; (d) the keys are staged in bucket order in shared memory and (e) written out in
+// coalesced runs.
+constexpr int kPtMaxItems = 16;                     // events per thread and round, at most (tile_cap <= 16 * kBkThreads)
 
-template <bool kPlace>
-__device__ __forceinline__ void bk_walk(const BucketArgs &B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt, int64_t tk0,
-                                        int64_t tk1, int64_t eb, int64_t ee, int *s_cnt, ull *s_key)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll 1
-    for (int64_t k0 = tk0 + warp * 32; k0 < tk1; k0 += kBkThreads) {
-        const int64_t k = k0 + lane;
-        int64_t a = kptr[k < B.K ? k : B.K];                       // lanes past the last kernel hold kernel_ptr[K] = E: no events
-        int64_t b = kptr[k + 1 < B.K ? k + 1 : B.K];
-        a = a > eb ? a : eb;
-        b = b < ee ? b : ee;
-        const bool wide = b - a > kBkWide;
-        if (!wide) {
-#pragma unroll 1
-            for (int64_t e = a; e < b; e += 4) {                   // four events of this lane's kernel at a time
-                int32_t id[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) id[u] = e + u < b ? kt[e + u] : -1;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) bk_take<kPlace>(B, id[u], k, s_cnt, s_key);
-            }
-        }
-        unsigned m = __ballot_sync(0xffffffffu, wide);
-#pragma unroll 1
-        while (m) {
-            const int src = __ffs(m) - 1;
-            m &= m - 1;
-            const int64_t wa = __shfl_sync(0xffffffffu, a, src), wb = __shfl_sync(0xffffffffu, b, src);
-#pragma unroll 1
-            for (int64_t e = wa + lane; e < wb; e += 32) bk_take<kPlace>(B, kt[e], k0 + src, s_cnt, s_key);
-        }
-    }
-}
-
-__global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
+__global__ void __launch_bounds__(kBkThreads, 2) k_bk_scatter(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
 {
     extern __shared__ __align__(16) int s_mem[];
     int *s_base = s_mem;                                   // [nb + 1] first key of each bucket
-    int *s_cnt = s_base + bk_pad(B.nb);                      // [nb + 1] events of this tile per bucket, then their scan, then fill cursors
-    int *s_off = s_cnt + bk_pad(B.nb);                      // [nb] global position of the tile's first key of the bucket minus its slot
-    ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [kBkKeyCap] keys of the tile in bucket order, the bucket in bits 48..59
+    int *s_cnt = s_base + bk_pad(B.nb);                      // [nb + 1] events of this round per bucket, then their scan
+    int *s_off = s_cnt + bk_pad(B.nb);                      // [nb] global position of the round's first key of the bucket minus its slot
+    ull *s_key = (ull *)(((uintptr_t)(s_off + B.nb) + 7) & ~(uintptr_t)7);   // [tile_cap] keys of the round in bucket order, the bucket in bits 48..59
+    unsigned short *s_krel = (unsigned short *)(s_key + B.tile_cap);         // [tile_cap] kernel of every event of the round, relative to the tile
     __shared__ int s_warp[2 * (kBkThreads / 32 + 1)];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // (launched with programmatic stream serialisation: the blocks are placed while k_bk_hist drains and wait here
     // until it has finished and its counts are visible; no effect on an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (*(volatile ull *)B.status & G10_DEV_BAD_KERNEL_PTR) return;          // (found by k_bk_hist: nothing is partitioned)
-#ifdef G10_PHASE_CLOCKS
-    __shared__ long long ph_acc[16];                     // (in shared memory: the register count stays that of the library build)
-    if (threadIdx.x == 0) { for (int i = 0; i < 15; ++i) ph_acc[i] = 0; ph_acc[15] = clock64(); }
-    int ph_n = 0;
-#endif
     block_scan_counts(B.bucket_count, B.nb, s_base, s_warp);
-    BK_CLOCK(0);
     const int64_t TK = B.tile_kernels;
     const int64_t tiles = (B.K + TK - 1) / TK;
+    const int cap = B.tile_cap;
 #pragma unroll 1
     for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         const int64_t tk0 = tile * TK, tk1 = tk0 + TK < B.K ? tk0 + TK : B.K;
         const int64_t T0 = kptr[tk0], T1 = kptr[tk1];
-        // (a tile with more events than the staging area holds goes through it in several rounds)
 #pragma unroll 1
-        for (int64_t eb = T0; eb < T1; eb += kBkKeyCap) {
-#ifdef G10_PHASE_CLOCKS
-            ++ph_n;
-#endif
-            const int64_t ee = eb + kBkKeyCap < T1 ? eb + kBkKeyCap : T1;
+        for (int64_t eb = T0; eb < T1; eb += cap) {
+            const int64_t ee = eb + cap < T1 ? eb + cap : T1;
+            const int n_round = (int)(ee - eb);
             for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_cnt[b] = 0;
+            // (a) kernel of every event of the round
+#pragma unroll 1
+            for (int64_t k0 = tk0 + warp * 32; k0 < tk1; k0 += kBkThreads) {
+                const int64_t k = k0 + lane;
+                int64_t a = kptr[k < tk1 ? k : tk1], b = kptr[k + 1 < tk1 ? k + 1 : tk1];
+                a = a > eb ? a : eb; a = a < ee ? a : ee;
+                b = b > eb ? b : eb; b = b < ee ? b : ee;
+                const bool wide = b - a > kBkWide;
+                const unsigned short rel = (unsigned short)(k - tk0);
+                if (!wide)
+                    for (int p = (int)(a - eb), q = (int)(b - eb); p < q; ++p) s_krel[p] = rel;
+                unsigned m = __ballot_sync(0xffffffffu, wide);
+#pragma unroll 1
+                while (m) {
+                    const int src = __ffs(m) - 1;
+                    m &= m - 1;
+                    const int wa = (int)(__shfl_sync(0xffffffffu, a, src) - eb), wb = (int)(__shfl_sync(0xffffffffu, b, src) - eb);
+                    const unsigned short wrel = (unsigned short)(k0 + src - tk0);
+                    for (int p = wa + lane; p < wb; p += 32) s_krel[p] = wrel;
+                }
+            }
             __syncthreads();
-            BK_CLOCK(1);
-            bk_walk<false>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key);
+            // (b) events, coalesced: bucket and rank inside (round, bucket)
+            int32_t id[kPtMaxItems];
+            int rank[kPtMaxItems];
+#pragma unroll
+            for (int j = 0; j < kPtMaxItems; ++j) {
+                const int p = j * kBkThreads + threadIdx.x;
+                id[j] = p < n_round ? kt[eb + p] : -1;
+            }
+#pragma unroll
+            for (int j = 0; j < kPtMaxItems; ++j) {
+                rank[j] = 0;
+                if (id[j] >= 0 && id[j] < B.N) rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1);
+                else id[j] = -1;
+            }
             __syncthreads();
-            BK_CLOCK(2);
-            // reserve this tile's room in every bucket it touches, then turn the tile counts into tile offsets
+            // (c) reserve this round's room in every bucket it touches, then turn the counts into offsets inside the round
             // (the global cursors answer while the block scans: their results stay in registers until after the scan)
             int cur[8];                                            // nb <= 4096 = 8 * kBkThreads
 #pragma unroll
@@ -267,32 +249,33 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_scatter(BucketArgs B, const i
                 const int b = j * kBkThreads + threadIdx.x;
                 cur[j] = (b < B.nb && s_cnt[b]) ? (int)atomicAdd(&B.bucket_cursor[b], (unsigned)s_cnt[b]) : 0;
             }
-            block_scan_counts((const unsigned *)s_cnt, B.nb, s_cnt, s_warp);      // in place: s_cnt[b] = first slot of bucket b in the tile
-            BK_CLOCK(3);
+            block_scan_counts((const unsigned *)s_cnt, B.nb, s_cnt, s_warp);      // in place: s_cnt[b] = first slot of bucket b in the round
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int b = j * kBkThreads + threadIdx.x;
                 if (b < B.nb) s_off[b] = cur[j] + s_base[b] - s_cnt[b];
             }
+            // (d) keys in bucket order
+#pragma unroll
+            for (int j = 0; j < kPtMaxItems; ++j) {
+                if (id[j] >= 0) {
+                    const int p = j * kBkThreads + threadIdx.x;
+                    const int b = id[j] >> B.shift;
+                    const unsigned k = (unsigned)(tk0 + s_krel[p]);
+                    s_key[s_cnt[b] + rank[j]] = ((ull)(unsigned)b << 48) | ((ull)(unsigned)(id[j] & (B.bt - 1)) << 32) | k;
+                }
+            }
             __syncthreads();
-            bk_walk<true>(B, kptr, kt, tk0, tk1, eb, ee, s_cnt, s_key);
-            __syncthreads();
-            BK_CLOCK(4);
-            const int n_valid = s_cnt[B.nb] < kBkKeyCap ? s_cnt[B.nb] : kBkKeyCap;
+            // (e) out, coalesced
+            const int n_valid = s_cnt[B.nb];
             for (int slot = threadIdx.x; slot < n_valid; slot += kBkThreads) {
                 const ull key = s_key[slot];                       // bits 48..59: the bucket (staging only)
                 const int64_t pos = (int64_t)s_off[(int)(key >> 48)] + slot;
                 if (pos >= 0 && pos < B.E) B.pairs[pos] = key & 0x0000ffffffffffffull;
             }
             __syncthreads();
-            BK_CLOCK(5);
         }
     }
-#ifdef G10_PHASE_CLOCKS
-    if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 100) && ph_n > 0)
-        printf("k_bk_scatter block %d (%d rounds): setup %lld; cycles/round: zero %lld count %lld cursors+scan %lld place %lld write %lld\n",
-               blockIdx.x, ph_n, ph_acc[0], ph_acc[1] / ph_n, ph_acc[2] / ph_n, ph_acc[3] / ph_n, ph_acc[4] / ph_n, ph_acc[5] / ph_n);
-#endif
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -597,7 +580,7 @@ bool vitality_buckets_supported(int64_t N, int64_t E)
 cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s)
 {
     BucketArgs B;
-    B.N = t.N; B.E = t.E; B.K = t.K; B.tile_kernels = kBkThreads;
+    B.N = t.N; B.E = t.E; B.K = t.K; B.tile_kernels = kBkThreads; B.tile_cap = kBkThreads;
     if (!choose_buckets(t.N, t.E, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
     B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
     B.ticket = w.emit_scan.ticket; B.status = w.status; B.spill = w.raw_uses;
@@ -617,13 +600,24 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
         k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
-        // kernels per partition tile: as many as fill the staging area on average, in steps of one sweep of the block
-        int64_t sweeps = ((int64_t)kBkKeyCap * t.K) / (t.E * kBkThreads);
-        sweeps = sweeps < 1 ? 1 : (sweeps > 8 ? 8 : sweeps);
-        B.tile_kernels = (int)(sweeps * kBkThreads);
-        const int64_t ktiles = (t.K + B.tile_kernels - 1) / B.tile_kernels;
-        const int g2 = (int)(ktiles < 3 * (int64_t)sms ? ktiles : 3 * (int64_t)sms);
-        const size_t sm2 = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8 + sizeof(ull) * kBkKeyCap;
+        // Shared memory of the partition kernel: three bucket tables and ten bytes per staged event; two blocks per SM.
+        const size_t tables = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8;
+        int64_t cap = ((int64_t)(100 << 10) - (int64_t)tables) / 10 / kBkThreads * kBkThreads;
+        cap = cap < kBkThreads ? kBkThreads : (cap > (int64_t)kPtMaxItems * kBkThreads ? (int64_t)kPtMaxItems * kBkThreads : cap);
+        B.tile_cap = (int)cap;
+        // Kernels per tile: as many as fill nine tenths of a round on average (so that few tiles need a second round),
+        // then evened out so that every block of the grid gets the same number of tiles.
+        const int g2max = 2 * sms;
+        int64_t tk = (cap * 9 / 10) * t.K / t.E;
+        tk = tk < 32 ? 32 : (tk > 32768 ? 32768 : tk);
+        const int64_t per_block = (t.K + tk * g2max - 1) / (tk * g2max);
+        tk = (t.K + per_block * g2max - 1) / (per_block * g2max);
+        tk = (tk + 31) / 32 * 32;
+        tk = tk > 32768 ? 32768 : tk;
+        B.tile_kernels = (int)tk;
+        const int64_t ktiles = (t.K + tk - 1) / tk;
+        const int g2 = (int)(ktiles < g2max ? ktiles : g2max);
+        const size_t sm2 = tables + (sizeof(ull) + sizeof(unsigned short)) * (size_t)cap;
         cudaError_t e = cudaFuncSetAttribute(k_bk_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
         if (e != cudaSuccess) return e;
         cfg.gridDim = dim3((unsigned)g2);
