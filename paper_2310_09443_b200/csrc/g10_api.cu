@@ -60,11 +60,14 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.bk_cursor = c.take<unsigned>(4096);
     w.bk_words = c.take<ull>(2 * 4096);
     w.xwords = c.take<ull>((2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16);
-    w.tl_words = c.take<ull>(2 * kTlMaxBlocks);
+    w.seg_words = c.take<ull>(512 * 16);
+    w.seg_words2 = c.take<ull>(512 * 16);
     w.zero_bytes = align_up(c.off);
     // arrays that must start at zero, cleared only by the calls that use them (the difference array sits right behind
     // the zero-initialised region, so that one memset covers both)
     w.diff = c.take<int64_t>(K + 1);
+    w.tl_point = c.take<int64_t>(K);
+    w.tl_pair = c.take<int>(2 * N);           // (both right behind the difference array: the timeline call clears both with the same memset)
     w.cnt = c.take<int32_t>(N);
     const size_t state_begin = align_up(c.off);
     w.busy = c.take<int64_t>(4 * K);       // busy, hocc and dead are contiguous: one memset
@@ -78,9 +81,6 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.heavy_info = c.take<int32_t>(2 * heavy);
     w.tile_max = c.take<int64_t>((size_t)ktiles);
     w.tile_slot = c.take<int32_t>((size_t)ktiles);
-    w.tl_pair = c.take<int>(2 * N);
-    w.tl_blk_max = c.take<int64_t>(kTlMaxBlocks);
-    w.tl_blk_slot = c.take<int32_t>(kTlMaxBlocks);
     w.first_use = c.take<int32_t>(N);
     w.last_use = c.take<int32_t>(N);
     w.num_uses = c.take<int32_t>(N);
@@ -160,7 +160,7 @@ int32_t check_ws(int32_t which, const g10_trace *t, void *ws, size_t ws_bytes)
     } while (0)
 
 // Prepares the workspace and returns the device view of the trace (staging it first in host mode).
-enum { kZeroCounts = 1, kZeroDiff = 2, kZeroState = 4 };
+enum { kZeroCounts = 1, kZeroDiff = 2, kZeroState = 4, kZeroPairs = 8 };
 
 int32_t begin_call(const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, cudaStream_t s, int zero_mask)
 {
@@ -169,6 +169,7 @@ int32_t begin_call(const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, c
     {
         size_t head = w.zero_bytes;
         if (zero_mask & kZeroDiff) head = (size_t)((char *)(w.diff + z.K + 1) - w.zero_begin);
+        if (zero_mask & kZeroPairs) head = (size_t)((char *)(w.tl_pair + 2 * z.N) - w.zero_begin);
         CU(cudaMemsetAsync(w.zero_begin, 0, head, s));
     }
     if ((zero_mask & kZeroCounts) && z.N > 0) CU(cudaMemsetAsync(w.cnt, 0, sizeof(int32_t) * (size_t)z.N, s));
@@ -318,7 +319,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(trace, ws, w, d, s, 0);
+    rc = begin_call(trace, ws, w, d, s, kZeroPairs);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     int64_t *start = host ? w.start : out->kernel_start_ns;
@@ -326,7 +327,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     int64_t *pk = host ? w.peak_bytes : out->peak_bytes;
     int32_t *ps = host ? w.peak_slot : out->peak_slot;
     int64_t *st = host ? w.counts + 2 : out->status;
-    CU(launch_timeline(d, w, start, P, pk, ps, s));
+    CU(launch_timeline_pairs(d, w, start, w.tl_pair, w.tl_point, P, pk, ps, s));
     CU(launch_publish_status(w, st, s));
     if (host) {
         CU(d2h(out->kernel_start_ns, w.start, (size_t)d.K + 1, s));

@@ -89,7 +89,7 @@ struct Workspace {
     unsigned *bk_count, *bk_cursor;   // [4096] events per tensor bucket, scatter cursors
     ull *bk_words;               // [2 * 4096] tagged per-bucket totals
     ull *xwords;                 // [2][kSmallMaxBlocks][16] tagged words of the proposal exchange
-    ull *tl_words;               // [2 * kTlMaxBlocks] tagged segment sums of the timeline call (slot clock, pressure)
+    ull *seg_words, *seg_words2; // [blocks * 16] each: tagged segment sums of the slot-clock scan and of the pressure scan, one 128-byte line per block
     // --- uninitialised region ---
     int32_t *raw_ptr;            // [N+1]
     int32_t *raw_uses;           // [E]
@@ -97,9 +97,8 @@ struct Workspace {
     int32_t *heavy_info;         // [2*(E/33+1)] distinct uses, periods
     int64_t *tile_max;           // [tiles(K)]
     int32_t *tile_slot;          // [tiles(K)]
+    int64_t *tl_point;           // [K] bytes of the tensors alive in one slot only (timeline call)
     int *tl_pair;                // [2 * N] first / last use of every tensor, encoded (timeline call)
-    int64_t *tl_blk_max;         // [kTlMaxBlocks] per-block pressure maxima of the timeline call
-    int32_t *tl_blk_slot;        // [kTlMaxBlocks] and their lowest slots
     // vitality / timeline outputs when the caller did not ask for them (planner) or passed host memory
     int32_t *first_use, *last_use, *num_uses;
     int64_t *use_ptr, *period_ptr;
@@ -164,14 +163,11 @@ struct PlanParams {
 };
 
 constexpr int kMaxPlanBlocks = 1024;
-constexpr int kTlMaxBlocks = 512;          // blocks of the timeline call's persistent grid, at most
 constexpr int kSmallMaxBlocks = 160;       // blocks of the small-trace planner (one per SM, at most)
 constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock fit in shared memory
 
 // passes (g10_passes.cu)
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);
-cudaError_t launch_clock_and_first_last(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *first_use, int32_t *last_use,
-                                        cudaStream_t s);
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 // bucketed formulation (g10_vitality_buckets.cu); supported for up to 4096 buckets of 4096 tensors
 bool vitality_buckets_supported(int64_t N, int64_t E);
@@ -182,9 +178,9 @@ cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int3
 cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, const int64_t *start, const int64_t *tensor_bytes,
                             const int32_t *per_t, const int32_t *per_u, const int32_t *per_v, uint64_t host_bw, uint64_t ssd_bw,
                             int64_t stride, int64_t *geo_t, int32_t *geo_a, int32_t *geo_b, cudaStream_t s);
-// timeline call (g10_timeline.cu): slot clock, pressure, peak from the trace alone
-cudaError_t launch_timeline(const DeviceTrace &t, const Workspace &w, int64_t *start, int64_t *pressure, int64_t *peak_bytes,
-                            int32_t *peak_slot, cudaStream_t s);
+// timeline call: slot clock, pressure, peak from the trace alone (g10_passes.cu)
+cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *pair, int64_t *point, int64_t *pressure,
+                                  int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);
 // eager prefetch pass (g10_prefetch.cu)
 cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *mig, const int64_t *start, const int64_t *bytes,
                                      uint64_t gpu_capacity_bytes, int64_t *P, int32_t *order, int32_t *new_last, int64_t *new_issue,

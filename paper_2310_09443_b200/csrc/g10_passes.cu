@@ -1,6 +1,8 @@
 // The HBM-bound passes: slot clock (Section 4.2: kernel times measure the inactive periods), tensor
 // vitality (Section 4.2: born / dead / inactive periods), memory-pressure timeline (Section 4.3) and
 // candidate geometry (Algorithm 1's t = size / BW; Section 4.4's latest safe prefetch time).
+#include <climits>
+
 #include "g10_device.cuh"
 #include "g10_internal.h"
 
@@ -20,6 +22,9 @@ constexpr int kSegWarps = kSegThreads / 32;
 constexpr int kSegItems = 8;
 constexpr int kSegChunk = kSegThreads * kSegItems;
 constexpr int kSegMaxBlocks = 512;
+// Every block's word sits in a 128-byte line of its own: a few hundred blocks each read all their predecessors' words at the
+// same moment, and words packed into a few lines would all be served by the same one or two L2 slices, one after the other.
+constexpr int kSegWordStride = 16;
 
 __device__ __forceinline__ ull seg_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
 __device__ __forceinline__ long long seg_unpack(ull w) { return (long long)(w << 2) >> 2; }     // sign-extend 62 bits
@@ -40,7 +45,8 @@ __device__ __forceinline__ long long seg_warp_totals(const long long *s_w, int l
 }
 
 // kind 0: exclusive scan of kernel_ns into start[0..K] with validation of kernel_ns and kernel_ptr
-// kind 1: inclusive scan of the difference array into the pressure, plus peak and lowest peak slot
+// kind 1: inclusive scan of the difference array into the pressure, plus peak and lowest peak slot; `kptr`, if not null, holds
+//         for every slot the bytes of the tensors that are alive in that slot alone (added to the scan's result, not carried on)
 template <int kind>
 __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t E, const int64_t *__restrict__ in, const int64_t *__restrict__ kptr,
                                                              int64_t *__restrict__ out, unsigned *ticket, unsigned *done, ull *words,
@@ -89,14 +95,14 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
     long long unused;
     const long long seg_total = seg_warp_totals(s_w, lane, warp, &unused);
     if (threadIdx.x == 0)
-        asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&words[g]), "l"(seg_pack(seg_total)) : "memory");
+        asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&words[(size_t)g * kSegWordStride]), "l"(seg_pack(seg_total)) : "memory");
     // ---- prefix of the segment: all predecessors' sums
     long long pre = 0;
     for (int j = threadIdx.x; j < g; j += kSegThreads) {
         ull w;
         unsigned polls = 0;
         for (;;) {
-            asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(w) : "l"(&words[j]) : "memory");
+            asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(w) : "l"(&words[(size_t)j * kSegWordStride]) : "memory");
             if (w >> 62) break;
             if (++polls > kSpinLimit) { raise_status(status, G10_DEV_TIMEOUT); w = 0; break; }
             __nanosleep(64);
@@ -135,7 +141,11 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
             if (kind == 0) { if (k < hi) out[k] = run; run += v[j]; }
             else {
                 run += v[j];
-                if (k < hi) { out[k] = run; if (sl < 0 || run > mx) { mx = run; sl = (int)k; } }
+                if (k < hi) {
+                    const long long p = kptr != nullptr ? run + kptr[k] : run;     // (kind 1: kptr = bytes alive in slot k only, or null)
+                    out[k] = p;
+                    if (sl < 0 || p > mx) { mx = p; sl = (int)k; }
+                }
             }
         }
         carry += ctot;
@@ -210,7 +220,7 @@ cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t 
 {
     const int G = seg_scan_blocks(t.K);
     k_seg_scan<0><<<G, kSegThreads, 0, s>>>(t.K, t.E, t.kernel_ns, t.kernel_ptr, start, w.clock_scan.ticket, w.clock_scan.done,
-                                          (ull *)w.clock_scan.agg, nullptr, nullptr, nullptr, nullptr, w.status);
+                                          w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status);
     return cudaGetLastError();
 }
 
@@ -371,6 +381,69 @@ __global__ void __launch_bounds__(kFlThreads) k_first_last_events(int64_t E, int
     if (bad) raise_status(status, bad);
 }
 
+// The same pass for the timeline call, on an interleaved array pair[2 i] = max(K - k), pair[2 i + 1] = max(k + 1): lanes l and
+// l + 16 of a warp share an event, one raises the tensor's first word, the other its last word.  Both words lie in one
+// 32-byte sector, so the two reductions reach the L2 as one request; the L2 serves such scattered requests at a fixed
+// rate per sector whatever they carry (about 170 G/s on this part), which is what bounds this pass.
+__global__ void __launch_bounds__(kFlThreads) k_first_last_pairs(int64_t E, int64_t N, int64_t K, const int64_t *__restrict__ kptr,
+                                                                 const int32_t *__restrict__ kt, int32_t *__restrict__ pair, ull *budget, ull *status)
+{
+    __shared__ int64_t s_span[2];
+    const int lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+    const int64_t kb0 = (int64_t)blockIdx.x * kFlThreads;
+    if (threadIdx.x == 0) {
+        const int64_t kb1 = kb0 + kFlThreads < K ? kb0 + kFlThreads : K;
+        int64_t b0 = kptr[kb0], b1 = kptr[kb1];
+        b0 = b0 < 0 ? 0 : (b0 > E ? E : b0);
+        b1 = b1 < 0 ? 0 : (b1 > E ? E : b1);
+        if (b1 < b0) b1 = b0;
+        if (b1 > b0 && atomicAdd(budget, (ull)(b1 - b0)) + (ull)(b1 - b0) > (ull)E) {
+            raise_status(status, G10_DEV_BAD_KERNEL_PTR);
+            b1 = b0;
+        }
+        s_span[0] = b0; s_span[1] = b1;
+    }
+    __syncthreads();
+    const int64_t b0 = s_span[0], b1 = s_span[1];
+    const int64_t k = kb0 + threadIdx.x, k0 = k - lane;
+    const bool idle = k0 >= K || b1 == b0;                       // (uniform in the warp)
+    int64_t mine = idle ? 0 : kptr[k < K ? k : K];               // lanes past the last kernel hold kernel_ptr[K]
+    int64_t span1 = idle ? 0 : kptr[k0 + 32 < K ? k0 + 32 : K];
+    mine = mine < b0 ? b0 : (mine > b1 ? b1 : mine);
+    span1 = span1 < b0 ? b0 : (span1 > b1 ? b1 : span1);
+    const int64_t span0 = __shfl_sync(0xffffffffu, mine, 0);
+    if (idle) span1 = span0;
+    ull bad = 0;
+#pragma unroll 1
+    for (int64_t base = span0; base < span1; base += 32) {       // two rows of sixteen events per step: both rows' loads in flight
+        int32_t id[2];
+        int kq[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const int64_t e = base + 16 * r + l16;
+            int lo = 0;                                          // last lane whose kernel starts at or before e
+#pragma unroll
+            for (int st = 16; st > 0; st >>= 1) {
+                const int64_t p = __shfl_sync(0xffffffffu, mine, (lo + st) & 31);
+                if (p <= e) lo += st;
+            }
+            kq[r] = (int)(k0 + lo);
+            id[r] = e < span1 ? kt[e] : INT32_MIN;
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            if (id[r] == INT32_MIN) continue;
+            if (id[r] < 0 || id[r] >= N) bad = G10_DEV_BAD_TENSOR_ID;
+            else atomicMax(&pair[2 * (size_t)id[r] + half], half ? kq[r] + 1 : (int)K - kq[r]);
+        }
+    }
+    if (bad) raise_status(status, bad);
+    // Launched with programmatic stream serialisation behind the slot-clock scan, which lets its dependents start early: this
+    // grid reads nothing of the scan's, but it must not complete before the scan has (the kernels behind it wait for this
+    // grid only, and the call's status word and slot clock have to be final by then).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s)
 {
     if (t.N == 0) return cudaSuccess;
@@ -381,39 +454,6 @@ cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t 
     if (t.E > 0 && t.K > 0) {
         const int blocks = (int)tiles_of(t.K, kFlThreads);
         k_first_last_events<<<blocks, kFlThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.event_budget, w.status);
-    }
-    return cudaGetLastError();
-}
-
-// Slot clock and first / last use for the timeline call: the two are independent, so the event kernel is launched
-// with programmatic stream serialisation and runs beside the clock scan (it never reads what the scan writes).
-cudaError_t launch_clock_and_first_last(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *first_use, int32_t *last_use,
-                                        cudaStream_t s)
-{
-    cudaError_t e;
-    if (t.N > 0) {
-        const ptrdiff_t gap = (const char *)last_use - (const char *)(first_use + t.N);
-        if (gap >= 0 && gap < 4096) {                 // the two arrays follow each other in the workspace: one memset
-            if ((e = cudaMemsetAsync(first_use, 0, (size_t)((const char *)(last_use + t.N) - (const char *)first_use), s)) != cudaSuccess) return e;
-        } else {
-            if ((e = cudaMemsetAsync(first_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
-            if ((e = cudaMemsetAsync(last_use, 0, sizeof(int32_t) * (size_t)t.N, s)) != cudaSuccess) return e;
-        }
-    }
-    if ((e = launch_slot_clock(t, w, start, s)) != cudaSuccess) return e;
-    if (t.N > 0 && t.E > 0 && t.K > 0) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)tiles_of(t.K, kFlThreads));
-        cfg.blockDim = dim3(kFlThreads);
-        cfg.dynamicSmemBytes = 0;
-        cfg.stream = s;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, k_first_last_events, t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.event_budget, w.status);
-        if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
 }
@@ -707,6 +747,40 @@ __global__ void __launch_bounds__(256) k_diff_scatter(int64_t N, int64_t K, cons
         if (tot != 0) atomicAdd(&diff[0], (ull)tot);
     }
 }
+// The same from the interleaved pair array of k_first_last_pairs.  A tensor that a single kernel uses (most tensors of a
+// trace) is alive in that slot alone: instead of a birth and a death next to each other in the difference array it is
+// booked once, in `point`, which the pressure scan adds to its result slot by slot.
+__global__ void __launch_bounds__(256) k_diff_scatter_pairs(int64_t N, int64_t K, const int64_t *__restrict__ bytes, const uint8_t *__restrict__ glob,
+                                                            const int2 *__restrict__ pair, ull *__restrict__ diff, ull *__restrict__ point, ull *status)
+{
+    __shared__ long long s_part[8];
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // (see k_diff_scatter)
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    long long gsum = 0;
+    if (i < N) {
+        const long long b = bytes[i];
+        if (b < 1 || b >= ((long long)1 << 40)) raise_status(status, G10_DEV_BAD_BYTES);
+        const int2 enc = pair[i];                                // K - first, last + 1; 0 = unused
+        if (enc.x > 0 && enc.x <= K && enc.y > 0 && enc.y <= K) {
+            const int64_t f = K - enc.x, l = (int64_t)enc.y - 1;
+            if (glob != nullptr && glob[i]) gsum = b;
+            else if (f == l) atomicAdd(&point[f], (ull)b);
+            else {
+                atomicAdd(&diff[f], (ull)b);
+                if (l + 1 < K) atomicAdd(&diff[l + 1], (ull)(-b));
+            }
+        }
+    }
+    gsum = warp_sum_i64(gsum);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = gsum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long tot = 0;
+        for (int w = 0; w < 8; ++w) tot += s_part[w];
+        if (tot != 0) atomicAdd(&diff[0], (ull)tot);
+    }
+}
+
 cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
 {
@@ -734,9 +808,43 @@ cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int3
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);
     e = cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)nullptr, pressure, w.pressure_scan.ticket,
-                           w.pressure_scan.done, (ull *)w.pressure_scan.agg, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
+                           w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
+}
+
+// The timeline call: slot clock beside the first / last pass (the two are independent), difference array from the pairs,
+// pressure scan.  `pair` [2 N], `point` [K] and the difference array start at zero (cleared by the caller).
+cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *pair, int64_t *point, int64_t *pressure,
+                                  int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
+{
+    cudaError_t e;
+    if ((e = launch_slot_clock(t, w, start, s)) != cudaSuccess) return e;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (t.N > 0 && t.E > 0 && t.K > 0) {
+        cfg.gridDim = dim3((unsigned)tiles_of(t.K, kFlThreads));
+        cfg.blockDim = dim3(kFlThreads);
+        if ((e = cudaLaunchKernelEx(&cfg, k_first_last_pairs, t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, pair, w.event_budget, w.status)) != cudaSuccess) return e;
+    }
+    if (t.N > 0 && t.K > 0) {
+        cfg.gridDim = dim3((unsigned)((t.N + 255) / 256));
+        cfg.blockDim = dim3(256);
+        const int64_t *bytes = t.tensor_bytes;
+        const uint8_t *glob = t.tensor_global;
+        const int2 *cpair = reinterpret_cast<const int2 *>(pair);
+        if ((e = cudaLaunchKernelEx(&cfg, k_diff_scatter_pairs, t.N, t.K, bytes, glob, cpair, (ull *)w.diff, (ull *)point, w.status)) != cudaSuccess) return e;
+    }
+    cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
+    cfg.blockDim = dim3(kSegThreads);
+    return cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)point, pressure, w.pressure_scan.ticket,
+                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
 }
 
 // =============================================================================================

@@ -93,6 +93,8 @@ extern "C" int32_t g10_pressure_timeline_static(const g10_trace *trace, g10_time
     w.event_budget = b.take<ull>(1);
     take_scan(b, w.clock_scan, ktiles);
     take_scan(b, w.pressure_scan, ktiles);
+    w.seg_words = b.take<ull>((ktiles + 1) * 16);        // (the scans run at most one block per 4096 kernels: fewer than ktiles)
+    w.seg_words2 = b.take<ull>((ktiles + 1) * 16);
     w.diff = b.take<int64_t>((size_t)K + 1);
     w.zero_bytes = align_up(b.off);
     w.first_use = b.take<int32_t>((size_t)N);
