@@ -121,8 +121,8 @@ typedef struct g10_geometry_out {
     int32_t *absent_last;       /* [2 * Pn]                                                         */
 } g10_geometry_out;
 
-/* One committed migration (Algorithm 1's "schedule pre-eviction(tensor, destination) at t_r"; the
-   matching prefetch is issued at prefetch_issue_ns).  Records appear in commit order. */
+/* One committed migration (the step of Algorithm 1 that schedules a tensor's pre-eviction to its destination
+   at the start of the period; the matching prefetch is issued at prefetch_issue_ns).  Records appear in commit order. */
 typedef struct g10_migration {
     int32_t period, tensor, dest;
     int32_t absent_first, absent_last;
@@ -320,7 +320,9 @@ int32_t g10_characterize(int64_t num_kernels, int64_t num_tensors, const int64_t
      - traces up to G10_STATIC_MAX_KERNELS kernels and G10_STATIC_MAX_TENSORS tensors; anything larger is
        refused with G10_ERR_LIMIT before any work is enqueued;
      - the first call on each device looks the array's address up (cudaGetSymbolAddress, with that device
-       current); make that first call outside any stream capture;
+       current); make that first call outside any stream capture.  The address is remembered for the life of the
+       process: after cudaDeviceReset() (or any teardown of the device's primary context) it is stale and this
+       entry point must not be called again in that process;
      - all calls on a device share the one array, which keeps the previous call's contents (the call clears
        what it needs zeroed); two calls that overlap on the GPU -- different streams, or one stream per thread --
        race on it and give wrong results, so serialise them;

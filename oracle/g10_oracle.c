@@ -222,8 +222,8 @@ static int64_t overlap(const plan_state *S, int64_t w0, int64_t w1, int64_t k)
     return hi > lo ? hi - lo : 0;
 }
 
-/* Bandwidth budget (Algorithm 1 asks whether the traffic to a device "is full" during the
-   transfer).  Reading: each slot offers dur[k] ns of channel time per device and direction; a
+/* Bandwidth budget (Algorithm 1 tests whether the link to a device is saturated for the duration
+   of the transfer).  Reading: each slot offers dur[k] ns of channel time per device and direction; a
    transfer may be booked iff, in every slot its window touches, the time already booked plus the
    window's overlap with that slot stays within dur[k]. */
 static int channel_free(const plan_state *S, int ch, int64_t w0, int64_t w1, int64_t k0, int64_t k1)
@@ -243,7 +243,7 @@ static int admissible(const plan_state *S, int64_t p, int X)
     if (!channel_free(S, out, t_r, t_r + g->t, a, g->a_abs - 1)) return 0;
     if (!channel_free(S, in, t_end - g->t, t_end, g->b_abs + 1, b)) return 0;
     if (X == DEST_HOST && S->host_capacity != 0) {
-        /* "host mem isn't full during periods[0]": the tensor sits in host memory for the whole period */
+        /* host-capacity test of Algorithm 1: the tensor occupies host memory for the whole period */
         uint64_t s = (uint64_t)S->bytes[S->per_tensor[p]];
         for (int64_t k = a; k <= b; ++k)
             if ((uint64_t)S->hocc[k] + s > S->host_capacity) return 0;

@@ -20,8 +20,26 @@ constexpr int kMaxDevices = 64;
 // device address and must never be handed to a kernel as one.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
+// The layout of the call below at the documented maxima, bounded from above (every array rounded up to the workspace
+// alignment): it has to fit the array, so that G10_ERR_LIMIT can only mean "trace larger than the documented maxima".
+constexpr size_t au(size_t bytes) { return (bytes + kAlign - 1) / kAlign * kAlign; }
+constexpr size_t static_layout_bound(size_t K, size_t N)
+{
+    const size_t tiles = (K + 2047) / 2048 + 1;
+    return 2 * au(8)                                                      // status word, event budget
+         + 2 * (2 * au(4) + au(4 * tiles) + 2 * au(8 * tiles))           // the two scans' slots
+         + 2 * au(8 * 16 * (tiles + 1))                                   // their tagged words, one line per block
+         + au(8 * (K + 1)) + 2 * au(4 * N)                                // difference array, first / last use
+         + au(8 * tiles) + au(4 * tiles);                                 // per-block maxima
+}
+static_assert(static_layout_bound(G10_STATIC_MAX_KERNELS, G10_STATIC_MAX_TENSORS) <= kStaticScratchBytes,
+              "the static scratch array is too small for the documented maxima");
+
 std::mutex g_setup_mutex;
-void *g_scratch_addr[kMaxDevices];      // device address of g_static_scratch on each device, once looked up
+// Device address of g_static_scratch on each device, once looked up.  It belongs to the context it was looked up in: after
+// cudaDeviceReset() (or any other teardown of the primary context) the remembered address is stale, and this entry
+// point must not be called again in that process (documented in g10.h).
+void *g_scratch_addr[kMaxDevices];
 
 // Looks the array's device address up once per device (with that device current) and remembers it.
 cudaError_t scratch_address(void **out)

@@ -315,8 +315,11 @@ def test_host_pointer_mode(gpu, oracle):
     ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
     pn = int(v.counts[1])
     assert int(v.counts[2]) == 0 and pn == len(ov.period_tensor)
-    assert np.array_equal(v.first_use.numpy(), ov.first_use) and np.array_equal(v.uses.numpy()[:int(v.counts[0])], ov.uses)
-    assert np.array_equal(v.period_next_use.numpy()[:pn], ov.period_next_use)
+    e2 = int(v.counts[0])
+    assert e2 == len(ov.uses)
+    for name, n in (("first_use", None), ("last_use", None), ("num_uses", None), ("use_ptr", None), ("period_ptr", None),
+                    ("uses", e2), ("period_tensor", pn), ("period_prev_use", pn), ("period_next_use", pn)):
+        assert np.array_equal(getattr(v, name).numpy()[:n], getattr(ov, name)), name
     tl = gpu.g10_pressure_timeline(tb)
     start, P0, peak, slot = oracle.timeline(tr)
     assert np.array_equal(tl.pressure.numpy(), P0) and int(tl.peak_bytes) == peak and int(tl.peak_slot) == slot

@@ -263,3 +263,47 @@ def test_lazy_equals_plain_scaled_stress(oracle):
     assert np.array_equal(a.migrations, b.migrations) and np.array_equal(a.summary, b.summary)
     assert np.array_equal(a.final_pressure, b.final_pressure)
     _replay(oracle, tr, cap, a)
+
+
+def _same_plan(a, b):
+    return (np.array_equal(a.migrations, b.migrations) and np.array_equal(a.summary, b.summary)
+            and np.array_equal(a.final_pressure, b.final_pressure))
+
+
+def test_lazy_equals_plain_config3(oracle):
+    """The lazy tier backs the GPU parity checks of the ViT-shaped trace: it has to give Algorithm 1's plan there."""
+    tr = traces.make_config(3)
+    start, P0, peak, slot = oracle.timeline(tr)
+    cap = tr.capacity_from_peak(peak)
+    a = oracle.plan(tr, cap)
+    b = oracle.plan(tr, cap, lazy=True)
+    assert len(a.migrations) > 1000 and _same_plan(a, b)
+
+
+def test_lazy_equals_plain_stress_20k(oracle):
+    """... and on the stress trace at K = 2*10^4, N = 8*10^4 (several scan tiles, periods hundreds of slots long),
+    before it stands in for the plain tier at full size."""
+    tr = traces.config4_stress_dag(K=20000, N=80000)
+    start, P0, peak, slot = oracle.timeline(tr)
+    cap = tr.capacity_from_peak(peak)
+    a = oracle.plan(tr, cap)
+    b = oracle.plan(tr, cap, lazy=True)
+    assert len(a.migrations) > 1000 and _same_plan(a, b)
+    _replay(oracle, tr, cap, a)
+
+
+@pytest.mark.parametrize("cfg,ssd_bw,host_bw,cap_num,host_cap", [
+    (1, 102_400_000_000, 32_000_000_000, 1, 0),
+    (1, 6_400_000_000, 512_000_000_000, 1, 8 << 30),
+    (2, 102_400_000_000, 512_000_000_000, 2, 0),
+    (2, 3_200_000_000, 32_000_000_000, 1, 8 << 30),
+    (2, 12_800_000_000, 512_000_000_000, 2, 8 << 30),
+])
+def test_lazy_equals_plain_on_the_sweep(oracle, cfg, ssd_bw, host_bw, cap_num, host_cap):
+    """Points of the bandwidth / capacity / host-memory sweep that the GPU parity test checks against the lazy tier
+    (fast SSD, fast host link, finite host memory, half the usual capacity): same plan from both tiers."""
+    tr = traces.make_config(cfg)
+    cap = tr.capacity_from_peak(0) // cap_num
+    a = oracle.plan(tr, cap, host_bw=host_bw, ssd_bw=ssd_bw, host_capacity_bytes=host_cap)
+    b = oracle.plan(tr, cap, host_bw=host_bw, ssd_bw=ssd_bw, host_capacity_bytes=host_cap, lazy=True)
+    assert len(a.migrations) > 100 and _same_plan(a, b)

@@ -31,6 +31,15 @@ def _same(a, b, K):
         assert np.array_equal(x, y), name      # integer outputs: the tolerance is bit-exact
 
 
+def _same_as_oracle(got, tr):
+    from oracle import g10_oracle as O
+    O.build()
+    start, P0, peak, slot = O.timeline(tr)
+    assert np.array_equal(got.kernel_start_ns.cpu().numpy(), start)
+    assert np.array_equal(got.pressure.cpu().numpy()[:tr.K], P0)
+    assert int(got.peak_bytes.item()) == peak and int(got.peak_slot.item()) == slot
+
+
 def test_static_scratch_matches_workspace_variant_on_consecutive_calls(gpu):
     import torch
     seq = [traces.config1_resnet152(), traces.config0_mlp_chain(), traces.config3_vit_huge(), traces.config1_resnet152()]
@@ -41,6 +50,7 @@ def test_static_scratch_matches_workspace_variant_on_consecutive_calls(gpu):
         torch.cuda.synchronize()
         assert int(got.status.item()) == 0
         _same(got, ref, tr.K)
+        _same_as_oracle(got, tr)                    # and both agree with the CPU oracle, not only with each other
     # twice in a row on the very same inputs, without anything in between
     tb = gpu.upload(seq[0])
     a = gpu.g10_pressure_timeline_static(tb)
@@ -49,6 +59,20 @@ def test_static_scratch_matches_workspace_variant_on_consecutive_calls(gpu):
     torch.cuda.synchronize()
     _same(a, ref, seq[0].K)
     _same(b, ref, seq[0].K)
+
+
+def test_static_variant_at_its_largest_trace(gpu):
+    """Exactly the documented maxima (32 768 kernels, 131 072 tensors): the scratch layout still fits the static
+    array and the result is the oracle's."""
+    import torch
+    tr = traces.config4_stress_dag(K=gpu.STATIC_MAX_KERNELS, N=gpu.STATIC_MAX_TENSORS)
+    assert tr.K == gpu.STATIC_MAX_KERNELS and tr.N == gpu.STATIC_MAX_TENSORS
+    tb = gpu.upload(tr)
+    for _ in range(2):
+        got = gpu.g10_pressure_timeline_static(tb)
+        torch.cuda.synchronize()
+        assert int(got.status.item()) == 0
+        _same_as_oracle(got, tr)
 
 
 def test_static_variant_refuses_what_does_not_fit(gpu):
