@@ -1,15 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the G10 planning path on B200.
 
-A step is one pass of the whole hot path -- slot clock, tensor vitality, pressure timeline, candidate
-geometry and the greedy eviction loop, i.e. one g10_plan_migrations call -- over the ResNet-152-shaped
-trace (config 1).  `value` = trace events planned per second with the trace resident in HBM; `plan_ms`
-is the same step as a latency.  Prints ONE JSON line (rank 0).
+Headline (`value`): trace events per second through the analysis passes S1-S3 -- slot clock, tensor vitality
+and pressure timeline, i.e. one g10_vitality call plus one g10_pressure_timeline call -- on the 1M-kernel /
+4M-tensor stress trace (config 4), the largest single-GPU workload and the only one whose arrays are large enough
+for an HBM fraction to mean something.  A step is one such pass with the trace resident in HBM; the L2 is flushed
+between steps.  Second headline (`plan_ms`): one whole g10_plan_migrations call (S1-S7) on the ResNet-152-shaped
+trace (config 1).  The same line carries the plan of every configuration (`plans`), the two analysis calls on a
+trace eight times the size (`scale_x8`), the calls behind the plan (prefetch pass, instruction stream, batched and
+cyclic planning), the roofline of the passes and the CPU oracle timed beside them.  Prints ONE JSON line (rank 0).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-stress]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick]
 
-With N > 1 (torchrun) every rank plans its own replica of the trace (the path does not shard: the greedy
-loop is a strict sequence); value is the aggregate over ranks, time the max over ranks.
+With N > 1 (torchrun) every rank works on its own replica of the trace (the path does not shard: the greedy loop
+is a strict sequence); value is the aggregate over ranks, time the max over ranks.
 """
 from __future__ import annotations
 
@@ -29,18 +33,29 @@ if ROOT not in sys.path:
 
 from paper_2310_09443_b200 import traces  # noqa: E402
 
-WORKLOAD = "config1_resnet152_b256"
+WORKLOAD = "config4_stress_dag"
+PLAN_WORKLOAD = "config1_resnet152_b256"
 L2_FLUSH_BYTES = 512 << 20
-PLAN_ONE_DRAM_BYTES = 211456    # dram__bytes_read.sum + dram__bytes_write.sum of one k_plan_one launch on config 1 (ncu --set full capture)
-# DRAM bytes per call on the stress trace, from an ncu capture of `bench.py --stress-only --stress-reps 1` (dram__bytes_read.sum +
-# dram__bytes_write.sum summed over the call's kernels): k_bk_hist 28.0 + k_bk_scatter 28.2 + k_bk_emit 138.0 MB; k_seg_scan<0> 16.0 +
-# k_first_last_events 59.9 + k_diff_scatter 76.1 + k_seg_scan<1> 8.0 MB
-STRESS_VITALITY_DRAM_BYTES = 194_200_000
-STRESS_TIMELINE_DRAM_BYTES = 160_000_000
-KERNELS_PER_PLAN = 10      # slot clock, bucket histogram, bucket scatter, bucket emit, diff, pressure scan, geometry,
-                           # single-block loop, multi-block loop (returns at once when the former did the work), status
-KERNELS_PER_VITALITY = 4   # bucket histogram, bucket scatter, bucket emit, status
-KERNELS_PER_TIMELINE = 5   # slot clock, first/last events, diff, pressure scan, status
+# DRAM bytes per call on the stress trace (dram__bytes_read.sum + dram__bytes_write.sum summed over the call's kernels), from
+# the one-pass ncu capture whose command and table are in profiles/passes_config4_stress.md.  SOURCES_SHA256 is the hash
+# of the kernel sources at the time of the capture: when the sources have changed since, the bench line says so
+# ("traffic_stale") instead of passing old traffic off as current.
+TRAFFIC = {"vitality": 194_200_000, "timeline": 160_000_000, "captured_at": "2026-11-25", "sources_sha256": "unset"}
+# kernels launched per call (counted from the launch lists in profiles/): vitality = bucket histogram, partition, emit,
+# status; timeline = slot-clock scan, first/last pairs, difference scatter, pressure scan, status (+ 1 memset node each)
+KERNELS_PER_VITALITY = 4
+KERNELS_PER_TIMELINE = 5
+
+
+def kernel_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2310_09443_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        if f.endswith((".cu", ".cuh", ".h")):
+            h.update(f.encode())
+            h.update(open(os.path.join(d, f), "rb").read())
+    return h.hexdigest()
 
 
 def measured_peaks():
@@ -100,33 +115,54 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+
+
+def pass_bytes(K, N, E, uses, periods):
+    """Algorithmic bytes of the two analysis calls.  Vitality reads kernel_ptr (8K) and kernel_tensors (4E) and writes
+    first/last/num_uses (12N), use_ptr (8N), uses (4E'), period_ptr (8N) and the periods (12 Pn); the timeline reads
+    kernel_ns (8K), tensor_bytes (8N), first/last (8N), the global flag (N) and writes start (8K) and pressure (8K)."""
+    return 8 * K + 4 * E + 28 * N + 4 * uses + 12 * periods, 24 * K + 17 * N
+
+
+def oracle_s123(O, tr):
+    """One pass S1-S3 of the CPU oracle: vitality, slot clock and the plain definition of the pressure."""
+    v = O.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+    start, P0, peak, slot = O.timeline(tr)
+    return v, peak
+
+
 def run_reference(args):
-    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only): the same metric on the same workload.
+    A step is one whole pass S1-S3 over the stress trace (about five seconds on one core)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from oracle import g10_oracle as O
     O.build()
-    tr = traces.config1_resnet152()
-    start, P0, peak, slot = O.timeline(tr)
-    cap = tr.capacity_from_peak(peak)
-    for _ in range(args.warmup):
-        O.plan(tr, cap)
+    tr = traces.config4_stress_dag()
+    steps, warm = max(1, min(args.steps, 12)), max(0, min(args.warmup, 1))      # bounded: the whole run ends within minutes
+    for _ in range(warm):
+        oracle_s123(O, tr)
     t0 = time.perf_counter()
-    for _ in range(args.steps):
-        r = O.plan(tr, cap)
+    for _ in range(steps):
+        v, peak = oracle_s123(O, tr)
     dt = time.perf_counter() - t0
-    value = tr.E * args.steps / dt
+    value = tr.E * steps / dt
+    t1 = time.perf_counter()
+    tr1 = traces.config1_resnet152()
+    r = O.plan(tr1, tr1.capacity_from_peak(0))
+    plan_ms = (time.perf_counter() - t1) * 1e3
     line = {
         "impl": "reference", "metric": "trace_events_per_s", "value": value, "unit": "events/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "steps": steps, "warmup": warm, "ms_per_step": dt / steps * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
         "config": {"workload": WORKLOAD, "trace_sha256": tr.sha256(), "K": tr.K, "N": tr.N, "E": tr.E,
-                   "migrations": int(r.summary[0]), "status": r.status},
+                   "uses": int(len(v.uses)), "periods": int(len(v.period_tensor)),
+                   "steps_note": "steps and warm-up bounded to 12 and 1: a step takes seconds on one core"},
         "cpu_baseline": {"value": value, "unit": "events/s", "cores": 1, "kind": "oracle",
-                         "sample": "whole config-1 plan (plain tier), %d repetitions" % args.steps, "cpu_model": cpu_model()},
+                         "sample": "%d whole passes S1-S3 over config 4" % steps, "cpu_model": cpu_model()},
         "e2e": {"value": value, "unit": "events/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "plan_ms": dt / args.steps * 1e3,
+        "plan_ms": plan_ms, "plan_workload": PLAN_WORKLOAD, "plan_migrations": int(r.summary[0]),
     }
     print(json.dumps(line))
 
@@ -144,20 +180,113 @@ def aggregate_events_per_s(world, events_per_step, steps, total_ms):
     return world * events_per_step * steps / (total_ms / 1e3)
 
 
-def time_calls(torch, fn, steps, warmup, flush):
-    """CUDA-event time of `steps` calls of fn on the current stream, L2 flushed between calls.  Returns seconds."""
+def timed(torch, fn, steps, warmup, flush):
+    """CUDA-event times (ms) of `steps` calls of fn on the current stream; `flush` (a buffer larger than the L2, or
+    None) is rewritten before every call, outside the event pair."""
     for _ in range(warmup):
-        flush.fill_(1)
+        if flush is not None:
+            flush.fill_(1)
         fn()
     torch.cuda.synchronize()
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     for a, b in evs:
-        flush.fill_(1)
+        if flush is not None:
+            flush.fill_(1)
         a.record()
         fn()
         b.record()
     torch.cuda.synchronize()
-    return sum(a.elapsed_time(b) for a, b in evs) / 1e3
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def time_calls(torch, fn, steps, warmup, flush):
+    """Sum of the timed calls, in seconds."""
+    return sum(timed(torch, fn, steps, warmup, flush)) / 1e3
+
+
+def roofline(nbytes, seconds, peak, peak_kind, **extra):
+    gbs = nbytes / seconds / 1e9
+    d = {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "frac_of_nominal_8000": gbs / 8000.0,
+         "algorithmic_bytes": nbytes, "peak_kind": peak_kind}
+    d.update(extra)
+    return d
+
+
+def replicate_trace(torch, binding, tb, times):
+    """The same trace `times` times back to back on the device (kernels, tensors and events of copy r follow those of copy
+    r - 1; tensor ids shifted by r * N): the stress trace scaled up for the roofline measurement."""
+    K, N, E = tb.K, tb.N, tb.E
+    kptr = torch.cat([tb.kernel_ptr[:-1] + r * E for r in range(times)] + [torch.tensor([times * E], dtype=torch.int64, device=tb.kernel_ptr.device)])
+    kt = torch.cat([tb.kernel_tensors + r * N for r in range(times)])
+    nbytes = tb.tensor_bytes.repeat(times)
+    ns = tb.kernel_ns.repeat(times)
+    glob = tb.tensor_global.repeat(times) if tb.tensor_global is not None else None
+    return binding.TraceBuffers(kptr, kt, nbytes, ns, glob, K=times * K, N=times * N, E=times * E)
+
+
+def scaled_passes(torch, binding, tb, times, flush, hbm_peak, peak_kind, reps=5):
+    """g10_vitality and g10_pressure_timeline alone on the stress trace replicated `times` times: with the fixed cost of
+    a call (launches, phase chains of tens of microseconds) spread over `times` as many events, what is left is throughput."""
+    big = replicate_trace(torch, binding, tb, times)
+    ws = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, big.K, big.N, big.E), dtype=torch.uint8, device=tb.kernel_ptr.device)
+    v = binding.g10_vitality(big, ws=ws)
+    tl = binding.g10_pressure_timeline(big, ws=ws)
+    torch.cuda.synchronize()
+    uses, periods = int(v.counts[0].item()), int(v.counts[1].item())
+    vb, tlb = pass_bytes(big.K, big.N, big.E, uses, periods)
+    out = {"times": times, "K": big.K, "N": big.N, "E": big.E, "uses": uses, "periods": periods,
+           "device_status": int(v.counts[2].item()) | int(tl.status.item()), "repetitions": reps,
+           "peak_bytes_is_that_of_one_copy": True}
+    del v, tl
+    for name, fn, nb in (("vitality", lambda: binding.g10_vitality(big, ws=ws), vb), ("timeline", lambda: binding.g10_pressure_timeline(big, ws=ws), tlb)):
+        cold = float(np.median(timed(torch, fn, reps, 2, flush)))
+        warm = float(np.median(timed(torch, fn, reps, 2, None)))
+        out[name + "_ms"] = cold
+        out[name + "_ms_warm_l2"] = warm
+        out[name + "_roofline"] = roofline(nb, cold / 1e3, hbm_peak, peak_kind)
+    out["events_per_s"] = big.E / ((out["vitality_ms"] + out["timeline_ms"]) / 1e3)
+    out["roofline"] = roofline(vb + tlb, (out["vitality_ms"] + out["timeline_ms"]) / 1e3, hbm_peak, peak_kind)
+    del big, ws
+    torch.cuda.empty_cache()
+    return out
+
+
+def plan_stats(torch, binding, tr, dev, flush, steps, warm, stage=False):
+    """Whole g10_plan_migrations calls on one trace (capacity from the trace's own recipe, applied to the peak this
+    library computed): median and spread of `steps` timed calls after `warm` warm-up calls."""
+    tb = binding.upload(tr, dev)
+    ws = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E), dtype=torch.uint8, device=dev)
+    tl = binding.g10_pressure_timeline(tb, ws=ws)
+    torch.cuda.synchronize()
+    cap = tr.capacity_from_peak(int(tl.peak_bytes.item()))
+    plan = binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)] if stage else None
+    if ev:
+        for e in ev:
+            e.record()                      # (an event owns a handle only once it has been recorded)
+    loop_ms = []
+
+    def call():
+        binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws, out=plan, stage_events=ev)
+
+    ms = []
+    for i in range(warm + steps):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); call(); b.record(); b.synchronize()
+        if i >= warm:
+            ms.append(a.elapsed_time(b))
+            if stage:
+                loop_ms.append(ev[3].elapsed_time(ev[4]))
+    s = plan.summary.cpu().numpy()
+    out = {"K": tr.K, "N": tr.N, "E": tr.E, "plan_ms": float(np.median(ms)), "plan_ms_min": float(min(ms)), "plan_ms_max": float(max(ms)),
+           "timed_calls": steps, "warmup_calls": warm, "migrations": int(s[0]), "iterations": int(s[1]), "status": binding.STATUS.get(int(s[2]), "?"),
+           "device_status": int(s[7]), "capacity_bytes": int(cap), "us_per_iteration": float(np.median(ms)) * 1e3 / max(int(s[1]), 1)}
+    if stage:
+        out["greedy_loop_ms"] = float(np.median(loop_ms))
+        out["greedy_loop_us_per_iteration"] = float(np.median(loop_ms)) * 1e3 / max(int(s[1]), 1)
+    return out, (tb, ws, plan, tl, cap)
 
 
 def run_ours(args):
@@ -171,6 +300,7 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the planner has no CPU path")
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
+    dist = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl")
@@ -186,25 +316,24 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     hbm_peak, peak_kind = measured_peaks()
-    tr = traces.config1_resnet152()
-    tb = binding.upload(tr, dev)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    cap = tr.capacity_from_peak(0)          # config 1 has an absolute capacity (16 GiB)
-    ws = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E), dtype=torch.uint8, device=dev)
-    plan = binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws)
-    torch.cuda.synchronize()
-    summary = plan.summary.cpu().numpy()
-    assert summary[7] == 0, "device status %x" % summary[7]
 
-    stage = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
-    for e in stage:
-        e.record()
-    stage_ms = np.zeros(4)
+    # ---- the headline: S1-S3 (one g10_vitality + one g10_pressure_timeline call) on the stress trace, device-resident
+    tr = traces.config4_stress_dag()
+    tb = binding.upload(tr, dev)
+    ws = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E), dtype=torch.uint8, device=dev)
+    v = binding.g10_vitality(tb, ws=ws)
+    tl = binding.g10_pressure_timeline(tb, ws=ws)
+    torch.cuda.synchronize()
+    assert int(v.counts[2].item()) == 0 and int(tl.status.item()) == 0, "device status"
+    uses, periods = int(v.counts[0].item()), int(v.counts[1].item())
+    K, N, E = tr.K, tr.N, tr.E
+    vit_bytes, tl_bytes = pass_bytes(K, N, E, uses, periods)
 
     def step():
-        binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws, out=plan, stage_events=stage)
+        binding.g10_vitality(tb, ws=ws, out=v)
+        binding.g10_pressure_timeline(tb, ws=ws, out=tl)
 
-    # ---- device-resident throughput: W warm-up steps, then exactly K timed steps
     for _ in range(args.warmup):
         flush.fill_(1)
         step()
@@ -212,248 +341,196 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     total_ms = 0.0
-    for a, b in evs:
+    for _ in range(args.steps):
         flush.fill_(1)                      # L2 flush between timed iterations (outside the event pair)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         step()
         b.record()
         b.synchronize()
         total_ms += a.elapsed_time(b)
-        stage_ms += np.array([stage[j].elapsed_time(stage[j + 1]) for j in range(4)])
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    total_s = max_over_ranks(torch, dist if world > 1 else None, world, total_ms, dev) / 1e3
-    value = aggregate_events_per_s(world, tr.E, args.steps, total_s * 1e3)
-    stage_ms /= args.steps
+    total_ms = max_over_ranks(torch, dist, world, total_ms, dev)
+    value = aggregate_events_per_s(world, E, args.steps, total_ms)
+    step_s = total_ms / args.steps / 1e3
 
-    # ---- the two analysis passes on their own (same workload)
-    vit_s = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), args.steps, args.warmup, flush)
-    tl_s = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), args.steps, args.warmup, flush)
-
-    # ---- the eager prefetch pass (Section 4.4) over the finished plan of the same workload
-    tl1 = binding.g10_pressure_timeline(tb, ws=ws)
-    torch.cuda.synchronize()
-    n_mig_dev = int(summary[0])
-
-    def prefetch_step():
-        binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws, out=plan)
-        return binding.g10_schedule_prefetch(tr.K, n_mig_dev, plan.migrations, tl1.kernel_start_ns, tb.tensor_bytes, cap, plan.final_pressure)
-
-    pf = prefetch_step()
-    torch.cuda.synchronize()
-    pf_summary = pf.summary.cpu().numpy()
-    both_s = time_calls(torch, prefetch_step, args.steps, args.warmup, flush)
-    prefetch_ms = both_s / args.steps * 1e3 - total_s / args.steps * 1e3
-
-    # ---- batched re-planning: one variant per SM, kernel durations jittered by +-10 % (seeded), variant 0 unperturbed
-    batch = None
-    if rank == 0:
-        sms = torch.cuda.get_device_properties(dev).multi_processor_count
-        rng = np.random.default_rng(20231009)
-        base_v = dict(gpu_capacity_bytes=cap, host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)
-        variants = [base_v]
-        for _ in range(sms - 1):
-            f = rng.uniform(0.9, 1.1, size=tr.K)
-            dur = np.maximum(1, np.rint(tr.kernel_ns.astype(np.float64) * f)).astype(np.int64)
-            variants.append(dict(base_v, kernel_ns=torch.from_numpy(dur).to(dev)))
-        wsb = torch.empty(binding.g10_workspace_bytes(binding.WS_BATCH, tb.K, tb.N, tb.E), dtype=torch.uint8, device=dev)
-        bsteps = max(3, args.steps // 4)
-        b_s = time_calls(torch, lambda: binding.g10_plan_batch(tb, variants, ws=wsb, migrations_cap=int(summary[0]) + 64), bsteps, 3, flush) / bsteps
-        bo = binding.g10_plan_batch(tb, variants, ws=wsb, migrations_cap=int(summary[0]) + 64)
-        torch.cuda.synchronize()
-        stab = bo.stability.cpu().numpy().astype(np.float64)
-        bsum = bo.summary.cpu().numpy()
-        batch = {"variants": len(variants), "ms": b_s * 1e3, "plans_per_s": len(variants) / b_s,
-                 "trace_events_per_s": len(variants) * tr.E / b_s, "jitter": "+-10 % per kernel, seeded",
-                 "mean_jaccard_vs_unperturbed": float(np.mean(stab[1:, 0] / np.maximum(stab[1:, 1], 1))),
-                 "device_status_or": int(np.bitwise_or.reduce(bsum[:, 7])),
-                 "note": "same planning path, one thread block per variant, all variants concurrently (binding allocates outputs inside the timed call)"}
-        del wsb, bo, variants
-
-    # ---- steady-state (cyclic) plan of the same trace: the weights' wrap-around periods become candidates
-    cyclic = None
-    if rank == 0:
-        csteps = max(3, args.steps // 4)
-        c_s = time_calls(torch, lambda: binding.g10_plan_cyclic(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws), csteps, 3, flush) / csteps
-        cp = binding.g10_plan_cyclic(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws)
-        torch.cuda.synchronize()
-        cs = cp.summary.cpu().numpy()
-        cyclic = {"plan_ms": c_s * 1e3, "migrations": int(cs[0]), "status": binding.STATUS.get(int(cs[2]), "?"),
-                  "final_peak_bytes": int(cs[3]), "final_peak_bytes_acyclic": int(summary[3]), "device_status": int(cs[7])}
-        del cp
-
-    # ---- end to end through the host-pointer form of the call: H2D of the trace and D2H of the plan inside
+    # ---- the same pass end to end through the host-pointer form of the calls: the library stages the trace (H2D) and
+    # copies every output back (D2H) inside the timed region
     tbh = binding.pin(tr)
-    wsh = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E, binding.MEM_HOST), dtype=torch.uint8, device=dev)
-    planh = binding.g10_plan_migrations(tbh, cap, tr.host_bw, tr.ssd_bw, ws=wsh, device=dev)
-    for _ in range(args.warmup):
-        binding.g10_plan_migrations(tbh, cap, tr.host_bw, tr.ssd_bw, ws=wsh, out=planh, device=dev)
+    wsh = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, K, N, E, binding.MEM_HOST), dtype=torch.uint8, device=dev)
+
+    outs = [None, None]                                               # pinned result buffers, allocated by the first call
+
+    def step_host():
+        outs[0] = binding.g10_vitality(tbh, ws=wsh, device=dev, out=outs[0])     # synchronous: results are in host memory on return
+        outs[1] = binding.g10_pressure_timeline(tbh, ws=wsh, device=dev, out=outs[1])
+        return outs[0], outs[1]
+
+    e2e_steps = max(3, args.steps // 4)
+    for _ in range(2):
+        step_host()
     barrier()
     e2e_ms = 0.0
-    for _ in range(args.steps):
+    for _ in range(e2e_steps):
         flush.fill_(1)
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        binding.g10_plan_migrations(tbh, cap, tr.host_bw, tr.ssd_bw, ws=wsh, out=planh, device=dev)   # synchronous
+        vh, th = step_host()
         b.record()
         b.synchronize()
         e2e_ms += a.elapsed_time(b)
-    e2e_total_ms = max_over_ranks(torch, dist if world > 1 else None, world, e2e_ms, dev)
-    e2e_value = aggregate_events_per_s(world, tr.E, args.steps, e2e_total_ms)
-    n_mig = int(planh.summary[0])
-    h2d = tbh.nbytes()
-    d2h = 8 * 8 + 48 * n_mig + 8 * tr.K
+    assert int(vh.counts[0]) == uses and int(th.peak_bytes) == int(tl.peak_bytes.item())
+    e2e_ms = max_over_ranks(torch, dist, world, e2e_ms, dev)
+    e2e_value = aggregate_events_per_s(world, E, e2e_steps, e2e_ms)
+    h2d = 2 * tbh.nbytes()                                            # each of the two calls stages the trace itself
+    d2h = (12 * N + 16 * (N + 1) + 4 * uses + 12 * periods + 24) + (8 * (K + 1) + 8 * K + 8 + 4 + 8)
+    del tbh, wsh, vh, th, outs
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel (the greedy loop).  Algorithmic bytes per launch: every scoring round
-    # reads pressure and duration (16 B) of each slot of each live candidate's absent range, a commit rewrites the
-    # range (16 B per slot) and appends a 48-byte record; counted from the plan itself.
-    mig = binding.migrations_numpy(plan)
-    loop_bytes = plan_loop_algorithmic_bytes(mig)
-    loop_s = stage_ms[3] / 1e3
-    roofline = {"kernel": "k_plan_one", "bound": "hbm", "achieved": loop_bytes / loop_s / 1e9, "peak": hbm_peak,
-                "unit": "GB/s", "frac": loop_bytes / loop_s / 1e9 / hbm_peak, "traffic": PLAN_ONE_DRAM_BYTES, "peak_kind": peak_kind,
-                "algorithmic_bytes": loop_bytes, "kernel_ms": stage_ms[3], "us_per_iteration": stage_ms[3] * 1e3 / max(int(summary[1]), 1),
-                "note": "the whole planner state of this workload (pressure, clock, bookings, %d periods) lives in the shared "
-                        "memory of one SM: the kernel is a chain of %d dependent iterations (search, rescore, commit), bound by "
-                        "latency, not by HBM; the HBM-meaningful fractions are in stress_passes"
-                        % (int(plan_periods(binding, tb, ws)), int(summary[1]))}
+    # ---- each call on its own (cold and warm L2), for the per-call rooflines
+    reps = max(5, args.steps)
+    vit_cold = float(np.median(timed(torch, lambda: binding.g10_vitality(tb, ws=ws), reps, 3, flush)))
+    tl_cold = float(np.median(timed(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), reps, 3, flush)))
+    vit_warm = float(np.median(timed(torch, lambda: binding.g10_vitality(tb, ws=ws), reps, 3, None)))
+    tl_warm = float(np.median(timed(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), reps, 3, None)))
+    sha = kernel_sources_sha256()
+    stale = sha != TRAFFIC["sources_sha256"]
+    traffic_note = {"captured_at": TRAFFIC["captured_at"], "sources_sha256_at_capture": TRAFFIC["sources_sha256"],
+                    "sources_sha256_now": sha, "traffic_stale": stale}
+    roof = roofline(vit_bytes + tl_bytes, step_s, hbm_peak, peak_kind,
+                    kernel="S1-S3: g10_vitality (k_bk_hist, k_bk_scatter, k_bk_emit) + g10_pressure_timeline "
+                           "(k_seg_scan<0>, k_first_last_pairs, k_diff_scatter_pairs, k_seg_scan<1>)",
+                    dominant_kernel="k_bk_emit", traffic=TRAFFIC["vitality"] + TRAFFIC["timeline"], traffic_note=traffic_note,
+                    ms=step_s * 1e3, algorithmic_bytes_per_event=(vit_bytes + tl_bytes) / E,
+                    roofline_events_per_s=E / ((vit_bytes + tl_bytes) / (hbm_peak * 1e9)),
+                    note="random accesses of the passes are bound by the L2's rate of scattered 32-byte sector requests "
+                         "(about 170 G/s measured on this part), not by HBM bytes: see DESIGN.md section 6")
+    passes = {"vitality_ms": vit_cold, "timeline_ms": tl_cold, "vitality_ms_warm_l2": vit_warm, "timeline_ms_warm_l2": tl_warm,
+              "vitality_roofline": roofline(vit_bytes, vit_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["vitality"]),
+              "timeline_roofline": roofline(tl_bytes, tl_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["timeline"]),
+              "repetitions": reps, "l2": "flushed between timed calls (the *_warm_l2 figures: not flushed)"}
+
+    # ---- whole plans, every configuration (median of >= 3 timed calls after warm-up; config 1 with stage events)
+    plans = {}
+    kept = None
+    for cfg in range(5):
+        trc = tr if cfg == 4 else traces.make_config(cfg)
+        n_t, n_w = (3, 1) if cfg == 4 else (max(5, args.steps) if cfg == 1 else 5, 3)
+        st, state = plan_stats(torch, binding, trc, dev, flush, n_t, n_w, stage=(cfg == 1))
+        plans["config%d" % cfg] = st
+        if cfg in (1, 4):
+            kept = kept or {}
+            kept[cfg] = (trc,) + state
+        else:
+            del state
+    plan1 = plans["config1"]
+
+    extras = {}
+    if not args.quick:
+        # ---- the calls behind the plan (Section 4.4) on the finished plans of config 1 and config 4
+        for cfg in (1, 4):
+            trc, tbc, wsc, planc, tlc, capc = kept[cfg]
+            n_mig = int(planc.summary[0].item())
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            P = planc.final_pressure.clone()
+            a.record()
+            pf = binding.g10_schedule_prefetch(trc.K, n_mig, planc.migrations, tlc.kernel_start_ns, tbc.tensor_bytes, capc, P)
+            b.record()
+            torch.cuda.synchronize()
+            vc = binding.g10_vitality(tbc, ws=wsc)
+            torch.cuda.synchronize()
+
+            def emit():
+                return binding.g10_emit_instructions(trc.K, trc.N, vc.first_use, vc.last_use, tbc.tensor_bytes, tbc.tensor_global,
+                                                     tlc.kernel_start_ns, n_mig, planc.migrations, pf.new_prefetch_issue_ns)
+
+            em_ms = float(np.median(timed(torch, emit, 3, 1, flush)))
+            em = emit()
+            torch.cuda.synchronize()
+            n_inst = int(em.counts[0].item())
+            em_bytes = 17 * trc.N + 56 * n_mig + 32 * n_inst + 8 * (trc.K + 2)
+            extras["config%d" % cfg] = {
+                "prefetch_pass": {"ms": a.elapsed_time(b), "moved": int(pf.summary[0].item()), "slots_regained": int(pf.summary[1].item()),
+                                  "note": "single call (it rewrites the pressure curve it is given)"},
+                "instruction_stream": {"ms": em_ms, "instructions": n_inst, "device_status": int(em.counts[1].item()),
+                                       "roofline": roofline(em_bytes, em_ms / 1e3, hbm_peak, peak_kind),
+                                       "note": "the binding allocates the record buffer inside the timed call"}}
+            del pf, em, vc, P
+        # ---- batched re-planning of config 1: one variant per SM, kernel durations jittered by +-10 % (seeded), variant 0 unperturbed
+        trc, tbc, wsc, planc, tlc, capc = kept[1]
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        rng = np.random.default_rng(20231009)
+        base_v = dict(gpu_capacity_bytes=capc, host_bw=trc.host_bw, ssd_bw=trc.ssd_bw)
+        variants = [base_v]
+        for _ in range(sms - 1):
+            f = rng.uniform(0.9, 1.1, size=trc.K)
+            dur = np.maximum(1, np.rint(trc.kernel_ns.astype(np.float64) * f)).astype(np.int64)
+            variants.append(dict(base_v, kernel_ns=torch.from_numpy(dur).to(dev)))
+        wsb = torch.empty(binding.g10_workspace_bytes(binding.WS_BATCH, tbc.K, tbc.N, tbc.E), dtype=torch.uint8, device=dev)
+        mcap = int(planc.summary[0].item()) + 64
+        b_ms = float(np.median(timed(torch, lambda: binding.g10_plan_batch(tbc, variants, ws=wsb, migrations_cap=mcap), 5, 3, flush)))
+        bo = binding.g10_plan_batch(tbc, variants, ws=wsb, migrations_cap=mcap)
+        torch.cuda.synchronize()
+        stab = bo.stability.cpu().numpy().astype(np.float64)
+        extras["batch_replan"] = {"workload": PLAN_WORKLOAD, "variants": len(variants), "ms": b_ms, "plans_per_s": len(variants) / (b_ms / 1e3),
+                                  "trace_events_per_s": len(variants) * trc.E / (b_ms / 1e3), "jitter": "+-10 % per kernel, seeded",
+                                  "mean_jaccard_vs_unperturbed": float(np.mean(stab[1:, 0] / np.maximum(stab[1:, 1], 1))),
+                                  "device_status_or": int(np.bitwise_or.reduce(bo.summary.cpu().numpy()[:, 7]))}
+        del wsb, bo, variants
+        # ---- steady-state (cyclic) plan of config 1
+        c_ms = float(np.median(timed(torch, lambda: binding.g10_plan_cyclic(tbc, capc, trc.host_bw, trc.ssd_bw, ws=wsc), 5, 3, flush)))
+        cp = binding.g10_plan_cyclic(tbc, capc, trc.host_bw, trc.ssd_bw, ws=wsc)
+        torch.cuda.synchronize()
+        cs = cp.summary.cpu().numpy()
+        extras["cyclic_plan"] = {"workload": PLAN_WORKLOAD, "plan_ms": c_ms, "migrations": int(cs[0]), "status": binding.STATUS.get(int(cs[2]), "?"),
+                                 "final_peak_bytes": int(cs[3]), "final_peak_bytes_acyclic": int(planc.summary[3].item()), "device_status": int(cs[7])}
+        del cp
+    kept = None
+    torch.cuda.empty_cache()
+
+    # ---- the two analysis calls on the stress trace eight (and four) times over: fixed cost against throughput
+    scale = {}
+    if not args.quick:
+        for times in (4, 8):
+            scale["x%d" % times] = scaled_passes(torch, binding, tb, times, flush, hbm_peak, peak_kind)
 
     line = {
         "metric": "trace_events_per_s", "value": value, "unit": "events/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": total_s / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "trace_sha256": tr.sha256(), "K": tr.K, "N": tr.N, "E": tr.E,
-                   "periods": int(plan_periods(binding, tb, ws)),
-                   "gpu_capacity_bytes": cap, "host_bw": tr.host_bw, "ssd_bw": tr.ssd_bw,
-                   "migrations": int(summary[0]), "scoring_rounds": int(summary[1]), "status": binding.STATUS[int(summary[2])],
+        "config": {"workload": WORKLOAD, "step": "S1-S3: one g10_vitality call + one g10_pressure_timeline call, trace resident in HBM",
+                   "trace_sha256": tr.sha256(), "K": K, "N": N, "E": E, "uses": uses, "periods": periods,
                    "l2": "flushed between timed iterations (%d MiB write)" % (L2_FLUSH_BYTES >> 20),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "plan_ms": total_s / args.steps * 1e3,
-        "stage_ms": {"clock_vitality": stage_ms[0], "pressure": stage_ms[1], "geometry": stage_ms[2], "greedy_loop": stage_ms[3]},
-        "passes": {"vitality_ms": vit_s / args.steps * 1e3, "timeline_ms": tl_s / args.steps * 1e3,
-                   "vitality_timeline_events_per_s": tr.E / ((vit_s + tl_s) / args.steps)},
+        "plan_ms": plan1["plan_ms"], "plan_workload": PLAN_WORKLOAD,
+        "plan_greedy_loop": {"kernel": "k_plan_one", "bound": "latency", "ms": plan1.get("greedy_loop_ms"),
+                             "us_per_iteration": plan1.get("greedy_loop_us_per_iteration"), "iterations": plan1["iterations"],
+                             "note": "the planner state of this workload lives in the shared memory of one SM: a chain of dependent "
+                                     "iterations (search, rescore, commit); reported per iteration, an HBM fraction would mean nothing"},
+        "plans": plans,
+        "passes": passes,
         "e2e": {"value": e2e_value, "unit": "events/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_total_ms / args.steps},
-        "prefetch_pass": {"ms": prefetch_ms, "moved": int(pf_summary[0]), "slots_regained": int(pf_summary[1]),
-                          "peak_after": int(pf_summary[2]), "note": "plan + pass timed together, plan time subtracted"},
-        "batch_replan": batch,
-        "cyclic_plan": cyclic,
-        "gpu_launches": args.steps * KERNELS_PER_PLAN,
+                "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
+                "note": "host-pointer form of both calls: each stages the trace itself and copies all its outputs back"},
+        "gpu_launches": args.steps * (KERNELS_PER_VITALITY + KERNELS_PER_TIMELINE),
+        "gpu_launches_note": "kernels of this library inside the timed region: %d per g10_vitality + %d per g10_pressure_timeline, "
+                             "from the ncu launch list in profiles/ (plus one memset node per call)" % (KERNELS_PER_VITALITY, KERNELS_PER_TIMELINE),
         "clocks": clocks,
-        "roofline": roofline,
+        "roofline": roof,
+        "behind_the_plan": extras,
+        "scale": scale,
     }
-    if not args.no_stress and world == 1:
-        line["stress_passes"] = stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, args.stress_reps)
     line["cpu_baseline"] = cpu_baseline(tr)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
-
-
-def plan_periods(binding, tb, ws):
-    import torch
-    v = binding.g10_vitality(tb, ws=ws)
-    torch.cuda.synchronize()
-    return int(v.counts[1].item())
-
-
-def plan_loop_algorithmic_bytes(mig):
-    """Bytes the greedy loop cannot avoid touching, counted from the plan itself: per commit the winner's absent
-    range is rescored once (pressure + duration, 16 B per slot) and rewritten once (16 B per slot), plus the
-    48-byte record.  Rescoring of periods that do not win is bookkeeping of the search, not algorithmic traffic."""
-    slots = int((mig["absent_last"].astype(np.int64) - mig["absent_first"].astype(np.int64) + 1).sum())
-    return 32 * slots + 48 * len(mig)
-
-
-def stress_passes(torch, binding, dev, flush, hbm_peak, peak_kind, reps=20):
-    """Vitality and timeline passes on the 1M-kernel / 4M-tensor stress trace (config 4): the only workload whose
-    arrays are large enough for an HBM fraction to mean something.  Algorithmic bytes: vitality reads kernel_ptr
-    (8K) and kernel_tensors (4E) and writes first/last/num_uses (12N), use_ptr (8N), uses (4E'), period_ptr (8N)
-    and the periods (12 Pn); the timeline reads kernel_ns (8K), tensor_bytes (8N), first/last (8N), the global flag
-    (N) and writes start (8K) and pressure (8K)."""
-    tr = traces.config4_stress_dag()
-    tb = binding.upload(tr, dev)
-    ws = torch.empty(binding.g10_workspace_bytes(binding.WS_PLAN, tb.K, tb.N, tb.E), dtype=torch.uint8, device=dev)
-    v = binding.g10_vitality(tb, ws=ws)
-    torch.cuda.synchronize()
-    e2, pn = int(v.counts[0].item()), int(v.counts[1].item())
-    K, N, E = tr.K, tr.N, tr.E
-    vit_bytes = 8 * K + 4 * E + 12 * N + 8 * N + 4 * e2 + 8 * N + 12 * pn
-    tl_bytes = 8 * K + 8 * N + 8 * N + N + 8 * K + 8 * K
-    steps, warm = reps, 3
-    vit_s = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), steps, warm, flush) / steps
-    tl_s = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), steps, warm, flush) / steps
-    no_flush = torch.empty(1, dtype=torch.uint8, device=dev)      # warm-L2 numbers: nothing written between the calls
-    vit_w = time_calls(torch, lambda: binding.g10_vitality(tb, ws=ws), steps, warm, no_flush) / steps
-    tl_w = time_calls(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), steps, warm, no_flush) / steps
-    out = {
-        "workload": "config4_stress_dag", "K": K, "N": N, "E": E, "uses": e2, "periods": pn,
-        "vitality_ms": vit_s * 1e3, "timeline_ms": tl_s * 1e3, "repetitions": steps,
-        "vitality_ms_warm_l2": vit_w * 1e3, "timeline_ms_warm_l2": tl_w * 1e3,
-        "events_per_s": E / (vit_s + tl_s),
-        "vitality_roofline": {"bound": "hbm", "achieved": vit_bytes / vit_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                              "frac": vit_bytes / vit_s / 1e9 / hbm_peak, "frac_of_nominal_8000": vit_bytes / vit_s / 1e9 / 8000.0,
-                              "algorithmic_bytes": vit_bytes, "traffic": STRESS_VITALITY_DRAM_BYTES,
-                              "peak_kind": peak_kind},
-        "timeline_roofline": {"bound": "hbm", "achieved": tl_bytes / tl_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                              "frac": tl_bytes / tl_s / 1e9 / hbm_peak, "frac_of_nominal_8000": tl_bytes / tl_s / 1e9 / 8000.0,
-                              "algorithmic_bytes": tl_bytes, "traffic": STRESS_TIMELINE_DRAM_BYTES,
-                              "peak_kind": peak_kind},
-        "l2": "flushed between timed calls (the *_warm_l2 figures: not flushed)",
-    }
-    # the whole plan of the stress trace (capacity = 3/10 of the unplanned peak), once
-    tl = binding.g10_pressure_timeline(tb, ws=ws)
-    torch.cuda.synchronize()
-    # characterisation statistics (Section 3): reads use_ptr (8N), uses (4E'), tensor_bytes (8N), the periods (12 Pn)
-    # and two clock entries per period (16 Pn), one 8-byte atomic per use (8E') into active_bytes (8K)
-    st_bytes = 8 * N + 4 * e2 + 8 * N + 12 * pn + 16 * pn + 8 * e2 + 8 * K
-    st_s = time_calls(torch, lambda: binding.g10_characterize(K, N, v.use_ptr, v.uses, tb.tensor_bytes, tl.kernel_start_ns, pn,
-                                                              v.period_tensor, v.period_prev_use, v.period_next_use,
-                                                              tr.host_bw, tr.ssd_bw), steps, warm, flush) / steps
-    out["characterize_ms"] = st_s * 1e3
-    out["characterize_roofline"] = {"bound": "hbm", "achieved": st_bytes / st_s / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                                    "frac": st_bytes / st_s / 1e9 / hbm_peak, "frac_of_nominal_8000": st_bytes / st_s / 1e9 / 8000.0,
-                                    "algorithmic_bytes": st_bytes, "peak_kind": peak_kind}
-    cap = tr.capacity_from_peak(int(tl.peak_bytes.item()))
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    plan = binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, ws=ws)
-    b.record()
-    torch.cuda.synchronize()
-    ps = plan.summary.cpu().numpy()
-    out["plan"] = {"plan_ms": a.elapsed_time(b), "migrations": int(ps[0]), "status": binding.STATUS.get(int(ps[2]), "?"),
-                   "device_status": int(ps[7]), "capacity_bytes": cap}
-    # Section 4.4 on the finished plan: the eager prefetch pass (once: it rewrites the pressure curve), then the
-    # instruction stream (alloc / free for every tensor, pre-evict / prefetch for every migration), three times
-    n_mig = int(ps[0])
-    a.record()
-    pf = binding.g10_schedule_prefetch(K, n_mig, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap, plan.final_pressure)
-    b.record()
-    torch.cuda.synchronize()
-    out["prefetch_pass"] = {"ms": a.elapsed_time(b), "moved": int(pf.summary[0].item()), "slots_regained": int(pf.summary[1].item())}
-    em_s = time_calls(torch, lambda: binding.g10_emit_instructions(K, N, v.first_use, v.last_use, tb.tensor_bytes, tb.tensor_global,
-                                                                   tl.kernel_start_ns, n_mig, plan.migrations, pf.new_prefetch_issue_ns),
-                      3, 1, flush) / 3
-    em = binding.g10_emit_instructions(K, N, v.first_use, v.last_use, tb.tensor_bytes, tb.tensor_global, tl.kernel_start_ns, n_mig,
-                                       plan.migrations, pf.new_prefetch_issue_ns)
-    torch.cuda.synchronize()
-    n_inst = int(em.counts[0].item())
-    em_bytes = 8 * N + 8 * N + N + 48 * n_mig + 8 * n_mig + 32 * n_inst + 8 * (K + 2)
-    out["instruction_stream"] = {"ms": em_s * 1e3, "instructions": n_inst, "device_status": int(em.counts[1].item()),
-                                 "algorithmic_bytes": em_bytes, "achieved_gbs": em_bytes / em_s / 1e9,
-                                 "frac": em_bytes / em_s / 1e9 / hbm_peak, "peak_kind": peak_kind,
-                                 "note": "binding allocates the 257 MB record buffer inside the timed call"}
-    del tb, ws, v, plan, tl, pf, em
-    torch.cuda.empty_cache()
-    return out
 
 
 def cpu_model():
@@ -468,35 +545,25 @@ def cpu_model():
 
 
 def cpu_baseline(tr):
-    """The oracle (plain tier, one thread) on the same workload, bounded to roughly ten seconds."""
+    """The oracle on the same workload, one thread: three whole passes S1-S3 over the stress trace (about fifteen seconds),
+    then the config-1 plan with both of its tiers."""
     from oracle import g10_oracle as O
     O.build()
-    start, P0, peak, slot = O.timeline(tr)
-    cap = tr.capacity_from_peak(peak)
-    O.plan(tr, cap)
-    reps, t0 = 0, time.perf_counter()
-    while time.perf_counter() - t0 < 10.0 and reps < 200:
-        O.plan(tr, cap)
-        reps += 1
+    t0 = time.perf_counter()
+    reps = 3
+    for _ in range(reps):
+        oracle_s123(O, tr)
     dt = time.perf_counter() - t0
-    # the analysis passes alone (slot clock, vitality, pressure), median of three
-    ts = []
+    tr1 = traces.config1_resnet152()
+    cap = tr1.capacity_from_peak(0)
+    ts, tl_ = [], []
     for _ in range(3):
-        t1 = time.perf_counter()
-        O.timeline(tr)
-        ts.append(time.perf_counter() - t1)
-    passes_s = sorted(ts)[1]
-    # the oracle's lazy tier (same plan, periods rescored only when their bound is on top of a heap), median of three
-    tl_ = []
-    for _ in range(3):
-        t1 = time.perf_counter()
-        O.plan(tr, cap, lazy=True)
-        tl_.append(time.perf_counter() - t1)
-    lazy_s = sorted(tl_)[1]
-    return {"value": tr.E * reps / dt, "unit": "events/s", "cores": 1, "kind": "oracle", "lazy_tier_plan_ms": lazy_s * 1e3,
-            "vitality_timeline_events_per_s": tr.E / passes_s,
-            "sample": "whole config-1 plan (plain tier), %d repetitions in %.1f s" % (reps, dt),
-            "plan_ms": dt / reps * 1e3, "host_cores_available": os.cpu_count(), "cpu_model": cpu_model()}
+        t1 = time.perf_counter(); O.plan(tr1, cap); ts.append(time.perf_counter() - t1)
+        t1 = time.perf_counter(); O.plan(tr1, cap, lazy=True); tl_.append(time.perf_counter() - t1)
+    return {"value": tr.E * reps / dt, "unit": "events/s", "cores": 1, "kind": "oracle",
+            "sample": "%d whole passes S1-S3 (vitality, slot clock, plain-definition pressure) over config 4 in %.1f s" % (reps, dt),
+            "ms_per_step": dt / reps * 1e3, "plan_ms_config1_plain_tier": sorted(ts)[1] * 1e3, "plan_ms_config1_lazy_tier": sorted(tl_)[1] * 1e3,
+            "host_cores_available": os.cpu_count(), "cpu_model": cpu_model()}
 
 
 def main():
@@ -505,22 +572,11 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-stress", action="store_true", help="skip the config-4 pass measurements")
-    ap.add_argument("--stress-only", action="store_true",
-                    help="only time the vitality / timeline passes on config 4 (small profiling target)")
-    ap.add_argument("--stress-reps", type=int, default=20)
+    ap.add_argument("--quick", action="store_true", help="headline, plans and per-call rooflines only (small profiling target)")
     args = ap.parse_args()
-    if args.warmup < 3:
+    if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    if args.stress_only:
-        import torch
-        from paper_2310_09443_b200 import binding, build
-        build.build()
-        torch.cuda.set_device(0)
-        flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda:0")
-        hbm_peak, peak_kind = measured_peaks()
-        print(json.dumps({"stress_passes": stress_passes(torch, binding, "cuda:0", flush, hbm_peak, peak_kind, args.stress_reps)}))
-    elif args.impl == "reference":
+    if args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -229,39 +229,40 @@ def _alloc(tb, shape, dtype, device):
     return torch.empty(shape, dtype=dtype).pin_memory()
 
 
-def g10_vitality(tb: TraceBuffers, ws=None, stream=None, device=None, uses_cap=None, periods_cap=None):
+def g10_vitality(tb: TraceBuffers, ws=None, stream=None, device=None, uses_cap=None, periods_cap=None, out=None):
     """Section 4.2 tensor vitality analysis.  Returns tensors in the memory space of `tb`; in device mode the
-    call is asynchronous on `stream` (trim `uses` / the period arrays with counts after synchronising)."""
+    call is asynchronous on `stream` (trim `uses` / the period arrays with counts after synchronising).
+    `out`: the result of an earlier call on a trace of the same sizes, to write into instead of allocating."""
     lib = load_library()
     ucap = tb.E if uses_cap is None else uses_cap
     pcap = tb.E if periods_cap is None else periods_cap
-    r = SimpleNamespace(
+    r = out if out is not None else SimpleNamespace(
         first_use=_alloc(tb, tb.N, torch.int32, device), last_use=_alloc(tb, tb.N, torch.int32, device),
         num_uses=_alloc(tb, tb.N, torch.int32, device), use_ptr=_alloc(tb, tb.N + 1, torch.int64, device),
         uses=_alloc(tb, max(ucap, 1), torch.int32, device), period_ptr=_alloc(tb, tb.N + 1, torch.int64, device),
         period_tensor=_alloc(tb, max(pcap, 1), torch.int32, device), period_prev_use=_alloc(tb, max(pcap, 1), torch.int32, device),
         period_next_use=_alloc(tb, max(pcap, 1), torch.int32, device), counts=_alloc(tb, 3, torch.int64, device))
     ws, ws_bytes = _workspace(tb, WS_VITALITY, ws, device)
-    out = _VitalityOut(_ptr(r.first_use), _ptr(r.last_use), _ptr(r.num_uses), _ptr(r.use_ptr), _ptr(r.uses), ucap,
+    vo = _VitalityOut(_ptr(r.first_use), _ptr(r.last_use), _ptr(r.num_uses), _ptr(r.use_ptr), _ptr(r.uses), ucap,
                        _ptr(r.period_ptr), _ptr(r.period_tensor), _ptr(r.period_prev_use), _ptr(r.period_next_use), pcap,
                        _ptr(r.counts))
     tr = tb.c_struct()
-    _check(lib.g10_vitality(C.byref(tr), C.byref(out), _ptr(ws), ws_bytes, _stream(stream)))
+    _check(lib.g10_vitality(C.byref(tr), C.byref(vo), _ptr(ws), ws_bytes, _stream(stream)))
     r.workspace = ws
     return r
 
 
-def g10_pressure_timeline(tb: TraceBuffers, ws=None, stream=None, device=None):
-    """Section 4.3 memory-pressure timeline before any migration."""
+def g10_pressure_timeline(tb: TraceBuffers, ws=None, stream=None, device=None, out=None):
+    """Section 4.3 memory-pressure timeline before any migration.  `out`: an earlier result to write into."""
     lib = load_library()
-    r = SimpleNamespace(
+    r = out if out is not None else SimpleNamespace(
         kernel_start_ns=_alloc(tb, tb.K + 1, torch.int64, device), pressure=_alloc(tb, max(tb.K, 1), torch.int64, device),
         peak_bytes=_alloc(tb, 1, torch.int64, device), peak_slot=_alloc(tb, 1, torch.int32, device),
         status=_alloc(tb, 1, torch.int64, device))
     ws, ws_bytes = _workspace(tb, WS_TIMELINE, ws, device)
-    out = _TimelineOut(_ptr(r.kernel_start_ns), _ptr(r.pressure), _ptr(r.peak_bytes), _ptr(r.peak_slot), _ptr(r.status))
+    to = _TimelineOut(_ptr(r.kernel_start_ns), _ptr(r.pressure), _ptr(r.peak_bytes), _ptr(r.peak_slot), _ptr(r.status))
     tr = tb.c_struct()
-    _check(lib.g10_pressure_timeline(C.byref(tr), C.byref(out), _ptr(ws), ws_bytes, _stream(stream)))
+    _check(lib.g10_pressure_timeline(C.byref(tr), C.byref(to), _ptr(ws), ws_bytes, _stream(stream)))
     r.workspace = ws
     return r
 

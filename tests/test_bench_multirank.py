@@ -43,4 +43,4 @@ def test_reference_arm_runs_on_cpu():
     import json
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["metric"] == "trace_events_per_s" and line["value"] > 0
-    assert line["config"]["workload"] == "config1_resnet152_b256" and line["cpu_baseline"]["kind"] == "oracle"
+    assert line["config"]["workload"] == "config4_stress_dag" and line["plan_workload"] == "config1_resnet152_b256" and line["cpu_baseline"]["kind"] == "oracle"
