@@ -161,6 +161,14 @@ typedef struct g10_options {
 #define G10_FLAG_MULTI_BLOCK 0x4    /* never let a single block run the greedy loop out of its shared memory (the path
                                        the smallest traces take); same plan                                  */
 
+#ifdef G10_TEST_HOOKS
+/* Honoured only by the test build of the library (compiled with -DG10_TEST_HOOKS, never shipped): one block of the
+   planner's cooperative grid skips its first grid-barrier arrival and every barrier wait of the call is limited to a
+   millisecond, so that the give-up path of the bounded waits can be exercised: the call returns with
+   G10_DEV_TIMEOUT in summary[7].  The product build ignores the bit. */
+#define G10_FLAG_TEST_SKIP_ARRIVAL 0x40000000
+#endif
+
 #define G10_WS_VITALITY 0
 #define G10_WS_TIMELINE 1
 #define G10_WS_PLAN 2

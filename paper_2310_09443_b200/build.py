@@ -12,8 +12,9 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
-OBJ = os.path.join(HERE, "build")
-LIB = os.path.join(HERE, "libg10.so")
+OBJ_PLAIN, OBJ_HOOKS = os.path.join(HERE, "build"), os.path.join(HERE, "build_hooks")
+LIB_PLAIN, LIB_HOOKS = os.path.join(HERE, "libg10.so"), os.path.join(HERE, "libg10_hooks.so")
+LIB = LIB_PLAIN
 SOURCES = ["g10_api.cu", "g10_passes.cu", "g10_planner.cu", "g10_planner_lazy.cu", "g10_planner_small.cu",
            "g10_planner_one.cu", "g10_vitality_buckets.cu", "g10_prefetch.cu", "g10_emit.cu", "g10_stats.cu", "g10_cyclic.cu",
            "g10_static.cu"]
@@ -25,8 +26,12 @@ def _newer(path: str, than: float) -> bool:
     return os.path.getmtime(path) > than
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, hooks: bool = False) -> str:
+    """hooks=True builds libg10_hooks.so instead: the same sources with -DG10_TEST_HOOKS (used by one test that makes a
+    bounded device wait run out; never loaded by the binding)."""
     nvcc = os.environ.get("NVCC", "nvcc")
+    OBJ, LIB = (OBJ_HOOKS, LIB_HOOKS) if hooks else (OBJ_PLAIN, LIB_PLAIN)
+    flags = NVCC_FLAGS + (["-DG10_TEST_HOOKS"] if hooks else [])
     headers = [os.path.join(CSRC, h) for h in HEADERS] + [os.path.join(ROOT, "include", "g10.h"), os.path.abspath(__file__)]
     os.makedirs(OBJ, exist_ok=True)
     sources = [f for f in SOURCES if os.path.exists(os.path.join(CSRC, f))]
@@ -39,7 +44,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     def compile_one(job):
         src, obj = job
         tmp = "%s.%d.tmp" % (obj, os.getpid())          # several processes may build at once: each renames a finished file
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-I" + os.path.join(ROOT, "include"), "-c", "-o", tmp, src]
+        cmd = [nvcc] + flags + (["-Xptxas", "-v"] if verbose else []) + ["-I" + os.path.join(ROOT, "include"), "-c", "-o", tmp, src]
         try:
             subprocess.check_call(cmd)
             os.replace(tmp, obj)
@@ -63,4 +68,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, hooks="--hooks" in sys.argv))

@@ -2,6 +2,7 @@
 #include <cstring>
 #include <vector>
 
+#include "g10_device.cuh"
 #include "g10_internal.h"
 
 namespace g10 {
@@ -508,6 +509,12 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
     rc = begin_call(trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff | (plan_keeps_state_on_chip(trace->num_kernels, trace->num_events, flags) ? 0 : kZeroState));
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
+#ifdef G10_TEST_HOOKS
+    if (flags & G10_FLAG_TEST_SKIP_ARRIVAL) {        // (test build: block 1 skips its first barrier arrival, waits give up after 1 ms)
+        static const unsigned hook = 2u;
+        CU(cudaMemcpyAsync(&((GridBarrier *)w.barrier)->pad, &hook, sizeof(hook), cudaMemcpyHostToDevice, s));
+    }
+#endif
     VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
                        w.period_tensor, w.period_prev_use, w.period_next_use, d.E, w.counts};
     PlanParams pp;

@@ -246,12 +246,26 @@ __device__ __forceinline__ bool grid_barrier(GridBarrier *b, unsigned nblocks, u
         // (no look at the error word before arriving: a block that arrives after another one gave up finds the word
         // set at its next check while polling, which costs one round trip less on every barrier that succeeds)
         unsigned ok = 1u;
+        ull limit_ns = kBarrierTimeoutNs;
+        bool arrive = true;
+#ifdef G10_TEST_HOOKS
+        // Test build only: in a call made with G10_FLAG_TEST_SKIP_ARRIVAL block (pad - 1) never arrives at a barrier (its
+        // own barrier calls fail at once) and every wait of the call gives up after a millisecond: the other blocks find
+        // that nobody completes the barrier, set the error word, and the kernel winds down with G10_DEV_TIMEOUT.
+        const unsigned hook = *(volatile unsigned *)&b->pad;
+        if (hook) {
+            limit_ns = 1000000ull;
+            if (blockIdx.x == hook - 1u) { arrive = false; ok = 0u; }
+        }
+#endif
         // arrival is an acquire-release add (it publishes this block's writes, ordered before it by the block barrier
         // above, and the last arrival has acquired everyone's); the generation is stored with release and polled with
         // acquire: no separate fences
-        unsigned arrived;
-        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(&b->count) : "memory");
-        if (arrived == nblocks - 1u) {
+        unsigned arrived = 0u;
+        if (arrive) asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(&b->count) : "memory");
+        if (!arrive) {
+            // (test build: this block does not arrive; ok is already 0)
+        } else if (arrived == nblocks - 1u) {
             b->count = 0u;
             st_release_u32(&b->gen, my_gen + 1u);
         } else {
@@ -260,7 +274,7 @@ __device__ __forceinline__ bool grid_barrier(GridBarrier *b, unsigned nblocks, u
             while (ld_acquire_u32(&b->gen) == my_gen) {
                 if ((++polls & 1023u) == 0u) {
                     if (ld_acquire_u32(&b->error)) { ok = 0u; break; }
-                    if (global_timer_ns() - t0 > kBarrierTimeoutNs) { atomicExch(&b->error, 1u); ok = 0u; break; }
+                    if (global_timer_ns() - t0 > limit_ns) { atomicExch(&b->error, 1u); ok = 0u; break; }
                 }
             }
         }
