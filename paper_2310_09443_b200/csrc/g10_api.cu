@@ -37,10 +37,14 @@ void carve_scan(Carver &c, ScanSlot &s, int64_t tiles, int nv)
     s.incl = c.take<long long>((size_t)tiles * nv);
 }
 
-size_t carve(void *base, const Sizes &z, Workspace &w)
+// `which` (G10_WS_*) decides what is laid out: the timeline call needs neither the partition scratch of the vitality
+// call nor the planner's state, the vitality call no timeline arrays; the planner calls need everything.
+size_t carve(void *base, const Sizes &z, Workspace &w, int32_t which)
 {
     std::memset(&w, 0, sizeof(w));
     Carver c(base);
+    const bool vit = which != G10_WS_TIMELINE, tl = which != G10_WS_VITALITY, plan = which != G10_WS_TIMELINE && which != G10_WS_VITALITY;
+    const bool inner = plan || z.host;             // results of the analysis calls kept inside the workspace
     const size_t K = (size_t)z.K, N = (size_t)z.N, E = (size_t)z.E;
     const size_t heavy = E / (kHeavyThreshold + 1) + 1;
     const int64_t ktiles = tiles_of(z.K, 2048), ntiles = tiles_of(z.N, 2048), etiles = tiles_of(z.N, 1024);
@@ -51,77 +55,77 @@ size_t carve(void *base, const Sizes &z, Workspace &w)
     w.peak_key = c.take<int>(1);
     w.barrier = c.take<unsigned>(4);
     carve_scan(c, w.clock_scan, ktiles, 1);
-    carve_scan(c, w.count_scan, ntiles, 1);
-    carve_scan(c, w.emit_scan, etiles, 2);
+    carve_scan(c, w.count_scan, vit ? ntiles : 1, 1);
+    carve_scan(c, w.emit_scan, vit ? etiles : 1, 2);
     carve_scan(c, w.pressure_scan, ktiles, 1);
     w.wl_count = c.take<unsigned>(2);
     w.one_done = c.take<unsigned>(1);
     w.event_budget = c.take<ull>(1);
-    w.bk_count = c.take<unsigned>(4096);
-    w.bk_cursor = c.take<unsigned>(4096);
-    w.bk_words = c.take<ull>(2 * 4096);
-    w.xwords = c.take<ull>((2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16);
+    w.bk_count = c.take<unsigned>(vit ? 4096 : 1);
+    w.bk_cursor = c.take<unsigned>(vit ? 4096 : 1);
+    w.bk_words = c.take<ull>(vit ? 2 * 4096 : 1);
+    w.xwords = c.take<ull>(plan ? (2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16 : 1);
     w.seg_words = c.take<ull>(512 * 16);
     w.seg_words2 = c.take<ull>(512 * 16);
     w.zero_bytes = align_up(c.off);
     // arrays that must start at zero, cleared only by the calls that use them (the difference array sits right behind
     // the zero-initialised region, so that one memset covers both)
-    w.diff = c.take<int64_t>(K + 1);
-    w.tl_point = c.take<int64_t>(K);
-    w.tl_pair = c.take<int>(2 * N);           // (both right behind the difference array: the timeline call clears both with the same memset)
-    w.cnt = c.take<int32_t>(N);
+    w.diff = c.take<int64_t>(tl ? K + 1 : 1);
+    w.tl_point = c.take<int64_t>(which == G10_WS_TIMELINE ? K : 1);
+    w.tl_pair = c.take<int>(which == G10_WS_TIMELINE ? 2 * N : 1);   // (both right behind the difference array: the timeline call clears all three with one memset)
+    w.cnt = c.take<int32_t>(vit ? N : 1);
     const size_t state_begin = align_up(c.off);
-    w.busy = c.take<int64_t>(4 * K);       // busy, hocc and dead are contiguous: one memset
-    w.hocc = c.take<int64_t>(K);
-    w.dead = c.take<unsigned char>(E);
+    w.busy = c.take<int64_t>(plan ? 4 * K : 1);       // busy, hocc and dead are contiguous: one memset
+    w.hocc = c.take<int64_t>(plan ? K : 1);
+    w.dead = c.take<unsigned char>(plan ? E : 1);
     w.state_bytes = align_up(c.off) - state_begin;
     // scratch
-    w.raw_ptr = c.take<int32_t>(N + 1);
-    w.raw_uses = c.take<int32_t>(E);
-    w.heavy_list = c.take<int32_t>(heavy);
-    w.heavy_info = c.take<int32_t>(2 * heavy);
+    w.raw_ptr = c.take<int32_t>(vit ? N + 1 : 1);
+    w.raw_uses = c.take<int32_t>(vit ? E : 1);
+    w.heavy_list = c.take<int32_t>(vit ? heavy : 1);
+    w.heavy_info = c.take<int32_t>(vit ? 2 * heavy : 1);
     w.tile_max = c.take<int64_t>((size_t)ktiles);
     w.tile_slot = c.take<int32_t>((size_t)ktiles);
-    w.first_use = c.take<int32_t>(N);
-    w.last_use = c.take<int32_t>(N);
-    w.num_uses = c.take<int32_t>(N);
-    w.use_ptr = c.take<int64_t>(N + 1);
-    w.period_ptr = c.take<int64_t>(N + 1);
-    w.uses = c.take<int32_t>(E);
-    w.period_tensor = c.take<int32_t>(E);
-    w.period_prev_use = c.take<int32_t>(E);
-    w.period_next_use = c.take<int32_t>(E);
+    w.first_use = c.take<int32_t>(vit && inner ? N : 1);
+    w.last_use = c.take<int32_t>(vit && inner ? N : 1);
+    w.num_uses = c.take<int32_t>(vit && inner ? N : 1);
+    w.use_ptr = c.take<int64_t>(vit && inner ? N + 1 : 1);
+    w.period_ptr = c.take<int64_t>(vit && inner ? N + 1 : 1);
+    w.uses = c.take<int32_t>(vit && inner ? E : 1);
+    w.period_tensor = c.take<int32_t>(vit && inner ? E : 1);
+    w.period_prev_use = c.take<int32_t>(vit && inner ? E : 1);
+    w.period_next_use = c.take<int32_t>(vit && inner ? E : 1);
     w.counts = c.take<int64_t>(4);
-    w.start = c.take<int64_t>(K + 1);
-    w.start2 = c.take<int64_t>(2 * K + 1);
-    w.pressure = c.take<int64_t>(K);
+    w.start = c.take<int64_t>(tl && inner ? K + 1 : 1);
+    w.start2 = c.take<int64_t>(plan ? 2 * K + 1 : 1);
+    w.pressure = c.take<int64_t>(tl && inner ? K : 1);
     w.peak_bytes = c.take<int64_t>(1);
     w.peak_slot = c.take<int32_t>(2);
-    w.geo_t = c.take<int64_t>(2 * E);
-    w.geo_a = c.take<int32_t>(2 * E);
-    w.geo_b = c.take<int32_t>(2 * E);
-    w.proposals = c.take<Proposal>(kMaxPlanBlocks);
-    w.prop_stale = c.take<Proposal>(kMaxPlanBlocks);
-    w.lazy_props = c.take<LazyProp>(2 * kLazyMaxBlocks);
-    w.lazy_partials = c.take<ull>((size_t)2 * kRoundM * kLazyMaxBlocks * 2);
-    w.lazy_tmin = c.take<int64_t>((size_t)tiles_of(z.K, 1024));
-    w.lazy_tmax = c.take<int64_t>((size_t)tiles_of(z.K, 1024));
-    w.c_state = c.take<unsigned char>(E);
-    w.c_ben_lo = c.take<ull>(E);
-    w.c_ben_hi = c.take<ull>(E);
-    w.c_cost = c.take<ull>(E);
-    w.c_key = c.take<double>(E);
-    w.worklist = c.take<int>(2 * E);
-    w.bk_pairs = c.take<ull>(E);
-    if (z.K <= kSmallMaxSlots) {
+    w.geo_t = c.take<int64_t>(plan ? 2 * E : 1);
+    w.geo_a = c.take<int32_t>(plan ? 2 * E : 1);
+    w.geo_b = c.take<int32_t>(plan ? 2 * E : 1);
+    w.proposals = c.take<Proposal>(plan ? kMaxPlanBlocks : 1);
+    w.prop_stale = c.take<Proposal>(plan ? kMaxPlanBlocks : 1);
+    w.lazy_props = c.take<LazyProp>(plan ? 2 * kLazyMaxBlocks : 1);
+    w.lazy_partials = c.take<ull>(plan ? (size_t)2 * kRoundM * kLazyMaxBlocks * 2 : 1);
+    w.lazy_tmin = c.take<int64_t>(plan ? (size_t)tiles_of(z.K, 1024) : 1);
+    w.lazy_tmax = c.take<int64_t>(plan ? (size_t)tiles_of(z.K, 1024) : 1);
+    w.c_state = c.take<unsigned char>(plan ? E : 1);
+    w.c_ben_lo = c.take<ull>(plan ? E : 1);
+    w.c_ben_hi = c.take<ull>(plan ? E : 1);
+    w.c_cost = c.take<ull>(plan ? E : 1);
+    w.c_key = c.take<double>(plan ? E : 1);
+    w.worklist = c.take<int>(plan ? 2 * E : 1);
+    w.bk_pairs = c.take<ull>(vit ? E : 1);
+    if (plan && z.K <= kSmallMaxSlots) {
         w.busy_rep = c.take<int64_t>((size_t)kSmallMaxBlocks * 4 * K);
         w.hocc_rep = c.take<int64_t>((size_t)kSmallMaxBlocks * K);
     }
-    w.peak_part = c.take<int64_t>(kMaxPlanBlocks);
+    w.peak_part = c.take<int64_t>(plan ? kMaxPlanBlocks : 1);
     w.summary = c.take<int64_t>(8);
-    w.batch_variants = c.take<BatchVariant>(kMaxVariants);
+    w.batch_variants = c.take<BatchVariant>(which == G10_WS_BATCH ? kMaxVariants : 1);
     if (z.host) {
-        w.migrations = c.take<g10_migration>(E);
+        w.migrations = c.take<g10_migration>(plan ? E : 1);
         w.s_kernel_ptr = c.take<int64_t>(K + 1);
         w.s_kernel_tensors = c.take<int32_t>(E);
         w.s_tensor_bytes = c.take<int64_t>(N);
@@ -163,10 +167,10 @@ int32_t check_ws(int32_t which, const g10_trace *t, void *ws, size_t ws_bytes)
 // Prepares the workspace and returns the device view of the trace (staging it first in host mode).
 enum { kZeroCounts = 1, kZeroDiff = 2, kZeroState = 4, kZeroPairs = 8 };
 
-int32_t begin_call(const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, cudaStream_t s, int zero_mask)
+int32_t begin_call(int32_t which, const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, cudaStream_t s, int zero_mask)
 {
     Sizes z{t->num_kernels, t->num_tensors, t->num_events, t->mem == G10_MEM_HOST};
-    carve(ws, z, w);
+    carve(ws, z, w, which);
     {
         size_t head = w.zero_bytes;
         if (zero_mask & kZeroDiff) head = (size_t)((char *)(w.diff + z.K + 1) - w.zero_begin);
@@ -250,10 +254,9 @@ int32_t g10_workspace_bytes(int32_t which, int64_t K, int64_t N, int64_t E, int3
         *out_bytes = carve_emit(nullptr, N, E, L, &zb, &zbytes);
         return G10_OK;
     }
-    // one layout serves the three calls (the planner uses all of it; the others a prefix-independent subset)
     Workspace w;
     Sizes z{K, N, E, mem == G10_MEM_HOST};
-    *out_bytes = carve(nullptr, z, w);
+    *out_bytes = carve(nullptr, z, w, which);
     return G10_OK;
 }
 
@@ -273,7 +276,7 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
     Workspace w;
     DeviceTrace d;
     const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
-    rc = begin_call(trace, ws, w, d, s, buckets ? 0 : kZeroCounts);
+    rc = begin_call(G10_WS_VITALITY, trace, ws, w, d, s, buckets ? 0 : kZeroCounts);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     VitalityBuffers vb;
@@ -320,7 +323,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(trace, ws, w, d, s, kZeroPairs);
+    rc = begin_call(G10_WS_TIMELINE, trace, ws, w, d, s, kZeroPairs);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     int64_t *start = host ? w.start : out->kernel_start_ns;
@@ -429,7 +432,7 @@ int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uin
     Workspace w;
     DeviceTrace d;
     const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
-    rc = begin_call(trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff);
+    rc = begin_call(G10_WS_PLAN, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff);
     if (rc != G10_OK) return rc;
     VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
                        w.period_tensor, w.period_prev_use, w.period_next_use, d.E, w.counts};
@@ -473,7 +476,7 @@ int32_t g10_plan_batch(const g10_trace *trace, int32_t V, const g10_variant *var
     Workspace w;
     DeviceTrace d;
     const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
-    rc = begin_call(trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff);
+    rc = begin_call(G10_WS_BATCH, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff);
     if (rc != G10_OK) return rc;
     CU(cudaMemcpyAsync(w.batch_variants, bv.data(), sizeof(BatchVariant) * (size_t)V, cudaMemcpyHostToDevice, s));
     VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
@@ -506,7 +509,7 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
     DeviceTrace d;
     const uint32_t flags = options ? options->flags : 0;
     const bool buckets = !(flags & G10_FLAG_RESCORE_ALL) && vitality_buckets_supported(trace->num_tensors, trace->num_events);
-    rc = begin_call(trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff | (plan_keeps_state_on_chip(trace->num_kernels, trace->num_events, flags) ? 0 : kZeroState));
+    rc = begin_call(G10_WS_PLAN, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff | (plan_keeps_state_on_chip(trace->num_kernels, trace->num_events, flags) ? 0 : kZeroState));
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
 #ifdef G10_TEST_HOOKS

@@ -14,8 +14,6 @@
 // beat the best exact score known to the whole grid, and then by the whole grid together (absent ranges of the
 // best candidates span a large part of a long timeline), so that when the iteration decides, the committed score
 // is the exact maximum over all live periods, ties included (see k_plan_lazy).
-#include <cstdio>
-
 #include "g10_planner.cuh"
 
 namespace g10 {
@@ -465,10 +463,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     __shared__ int s_mix[kMixCap];
     __shared__ int s_nmix;
     __shared__ int s_flag;
-#ifdef G10_PHASE_CLOCKS
-    __shared__ ull s_dbg_slots, s_dbg_mixed, s_dbg_tiles, s_dbg_over;
-    if (threadIdx.x == 0) { s_dbg_slots = 0; s_dbg_mixed = 0; s_dbg_tiles = 0; s_dbg_over = 0; }
-#endif
     __shared__ unsigned char s_refresh[kLazyMaxBlocks];
     const int G = gridDim.x, c = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -481,13 +475,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     int par = 0;                               // which worklist buffer this iteration fills
     int pbuf = 0;                              // which publication buffer is written next
     int pp = 0;                                // which slice buffer is written next
-#ifdef G10_PHASE_CLOCKS
-    long long dbg_dirty = 0, dbg_coop = 0, dbg_rounds = 0, dbg_refresh = 0;
-    long long pc_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, pc_last = clock64();
-#define LAZY_CLOCK(i) do { if (threadIdx.x == 0) { const long long now_ = clock64(); pc_acc[i] += now_ - pc_last; pc_last = now_; } } while (0)
-#else
-#define LAZY_CLOCK(i)
-#endif
 
     if (c == 0) for (int j = threadIdx.x; j < 3 * kRoundM * 2; j += kPlanThreads) L.partials[j] = 0;
     // every period starts DIRTY: its first evaluation chooses the destination
@@ -540,13 +527,11 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         // ---------------- A: apply the pending commit to the slots this block owns (bookings: after the barrier)
         if (pending) {
             const bool touched = commit_lazy(A, L, win.idx, win.dest, it - 1, n_mig - 1, c, G, s_max);
-            LAZY_CLOCK(10);
             if (touched) {
                 __syncthreads();
                 const long long m = own_tiles_max(A, L, c, G, s_max);
                 if (threadIdx.x == 0) A.peak_part[c] = m;
             }
-            LAZY_CLOCK(11);
         }
         // classify the owned periods against the commit, collect DIRTY ones, local bests
         // (on the first iteration `win` matches nothing and every period is DIRTY)
@@ -554,9 +539,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
             const Cand bestF = scan_owned(A, L, Pn, true, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti);
             if (threadIdx.x == 0) store_prop(&L.props[(size_t)pbuf * kLazyMaxBlocks + c], bestF, s_tk, s_ti);
         }
-        LAZY_CLOCK(0);
         if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
-        LAZY_CLOCK(1);
         int rbuf = pbuf;
         pbuf ^= 1;
 
@@ -579,25 +562,18 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         if (c == 0 && threadIdx.x == 0) L.wl_count[par ^ 1] = 0;
         par ^= 1;
         const bool few_dirty = W > 0 && W <= (unsigned)kDirtyPool && G * kTopT + kDirtyPool <= kLazyMaxBlocks * kTopT;
-        LAZY_CLOCK(2);
         if (few_dirty) {
             // DIRTY periods need the bookings in place: barrier; one warp re-chooses each one's destination; barrier.
             // They join the published bounds below with an unbounded score and are rescored with the others.
             if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
             barrier_since_booking = true;
             for (unsigned e = (unsigned)c * kPlanWarps + warp; e < W; e += (unsigned)G * kPlanWarps) dest_warp(A, L, wl[e], lane);
-#ifdef G10_PHASE_CLOCKS
-            dbg_dirty += W;
-#endif
             if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
         } else if (W > 0) {
             // very many DIRTY periods (the first iteration): rescore them at once, shared out, and look again
             if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
             barrier_since_booking = true;
             for (unsigned e = (unsigned)c * kPlanWarps + warp; e < W; e += (unsigned)G * kPlanWarps) eval_warp(A, L, wl[e], lane);
-#ifdef G10_PHASE_CLOCKS
-            dbg_dirty += W;
-#endif
             if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
             {
                 const Cand bestF = scan_owned(A, L, Pn, false, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti);
@@ -621,7 +597,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
             n_pool += (int)W;
             __syncthreads();
         }
-        LAZY_CLOCK(3);
 
         // ---------------- R: rounds of joint rescoring
         bool failed = false;
@@ -675,7 +650,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                 }
             }
             __syncthreads();
-            LAZY_CLOCK(4);
             if (msel == 0) {
                 if (round_no == 0) { round_no = 1; continue; }      // (the first round only looks at the best bounds)
                 // nothing published may beat the best score.  A block that has used all its bounds may hold more.
@@ -691,9 +665,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                 }
                 __syncthreads();
                 if (!s_flag) break;
-#ifdef G10_PHASE_CLOCKS
-                dbg_refresh += 1;
-#endif
                 if (s_refresh[c]) {
                     const Cand bestF = scan_owned(A, L, Pn, false, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti, &gBest);
                     if (threadIdx.x == 0) store_prop(&L.props[(size_t)pbuf * kLazyMaxBlocks + c], bestF, s_tk, s_ti);
@@ -702,13 +673,9 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                 barrier_since_booking = true;
                 load_bounds(pbuf, true);
                 pbuf ^= 1;
-                LAZY_CLOCK(8);
                 continue;
             }
             round_no += 1;
-#ifdef G10_PHASE_CLOCKS
-            dbg_rounds += 1; dbg_coop += msel;
-#endif
             // every block sums its share of each chosen period's absent range: tiles ta + c, ta + c + G, ... of the
             // range.  One thread per period classifies its tiles from their pressure minima / maxima (a tile wholly
             // at least s above capacity counts s for its whole time, one wholly within capacity nothing); the few
@@ -723,23 +690,14 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                 if (r < msel) {
                     const int ap = s_it_ap[r], bp = s_it_bp[r];
                     const int64_t sz = s_it_s[r];
-#ifdef G10_PHASE_CLOCKS
-                    if (sub == 0) atomicAdd((ull *)&s_dbg_slots, (ull)(bp - ap + 1));
-#endif
                     u128 acc = 0;
                     const int ta = ap / kSlotTile, tb = bp / kSlotTile;
                     for (int tl = ta + c + sub * G; tl <= tb; tl += nsub * G) {
                         const int64_t t0 = (int64_t)tl * kSlotTile, t1 = t0 + kSlotTile - 1;
                         const int k_lo = (int)(t0 > ap ? t0 : ap), k_hi = (int)(t1 < bp ? t1 : bp);
                         const long long mn = L.tmin[tl], mx = L.tmax[tl];
-#ifdef G10_PHASE_CLOCKS
-                        atomicAdd((ull *)&s_dbg_tiles, 1ull);
-#endif
                         if (mx <= A.cap) continue;
                         if (mn >= A.cap && mn - A.cap >= sz) { acc += (u128)(ull)sz * (u128)(ull)(A.start[k_hi + 1] - A.start[k_lo]); continue; }
-#ifdef G10_PHASE_CLOCKS
-                        atomicAdd((ull *)&s_dbg_mixed, 1ull);
-#endif
                         const int pos = atomicAdd(&s_nmix, 1);
                         if (pos < kMixCap) s_mix[pos] = (r << 22) | tl;
                         else acc += benefit_partial(A, k_lo, k_hi, sz, 0, 1);          // list full: this thread reads the tile itself
@@ -754,10 +712,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
             __syncthreads();
             {
                 const int nmix = s_nmix < kMixCap ? s_nmix : kMixCap;
-#ifdef G10_PHASE_CLOCKS
-                if (threadIdx.x == 0 && s_nmix > kMixCap) s_dbg_over += s_nmix - kMixCap;
-                LAZY_CLOCK(10);
-#endif
 #pragma unroll 1
                 for (int m = warp; m < nmix; m += kPlanWarps) {
                     const int r = s_mix[m] >> 22, tl = s_mix[m] & ((1 << 22) - 1);
@@ -783,10 +737,8 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                     if (up) atomicAdd(&dst[1], up);
                 }
             }
-            LAZY_CLOCK(5);
             if (!grid_barrier(A.bar, G, gen)) { failed = true; break; }
             barrier_since_booking = true;
-            LAZY_CLOCK(6);
             // the buffer used two rounds from now was last read one round ago: block 0 clears it
             if (c == 0)
                 for (int j = threadIdx.x; j < kRoundM * 2; j += kPlanThreads) L.partials[(size_t)((pp + 2) % 3) * kRoundM * 2 + j] = 0;
@@ -811,7 +763,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
             }
             pp = (pp + 1) % 3;
             __syncthreads();
-            LAZY_CLOCK(7);
         }
         if (failed) { status = -2; break; }
         if (!barrier_since_booking) { if (!grid_barrier(A.bar, G, gen)) { status = -2; break; } }
@@ -831,20 +782,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         }
         n_mig += 1;
         pending = true;
-        LAZY_CLOCK(9);
     }
-#ifdef G10_PHASE_CLOCKS
-    if (threadIdx.x == 0 && c == 0) {
-        const long long r_ = rounds ? rounds : 1;
-        printf("k_plan_lazy cycles/iteration: A %lld bar1 %lld B %lld dirty %lld select %lld slices %lld bar %lld combine %lld refresh %lld decide %lld\n",
-               pc_acc[0] / r_, pc_acc[1] / r_, pc_acc[2] / r_, pc_acc[3] / r_, pc_acc[4] / r_, pc_acc[5] / r_, pc_acc[6] / r_, pc_acc[7] / r_, pc_acc[8] / r_, pc_acc[9] / r_);
-        printf("  within A: commit %lld own-slots max %lld\n", pc_acc[10] / r_, pc_acc[11] / r_);
-    }
-    if (threadIdx.x == 0 && c == 0) printf("slots of jointly rescored ranges: %llu; tiles looked at by block 0: %llu, read slot by slot %llu, beyond the list %llu\n", s_dbg_slots, s_dbg_tiles, s_dbg_mixed, s_dbg_over);
-    if (threadIdx.x == 0 && (c == 0 || c == 77))
-        printf("k_plan_lazy block %d: iterations %lld, DIRTY rescored (grid) %lld, rounds %lld, periods rescored jointly %lld, refreshes %lld\n",
-               c, (long long)rounds, dbg_dirty, dbg_rounds, dbg_coop, dbg_refresh);
-#endif
     plan_epilogue(A, c, G, gen, status, peak, n_mig, rounds, bytes_ssd, bytes_host);
 }
 

@@ -20,8 +20,6 @@
 // capacities -- each running the whole loop independently of the others (re-planning under profiling error,
 // other SSD bandwidths or host capacities).  A variant's block builds its own slot clock (block-wide scan of its
 // durations) and derives the geometry of a period when it needs it, from that clock in shared memory.
-#include <cstdio>
-
 #include "g10_planner.cuh"
 
 namespace g10 {
@@ -116,28 +114,12 @@ __device__ __forceinline__ void warp_argmax_u64(ull k, int idx, ull *mk, int *mi
     *mi = (int)__reduce_min_sync(0xffffffffu, top ? (unsigned)idx : 0x7fffffffu);
 }
 
-// Developer aid (off in the library build): with -DG10_PHASE_CLOCKS thread 0 accumulates the cycles between the
-// marked points of an iteration and prints the averages when the loop ends.
-#ifdef G10_PHASE_CLOCKS
-#define W0_CLOCK(i) do { if (threadIdx.x == 0) { const long long now_ = clock64(); w0_acc[i] += now_ - w0_last; w0_last = now_; } } while (0)
-#define ONE_COUNT(i) do { if ((threadIdx.x & 31) == 0) atomicAdd(&s_dbg[i], 1); } while (0)
-#define ONE_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
-                           ph_acc[i] += now_ - ph_last; ph_last = now_; ph_cnt[i] += 1; asm volatile("" ::: "memory"); } } while (0)
-#else
-#define ONE_CLOCK(i)
-#define ONE_COUNT(i)
-#define W0_CLOCK(i)
-#endif
 
 template <bool kBatch, bool kCyclic>
 __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs O, BatchArgs B)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_fin[kOneMaxFin];
-#ifdef G10_PHASE_CLOCKS
-    __shared__ int s_dbg[4];
-    if (threadIdx.x < 4) s_dbg[threadIdx.x] = 0;
-#endif
     __shared__ OneDirty s_dirty[kOneDirtyCap];
     __shared__ int s_n_over, s_ndirty, s_nlist, s_nfin, s_force, s_win, s_top, s_flagged;
     __shared__ ull s_topkey;
@@ -257,16 +239,11 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
 
     int64_t n_mig = 0, rounds = 0, bytes_ssd = 0, bytes_host = 0;
     int status = -1;
-#ifdef G10_PHASE_CLOCKS
-    long long ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_cnt[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
-    long long w0_acc[4] = {0, 0, 0, 0}, w0_last = clock64();
-#endif
 #pragma unroll 1
     for (int64_t it = 0;; ++it) {
         if (A.fits_always || s_n_over == 0) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
         if (it >= limit) { status = limit < Pn64 ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
         rounds += 1;
-        ONE_CLOCK(0);
         // ---------------- 1. DIRTY periods: destination (SSD first, then host), one warp per period; a new score
         // only if the destination changed
         if (s_ndirty > 0) {
@@ -284,7 +261,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                     const int j = base + __ffs(m) - 1;
                     m &= m - 1;
                     const int li = listed ? s_dirty[j].li : j;
-                    ONE_COUNT(0);
                     const unsigned char st = cstate[li];
                     const OneRanges r = crng[li];
                     const int a = r.a, b = r.b;
@@ -314,7 +290,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                         d = X;
                     }
                     if (d < 0) {                                  // channels only fill up: gone for good
-                        ONE_COUNT(2);
                         if (lane == 0) { cstate[li] = 0; ckey[li] = 0; gflag[li >> 5] = 1; s_flagged = 1; }
                         continue;
                     }
@@ -322,7 +297,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                         if (lane == 0) cstate[li] = (unsigned char)(st & ~kDirtyO);
                         continue;
                     }
-                    ONE_COUNT(1);
                     const u128 acc = warp_sum_u128(benefit_range_warp(sP, sStart, tmin, tmax, A.cap, s, ap, bp, Kc, lane));
                     if (lane == 0) {
                         Cand cd;
@@ -339,7 +313,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             }
             __syncthreads();
             if (tid == 0) { s_ndirty = 0; s_nlist = 0; }
-            ONE_CLOCK(1);
         }
         // ---------------- 2. search: warp 0 refreshes the group maxima that changed, takes the top and, while the top is
         // STALE, rescores it (from the pressure tiles) and looks again; the other warps wait at the barrier
@@ -364,7 +337,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             if (warp == 0) {
 #pragma unroll 1
                 for (;;) {
-                    W0_CLOCK(0);
                     if (s_flagged) {
                         __syncwarp();
                         if (lane == 0) s_flagged = 0;
@@ -382,7 +354,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                         }
                     }
                     __syncwarp();
-                    W0_CLOCK(1);
                     ull bk = 0; int bi = 0x7fffffff;
 #pragma unroll 4
                     for (int g = lane; g < G1; g += 32) {
@@ -391,18 +362,14 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                     }
                     ull mk; int mi;
                     warp_argmax_u64(bk, bi, &mk, &mi);
-                    W0_CLOCK(2);
                     if (mk == 0 || (cstate[mi] & kStateMaskO) != kStaleO) {
                         if (lane == 0) { s_topkey = mk; s_top = mi; }
                         break;
                     }
-                    ONE_COUNT(3);
                     rescore_warp0(mi);
-                    W0_CLOCK(3);
                 }
             }
             __syncthreads();
-            ONE_CLOCK(2);
             const ull topkey = s_topkey;
             const int top = s_top;
             if (topkey == 0) { exhausted = true; break; }
@@ -434,7 +401,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
                     if (lane == 0) { s_force = 0x7fffffff; s_nfin = 0; }
                     __syncwarp();
                 }
-                ONE_CLOCK(4);
                 continue;
             }
             if (tid == 0) {
@@ -463,7 +429,6 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             break;
         }
         if (exhausted) { status = G10_EXHAUSTED; break; }
-        ONE_CLOCK(5);
         // ---------------- 3. apply the winner
         {
             const OneRanges r = crng[win];
@@ -567,18 +532,7 @@ __global__ void __launch_bounds__(kOneThreads, 1) k_plan_one(PlanArgs A, OneArgs
             if (X == G10_DEST_SSD) bytes_ssd += s; else bytes_host += s;
         }
         __syncthreads();
-        ONE_CLOCK(6);
     }
-#ifdef G10_PHASE_CLOCKS
-    if (threadIdx.x == 0) {
-        const long long r = rounds ? rounds : 1;
-        printf("one-block cycles/iteration: top %lld dirty %lld (x%lld) topscan %lld (x%lld) tiescan %lld (x%lld) rescore %lld (x%lld) winner %lld apply %lld (n=%lld)\n",
-               ph_acc[0] / r, ph_acc[1] / r, ph_cnt[1], ph_acc[2] / r, ph_cnt[2], ph_acc[3] / r, ph_cnt[3], ph_acc[4] / r, ph_cnt[4], ph_acc[5] / r,
-               ph_acc[6] / r, (long long)rounds);
-        printf("dirty periods examined %d, rescored %d, erased %d; search-loop rescorings %d\n", s_dbg[0], s_dbg[1], s_dbg[2], s_dbg[3]);
-        printf("warp 0 search loop cycles/iteration: other %lld flag refresh %lld top scan %lld rescore %lld\n", w0_acc[0] / r, w0_acc[1] / r, w0_acc[2] / r, w0_acc[3] / r);
-    }
-#endif
     // ---------------- epilogue: final pressure, peak and its lowest slot, summary
     __syncthreads();
     long long pk = 0;

@@ -9,8 +9,6 @@
 //   3. every block applies the winner to its own copy of the state and reclassifies its own periods.
 // Because all copies evolve identically no block ever reads another block's state, so no barrier separates
 // the commit from the next scoring round.
-#include <cstdio>
-
 #include "g10_planner.cuh"
 
 namespace g10 {
@@ -104,14 +102,6 @@ __device__ __forceinline__ bool poll_record_halfwarp(const ull *rec, bool active
     return ok;
 }
 
-// Developer aid (off in the library build): with -DG10_PHASE_CLOCKS thread 0 of blocks 0 and 1 accumulates
-// the cycles between the marked points of an iteration and prints the averages when the loop ends.
-#ifdef G10_PHASE_CLOCKS
-#define PHASE_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
-                             ph_acc[i] += now_ - ph_last; ph_last = now_; asm volatile("" ::: "memory"); } } while (0)
-#else
-#define PHASE_CLOCK(i)
-#endif
 
 // kFew: every block owns at most 256 periods (warp 0 alone finds the block's best candidate).
 template <bool kFew>
@@ -146,9 +136,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
     int64_t *tmax = tmin + NT;                                                             // [NT] largest
     int64_t *busy = S.busy_rep + (size_t)c * 4 * K;
     int64_t *hocc = S.hocc_rep + (size_t)c * K;
-#ifdef G10_PHASE_CLOCKS
-    long long ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_last = clock64();
-#endif
 
     if (threadIdx.x == 0) { s_n_over = 0; s_err = 0; }
     __syncthreads();
@@ -197,7 +184,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
         if (A.fits_always || s_n_over == 0) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
         if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
         rounds += 1;
-        PHASE_CLOCK(0);     // loop top (stop tests)
         if (kFew) for (int li = threadIdx.x; li < n_local; li += kPlanThreads) cskip[li] = 0;
         // ---------------- 1. bring this block's periods up to date (one warp per period).  With few periods per
         // block only the DIRTY ones are done here (rare); STALE ones are rescored on demand in step 2.
@@ -251,7 +237,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             }
         }
         __syncthreads();
-        PHASE_CLOCK(1);     // evaluation + barrier
         // ---------------- 2. block-local argmax, published as tagged words
         const int par = (int)(it & 1);
         const ull tag = (ull)(unsigned)(it + 1) << 32;
@@ -429,7 +414,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                 st_volatile_u64(&S.xwords[((size_t)par * G + c) * kXWords + threadIdx.x], tag | ((const unsigned *)&s_pay)[threadIdx.x]);
             __syncthreads();                               // s_pay is reused for the winner's record below
         }
-        PHASE_CLOCK(2);     // local argmax + publish
         // ---------------- block 0 reads all G proposals (one half-warp per record), reduces them and writes one
         // copy of the winner's record per block; every other block polls its own copy (no hot line)
         ull *win_words = &S.xwords[((size_t)2 * G + (size_t)par * G) * kXWords];      // [G] copies for this parity
@@ -455,9 +439,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
                 cy.ben = ((u128)y.ben_hi << 64) | y.ben_lo; cy.cost = 2ull * (ull)y.t; cy.idx = y.idx; cy.dest = y.dest;
                 if (cand_beats(cy, x)) x = cy;
             }
-            PHASE_CLOCK(3);     // leader: all proposals arrived and compared per thread
             const Cand gw = block_best_fast(x, &s_best, s_cand);         // (its barriers also publish s_err)
-            PHASE_CLOCK(4);     // leader: block argmax
             if (threadIdx.x == 0) {
                 if (gw.idx < 0) { s_pay.idx = -1; s_pay.dest = -1; }
                 else s_pay = recs[gw.idx % G];             // period p was proposed by block p mod G
@@ -479,7 +461,6 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
         if (s_err) { status = -2; break; }
         const XPayload win = s_pay;
         if (win.idx < 0) { status = G10_EXHAUSTED; break; }
-        PHASE_CLOCK(5);     // leader: copies written / follower: winner record arrived
         // ---------------- 3. apply the winner to this block's copy of the state
         {
             const int64_t p = win.idx;
@@ -554,15 +535,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_small(PlanArgs A, Smal
             for (int tl = wap / kTileO + warp; tl <= wbp / kTileO; tl += kPlanWarps) tile_refresh_warp(sP, K, tl, tmin, tmax, lane);
         }
         __syncthreads();
-        PHASE_CLOCK(6);     // apply + barrier
     }
-#ifdef G10_PHASE_CLOCKS
-    if (threadIdx.x == 0 && c < 2) {
-        const long long r = rounds ? rounds : 1;
-        printf("block %d cycles/iteration: top %lld eval %lld local+publish %lld gather %lld argmax %lld winner %lld apply %lld [7: %lld] (n=%lld)\n", c,
-               ph_acc[0] / r, ph_acc[1] / r, ph_acc[2] / r, ph_acc[3] / r, ph_acc[4] / r, ph_acc[5] / r, ph_acc[6] / r, ph_acc[7] / r, (long long)rounds);
-    }
-#endif
     // ---------------- epilogue: block 0 writes the final pressure and the summary
     if (c != 0) return;
     __syncthreads();

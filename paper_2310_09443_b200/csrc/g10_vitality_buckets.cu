@@ -15,8 +15,6 @@
 // Everything random happens in shared memory (atomics included); HBM sees the events twice, the keys once each
 // way and the outputs once.  A bucket with more events than fit in shared memory (a tensor listed by a great many
 // kernels) keeps its segments in global memory instead: slower, same result.
-#include <cstdio>
-
 #include "g10_device.cuh"
 #include "g10_internal.h"
 
@@ -119,14 +117,6 @@ __device__ __forceinline__ void block_scan_counts(const unsigned *cnt, int n, in
     bk_block_scan<1>((const int *)cnt, out, nullptr, nullptr, n, s_w);
 }
 
-// Developer aid (off in the library build): with -DG10_PHASE_CLOCKS thread 0 of two blocks adds up the cycles
-// between the marked points and prints the averages at the end.
-#ifdef G10_PHASE_CLOCKS
-#define BK_CLOCK(i) do { if (threadIdx.x == 0) { asm volatile("" ::: "memory"); const long long now_ = clock64(); \
-                         ph_acc[i] += now_ - ph_acc[15]; ph_acc[15] = now_; asm volatile("" ::: "memory"); } } while (0)
-#else
-#define BK_CLOCK(i)
-#endif
 
 // ---------------------------------------------------------------------------------------------
 // 1. events per bucket
@@ -307,11 +297,6 @@ __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ul
 
 __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBuffers out)
 {
-#ifdef G10_PHASE_CLOCKS
-    __shared__ long long ph_acc[16];                     // (in shared memory: the register count stays that of the library build)
-    if (threadIdx.x == 0) { for (int i = 0; i < 15; ++i) ph_acc[i] = 0; ph_acc[15] = clock64(); }
-    int ph_n = 0;
-#endif
     extern __shared__ __align__(16) int s_mem[];
     int *s_base = s_mem;                       // [nb + 1] first key of each bucket
     int *t_off = s_base + bk_pad(B.nb);          // [bt + 1] raw events per tensor, then segment offsets
@@ -340,10 +325,6 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         __syncthreads();
         const int b = s_bucket;
         if (b >= B.nb) break;
-        BK_CLOCK(0);
-#ifdef G10_PHASE_CLOCKS
-        ph_n += 1;
-#endif
         const int n = s_base[b + 1] - s_base[b];
         const int64_t t0 = (int64_t)b * B.bt;
         const int bt_eff = (int)((B.N - t0) < B.bt ? (B.N - t0) : B.bt);
@@ -364,9 +345,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             if (rk[q] != ~0ull) atomicAdd(&t_off[(int)(rk[q] >> 32)], 1);
         for (int j = kRegKeys * kBkThreads + threadIdx.x; j < n; j += kBkThreads) atomicAdd(&t_off[(int)(gk[j] >> 32)], 1);
         __syncthreads();
-        BK_CLOCK(1);
         bk_block_scan<1>(t_off, t_off, nullptr, nullptr, bt_eff, s_scan);
-        BK_CLOCK(2);
 #pragma unroll
         for (int q = 0; q < kRegKeys; ++q)
             if (rk[q] != ~0ull) {
@@ -379,7 +358,6 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             ks[t_off[tl] + atomicAdd(&t_d[tl], 1)] = (int32_t)(unsigned)key;
         }
         __syncthreads();
-        BK_CLOCK(3);
         // ---- short segments: one or two raw uses are settled on the spot; three to kBkHeavy go to a list that the
         // threads then take one tensor each from (one thread sorts, removes repeats in place and counts the periods),
         // so that a warp is not held up eight times over by its longest segment
@@ -421,7 +399,6 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             my_d += dd; my_p += pp;
         }
         __syncthreads();
-        BK_CLOCK(4);
         // ---- long segments: the whole block sorts, compacts and counts, one tensor after the other
         const int nheavy = s_nheavy;
         for (int hq = 0; hq < (nheavy <= 64 ? nheavy : bt_eff); ++hq) {
@@ -459,7 +436,6 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         }
         // ---- the bucket's totals go out first (later buckets wait for them), then the offsets of every tensor's
         // distinct uses and periods inside the bucket
-        BK_CLOCK(5);
         {
             const int wd = __reduce_add_sync(0xffffffffu, my_d), wp = __reduce_add_sync(0xffffffffu, my_p);
             if (lane == 0) { s_wa[warp] = wd; s_wb[warp] = wp; }
@@ -472,7 +448,6 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             }
         }
         bk_block_scan<2>(t_d, t_d, t_np, t_np, bt_eff, s_scan);
-        BK_CLOCK(6);
         const long long D = t_d[bt_eff], PC = t_np[bt_eff];
         long long pu = 0, pq = 0;
         for (int j0 = threadIdx.x; j0 < 2 * b; j0 += 4 * kBkThreads) {
@@ -509,7 +484,6 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         }
         __syncthreads();
         const long long U = s_pre[0], PB = s_pre[1];
-        BK_CLOCK(7);
         ull bad = 0;
         if (U + D > out.uses_cap) bad |= G10_DEV_USES_OVERFLOW;
         if (PB + PC > out.periods_cap) bad |= G10_DEV_PERIODS_OVERFLOW;
@@ -547,14 +521,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             out.use_ptr[B.N] = U + D; out.period_ptr[B.N] = PB + PC;
             out.counts[0] = U + D; out.counts[1] = PB + PC;
         }
-        BK_CLOCK(8);
     }
-#ifdef G10_PHASE_CLOCKS
-    if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 100) && ph_n > 0)
-        printf("k_bk_emit block %d (%d buckets) cycles/bucket: ticket %lld load+count %lld scan %lld scatter %lld short %lld heavy %lld scan2 %lld prefix %lld outputs %lld\n",
-               blockIdx.x, ph_n, ph_acc[0] / ph_n, ph_acc[1] / ph_n, ph_acc[2] / ph_n, ph_acc[3] / ph_n, ph_acc[4] / ph_n, ph_acc[5] / ph_n,
-               ph_acc[6] / ph_n, ph_acc[7] / ph_n, ph_acc[8] / ph_n);
-#endif
 }
 
 // Picks the bucket width for a trace; false if the trace is outside what the bucket path handles.

@@ -85,4 +85,10 @@ def test_argument_errors_of_the_later_entry_points(lib):
     eo = binding._EmitOut()
     assert lib.g10_emit_instructions(1, 1, None, None, None, None, None, 0, None, None, C.byref(eo), None, 0, None) == -1
     # the workspace of the batch call is the planner's
-    assert binding.g10_workspace_bytes(binding.WS_BATCH, 96, 130, 320) == binding.g10_workspace_bytes(binding.WS_PLAN, 96, 130, 320)
+    plan_ws = binding.g10_workspace_bytes(binding.WS_PLAN, 96, 130, 320)
+    assert binding.g10_workspace_bytes(binding.WS_BATCH, 96, 130, 320) >= plan_ws       # the planner's, plus the variant table
+    # the analysis calls ask only for what they use
+    big = (1_000_000, 4_000_000, 5_000_000)
+    assert binding.g10_workspace_bytes(binding.WS_TIMELINE, *big) < 64 << 20
+    assert binding.g10_workspace_bytes(binding.WS_VITALITY, *big) < 128 << 20
+    assert binding.g10_workspace_bytes(binding.WS_PLAN, *big) > binding.g10_workspace_bytes(binding.WS_VITALITY, *big)
