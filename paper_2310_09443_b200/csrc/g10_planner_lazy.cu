@@ -180,25 +180,49 @@ __device__ __forceinline__ long long own_tiles_max(const PlanArgs &A, const Lazy
 // minima / maxima) and host occupancy; block 0 also writes the plan record and the erase flag.  The channel
 // bookings are added later (book_winner).  Returns true if a tile of this block changed.
 __device__ __forceinline__ bool commit_lazy(const PlanArgs &A, const LazyArgs &L, int64_t p, int X, int64_t it, int64_t n_mig, int c, int G,
-                                            long long *s_red)
+                                            long long *s_red, int a, int ap, int bp, int b, int64_t t)
 {
+    // (the winner's slot ranges and transfer time come from the caller, which looked them up when it decided; only the
+    // tensor's size is fetched here)
     const int64_t K = A.K;
-    const int i = A.per_t[p], u = A.per_u[p], v = A.per_v[p];
-    const int a = u + 1, b = v - 1;
+    const int i = A.per_t[p];
     const int64_t s = A.bytes[i];
-    const int ap = A.geo_a[X * A.geo_stride + p], bp = A.geo_b[X * A.geo_stride + p];
-    const int64_t t = A.geo_t[X * A.geo_stride + p];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     bool touched = false;
     {
         const int ta = ap / kSlotTile, tb = bp / kSlotTile;
         int tl = ta + ((c - ta % G) % G + G) % G;            // first tile >= ta that this block owns
         for (; tl <= tb; tl += G) {
             touched = true;
+            // one pass over the tile: subtract inside the range, and the tile's new minimum and maximum from the same values
             const int64_t k0 = (int64_t)tl * kSlotTile;
-            for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < K; k += kPlanThreads)
-                if (k >= ap && k <= bp) A.P[k] -= s;
+            long long mn = 0x7fffffffffffffffll, mx = -0x7fffffffffffffffll - 1;
+            for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < K; k += kPlanThreads) {
+                long long pv = A.P[k];
+                if (k >= ap && k <= bp) { pv -= s; A.P[k] = pv; }
+                if (pv < mn) mn = pv;
+                if (pv > mx) mx = pv;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const long long x = __shfl_xor_sync(0xffffffffu, mn, o), y = __shfl_xor_sync(0xffffffffu, mx, o);
+                if (x < mn) mn = x;
+                if (y > mx) mx = y;
+            }
+            __syncthreads();                                   // (s_red free)
+            if (lane == 0) { s_red[2 * warp] = mn; s_red[2 * warp + 1] = mx; }
             __syncthreads();
-            tile_minmax(A, L, tl, s_red);
+            if (warp == 0) {
+                long long x = lane < kPlanWarps ? s_red[2 * lane] : 0x7fffffffffffffffll;
+                long long y = lane < kPlanWarps ? s_red[2 * lane + 1] : -0x7fffffffffffffffll - 1;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const long long x2 = __shfl_xor_sync(0xffffffffu, x, o), y2 = __shfl_xor_sync(0xffffffffu, y, o);
+                    if (x2 < x) x = x2;
+                    if (y2 > y) y = y2;
+                }
+                if (lane == 0) { L.tmin[tl] = x; L.tmax[tl] = y; }
+            }
         }
     }
     if (X == G10_DEST_HOST && A.host_capacity != 0) {
@@ -215,7 +239,7 @@ __device__ __forceinline__ bool commit_lazy(const PlanArgs &A, const LazyArgs &L
         if (n_mig < A.out_cap) {
             g10_migration m;
             m.period = (int32_t)p; m.tensor = i; m.dest = X; m.absent_first = ap; m.absent_last = bp;
-            m.iteration = (int32_t)it; m.evict_issue_ns = A.start[a]; m.prefetch_issue_ns = A.start[v] - t; m.transfer_ns = t;
+            m.iteration = (int32_t)it; m.evict_issue_ns = A.start[a]; m.prefetch_issue_ns = A.start[b + 1] - t; m.transfer_ns = t;
             A.out[n_mig] = m;
         } else raise_status(A.status, G10_DEV_PLAN_OVERFLOW);
     }
@@ -314,25 +338,28 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
 #pragma unroll
     for (int j = 0; j < kTopT; ++j) { tk[j] = -1.0; ti[j] = -1; }
     const int64_t *bo = A.busy + (size_t)(2 * (w.dest < 0 ? 0 : w.dest)) * A.K, *bi = bo + A.K;
-    // The pass is a chain of L2 latencies: the loads of the next period of this thread are issued before the
-    // current one is worked on.
-    unsigned char st_nx = 0;
-    double key_nx = 0.0;
-    int u_nx = 0, v_nx = 0;
-    {
-        const int64_t p = (int64_t)c * kPlanThreads + threadIdx.x;
-        if (p < Pn) { st_nx = L.c_state[p]; key_nx = L.c_key[p]; if (classify) { u_nx = A.per_u[p]; v_nx = A.per_v[p]; } }
-    }
-    for (int64_t p0 = (int64_t)c * kPlanThreads; p0 < Pn; p0 += (int64_t)G * kPlanThreads) {
+    // The pass is a chain of L2 latencies: the loads of four periods of this thread are in flight together.
+    constexpr int kAhead = 4;
+    const int64_t step = (int64_t)G * kPlanThreads;
+    for (int64_t p00 = (int64_t)c * kPlanThreads; p00 < Pn; p00 += kAhead * step) {
+      unsigned char st_q[kAhead];
+      double key_q[kAhead];
+      int u_q[kAhead], v_q[kAhead];
+#pragma unroll
+      for (int q = 0; q < kAhead; ++q) {
+          const int64_t pq = p00 + q * step + threadIdx.x;
+          st_q[q] = 0; key_q[q] = 0.0; u_q[q] = 0; v_q[q] = 0;
+          if (pq < Pn) { st_q[q] = L.c_state[pq]; key_q[q] = L.c_key[pq]; if (classify) { u_q[q] = A.per_u[pq]; v_q[q] = A.per_v[pq]; } }
+      }
+#pragma unroll
+      for (int q = 0; q < kAhead; ++q) {
+        const int64_t p0 = p00 + q * step;
+        if (p0 >= Pn) break;                                  // (uniform in the block)
         const int64_t p = p0 + threadIdx.x;
         bool dirty = false;
-        unsigned char st = st_nx;
-        const double key_ld = key_nx;
-        const int u = u_nx, v = v_nx;
-        {
-            const int64_t pn = p + (int64_t)G * kPlanThreads;
-            if (pn < Pn) { st_nx = L.c_state[pn]; key_nx = L.c_key[pn]; if (classify) { u_nx = A.per_u[pn]; v_nx = A.per_v[pn]; } }
-        }
+        unsigned char st = st_q[q];
+        const double key_ld = key_q[q];
+        const int u = u_q[q], v = v_q[q];
         if (p < Pn) {
             if (st != 0) {
                 int state = st >> 2;
@@ -396,6 +423,7 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
                 if (dirty) L.worklist[(size_t)par * L.stride + base + __popc(md & ((1u << lane) - 1u))] = (int)p;
             }
         }
+      }
     }
     Cand x;
     x.ben = 0; x.cost = 1; x.idx = -1; x.dest = -1;
@@ -526,7 +554,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         bool barrier_since_booking = true;
         // ---------------- A: apply the pending commit to the slots this block owns (bookings: after the barrier)
         if (pending) {
-            const bool touched = commit_lazy(A, L, win.idx, win.dest, it - 1, n_mig - 1, c, G, s_max);
+            const bool touched = commit_lazy(A, L, win.idx, win.dest, it - 1, n_mig - 1, c, G, s_max, win.a, win.ap, win.bp, win.b, win.t);
             if (touched) {
                 __syncthreads();
                 const long long m = own_tiles_max(A, L, c, G, s_max);
@@ -692,7 +720,10 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                     const int64_t sz = s_it_s[r];
                     u128 acc = 0;
                     const int ta = ap / kSlotTile, tb = bp / kSlotTile;
-                    for (int tl = ta + c + sub * G; tl <= tb; tl += nsub * G) {
+                    // (which block takes the range's first tile rotates with the period: ranges shorter than G tiles would
+                    // otherwise all land on the low-numbered blocks)
+                    const int ce = (c + r * 37) % G;
+                    for (int tl = ta + ce + sub * G; tl <= tb; tl += nsub * G) {
                         const int64_t t0 = (int64_t)tl * kSlotTile, t1 = t0 + kSlotTile - 1;
                         const int k_lo = (int)(t0 > ap ? t0 : ap), k_hi = (int)(t1 < bp ? t1 : bp);
                         const long long mn = L.tmin[tl], mx = L.tmax[tl];
