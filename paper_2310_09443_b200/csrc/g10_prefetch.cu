@@ -21,6 +21,58 @@ __device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y
     return kx < ky || (kx == ky && x < y);
 }
 
+// Orders the records by (latest safe prefetch time, record index) into `order`, with the whole block: a bitonic network
+// over (time, record) pairs in shared memory (`scratch`: n2 * 12 bytes) when they fit, else over the indices in global memory.
+__device__ void pf_order_records(int64_t n, int64_t n2, const g10_migration *__restrict__ mig, int32_t *order, long long *scratch,
+                                 int sort_in_smem, int nthreads)
+{
+    if (sort_in_smem) {
+        // (time, record) pairs sorted in shared memory: the network's comparisons would otherwise each cost two
+        // dependent global loads
+        long long *s_key = scratch;
+        int *s_idx = (int *)(s_key + n2);
+        for (int64_t i = threadIdx.x; i < n2; i += nthreads) {
+            s_key[i] = i < n ? mig[i].prefetch_issue_ns : 0x7fffffffffffffffll;
+            s_idx[i] = i < n ? (int)i : 0x7fffffff;
+        }
+        __syncthreads();
+        for (int64_t k = 2; k <= n2; k <<= 1) {
+            for (int64_t j = k >> 1; j > 0; j >>= 1) {
+                const bool mirror = (j == (k >> 1));
+                for (int64_t t = threadIdx.x; t < n2 / 2; t += nthreads) {
+                    const int64_t blk = t / j, off = t % j;
+                    const int64_t i = blk * 2 * j + off;
+                    const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
+                    const long long kx = s_key[i], ky = s_key[p];
+                    const int ix = s_idx[i], iy = s_idx[p];
+                    if (ky < kx || (ky == kx && iy < ix)) { s_key[i] = ky; s_key[p] = kx; s_idx[i] = iy; s_idx[p] = ix; }
+                }
+                __syncthreads();
+            }
+        }
+        for (int64_t i = threadIdx.x; i < n; i += nthreads) order[i] = s_idx[i];
+        __syncthreads();
+    } else {
+        for (int64_t i = threadIdx.x; i < n; i += nthreads) order[i] = (int32_t)i;
+        __syncthreads();
+        for (int64_t k = 2; k <= n2; k <<= 1) {
+            for (int64_t j = k >> 1; j > 0; j >>= 1) {
+                const bool mirror = (j == (k >> 1));
+                for (int64_t t = threadIdx.x; t < n2 / 2; t += nthreads) {
+                    const int64_t blk = t / j, off = t % j;
+                    const int64_t i = blk * 2 * j + off;
+                    const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
+                    if (p < n) {
+                        const int32_t x = order[i], y = order[p];
+                        if (pf_before(mig, y, x)) { order[i] = y; order[p] = x; }
+                    }
+                }
+                __syncthreads();
+            }
+        }
+    }
+}
+
 template <int kPfThreads>
 __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int64_t n, const g10_migration *__restrict__ mig,
                                                                   const int64_t *__restrict__ start, const int64_t *__restrict__ bytes,
@@ -43,51 +95,7 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
     // ---- order the records by (latest safe prefetch time, record index)
     int64_t n2 = 1;
     while (n2 < n) n2 <<= 1;
-    if (sort_in_smem) {
-        // (time, record) pairs sorted in shared memory: the network's comparisons would otherwise each cost two
-        // dependent global loads
-        long long *s_key = s_dyn + (p_in_smem ? K : 0);
-        int *s_idx = (int *)(s_key + n2);
-        for (int64_t i = threadIdx.x; i < n2; i += kPfThreads) {
-            s_key[i] = i < n ? mig[i].prefetch_issue_ns : 0x7fffffffffffffffll;
-            s_idx[i] = i < n ? (int)i : 0x7fffffff;
-        }
-        __syncthreads();
-        for (int64_t k = 2; k <= n2; k <<= 1) {
-            for (int64_t j = k >> 1; j > 0; j >>= 1) {
-                const bool mirror = (j == (k >> 1));
-                for (int64_t t = threadIdx.x; t < n2 / 2; t += kPfThreads) {
-                    const int64_t blk = t / j, off = t % j;
-                    const int64_t i = blk * 2 * j + off;
-                    const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
-                    const long long kx = s_key[i], ky = s_key[p];
-                    const int ix = s_idx[i], iy = s_idx[p];
-                    if (ky < kx || (ky == kx && iy < ix)) { s_key[i] = ky; s_key[p] = kx; s_idx[i] = iy; s_idx[p] = ix; }
-                }
-                __syncthreads();
-            }
-        }
-        for (int64_t i = threadIdx.x; i < n; i += kPfThreads) order[i] = s_idx[i];
-        __syncthreads();
-    } else {
-        for (int64_t i = threadIdx.x; i < n; i += kPfThreads) order[i] = (int32_t)i;
-        __syncthreads();
-        for (int64_t k = 2; k <= n2; k <<= 1) {
-            for (int64_t j = k >> 1; j > 0; j >>= 1) {
-                const bool mirror = (j == (k >> 1));
-                for (int64_t t = threadIdx.x; t < n2 / 2; t += kPfThreads) {
-                    const int64_t blk = t / j, off = t % j;
-                    const int64_t i = blk * 2 * j + off;
-                    const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
-                    if (p < n) {
-                        const int32_t x = order[i], y = order[p];
-                        if (pf_before(mig, y, x)) { order[i] = y; order[p] = x; }
-                    }
-                }
-                __syncthreads();
-            }
-        }
-    }
+    pf_order_records(n, n2, mig, order, s_dyn + (p_in_smem ? K : 0), sort_in_smem, kPfThreads);
     // ---- visit the records in that order, a batch of kPfThreads at a time: the batch's fields are fetched together
     // (one thread per record), the visits read them from shared memory; the pressure curve sits in shared memory
     // too when it fits (Pw), else in global memory
@@ -180,6 +188,192 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same pass for a pressure curve too long for shared memory.  The curve stays in global memory, but the block
+// keeps two numbers per tile of kPfTile slots in shared memory: an upper bound of the tile's largest pressure and an
+// amount still to be added to every slot of the tile.  A search walks the tiles of the range (shared memory only) and
+// looks at slots only in a tile whose bound says that it may hold a slot that cannot take the tensor -- one trip to
+// global memory, which also makes the tile's bound exact again; a regained range adds the tensor's size to the
+// tiles it covers whole (shared memory) and to the slots of the at most two tiles it covers in part (reductions that
+// nobody waits for).  The amounts still to be added go into the curve at the end.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPfTile = 1024;                    // slots per tile
+constexpr int kPfNT = 256;                       // threads of the block (few warps: the many block-wide barriers stay cheap)
+constexpr int kPfMaxTiles = 8192;
+constexpr int kPfBatch = 256;                    // records whose fields are fetched together
+
+// largest of one int per thread over the block (-1 = none); `s_buf` [32], used by one call at a time between barriers
+__device__ __forceinline__ int pf_block_max(int v, int *s_buf, int lane, int warp)
+{
+    v = (int)__reduce_max_sync(0xffffffffu, v);
+    __syncthreads();                                       // (s_buf free)
+    if (lane == 0) s_buf[warp] = v;
+    __syncthreads();
+    return (int)__reduce_max_sync(0xffffffffu, lane < kPfNT / 32 ? s_buf[lane] : -1);
+}
+
+__global__ void __launch_bounds__(kPfNT) k_schedule_prefetch_tiled(int64_t K, int64_t n, const g10_migration *__restrict__ mig,
+                                                                     const int64_t *__restrict__ start, const int64_t *__restrict__ bytes,
+                                                                     int64_t cap, int64_t *P, int32_t *order, int32_t *new_last,
+                                                                     int64_t *new_issue, int64_t *summary, int sort_in_smem)
+{
+    extern __shared__ long long s_dyn[];
+    __shared__ int s_ra[kPfBatch], s_rb[kPfBatch], s_rj[kPfBatch];
+    __shared__ long long s_rs[kPfBatch];
+    __shared__ int s_red[32];
+    __shared__ long long s_redl[32];
+    __shared__ long long s_mx[32];
+    __shared__ int s_sl[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int T = (int)((K + kPfTile - 1) / kPfTile);
+    int64_t n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    long long *tmax = s_dyn + (sort_in_smem ? (n2 * 12 + 7) / 8 : 0);      // [T] upper bound of the tile's largest pressure (amount to add included)
+    long long *toff = tmax + T;                                             // [T] still to be added to every slot of the tile
+    pf_order_records(n, n2, mig, order, s_dyn, sort_in_smem, kPfNT);
+    __syncthreads();
+    // ---- tile maxima, a warp per tile
+    for (int t = warp; t < T; t += kPfNT / 32) {
+        long long m = -0x7fffffffffffffffll - 1;
+        for (int k0 = t * kPfTile + lane; k0 < (t + 1) * kPfTile; k0 += 8 * 32) {
+            long long v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = k0 + 32 * u < K ? __ldcg(&P[k0 + 32 * u]) : m;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) if (v[u] > m) m = v[u];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { const long long x = __shfl_xor_sync(0xffffffffu, m, o); if (x > m) m = x; }
+        if (lane == 0) { tmax[t] = m; toff[t] = 0; }
+    }
+    __syncthreads();
+    long long moved = 0, regained = 0;
+    for (int64_t q0 = 0; q0 < n; q0 += kPfBatch) {
+        const int nb = (int)(n - q0 < kPfBatch ? n - q0 : kPfBatch);
+        __syncthreads();
+        if ((int)threadIdx.x < nb) {
+            const int r = order[q0 + threadIdx.x];
+            s_ra[threadIdx.x] = mig[r].absent_first; s_rb[threadIdx.x] = mig[r].absent_last;
+            s_rs[threadIdx.x] = bytes[mig[r].tensor];
+        }
+        __syncthreads();
+        for (int q = 0; q < nb; ++q) {
+            const int a_abs = s_ra[q], b_abs = s_rb[q];
+            const long long s = s_rs[q], lim = cap - s;        // a slot takes the tensor iff its pressure is at most lim
+            int j = a_abs - 1;                                  // result: last slot that stays absent
+            const int lo_t = a_abs / kPfTile;
+            int t_cur = b_abs / kPfTile;
+            while (t_cur >= lo_t) {
+                // highest tile at or below t_cur whose bound says it may hold a slot that cannot take the tensor
+                int found = -1;
+                for (int base = t_cur; base >= lo_t && found < 0; base -= kPfNT) {
+                    const int t = base - (int)threadIdx.x;
+                    found = pf_block_max((t >= lo_t && tmax[t] > lim) ? t : -1, s_red, lane, warp);
+                }
+                if (found < 0) break;
+                // its slots: the highest one inside the range that cannot take the tensor, and the tile's exact maximum
+                long long m = -0x7fffffffffffffffll - 1;
+                int jt = -1;
+                {
+                    long long val[kPfTile / kPfNT];
+                    const long long add = toff[found];
+#pragma unroll
+                    for (int u = 0; u < kPfTile / kPfNT; ++u) {
+                        const int64_t k = (int64_t)found * kPfTile + u * kPfNT + threadIdx.x;
+                        val[u] = k < K ? __ldcg(&P[k]) + add : m;   // (L2: earlier reductions are there, not in L1)
+                    }
+#pragma unroll
+                    for (int u = 0; u < kPfTile / kPfNT; ++u) {
+                        const int64_t k = (int64_t)found * kPfTile + u * kPfNT + threadIdx.x;
+                        if (val[u] > m) m = val[u];
+                        if (k >= a_abs && k <= b_abs && val[u] > lim) jt = (int)k;     // (k grows with u: the highest one stays)
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) { const long long x = __shfl_xor_sync(0xffffffffu, m, o); if (x > m) m = x; }
+                const int jw = (int)__reduce_max_sync(0xffffffffu, jt);
+                __syncthreads();                                   // (s_red, s_redl free)
+                if (lane == 0) { s_red[warp] = jw; s_redl[warp] = m; }
+                __syncthreads();
+                const int jj = (int)__reduce_max_sync(0xffffffffu, lane < kPfNT / 32 ? s_red[lane] : -1);
+                if (warp == 0) {
+                    long long mm = lane < kPfNT / 32 ? s_redl[lane] : -0x7fffffffffffffffll - 1;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) { const long long x = __shfl_xor_sync(0xffffffffu, mm, o); if (x > mm) mm = x; }
+                    if (lane == 0) tmax[found] = mm;
+                }
+                if (jj >= 0) { j = jj; break; }
+                t_cur = found - 1;
+                __syncthreads();                                   // (the refreshed bound is read by the next search)
+            }
+            __syncthreads();
+            if (j < b_abs) {
+                // the regained slots (j, b_abs] take the tensor back
+                const int k0 = j + 1;
+                const int t0 = k0 / kPfTile, t1 = b_abs / kPfTile;
+                const int first_full = (k0 % kPfTile) ? t0 + 1 : t0, last_full = (b_abs % kPfTile == kPfTile - 1) ? t1 : t1 - 1;
+                for (int t = first_full + (int)threadIdx.x; t <= last_full; t += kPfNT) { toff[t] += s; tmax[t] += s; }
+                if (first_full > t0) {                             // the tile the range starts in, covered in part
+#pragma unroll
+                    for (int u = 0; u < kPfTile / kPfNT; ++u) {
+                        const int64_t k = (int64_t)t0 * kPfTile + u * kPfNT + threadIdx.x;
+                        if (k >= k0 && k <= b_abs) atomicAdd((ull *)&P[k], (ull)s);
+                    }
+                    if (threadIdx.x == 0) tmax[t0] += s;
+                }
+                if (last_full < t1 && (t1 > t0 || first_full == t0)) {   // the tile it ends in, covered in part (and not done above)
+#pragma unroll
+                    for (int u = 0; u < kPfTile / kPfNT; ++u) {
+                        const int64_t k = (int64_t)t1 * kPfTile + u * kPfNT + threadIdx.x;
+                        if (k >= k0 && k <= b_abs) atomicAdd((ull *)&P[k], (ull)s);
+                    }
+                    if (threadIdx.x == 0) tmax[t1] += s;
+                }
+                moved += 1; regained += b_abs - j;
+            }
+            if (threadIdx.x == 0) s_rj[q] = j;
+            __syncthreads();
+        }
+        if ((int)threadIdx.x < nb) {
+            const int r = order[q0 + threadIdx.x];
+            const int j = s_rj[threadIdx.x];
+            new_last[r] = j;
+            new_issue[r] = j < s_rb[threadIdx.x] ? start[j + 1] : mig[r].prefetch_issue_ns;
+        }
+    }
+    __syncthreads();
+    // ---- what is still to be added goes into the curve; new peak and its lowest slot
+    long long mx = 0;
+    int sl = -1;
+    for (int64_t k0 = threadIdx.x; k0 < K; k0 += 8 * kPfNT) {           // eight slots per thread in flight
+        long long pv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) pv[u] = k0 + u * kPfNT < K ? __ldcg(&P[k0 + u * kPfNT]) : 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int64_t k = k0 + u * kPfNT;
+            if (k < K) {
+                const long long add = toff[k / kPfTile];
+                if (add) { pv[u] += add; P[k] = pv[u]; }
+                if (sl < 0 || pv[u] > mx) { mx = pv[u]; sl = (int)k; }
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long omx = __shfl_down_sync(0xffffffffu, mx, o);
+        const int osl = __shfl_down_sync(0xffffffffu, sl, o);
+        if (osl >= 0 && (sl < 0 || omx > mx || (omx == mx && osl < sl))) { mx = omx; sl = osl; }
+    }
+    if (lane == 0) { s_mx[warp] = mx; s_sl[warp] = sl; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kPfNT / 32; ++w)
+            if (s_sl[w] >= 0 && (sl < 0 || s_mx[w] > mx || (s_mx[w] == mx && s_sl[w] < sl))) { mx = s_mx[w]; sl = s_sl[w]; }
+        summary[0] = moved; summary[1] = regained; summary[2] = sl < 0 ? 0 : mx; summary[3] = sl;
+    }
+}
+
 cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *mig, const int64_t *start, const int64_t *bytes,
                                      uint64_t gpu_capacity_bytes, int64_t *P, int32_t *order, int32_t *new_last, int64_t *new_issue,
                                      int64_t *summary, cudaStream_t s)
@@ -193,12 +387,19 @@ cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *
     while (n2 < n) n2 <<= 1;
     int sort_smem = 0;
     if (n > 0 && (size_t)n2 * 12 <= 64 * 1024) { dyn += (size_t)n2 * 12; sort_smem = 1; }
+    const int64_t tiles = (K + kPfTile - 1) / kPfTile;
     if (in_smem) {
         if (dyn > 0) {
             const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
             if (e != cudaSuccess) return e;
         }
         k_schedule_prefetch<256><<<1, 256, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem);
+    } else if (tiles <= kPfMaxTiles) {
+        sort_smem = (n > 0 && (size_t)n2 * 12 + (size_t)tiles * 16 <= 200 * 1024) ? 1 : 0;   // (this kernel has most of the SM's shared memory to itself)
+        dyn = (sort_smem ? ((size_t)n2 * 12 + 7) / 8 * 8 : 0) + (size_t)tiles * 16;
+        const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch_tiled, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+        if (e != cudaSuccess) return e;
+        k_schedule_prefetch_tiled<<<1, kPfNT, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, sort_smem);
     } else {
         if (dyn > 0) {
             const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
