@@ -663,6 +663,12 @@ int32_t g10o_plan_cyclic(int64_t K, int64_t N, const int64_t *kernel_ptr, const 
  * record; (3) only memory is examined, as the section says -- channel bookings are not revisited;
  * (4) a prefetch that moves is issued at the start of the first slot in which the tensor is resident
  * again; one that cannot move keeps its time.
+ * Plans of the steady-state planner (g10o_plan_cyclic) are accepted too.  Readings for them: (5) their
+ * records carry unrolled slots and times (reading (4) there); the pressure curve belongs to the physical
+ * slots, so slot x stands for slot x mod K, and a prefetch that moves is issued at the unrolled time of
+ * its first regained slot; (6) on the cycle no prefetch comes "first": the visiting order is that of the
+ * position inside the iteration, i.e. of the latest safe prefetch time modulo the iteration's length T.
+ * For an ordinary plan every slot is below K and every time below T, and nothing changes.
  * order[i] = plan record visited i-th; new_absent_last / new_issue_ns are indexed by plan record.
  * summary[4] = { prefetches moved, slots regained in total, peak pressure after, its lowest slot }.
  * ---------------------------------------------------------------------------------------- */
@@ -671,12 +677,13 @@ void g10o_schedule_prefetch(int64_t K, int64_t n, const g10o_migration *mig, con
                             int32_t *order, int32_t *new_absent_last, int64_t *new_issue_ns, int64_t *summary)
 {
     int64_t cap = gpu_capacity_bytes >= ((uint64_t)1 << 63) ? INT64_MAX : (int64_t)gpu_capacity_bytes;
+    const int64_t T = K > 0 ? start[K] : 1;
     for (int64_t i = 0; i < n; ++i) order[i] = (int32_t)i;
-    /* insertion sort by (latest safe prefetch time, record): plain and stable */
+    /* insertion sort by (latest safe prefetch time inside the iteration, record): plain and stable */
     for (int64_t i = 1; i < n; ++i) {
         int32_t x = order[i];
         int64_t j = i - 1;
-        while (j >= 0 && (mig[order[j]].prefetch_issue_ns > mig[x].prefetch_issue_ns)) { order[j + 1] = order[j]; --j; }
+        while (j >= 0 && (mig[order[j]].prefetch_issue_ns % T > mig[x].prefetch_issue_ns % T)) { order[j + 1] = order[j]; --j; }
         order[j + 1] = x;
     }
     int64_t moved = 0, regained = 0;
@@ -684,10 +691,11 @@ void g10o_schedule_prefetch(int64_t K, int64_t n, const g10o_migration *mig, con
         const g10o_migration *m = &mig[order[i]];
         int64_t s = tensor_bytes[m->tensor];
         int64_t j = m->absent_last;
-        while (j >= m->absent_first && pressure[j] <= cap - s) --j;      /* pressure + s <= cap, without overflow */
-        for (int64_t k = j + 1; k <= m->absent_last; ++k) pressure[k] += s;
+        while (j >= m->absent_first && pressure[j % K] <= cap - s) --j;  /* pressure + s <= cap, without overflow */
+        for (int64_t k = j + 1; k <= m->absent_last; ++k) pressure[k % K] += s;
         new_absent_last[order[i]] = (int32_t)j;
-        new_issue_ns[order[i]] = j < m->absent_last ? start[j + 1] : m->prefetch_issue_ns;
+        const int64_t first = j + 1;                                     /* first regained slot, unrolled */
+        new_issue_ns[order[i]] = j < m->absent_last ? (first <= K ? start[first] : start[first - K] + T) : m->prefetch_issue_ns;
         if (j < m->absent_last) { moved += 1; regained += m->absent_last - j; }
     }
     int64_t pk, ps;
@@ -710,6 +718,9 @@ void g10o_schedule_prefetch(int64_t K, int64_t n, const g10o_migration *mig, con
  * PREFETCH (get ready for the next), as in Figure 9; then by tensor id.  A tensor never has two
  * instructions of the same kind at one boundary, so the order is total.
  * new_issue_ns (optional): prefetch times from the eager prefetch pass, indexed by plan record.
+ * A plan of the steady-state planner is accepted too: the stream is that of one iteration of the cycle, and a
+ * prefetch whose time lies in the next iteration (a wrap-around period's) stands where the program is at
+ * that moment of every iteration: its time is taken modulo the iteration's length, and so is its boundary.
  * Returns the number of instructions (records beyond out_cap are not written).
  * ---------------------------------------------------------------------------------------- */
 enum { OP_FREE = 0, OP_PRE_EVICT = 1, OP_ALLOC = 2, OP_PREFETCH = 3 };
@@ -758,6 +769,7 @@ int64_t g10o_emit_instructions(int64_t K, int64_t N, const int32_t *first_use, c
         list[m++] = e;
         keyed_ins p = e;
         int64_t t = new_issue_ns ? new_issue_ns[r] : mig[r].prefetch_issue_ns;
+        if (t >= start[K]) t -= start[K];                        /* (steady-state plans only: a time in the next iteration) */
         b = K;
         while (start[b] > t) --b;                                /* last boundary at or before the issue time */
         p.boundary = b; p.ins.opcode = OP_PREFETCH; p.ins.target = -1; p.ins.time_ns = t;
