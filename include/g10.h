@@ -209,7 +209,11 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
    All pointers are DEVICE pointers.  `pressure` [K] is the final pressure of the eviction plan on entry and the
    pressure after the pass on return; order [n] receives the visiting order; new_absent_last [n] and
    new_prefetch_issue_ns [n] are indexed by plan record; summary [4] = prefetches moved, slots regained, new peak,
-   its lowest slot.  Needs no workspace; one block does the (strictly sequential) pass. */
+   its lowest slot.  Needs no workspace; one block does the (strictly sequential) pass.
+   Records of g10_plan_cyclic are accepted as they are: a slot beyond K stands for the same slot of the cycle (the
+   pressure curve has K slots), a moved prefetch is issued at the unrolled time of its first regained slot, and the
+   visiting order is that of the prefetch's moment inside the iteration (its time modulo the iteration's length).
+   For an ordinary plan nothing changes. */
 typedef struct g10_prefetch_out {
     int64_t *pressure;
     int32_t *order;
@@ -230,7 +234,10 @@ int32_t g10_schedule_prefetch(int64_t num_kernels, int64_t num_migrations, const
    inst_ptr [K + 2] is the CSR by boundary; counts [2] = number of instructions, device status word
    (G10_DEV_PLAN_OVERFLOW if instructions_cap is too small).  new_prefetch_issue_ns (optional) are the times from
    g10_schedule_prefetch.  All pointers are DEVICE pointers; `ws` as for the other calls (G10_WS_EMIT, with the
-   number of migrations in place of E).  Limits: K + 1 <= 4096 * 4096 boundaries. */
+   number of migrations in place of E).  Limits: K + 1 <= 4096 * 4096 boundaries.
+   Records of g10_plan_cyclic are accepted as they are: the stream is that of one iteration of the cycle, and the
+   prefetch of a wrap-around period, whose time lies in the next iteration, stands at the same moment of this one
+   (time and boundary modulo the iteration). */
 #define G10_OP_FREE 0
 #define G10_OP_PRE_EVICT 1
 #define G10_OP_ALLOC 2
@@ -261,7 +268,8 @@ int32_t g10_emit_instructions(int64_t num_kernels, int64_t num_tensors, const in
    g10_plan_migrations on the unrolled clock, while pressure, channel bookings and host occupancy belong to the
    physical slot k mod K.  Records carry unrolled slots and times (absent_last may be >= K, the prefetch time may lie
    in the next iteration).  Same arguments, outputs and workspace (G10_WS_PLAN) as g10_plan_migrations; of the
-   options only host_capacity_bytes and max_iterations are used.
+   options only host_capacity_bytes and max_iterations are used.  g10_schedule_prefetch and g10_emit_instructions take
+   the records as they are.
    Limits: device-resident traces (G10_MEM_DEVICE); one thread block plans, so pressure, clock, bookings and periods
    must fit the shared memory of one SM (K <= 32000), else summary[2] = -1 and summary[7] has G10_DEV_BATCH_UNFIT. */
 int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,

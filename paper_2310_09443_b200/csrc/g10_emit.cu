@@ -51,7 +51,10 @@ __device__ __forceinline__ bool emit_item(const EmitArgs &A, int64_t item, int64
     const int64_t r = item - 2 * A.N < A.n ? item - 2 * A.N : item - 2 * A.N - A.n;
     const bool evict = item - 2 * A.N < A.n;
     *record = (int)r; *tensor = A.mig[r].tensor;
-    const int64_t t = evict ? A.mig[r].evict_issue_ns : (A.new_issue ? A.new_issue[r] : A.mig[r].prefetch_issue_ns);
+    int64_t t = evict ? A.mig[r].evict_issue_ns : (A.new_issue ? A.new_issue[r] : A.mig[r].prefetch_issue_ns);
+    // (a steady-state plan: the prefetch of a wrap-around period may lie in the next iteration; it stands at the same
+    // moment of this one)
+    if (!evict && t >= A.start[A.K]) t -= A.start[A.K];
     // last boundary b in [0, K] with start[b] <= t (for a pre-eviction start[b] == t_r exactly)
     int lo = 0, hi = (int)A.K;
     while (lo < hi) { const int mid = lo + (hi - lo + 1) / 2; if (A.start[mid] <= t) lo = mid; else hi = mid - 1; }
@@ -281,8 +284,10 @@ __global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int6
             ins.bytes = A.bytes[ins.tensor];
             ins.time_ns = A.start[boundary];
             if (ins.opcode == kOpPreEvict) { ins.target = A.mig[ins.record].dest; ins.time_ns = A.mig[ins.record].evict_issue_ns; }
-            if (ins.opcode == kOpPrefetch)
+            if (ins.opcode == kOpPrefetch) {
                 ins.time_ns = A.new_issue ? A.new_issue[ins.record] : A.mig[ins.record].prefetch_issue_ns;
+                if (ins.time_ns >= A.start[A.K]) ins.time_ns -= A.start[A.K];      // (steady-state plans: see emit_item)
+            }
             inst[pos] = ins;
         }
     }

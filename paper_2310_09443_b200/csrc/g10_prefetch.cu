@@ -15,16 +15,18 @@ namespace g10 {
 // and per record: few warps keep it cheap), 1024 for a long one in global memory (its ranges are long: width pays)
 constexpr int kPfRows = 8;                       // slots a thread looks at per search chunk
 
-__device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y)
+// (T = length of the iteration: the prefetch of a steady-state plan's wrap-around period may lie in the next iteration; what
+// orders the visits is its moment inside the iteration.  Times of an ordinary plan are all below T.)
+__device__ __forceinline__ bool pf_before(const g10_migration *mig, int x, int y, int64_t T)
 {
-    const int64_t kx = mig[x].prefetch_issue_ns, ky = mig[y].prefetch_issue_ns;
+    const int64_t kx = mig[x].prefetch_issue_ns % T, ky = mig[y].prefetch_issue_ns % T;
     return kx < ky || (kx == ky && x < y);
 }
 
 // Orders the records by (latest safe prefetch time, record index) into `order`, with the whole block: a bitonic network
 // over (time, record) pairs in shared memory (`scratch`: n2 * 12 bytes) when they fit, else over the indices in global memory.
 __device__ void pf_order_records(int64_t n, int64_t n2, const g10_migration *__restrict__ mig, int32_t *order, long long *scratch,
-                                 int sort_in_smem, int nthreads)
+                                 int sort_in_smem, int nthreads, int64_t T)
 {
     if (sort_in_smem) {
         // (time, record) pairs sorted in shared memory: the network's comparisons would otherwise each cost two
@@ -32,7 +34,7 @@ __device__ void pf_order_records(int64_t n, int64_t n2, const g10_migration *__r
         long long *s_key = scratch;
         int *s_idx = (int *)(s_key + n2);
         for (int64_t i = threadIdx.x; i < n2; i += nthreads) {
-            s_key[i] = i < n ? mig[i].prefetch_issue_ns : 0x7fffffffffffffffll;
+            s_key[i] = i < n ? mig[i].prefetch_issue_ns % T : 0x7fffffffffffffffll;
             s_idx[i] = i < n ? (int)i : 0x7fffffff;
         }
         __syncthreads();
@@ -64,7 +66,7 @@ __device__ void pf_order_records(int64_t n, int64_t n2, const g10_migration *__r
                     const int64_t p = mirror ? (blk * 2 * j + 2 * j - 1 - off) : (i + j);
                     if (p < n) {
                         const int32_t x = order[i], y = order[p];
-                        if (pf_before(mig, y, x)) { order[i] = y; order[p] = x; }
+                        if (pf_before(mig, y, x, T)) { order[i] = y; order[p] = x; }
                     }
                 }
                 __syncthreads();
@@ -95,7 +97,8 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
     // ---- order the records by (latest safe prefetch time, record index)
     int64_t n2 = 1;
     while (n2 < n) n2 <<= 1;
-    pf_order_records(n, n2, mig, order, s_dyn + (p_in_smem ? K : 0), sort_in_smem, kPfThreads);
+    const int64_t T = K > 0 ? start[K] : 1;
+    pf_order_records(n, n2, mig, order, s_dyn + (p_in_smem ? K : 0), sort_in_smem, kPfThreads, T);
     // ---- visit the records in that order, a batch of kPfThreads at a time: the batch's fields are fetched together
     // (one thread per record), the visits read them from shared memory; the pressure curve sits in shared memory
     // too when it fits (Pw), else in global memory
@@ -111,15 +114,24 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
         }
         __syncthreads();
         for (int q = 0; q < nb; ++q) {
-            const int a_abs = s_ra[q], b_abs = s_rb[q];
+            const int a_abs = s_ra[q], b_abs = s_rb[q];          // unrolled slots; beyond K only for a steady-state plan
             const int64_t s = s_rs[q];
-            int hi = b_abs;                     // slots (j, b_abs] are known to take the tensor
-            int j = a_abs - 1;                  // result: last slot that stays absent
-            while (hi >= a_abs) {
+            int j = a_abs - 1;                  // result: last slot that stays absent (unrolled)
+            // The range as at most two runs of physical slots, the later one first: the part in the next iteration
+            // (slot x stands for slot x - K), then the part in this one.
+            const int Ki = (int)K;
+            int seg_lo[2], seg_hi[2], seg_off[2], nseg = 0;
+            if (b_abs >= Ki) { seg_lo[nseg] = (a_abs > Ki ? a_abs : Ki) - Ki; seg_hi[nseg] = b_abs - Ki; seg_off[nseg] = Ki; ++nseg; }
+            if (a_abs < Ki) { seg_lo[nseg] = a_abs; seg_hi[nseg] = b_abs < Ki ? b_abs : Ki - 1; seg_off[nseg] = 0; ++nseg; }
+            bool stopped = false;
+            for (int g = 0; g < nseg && !stopped; ++g) {
+              const int lo_p = seg_lo[g];
+              int hi = seg_hi[g];                 // slots (.., seg_hi] above hi are known to take the tensor
+              while (hi >= lo_p) {
                 // a chunk of kPfRows rows of kPfThreads slots, from hi downwards: row r, thread t looks at slot
                 // hi - (r * kPfThreads + t); all loads of a thread are in flight together.  The highest slot that
                 // cannot take the tensor is the failing one with the smallest offset r * kPfThreads + t.
-                const int span = hi - a_abs + 1;                     // slots still to look at
+                const int span = hi - lo_p + 1;                      // slots still to look at
                 int first = 0x7fffffff;                             // this warp's smallest failing offset
                 long long pv[kPfRows];
 #pragma unroll
@@ -138,18 +150,20 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
                 const int mine = lane < kPfThreads / 32 ? s_wstop[turn][lane] : 0x7fffffff;      // one warp result per lane
                 const int best = (int)__reduce_min_sync(0xffffffffu, (unsigned)mine);
                 turn ^= 1;                                                   // (the other copy was last read two barriers ago)
-                if (best != 0x7fffffff) { j = hi - best; break; }
+                if (best != 0x7fffffff) { j = hi - best + seg_off[g]; stopped = true; break; }
                 hi -= kPfRows * kPfThreads;
+              }
             }
-            {   // the regained slots take the tensor back: read-modify-write, eight per thread in flight
-                const int k0 = j + 1 + (int)threadIdx.x;
+            for (int g = 0; g < nseg; ++g) {   // the regained slots (j, b_abs] take the tensor back: read-modify-write, eight per thread in flight
+                const int lo_p = (j + 1 - seg_off[g] > seg_lo[g] ? j + 1 - seg_off[g] : seg_lo[g]), hi_p = seg_hi[g];
+                const int k0 = lo_p + (int)threadIdx.x;
 #pragma unroll 1
-                for (int k = k0; k <= b_abs; k += 8 * kPfThreads) {
+                for (int k = k0; k <= hi_p; k += 8 * kPfThreads) {
                     long long v[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) v[u] = k + u * kPfThreads <= b_abs ? Pw[k + u * kPfThreads] : 0;
+                    for (int u = 0; u < 8; ++u) v[u] = k + u * kPfThreads <= hi_p ? Pw[k + u * kPfThreads] : 0;
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) if (k + u * kPfThreads <= b_abs) Pw[k + u * kPfThreads] = v[u] + s;
+                    for (int u = 0; u < 8; ++u) if (k + u * kPfThreads <= hi_p) Pw[k + u * kPfThreads] = v[u] + s;
                 }
             }
             if (threadIdx.x == 0) s_rj[q] = j;
@@ -160,7 +174,7 @@ __global__ void __launch_bounds__(kPfThreads) k_schedule_prefetch(int64_t K, int
             const int r = order[q0 + threadIdx.x];
             const int j = s_rj[threadIdx.x];
             new_last[r] = j;
-            new_issue[r] = j < s_rb[threadIdx.x] ? start[j + 1] : mig[r].prefetch_issue_ns;
+            new_issue[r] = j < s_rb[threadIdx.x] ? (j + 1 <= K ? start[j + 1] : start[j + 1 - K] + T) : mig[r].prefetch_issue_ns;
         }
     }
     __syncthreads();
@@ -225,15 +239,16 @@ __global__ void __launch_bounds__(kPfNT) k_schedule_prefetch_tiled(int64_t K, in
     __shared__ long long s_mx[32];
     __shared__ int s_sl[32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int T = (int)((K + kPfTile - 1) / kPfTile);
+    const int nT = (int)((K + kPfTile - 1) / kPfTile);
     int64_t n2 = 1;
     while (n2 < n) n2 <<= 1;
     long long *tmax = s_dyn + (sort_in_smem ? (n2 * 12 + 7) / 8 : 0);      // [T] upper bound of the tile's largest pressure (amount to add included)
-    long long *toff = tmax + T;                                             // [T] still to be added to every slot of the tile
-    pf_order_records(n, n2, mig, order, s_dyn, sort_in_smem, kPfNT);
+    long long *toff = tmax + nT;                                             // [T] still to be added to every slot of the tile
+    const int64_t T = K > 0 ? start[K] : 1;
+    pf_order_records(n, n2, mig, order, s_dyn, sort_in_smem, kPfNT, T);
     __syncthreads();
     // ---- tile maxima, a warp per tile
-    for (int t = warp; t < T; t += kPfNT / 32) {
+    for (int t = warp; t < nT; t += kPfNT / 32) {
         long long m = -0x7fffffffffffffffll - 1;
         for (int k0 = t * kPfTile + lane; k0 < (t + 1) * kPfTile; k0 += 8 * 32) {
             long long v[8];
@@ -258,9 +273,18 @@ __global__ void __launch_bounds__(kPfNT) k_schedule_prefetch_tiled(int64_t K, in
         }
         __syncthreads();
         for (int q = 0; q < nb; ++q) {
-            const int a_abs = s_ra[q], b_abs = s_rb[q];
+            const int ua = s_ra[q], ub = s_rb[q];              // unrolled slots; beyond K only for a steady-state plan
             const long long s = s_rs[q], lim = cap - s;        // a slot takes the tensor iff its pressure is at most lim
-            int j = a_abs - 1;                                  // result: last slot that stays absent
+            int j = ua - 1;                                     // result: last slot that stays absent (unrolled)
+            // the range as at most two runs of physical slots, the later one first: the part in the next iteration (slot x
+            // stands for slot x - K), then the part in this one
+            const int Ki = (int)K;
+            int seg_lo[2], seg_hi[2], seg_off[2], nseg = 0;
+            if (ub >= Ki) { seg_lo[nseg] = (ua > Ki ? ua : Ki) - Ki; seg_hi[nseg] = ub - Ki; seg_off[nseg] = Ki; ++nseg; }
+            if (ua < Ki) { seg_lo[nseg] = ua; seg_hi[nseg] = ub < Ki ? ub : Ki - 1; seg_off[nseg] = 0; ++nseg; }
+            bool stopped = false;
+            for (int g = 0; g < nseg && !stopped; ++g) {
+            const int a_abs = seg_lo[g], b_abs = seg_hi[g];
             const int lo_t = a_abs / kPfTile;
             int t_cur = b_abs / kPfTile;
             while (t_cur >= lo_t) {
@@ -302,14 +326,17 @@ __global__ void __launch_bounds__(kPfNT) k_schedule_prefetch_tiled(int64_t K, in
                     for (int o = 16; o > 0; o >>= 1) { const long long x = __shfl_xor_sync(0xffffffffu, mm, o); if (x > mm) mm = x; }
                     if (lane == 0) tmax[found] = mm;
                 }
-                if (jj >= 0) { j = jj; break; }
+                if (jj >= 0) { j = jj + seg_off[g]; stopped = true; break; }
                 t_cur = found - 1;
                 __syncthreads();                                   // (the refreshed bound is read by the next search)
             }
             __syncthreads();
-            if (j < b_abs) {
-                // the regained slots (j, b_abs] take the tensor back
-                const int k0 = j + 1;
+            }
+            for (int g = 0; g < nseg; ++g) {
+            // the regained slots (j, ub] take the tensor back: this run's share of them
+            const int b_abs = seg_hi[g];
+            const int k0 = j + 1 - seg_off[g] > seg_lo[g] ? j + 1 - seg_off[g] : seg_lo[g];
+            if (k0 <= b_abs) {
                 const int t0 = k0 / kPfTile, t1 = b_abs / kPfTile;
                 const int first_full = (k0 % kPfTile) ? t0 + 1 : t0, last_full = (b_abs % kPfTile == kPfTile - 1) ? t1 : t1 - 1;
                 for (int t = first_full + (int)threadIdx.x; t <= last_full; t += kPfNT) { toff[t] += s; tmax[t] += s; }
@@ -329,8 +356,10 @@ __global__ void __launch_bounds__(kPfNT) k_schedule_prefetch_tiled(int64_t K, in
                     }
                     if (threadIdx.x == 0) tmax[t1] += s;
                 }
-                moved += 1; regained += b_abs - j;
             }
+            __syncthreads();                                       // (a tile may belong to both runs)
+            }
+            if (j < ub) { moved += 1; regained += ub - j; }
             if (threadIdx.x == 0) s_rj[q] = j;
             __syncthreads();
         }
@@ -338,7 +367,7 @@ __global__ void __launch_bounds__(kPfNT) k_schedule_prefetch_tiled(int64_t K, in
             const int r = order[q0 + threadIdx.x];
             const int j = s_rj[threadIdx.x];
             new_last[r] = j;
-            new_issue[r] = j < s_rb[threadIdx.x] ? start[j + 1] : mig[r].prefetch_issue_ns;
+            new_issue[r] = j < s_rb[threadIdx.x] ? (j + 1 <= K ? start[j + 1] : start[j + 1 - K] + T) : mig[r].prefetch_issue_ns;
         }
     }
     __syncthreads();

@@ -626,7 +626,69 @@ def check_cyclic(gpu, oracle, tr, cap, host_capacity=0, max_iterations=0):
     assert np.array_equal(summary[:7], ref.summary[:7]), (summary, ref.summary)
     assert np.array_equal(gpu.migrations_numpy(plan), ref.migrations)
     assert np.array_equal(_np(plan.final_pressure)[:tr.K], ref.final_pressure)
+    # the calls behind the plan take the steady-state plan as it is (Section 4.4): eager prefetch pass (with the plan's
+    # capacity and with more room, so that wrap-around prefetches move too), then the instruction stream of one iteration
+    if tr.K > 0 and len(ref.migrations) > 0 and max_iterations == 0:
+        n = len(ref.migrations)
+        tl = gpu.g10_pressure_timeline(tb)
+        v = gpu.g10_vitality(tb)
+        ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+        start = oracle.slot_clock(tr.kernel_ns)
+        for cap2 in (cap, cap + int(tr.tensor_bytes.max())):
+            P = plan.final_pressure.clone()
+            pf = gpu.g10_schedule_prefetch(tr.K, n, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap2, P)
+            em = gpu.g10_emit_instructions(tr.K, tr.N, v.first_use, v.last_use, tb.tensor_bytes, tb.tensor_global, tl.kernel_start_ns,
+                                           n, plan.migrations, pf.new_prefetch_issue_ns)
+            torch.cuda.synchronize()
+            opf = oracle.schedule_prefetch(tr.K, ref.migrations, start, tr.tensor_bytes, cap2, ref.final_pressure)
+            assert np.array_equal(_np(pf.order)[:n], opf.order) and np.array_equal(_np(pf.new_absent_last)[:n], opf.new_absent_last)
+            assert np.array_equal(_np(pf.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
+            assert np.array_equal(_np(P)[:tr.K], opf.pressure) and np.array_equal(_np(pf.summary), opf.summary)
+            oe = oracle.emit_instructions(tr.K, ov.first_use, ov.last_use, tr.tensor_bytes, tr.tensor_global, start, ref.migrations,
+                                          opf.new_prefetch_issue_ns)
+            assert int(em.counts[1].item()) == 0 and int(em.counts[0].item()) == len(oe.instructions)
+            assert np.array_equal(_np(em.inst_ptr), oe.inst_ptr)
+            got = gpu.instructions_numpy(em)
+            for name in oe.instructions.dtype.names:
+                assert np.array_equal(got[name], oe.instructions[name]), name
     return ref
+
+
+@pytest.mark.gpu
+def test_prefetch_pass_on_wrapping_records(gpu, oracle):
+    """The eager prefetch pass on synthetic records whose absent ranges reach into the next iteration, for every kernel the
+    call can choose: pressure curve in shared memory (K = 5000), per-tile bounds in shared memory (K = 40 000, several
+    tiles and a ragged last one)."""
+    import torch
+    rng = np.random.default_rng(60221023)
+    for K, n in ((5000, 400), (40000, 1500), (40000, 6000)):
+        dur = rng.integers(1, 1000, size=K).astype(np.int64)
+        start = np.concatenate([[0], np.cumsum(dur)]).astype(np.int64)
+        T = int(start[K])
+        N = 64
+        nbytes = rng.integers(1, 1 << 20, size=N).astype(np.int64)
+        P = rng.integers(0, 1 << 22, size=K).astype(np.int64)
+        cap = int(1 << 22)
+        mig = np.zeros(n, dtype=gpu.MIGRATION_DTYPE)
+        a = rng.integers(0, K, size=n)
+        length = np.where(rng.random(n) < 0.3, rng.integers(1, K - 1, size=n), rng.integers(1, 64, size=n))
+        b = np.minimum(a + length - 1, a + K - 2)
+        mig["absent_first"], mig["absent_last"] = a, b
+        mig["tensor"] = rng.integers(0, N, size=n)
+        issue = np.where(b + 1 <= K, start[np.minimum(b + 1, K)], start[(b + 1) % K] + T) - rng.integers(0, 2, size=n)
+        mig["prefetch_issue_ns"] = issue
+        mig["period"] = np.arange(n)
+        assert (b >= K).sum() > 20
+        dm = torch.from_numpy(mig.view(np.uint8).copy()).cuda()
+        dP = torch.from_numpy(P.copy()).cuda()
+        pf = gpu.g10_schedule_prefetch(K, n, dm, torch.from_numpy(start).cuda(), torch.from_numpy(nbytes).cuda(), cap, dP)
+        torch.cuda.synchronize()
+        opf = oracle.schedule_prefetch(K, mig, start, nbytes, cap, P)
+        assert np.array_equal(_np(pf.order)[:n], opf.order)
+        assert np.array_equal(_np(pf.new_absent_last)[:n], opf.new_absent_last)
+        assert np.array_equal(_np(pf.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
+        assert np.array_equal(_np(dP), opf.pressure) and np.array_equal(_np(pf.summary), opf.summary)
+        assert int(opf.summary[0]) > n // 10
 
 
 @pytest.mark.gpu
