@@ -56,7 +56,7 @@ extern "C" {
 #define G10_DEV_PERIODS_OVERFLOW 0x20 /* periods_cap too small (counts[1] holds the need)         */
 #define G10_DEV_PLAN_OVERFLOW 0x40   /* migrations_cap too small (summary[0] holds the need)      */
 #define G10_DEV_TIMEOUT 0x80         /* an internal wait gave up; the kernel returned early       */
-#define G10_DEV_BATCH_UNFIT 0x100    /* g10_plan_batch / g10_plan_cyclic: the trace does not fit one SM (no plan) */
+#define G10_DEV_BATCH_UNFIT 0x100    /* g10_plan_batch: the trace does not fit one SM (no plan)   */
 
 /* exit status of the planner (summary[2]) */
 #define G10_ALREADY_FITS 0      /* unplanned peak pressure <= capacity, empty plan                 */
@@ -270,8 +270,9 @@ int32_t g10_emit_instructions(int64_t num_kernels, int64_t num_tensors, const in
    in the next iteration).  Same arguments, outputs and workspace (G10_WS_PLAN) as g10_plan_migrations; of the
    options only host_capacity_bytes and max_iterations are used.  g10_schedule_prefetch and g10_emit_instructions take
    the records as they are.
-   Limits: device-resident traces (G10_MEM_DEVICE); one thread block plans, so pressure, clock, bookings and periods
-   must fit the shared memory of one SM (K <= 32000), else summary[2] = -1 and summary[7] has G10_DEV_BATCH_UNFIT. */
+   A trace whose pressure, clock, bookings and periods fit the shared memory of one SM (K <= 32000) is planned by one
+   thread block; a larger one by the multi-block formulation of Algorithm 1 as printed (every live period rescored
+   every iteration: the same plan, slower). */
 int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uint64_t host_bw, uint64_t ssd_bw,
                         const g10_options *options /* NULL = defaults */, g10_plan_out *out,
                         void *ws, size_t ws_bytes, void *stream);

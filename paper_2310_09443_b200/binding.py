@@ -327,16 +327,15 @@ def g10_plan_migrations(tb: TraceBuffers, gpu_capacity_bytes, host_bw, ssd_bw, h
 
 
 def g10_plan_cyclic(tb: TraceBuffers, gpu_capacity_bytes, host_bw, ssd_bw, host_capacity_bytes=0, max_iterations=0, ws=None,
-                    stream=None, migrations_cap=None):
-    """Steady-state plan on the cyclic timeline (wrap-around periods of global tensors).  Device traces only; records as in
-    g10_plan_migrations with unrolled slots and times."""
+                    stream=None, migrations_cap=None, device=None):
+    """Steady-state plan on the cyclic timeline (wrap-around periods of global tensors).  Records as in
+    g10_plan_migrations with unrolled slots and times; results in the memory space of `tb`."""
     lib = load_library()
     mcap = tb.E if migrations_cap is None else migrations_cap
-    dev = tb.kernel_ptr.device
-    out = SimpleNamespace(migrations=torch.empty(max(mcap, 1) * 48, dtype=torch.uint8, device=dev),
-                          final_pressure=torch.empty(max(tb.K, 1), dtype=torch.int64, device=dev),
-                          summary=torch.empty(8, dtype=torch.int64, device=dev))
-    ws, ws_bytes = _workspace(tb, WS_PLAN, ws, None)
+    out = SimpleNamespace(migrations=_alloc(tb, max(mcap, 1) * 48, torch.uint8, device),
+                          final_pressure=_alloc(tb, max(tb.K, 1), torch.int64, device),
+                          summary=_alloc(tb, 8, torch.int64, device))
+    ws, ws_bytes = _workspace(tb, WS_PLAN, ws, device)
     po = _PlanOut(_ptr(out.migrations), mcap, _ptr(out.final_pressure), _ptr(out.summary))
     opt = _Options(host_capacity_bytes, max_iterations, 0, None, 0)
     tr = tb.c_struct()

@@ -422,7 +422,7 @@ int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uin
 {
     int32_t rc = check_trace(trace);
     if (rc != G10_OK) return rc;
-    if (trace->mem != G10_MEM_DEVICE || host_bw == 0 || ssd_bw == 0 || !out || !out->summary) return G10_ERR_ARG;
+    if (host_bw == 0 || ssd_bw == 0 || !out || !out->summary) return G10_ERR_ARG;
     if (out->migrations_cap < 0 || (out->migrations_cap > 0 && !out->migrations)) return G10_ERR_ARG;
     if (trace->num_kernels > 0 && !out->final_pressure) return G10_ERR_ARG;
     if (options && options->max_iterations < 0) return G10_ERR_ARG;
@@ -432,7 +432,8 @@ int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uin
     Workspace w;
     DeviceTrace d;
     const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
-    rc = begin_call(G10_WS_PLAN, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff);
+    // (the planner state in global memory is cleared too: a trace too large for the single-block planner is planned there)
+    rc = begin_call(G10_WS_PLAN, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | kZeroDiff | kZeroState);
     if (rc != G10_OK) return rc;
     VitalityBuffers vb{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, d.E, w.period_ptr,
                        w.period_tensor, w.period_prev_use, w.period_next_use, d.E, w.counts};
@@ -441,8 +442,11 @@ int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uin
     pp.host_capacity_bytes = options ? options->host_capacity_bytes : 0;
     pp.max_iterations = options ? options->max_iterations : 0;
     pp.flags = 0;
-    pp.migrations = out->migrations; pp.migrations_cap = out->migrations_cap;
-    pp.final_pressure = out->final_pressure; pp.summary = out->summary;
+    const bool host = trace->mem == G10_MEM_HOST;
+    pp.migrations = host ? w.migrations : out->migrations;
+    pp.migrations_cap = host ? (out->migrations_cap < d.E ? out->migrations_cap : d.E) : out->migrations_cap;
+    pp.final_pressure = host ? w.pressure : out->final_pressure;
+    pp.summary = host ? w.summary : out->summary;
     CU(launch_slot_clock(d, w, w.start, s));
     CU(buckets ? launch_vitality_buckets(d, w, vb, s) : launch_vitality(d, w, vb, s));
     CU(launch_pressure(d, w, w.first_use, w.last_use, false, pp.final_pressure, w.peak_bytes, w.peak_slot, s));
@@ -451,6 +455,16 @@ int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uin
                        host_bw, ssd_bw, d.E > 0 ? d.E : 1, w.geo_t, w.geo_a, w.geo_b, s));
     CU(launch_plan_cyclic(d, w, pp, s));
     CU(launch_publish_status_or(w, pp.summary + 7, s));
+    if (host) {
+        int64_t summary[8];
+        CU(cudaMemcpyAsync(summary, w.summary, sizeof(summary), cudaMemcpyDeviceToHost, s));
+        CU(cudaStreamSynchronize(s));
+        std::memcpy(out->summary, summary, sizeof(summary));
+        const size_t nm = (size_t)(summary[0] < pp.migrations_cap ? (summary[0] > 0 ? summary[0] : 0) : pp.migrations_cap);
+        CU(d2h(out->migrations, w.migrations, nm, s));
+        CU(d2h(out->final_pressure, w.pressure, (size_t)d.K, s));
+        CU(cudaStreamSynchronize(s));
+    }
     return G10_OK;
 }
 

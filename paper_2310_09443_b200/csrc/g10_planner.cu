@@ -6,8 +6,14 @@
 
 namespace g10 {
 
-__global__ void __launch_bounds__(kPlanThreads, 1) k_plan_loop(PlanArgs A)
+// kCyclic: steady-state planning (period and geometry arrays hold slots unrolled over two iterations, A.start is the
+// unrolled clock; see phys_slot) for traces too large for the single-block planner, which runs first: when it has
+// produced the plan (`done`), this grid returns at once.
+template <bool kCyclic>
+__global__ void __launch_bounds__(kPlanThreads, 1) k_plan_loop(PlanArgs A, const unsigned *done)
 {
+    if (kCyclic && *done) return;          // (same answer in every thread of the grid: written by an earlier launch)
+    if (kCyclic && blockIdx.x == 0 && threadIdx.x == 0) A.summary[7] = 0;      // (the single-block planner left "does not fit" there)
     __shared__ Cand s_cand[kPlanWarps + 1];
     __shared__ long long s_max[kPlanWarps + 1];
     const int G = gridDim.x, c = blockIdx.x;
@@ -32,7 +38,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_loop(PlanArgs A)
         for (int64_t p = (int64_t)c * kPlanWarps + warp; p < Pn; p += (int64_t)G * kPlanWarps) {
             if (A.dead[p]) continue;
             Cand cd;
-            if (!score_period(A, p, lane, &cd)) {
+            if (!score_period<kCyclic>(A, p, lane, &cd)) {
                 if (lane == 0) A.dead[p] = 1;       // channels only fill up: never admissible again
                 continue;
             }
@@ -69,7 +75,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_loop(PlanArgs A)
         if (win.idx < 0) { status = G10_EXHAUSTED; break; }
 
         int64_t sz = 0;
-        if (commit_winner(A, win.idx, win.dest, it, n_mig, c, G, &sz)) own_dirty = true;
+        if (commit_winner<kCyclic>(A, win.idx, win.dest, it, n_mig, c, G, &sz)) own_dirty = true;
         n_mig += 1;
         if (win.dest == G10_DEST_SSD) bytes_ssd += sz; else bytes_host += sz;
         if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
@@ -150,7 +156,15 @@ cudaError_t launch_plan_cyclic(const DeviceTrace &t, const Workspace &w, const P
     PlanArgs A;
     fill_plan_args(t, w, p, A);
     A.start = w.start2;
-    return launch_plan_one_cyclic(A, w, s);
+    // one block plans when everything fits its shared memory (decided on the device); the multi-block planner queued
+    // behind it does the work otherwise
+    cudaError_t e = launch_plan_one_cyclic(A, w, s);
+    if (e != cudaSuccess) return e;
+    const int G = blocks_for((const void *)k_plan_loop<true>);
+    if (G < 1) return cudaErrorLaunchFailure;
+    const unsigned *done = w.one_done;
+    void *args[] = {&A, &done};
+    return cudaLaunchCooperativeKernel((const void *)k_plan_loop<true>, dim3(G), dim3(kPlanThreads), args, 0, s);
 }
 
 // ORs the call's status word into *dst (which the planner may already have written)
@@ -167,10 +181,11 @@ cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const Pla
     PlanArgs A;
     fill_plan_args(t, w, p, A);
     if (p.flags & G10_FLAG_RESCORE_ALL) {
-        const int G = blocks_for((const void *)k_plan_loop);
+        const int G = blocks_for((const void *)k_plan_loop<false>);
         if (G < 1) return cudaErrorLaunchFailure;
-        void *args[] = {&A};
-        return cudaLaunchCooperativeKernel((const void *)k_plan_loop, dim3(G), dim3(kPlanThreads), args, 0, s);
+        const unsigned *done = w.one_done;
+        void *args[] = {&A, &done};
+        return cudaLaunchCooperativeKernel((const void *)k_plan_loop<false>, dim3(G), dim3(kPlanThreads), args, 0, s);
     }
     if (plan_keeps_state_on_chip(t.K, t.E, p.flags)) {
         int Gs = plan_small_blocks();

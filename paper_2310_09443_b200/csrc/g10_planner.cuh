@@ -81,6 +81,12 @@ __device__ __forceinline__ Cand cand_shfl_xor(const Cand &c, int o)
 // Is the channel free for the window [w0, w1) over slots k0..k1?  Each slot offers dur[k] ns of channel
 // time per device and direction; the window may be booked iff booked + overlap <= dur in every slot.
 // Called by a whole warp; returns the same answer in every lane.
+// kCyclic (steady-state planning): slot indices and A.start are unrolled over two iterations, while pressure, bookings,
+// host occupancy and durations belong to the physical slot (index - K beyond the first iteration).
+template <bool kCyclic>
+__device__ __forceinline__ int phys_slot(int64_t K, int k) { return kCyclic && k >= K ? k - (int)K : k; }
+
+template <bool kCyclic = false>
 __device__ __forceinline__ bool window_free(const PlanArgs &A, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane)
 {
     bool ok = true;
@@ -88,7 +94,7 @@ __device__ __forceinline__ bool window_free(const PlanArgs &A, const int64_t *bu
         const int64_t s0 = A.start[k], s1 = A.start[k + 1];
         const int64_t lo = w0 > s0 ? w0 : s0, hi = w1 < s1 ? w1 : s1;
         const int64_t ov = hi > lo ? hi - lo : 0;
-        if (busy[k] + ov > s1 - s0) ok = false;
+        if (busy[phys_slot<kCyclic>(A.K, k)] + ov > s1 - s0) ok = false;
     }
     return __all_sync(0xffffffffu, ok);
 }
@@ -179,6 +185,7 @@ __device__ __forceinline__ u128 benefit_tiles_warp(const int64_t *sP, const int6
 
 // Scores period p against the current state: destination (SSD first, then host) and benefit.
 // Whole warp; result valid in lane 0.  Returns false if no destination is admissible (permanent).
+template <bool kCyclic = false>
 __device__ __forceinline__ bool score_period(const PlanArgs &A, int64_t p, int lane, Cand *out)
 {
     const int i = A.per_t[p];
@@ -193,12 +200,12 @@ __device__ __forceinline__ bool score_period(const PlanArgs &A, int64_t p, int l
         if (ap < 0) continue;
         bp = A.geo_b[X * A.geo_stride + p];
         t = A.geo_t[X * A.geo_stride + p];
-        if (!window_free(A, A.busy + (size_t)(2 * X) * A.K, t_r, t_r + t, a, ap - 1, lane)) continue;
-        if (!window_free(A, A.busy + (size_t)(2 * X + 1) * A.K, t_end - t, t_end, bp + 1, b, lane)) continue;
+        if (!window_free<kCyclic>(A, A.busy + (size_t)(2 * X) * A.K, t_r, t_r + t, a, ap - 1, lane)) continue;
+        if (!window_free<kCyclic>(A, A.busy + (size_t)(2 * X + 1) * A.K, t_end - t, t_end, bp + 1, b, lane)) continue;
         if (X == G10_DEST_HOST && A.host_capacity != 0) {
             bool ok = true;
             for (int k = a + lane; k <= b; k += 32)
-                if ((uint64_t)A.hocc[k] + (uint64_t)s > A.host_capacity) ok = false;
+                if ((uint64_t)A.hocc[phys_slot<kCyclic>(A.K, k)] + (uint64_t)s > A.host_capacity) ok = false;
             if (!__all_sync(0xffffffffu, ok)) continue;
         }
         dest = X;
@@ -206,10 +213,11 @@ __device__ __forceinline__ bool score_period(const PlanArgs &A, int64_t p, int l
     if (dest < 0) return false;
     u128 acc = 0;
     for (int k = ap + lane; k <= bp; k += 32) {
-        int64_t ex = A.P[k] - A.cap;
+        const int kp = phys_slot<kCyclic>(A.K, k);
+        int64_t ex = A.P[kp] - A.cap;
         if (ex > 0) {
             if (ex > s) ex = s;
-            acc += (u128)(ull)ex * (u128)(ull)A.dur[k];
+            acc += (u128)(ull)ex * (u128)(ull)A.dur[kp];
         }
     }
     acc = warp_sum_u128(acc);
@@ -327,6 +335,7 @@ __device__ __forceinline__ long long own_slots_max(const PlanArgs &A, int c, int
 // Commits period p with destination X: pressure range-subtract and host occupancy on the slots this block
 // owns, channel bookings, the plan record and the erase flag by block 0.  Returns true if this block's
 // pressure slots changed.
+template <bool kCyclic = false>
 __device__ __forceinline__ bool commit_winner(const PlanArgs &A, int64_t p, int X, int64_t it, int64_t n_mig, int c, int G,
                                               int64_t *bytes_out, bool with_bookings = true)
 {
@@ -338,33 +347,38 @@ __device__ __forceinline__ bool commit_winner(const PlanArgs &A, int64_t p, int 
     const int64_t t = A.geo_t[X * A.geo_stride + p];
     const int64_t t_r = A.start[a], t_end = A.start[v];
     bool touched = false;
-    for (int tl = ap / kSlotTile; tl <= bp / kSlotTile; ++tl) {
-        if (tl % G != c) continue;
-        touched = true;
-        const int64_t k0 = (int64_t)tl * kSlotTile;
-        for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < K; k += kPlanThreads)
-            if (k >= ap && k <= bp) A.P[k] -= s;
-    }
-    if (X == G10_DEST_HOST && A.host_capacity != 0) {
-        for (int tl = a / kSlotTile; tl <= b / kSlotTile; ++tl) {
-            if (tl % G != c) continue;
-            const int64_t k0 = (int64_t)tl * kSlotTile;
-            for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < K; k += kPlanThreads)
-                if (k >= a && k <= b) A.hocc[k] += s;
+    // adds `delta` to arr over the unrolled slots [lo, hi], on the tiles this block owns (a range that reaches into the next
+    // iteration -- steady-state planning only -- is two runs of physical slots)
+    auto range_add = [&](int64_t *arr, int lo, int hi, int64_t delta, bool mark) {
+        for (int part = 0; part < (kCyclic ? 2 : 1); ++part) {
+            int plo = lo, phi = hi;
+            if (kCyclic) {
+                if (part == 0) { if (lo >= K) continue; phi = hi < K ? hi : (int)K - 1; }
+                else { if (hi < K) continue; plo = (lo > K ? lo : (int)K) - (int)K; phi = hi - (int)K; }
+            }
+            for (int tl = plo / kSlotTile; tl <= phi / kSlotTile; ++tl) {
+                if (tl % G != c) continue;
+                if (mark) touched = true;
+                const int64_t k0 = (int64_t)tl * kSlotTile;
+                for (int64_t k = k0 + threadIdx.x; k < k0 + kSlotTile && k < K; k += kPlanThreads)
+                    if (k >= plo && k <= phi) arr[k] += delta;
+            }
         }
-    }
+    };
+    range_add(A.P, ap, bp, -s, true);
+    if (X == G10_DEST_HOST && A.host_capacity != 0) range_add(A.hocc, a, b, s, false);
     if (c == 0) {
         if (with_bookings) {
             int64_t *bo = A.busy + (size_t)(2 * X) * K, *bi = A.busy + (size_t)(2 * X + 1) * K;
             for (int k = a + threadIdx.x; k <= ap - 1; k += kPlanThreads) {
                 const int64_t s0 = A.start[k], s1 = A.start[k + 1];
                 const int64_t lo = t_r > s0 ? t_r : s0, hi = (t_r + t) < s1 ? (t_r + t) : s1;
-                if (hi > lo) bo[k] += hi - lo;
+                if (hi > lo) bo[phys_slot<kCyclic>(K, k)] += hi - lo;
             }
             for (int k = bp + 1 + threadIdx.x; k <= b; k += kPlanThreads) {
                 const int64_t s0 = A.start[k], s1 = A.start[k + 1];
                 const int64_t lo = (t_end - t) > s0 ? (t_end - t) : s0, hi = t_end < s1 ? t_end : s1;
-                if (hi > lo) bi[k] += hi - lo;
+                if (hi > lo) bi[phys_slot<kCyclic>(K, k)] += hi - lo;
             }
         }
         if (threadIdx.x == 0) {
