@@ -41,10 +41,6 @@ L2_FLUSH_BYTES = 512 << 20
 # of the kernel sources at the time of the capture: when the sources have changed since, the bench line says so
 # ("traffic_stale") instead of passing old traffic off as current.
 TRAFFIC = {"vitality": 194_200_000, "timeline": 160_000_000, "captured_at": "2026-11-25", "sources_sha256": "unset"}
-# kernels launched per call (counted from the launch lists in profiles/): vitality = bucket histogram, partition, emit,
-# status; timeline = slot-clock scan, first/last pairs, difference scatter, pressure scan, status (+ 1 memset node each)
-KERNELS_PER_VITALITY = 4
-KERNELS_PER_TIMELINE = 5
 
 
 def kernel_sources_sha256():
@@ -341,6 +337,7 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    launches0 = binding.g10_launch_count()
     total_ms = 0.0
     for _ in range(args.steps):
         flush.fill_(1)                      # L2 flush between timed iterations (outside the event pair)
@@ -350,6 +347,7 @@ def run_ours(args):
         b.record()
         b.synchronize()
         total_ms += a.elapsed_time(b)
+    gpu_launches = binding.g10_launch_count() - launches0
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = max_over_ranks(torch, dist, world, total_ms, dev)
@@ -519,9 +517,9 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": "events/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
                 "note": "host-pointer form of both calls: each stages the trace itself and copies all its outputs back"},
-        "gpu_launches": args.steps * (KERNELS_PER_VITALITY + KERNELS_PER_TIMELINE),
-        "gpu_launches_note": "kernels of this library inside the timed region: %d per g10_vitality + %d per g10_pressure_timeline, "
-                             "from the ncu launch list in profiles/ (plus one memset node per call)" % (KERNELS_PER_VITALITY, KERNELS_PER_TIMELINE),
+        "gpu_launches": gpu_launches,
+        "gpu_launches_note": "counted by the library itself (g10_launch_count before and after the timed region): its own kernels only, "
+                             "%d per step; memset nodes and the L2 flush are not counted" % (gpu_launches // max(args.steps, 1)),
         "clocks": clocks,
         "roofline": roof,
         "behind_the_plan": extras,

@@ -355,6 +355,9 @@ int32_t g10_workspace_bytes(int32_t which, int64_t num_kernels, int64_t num_tens
 
 const char *g10_strerror(int32_t code);
 int32_t g10_version(void);
+/* Diagnostic: kernels this library has launched in the process so far (a benchmark reads it before and after its timed
+   region to say how many of the library's own kernels ran there). */
+uint64_t g10_launch_count(void);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,7 @@ FLAG_GLOBAL_STATE = 2
 FLAG_MULTI_BLOCK = 4
 STATUS = {0: "ALREADY_FITS", 1: "FIT", 2: "EXHAUSTED", 3: "ITERATION_LIMIT"}
 EXPORTS = ("g10_vitality", "g10_pressure_timeline", "g10_candidate_geometry", "g10_plan_migrations",
-           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize", "g10_plan_batch", "g10_plan_cyclic")
+           "g10_workspace_bytes", "g10_strerror", "g10_version", "g10_pressure_timeline_static", "g10_schedule_prefetch", "g10_emit_instructions", "g10_characterize", "g10_plan_batch", "g10_plan_cyclic", "g10_launch_count")
 STATIC_MAX_KERNELS, STATIC_MAX_TENSORS = 32768, 131072
 
 INSTRUCTION_DTYPE = np.dtype([("opcode", "<i4"), ("tensor", "<i4"), ("target", "<i4"), ("record", "<i4"),
@@ -107,6 +107,8 @@ def load_library():
         lib.g10_strerror.restype = C.c_char_p
         lib.g10_strerror.argtypes = [C.c_int32]
         lib.g10_version.restype = C.c_int32
+        lib.g10_launch_count.restype = C.c_uint64
+        lib.g10_launch_count.argtypes = []
         lib.g10_workspace_bytes.restype = C.c_int32
         lib.g10_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.POINTER(C.c_size_t)]
         lib.g10_vitality.restype = C.c_int32
@@ -201,6 +203,11 @@ def pin(trace) -> TraceBuffers:
     f = lambda a: torch.from_numpy(_nonempty(a)).pin_memory()
     return TraceBuffers(f(trace.kernel_ptr), f(trace.kernel_tensors), f(trace.tensor_bytes), f(trace.kernel_ns),
                         f(trace.tensor_global) if trace.tensor_global is not None else None, trace.K, trace.N, trace.E)
+
+
+def g10_launch_count() -> int:
+    """Kernels the library has launched in this process so far."""
+    return int(load_library().g10_launch_count())
 
 
 def g10_workspace_bytes(which, K, N, E, mem=MEM_DEVICE) -> int:

@@ -6,6 +6,7 @@
 #include "g10_internal.h"
 
 namespace g10 {
+ull g_launch_count = 0;
 namespace {
 
 struct Sizes {
@@ -226,6 +227,8 @@ using namespace g10;
 extern "C" {
 
 int32_t g10_version(void) { return G10_VERSION; }
+
+uint64_t g10_launch_count(void) { return __atomic_load_n(&g_launch_count, __ATOMIC_RELAXED); }
 
 const char *g10_strerror(int32_t code)
 {

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(kCycThreads) k_cyclic_prepare(int64_t K, int64
 cudaError_t launch_cyclic_prepare(const DeviceTrace &t, const Workspace &w, cudaStream_t s)
 {
     k_cyclic_prepare<<<1, kCycThreads, 0, s>>>(t.K, t.N, w.start, w.start2, t.tensor_global, w.first_use, w.last_use, t.E,
-                                               w.period_tensor, w.period_prev_use, w.period_next_use, w.counts, w.status);
+                                               w.period_tensor, w.period_prev_use, w.period_next_use, w.counts, w.status); count_launch();
     return cudaGetLastError();
 }
 

@@ -322,14 +322,14 @@ cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s)
     int64_t g = (total + kEmitThreads - 1) / kEmitThreads;
     if (g > 4 * (int64_t)sms) g = 4 * (int64_t)sms;
     if (g < 1) g = 1;
-    k_emit_hist<<<(int)g, kEmitThreads, sizeof(unsigned) * (size_t)A.nb, s>>>(A);
-    k_emit_scatter<<<(int)g, kEmitThreads, sizeof(long long) * (size_t)(A.nb + 1), s>>>(A);
+    k_emit_hist<<<(int)g, kEmitThreads, sizeof(unsigned) * (size_t)A.nb, s>>>(A); count_launch();
+    k_emit_scatter<<<(int)g, kEmitThreads, sizeof(long long) * (size_t)(A.nb + 1), s>>>(A); count_launch();
     const size_t sm3 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(int) * (size_t)(2 * (1 << A.shift) + 2) + 8 +
                        (sizeof(ull) + sizeof(int32_t)) * kEmitCap;
     cudaError_t e = cudaFuncSetAttribute(k_emit_write, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
     const int g3 = A.nb < 2 * sms ? A.nb : 2 * sms;
-    k_emit_write<<<g3, kEmitThreads, sm3, s>>>(A, L.inst_ptr, L.inst, L.inst_cap, L.counts);
+    k_emit_write<<<g3, kEmitThreads, sm3, s>>>(A, L.inst_ptr, L.inst, L.inst_cap, L.counts); count_launch();
     return cudaGetLastError();
 }
 

@@ -11,6 +11,15 @@ namespace g10 {
 
 typedef unsigned long long ull;
 
+// Kernels this library has launched in the process so far (every launch site counts itself; read through
+// g10_launch_count, which benchmarks use to report how many of the library's kernels ran inside a timed region).
+extern ull g_launch_count;
+inline void count_launch() { __atomic_fetch_add(&g_launch_count, 1ull, __ATOMIC_RELAXED); }
+}  // namespace g10
+#define cudaLaunchKernelEx(...) (g10::count_launch(), ::cudaLaunchKernelEx(__VA_ARGS__))
+#define cudaLaunchCooperativeKernel(...) (g10::count_launch(), ::cudaLaunchCooperativeKernel(__VA_ARGS__))
+namespace g10 {
+
 constexpr size_t kAlign = 256;
 constexpr int kHeavyThreshold = 32;      // tensors with more raw uses than this are sorted by a whole block
 

@@ -220,7 +220,7 @@ cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t 
 {
     const int G = seg_scan_blocks(t.K);
     k_seg_scan<0><<<G, kSegThreads, 0, s>>>(t.K, t.E, t.kernel_ns, t.kernel_ptr, start, w.clock_scan.ticket, w.clock_scan.done,
-                                          w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status);
+                                          w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status); count_launch();
     return cudaGetLastError();
 }
 
@@ -453,7 +453,7 @@ cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t 
     if (e != cudaSuccess) return e;
     if (t.E > 0 && t.K > 0) {
         const int blocks = (int)tiles_of(t.K, kFlThreads);
-        k_first_last_events<<<blocks, kFlThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.event_budget, w.status);
+        k_first_last_events<<<blocks, kFlThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, first_use, last_use, w.event_budget, w.status); count_launch();
     }
     return cudaGetLastError();
 }
@@ -686,22 +686,22 @@ __global__ void __launch_bounds__(kEmThreads) k_vitality_emit(int64_t N, const i
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s)
 {
     if (t.E > 0 && t.N > 0) {
-        k_count_events<<<(unsigned)tiles_of(t.E, kEvTile), kEvThreads, 0, s>>>(t.E, t.N, t.kernel_tensors, w.cnt, w.status);
+        k_count_events<<<(unsigned)tiles_of(t.E, kEvTile), kEvThreads, 0, s>>>(t.E, t.N, t.kernel_tensors, w.cnt, w.status); count_launch();
     }
     {
         const int tiles = (int)tiles_of(t.N, kScanTile);
         TileState<1> st{w.count_scan.ticket, w.count_scan.flag, w.count_scan.agg, w.count_scan.incl};
-        k_scan_counts<<<tiles, kScanThreads, 0, s>>>(t.N, w.cnt, w.raw_ptr, w.heavy_list, w.heavy_count, st, tiles, w.status);
+        k_scan_counts<<<tiles, kScanThreads, 0, s>>>(t.N, w.cnt, w.raw_ptr, w.heavy_list, w.heavy_count, st, tiles, w.status); count_launch();
     }
     if (t.E > 0 && t.N > 0 && t.K > 0) {
         k_scatter_events<<<(unsigned)tiles_of(t.E, kEvTile), kEvThreads, 0, s>>>(t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors,
-                                                                                 w.raw_ptr, w.cnt, w.raw_uses);
-        k_sort_heavy<<<64, kHeavyThreads, 0, s>>>(w.heavy_count, w.heavy_list, w.raw_ptr, w.raw_uses, w.cnt, w.heavy_info);
+                                                                                 w.raw_ptr, w.cnt, w.raw_uses); count_launch();
+        k_sort_heavy<<<64, kHeavyThreads, 0, s>>>(w.heavy_count, w.heavy_list, w.raw_ptr, w.raw_uses, w.cnt, w.heavy_info); count_launch();
     }
     {
         const int tiles = (int)tiles_of(t.N, kEmTile);
         TileState<2> st{w.emit_scan.ticket, w.emit_scan.flag, w.emit_scan.agg, w.emit_scan.incl};
-        k_vitality_emit<<<tiles, kEmThreads, 0, s>>>(t.N, w.raw_ptr, w.raw_uses, w.cnt, w.heavy_info, out, st, tiles, w.status);
+        k_vitality_emit<<<tiles, kEmThreads, 0, s>>>(t.N, w.raw_ptr, w.raw_uses, w.cnt, w.heavy_info, out, st, tiles, w.status); count_launch();
     }
     return cudaGetLastError();
 }
@@ -879,7 +879,7 @@ cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, 
 {
     if (Pn_bound <= 0) return cudaSuccess;
     k_geometry<<<(unsigned)((Pn_bound + 255) / 256), 256, 0, s>>>(K, Pn_bound, Pn_dev, start, tensor_bytes, per_t, per_u, per_v,
-                                                                  host_bw, ssd_bw, stride, geo_t, geo_a, geo_b);
+                                                                  host_bw, ssd_bw, stride, geo_t, geo_a, geo_b); count_launch();
     return cudaGetLastError();
 }
 

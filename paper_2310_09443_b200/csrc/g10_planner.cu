@@ -88,7 +88,7 @@ __global__ void k_publish_status(const ull *status, int64_t *dst) { *dst = (int6
 
 cudaError_t launch_publish_status(const Workspace &w, int64_t *dst, cudaStream_t s)
 {
-    k_publish_status<<<1, 1, 0, s>>>(w.status, dst);
+    k_publish_status<<<1, 1, 0, s>>>(w.status, dst); count_launch();
     return cudaGetLastError();
 }
 
@@ -172,7 +172,7 @@ __global__ void k_publish_status_or(const ull *status, int64_t *dst) { *dst |= (
 
 cudaError_t launch_publish_status_or(const Workspace &w, int64_t *dst, cudaStream_t s)
 {
-    k_publish_status_or<<<1, 1, 0, s>>>(w.status, dst);
+    k_publish_status_or<<<1, 1, 0, s>>>(w.status, dst); count_launch();
     return cudaGetLastError();
 }
 

@@ -605,7 +605,7 @@ cudaError_t launch_plan_one(const PlanArgs &A_in, const Workspace &w, cudaStream
     O.smem_bytes = one_smem_budget<false, false>();
     cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
     if (e != cudaSuccess) return e;
-    k_plan_one<false, false><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    k_plan_one<false, false><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B); count_launch();
     return cudaGetLastError();
 }
 
@@ -620,7 +620,7 @@ cudaError_t launch_plan_one_cyclic(const PlanArgs &A_in, const Workspace &w, cud
     O.smem_bytes = one_smem_budget<false, true>();
     cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
     if (e != cudaSuccess) return e;
-    k_plan_one<false, true><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    k_plan_one<false, true><<<1, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B); count_launch();
     return cudaGetLastError();
 }
 
@@ -672,10 +672,10 @@ cudaError_t launch_plan_batch(const PlanArgs &A_in, const Workspace &w, int V, c
     O.smem_bytes = one_smem_budget<true, false>();
     cudaError_t e = cudaFuncSetAttribute((const void *)k_plan_one<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, O.smem_bytes);
     if (e != cudaSuccess) return e;
-    k_plan_one<true, false><<<V, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B);
+    k_plan_one<true, false><<<V, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B); count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const int64_t bound = A.geo_stride < batch_max_periods() ? A.geo_stride : batch_max_periods();
-    k_batch_finish<<<V, 256, (size_t)((bound + 31) / 32) * 4, s>>>(bound, A.Pn_dev, A.out, A.out_cap, A.summary, stability, A.status);
+    k_batch_finish<<<V, 256, (size_t)((bound + 31) / 32) * 4, s>>>(bound, A.Pn_dev, A.out, A.out_cap, A.summary, stability, A.status); count_launch();
     return cudaGetLastError();
 }
 

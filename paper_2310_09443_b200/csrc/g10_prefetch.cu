@@ -422,19 +422,19 @@ cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *
             const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
             if (e != cudaSuccess) return e;
         }
-        k_schedule_prefetch<256><<<1, 256, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem);
+        k_schedule_prefetch<256><<<1, 256, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem); count_launch();
     } else if (tiles <= kPfMaxTiles) {
         sort_smem = (n > 0 && (size_t)n2 * 12 + (size_t)tiles * 16 <= 200 * 1024) ? 1 : 0;   // (this kernel has most of the SM's shared memory to itself)
         dyn = (sort_smem ? ((size_t)n2 * 12 + 7) / 8 * 8 : 0) + (size_t)tiles * 16;
         const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch_tiled, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
         if (e != cudaSuccess) return e;
-        k_schedule_prefetch_tiled<<<1, kPfNT, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, sort_smem);
+        k_schedule_prefetch_tiled<<<1, kPfNT, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, sort_smem); count_launch();
     } else {
         if (dyn > 0) {
             const cudaError_t e = cudaFuncSetAttribute(k_schedule_prefetch<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
             if (e != cudaSuccess) return e;
         }
-        k_schedule_prefetch<1024><<<1, 1024, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem);
+        k_schedule_prefetch<1024><<<1, 1024, dyn, s>>>(K, n, mig, start, bytes, cap, P, order, new_last, new_issue, summary, in_smem, sort_smem); count_launch();
     }
     return cudaGetLastError();
 }

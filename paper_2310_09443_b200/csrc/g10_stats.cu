@@ -117,12 +117,13 @@ cudaError_t launch_characterize(int64_t K, int64_t N, const int64_t *use_ptr, co
     if ((e = cudaMemsetAsync(size_len_hist, 0, kSizeBins * kLen2Bins * 8, s)) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(hide, 0, 16, s)) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(summary, 0, 16, s)) != cudaSuccess) return e;
-    if (N > 0 && K > 0) k_active_bytes<<<stat_grid(N, kStatThreads), kStatThreads, 0, s>>>(N, use_ptr, uses, bytes, (ull *)active);
-    if (Pn > 0)
+    if (N > 0 && K > 0) { k_active_bytes<<<stat_grid(N, kStatThreads), kStatThreads, 0, s>>>(N, use_ptr, uses, bytes, (ull *)active); count_launch(); }
+    if (Pn > 0) {
         k_period_hist<<<stat_grid(Pn, kStatThreads * 4), kStatThreads, 0, s>>>(Pn, start, bytes, per_t, per_u, per_v, host_bw, ssd_bw,
-                                                                               (ull *)len_hist, (ull *)size_len_hist, (ull *)hide);
-    k_active_max<<<stat_grid(K, kStatThreads * 4), kStatThreads, 0, s>>>(K, (const long long *)active, (long long *)summary);
-    if (K > 0) k_active_argmax<<<stat_grid(K, kStatThreads * 4), kStatThreads, 0, s>>>(K, (const long long *)active, (long long *)summary);
+                                                                               (ull *)len_hist, (ull *)size_len_hist, (ull *)hide); count_launch();
+    }
+    k_active_max<<<stat_grid(K, kStatThreads * 4), kStatThreads, 0, s>>>(K, (const long long *)active, (long long *)summary); count_launch();
+    if (K > 0) { k_active_argmax<<<stat_grid(K, kStatThreads * 4), kStatThreads, 0, s>>>(K, (const long long *)active, (long long *)summary); count_launch(); }
     return cudaGetLastError();
 }
 

@@ -566,7 +566,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     cfg.numAttrs = 1;
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
-        k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
+        k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors); count_launch();
         // Shared memory of the partition kernel: three bucket tables and ten bytes per staged event; two blocks per SM.
         const size_t tables = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8;
         int64_t cap = ((int64_t)(100 << 10) - (int64_t)tables) / 10 / kBkThreads * kBkThreads;
