@@ -56,7 +56,7 @@ extern "C" {
 #define G10_DEV_PERIODS_OVERFLOW 0x20 /* periods_cap too small (counts[1] holds the need)         */
 #define G10_DEV_PLAN_OVERFLOW 0x40   /* migrations_cap too small (summary[0] holds the need)      */
 #define G10_DEV_TIMEOUT 0x80         /* an internal wait gave up; the kernel returned early       */
-#define G10_DEV_BATCH_UNFIT 0x100    /* g10_plan_batch: the trace does not fit one SM (no plan)   */
+#define G10_DEV_BATCH_UNFIT 0x100    /* internal: the trace does not fit one SM (g10_plan_batch then plans the variants one by one) */
 
 /* exit status of the planner (summary[2]) */
 #define G10_ALREADY_FITS 0      /* unplanned peak pressure <= capacity, empty plan                 */
@@ -285,9 +285,12 @@ int32_t g10_plan_cyclic(const g10_trace *trace, uint64_t gpu_capacity_bytes, uin
    final_pressure [V][K], summary [V][8] (as in g10_plan_out; summary[8 v + 7] holds the status bits of variant v),
    stability [V][2] = (|M_v & M_0|, |M_v | M_0|) over the sets of migrated periods of variant v and variant 0 (their
    quotient is the Jaccard index; (-1, -1) when a plan is missing).
-   Limits: the trace has to be device resident (G10_MEM_DEVICE); 1 <= V <= 1024; pressure, clock, bookings and the
-   periods of the trace must fit the shared memory of one SM (the DNN-shaped traces of a few thousand kernels do),
-   else every variant reports G10_DEV_BATCH_UNFIT and summary[2] = -1: plan such traces one by one.
+   Limits: the trace has to be device resident (G10_MEM_DEVICE); 1 <= V <= 1024.
+   One block per variant requires that pressure, clock, bookings and the periods of the trace fit the shared memory of
+   one SM (the DNN-shaped traces of a few thousand kernels do).  Only the device can tell, so the call reads variant
+   0's summary back (one small copy and a synchronisation of `stream`: unlike the other calls this one returns with
+   its kernels finished); if the trace did not fit, the variants are then planned one after the other by the planners
+   that use the whole GPU -- the same results, V times the time of one plan.
    Workspace: G10_WS_BATCH. */
 typedef struct g10_variant {
     const int64_t *kernel_ns;       /* [K] device pointer, or NULL: the trace's own durations */

@@ -507,6 +507,34 @@ int32_t g10_plan_batch(const g10_trace *trace, int32_t V, const g10_variant *var
     CU(buckets ? launch_vitality_buckets(d, w, vb, s) : launch_vitality(d, w, vb, s));
     CU(launch_pressure(d, w, w.first_use, w.last_use, false, w.pressure, w.peak_bytes, w.peak_slot, s));
     CU(launch_plan_variants(d, w, pp, V, out->stability, s));
+    // One block per variant needs the trace to fit the shared memory of one SM, which only the device can tell (the
+    // number of periods is counted there).  Variant 0 says so: if it could not be planned, the variants are planned one
+    // after the other by the planners that use the whole GPU.  Asking costs one small copy and a synchronisation.
+    int64_t first[8];
+    CU(cudaMemcpyAsync(first, out->summary, sizeof(first), cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    if (!(first[2] == -1 && (first[7] & G10_DEV_BATCH_UNFIT))) return G10_OK;
+    CU(launch_publish_status(w, w.counts + 3, s));              // what trace validation found: folded into every variant at the end
+    for (int32_t v = 0; v < V; ++v) {
+        CU(cudaMemsetAsync(w.zero_begin, 0, w.zero_bytes, s));
+        CU(cudaMemsetAsync(w.busy, 0, w.state_bytes, s));
+        DeviceTrace dv = d;
+        dv.kernel_ns = bv[v].kernel_ns;
+        PlanParams pv;
+        pv.gpu_capacity_bytes = bv[v].cap; pv.host_bw = bv[v].host_bw; pv.ssd_bw = bv[v].ssd_bw; pv.host_capacity_bytes = bv[v].host_capacity;
+        pv.max_iterations = max_iterations; pv.flags = 0;
+        pv.migrations = out->migrations ? out->migrations + (size_t)v * (size_t)out->migrations_cap : nullptr;
+        pv.migrations_cap = out->migrations_cap;
+        pv.final_pressure = out->final_pressure + (size_t)v * (size_t)d.K;
+        pv.summary = out->summary + (size_t)v * 8;
+        CU(launch_slot_clock(dv, w, w.start, s));               // this variant's clock (and the check of its durations)
+        if (d.K > 0) CU(cudaMemcpyAsync(pv.final_pressure, w.pressure, sizeof(int64_t) * (size_t)d.K, cudaMemcpyDeviceToDevice, s));
+        CU(launch_geometry(d.K, d.E, w.counts + 1, w.start, d.tensor_bytes, w.period_tensor, w.period_prev_use, w.period_next_use,
+                           pv.host_bw, pv.ssd_bw, d.E > 0 ? d.E : 1, w.geo_t, w.geo_a, w.geo_b, s));
+        CU(launch_plan_loop(dv, w, pv, s));
+        CU(launch_publish_status(w, pv.summary + 7, s));
+    }
+    CU(launch_batch_finish(d, w, pp, V, out->stability, (const ull *)(w.counts + 3), s));
     return G10_OK;
 }
 

@@ -222,6 +222,9 @@ cudaError_t launch_plan_loop(const DeviceTrace &t, const Workspace &w, const Pla
 cudaError_t launch_cyclic_prepare(const DeviceTrace &t, const Workspace &w, cudaStream_t s);
 cudaError_t launch_plan_cyclic(const DeviceTrace &t, const Workspace &w, const PlanParams &p, cudaStream_t s);
 cudaError_t launch_plan_variants(const DeviceTrace &t, const Workspace &w, const PlanParams &p, int V, int64_t *stability, cudaStream_t s);
+// stability pairs of V finished plans against plan 0; ORs *status_word into every plan's summary[7]
+cudaError_t launch_batch_finish(const DeviceTrace &t, const Workspace &w, const PlanParams &p, int V, int64_t *stability, const ull *status_word,
+                                cudaStream_t s);
 int plan_loop_max_blocks();
 bool plan_keeps_state_on_chip(int64_t K, int64_t E, uint32_t flags);   // true: the small-trace planner will run
 cudaError_t launch_publish_status(const Workspace &w, int64_t *dst, cudaStream_t s);

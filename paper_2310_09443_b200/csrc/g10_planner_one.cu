@@ -661,7 +661,24 @@ __global__ void __launch_bounds__(256) k_batch_finish(int64_t Pn_bound, const in
 
 int batch_max_periods()          // periods whose bitmap fits the finishing kernel's shared memory
 {
-    return 40 * 1024 * 8;
+    return 200 * 1024 * 8;
+}
+
+static cudaError_t run_batch_finish(int64_t geo_stride, const int64_t *Pn_dev, const g10_migration *mig, int64_t out_cap, int64_t *summary,
+                                    int V, int64_t *stability, const ull *status_word, cudaStream_t s)
+{
+    const int64_t bound = geo_stride < batch_max_periods() ? geo_stride : batch_max_periods();
+    const size_t smem = (size_t)((bound + 31) / 32) * 4;
+    cudaError_t e = cudaFuncSetAttribute((const void *)k_batch_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_batch_finish<<<V, 256, smem, s>>>(bound, Pn_dev, mig, out_cap, summary, stability, status_word); count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_batch_finish(const DeviceTrace &t, const Workspace &w, const PlanParams &p, int V, int64_t *stability, const ull *status_word,
+                                cudaStream_t s)
+{
+    return run_batch_finish(t.E > 0 ? t.E : 1, w.counts + 1, p.migrations, p.migrations_cap, p.summary, V, stability, status_word, s);
 }
 
 cudaError_t launch_plan_batch(const PlanArgs &A_in, const Workspace &w, int V, const BatchArgs &B, int64_t *stability, cudaStream_t s)
@@ -674,9 +691,7 @@ cudaError_t launch_plan_batch(const PlanArgs &A_in, const Workspace &w, int V, c
     if (e != cudaSuccess) return e;
     k_plan_one<true, false><<<V, kOneThreads, (size_t)O.smem_bytes, s>>>(A, O, B); count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    const int64_t bound = A.geo_stride < batch_max_periods() ? A.geo_stride : batch_max_periods();
-    k_batch_finish<<<V, 256, (size_t)((bound + 31) / 32) * 4, s>>>(bound, A.Pn_dev, A.out, A.out_cap, A.summary, stability, A.status); count_launch();
-    return cudaGetLastError();
+    return run_batch_finish(A.geo_stride, A.Pn_dev, A.out, A.out_cap, A.summary, V, stability, A.status, s);
 }
 
 }  // namespace g10

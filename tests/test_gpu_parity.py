@@ -605,13 +605,17 @@ def test_batched_replanning(gpu, oracle):
     torch.cuda.synchronize()
     s7 = _np(got.summary)[:, 7]
     assert s7[0] == 0 and (s7[1] & 0x8) and s7[2] == 0
-    # a trace too large for one SM: every variant says so, nothing else is written
+    # a trace too large for one SM: the variants are planned one after the other by the planners that use the whole GPU
     tr = traces.make_config(3)
-    tb = gpu.upload(tr)
-    got = gpu.g10_plan_batch(tb, [dict(gpu_capacity_bytes=1 << 30, host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)] * 2)
-    torch.cuda.synchronize()
-    s = _np(got.summary)
-    assert (s[:, 7] & 0x100).all() and (s[:, 2] == -1).all() and (_np(got.stability) == -1).all()
+    start, P0, peak, slot = oracle.timeline(tr)
+    base = dict(gpu_capacity_bytes=tr.capacity_from_peak(peak), host_bw=tr.host_bw, ssd_bw=tr.ssd_bw)
+    variants = [base, dict(base, kernel_ns=_jitter(rng, tr.kernel_ns, 10)), dict(base, ssd_bw=4 * tr.ssd_bw),
+                dict(base, gpu_capacity_bytes=base["gpu_capacity_bytes"] * 3 // 4, host_capacity_bytes=64 << 30),
+                dict(base, kernel_ns=_jitter(rng, tr.kernel_ns, 25), host_bw=2 * tr.host_bw)]
+    ref = check_batch(gpu, oracle, tr, variants)
+    assert ref.stability[0, 0] == ref.stability[0, 1] == len(ref.plans[0].migrations) > 1000
+    ref = check_batch(gpu, oracle, tr, variants[:2], max_iterations=50)
+    assert len(ref.plans[1].migrations) == 50
 
 
 def check_cyclic(gpu, oracle, tr, cap, host_capacity=0, max_iterations=0):
