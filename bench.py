@@ -10,7 +10,7 @@ trace (config 1).  The same line carries the plan of every configuration (`plans
 trace eight times the size (`scale_x8`), the calls behind the plan (prefetch pass, instruction stream, batched and
 cyclic planning), the roofline of the passes and the CPU oracle timed beside them.  Prints ONE JSON line (rank 0).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick | --passes-only]
 
 With N > 1 (torchrun) every rank works on its own replica of the trace (the path does not shard: the greedy loop
 is a strict sequence); value is the aggregate over ranks, time the max over ranks.
@@ -415,6 +415,11 @@ def run_ours(args):
               "timeline_roofline": roofline(tl_bytes, tl_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["timeline"]),
               "repetitions": reps, "l2": "flushed between timed calls (the *_warm_l2 figures: not flushed)"}
 
+    if args.passes_only:                   # (small profiling target: the headline and the per-call figures only)
+        print(json.dumps({"metric": "trace_events_per_s", "value": value, "unit": "events/s", "ms_per_step": step_s * 1e3, "steps": args.steps,
+                          "config": {"workload": WORKLOAD, "K": K, "N": N, "E": E}, "passes": passes, "roofline": roof, "gpu_launches": gpu_launches}))
+        return
+
     # ---- whole plans, every configuration (median of >= 3 timed calls after warm-up; config 1 with stage events)
     plans = {}
     kept = None
@@ -570,7 +575,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--quick", action="store_true", help="headline, plans and per-call rooflines only (small profiling target)")
+    ap.add_argument("--quick", action="store_true", help="headline, plans and per-call rooflines only")
+    ap.add_argument("--passes-only", action="store_true", help="headline and per-call rooflines only (small profiling target)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
