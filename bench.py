@@ -37,10 +37,12 @@ WORKLOAD = "config4_stress_dag"
 PLAN_WORKLOAD = "config1_resnet152_b256"
 L2_FLUSH_BYTES = 512 << 20
 # DRAM bytes per call on the stress trace (dram__bytes_read.sum + dram__bytes_write.sum summed over the call's kernels), from
-# the one-pass ncu capture whose command and table are in profiles/passes_config4_stress.md.  SOURCES_SHA256 is the hash
-# of the kernel sources at the time of the capture: when the sources have changed since, the bench line says so
-# ("traffic_stale") instead of passing old traffic off as current.
-TRAFFIC = {"vitality": 194_200_000, "timeline": 160_000_000, "captured_at": "2026-11-25", "sources_sha256": "unset"}
+# the one-pass ncu capture whose command and table are in profiles/passes_config4_stress.md (the capture that leaves the
+# caches alone between launches, as this program does: the write-back of the L2 flush's dirty lines is part of it).
+# "sources_sha256" is the hash of the kernel sources at the time of the capture: when the sources have changed since, the
+# bench line says so ("traffic_stale") instead of passing old traffic off as current, and a CPU test warns.
+TRAFFIC = {"vitality": 242_500_000, "timeline": 110_000_000, "captured_at": "2026-11-25",
+           "sources_sha256": "277666adb10f5bf245a5b4acd77d73e540cdfbe8fd3a12fc8bbb6aa9fa3787c1"}
 
 
 def kernel_sources_sha256():
@@ -409,7 +411,7 @@ def run_ours(args):
                     ms=step_s * 1e3, algorithmic_bytes_per_event=(vit_bytes + tl_bytes) / E,
                     roofline_events_per_s=E / ((vit_bytes + tl_bytes) / (hbm_peak * 1e9)),
                     note="random accesses of the passes are bound by the L2's rate of scattered 32-byte sector requests "
-                         "(about 170 G/s measured on this part), not by HBM bytes: see DESIGN.md section 6")
+                         "(about 170 G/s measured on this part), not by HBM bytes")
     passes = {"vitality_ms": vit_cold, "timeline_ms": tl_cold, "vitality_ms_warm_l2": vit_warm, "timeline_ms_warm_l2": tl_warm,
               "vitality_roofline": roofline(vit_bytes, vit_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["vitality"]),
               "timeline_roofline": roofline(tl_bytes, tl_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["timeline"]),

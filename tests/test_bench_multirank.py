@@ -44,3 +44,21 @@ def test_reference_arm_runs_on_cpu():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["metric"] == "trace_events_per_s" and line["value"] > 0
     assert line["config"]["workload"] == "config4_stress_dag" and line["plan_workload"] == "config1_resnet152_b256" and line["cpu_baseline"]["kind"] == "oracle"
+
+
+def test_traffic_constants_carry_the_hash_of_the_sources_they_were_captured_on():
+    """The DRAM traffic in the bench line is a stored ncu figure: it is tagged with the hash of the kernel sources it was
+    captured on, and a bench line on other sources says "traffic_stale".  A stale tag is reported here as a warning."""
+    import warnings
+
+    sys.path.insert(0, ROOT)
+    import bench
+
+    now = bench.kernel_sources_sha256()
+    assert len(now) == 64 and int(now, 16) >= 0
+    assert set(bench.TRAFFIC) == {"vitality", "timeline", "captured_at", "sources_sha256"}
+    assert len(bench.TRAFFIC["sources_sha256"]) == 64, "the traffic constants carry no source hash"
+    assert bench.TRAFFIC["vitality"] > 0 and bench.TRAFFIC["timeline"] > 0
+    if now != bench.TRAFFIC["sources_sha256"]:
+        warnings.warn("kernel sources changed since the DRAM traffic in bench.py was captured: re-capture it "
+                      "(profiles/passes_config4_stress.md has the command)")
