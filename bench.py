@@ -443,12 +443,18 @@ def run_ours(args):
         for cfg in (1, 4):
             trc, tbc, wsc, planc, tlc, capc = kept[cfg]
             n_mig = int(planc.summary[0].item())
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            P = planc.final_pressure.clone()
-            a.record()
-            pf = binding.g10_schedule_prefetch(trc.K, n_mig, planc.migrations, tlc.kernel_start_ns, tbc.tensor_bytes, capc, P)
-            b.record()
-            torch.cuda.synchronize()
+            pws = torch.empty(max(256, binding.g10_workspace_bytes(binding.WS_PREFETCH, trc.K, 0, n_mig)), dtype=torch.uint8, device=dev)
+            pf_ms = []
+            for _ in range(4):                                        # (the pass rewrites the pressure curve it is given: a fresh copy per call)
+                P = planc.final_pressure.clone()
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                pf = binding.g10_schedule_prefetch(trc.K, n_mig, planc.migrations, tlc.kernel_start_ns, tbc.tensor_bytes, capc, P, ws=pws)
+                b.record()
+                torch.cuda.synchronize()
+                pf_ms.append(a.elapsed_time(b))
+            assert int(pf.summary[4].item()) == 0, "device status of the prefetch pass"
             vc = binding.g10_vitality(tbc, ws=wsc)
             torch.cuda.synchronize()
 
@@ -462,12 +468,12 @@ def run_ours(args):
             n_inst = int(em.counts[0].item())
             em_bytes = 17 * trc.N + 56 * n_mig + 32 * n_inst + 8 * (trc.K + 2)
             extras["config%d" % cfg] = {
-                "prefetch_pass": {"ms": a.elapsed_time(b), "moved": int(pf.summary[0].item()), "slots_regained": int(pf.summary[1].item()),
-                                  "note": "single call (it rewrites the pressure curve it is given)"},
+                "prefetch_pass": {"ms": float(np.median(pf_ms[1:])), "moved": int(pf.summary[0].item()), "slots_regained": int(pf.summary[1].item()),
+                                  "records": n_mig, "note": "median of 3 calls after one warm-up, L2 flushed, each on a fresh copy of the plan's pressure curve"},
                 "instruction_stream": {"ms": em_ms, "instructions": n_inst, "device_status": int(em.counts[1].item()),
                                        "roofline": roofline(em_bytes, em_ms / 1e3, hbm_peak, peak_kind),
                                        "note": "the binding allocates the record buffer inside the timed call"}}
-            del pf, em, vc, P
+            del pf, em, vc, P, pws
         # ---- batched re-planning of config 1: one variant per SM, kernel durations jittered by +-10 % (seeded), variant 0 unperturbed
         trc, tbc, wsc, planc, tlc, capc = kept[1]
         sms = torch.cuda.get_device_properties(dev).multi_processor_count

@@ -175,6 +175,7 @@ typedef struct g10_options {
 #define G10_WS_GEOMETRY 3
 #define G10_WS_EMIT 4
 #define G10_WS_BATCH 5
+#define G10_WS_PREFETCH 6
 
 /* Section 4.2, tensor vitality analysis.  Device-found errors land in counts[2]; with G10_DEV_BAD_KERNEL_PTR every
    tensor is reported unused (no uses, no periods), with G10_DEV_BAD_TENSOR_ID the offending entries are skipped. */
@@ -208,12 +209,18 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
    of bandwidth); a prefetch that moves is issued at the start of its first newly resident slot.
    All pointers are DEVICE pointers.  `pressure` [K] is the final pressure of the eviction plan on entry and the
    pressure after the pass on return; order [n] receives the visiting order; new_absent_last [n] and
-   new_prefetch_issue_ns [n] are indexed by plan record; summary [4] = prefetches moved, slots regained, new peak,
-   its lowest slot.  Needs no workspace; one block does the (strictly sequential) pass.
+   new_prefetch_issue_ns [n] are indexed by plan record; summary [5] = prefetches moved, slots regained, new peak,
+   its lowest slot, device status word (0, or G10_DEV_TIMEOUT when a wait between thread blocks ran out: the other
+   outputs are then not valid).
+   `ws` (optional; G10_WS_PREFETCH, with the number of migrations in place of E; contents are scratch): with it, a
+   timeline too long for one SM's shared memory (more than 15 360 slots, up to about 25 000 slots per SM of the GPU)
+   is cut into slices, one per thread block of a cooperative launch, and every block walks the records in visiting
+   order, waiting only for the records that can still reach its slice; the result is that of the sequential pass.
+   With ws == NULL (ws_bytes ignored) one block does the whole pass, record by record.
    Records of g10_plan_cyclic are accepted as they are: a slot beyond K stands for the same slot of the cycle (the
    pressure curve has K slots), a moved prefetch is issued at the unrolled time of its first regained slot, and the
-   visiting order is that of the prefetch's moment inside the iteration (its time modulo the iteration's length).
-   For an ordinary plan nothing changes. */
+   visiting order is that of the prefetch's moment inside the iteration (its time modulo the iteration's length);
+   records that wrap around are always visited by one block.  For an ordinary plan nothing changes. */
 typedef struct g10_prefetch_out {
     int64_t *pressure;
     int32_t *order;
@@ -223,7 +230,7 @@ typedef struct g10_prefetch_out {
 } g10_prefetch_out;
 int32_t g10_schedule_prefetch(int64_t num_kernels, int64_t num_migrations, const g10_migration *migrations,
                               const int64_t *kernel_start_ns, const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes,
-                              g10_prefetch_out *out, void *stream);
+                              g10_prefetch_out *out, void *ws, size_t ws_bytes, void *stream);
 
 /* Section 4.4, code instrumentation (the instrumented program of Figure 9): the g10_alloc / g10_free /
    g10_pre_evict / g10_prefetch calls to insert between the kernels.  Boundary b (0 <= b <= K) is the gap before

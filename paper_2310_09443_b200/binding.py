@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libg10.so")
 
 MEM_DEVICE, MEM_HOST = 0, 1
-WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT, WS_BATCH = 0, 1, 2, 3, 4, 5
+WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT, WS_BATCH, WS_PREFETCH = 0, 1, 2, 3, 4, 5, 6
 DEST_SSD, DEST_HOST = 0, 1
 FLAG_RESCORE_ALL = 1
 FLAG_GLOBAL_STATE = 2
@@ -122,7 +122,7 @@ def load_library():
                                                C.c_uint64, C.c_uint64, C.POINTER(_GeometryOut), C.c_void_p]
         lib.g10_schedule_prefetch.restype = C.c_int32
         lib.g10_schedule_prefetch.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
-                                              C.POINTER(_PrefetchOut), C.c_void_p]
+                                              C.POINTER(_PrefetchOut), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.g10_emit_instructions.restype = C.c_int32
         lib.g10_emit_instructions.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                               C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(_EmitOut), C.c_void_p, C.c_size_t,
@@ -389,19 +389,28 @@ def batch_migrations_numpy(batch, v) -> np.ndarray:
 
 
 def g10_schedule_prefetch(K, num_migrations, migrations, kernel_start_ns, tensor_bytes, gpu_capacity_bytes, pressure,
-                          stream=None):
+                          ws=None, one_block=False, stream=None):
     """Section 4.4 eager prefetch pass.  `migrations` is the uint8 record tensor of a finished plan, `pressure` its
-    final pressure (updated in place).  Device tensors only."""
+    final pressure (updated in place).  Device tensors only.  `ws`: a uint8 device tensor of at least
+    g10_workspace_bytes(WS_PREFETCH, K, 0, n) bytes (allocated here when None); one_block=True calls without a
+    workspace, which makes one thread block do the whole pass.  summary[4] is the device status word."""
     lib = load_library()
     dev = kernel_start_ns.device
     n = int(num_migrations)
     r = SimpleNamespace(pressure=pressure, order=torch.empty(max(n, 1), dtype=torch.int32, device=dev),
                         new_absent_last=torch.empty(max(n, 1), dtype=torch.int32, device=dev),
                         new_prefetch_issue_ns=torch.empty(max(n, 1), dtype=torch.int64, device=dev),
-                        summary=torch.empty(4, dtype=torch.int64, device=dev))
+                        summary=torch.empty(5, dtype=torch.int64, device=dev))
     out = _PrefetchOut(_ptr(r.pressure), _ptr(r.order), _ptr(r.new_absent_last), _ptr(r.new_prefetch_issue_ns), _ptr(r.summary))
+    ws_ptr, ws_bytes = None, 0
+    if not one_block:
+        need = g10_workspace_bytes(WS_PREFETCH, K, 0, n)
+        if ws is None:
+            ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        ws_ptr, ws_bytes = _ptr(ws), ws.numel()
+        r.ws = ws
     _check(lib.g10_schedule_prefetch(K, n, _ptr(migrations), _ptr(kernel_start_ns), _ptr(tensor_bytes), gpu_capacity_bytes,
-                                     C.byref(out), _stream(stream)))
+                                     C.byref(out), ws_ptr, ws_bytes, _stream(stream)))
     return r
 
 

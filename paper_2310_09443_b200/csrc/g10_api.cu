@@ -219,6 +219,24 @@ size_t carve_emit(void *base, int64_t N, int64_t n, EmitLaunch &L, char **zero_b
     return align_up(c.off);
 }
 
+// Scratch of the eager prefetch pass (many-block form): what must start at zero first.
+size_t carve_prefetch(void *base, int64_t n, PrefetchScratch &p, size_t *zero_bytes)
+{
+    Carver c(base);
+    p.status = c.take<ull>(1);
+    p.ticket = c.take<unsigned>(1);
+    p.fallback = c.take<unsigned>(1);
+    p.word = c.take<unsigned>((size_t)n);
+    p.rank = c.take<unsigned>((size_t)n);
+    *zero_bytes = align_up(c.off);
+    p.first = c.take<int32_t>((size_t)n);
+    p.last = c.take<int32_t>((size_t)n);
+    p.size = c.take<int64_t>((size_t)n);
+    p.block_max = c.take<int64_t>(kPfMaxBlocks);
+    p.block_slot = c.take<int32_t>(kPfMaxBlocks);
+    return align_up(c.off);
+}
+
 }  // namespace
 }  // namespace g10
 
@@ -245,7 +263,7 @@ const char *g10_strerror(int32_t code)
 int32_t g10_workspace_bytes(int32_t which, int64_t K, int64_t N, int64_t E, int32_t mem, size_t *out_bytes)
 {
     if (!out_bytes || K < 0 || N < 0 || E < 0) return G10_ERR_ARG;
-    if (which < G10_WS_VITALITY || which > G10_WS_BATCH) return G10_ERR_ARG;
+    if (which < G10_WS_VITALITY || which > G10_WS_PREFETCH) return G10_ERR_ARG;
     if (mem != G10_MEM_DEVICE && mem != G10_MEM_HOST) return G10_ERR_ARG;
     const int64_t lim = ((int64_t)1 << 31) - 1;
     if (K >= lim || N >= lim || E >= lim) return G10_ERR_LIMIT;
@@ -255,6 +273,12 @@ int32_t g10_workspace_bytes(int32_t which, int64_t K, int64_t N, int64_t E, int3
         char *zb = nullptr;
         size_t zbytes = 0;
         *out_bytes = carve_emit(nullptr, N, E, L, &zb, &zbytes);
+        return G10_OK;
+    }
+    if (which == G10_WS_PREFETCH) {                // E stands for the number of migrations here
+        PrefetchScratch p;
+        size_t zbytes = 0;
+        *out_bytes = carve_prefetch(nullptr, E, p, &zbytes);
         return G10_OK;
     }
     Workspace w;
@@ -408,15 +432,26 @@ int32_t g10_characterize(int64_t K, int64_t N, const int64_t *use_ptr, const int
 }
 
 int32_t g10_schedule_prefetch(int64_t K, int64_t n, const g10_migration *migrations, const int64_t *kernel_start_ns,
-                              const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes, g10_prefetch_out *out, void *stream)
+                              const int64_t *tensor_bytes, uint64_t gpu_capacity_bytes, g10_prefetch_out *out, void *ws, size_t ws_bytes,
+                              void *stream)
 {
     if (K < 0 || n < 0 || !out || !out->summary) return G10_ERR_ARG;
     if (K >= (((int64_t)1 << 31) - 1) || n >= (((int64_t)1 << 31) - 1)) return G10_ERR_LIMIT;
     if (K > 0 && !out->pressure) return G10_ERR_ARG;
     if (n > 0 && (!migrations || !kernel_start_ns || !tensor_bytes || !out->order || !out->new_absent_last || !out->new_prefetch_issue_ns))
         return G10_ERR_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    PrefetchScratch p{};
+    if (ws) {                                      // (without a workspace one block does the pass)
+        if (((uintptr_t)ws & (kAlign - 1)) != 0) return G10_ERR_WORKSPACE;
+        PrefetchScratch probe;
+        size_t zbytes = 0;
+        if (carve_prefetch(nullptr, n, probe, &zbytes) > ws_bytes) return G10_ERR_WORKSPACE;
+        carve_prefetch(ws, n, p, &zbytes);
+        CU(cudaMemsetAsync(ws, 0, zbytes, s));
+    }
     CU(launch_schedule_prefetch(K, n, migrations, kernel_start_ns, tensor_bytes, gpu_capacity_bytes, out->pressure, out->order,
-                                out->new_absent_last, out->new_prefetch_issue_ns, out->summary, (cudaStream_t)stream));
+                                out->new_absent_last, out->new_prefetch_issue_ns, out->summary, p, s));
     return G10_OK;
 }
 

@@ -191,9 +191,22 @@ cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, 
 cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *pair, int64_t *point, int64_t *pressure,
                                   int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);
 // eager prefetch pass (g10_prefetch.cu)
+constexpr int kPfMaxBlocks = 2048;         // most blocks the many-block form of the pass may use (one slice of the timeline each)
+// Scratch of the many-block form, carved from the caller's workspace (all null: the call came without one).
+struct PrefetchScratch {
+    ull *status;              // device status word                                      }
+    unsigned *ticket;         // blocks that have finished                               } cleared before the launch
+    unsigned *fallback;       // set when the records need the one-block form after all  }
+    unsigned *word;           // [n] where each record's search stands                   }
+    unsigned *rank;           // [n] position of each record in the visiting order       }
+    int32_t *first, *last;    // [n] absent_first / absent_last in visiting order
+    int64_t *size;            // [n] tensor size in visiting order
+    int64_t *block_max;       // [kPfMaxBlocks] largest pressure of each block's slice ...
+    int32_t *block_slot;      // [kPfMaxBlocks] ... and its lowest slot
+};
 cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *mig, const int64_t *start, const int64_t *bytes,
                                      uint64_t gpu_capacity_bytes, int64_t *P, int32_t *order, int32_t *new_last, int64_t *new_issue,
-                                     int64_t *summary, cudaStream_t s);
+                                     int64_t *summary, const PrefetchScratch &scratch, cudaStream_t s);
 // instruction-stream emission (g10_emit.cu)
 struct EmitLaunch {
     int64_t K, N, n;

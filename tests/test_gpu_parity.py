@@ -386,9 +386,9 @@ def test_full_size_stress_plan_digest(gpu):
     n = int(summary[0])
     pf = gpu.g10_schedule_prefetch(tr.K, n, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap, plan.final_pressure)
     torch.cuda.synchronize()
-    assert _np(pf.summary).tolist() == gold["prefetch_summary"]
+    assert _np(pf.summary)[:4].tolist() == gold["prefetch_summary"] and int(_np(pf.summary)[4]) == 0
     hp = hashlib.sha256()
-    for a in (_np(pf.order)[:n], _np(pf.new_absent_last)[:n], _np(pf.new_prefetch_issue_ns)[:n], _np(pf.pressure)[:tr.K], _np(pf.summary)):
+    for a in (_np(pf.order)[:n], _np(pf.new_absent_last)[:n], _np(pf.new_prefetch_issue_ns)[:n], _np(pf.pressure)[:tr.K], _np(pf.summary)[:4]):
         hp.update(np.ascontiguousarray(a).tobytes())
     assert hp.hexdigest() == gold["prefetch_sha256"]
     # the instruction stream of that plan with the eager prefetch times (8 M records), field by field
@@ -413,17 +413,20 @@ def check_prefetch(gpu, oracle, tr, cap):
     plan = gpu.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw)
     torch.cuda.synchronize()
     n = int(plan.summary[0].item())
+    P1 = plan.final_pressure.clone()
     pf = gpu.g10_schedule_prefetch(tr.K, n, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap, plan.final_pressure)
+    pf1 = gpu.g10_schedule_prefetch(tr.K, n, plan.migrations, tl.kernel_start_ns, tb.tensor_bytes, cap, P1, one_block=True)
     torch.cuda.synchronize()
     start = oracle.slot_clock(tr.kernel_ns)
     ref = oracle.plan(tr, cap, lazy=True)
     opf = oracle.schedule_prefetch(tr.K, ref.migrations, start, tr.tensor_bytes, cap, ref.final_pressure)
     assert n == len(ref.migrations)
-    assert np.array_equal(_np(pf.order)[:n], opf.order)
-    assert np.array_equal(_np(pf.new_absent_last)[:n], opf.new_absent_last)
-    assert np.array_equal(_np(pf.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
-    assert np.array_equal(_np(pf.pressure)[:tr.K], opf.pressure)
-    assert np.array_equal(_np(pf.summary), opf.summary)
+    for got in (pf, pf1):                         # with a workspace (many blocks on a long timeline) and without (one block)
+        assert np.array_equal(_np(got.order)[:n], opf.order)
+        assert np.array_equal(_np(got.new_absent_last)[:n], opf.new_absent_last)
+        assert np.array_equal(_np(got.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
+        assert np.array_equal(_np(got.pressure)[:tr.K], opf.pressure)
+        assert np.array_equal(_np(got.summary)[:4], opf.summary) and int(_np(got.summary)[4]) == 0
     return opf
 
 
@@ -647,7 +650,7 @@ def check_cyclic(gpu, oracle, tr, cap, host_capacity=0, max_iterations=0):
             opf = oracle.schedule_prefetch(tr.K, ref.migrations, start, tr.tensor_bytes, cap2, ref.final_pressure)
             assert np.array_equal(_np(pf.order)[:n], opf.order) and np.array_equal(_np(pf.new_absent_last)[:n], opf.new_absent_last)
             assert np.array_equal(_np(pf.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
-            assert np.array_equal(_np(P)[:tr.K], opf.pressure) and np.array_equal(_np(pf.summary), opf.summary)
+            assert np.array_equal(_np(P)[:tr.K], opf.pressure) and np.array_equal(_np(pf.summary)[:4], opf.summary) and int(_np(pf.summary)[4]) == 0
             oe = oracle.emit_instructions(tr.K, ov.first_use, ov.last_use, tr.tensor_bytes, tr.tensor_global, start, ref.migrations,
                                           opf.new_prefetch_issue_ns)
             assert int(em.counts[1].item()) == 0 and int(em.counts[0].item()) == len(oe.instructions)
@@ -659,40 +662,83 @@ def check_cyclic(gpu, oracle, tr, cap, host_capacity=0, max_iterations=0):
 
 
 @pytest.mark.gpu
+def synthetic_prefetch_records(gpu, rng, K, n, wrap, long_share=0.3):
+    """Seeded records over a random pressure curve: absent ranges that are short or (a share of them) as long as most of
+    the timeline, capacity such that about one slot in sixteen cannot take a mid-sized tensor."""
+    dur = rng.integers(1, 1000, size=K).astype(np.int64)
+    start = np.concatenate([[0], np.cumsum(dur)]).astype(np.int64)
+    T = int(start[K])
+    N = 64
+    nbytes = rng.integers(1, 1 << 20, size=N).astype(np.int64)
+    P = rng.integers(0, 1 << 22, size=K).astype(np.int64)
+    mig = np.zeros(n, dtype=gpu.MIGRATION_DTYPE)
+    a = rng.integers(0, K, size=n)
+    length = np.where(rng.random(n) < long_share, rng.integers(1, K - 1, size=n), rng.integers(1, 64, size=n))
+    b = np.minimum(a + length - 1, a + K - 2)
+    if not wrap:
+        b = np.minimum(b, K - 1)
+    mig["absent_first"], mig["absent_last"] = a, b
+    mig["tensor"] = rng.integers(0, N, size=n)
+    issue = np.where(b + 1 <= K, start[np.minimum(b + 1, K)], start[(b + 1) % K] + T) - rng.integers(0, 2, size=n)
+    mig["prefetch_issue_ns"] = issue
+    mig["period"] = np.arange(n)
+    return mig, start, nbytes, P
+
+
+def check_prefetch_records(gpu, oracle, K, mig, start, nbytes, cap, P, **kw):
+    import torch
+    n = len(mig)
+    dm = torch.from_numpy(mig.view(np.uint8).copy()).cuda()
+    dP = torch.from_numpy(P.copy()).cuda()
+    pf = gpu.g10_schedule_prefetch(K, n, dm, torch.from_numpy(start).cuda(), torch.from_numpy(nbytes).cuda(), cap, dP, **kw)
+    torch.cuda.synchronize()
+    opf = oracle.schedule_prefetch(K, mig, start, nbytes, cap, P)
+    assert np.array_equal(_np(pf.order)[:n], opf.order)
+    assert np.array_equal(_np(pf.new_absent_last)[:n], opf.new_absent_last)
+    assert np.array_equal(_np(pf.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
+    assert np.array_equal(_np(dP), opf.pressure)
+    assert np.array_equal(_np(pf.summary)[:4], opf.summary) and int(_np(pf.summary)[4]) == 0
+    return opf
+
+
+@pytest.mark.gpu
 def test_prefetch_pass_on_wrapping_records(gpu, oracle):
     """The eager prefetch pass on synthetic records whose absent ranges reach into the next iteration, for every kernel the
     call can choose: pressure curve in shared memory (K = 5000), per-tile bounds in shared memory (K = 40 000, several
-    tiles and a ragged last one)."""
-    import torch
+    tiles and a ragged last one) -- called without a workspace, and with one (the many-block form then hands such
+    records to the one-block form behind it)."""
     rng = np.random.default_rng(60221023)
     for K, n in ((5000, 400), (40000, 1500), (40000, 6000)):
-        dur = rng.integers(1, 1000, size=K).astype(np.int64)
-        start = np.concatenate([[0], np.cumsum(dur)]).astype(np.int64)
-        T = int(start[K])
-        N = 64
-        nbytes = rng.integers(1, 1 << 20, size=N).astype(np.int64)
-        P = rng.integers(0, 1 << 22, size=K).astype(np.int64)
-        cap = int(1 << 22)
-        mig = np.zeros(n, dtype=gpu.MIGRATION_DTYPE)
-        a = rng.integers(0, K, size=n)
-        length = np.where(rng.random(n) < 0.3, rng.integers(1, K - 1, size=n), rng.integers(1, 64, size=n))
-        b = np.minimum(a + length - 1, a + K - 2)
-        mig["absent_first"], mig["absent_last"] = a, b
-        mig["tensor"] = rng.integers(0, N, size=n)
-        issue = np.where(b + 1 <= K, start[np.minimum(b + 1, K)], start[(b + 1) % K] + T) - rng.integers(0, 2, size=n)
-        mig["prefetch_issue_ns"] = issue
-        mig["period"] = np.arange(n)
-        assert (b >= K).sum() > 20
-        dm = torch.from_numpy(mig.view(np.uint8).copy()).cuda()
-        dP = torch.from_numpy(P.copy()).cuda()
-        pf = gpu.g10_schedule_prefetch(K, n, dm, torch.from_numpy(start).cuda(), torch.from_numpy(nbytes).cuda(), cap, dP)
-        torch.cuda.synchronize()
-        opf = oracle.schedule_prefetch(K, mig, start, nbytes, cap, P)
-        assert np.array_equal(_np(pf.order)[:n], opf.order)
-        assert np.array_equal(_np(pf.new_absent_last)[:n], opf.new_absent_last)
-        assert np.array_equal(_np(pf.new_prefetch_issue_ns)[:n], opf.new_prefetch_issue_ns)
-        assert np.array_equal(_np(dP), opf.pressure) and np.array_equal(_np(pf.summary), opf.summary)
+        mig, start, nbytes, P = synthetic_prefetch_records(gpu, rng, K, n, wrap=True)
+        assert (mig["absent_last"] >= K).sum() > 20
+        for one_block in (True, False):
+            opf = check_prefetch_records(gpu, oracle, K, mig, start, nbytes, int(1 << 22), P, one_block=one_block)
         assert int(opf.summary[0]) > n // 10
+
+
+@pytest.mark.gpu
+def test_prefetch_pass_in_slices(gpu, oracle):
+    """The many-block form of the eager prefetch pass (timeline cut into one slice per thread block) on synthetic records
+    that do not wrap: short and very long absent ranges mixed, so that searches start everywhere at once, run through many
+    slices and wait for one another; slice counts from a handful to every block the GPU holds, ragged last slice; a curve
+    where nothing blocks (every search runs to absent_first) and one where everything does; empty ranges."""
+    rng = np.random.default_rng(2310094431)
+    for K, n, long_share in ((15361, 300, 0.3), (40000, 6000, 0.3), (151552 + 77, 9000, 0.1), (400003, 12000, 0.02), (1200007, 5000, 0.01)):
+        mig, start, nbytes, P = synthetic_prefetch_records(gpu, rng, K, n, wrap=False, long_share=long_share)
+        opf = check_prefetch_records(gpu, oracle, K, mig, start, nbytes, int(1 << 22), P)
+        assert int(opf.summary[0]) > n // 10
+    K, n = 60000, 3000
+    mig, start, nbytes, P = synthetic_prefetch_records(gpu, rng, K, n, wrap=False, long_share=0.5)
+    check_prefetch_records(gpu, oracle, K, mig, start, nbytes, int(1 << 62), P)          # nothing ever blocks
+    check_prefetch_records(gpu, oracle, K, mig, start, nbytes, 0, P)                     # every slot blocks: nothing moves
+    mig2 = mig.copy()
+    empty = rng.random(n) < 0.2
+    mig2["absent_first"] = np.where(empty, mig2["absent_last"] + 1, mig2["absent_first"])   # ranges without a slot
+    check_prefetch_records(gpu, oracle, K, mig2, start, nbytes, int(1 << 22), P)
+    # equal prefetch times: the visiting order falls back to the record index
+    mig3 = mig.copy()
+    mig3["prefetch_issue_ns"] = (mig3["prefetch_issue_ns"] // 100000) * 100000
+    check_prefetch_records(gpu, oracle, K, mig3, start, nbytes, int(1 << 22), P)
 
 
 @pytest.mark.gpu

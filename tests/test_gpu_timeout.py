@@ -72,3 +72,63 @@ def test_a_wait_that_runs_out_returns_with_the_timeout_bit(oracle):
     plan = binding.g10_plan_migrations(tb, cap, tr.host_bw, tr.ssd_bw, flags=FLAG_RESCORE_ALL)
     torch.cuda.synchronize()
     assert int(plan.summary[7].item()) == 0 and np.array_equal(binding.migrations_numpy(plan), ref.migrations)
+
+
+def test_a_prefetch_hand_over_that_never_comes(oracle):
+    """The many-block form of the eager prefetch pass: blocks wait for records handed over by the block on their right.  In
+    the test build one block (named by an environment variable that only that build reads) keeps its records to itself
+    and waits last a millisecond: the blocks that wait for it give up, the others stop as soon as they see the status
+    word, summary[4] carries G10_DEV_TIMEOUT, and the same call without the injection matches the oracle."""
+    import os
+    import torch
+    from paper_2310_09443_b200 import binding, build
+    from test_gpu_parity import synthetic_prefetch_records
+    build.build()
+    binding.load_library()
+    hooks = C.CDLL(build.build(hooks=True))
+    hooks.g10_schedule_prefetch.restype = C.c_int32
+    hooks.g10_schedule_prefetch.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
+                                            C.POINTER(binding._PrefetchOut), C.c_void_p, C.c_size_t, C.c_void_p]
+    rng = np.random.default_rng(77)
+    K, n, cap = 40000, 6000, 1 << 22
+    mig, start, nbytes, P = synthetic_prefetch_records(binding, rng, K, n, wrap=False)
+    ref = oracle.schedule_prefetch(K, mig, start, nbytes, cap, P)
+    dm = torch.from_numpy(mig.view(np.uint8).copy()).cuda()
+    dstart, dbytes = torch.from_numpy(start).cuda(), torch.from_numpy(nbytes).cuda()
+    ws = torch.zeros(binding.g10_workspace_bytes(binding.WS_PREFETCH, K, 0, n), dtype=torch.uint8, device="cuda")
+    order = torch.zeros(n, dtype=torch.int32, device="cuda")
+    new_last = torch.zeros(n, dtype=torch.int32, device="cuda")
+    new_issue = torch.zeros(n, dtype=torch.int64, device="cuda")
+    summary = torch.zeros(5, dtype=torch.int64, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        dP = torch.from_numpy(P.copy()).cuda()
+        out = binding._PrefetchOut(dP.data_ptr(), order.data_ptr(), new_last.data_ptr(), new_issue.data_ptr(), summary.data_ptr())
+        t0 = time.perf_counter()
+        rc = hooks.g10_schedule_prefetch(K, n, dm.data_ptr(), dstart.data_ptr(), dbytes.data_ptr(), cap, C.byref(out), ws.data_ptr(),
+                                         ws.numel(), stream)
+        torch.cuda.synchronize()
+        return rc, time.perf_counter() - t0, dP
+
+    def check_against_oracle(dP):
+        s = summary.cpu().numpy()
+        assert s[4] == 0 and np.array_equal(s[:4], ref.summary)
+        assert np.array_equal(order.cpu().numpy(), ref.order) and np.array_equal(new_last.cpu().numpy(), ref.new_absent_last)
+        assert np.array_equal(new_issue.cpu().numpy(), ref.new_prefetch_issue_ns) and np.array_equal(dP.cpu().numpy(), ref.pressure)
+
+    os.environ.pop("G10_TEST_PREFETCH_MUTE_BLOCK", None)
+    rc, _, dP = call()
+    assert rc == 0
+    check_against_oracle(dP)
+    os.environ["G10_TEST_PREFETCH_MUTE_BLOCK"] = "100"
+    try:
+        rc, dt, dP = call()
+    finally:
+        os.environ.pop("G10_TEST_PREFETCH_MUTE_BLOCK", None)
+    assert rc == 0
+    assert int(summary[4].item()) & DEV_TIMEOUT, "summary[4] must carry G10_DEV_TIMEOUT"
+    assert dt < 1.0, "the call must come back within milliseconds (%.3f s)" % dt
+    rc, _, dP = call()
+    assert rc == 0
+    check_against_oracle(dP)

@@ -81,7 +81,8 @@ def test_argument_errors_of_the_later_entry_points(lib):
     assert lib.g10_plan_batch(C.byref(tr_dev), 1, var, 0, C.byref(bo), None, 0, None) == -3
     # prefetch pass and instruction stream
     pf = binding._PrefetchOut()
-    assert lib.g10_schedule_prefetch(1, 1, None, None, None, 1, C.byref(pf), None) == -1
+    assert lib.g10_schedule_prefetch(1, 1, None, None, None, 1, C.byref(pf), None, 0, None) == -1
+    assert binding.g10_workspace_bytes(binding.WS_PREFETCH, 1000000, 0, 13505) < (1 << 20)        # a few words per record
     eo = binding._EmitOut()
     assert lib.g10_emit_instructions(1, 1, None, None, None, None, None, 0, None, None, C.byref(eo), None, 0, None) == -1
     # the workspace of the batch call is the planner's
