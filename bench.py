@@ -7,7 +7,7 @@ and pressure timeline, i.e. one g10_vitality call plus one g10_pressure_timeline
 for an HBM fraction to mean something.  A step is one such pass with the trace resident in HBM; the L2 is flushed
 between steps.  Second headline (`plan_ms`): one whole g10_plan_migrations call (S1-S7) on the ResNet-152-shaped
 trace (config 1).  The same line carries the plan of every configuration (`plans`), the two analysis calls on a
-trace eight times the size (`scale_x8`), the calls behind the plan (prefetch pass, instruction stream, batched and
+trace four and eight times the size (`scale`), the calls behind the plan (prefetch pass, instruction stream, batched and
 cyclic planning), the roofline of the passes and the CPU oracle timed beside them.  Prints ONE JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick | --passes-only]
@@ -42,17 +42,20 @@ L2_FLUSH_BYTES = 512 << 20
 # "sources_sha256" is the hash of the kernel sources at the time of the capture: when the sources have changed since, the
 # bench line says so ("traffic_stale") instead of passing old traffic off as current, and a CPU test warns.
 TRAFFIC = {"vitality": 242_500_000, "timeline": 110_000_000, "captured_at": "2026-11-25",
-           "sources_sha256": "277666adb10f5bf245a5b4acd77d73e540cdfbe8fd3a12fc8bbb6aa9fa3787c1"}
+           "sources_sha256": "ac29ffd5ce9d5251e4fb839bdb2b35f20f5d1142fd9b8062e57e75a4201d05e4"}
+
+
+PASS_SOURCES = ("g10_passes.cu", "g10_vitality_buckets.cu")     # the kernels of g10_vitality and g10_pressure_timeline
 
 
 def kernel_sources_sha256():
+    """Hash of the sources that hold the kernels of the two analysis calls (what the stored traffic was measured on)."""
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2310_09443_b200", "csrc")
-    for f in sorted(os.listdir(d)):
-        if f.endswith((".cu", ".cuh", ".h")):
-            h.update(f.encode())
-            h.update(open(os.path.join(d, f), "rb").read())
+    for f in PASS_SOURCES:
+        h.update(f.encode())
+        h.update(open(os.path.join(d, f), "rb").read())
     return h.hexdigest()
 
 
