@@ -116,6 +116,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w, int32_t which)
     w.c_ben_hi = c.take<ull>(plan ? E : 1);
     w.c_cost = c.take<ull>(plan ? E : 1);
     w.c_key = c.take<double>(plan ? E : 1);
+    w.c_rng = c.take<int2>(plan ? E : 1);
     w.worklist = c.take<int>(plan ? 2 * E : 1);
     w.bk_pairs = c.take<ull>(vit ? E : 1);
     if (plan && z.K <= kSmallMaxSlots) {

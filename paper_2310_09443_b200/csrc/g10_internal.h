@@ -128,6 +128,7 @@ struct Workspace {
     unsigned char *c_state;      // [E] per-period state of the lazy planner
     ull *c_ben_lo, *c_ben_hi, *c_cost;   // [E] cached benefit and cost
     double *c_key;               // [E] rounded benefit / cost
+    int2 *c_rng;                 // [E] absent range of the current destination
     int *worklist;               // [2*E]
     ull *bk_pairs;               // [E] events as (tensor in bucket, kernel) keys, bucket after bucket
     int64_t *busy_rep, *hocc_rep; // per-block copies of the channel bookings / host occupancy (small-trace planner)

@@ -26,6 +26,8 @@ struct LazyArgs {
     ull *c_ben_lo, *c_ben_hi;   // last computed benefit
     ull *c_cost;                // 2 t of the current destination
     double *c_key;              // rounded benefit / cost of the cached score (steers the search; decisions are exact)
+    int2 *c_rng;                // absent range [a', b'] of the current destination (a copy of the geometry, so that the
+                                // pass over the periods has it in one load, with no look-up by destination)
     int *worklist;              // [2][stride] DIRTY periods of the current round
     unsigned *wl_count;         // [2]
     LazyProp *props;            // [2][kLazyMaxBlocks] each block's best FRESH candidate and best STALE bounds
@@ -72,8 +74,9 @@ __device__ __forceinline__ u128 benefit_tile_warp(const PlanArgs &A, int k_lo, i
     return acc;
 }
 
-__device__ __forceinline__ void store_score(const LazyArgs &L, int64_t p, int dest, int state, u128 ben, ull cost)
+__device__ __forceinline__ void store_score(const PlanArgs &A, const LazyArgs &L, int64_t p, int dest, int state, u128 ben, ull cost)
 {
+    L.c_rng[p] = make_int2(A.geo_a[dest * A.geo_stride + p], A.geo_b[dest * A.geo_stride + p]);
     L.c_ben_lo[p] = (ull)ben;
     L.c_ben_hi[p] = (ull)(ben >> 64);
     L.c_cost[p] = cost;
@@ -91,14 +94,14 @@ __device__ __forceinline__ void eval_warp(const PlanArgs &A, const LazyArgs &L, 
     if ((st >> 2) == kDirty) {
         Cand cd;
         if (!score_period(A, p, lane, &cd)) { if (lane == 0) L.c_state[p] = 0; return; }
-        if (lane == 0) store_score(L, p, cd.dest, kFresh, cd.ben, cd.cost);
+        if (lane == 0) store_score(A, L, p, cd.dest, kFresh, cd.ben, cd.cost);
         return;
     }
     const int d = (st & 3) - 1;
     const int ap = A.geo_a[d * A.geo_stride + p], bp = A.geo_b[d * A.geo_stride + p];
     const int64_t s = A.bytes[A.per_t[p]];
     u128 acc = warp_sum_u128(benefit_partial(A, ap, bp, s, lane, 32));
-    if (lane == 0) store_score(L, p, d, kFresh, acc, 2ull * (ull)A.geo_t[d * A.geo_stride + p]);
+    if (lane == 0) store_score(A, L, p, d, kFresh, acc, 2ull * (ull)A.geo_t[d * A.geo_stride + p]);
 }
 
 // One warp re-chooses the destination of DIRTY period p (SSD first, then host).  The period is erased if no
@@ -131,6 +134,7 @@ __device__ __forceinline__ void dest_warp(const PlanArgs &A, const LazyArgs &L, 
         if (dest < 0) L.c_state[p] = 0;
         else {
             L.c_ben_lo[p] = 0; L.c_ben_hi[p] = 0; L.c_cost[p] = 2ull * (ull)t;
+            L.c_rng[p] = make_int2(A.geo_a[dest * A.geo_stride + p], A.geo_b[dest * A.geo_stride + p]);
             L.c_key[p] = __longlong_as_double(0x7ff0000000000000ll);      // +infinity: rescored before anything is decided
             L.c_state[p] = (unsigned char)((dest + 1) | (kStale << 2));
         }
@@ -345,11 +349,15 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
       unsigned char st_q[kAhead];
       double key_q[kAhead];
       int u_q[kAhead], v_q[kAhead];
+      int2 rng_q[kAhead];
 #pragma unroll
       for (int q = 0; q < kAhead; ++q) {
           const int64_t pq = p00 + q * step + threadIdx.x;
-          st_q[q] = 0; key_q[q] = 0.0; u_q[q] = 0; v_q[q] = 0;
-          if (pq < Pn) { st_q[q] = L.c_state[pq]; key_q[q] = L.c_key[pq]; if (classify) { u_q[q] = A.per_u[pq]; v_q[q] = A.per_v[pq]; } }
+          st_q[q] = 0; key_q[q] = 0.0; u_q[q] = 0; v_q[q] = 0; rng_q[q] = make_int2(0, -1);
+          if (pq < Pn) {
+              st_q[q] = L.c_state[pq]; key_q[q] = L.c_key[pq];
+              if (classify) { u_q[q] = A.per_u[pq]; v_q[q] = A.per_v[pq]; rng_q[q] = L.c_rng[pq]; }     // (the range: rubbish while the period is DIRTY, not used then)
+          }
       }
 #pragma unroll
       for (int q = 0; q < kAhead; ++q) {
@@ -368,7 +376,7 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
                     if (p == w.idx) { L.c_state[p] = 0; st = 0; }
                     else if (state != kDirty) {
                         if (u + 1 <= w.b && w.a <= v - 1) {          // the two periods share slots
-                            const int ap = A.geo_a[d * A.geo_stride + p], bp = A.geo_b[d * A.geo_stride + p];
+                            const int ap = rng_q[q].x, bp = rng_q[q].y;
                             bool hit = false;
                             if (d == w.dest) {
                                 const bool meet_out = u + 1 <= w.ap - 1 && w.a <= ap - 1, meet_in = bp + 1 <= w.b && w.bp + 1 <= v - 1;
@@ -782,7 +790,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
                 Cand x;
                 x.ben = tot; x.cost = s_it_cost[r]; x.idx = tot == 0 ? -1 : p; x.dest = d;
                 s_new[r] = x;
-                if ((int)((p / kPlanThreads) % G) == c) store_score(L, p, d, kFresh, tot, x.cost);
+                if ((int)((p / kPlanThreads) % G) == c) store_score(A, L, p, d, kFresh, tot, x.cost);
             }
             __syncthreads();
             {
@@ -832,7 +840,7 @@ cudaError_t launch_plan_lazy(const PlanArgs &A_in, const Workspace &w, int G, cu
     PlanArgs A = A_in;
     LazyArgs L;
     L.c_state = w.c_state; L.c_ben_lo = w.c_ben_lo; L.c_ben_hi = w.c_ben_hi; L.c_cost = w.c_cost; L.c_key = w.c_key;
-    L.worklist = w.worklist; L.wl_count = w.wl_count; L.props = w.lazy_props; L.partials = w.lazy_partials; L.stride = A.geo_stride;
+    L.c_rng = w.c_rng; L.worklist = w.worklist; L.wl_count = w.wl_count; L.props = w.lazy_props; L.partials = w.lazy_partials; L.stride = A.geo_stride;
     L.tmin = w.lazy_tmin; L.tmax = w.lazy_tmax;
     void *args[] = {&A, &L};
     return cudaLaunchCooperativeKernel((const void *)k_plan_lazy, dim3(G), dim3(kPlanThreads), args, 0, s);
