@@ -59,7 +59,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w, int32_t which)
     carve_scan(c, w.count_scan, vit ? ntiles : 1, 1);
     carve_scan(c, w.emit_scan, vit ? etiles : 1, 2);
     carve_scan(c, w.pressure_scan, ktiles, 1);
-    w.wl_count = c.take<unsigned>(2);
+    w.wl_count = c.take<unsigned>(4);           // (two list lengths, two overflow flags)
     w.one_done = c.take<unsigned>(1);
     w.event_budget = c.take<ull>(1);
     w.bk_count = c.take<unsigned>(vit ? 4096 : 1);

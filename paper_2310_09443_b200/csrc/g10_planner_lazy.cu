@@ -20,6 +20,7 @@ namespace g10 {
 
 enum { kFresh = 1, kStale = 2, kDirty = 3 };
 constexpr int kMixCap = 1024;            // tiles of one round that a block reads slot by slot, listed
+constexpr int kLocalDirty = 128;         // DIRTY periods a block re-examines itself right after its pass
 
 struct LazyArgs {
     unsigned char *c_state;     // 0 = erased; else (dest + 1) | (state << 2)
@@ -29,7 +30,7 @@ struct LazyArgs {
     int2 *c_rng;                // absent range [a', b'] of the current destination (a copy of the geometry, so that the
                                 // pass over the periods has it in one load, with no look-up by destination)
     int *worklist;              // [2][stride] DIRTY periods of the current round
-    unsigned *wl_count;         // [2]
+    unsigned *wl_count;         // [2] lengths of the two work lists; [2..3]: a block could not take its DIRTY periods itself
     LazyProp *props;            // [2][kLazyMaxBlocks] each block's best FRESH candidate and best STALE bounds
     ull *partials;              // [3][kRoundM][2] 128-bit sums of the benefits rescored together (three buffers in turn)
     int64_t *tmin, *tmax;       // [tiles of kSlotTile slots] smallest / largest pressure of each tile
@@ -106,7 +107,29 @@ __device__ __forceinline__ void eval_warp(const PlanArgs &A, const LazyArgs &L, 
 
 // One warp re-chooses the destination of DIRTY period p (SSD first, then host).  The period is erased if no
 // destination is left; otherwise it becomes STALE with an unbounded score, so that it is rescored with the others.
-__device__ __forceinline__ void dest_warp(const PlanArgs &A, const LazyArgs &L, int64_t p, int lane)
+// pend (optional): a commit whose channel bookings are not in A.busy yet; its share of every slot is added on the fly
+// (the same amounts book_winner adds later), so that the answer is the one the booked arrays will give.
+struct Winner;
+__device__ __forceinline__ bool window_free_pending(const PlanArgs &A, const int64_t *busy, int64_t w0, int64_t w1, int k0, int k1, int lane,
+                                                    int vk0, int vk1, int64_t v0, int64_t v1)
+{
+    bool ok = true;
+    for (int k = k0 + lane; k <= k1; k += 32) {
+        const int64_t s0 = A.start[k], s1 = A.start[k + 1];
+        const int64_t lo = w0 > s0 ? w0 : s0, hi = w1 < s1 ? w1 : s1;
+        const int64_t ov = hi > lo ? hi - lo : 0;
+        int64_t extra = 0;
+        if (k >= vk0 && k <= vk1) {
+            const int64_t vl = v0 > s0 ? v0 : s0, vh = v1 < s1 ? v1 : s1;
+            extra = vh > vl ? vh - vl : 0;
+        }
+        if (busy[k] + extra + ov > s1 - s0) ok = false;
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void dest_warp(const PlanArgs &A, const LazyArgs &L, int64_t p, int lane, int pend_dest = -1, int pa = 0, int pap = 0,
+                                          int pbp = 0, int pb = 0, int64_t pt = 0, int64_t pt_r = 0, int64_t pt_end = 0)
 {
     if (L.c_state[p] == 0) return;
     const int u = A.per_u[p], v = A.per_v[p];
@@ -120,8 +143,13 @@ __device__ __forceinline__ void dest_warp(const PlanArgs &A, const LazyArgs &L, 
         if (ap < 0) continue;
         const int bp = A.geo_b[X * A.geo_stride + p];
         t = A.geo_t[X * A.geo_stride + p];
-        if (!window_free(A, A.busy + (size_t)(2 * X) * A.K, t_r, t_r + t, a, ap - 1, lane)) continue;
-        if (!window_free(A, A.busy + (size_t)(2 * X + 1) * A.K, t_end - t, t_end, bp + 1, b, lane)) continue;
+        if (X == pend_dest) {
+            if (!window_free_pending(A, A.busy + (size_t)(2 * X) * A.K, t_r, t_r + t, a, ap - 1, lane, pa, pap - 1, pt_r, pt_r + pt)) continue;
+            if (!window_free_pending(A, A.busy + (size_t)(2 * X + 1) * A.K, t_end - t, t_end, bp + 1, b, lane, pbp + 1, pb, pt_end - pt, pt_end)) continue;
+        } else {
+            if (!window_free(A, A.busy + (size_t)(2 * X) * A.K, t_r, t_r + t, a, ap - 1, lane)) continue;
+            if (!window_free(A, A.busy + (size_t)(2 * X + 1) * A.K, t_end - t, t_end, bp + 1, b, lane)) continue;
+        }
         if (X == G10_DEST_HOST && A.host_capacity != 0) {
             bool ok = true;
             for (int k = a + lane; k <= b; k += 32)
@@ -330,7 +358,7 @@ struct Winner {
 // and leaves its kTopT best STALE bounds in s_tk / s_ti (uniform).
 __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L, int64_t Pn, bool classify, const Winner &w,
                                            int par, BestScratch *sc, Cand *s_cand, double *s_k, int *s_i, double *s_tk, int *s_ti,
-                                           const Cand *floor = nullptr)
+                                           const Cand *floor = nullptr, int *s_dl = nullptr, int *s_ndl = nullptr)
 {
     // with a floor (the best exact score known to the grid) only the STALE bounds that can beat it are listed
     const double floor_key = floor && floor->idx >= 0 ? cand_key(*floor) : -1.0;
@@ -429,6 +457,13 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
                 if (lane == 0) base = atomicAdd(&L.wl_count[par], (unsigned)__popc(md));
                 base = __shfl_sync(0xffffffffu, base, 0);
                 if (dirty) L.worklist[(size_t)par * L.stride + base + __popc(md & ((1u << lane) - 1u))] = (int)p;
+                if (s_dl != nullptr) {                         // ... and on the block's own list
+                    int lb = 0;
+                    if (lane == 0) lb = atomicAdd(s_ndl, __popc(md));
+                    lb = __shfl_sync(0xffffffffu, lb, 0);
+                    const int q2 = lb + __popc(md & ((1u << lane) - 1u));
+                    if (dirty && q2 < kLocalDirty) s_dl[q2] = (int)p;
+                }
             }
         }
       }
@@ -500,6 +535,8 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     __shared__ int s_nmix;
     __shared__ int s_flag;
     __shared__ unsigned char s_refresh[kLazyMaxBlocks];
+    __shared__ int s_dl[kLocalDirty];
+    __shared__ int s_ndl;
     const int G = gridDim.x, c = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t Pn = *A.Pn_dev < A.geo_stride ? *A.Pn_dev : A.geo_stride;
@@ -571,9 +608,23 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         }
         // classify the owned periods against the commit, collect DIRTY ones, local bests
         // (on the first iteration `win` matches nothing and every period is DIRTY)
+        // With unlimited host memory a DIRTY period's new destination depends on the channel bookings alone, and the
+        // pending commit's share of them is known here: the block re-examines its DIRTY periods itself, at once, which
+        // spares the grid two barriers (with finite host memory the occupancy of other blocks' slots is needed too).
+        const bool own_dirty = pending && A.host_capacity == 0;
+        if (threadIdx.x == 0) s_ndl = 0;
+        __syncthreads();
         {
-            const Cand bestF = scan_owned(A, L, Pn, true, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti);
+            const Cand bestF = scan_owned(A, L, Pn, true, win, par, &s_best, s_cand, s_k, s_i, s_tk, s_ti, nullptr,
+                                          own_dirty ? s_dl : nullptr, &s_ndl);
             if (threadIdx.x == 0) store_prop(&L.props[(size_t)pbuf * kLazyMaxBlocks + c], bestF, s_tk, s_ti);
+        }
+        if (own_dirty) {
+            const int ndl = s_ndl;                              // (scan_owned ends with a barrier)
+            if (ndl > kLocalDirty) { if (threadIdx.x == 0) atomicOr(&L.wl_count[2 + par], 1u); }
+            else
+                for (int e = warp; e < ndl; e += kPlanWarps)
+                    dest_warp(A, L, s_dl[e], lane, win.dest, win.a, win.ap, win.bp, win.b, win.t, win.t_r, win.t_end);
         }
         if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
         int rbuf = pbuf;
@@ -588,6 +639,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         peak = block_max_i64(m, s_max);
         gBest = load_best(rbuf);
         const unsigned W = __ldcg(&L.wl_count[par]);
+        const bool dirty_done = own_dirty && __ldcg(&L.wl_count[2 + par]) == 0u;     // every block took its own
         if (A.fits_always || peak <= A.cap) { status = n_mig == 0 ? G10_ALREADY_FITS : G10_FIT; break; }
         if (it >= limit) { status = limit < Pn ? G10_ITERATION_LIMIT : G10_EXHAUSTED; break; }
         rounds += 1;
@@ -595,10 +647,12 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
         if (pending) barrier_since_booking = false;
         pending = false;
         const int *wl = L.worklist + (size_t)par * L.stride;
-        if (c == 0 && threadIdx.x == 0) L.wl_count[par ^ 1] = 0;
+        if (c == 0 && threadIdx.x == 0) { L.wl_count[par ^ 1] = 0; L.wl_count[2 + (par ^ 1)] = 0; }
         par ^= 1;
         const bool few_dirty = W > 0 && W <= (unsigned)kDirtyPool && G * kTopT + kDirtyPool <= kLazyMaxBlocks * kTopT;
-        if (few_dirty) {
+        if (few_dirty && dirty_done) {
+            // (their owners have re-chosen the destinations already; they join the published bounds below)
+        } else if (few_dirty) {
             // DIRTY periods need the bookings in place: barrier; one warp re-chooses each one's destination; barrier.
             // They join the published bounds below with an unbounded score and are rescored with the others.
             if (!grid_barrier(A.bar, G, gen)) { status = -2; break; }
