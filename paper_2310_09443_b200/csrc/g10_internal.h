@@ -54,7 +54,7 @@ struct Proposal {          // a block's best candidate of one scoring round (32 
 // bounds) and the sizes of its joint rescoring rounds.
 constexpr int kLazyMaxBlocks = 256;
 constexpr int kTopT = 4;
-constexpr int kRoundM = 256;      // periods rescored together in one round, at most
+constexpr int kRoundM = 512;      // periods rescored together in one round, at most
 constexpr int kDirtyPool = 256;   // DIRTY periods of one commit that join a round (more: rescored at once, shared out)
 constexpr int kFirstM = 8;        // ... in the first round of an iteration (best bounds first)
 struct __align__(16) LazyProp {

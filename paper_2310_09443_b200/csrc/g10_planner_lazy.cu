@@ -524,13 +524,15 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     __shared__ double s_pkey[kLazyMaxBlocks * kTopT];      // published bounds of all blocks
     __shared__ int s_pidx[kLazyMaxBlocks * kTopT];
     __shared__ unsigned char s_pdone[kLazyMaxBlocks * kTopT];
-    __shared__ int s_sel[kRoundM];
-    __shared__ Cand s_new[kRoundM];
+    // what a round keeps per rescored period, in dynamic shared memory (kLazyDynBytes)
+    extern __shared__ __align__(16) unsigned char s_dyn_lazy[];
+    Cand *s_new = (Cand *)s_dyn_lazy;                                   // [kRoundM]
+    ull *s_acc = (ull *)(s_new + kRoundM);                              // [2 * kRoundM]
+    long long *s_it_s = (long long *)(s_acc + 2 * kRoundM);             // [kRoundM]
+    ull *s_it_cost = (ull *)(s_it_s + kRoundM);                         // [kRoundM]
+    int *s_sel = (int *)(s_it_cost + kRoundM);                          // [kRoundM]
+    int *s_it_d = s_sel + kRoundM, *s_it_ap = s_it_d + kRoundM, *s_it_bp = s_it_ap + kRoundM;
     __shared__ int s_wcnt[kPlanWarps];
-    __shared__ int s_it_d[kRoundM], s_it_ap[kRoundM], s_it_bp[kRoundM];
-    __shared__ long long s_it_s[kRoundM];
-    __shared__ ull s_it_cost[kRoundM];
-    __shared__ ull s_acc[2 * kRoundM];
     __shared__ int s_mix[kMixCap];
     __shared__ int s_nmix;
     __shared__ int s_flag;
@@ -879,12 +881,15 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_lazy(PlanArgs A, LazyA
     plan_epilogue(A, c, G, gen, status, peak, n_mig, rounds, bytes_ssd, bytes_host);
 }
 
+constexpr size_t kLazyDynBytes = (size_t)kRoundM * (sizeof(Cand) + 2 * sizeof(ull) + sizeof(long long) + sizeof(ull) + 4 * sizeof(int));
+
 int plan_lazy_blocks()
 {
     int dev = 0, sms = 0, per_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_plan_lazy, kPlanThreads, 0) != cudaSuccess) return 0;
+    if (cudaFuncSetAttribute(k_plan_lazy, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLazyDynBytes) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_plan_lazy, kPlanThreads, kLazyDynBytes) != cudaSuccess) return 0;
     if (per_sm < 1) return 0;
     return sms > kLazyMaxBlocks ? kLazyMaxBlocks : sms;
 }
@@ -897,7 +902,9 @@ cudaError_t launch_plan_lazy(const PlanArgs &A_in, const Workspace &w, int G, cu
     L.c_rng = w.c_rng; L.worklist = w.worklist; L.wl_count = w.wl_count; L.props = w.lazy_props; L.partials = w.lazy_partials; L.stride = A.geo_stride;
     L.tmin = w.lazy_tmin; L.tmax = w.lazy_tmax;
     void *args[] = {&A, &L};
-    return cudaLaunchCooperativeKernel((const void *)k_plan_lazy, dim3(G), dim3(kPlanThreads), args, 0, s);
+    const cudaError_t e = cudaFuncSetAttribute(k_plan_lazy, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLazyDynBytes);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchCooperativeKernel((const void *)k_plan_lazy, dim3(G), dim3(kPlanThreads), args, kLazyDynBytes, s);
 }
 
 }  // namespace g10

@@ -433,7 +433,7 @@ __global__ void __launch_bounds__(kPfNT) k_schedule_prefetch_tiled(int64_t K, in
 // ---------------------------------------------------------------------------------------------
 constexpr int kPpBatch = 512;                    // records fetched together
 constexpr int kPpResults = 256;                  // finished records a block keeps before it writes them out
-constexpr unsigned kPpPassed = 0xfffffff0u, kPpEnded = 0xfffffff1u, kPpGaveUp = 0xffffffffu;
+constexpr unsigned kPpGaveUp = 0xffffffffu;       // (in place of a record's word: the wait for it ran out)
 
 // Visiting order by counting: the position of a record is the number of records that come before it -- earlier
 // moment of the prefetch inside the iteration, or the same moment and a lower index.  Every (record, record) pair is
