@@ -213,8 +213,8 @@ int32_t g10_plan_migrations(const g10_trace *trace, uint64_t gpu_capacity_bytes,
    its lowest slot, device status word (0, or G10_DEV_TIMEOUT when a wait between thread blocks ran out: the other
    outputs are then not valid).
    `ws` (optional; G10_WS_PREFETCH, with the number of migrations in place of E; contents are scratch): with it, a
-   timeline too long for one SM's shared memory (more than 15 360 slots, up to about 25 000 slots per SM of the GPU)
-   is cut into slices, one per thread block of a cooperative launch, and every block walks the records in visiting
+   timeline too long for one SM's shared memory (more than 15 360 slots, up to about 25 000 slots per SM of the GPU;
+   at most 262 144 migrations) is cut into slices, one per thread block of a cooperative launch, and every block walks the records in visiting
    order, waiting only for the records that can still reach its slice; the result is that of the sequential pass.
    With ws == NULL (ws_bytes ignored) one block does the whole pass, record by record.
    Records of g10_plan_cyclic are accepted as they are: a slot beyond K stands for the same slot of the cycle (the

@@ -818,7 +818,10 @@ cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *
     int G = 0, L = 0, per_sm = 0;
     const unsigned *only_if = nullptr;
     int presorted = 0;
-    if (scratch.word != nullptr && tiles <= kPfMaxTiles && pf_pipe_geometry(K, &G, &L, &per_sm)) {
+    // (the visiting order by counting compares all pairs of records: fine for the tens of thousands of a plan, too slow
+    // far beyond that)
+    constexpr int64_t kPfMaxRanked = 262144;
+    if (scratch.word != nullptr && n <= kPfMaxRanked && tiles <= kPfMaxTiles && pf_pipe_geometry(K, &G, &L, &per_sm)) {
         // many blocks, one slice of the timeline each; behind them the one-block form, which runs only if the records ask for it
         k_pf_rank<<<dim3((unsigned)((n + kRankNT - 1) / kRankNT), (unsigned)((n + kRankChunk - 1) / kRankChunk)), kRankNT, 0, s>>>(n, mig, start, K, scratch.rank); count_launch();
         k_pf_prepare<<<(unsigned)((n + kRankNT - 1) / kRankNT), kRankNT, 0, s>>>(K, n, mig, bytes, order, scratch, summary); count_launch();
