@@ -65,6 +65,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w, int32_t which)
     w.bk_count = c.take<unsigned>(vit ? 4096 : 1);
     w.bk_cursor = c.take<unsigned>(vit ? 4096 : 1);
     w.bk_words = c.take<ull>(vit ? 2 * 4096 : 1);
+    w.bk_carry = c.take<long long>(4);
     w.xwords = c.take<ull>(plan ? (2 * kSmallMaxBlocks + 2 * kSmallMaxBlocks) * 16 : 1);
     w.seg_words = c.take<ull>(512 * 16);
     w.seg_words2 = c.take<ull>(512 * 16);

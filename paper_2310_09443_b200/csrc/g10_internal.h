@@ -97,6 +97,7 @@ struct Workspace {
     ull *event_budget;           // [1] events booked by the blocks of the first / last pass (at most E for a valid trace)
     unsigned *bk_count, *bk_cursor;   // [4096] events per tensor bucket, scatter cursors
     ull *bk_words;               // [2 * 4096] tagged per-bucket totals
+    long long *bk_carry;         // [4] distinct uses and periods of all tensors before the current pass (two copies used in turn)
     ull *xwords;                 // [2][kSmallMaxBlocks][16] tagged words of the proposal exchange
     ull *seg_words, *seg_words2; // [blocks * 16] each: tagged segment sums of the slot-clock scan and of the pressure scan, one 128-byte line per block
     // --- uninitialised region ---
@@ -179,7 +180,7 @@ constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock f
 // passes (g10_passes.cu)
 cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
-// bucketed formulation (g10_vitality_buckets.cu); supported for up to 4096 buckets of 4096 tensors
+// bucketed formulation (g10_vitality_buckets.cu); 4096 buckets of 4096 tensors per pass over the events, up to 16 passes
 bool vitality_buckets_supported(int64_t N, int64_t E);
 cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s);

@@ -27,8 +27,15 @@ constexpr int kBkCap = 10240;                      // events of a bucket kept in
 constexpr int kBkWide = 64;                        // a kernel with more events is walked by its whole warp in the partition
 constexpr int kBkHeavy = 32;                       // longer segments are sorted by the whole block
 
+// A trace with more tensors than 4096 buckets of 4096 hold is taken in passes over the events, each for a run of
+// consecutive tensor ids (t_begin, N of them): events of other tensors are skipped, tensor numbers inside a pass are
+// relative to t_begin, and the totals of the earlier passes come in through `carry_in`.
 struct BucketArgs {
-    int64_t N, E, K;
+    int64_t N, E, K;           // N: tensors of this pass
+    int64_t t_begin, N_total;  // first tensor id of the pass; tensors of the trace
+    int last_pass;
+    const long long *carry_in; // [2] distinct uses and periods of all tensors before the pass (nullptr: none)
+    long long *carry_out;      // [2] the same after the pass
     int shift;                 // log2(bt)
     int bt;                    // tensors per bucket
     int nb;                    // number of buckets
@@ -144,8 +151,11 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
 #pragma unroll
         for (int j = 0; j < kBkItems; ++j) {
             if (id[j] == -2) continue;
-            if (id[j] < 0 || id[j] >= B.N) bad |= G10_DEV_BAD_TENSOR_ID;
-            else atomicAdd(&s_hist[id[j] >> B.shift], 1u);
+            if (id[j] < 0 || id[j] >= B.N_total) { if (B.t_begin == 0) bad |= G10_DEV_BAD_TENSOR_ID; }
+            else {
+                const int64_t rel = (int64_t)id[j] - B.t_begin;
+                if (rel >= 0 && rel < B.N) atomicAdd(&s_hist[rel >> B.shift], 1u);
+            }
         }
     }
     if (bad) raise_status(B.status, bad);
@@ -227,7 +237,8 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_scatter(BucketArgs B, cons
 #pragma unroll
             for (int j = 0; j < kPtMaxItems; ++j) {
                 rank[j] = 0;
-                if (id[j] >= 0 && id[j] < B.N) rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1);
+                const int64_t rel = (int64_t)id[j] - B.t_begin;              // (the tensor's number inside the pass from here on)
+                if (id[j] >= 0 && rel >= 0 && rel < B.N) { id[j] = (int)rel; rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1); }
                 else id[j] = -1;
             }
             __syncthreads();
@@ -326,8 +337,8 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         const int b = s_bucket;
         if (b >= B.nb) break;
         const int n = s_base[b + 1] - s_base[b];
-        const int64_t t0 = (int64_t)b * B.bt;
-        const int bt_eff = (int)((B.N - t0) < B.bt ? (B.N - t0) : B.bt);
+        const int64_t t0 = B.t_begin + (int64_t)b * B.bt;        // first tensor id of the bucket
+        const int bt_eff = (int)((B.N - (int64_t)b * B.bt) < B.bt ? (B.N - (int64_t)b * B.bt) : B.bt);
         const ull *gk = B.pairs + s_base[b];
         int32_t *ks = n <= kBkCap ? s_ks : B.spill + s_base[b];
         for (int tl = threadIdx.x; tl <= bt_eff; tl += kBkThreads) { t_off[tl] = 0; t_d[tl] = 0; }
@@ -480,6 +491,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         if (threadIdx.x == 0) {
             long long a = 0, c2 = 0;
             for (int w = 0; w < kBkThreads / 32; ++w) { a += s_pu[w]; c2 += s_pp[w]; }
+            if (B.carry_in != nullptr) { a += B.carry_in[0]; c2 += B.carry_in[1]; }    // (the tensors of the earlier passes)
             s_pre[0] = a; s_pre[1] = c2;
         }
         __syncthreads();
@@ -518,13 +530,16 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             }
         }
         if (b == B.nb - 1 && threadIdx.x == 0) {
-            out.use_ptr[B.N] = U + D; out.period_ptr[B.N] = PB + PC;
-            out.counts[0] = U + D; out.counts[1] = PB + PC;
+            B.carry_out[0] = U + D; B.carry_out[1] = PB + PC;
+            if (B.last_pass) {
+                out.use_ptr[B.N_total] = U + D; out.period_ptr[B.N_total] = PB + PC;
+                out.counts[0] = U + D; out.counts[1] = PB + PC;
+            }
         }
     }
 }
 
-// Picks the bucket width for a trace; false if the trace is outside what the bucket path handles.
+// Picks the bucket width for (a pass over) N tensors with about E events; false if that is outside what the bucket path handles.
 static bool choose_buckets(int64_t N, int64_t E, int *shift, int *bt, int *nb)
 {
     if (N <= 0) return false;
@@ -538,21 +553,18 @@ static bool choose_buckets(int64_t N, int64_t E, int *shift, int *bt, int *nb)
     return true;
 }
 
+constexpr int64_t kBkPassTensors = (int64_t)4096 * 4096;       // tensors one pass can take (4096 buckets of 4096)
+constexpr int64_t kBkMaxPasses = 16;                           // (every pass reads all events: beyond this the plain formulation is used)
+
 bool vitality_buckets_supported(int64_t N, int64_t E)
 {
-    int a, b, c;
-    return choose_buckets(N, E, &a, &b, &c);
+    (void)E;
+    return N > 0 && N <= kBkMaxPasses * kBkPassTensors;
 }
 
-cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s)
+// One pass: the three kernels for tensors [B.t_begin, B.t_begin + B.N).
+static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const VitalityBuffers &out, int sms, cudaStream_t s)
 {
-    BucketArgs B;
-    B.N = t.N; B.E = t.E; B.K = t.K; B.tile_kernels = kBkThreads; B.tile_cap = kBkThreads;
-    if (!choose_buckets(t.N, t.E, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
-    B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
-    B.ticket = w.emit_scan.ticket; B.status = w.status; B.spill = w.raw_uses;
-    const int sms = current_sm_count();
-    if (sms <= 0) return cudaErrorInvalidDevice;
     const int64_t tiles = (t.E + kBkTile - 1) / kBkTile;
     // the second and third kernel are launched with programmatic stream serialisation (they wait for their
     // predecessor themselves): launch and block placement overlap its tail
@@ -601,6 +613,39 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
     cfg.dynamicSmemBytes = sm3;
     if ((e = cudaLaunchKernelEx(&cfg, k_bk_emit, B, out)) != cudaSuccess) return e;
     return cudaGetLastError();
+}
+
+cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s)
+{
+    if (!vitality_buckets_supported(t.N, t.E)) return cudaErrorInvalidValue;
+    const int sms = current_sm_count();
+    if (sms <= 0) return cudaErrorInvalidDevice;
+    const int64_t passes = (t.N + kBkPassTensors - 1) / kBkPassTensors;
+    for (int64_t p = 0; p < passes; ++p) {
+        BucketArgs B;
+        B.t_begin = p * kBkPassTensors;
+        B.N_total = t.N;
+        B.N = t.N - B.t_begin < kBkPassTensors ? t.N - B.t_begin : kBkPassTensors;
+        B.E = t.E; B.K = t.K; B.tile_kernels = kBkThreads; B.tile_cap = kBkThreads;
+        B.last_pass = p == passes - 1 ? 1 : 0;
+        B.carry_in = p > 0 ? w.bk_carry + 2 * ((p - 1) & 1) : nullptr;
+        B.carry_out = w.bk_carry + 2 * (p & 1);
+        // (bucket width from the pass's share of the events, taken as proportional to its share of the tensors)
+        const int64_t e_share = passes > 1 ? (int64_t)((double)t.E * (double)B.N / (double)t.N) : t.E;
+        if (!choose_buckets(B.N, e_share, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
+        B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
+        B.ticket = w.emit_scan.ticket; B.status = w.status; B.spill = w.raw_uses;
+        if (p > 0) {                                   // what the call's opening memset cleared for the first pass
+            cudaError_t e;
+            if ((e = cudaMemsetAsync(w.bk_count, 0, sizeof(unsigned) * 4096, s)) != cudaSuccess) return e;
+            if ((e = cudaMemsetAsync(w.bk_cursor, 0, sizeof(unsigned) * 4096, s)) != cudaSuccess) return e;
+            if ((e = cudaMemsetAsync(w.bk_words, 0, sizeof(ull) * 2 * 4096, s)) != cudaSuccess) return e;
+            if ((e = cudaMemsetAsync(w.emit_scan.ticket, 0, sizeof(unsigned), s)) != cudaSuccess) return e;
+        }
+        const cudaError_t e = launch_bucket_pass(B, t, out, sms, s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace g10

@@ -203,6 +203,20 @@ def test_pass_shapes(gpu, oracle, shape):
     check_timeline(gpu, oracle, tr, tb)
 
 
+def test_more_tensors_than_one_pass_of_buckets(gpu, oracle):
+    """Vitality on 18 M tensors: more than the 4096 buckets of 4096 tensors one pass of the bucketed formulation takes, so
+    the events are walked twice, the second time for the tensors from 16 777 216 on, with the first pass's totals
+    carried over.  Events concentrate around the pass boundary (a third of them within 3000 ids of it)."""
+    rng = np.random.default_rng(16777216)
+    K, N = 400_000, 18_000_000
+    deg = rng.integers(0, 9, size=K)
+    tr = _csr_trace("two_passes", rng, K, N, deg)
+    near = rng.random(tr.E) < 0.33
+    tr.kernel_tensors[near] = (16_777_216 + rng.integers(-3000, 3000, size=int(near.sum()))).astype(np.int32)
+    tb = gpu.upload(tr)
+    check_vitality(gpu, oracle, tr, tb)
+
+
 def test_inplace_relu_variant(gpu, oracle):
     tr = traces.config1_resnet152(inplace_relu=True)
     full_parity(gpu, oracle, tr)
