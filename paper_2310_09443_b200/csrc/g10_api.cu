@@ -317,8 +317,11 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
         vb = VitalityBuffers{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, ucap, w.period_ptr,
                              w.period_tensor, w.period_prev_use, w.period_next_use, pcap, w.counts};
     }
-    CU(buckets ? launch_vitality_buckets(d, w, vb, s) : launch_vitality(d, w, vb, s));
-    CU(launch_publish_status(w, vb.counts + 2, s));
+    if (buckets) CU(launch_vitality_buckets(d, w, vb, s, vb.counts + 2));     // (its last block publishes the status word)
+    else {
+        CU(launch_vitality(d, w, vb, s));
+        CU(launch_publish_status(w, vb.counts + 2, s));
+    }
     if (host) {
         int64_t counts[3];
         CU(cudaMemcpyAsync(counts, w.counts, sizeof(counts), cudaMemcpyDeviceToHost, s));
@@ -360,8 +363,7 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     int64_t *pk = host ? w.peak_bytes : out->peak_bytes;
     int32_t *ps = host ? w.peak_slot : out->peak_slot;
     int64_t *st = host ? w.counts + 2 : out->status;
-    CU(launch_timeline_pairs(d, w, start, w.tl_pair, w.tl_point, P, pk, ps, s));
-    CU(launch_publish_status(w, st, s));
+    CU(launch_timeline_pairs(d, w, start, w.tl_pair, w.tl_point, P, pk, ps, st, s));      // (its last block publishes the status word)
     if (host) {
         CU(d2h(out->kernel_start_ns, w.start, (size_t)d.K + 1, s));
         CU(d2h(out->pressure, w.pressure, (size_t)d.K, s));

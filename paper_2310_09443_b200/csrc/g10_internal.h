@@ -182,7 +182,8 @@ cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t 
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 // bucketed formulation (g10_vitality_buckets.cu); 4096 buckets of 4096 tensors per pass over the events, up to 16 passes
 bool vitality_buckets_supported(int64_t N, int64_t E);
-cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
+// (status_out, if not null, receives the device status word when the last block of the last kernel finishes)
+cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s, int64_t *status_out = nullptr);
 cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s);
 cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);
@@ -191,7 +192,7 @@ cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, 
                             int64_t stride, int64_t *geo_t, int32_t *geo_a, int32_t *geo_b, cudaStream_t s);
 // timeline call: slot clock, pressure, peak from the trace alone (g10_passes.cu)
 cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *pair, int64_t *point, int64_t *pressure,
-                                  int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);
+                                  int64_t *peak_bytes, int32_t *peak_slot, int64_t *status_out /* receives the device status word */, cudaStream_t s);
 // eager prefetch pass (g10_prefetch.cu)
 constexpr int kPfMaxBlocks = 2048;         // most blocks the many-block form of the pass may use (one slice of the timeline each)
 // Scratch of the many-block form, carved from the caller's workspace (all null: the call came without one).

@@ -50,7 +50,8 @@ __device__ __forceinline__ long long seg_warp_totals(const long long *s_w, int l
 template <int kind>
 __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t E, const int64_t *__restrict__ in, const int64_t *__restrict__ kptr,
                                                              int64_t *__restrict__ out, unsigned *ticket, unsigned *done, ull *words,
-                                                             int64_t *blk_max, int32_t *blk_slot, int64_t *peak_bytes, int32_t *peak_slot, ull *status)
+                                                             int64_t *blk_max, int32_t *blk_slot, int64_t *peak_bytes, int32_t *peak_slot, ull *status,
+                                                             int64_t *status_out)
 {
     __shared__ long long s_w[kSegWarps];
     __shared__ int s_sl[kSegWarps];
@@ -200,6 +201,9 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
                 if (s_sl[w] >= 0 && (bs < 0 || s_w[w] > bm || (s_w[w] == bm && s_sl[w] < bs))) { bm = s_w[w]; bs = s_sl[w]; }
             *peak_bytes = bs < 0 ? 0 : bm;
             *peak_slot = bs;
+            // (kind 1, the last kernel of a timeline call: every block of this grid has arrived, every earlier kernel of the
+            // call has completed, so the status word is final)
+            if (status_out != nullptr) *status_out = (int64_t)*(volatile ull *)status;
         }
     }
     }
@@ -220,7 +224,7 @@ cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t 
 {
     const int G = seg_scan_blocks(t.K);
     k_seg_scan<0><<<G, kSegThreads, 0, s>>>(t.K, t.E, t.kernel_ns, t.kernel_ptr, start, w.clock_scan.ticket, w.clock_scan.done,
-                                          w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status); count_launch();
+                                          w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status, nullptr); count_launch();
     return cudaGetLastError();
 }
 
@@ -808,7 +812,7 @@ cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int3
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);
     e = cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)nullptr, pressure, w.pressure_scan.ticket,
-                           w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
+                           w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, (int64_t *)nullptr);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
@@ -816,7 +820,7 @@ cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int3
 // The timeline call: slot clock beside the first / last pass (the two are independent), difference array from the pairs,
 // pressure scan.  `pair` [2 N], `point` [K] and the difference array start at zero (cleared by the caller).
 cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *pair, int64_t *point, int64_t *pressure,
-                                  int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
+                                  int64_t *peak_bytes, int32_t *peak_slot, int64_t *status_out, cudaStream_t s)
 {
     cudaError_t e;
     if ((e = launch_slot_clock(t, w, start, s)) != cudaSuccess) return e;
@@ -844,7 +848,7 @@ cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int6
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);
     return cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)point, pressure, w.pressure_scan.ticket,
-                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status);
+                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out);
 }
 
 // =============================================================================================

@@ -47,6 +47,8 @@ struct BucketArgs {
     ull *words;                // [2 * nb] tagged totals of each bucket: distinct uses, periods
     int32_t *spill;            // [E] per-tensor segments of buckets too large for shared memory
     unsigned *ticket;
+    unsigned *done;            // blocks of the last kernel that have finished (starts at zero)
+    int64_t *status_out;       // receives the status word when the last of them finishes the last pass (nullptr: nobody asked)
     ull *status;
 };
 
@@ -128,6 +130,8 @@ __device__ __forceinline__ void block_scan_counts(const unsigned *cnt, int n, in
 // ---------------------------------------------------------------------------------------------
 // 1. events per bucket
 // ---------------------------------------------------------------------------------------------
+// (kMulti: the trace is taken in several passes; with one pass the tensor ids are used as they are)
+template <bool kMulti>
 __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
 {
     extern __shared__ unsigned s_hist[];
@@ -151,7 +155,10 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
 #pragma unroll
         for (int j = 0; j < kBkItems; ++j) {
             if (id[j] == -2) continue;
-            if (id[j] < 0 || id[j] >= B.N_total) { if (B.t_begin == 0) bad |= G10_DEV_BAD_TENSOR_ID; }
+            if (!kMulti) {
+                if (id[j] < 0 || id[j] >= B.N) bad |= G10_DEV_BAD_TENSOR_ID;
+                else atomicAdd(&s_hist[id[j] >> B.shift], 1u);
+            } else if (id[j] < 0 || id[j] >= B.N_total) { if (B.t_begin == 0) bad |= G10_DEV_BAD_TENSOR_ID; }
             else {
                 const int64_t rel = (int64_t)id[j] - B.t_begin;
                 if (rel >= 0 && rel < B.N) atomicAdd(&s_hist[rel >> B.shift], 1u);
@@ -177,6 +184,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
 // coalesced runs.
 constexpr int kPtMaxItems = 16;                     // events per thread and round, at most (tile_cap <= 16 * kBkThreads)
 
+template <bool kMulti>
 __global__ void __launch_bounds__(kBkThreads, 2) k_bk_scatter(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
 {
     extern __shared__ __align__(16) int s_mem[];
@@ -237,9 +245,14 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_scatter(BucketArgs B, cons
 #pragma unroll
             for (int j = 0; j < kPtMaxItems; ++j) {
                 rank[j] = 0;
-                const int64_t rel = (int64_t)id[j] - B.t_begin;              // (the tensor's number inside the pass from here on)
-                if (id[j] >= 0 && rel >= 0 && rel < B.N) { id[j] = (int)rel; rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1); }
-                else id[j] = -1;
+                if (!kMulti) {
+                    if (id[j] >= 0 && id[j] < B.N) rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1);
+                    else id[j] = -1;
+                } else {
+                    const int64_t rel = (int64_t)id[j] - B.t_begin;          // (the tensor's number inside the pass from here on)
+                    if (id[j] >= 0 && rel >= 0 && rel < B.N) { id[j] = (int)rel; rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1); }
+                    else id[j] = -1;
+                }
             }
             __syncthreads();
             // (c) reserve this round's room in every bucket it touches, then turn the counts into offsets inside the round
@@ -537,6 +550,12 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             }
         }
     }
+    // the last block out, on the last pass, hands the status word over (every block's bits are in: acquire-release count)
+    if (threadIdx.x == 0 && B.last_pass && B.status_out != nullptr) {
+        unsigned arrived;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(B.done) : "memory");
+        if (arrived == gridDim.x - 1u) *B.status_out = (int64_t)*(volatile ull *)B.status;
+    }
 }
 
 // Picks the bucket width for (a pass over) N tensors with about E events; false if that is outside what the bucket path handles.
@@ -563,7 +582,7 @@ bool vitality_buckets_supported(int64_t N, int64_t E)
 }
 
 // One pass: the three kernels for tensors [B.t_begin, B.t_begin + B.N).
-static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const VitalityBuffers &out, int sms, cudaStream_t s)
+static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const VitalityBuffers &out, int sms, bool multi, cudaStream_t s)
 {
     const int64_t tiles = (t.E + kBkTile - 1) / kBkTile;
     // the second and third kernel are launched with programmatic stream serialisation (they wait for their
@@ -578,7 +597,9 @@ static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const 
     cfg.numAttrs = 1;
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
-        k_bk_hist<<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors); count_launch();
+        if (multi) k_bk_hist<true><<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
+        else k_bk_hist<false><<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
+        count_launch();
         // Shared memory of the partition kernel: three bucket tables and ten bytes per staged event; two blocks per SM.
         const size_t tables = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8;
         int64_t cap = ((int64_t)(100 << 10) - (int64_t)tables) / 10 / kBkThreads * kBkThreads;
@@ -597,13 +618,15 @@ static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const 
         const int64_t ktiles = (t.K + tk - 1) / tk;
         const int g2 = (int)(ktiles < g2max ? ktiles : g2max);
         const size_t sm2 = tables + (sizeof(ull) + sizeof(unsigned short)) * (size_t)cap;
-        cudaError_t e = cudaFuncSetAttribute(k_bk_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
+        cudaError_t e = multi ? cudaFuncSetAttribute(k_bk_scatter<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2)
+                              : cudaFuncSetAttribute(k_bk_scatter<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
         if (e != cudaSuccess) return e;
         cfg.gridDim = dim3((unsigned)g2);
         cfg.dynamicSmemBytes = sm2;
         const int64_t *kp = t.kernel_ptr;
         const int32_t *kt = t.kernel_tensors;
-        if ((e = cudaLaunchKernelEx(&cfg, k_bk_scatter, B, kp, kt)) != cudaSuccess) return e;
+        e = multi ? cudaLaunchKernelEx(&cfg, k_bk_scatter<true>, B, kp, kt) : cudaLaunchKernelEx(&cfg, k_bk_scatter<false>, B, kp, kt);
+        if (e != cudaSuccess) return e;
     }
     const size_t sm3 = sizeof(int) * (size_t)(bk_pad(B.nb) + 3 * bk_pad(B.bt) + kBkCap) + sizeof(unsigned short) * (size_t)B.bt;
     cudaError_t e = cudaFuncSetAttribute(k_bk_emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
@@ -615,7 +638,7 @@ static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const 
     return cudaGetLastError();
 }
 
-cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s)
+cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s, int64_t *status_out)
 {
     if (!vitality_buckets_supported(t.N, t.E)) return cudaErrorInvalidValue;
     const int sms = current_sm_count();
@@ -634,7 +657,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         const int64_t e_share = passes > 1 ? (int64_t)((double)t.E * (double)B.N / (double)t.N) : t.E;
         if (!choose_buckets(B.N, e_share, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
         B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
-        B.ticket = w.emit_scan.ticket; B.status = w.status; B.spill = w.raw_uses;
+        B.ticket = w.emit_scan.ticket; B.done = w.emit_scan.done; B.status_out = status_out; B.status = w.status; B.spill = w.raw_uses;
         if (p > 0) {                                   // what the call's opening memset cleared for the first pass
             cudaError_t e;
             if ((e = cudaMemsetAsync(w.bk_count, 0, sizeof(unsigned) * 4096, s)) != cudaSuccess) return e;
@@ -642,7 +665,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
             if ((e = cudaMemsetAsync(w.bk_words, 0, sizeof(ull) * 2 * 4096, s)) != cudaSuccess) return e;
             if ((e = cudaMemsetAsync(w.emit_scan.ticket, 0, sizeof(unsigned), s)) != cudaSuccess) return e;
         }
-        const cudaError_t e = launch_bucket_pass(B, t, out, sms, s);
+        const cudaError_t e = launch_bucket_pass(B, t, out, sms, passes > 1, s);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
