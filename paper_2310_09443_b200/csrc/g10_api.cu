@@ -72,9 +72,17 @@ size_t carve(void *base, const Sizes &z, Workspace &w, int32_t which)
     w.zero_bytes = align_up(c.off);
     // arrays that must start at zero, cleared only by the calls that use them (the difference array sits right behind
     // the zero-initialised region, so that one memset covers both)
-    w.diff = c.take<int64_t>(tl ? K + 1 : 1);
-    w.tl_point = c.take<int64_t>(which == G10_WS_TIMELINE ? K : 1);
-    w.tl_pair = c.take<int>(which == G10_WS_TIMELINE ? 2 * N : 1);   // (both right behind the difference array: the timeline call clears all three with one memset)
+    if (which == G10_WS_TIMELINE) {
+        // (the first / last pairs right behind the zero-initialised region: one memset covers both; the difference array and
+        // the point masses are cleared by the kernel that fills the pairs)
+        w.tl_pair = c.take<int>(2 * N);
+        w.diff = c.take<int64_t>(K + 1);
+        w.tl_point = c.take<int64_t>(K);
+    } else {
+        w.diff = c.take<int64_t>(tl ? K + 1 : 1);
+        w.tl_point = c.take<int64_t>(1);
+        w.tl_pair = c.take<int>(1);
+    }
     w.cnt = c.take<int32_t>(vit ? N : 1);
     const size_t state_begin = align_up(c.off);
     w.busy = c.take<int64_t>(plan ? 4 * K : 1);       // busy, hocc and dead are contiguous: one memset

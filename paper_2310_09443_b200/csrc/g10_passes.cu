@@ -390,11 +390,19 @@ __global__ void __launch_bounds__(kFlThreads) k_first_last_events(int64_t E, int
 // 32-byte sector, so the two reductions reach the L2 as one request; the L2 serves such scattered requests at a fixed
 // rate per sector whatever they carry (about 170 G/s on this part), which is what bounds this pass.
 __global__ void __launch_bounds__(kFlThreads) k_first_last_pairs(int64_t E, int64_t N, int64_t K, const int64_t *__restrict__ kptr,
-                                                                 const int32_t *__restrict__ kt, int32_t *__restrict__ pair, ull *budget, ull *status)
+                                                                 const int32_t *__restrict__ kt, int32_t *__restrict__ pair, ull *budget, ull *status,
+                                                                 int64_t *zero_diff, int64_t *zero_point)
 {
     __shared__ int64_t s_span[2];
     const int lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
     const int64_t kb0 = (int64_t)blockIdx.x * kFlThreads;
+    // the difference array [K + 1] and the point masses [K], which the NEXT kernel adds into, are cleared here (the grid has
+    // a thread per kernel): 16 bytes per thread instead of a third of the call's opening memset
+    if (zero_diff != nullptr) {
+        const int64_t z = kb0 + threadIdx.x;
+        if (z < K) { zero_diff[z] = 0; zero_point[z] = 0; }
+        if (z == 0) zero_diff[K] = 0;
+    }
     if (threadIdx.x == 0) {
         const int64_t kb1 = kb0 + kFlThreads < K ? kb0 + kFlThreads : K;
         int64_t b0 = kptr[kb0], b1 = kptr[kb1];
@@ -835,7 +843,11 @@ cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int6
     if (t.N > 0 && t.E > 0 && t.K > 0) {
         cfg.gridDim = dim3((unsigned)tiles_of(t.K, kFlThreads));
         cfg.blockDim = dim3(kFlThreads);
-        if ((e = cudaLaunchKernelEx(&cfg, k_first_last_pairs, t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, pair, w.event_budget, w.status)) != cudaSuccess) return e;
+        if ((e = cudaLaunchKernelEx(&cfg, k_first_last_pairs, t.E, t.N, t.K, t.kernel_ptr, t.kernel_tensors, pair, w.event_budget, w.status, w.diff, point)) != cudaSuccess) return e;
+    } else if (t.K > 0) {
+        // (no events: nothing clears the difference array and the point masses on the way)
+        if ((e = cudaMemsetAsync(w.diff, 0, sizeof(int64_t) * (size_t)(t.K + 1), s)) != cudaSuccess) return e;
+        if ((e = cudaMemsetAsync(point, 0, sizeof(int64_t) * (size_t)t.K, s)) != cudaSuccess) return e;
     }
     if (t.N > 0 && t.K > 0) {
         cfg.gridDim = dim3((unsigned)((t.N + 255) / 256));
