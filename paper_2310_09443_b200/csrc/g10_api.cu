@@ -226,6 +226,7 @@ size_t carve_emit(void *base, int64_t N, int64_t n, EmitLaunch &L, char **zero_b
     *zero_bytes = align_up(c.off);
     L.keys = c.take<ull>(total);
     L.payload = c.take<int32_t>(total);
+    L.block_count = c.take<unsigned>((size_t)4096 * kEmitMaxBlocks);
     return align_up(c.off);
 }
 

@@ -3,7 +3,9 @@
 //
 // Every instruction is one 64-bit key (boundary << 33 | opcode << 31 | tensor; unique) plus the plan record it
 // came from.  The keys are sorted with the same shape as the vitality pass: boundaries are cut into buckets of
-// consecutive boundaries holding a couple of thousand instructions, a histogram sizes the buckets, the keys are
+// consecutive boundaries holding a couple of thousand instructions, a histogram sizes the buckets -- kept per block of
+// the counting kernel, so that the scatter kernel, whose blocks walk the same items, knows each block's own run inside
+// every bucket and places its keys with shared-memory counters alone (no global cursor) --, the keys are
 // scattered into their bucket's slice, and one block per bucket sorts its slice in shared memory (counting sort by
 // boundary, then the few instructions of every boundary in key order by one thread; a boundary with more than 32
 // by a bitonic network), which also gives the CSR pointers, and writes the records out in order.
@@ -27,6 +29,8 @@ struct EmitArgs {
     const int64_t *new_issue;
     int shift, nb;                        // boundaries per bucket = 1 << shift
     unsigned *bucket_count, *bucket_cursor;
+    unsigned *block_count;                // [nb][G] per bucket: what each block of the counting kernel saw, then the running sums
+    int G;                                // blocks of the counting and of the scatter kernel (the same items go to the same block)
     ull *keys;
     int32_t *payload;
     unsigned *ticket;
@@ -78,8 +82,29 @@ __global__ void __launch_bounds__(kEmitThreads) k_emit_hist(EmitArgs A)
         if (emit_item(A, item, &bd, &op, &tn, &rc)) atomicAdd(&s_hist[bd >> A.shift], 1u);
     }
     __syncthreads();
-    for (int b = threadIdx.x; b < A.nb; b += kEmitThreads)
-        if (s_hist[b]) atomicAdd(&A.bucket_count[b], s_hist[b]);
+    // what this block saw of every bucket: the scatter kernel, whose blocks walk the same items, gets from it the block's own
+    // run inside every bucket's slice and needs no global cursor
+    for (int b = threadIdx.x; b < A.nb; b += kEmitThreads) A.block_count[(size_t)b * A.G + blockIdx.x] = s_hist[b];
+}
+
+// Per bucket: running sums over the blocks (in place) and the bucket's total.  One warp per bucket.
+__global__ void __launch_bounds__(kEmitThreads) k_emit_block_offsets(EmitArgs A)
+{
+    const int lane = threadIdx.x & 31;
+    const int b = (int)(blockIdx.x * (kEmitThreads / 32) + (threadIdx.x >> 5));
+    if (b >= A.nb) return;
+    unsigned *row = A.block_count + (size_t)b * A.G;
+    unsigned carry = 0;
+    for (int j0 = 0; j0 < A.G; j0 += 32) {
+        const int j = j0 + lane;
+        const unsigned v = j < A.G ? row[j] : 0u;
+        unsigned incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const unsigned y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        if (j < A.G) row[j] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) A.bucket_count[b] = carry;
 }
 
 // exclusive scan of the bucket counts (nb <= 4096) into s_base[0..nb]
@@ -106,17 +131,21 @@ __device__ __forceinline__ void emit_scan_buckets(const unsigned *cnt, int nb, l
 
 __global__ void __launch_bounds__(kEmitThreads) k_emit_scatter(EmitArgs A)
 {
-    extern __shared__ long long s_base[];            // [nb + 1]
+    extern __shared__ long long s_base[];            // [nb + 1] first slot of each bucket, then [nb] (unsigned) this block's next slot inside it
     __shared__ long long s_w[kEmitThreads / 32];
     emit_scan_buckets(A.bucket_count, A.nb, s_base, s_w);
+    unsigned *s_next = (unsigned *)(s_base + A.nb + 1);
+    for (int b = threadIdx.x; b < A.nb; b += kEmitThreads) s_next[b] = A.block_count[(size_t)b * A.G + blockIdx.x];
+    __syncthreads();
     const int64_t total = 2 * A.N + 2 * A.n;
     for (int64_t item = (int64_t)blockIdx.x * kEmitThreads + threadIdx.x; item < total; item += (int64_t)gridDim.x * kEmitThreads) {
         int64_t bd; int op, tn, rc;
         if (emit_item(A, item, &bd, &op, &tn, &rc)) {
             const int b = (int)(bd >> A.shift);
-            const long long pos = s_base[b] + atomicAdd(&A.bucket_cursor[b], 1u);
+            const long long pos = s_base[b] + atomicAdd(&s_next[b], 1u);       // (shared memory: the block's own run of the bucket)
             A.keys[pos] = emit_key(bd, op, tn);
-            A.payload[pos] = rc;
+            if (rc >= 0) A.payload[pos] = rc;          // (only the few instructions that come from a plan record carry one: the
+                                                       // others' payload is never read, which spares a scattered store per tensor)
         }
     }
 }
@@ -216,7 +245,7 @@ __global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int6
                     const int bd = (int)((rk[q] >> 33) - b0);
                     const int slot = s_cnt[bd] + atomicAdd(&s_cur[bd], 1);
                     s_keys[slot] = rk[q];
-                    s_pay[slot] = gp[j];
+                    s_pay[slot] = ((rk[q] >> 31) & 1u) ? gp[j] : -1;       // (PRE_EVICT = 1 and PREFETCH = 3 come from a plan record)
                 }
             __syncthreads();
             for (int bd = threadIdx.x; bd < bw_eff; bd += kEmitThreads) {
@@ -280,7 +309,7 @@ __global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int6
             const ull key = kp[j];
             const int64_t boundary = (int64_t)(key >> 33);
             g10_instruction ins;
-            ins.opcode = (int)((key >> 31) & 3u); ins.tensor = (int)(key & 0x7fffffffu); ins.record = pp[j]; ins.target = -1;
+            ins.opcode = (int)((key >> 31) & 3u); ins.tensor = (int)(key & 0x7fffffffu); ins.record = (ins.opcode & 1) ? pp[j] : -1; ins.target = -1;
             ins.bytes = A.bytes[ins.tensor];
             ins.time_ns = A.start[boundary];
             if (ins.opcode == kOpPreEvict) { ins.target = A.mig[ins.record].dest; ins.time_ns = A.mig[ins.record].evict_issue_ns; }
@@ -321,9 +350,15 @@ cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s)
     const int64_t total = 2 * L.N + 2 * L.n;
     int64_t g = (total + kEmitThreads - 1) / kEmitThreads;
     if (g > 4 * (int64_t)sms) g = 4 * (int64_t)sms;
+    if (g > kEmitMaxBlocks) g = kEmitMaxBlocks;
     if (g < 1) g = 1;
+    A.block_count = L.block_count; A.G = (int)g;
     k_emit_hist<<<(int)g, kEmitThreads, sizeof(unsigned) * (size_t)A.nb, s>>>(A); count_launch();
-    k_emit_scatter<<<(int)g, kEmitThreads, sizeof(long long) * (size_t)(A.nb + 1), s>>>(A); count_launch();
+    k_emit_block_offsets<<<(A.nb + kEmitThreads / 32 - 1) / (kEmitThreads / 32), kEmitThreads, 0, s>>>(A); count_launch();
+    const size_t sm2 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(unsigned) * (size_t)A.nb;
+    cudaError_t e2 = cudaFuncSetAttribute(k_emit_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
+    if (e2 != cudaSuccess) return e2;
+    k_emit_scatter<<<(int)g, kEmitThreads, sm2, s>>>(A); count_launch();
     const size_t sm3 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(int) * (size_t)(2 * (1 << A.shift) + 2) + 8 +
                        (sizeof(ull) + sizeof(int32_t)) * kEmitCap;
     cudaError_t e = cudaFuncSetAttribute(k_emit_write, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);

@@ -211,6 +211,7 @@ cudaError_t launch_schedule_prefetch(int64_t K, int64_t n, const g10_migration *
                                      uint64_t gpu_capacity_bytes, int64_t *P, int32_t *order, int32_t *new_last, int64_t *new_issue,
                                      int64_t *summary, const PrefetchScratch &scratch, cudaStream_t s);
 // instruction-stream emission (g10_emit.cu)
+constexpr int kEmitMaxBlocks = 1024;       // most blocks the counting and the scatter kernel run with
 struct EmitLaunch {
     int64_t K, N, n;
     const int32_t *first_use, *last_use;
@@ -220,6 +221,7 @@ struct EmitLaunch {
     const g10_migration *mig;
     const int64_t *new_issue;
     unsigned *bucket_count, *bucket_cursor, *ticket;
+    unsigned *block_count;       // [4096][kEmitMaxBlocks] instructions of each bucket seen by each block of the counting kernel
     ull *keys;
     int32_t *payload;
     ull *status;
