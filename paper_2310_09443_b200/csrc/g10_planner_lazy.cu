@@ -475,18 +475,56 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
         x.dest = (L.c_state[pf] & 3) - 1;
     }
     const Cand bestF = block_best_fast(x, sc, s_cand);
-    // the block's kTopT best bounds: kTopT rounds of block-wide maximum over the threads' current heads
+    // the block's kTopT best bounds: every warp takes the kTopT best of its lanes' lists with shuffles alone (kTopT rounds
+    // of a warp-wide maximum over the lanes' current heads; larger index on equal keys), then warp 0 takes the kTopT best
+    // of the warps' results the same way
+    __shared__ double s_wk[kPlanWarps * kTopT];
+    __shared__ int s_wi[kPlanWarps * kTopT];
+    const int warp = threadIdx.x >> 5;
+    auto warp_take = [&](double &hk, int &hi) {              // warp-wide maximum of (hk, hi); uniform result
+        double k = hk;
+        int idx = hi;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const double yk = __shfl_xor_sync(0xffffffffu, k, o);
+            const int yi = __shfl_xor_sync(0xffffffffu, idx, o);
+            if (yk > k || (yk == k && yi > idx)) { k = yk; idx = yi; }
+        }
+        hk = k; hi = idx;
+    };
 #pragma unroll 1
     for (int r = 0; r < kTopT; ++r) {
         double k = tk[0];
         int idx = ti[0];
-        block_max_key(k, idx, s_k, s_i);
-        if (idx >= 0 && idx == ti[0]) {                 // this thread's head was taken: next one moves up
+        warp_take(k, idx);
+        if (idx >= 0 && idx == ti[0]) {                 // this lane's head was taken: next one moves up
 #pragma unroll
             for (int q = 0; q < kTopT - 1; ++q) { tk[q] = tk[q + 1]; ti[q] = ti[q + 1]; }
             tk[kTopT - 1] = -1.0; ti[kTopT - 1] = -1;
         }
-        if (threadIdx.x == 0) { s_tk[r] = idx >= 0 ? k : -1.0; s_ti[r] = idx; }
+        if (lane == 0) { s_wk[warp * kTopT + r] = idx >= 0 ? k : -1.0; s_wi[warp * kTopT + r] = idx; }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // kPlanWarps * kTopT entries, two per lane (each warp's are in descending order; a lane's two need not be)
+        static_assert(kPlanWarps * kTopT <= 64, "two entries per lane of warp 0");
+        double ek[2];
+        int ei[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int e = lane + 32 * h;
+            ek[h] = e < kPlanWarps * kTopT ? s_wk[e] : -1.0;
+            ei[h] = e < kPlanWarps * kTopT ? s_wi[e] : -1;
+        }
+        if (ek[1] > ek[0] || (ek[1] == ek[0] && ei[1] > ei[0])) { const double a = ek[0]; ek[0] = ek[1]; ek[1] = a; const int b2 = ei[0]; ei[0] = ei[1]; ei[1] = b2; }
+#pragma unroll 1
+        for (int r = 0; r < kTopT; ++r) {
+            double k = ek[0];
+            int idx = ei[0];
+            warp_take(k, idx);
+            if (idx >= 0 && idx == ei[0]) { ek[0] = ek[1]; ei[0] = ei[1]; ek[1] = -1.0; ei[1] = -1; }
+            if (lane == 0) { s_tk[r] = idx >= 0 ? k : -1.0; s_ti[r] = idx; }
+        }
     }
     __syncthreads();
     return bestF;
