@@ -506,23 +506,33 @@ __device__ __forceinline__ Cand scan_owned(const PlanArgs &A, const LazyArgs &L,
     }
     __syncthreads();
     if (warp == 0) {
-        // kPlanWarps * kTopT entries, two per lane (each warp's are in descending order; a lane's two need not be)
-        static_assert(kPlanWarps * kTopT <= 64, "two entries per lane of warp 0");
-        double ek[2];
-        int ei[2];
+        // kPlanWarps * kTopT entries, kPerLane per lane, kept in descending order by the lane
+        constexpr int kPerLane = (kPlanWarps * kTopT + 31) / 32;
+        double ek[kPerLane];
+        int ei[kPerLane];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < kPerLane; ++h) {
             const int e = lane + 32 * h;
-            ek[h] = e < kPlanWarps * kTopT ? s_wk[e] : -1.0;
-            ei[h] = e < kPlanWarps * kTopT ? s_wi[e] : -1;
+            double k = e < kPlanWarps * kTopT ? s_wk[e] : -1.0;
+            int idx = e < kPlanWarps * kTopT ? s_wi[e] : -1;
+            if (idx < 0) k = -1.0;
+            // insertion into ek[0..h)
+#pragma unroll
+            for (int q = 0; q < kPerLane; ++q) {
+                if (q < h && (k > ek[q] || (k == ek[q] && idx > ei[q]))) { const double a = ek[q]; ek[q] = k; k = a; const int b2 = ei[q]; ei[q] = idx; idx = b2; }
+            }
+            ek[h] = k; ei[h] = idx;
         }
-        if (ek[1] > ek[0] || (ek[1] == ek[0] && ei[1] > ei[0])) { const double a = ek[0]; ek[0] = ek[1]; ek[1] = a; const int b2 = ei[0]; ei[0] = ei[1]; ei[1] = b2; }
 #pragma unroll 1
         for (int r = 0; r < kTopT; ++r) {
             double k = ek[0];
             int idx = ei[0];
             warp_take(k, idx);
-            if (idx >= 0 && idx == ei[0]) { ek[0] = ek[1]; ei[0] = ei[1]; ek[1] = -1.0; ei[1] = -1; }
+            if (idx >= 0 && idx == ei[0]) {
+#pragma unroll
+                for (int q = 0; q < kPerLane - 1; ++q) { ek[q] = ek[q + 1]; ei[q] = ei[q + 1]; }
+                ek[kPerLane - 1] = -1.0; ei[kPerLane - 1] = -1;
+            }
             if (lane == 0) { s_tk[r] = idx >= 0 ? k : -1.0; s_ti[r] = idx; }
         }
     }
