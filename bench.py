@@ -41,8 +41,8 @@ L2_FLUSH_BYTES = 512 << 20
 # caches alone between launches, as this program does: the write-back of the L2 flush's dirty lines is part of it).
 # "sources_sha256" is the hash of the kernel sources at the time of the capture: when the sources have changed since, the
 # bench line says so ("traffic_stale") instead of passing old traffic off as current, and a CPU test warns.
-TRAFFIC = {"vitality": 242_500_000, "timeline": 110_000_000, "captured_at": "2026-11-25",
-           "sources_sha256": "ac29ffd5ce9d5251e4fb839bdb2b35f20f5d1142fd9b8062e57e75a4201d05e4"}
+TRAFFIC = {"vitality": 242_600_000, "timeline": 113_900_000, "captured_at": "2026-11-25",
+           "sources_sha256": "c33140bd1ea69c88067b5bf3a564020ec54dc057ba2a91ee4f9d54674fb747dd"}
 
 
 PASS_SOURCES = ("g10_passes.cu", "g10_vitality_buckets.cu")     # the kernels of g10_vitality and g10_pressure_timeline
