@@ -356,8 +356,10 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         int32_t *ks = n <= kBkCap ? s_ks : B.spill + s_base[b];
         for (int tl = threadIdx.x; tl <= bt_eff; tl += kBkThreads) { t_off[tl] = 0; t_d[tl] = 0; }
         __syncthreads();
-        // ---- raw events per tensor, segment offsets, scatter (the keys of a usual bucket stay in registers)
-        constexpr int kRegKeys = 12;
+        // ---- raw events per tensor, segment offsets, scatter.  The first keys of the bucket stay in registers between the
+        // counting and the scatter; the rest is read again (from L2).  Six per thread: with twelve -- every key of a usual
+        // bucket -- the kernel needs more than the 64 registers that let two blocks share an SM, and spills.
+        constexpr int kRegKeys = 6;
         ull rk[kRegKeys];
 #pragma unroll
         for (int q = 0; q < kRegKeys; ++q) {
@@ -519,16 +521,35 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         if (dense)
             for (int j = threadIdx.x; j < n; j += kBkThreads)
                 if (U + j < out.uses_cap) out.uses[U + j] = ks[j];
-        for (int tl = threadIdx.x; tl < bt_eff; tl += kBkThreads) {
+        // (two tensors of the thread at a time: their table entries, then their first and last use, are loaded together --
+        // the loop is a chain of dependent shared-memory reads otherwise)
+        for (int tl0 = threadIdx.x; tl0 < bt_eff; tl0 += 2 * kBkThreads) {
+            int d04[2], dd4[2], of4[2], np4[2];
+            int32_t f4[2], l4[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int tl = tl0 + q * kBkThreads;
+                d04[q] = 0; dd4[q] = -1; of4[q] = 0; np4[q] = 0;
+                if (tl < bt_eff) { d04[q] = t_d[tl]; dd4[q] = t_d[tl + 1] - d04[q]; of4[q] = t_off[tl]; np4[q] = t_np[tl]; }
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                f4[q] = -1; l4[q] = -1;
+                if (dd4[q] > 0) { f4[q] = ks[of4[q]]; l4[q] = ks[of4[q] + dd4[q] - 1]; }
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+            const int tl = tl0 + q * kBkThreads;
+            if (dd4[q] < 0) continue;
             const int64_t t = t0 + tl;
-            const int dd = t_d[tl + 1] - t_d[tl];
-            const int32_t *seg = ks + t_off[tl];
-            out.first_use[t] = dd > 0 ? seg[0] : -1;
-            out.last_use[t] = dd > 0 ? seg[dd - 1] : -1;
+            const int dd = dd4[q];
+            const int32_t *seg = ks + of4[q];
+            out.first_use[t] = f4[q];
+            out.last_use[t] = l4[q];
             out.num_uses[t] = dd;
-            out.use_ptr[t] = U + t_d[tl];
-            out.period_ptr[t] = PB + t_np[tl];
-            long long uo = U + t_d[tl], po = PB + t_np[tl];
+            out.use_ptr[t] = U + d04[q];
+            out.period_ptr[t] = PB + np4[q];
+            long long uo = U + d04[q], po = PB + np4[q];
             for (int a = dense ? 1 : 0; a < dd; ++a) {
                 const int32_t x = seg[a];
                 if (!dense && uo + a < out.uses_cap) out.uses[uo + a] = x;
@@ -540,6 +561,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
                     }
                     ++po;
                 }
+            }
             }
         }
         if (b == B.nb - 1 && threadIdx.x == 0) {
