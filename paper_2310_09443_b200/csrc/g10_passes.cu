@@ -60,8 +60,10 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
     // Nothing later in a call reads the slot clock, so a kernel launched behind this one with programmatic stream
     // serialisation may start as soon as every block of this grid is running (no effect on ordinary launches).
     if (kind == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    else asm volatile("griddepcontrol.wait;" ::: "memory");   // (the difference array is complete; see k_diff_scatter)
+    // (the segment number comes from a counter that the call's opening memset cleared, before any kernel: it can be taken
+    // while the predecessor still runs)
     const int g = next_tile(ticket);
+    if (kind != 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // (the difference array is complete; see k_diff_scatter)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t seg = ((n + G - 1) / G + kSegChunk - 1) / kSegChunk * kSegChunk;
     const int64_t lo = (int64_t)g * seg, hi = lo + seg < n ? lo + seg : n;
