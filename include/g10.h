@@ -56,6 +56,7 @@ extern "C" {
 #define G10_DEV_PERIODS_OVERFLOW 0x20 /* periods_cap too small (counts[1] holds the need)         */
 #define G10_DEV_PLAN_OVERFLOW 0x40   /* migrations_cap too small (summary[0] holds the need)      */
 #define G10_DEV_TIMEOUT 0x80         /* an internal wait gave up; the kernel returned early       */
+#define G10_DEV_BAD_FIRST_LAST 0x200 /* first_use / last_use handed to g10_pressure_timeline: last < first or last >= K (tensor skipped) */
 #define G10_DEV_BATCH_UNFIT 0x100    /* internal: the trace does not fit one SM (g10_plan_batch then plans the variants one by one) */
 
 /* exit status of the planner (summary[2]) */
@@ -107,6 +108,13 @@ typedef struct g10_timeline_out {
     int64_t *peak_bytes;        /* [1] max pressure (0 if K = 0)                                    */
     int32_t *peak_slot;         /* [1] lowest slot attaining it (-1 if K = 0)                       */
     int64_t *status;            /* [1] device status word                                           */
+    /* Optional INPUTS (both or neither; device traces only): first / last use of every tensor as
+       g10_vitality returned them ([N], -1 = unused).  A caller that runs the vitality analysis anyway
+       hands them over and the timeline call does not walk kernel_tensors a second time: it books every
+       tensor's size at the slots given (a pair with last < first or last >= K sets
+       G10_DEV_BAD_FIRST_LAST and is skipped).  Without them the call derives both from the trace. */
+    const int32_t *first_use;
+    const int32_t *last_use;
 } g10_timeline_out;
 
 /* Candidate geometry of a period for one destination (Algorithm 1: t = tensor_size / BW; Section 4.4:

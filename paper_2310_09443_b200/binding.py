@@ -53,7 +53,7 @@ class _VitalityOut(C.Structure):
 
 class _TimelineOut(C.Structure):
     _fields_ = [("kernel_start_ns", C.c_void_p), ("pressure", C.c_void_p), ("peak_bytes", C.c_void_p),
-                ("peak_slot", C.c_void_p), ("status", C.c_void_p)]
+                ("peak_slot", C.c_void_p), ("status", C.c_void_p), ("first_use", C.c_void_p), ("last_use", C.c_void_p)]
 
 
 class _GeometryOut(C.Structure):
@@ -259,15 +259,18 @@ def g10_vitality(tb: TraceBuffers, ws=None, stream=None, device=None, uses_cap=N
     return r
 
 
-def g10_pressure_timeline(tb: TraceBuffers, ws=None, stream=None, device=None, out=None):
-    """Section 4.3 memory-pressure timeline before any migration.  `out`: an earlier result to write into."""
+def g10_pressure_timeline(tb: TraceBuffers, ws=None, stream=None, device=None, out=None, first_last=None):
+    """Section 4.3 memory-pressure timeline before any migration.  `out`: an earlier result to write into.
+    first_last: (first_use, last_use) device tensors of an earlier g10_vitality call on the same trace; with them the
+    call does not derive first / last use from the trace again."""
     lib = load_library()
     r = out if out is not None else SimpleNamespace(
         kernel_start_ns=_alloc(tb, tb.K + 1, torch.int64, device), pressure=_alloc(tb, max(tb.K, 1), torch.int64, device),
         peak_bytes=_alloc(tb, 1, torch.int64, device), peak_slot=_alloc(tb, 1, torch.int32, device),
         status=_alloc(tb, 1, torch.int64, device))
     ws, ws_bytes = _workspace(tb, WS_TIMELINE, ws, device)
-    to = _TimelineOut(_ptr(r.kernel_start_ns), _ptr(r.pressure), _ptr(r.peak_bytes), _ptr(r.peak_slot), _ptr(r.status))
+    to = _TimelineOut(_ptr(r.kernel_start_ns), _ptr(r.pressure), _ptr(r.peak_bytes), _ptr(r.peak_slot), _ptr(r.status),
+                      _ptr(first_last[0]) if first_last is not None else None, _ptr(first_last[1]) if first_last is not None else None)
     tr = tb.c_struct()
     _check(lib.g10_pressure_timeline(C.byref(tr), C.byref(to), _ptr(ws), ws_bytes, _stream(stream)))
     r.workspace = ws

@@ -364,7 +364,10 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
-    rc = begin_call(G10_WS_TIMELINE, trace, ws, w, d, s, kZeroPairs);
+    if ((out->first_use == nullptr) != (out->last_use == nullptr)) return G10_ERR_ARG;
+    const bool given = out->first_use != nullptr;          // first / last use from the caller's vitality analysis
+    if (given && trace->mem != G10_MEM_DEVICE) return G10_ERR_ARG;
+    rc = begin_call(G10_WS_TIMELINE, trace, ws, w, d, s, given ? 0 : kZeroPairs);
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     int64_t *start = host ? w.start : out->kernel_start_ns;
@@ -372,7 +375,13 @@ int32_t g10_pressure_timeline(const g10_trace *trace, g10_timeline_out *out, voi
     int64_t *pk = host ? w.peak_bytes : out->peak_bytes;
     int32_t *ps = host ? w.peak_slot : out->peak_slot;
     int64_t *st = host ? w.counts + 2 : out->status;
-    CU(launch_timeline_pairs(d, w, start, w.tl_pair, w.tl_point, P, pk, ps, st, s));      // (its last block publishes the status word)
+    if (given) {
+        // (difference array and point masses sit next to each other: one memset; the pair array is not used)
+        CU(cudaMemsetAsync(w.diff, 0, (size_t)((char *)(w.tl_point + d.K) - (char *)w.diff), s));
+        CU(launch_timeline_given(d, w, start, out->first_use, out->last_use, w.tl_point, P, pk, ps, st, s));
+    } else {
+        CU(launch_timeline_pairs(d, w, start, w.tl_pair, w.tl_point, P, pk, ps, st, s));  // (its last block publishes the status word)
+    }
     if (host) {
         CU(d2h(out->kernel_start_ns, w.start, (size_t)d.K + 1, s));
         CU(d2h(out->pressure, w.pressure, (size_t)d.K, s));

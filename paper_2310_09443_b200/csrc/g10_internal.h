@@ -193,6 +193,9 @@ cudaError_t launch_geometry(int64_t K, int64_t Pn_bound, const int64_t *Pn_dev, 
 // timeline call: slot clock, pressure, peak from the trace alone (g10_passes.cu)
 cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int64_t *start, int32_t *pair, int64_t *point, int64_t *pressure,
                                   int64_t *peak_bytes, int32_t *peak_slot, int64_t *status_out /* receives the device status word */, cudaStream_t s);
+// timeline call with first / last use handed over by the caller (g10_passes.cu)
+cudaError_t launch_timeline_given(const DeviceTrace &t, const Workspace &w, int64_t *start, const int32_t *first_use, const int32_t *last_use,
+                                  int64_t *point, int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, int64_t *status_out, cudaStream_t s);
 // eager prefetch pass (g10_prefetch.cu)
 constexpr int kPfMaxBlocks = 2048;         // most blocks the many-block form of the pass may use (one slice of the timeline each)
 // Scratch of the many-block form, carved from the caller's workspace (all null: the call came without one).

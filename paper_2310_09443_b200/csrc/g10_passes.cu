@@ -795,6 +795,39 @@ __global__ void __launch_bounds__(256) k_diff_scatter_pairs(int64_t N, int64_t K
     }
 }
 
+// The same from first / last use as the vitality analysis reports them (-1 = unused), handed over by the caller.
+__global__ void __launch_bounds__(256) k_diff_scatter_given(int64_t N, int64_t K, const int64_t *__restrict__ bytes, const uint8_t *__restrict__ glob,
+                                                            const int32_t *__restrict__ first_use, const int32_t *__restrict__ last_use,
+                                                            ull *__restrict__ diff, ull *__restrict__ point, ull *status)
+{
+    __shared__ long long s_part[8];
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // (see k_diff_scatter)
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    long long gsum = 0;
+    if (i < N) {
+        const long long b = bytes[i];
+        if (b < 1 || b >= ((long long)1 << 40)) raise_status(status, G10_DEV_BAD_BYTES);
+        const int64_t f = first_use[i], l = last_use[i];
+        if (f >= 0) {
+            if (l < f || l >= K) raise_status(status, G10_DEV_BAD_FIRST_LAST);
+            else if (glob != nullptr && glob[i]) gsum = b;
+            else if (f == l) atomicAdd(&point[f], (ull)b);
+            else {
+                atomicAdd(&diff[f], (ull)b);
+                if (l + 1 < K) atomicAdd(&diff[l + 1], (ull)(-b));
+            }
+        }
+    }
+    gsum = warp_sum_i64(gsum);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = gsum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long tot = 0;
+        for (int w = 0; w < 8; ++w) tot += s_part[w];
+        if (tot != 0) atomicAdd(&diff[0], (ull)tot);
+    }
+}
+
 cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s)
 {
@@ -858,6 +891,34 @@ cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int6
         const uint8_t *glob = t.tensor_global;
         const int2 *cpair = reinterpret_cast<const int2 *>(pair);
         if ((e = cudaLaunchKernelEx(&cfg, k_diff_scatter_pairs, t.N, t.K, bytes, glob, cpair, (ull *)w.diff, (ull *)point, w.status)) != cudaSuccess) return e;
+    }
+    cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
+    cfg.blockDim = dim3(kSegThreads);
+    return cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)point, pressure, w.pressure_scan.ticket,
+                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out);
+}
+
+// The timeline call when the caller hands first / last use over: slot clock, then (beside it) the bookings, then the scan.
+// The caller has cleared w.diff [K + 1] and point [K].
+cudaError_t launch_timeline_given(const DeviceTrace &t, const Workspace &w, int64_t *start, const int32_t *first_use, const int32_t *last_use,
+                                  int64_t *point, int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, int64_t *status_out, cudaStream_t s)
+{
+    cudaError_t e;
+    if ((e = launch_slot_clock(t, w, start, s)) != cudaSuccess) return e;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (t.N > 0 && t.K > 0) {
+        cfg.gridDim = dim3((unsigned)((t.N + 255) / 256));
+        cfg.blockDim = dim3(256);
+        const int64_t *bytes = t.tensor_bytes;
+        const uint8_t *glob = t.tensor_global;
+        if ((e = cudaLaunchKernelEx(&cfg, k_diff_scatter_given, t.N, t.K, bytes, glob, first_use, last_use, (ull *)w.diff, (ull *)point, w.status)) != cudaSuccess) return e;
     }
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);

@@ -51,6 +51,13 @@ def check_timeline(gpu, oracle, tr, tb):
     assert np.array_equal(_np(tl.kernel_start_ns)[:tr.K + 1], start)
     assert np.array_equal(_np(tl.pressure)[:tr.K], P0)
     assert int(tl.peak_bytes.item()) == peak and int(tl.peak_slot.item()) == slot
+    # the same call with first / last use handed over from the vitality call
+    v = gpu.g10_vitality(tb)
+    tg = gpu.g10_pressure_timeline(tb, first_last=(v.first_use, v.last_use))
+    torch.cuda.synchronize()
+    assert int(tg.status.item()) == 0
+    assert np.array_equal(_np(tg.kernel_start_ns)[:tr.K + 1], start) and np.array_equal(_np(tg.pressure)[:tr.K], P0)
+    assert int(tg.peak_bytes.item()) == peak and int(tg.peak_slot.item()) == slot
     return tl, (start, P0, peak, slot)
 
 
@@ -296,6 +303,19 @@ def test_bad_trace_sets_status_bits(gpu):
     assert _np(v.counts)[2] & 0x1
     st = int(tl.status.item())
     assert (st & 0x1) and (st & 0x8) and (st & 0x4)
+    # first / last use handed over but wrong (last before first, last beyond the trace): flagged, skipped, in bounds
+    good = traces.config0_mlp_chain()
+    tbg = gpu.upload(good)
+    vg = gpu.g10_vitality(tbg)
+    torch.cuda.synchronize()
+    first, last = vg.first_use.clone(), vg.last_use.clone()
+    last[3] = first[3] - 1 if int(first[3]) > 0 else -5
+    last[9] = good.K + 7
+    tg = gpu.g10_pressure_timeline(tbg, first_last=(first, last))
+    ok = gpu.g10_pressure_timeline(tbg)
+    torch.cuda.synchronize()
+    assert int(tg.status.item()) == 0x200 and int(ok.status.item()) == 0
+    assert int(tg.peak_bytes.item()) <= int(ok.peak_bytes.item())
 
 
 def test_bad_kernel_ptr_is_flagged(gpu):
