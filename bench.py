@@ -238,8 +238,10 @@ def scaled_passes(torch, binding, tb, times, flush, hbm_peak, peak_kind, reps=5)
     out = {"times": times, "K": big.K, "N": big.N, "E": big.E, "uses": uses, "periods": periods,
            "device_status": int(v.counts[2].item()) | int(tl.status.item()), "repetitions": reps,
            "peak_bytes_is_that_of_one_copy": True}
+    fl = (v.first_use.clone(), v.last_use.clone())          # (as in the headline step: first / last use handed over to the timeline call)
     del v, tl
-    for name, fn, nb in (("vitality", lambda: binding.g10_vitality(big, ws=ws), vb), ("timeline", lambda: binding.g10_pressure_timeline(big, ws=ws), tlb)):
+    for name, fn, nb in (("vitality", lambda: binding.g10_vitality(big, ws=ws), vb),
+                         ("timeline", lambda: binding.g10_pressure_timeline(big, ws=ws, first_last=fl), tlb)):
         cold = float(np.median(timed(torch, fn, reps, 2, flush)))
         warm = float(np.median(timed(torch, fn, reps, 2, None)))
         out[name + "_ms"] = cold
@@ -247,7 +249,8 @@ def scaled_passes(torch, binding, tb, times, flush, hbm_peak, peak_kind, reps=5)
         out[name + "_roofline"] = roofline(nb, cold / 1e3, hbm_peak, peak_kind)
     out["events_per_s"] = big.E / ((out["vitality_ms"] + out["timeline_ms"]) / 1e3)
     out["roofline"] = roofline(vb + tlb, (out["vitality_ms"] + out["timeline_ms"]) / 1e3, hbm_peak, peak_kind)
-    del big, ws
+    out["timeline_note"] = "first / last use handed over from the vitality call, as in the headline step"
+    del big, ws, fl
     torch.cuda.empty_cache()
     return out
 
