@@ -41,8 +41,8 @@ L2_FLUSH_BYTES = 512 << 20
 # caches alone between launches, as this program does: the write-back of the L2 flush's dirty lines is part of it).
 # "sources_sha256" is the hash of the kernel sources at the time of the capture: when the sources have changed since, the
 # bench line says so ("traffic_stale") instead of passing old traffic off as current, and a CPU test warns.
-TRAFFIC = {"vitality": 228_600_000, "timeline": 118_500_000, "timeline_given": 133_500_000, "captured_at": "2026-11-25",
-           "sources_sha256": "7167c4b4a8eae54401e81f0c01ccd4f560b8902ddd683c39e0133d545ba22196"}
+TRAFFIC = {"vitality": 228_600_000, "timeline": 118_500_000, "timeline_given": 133_500_000, "fused": 327_800_000, "captured_at": "2026-11-25",
+           "sources_sha256": "ae10dc0f9199f2b40fd454d3918e240de7e5e68966304de51b85aced14a28358"}
 
 
 PASS_SOURCES = ("g10_passes.cu", "g10_vitality_buckets.cu")     # the kernels of g10_vitality and g10_pressure_timeline
@@ -247,10 +247,14 @@ def scaled_passes(torch, binding, tb, times, flush, hbm_peak, peak_kind, reps=5)
         out[name + "_ms"] = cold
         out[name + "_ms_warm_l2"] = warm
         out[name + "_roofline"] = roofline(nb, cold / 1e3, hbm_peak, peak_kind)
-    out["events_per_s"] = big.E / ((out["vitality_ms"] + out["timeline_ms"]) / 1e3)
-    out["roofline"] = roofline(vb + tlb, (out["vitality_ms"] + out["timeline_ms"]) / 1e3, hbm_peak, peak_kind)
-    out["timeline_note"] = "first / last use handed over from the vitality call, as in the headline step"
-    del big, ws, fl
+    # both analyses from one call, as in the headline step
+    vf = binding.g10_vitality(big, ws=ws, timeline=True)
+    fused = float(np.median(timed(torch, lambda: binding.g10_vitality(big, ws=ws, out=vf, timeline=vf.timeline), reps, 2, flush)))
+    out["s123_one_call_ms"] = fused
+    out["events_per_s"] = big.E / (fused / 1e3)
+    out["roofline"] = roofline(vb + tlb, fused / 1e3, hbm_peak, peak_kind)
+    out["timeline_note"] = "timeline_ms: first / last use handed over from an earlier vitality call; events_per_s and roofline: both analyses from one g10_vitality call, as in the headline step"
+    del big, ws, fl, vf
     torch.cuda.empty_cache()
     return out
 
@@ -335,10 +339,10 @@ def run_ours(args):
     vit_bytes, tl_bytes = pass_bytes(K, N, E, uses, periods)
 
     def step():
-        # (the timeline call takes first / last use from the vitality call of the same step instead of walking the events
-        # a second time; the e2e leg below and `passes.timeline_ms` use the form that derives them from the trace)
-        binding.g10_vitality(tb, ws=ws, out=v)
-        binding.g10_pressure_timeline(tb, ws=ws, out=tl, first_last=(v.first_use, v.last_use))
+        # (one call gives both analyses: the vitality kernel that writes first / last use books every tensor's size on its
+        # way, so that the events are walked once and only the slot clock and the pressure scan are left; the e2e leg
+        # below and `passes.vitality_ms` / `passes.timeline_ms` time the two calls on their own)
+        binding.g10_vitality(tb, ws=ws, out=v, timeline=tl)
 
     for _ in range(args.warmup):
         flush.fill_(1)
@@ -407,6 +411,7 @@ def run_ours(args):
     vit_cold = float(np.median(timed(torch, lambda: binding.g10_vitality(tb, ws=ws), reps, 3, flush)))
     tl_cold = float(np.median(timed(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), reps, 3, flush)))
     tlg_cold = float(np.median(timed(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws, first_last=(v.first_use, v.last_use)), reps, 3, flush)))
+    fused_cold = float(np.median(timed(torch, lambda: binding.g10_vitality(tb, ws=ws, out=v, timeline=tl), reps, 3, flush)))
     vit_warm = float(np.median(timed(torch, lambda: binding.g10_vitality(tb, ws=ws), reps, 3, None)))
     tl_warm = float(np.median(timed(torch, lambda: binding.g10_pressure_timeline(tb, ws=ws), reps, 3, None)))
     sha = kernel_sources_sha256()
@@ -414,9 +419,9 @@ def run_ours(args):
     traffic_note = {"captured_at": TRAFFIC["captured_at"], "sources_sha256_at_capture": TRAFFIC["sources_sha256"],
                     "sources_sha256_now": sha, "traffic_stale": stale}
     roof = roofline(vit_bytes + tl_bytes, step_s, hbm_peak, peak_kind,
-                    kernel="S1-S3: g10_vitality (k_bk_hist, k_bk_scatter, k_bk_emit) + g10_pressure_timeline with first / last use "
-                           "from the vitality call (k_seg_scan<0>, k_diff_scatter_given, k_seg_scan<1>)",
-                    dominant_kernel="k_bk_emit", traffic=TRAFFIC["vitality"] + TRAFFIC["timeline_given"], traffic_note=traffic_note,
+                    kernel="S1-S3 in one call, g10_vitality with its timeline output: k_seg_scan<0> (slot clock), k_bk_hist, k_bk_scatter, "
+                           "k_bk_emit<true> (uses, periods and the bookings of the tensors' sizes), k_seg_scan<1> (pressure, peak)",
+                    dominant_kernel="k_bk_emit", traffic=TRAFFIC["fused"], traffic_note=traffic_note,
                     ms=step_s * 1e3, algorithmic_bytes_per_event=(vit_bytes + tl_bytes) / E,
                     roofline_events_per_s=E / ((vit_bytes + tl_bytes) / (hbm_peak * 1e9)),
                     note="random accesses of the passes are bound by the L2's rate of scattered 32-byte sector requests "
@@ -425,9 +430,10 @@ def run_ours(args):
               "vitality_roofline": roofline(vit_bytes, vit_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["vitality"]),
               "timeline_roofline": roofline(tl_bytes, tl_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["timeline"]),
               "timeline_after_vitality_ms": tlg_cold,
+              "s123_one_call_ms": fused_cold,
               "timeline_after_vitality_roofline": roofline(tl_bytes, tlg_cold / 1e3, hbm_peak, peak_kind, traffic=TRAFFIC["timeline_given"]),
               "timeline_note": "timeline_ms: first / last use derived from the trace (k_first_last_pairs); timeline_after_vitality_ms: "
-                               "handed over from the vitality call, as in the timed step",
+                               "handed over from an earlier vitality call; the timed step gets both analyses from one g10_vitality call",
               "repetitions": reps, "l2": "flushed between timed calls (the *_warm_l2 figures: not flushed)"}
 
     if args.passes_only:                   # (small profiling target: the headline and the per-call figures only)

@@ -97,6 +97,12 @@ typedef struct g10_vitality_out {
     int32_t *period_tensor, *period_prev_use, *period_next_use;   /* [periods_cap] (E always suffices) */
     int64_t periods_cap;
     int64_t *counts;                            /* [3]: number of uses E', number of periods Pn, device status word */
+    /* Optional (NULL = no): the memory-pressure timeline of the same trace from the same call (device traces
+       only; workspace G10_WS_ANALYSIS).  The kernel that writes first / last use books every tensor's size
+       on the way, so that S1 - S3 walk the events once and only the slot clock and the pressure scan are
+       left.  Its first_use / last_use inputs must be NULL; its outputs and status word are those of
+       g10_pressure_timeline. */
+    struct g10_timeline_out *timeline;
 } g10_vitality_out;
 
 /* Memory-pressure timeline (Section 4.3: pressure = total size of the tensors resident in GPU memory
@@ -184,6 +190,7 @@ typedef struct g10_options {
 #define G10_WS_EMIT 4
 #define G10_WS_BATCH 5
 #define G10_WS_PREFETCH 6
+#define G10_WS_ANALYSIS 7   /* g10_vitality with its `timeline` output */
 
 /* Section 4.2, tensor vitality analysis.  Device-found errors land in counts[2]; with G10_DEV_BAD_KERNEL_PTR every
    tensor is reported unused (no uses, no periods), with G10_DEV_BAD_TENSOR_ID the offending entries are skipped. */

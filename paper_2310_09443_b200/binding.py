@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libg10.so")
 
 MEM_DEVICE, MEM_HOST = 0, 1
-WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT, WS_BATCH, WS_PREFETCH = 0, 1, 2, 3, 4, 5, 6
+WS_VITALITY, WS_TIMELINE, WS_PLAN, WS_GEOMETRY, WS_EMIT, WS_BATCH, WS_PREFETCH, WS_ANALYSIS = 0, 1, 2, 3, 4, 5, 6, 7
 DEST_SSD, DEST_HOST = 0, 1
 FLAG_RESCORE_ALL = 1
 FLAG_GLOBAL_STATE = 2
@@ -44,16 +44,17 @@ class _Trace(C.Structure):
                 ("kernel_ns", C.c_void_p), ("tensor_global", C.c_void_p), ("mem", C.c_int32)]
 
 
+class _TimelineOut(C.Structure):
+    _fields_ = [("kernel_start_ns", C.c_void_p), ("pressure", C.c_void_p), ("peak_bytes", C.c_void_p),
+                ("peak_slot", C.c_void_p), ("status", C.c_void_p), ("first_use", C.c_void_p), ("last_use", C.c_void_p)]
+
+
 class _VitalityOut(C.Structure):
     _fields_ = [("first_use", C.c_void_p), ("last_use", C.c_void_p), ("num_uses", C.c_void_p),
                 ("use_ptr", C.c_void_p), ("uses", C.c_void_p), ("uses_cap", C.c_int64),
                 ("period_ptr", C.c_void_p), ("period_tensor", C.c_void_p), ("period_prev_use", C.c_void_p),
-                ("period_next_use", C.c_void_p), ("periods_cap", C.c_int64), ("counts", C.c_void_p)]
-
-
-class _TimelineOut(C.Structure):
-    _fields_ = [("kernel_start_ns", C.c_void_p), ("pressure", C.c_void_p), ("peak_bytes", C.c_void_p),
-                ("peak_slot", C.c_void_p), ("status", C.c_void_p), ("first_use", C.c_void_p), ("last_use", C.c_void_p)]
+                ("period_next_use", C.c_void_p), ("periods_cap", C.c_int64), ("counts", C.c_void_p),
+                ("timeline", C.POINTER(_TimelineOut))]
 
 
 class _GeometryOut(C.Structure):
@@ -236,10 +237,12 @@ def _alloc(tb, shape, dtype, device):
     return torch.empty(shape, dtype=dtype).pin_memory()
 
 
-def g10_vitality(tb: TraceBuffers, ws=None, stream=None, device=None, uses_cap=None, periods_cap=None, out=None):
+def g10_vitality(tb: TraceBuffers, ws=None, stream=None, device=None, uses_cap=None, periods_cap=None, out=None, timeline=False):
     """Section 4.2 tensor vitality analysis.  Returns tensors in the memory space of `tb`; in device mode the
     call is asynchronous on `stream` (trim `uses` / the period arrays with counts after synchronising).
-    `out`: the result of an earlier call on a trace of the same sizes, to write into instead of allocating."""
+    `out`: the result of an earlier call on a trace of the same sizes, to write into instead of allocating.
+    timeline=True (device traces): the same call also produces the Section 4.3 pressure timeline, returned as
+    `.timeline` (the fields of g10_pressure_timeline); pass an earlier such result as `timeline` to write into it."""
     lib = load_library()
     ucap = tb.E if uses_cap is None else uses_cap
     pcap = tb.E if periods_cap is None else periods_cap
@@ -249,10 +252,18 @@ def g10_vitality(tb: TraceBuffers, ws=None, stream=None, device=None, uses_cap=N
         uses=_alloc(tb, max(ucap, 1), torch.int32, device), period_ptr=_alloc(tb, tb.N + 1, torch.int64, device),
         period_tensor=_alloc(tb, max(pcap, 1), torch.int32, device), period_prev_use=_alloc(tb, max(pcap, 1), torch.int32, device),
         period_next_use=_alloc(tb, max(pcap, 1), torch.int32, device), counts=_alloc(tb, 3, torch.int64, device))
-    ws, ws_bytes = _workspace(tb, WS_VITALITY, ws, device)
+    to = None
+    if timeline:
+        t = timeline if not isinstance(timeline, bool) else SimpleNamespace(
+            kernel_start_ns=_alloc(tb, tb.K + 1, torch.int64, device), pressure=_alloc(tb, max(tb.K, 1), torch.int64, device),
+            peak_bytes=_alloc(tb, 1, torch.int64, device), peak_slot=_alloc(tb, 1, torch.int32, device),
+            status=_alloc(tb, 1, torch.int64, device))
+        to = _TimelineOut(_ptr(t.kernel_start_ns), _ptr(t.pressure), _ptr(t.peak_bytes), _ptr(t.peak_slot), _ptr(t.status), None, None)
+        r.timeline = t
+    ws, ws_bytes = _workspace(tb, WS_ANALYSIS if timeline else WS_VITALITY, ws, device)
     vo = _VitalityOut(_ptr(r.first_use), _ptr(r.last_use), _ptr(r.num_uses), _ptr(r.use_ptr), _ptr(r.uses), ucap,
                        _ptr(r.period_ptr), _ptr(r.period_tensor), _ptr(r.period_prev_use), _ptr(r.period_next_use), pcap,
-                       _ptr(r.counts))
+                       _ptr(r.counts), C.pointer(to) if to is not None else None)
     tr = tb.c_struct()
     _check(lib.g10_vitality(C.byref(tr), C.byref(vo), _ptr(ws), ws_bytes, _stream(stream)))
     r.workspace = ws

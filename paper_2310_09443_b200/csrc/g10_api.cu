@@ -44,7 +44,8 @@ size_t carve(void *base, const Sizes &z, Workspace &w, int32_t which)
 {
     std::memset(&w, 0, sizeof(w));
     Carver c(base);
-    const bool vit = which != G10_WS_TIMELINE, tl = which != G10_WS_VITALITY, plan = which != G10_WS_TIMELINE && which != G10_WS_VITALITY;
+    const bool vit = which != G10_WS_TIMELINE, tl = which != G10_WS_VITALITY;
+    const bool plan = which != G10_WS_TIMELINE && which != G10_WS_VITALITY && which != G10_WS_ANALYSIS;
     const bool inner = plan || z.host;             // results of the analysis calls kept inside the workspace
     const size_t K = (size_t)z.K, N = (size_t)z.N, E = (size_t)z.E;
     const size_t heavy = E / (kHeavyThreshold + 1) + 1;
@@ -80,7 +81,7 @@ size_t carve(void *base, const Sizes &z, Workspace &w, int32_t which)
         w.tl_point = c.take<int64_t>(K);
     } else {
         w.diff = c.take<int64_t>(tl ? K + 1 : 1);
-        w.tl_point = c.take<int64_t>(1);
+        w.tl_point = c.take<int64_t>(which == G10_WS_ANALYSIS ? K : 1);   // (right behind the difference array: one memset)
         w.tl_pair = c.take<int>(1);
     }
     w.cnt = c.take<int32_t>(vit ? N : 1);
@@ -176,7 +177,7 @@ int32_t check_ws(int32_t which, const g10_trace *t, void *ws, size_t ws_bytes)
     } while (0)
 
 // Prepares the workspace and returns the device view of the trace (staging it first in host mode).
-enum { kZeroCounts = 1, kZeroDiff = 2, kZeroState = 4, kZeroPairs = 8 };
+enum { kZeroCounts = 1, kZeroDiff = 2, kZeroState = 4, kZeroPairs = 8, kZeroDiffPoint = 16 };
 
 int32_t begin_call(int32_t which, const g10_trace *t, void *ws, Workspace &w, DeviceTrace &d, cudaStream_t s, int zero_mask)
 {
@@ -186,6 +187,7 @@ int32_t begin_call(int32_t which, const g10_trace *t, void *ws, Workspace &w, De
         size_t head = w.zero_bytes;
         if (zero_mask & kZeroDiff) head = (size_t)((char *)(w.diff + z.K + 1) - w.zero_begin);
         if (zero_mask & kZeroPairs) head = (size_t)((char *)(w.tl_pair + 2 * z.N) - w.zero_begin);
+        if (zero_mask & kZeroDiffPoint) head = (size_t)((char *)(w.tl_point + z.K) - w.zero_begin);
         CU(cudaMemsetAsync(w.zero_begin, 0, head, s));
     }
     if ((zero_mask & kZeroCounts) && z.N > 0) CU(cudaMemsetAsync(w.cnt, 0, sizeof(int32_t) * (size_t)z.N, s));
@@ -274,7 +276,7 @@ const char *g10_strerror(int32_t code)
 int32_t g10_workspace_bytes(int32_t which, int64_t K, int64_t N, int64_t E, int32_t mem, size_t *out_bytes)
 {
     if (!out_bytes || K < 0 || N < 0 || E < 0) return G10_ERR_ARG;
-    if (which < G10_WS_VITALITY || which > G10_WS_PREFETCH) return G10_ERR_ARG;
+    if (which < G10_WS_VITALITY || which > G10_WS_ANALYSIS) return G10_ERR_ARG;
     if (mem != G10_MEM_DEVICE && mem != G10_MEM_HOST) return G10_ERR_ARG;
     const int64_t lim = ((int64_t)1 << 31) - 1;
     if (K >= lim || N >= lim || E >= lim) return G10_ERR_LIMIT;
@@ -308,13 +310,19 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
     if ((out->uses_cap > 0 && !out->uses) ||
         (out->periods_cap > 0 && (!out->period_tensor || !out->period_prev_use || !out->period_next_use)))
         return G10_ERR_ARG;
-    rc = check_ws(G10_WS_VITALITY, trace, ws, ws_bytes);
+    g10_timeline_out *to = out->timeline;                  // the pressure timeline from the same call, if wanted
+    if (to) {
+        if (trace->mem != G10_MEM_DEVICE || to->first_use || to->last_use) return G10_ERR_ARG;
+        if (!to->kernel_start_ns || !to->peak_bytes || !to->peak_slot || !to->status || (trace->num_kernels > 0 && !to->pressure)) return G10_ERR_ARG;
+    }
+    const int32_t wsk = to ? G10_WS_ANALYSIS : G10_WS_VITALITY;
+    rc = check_ws(wsk, trace, ws, ws_bytes);
     if (rc != G10_OK) return rc;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w;
     DeviceTrace d;
     const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
-    rc = begin_call(G10_WS_VITALITY, trace, ws, w, d, s, buckets ? 0 : kZeroCounts);
+    rc = begin_call(wsk, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | (to ? kZeroDiffPoint : 0));
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     VitalityBuffers vb;
@@ -326,10 +334,17 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
         vb = VitalityBuffers{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, ucap, w.period_ptr,
                              w.period_tensor, w.period_prev_use, w.period_next_use, pcap, w.counts};
     }
-    if (buckets) CU(launch_vitality_buckets(d, w, vb, s, vb.counts + 2));     // (its last block publishes the status word)
+    if (to && buckets) {
+        // slot clock; beside it the vitality kernels, the last of which books the tensors' sizes; then the pressure scan alone
+        CU(launch_slot_clock(d, w, to->kernel_start_ns, s));
+        vb.tl_diff = (ull *)w.diff; vb.tl_point = (ull *)w.tl_point; vb.tl_bytes = d.tensor_bytes; vb.tl_glob = d.tensor_global; vb.tl_K = d.K;
+        CU(launch_vitality_buckets(d, w, vb, s, vb.counts + 2, true));
+        CU(launch_pressure_scan(d, w, w.tl_point, to->pressure, to->peak_bytes, to->peak_slot, to->status, s));
+    } else if (buckets) CU(launch_vitality_buckets(d, w, vb, s, vb.counts + 2));     // (its last block publishes the status word)
     else {
         CU(launch_vitality(d, w, vb, s));
         CU(launch_publish_status(w, vb.counts + 2, s));
+        if (to) CU(launch_timeline_given(d, w, to->kernel_start_ns, vb.first_use, vb.last_use, w.tl_point, to->pressure, to->peak_bytes, to->peak_slot, to->status, s));
     }
     if (host) {
         int64_t counts[3];

@@ -161,6 +161,13 @@ struct VitalityBuffers {
     int32_t *period_tensor, *period_prev_use, *period_next_use;
     int64_t periods_cap;
     int64_t *counts;   // [3]
+    // When the caller wants the pressure timeline from the same call (bucketed formulation only): the kernel that writes
+    // first / last use also books every tensor's size into the difference array [K + 1] and the point masses [K] (both
+    // cleared beforehand), so that only the scan is left to do.  All null otherwise.
+    ull *tl_diff = nullptr, *tl_point = nullptr;
+    const int64_t *tl_bytes = nullptr;
+    const uint8_t *tl_glob = nullptr;
+    int64_t tl_K = 0;
 };
 
 struct PlanParams {
@@ -183,7 +190,12 @@ cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const Vita
 // bucketed formulation (g10_vitality_buckets.cu); 4096 buckets of 4096 tensors per pass over the events, up to 16 passes
 bool vitality_buckets_supported(int64_t N, int64_t E);
 // (status_out, if not null, receives the device status word when the last block of the last kernel finishes)
-cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s, int64_t *status_out = nullptr);
+// (pdl_first: the first kernel may start while its predecessor in the stream, which has released its dependents, still runs)
+cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s, int64_t *status_out = nullptr,
+                                    bool pdl_first = false);
+// the pressure scan alone (difference array and point masses are complete when its predecessor in the stream is)
+cudaError_t launch_pressure_scan(const DeviceTrace &t, const Workspace &w, const int64_t *point, int64_t *pressure, int64_t *peak_bytes,
+                                 int32_t *peak_slot, int64_t *status_out, cudaStream_t s);
 cudaError_t launch_first_last(const DeviceTrace &t, const Workspace &w, int32_t *first_use, int32_t *last_use, cudaStream_t s);
 cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int32_t *first_use, const int32_t *last_use, bool encoded,
                             int64_t *pressure, int64_t *peak_bytes, int32_t *peak_slot, cudaStream_t s);

@@ -898,6 +898,23 @@ cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int6
                               w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out);
 }
 
+cudaError_t launch_pressure_scan(const DeviceTrace &t, const Workspace &w, const int64_t *point, int64_t *pressure, int64_t *peak_bytes,
+                                 int32_t *peak_slot, int64_t *status_out, cudaStream_t s)
+{
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
+    cfg.blockDim = dim3(kSegThreads);
+    return cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, point, pressure, w.pressure_scan.ticket,
+                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out);
+}
+
 // The timeline call when the caller hands first / last use over: slot clock, then (beside it) the bookings, then the scan.
 // The caller has cleared w.diff [K + 1] and point [K].
 cudaError_t launch_timeline_given(const DeviceTrace &t, const Workspace &w, int64_t *start, const int32_t *first_use, const int32_t *last_use,

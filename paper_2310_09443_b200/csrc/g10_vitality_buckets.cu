@@ -169,6 +169,8 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
     __syncthreads();
     for (int b = threadIdx.x; b < B.nb; b += kBkThreads)
         if (s_hist[b]) atomicAdd(&B.bucket_count[b], s_hist[b]);
+    // (when this kernel was allowed to start beside its predecessor in the stream: its completion must imply that one's)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -319,6 +321,8 @@ __device__ void bk_bitonic_sort_i32(int32_t *a, int n)    // arbitrary n: the ne
 __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
 
 
+// (kTimeline: the call also wants the pressure timeline; the outputs loop then books every tensor's size, see VitalityBuffers)
+template <bool kTimeline>
 __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBuffers out)
 {
     extern __shared__ __align__(16) int s_mem[];
@@ -341,6 +345,8 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         for (int b = threadIdx.x; b <= B.nb; b += kBkThreads) s_base[b] = 0;
         __syncthreads();
     }
+    long long tl_gsum = 0;                     // (timeline wanted too: bytes of the global tensors this thread met)
+    bool tl_bad = false;
     for (;;) {
         __syncthreads();
         // (the number is taken when the work starts, not earlier: a later bucket waits for the totals of all earlier
@@ -359,7 +365,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         // ---- raw events per tensor, segment offsets, scatter.  The first keys of the bucket stay in registers between the
         // counting and the scatter; the rest is read again (from L2).  Six per thread: with twelve -- every key of a usual
         // bucket -- the kernel needs more than the 64 registers that let two blocks share an SM, and spills.
-        constexpr int kRegKeys = 6;
+        constexpr int kRegKeys = kTimeline ? 4 : 6;          // (the bookings of the timeline form need registers of their own)
         ull rk[kRegKeys];
 #pragma unroll
         for (int q = 0; q < kRegKeys; ++q) {
@@ -526,11 +532,15 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         for (int tl0 = threadIdx.x; tl0 < bt_eff; tl0 += 2 * kBkThreads) {
             int d04[2], dd4[2], of4[2], np4[2];
             int32_t f4[2], l4[2];
+            long long bz4[2];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int tl = tl0 + q * kBkThreads;
-                d04[q] = 0; dd4[q] = -1; of4[q] = 0; np4[q] = 0;
-                if (tl < bt_eff) { d04[q] = t_d[tl]; dd4[q] = t_d[tl + 1] - d04[q]; of4[q] = t_off[tl]; np4[q] = t_np[tl]; }
+                d04[q] = 0; dd4[q] = -1; of4[q] = 0; np4[q] = 0; bz4[q] = 1;
+                if (tl < bt_eff) {
+                    d04[q] = t_d[tl]; dd4[q] = t_d[tl + 1] - d04[q]; of4[q] = t_off[tl]; np4[q] = t_np[tl];
+                    if (kTimeline) bz4[q] = out.tl_bytes[t0 + tl];
+                }
             }
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
@@ -549,6 +559,21 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
             out.num_uses[t] = dd;
             out.use_ptr[t] = U + d04[q];
             out.period_ptr[t] = PB + np4[q];
+            if (kTimeline) {
+                // the pressure timeline is wanted from the same call: the tensor's size is booked where it is born and where it dies
+                // (a tensor of one kernel in that slot's point mass; a global tensor in slot 0, summed per thread first)
+                const long long bsz = bz4[q];
+                if (bsz < 1 || bsz >= ((long long)1 << 40)) tl_bad = true;
+                if (dd > 0) {
+                    const int64_t f = f4[q], l = l4[q];
+                    if (out.tl_glob != nullptr && out.tl_glob[t]) tl_gsum += bsz;
+                    else if (f == l) atomicAdd(&out.tl_point[f], (ull)bsz);
+                    else {
+                        atomicAdd(&out.tl_diff[f], (ull)bsz);
+                        if (l + 1 < out.tl_K) atomicAdd(&out.tl_diff[l + 1], (ull)(-bsz));
+                    }
+                }
+            }
             long long uo = U + d04[q], po = PB + np4[q];
             for (int a = dense ? 1 : 0; a < dd; ++a) {
                 const int32_t x = seg[a];
@@ -571,6 +596,11 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
                 out.counts[0] = U + D; out.counts[1] = PB + PC;
             }
         }
+    }
+    if (kTimeline) {
+        if (tl_bad) raise_status(B.status, G10_DEV_BAD_BYTES);
+        tl_gsum = warp_sum_i64(tl_gsum);
+        if (lane == 0 && tl_gsum != 0) atomicAdd(&out.tl_diff[0], (ull)tl_gsum);
     }
     // the last block out, on the last pass, hands the status word over (every block's bits are in: acquire-release count)
     if (threadIdx.x == 0 && B.last_pass && B.status_out != nullptr) {
@@ -604,7 +634,7 @@ bool vitality_buckets_supported(int64_t N, int64_t E)
 }
 
 // One pass: the three kernels for tensors [B.t_begin, B.t_begin + B.N).
-static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const VitalityBuffers &out, int sms, bool multi, cudaStream_t s)
+static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const VitalityBuffers &out, int sms, bool multi, bool pdl_first, cudaStream_t s)
 {
     const int64_t tiles = (t.E + kBkTile - 1) / kBkTile;
     // the second and third kernel are launched with programmatic stream serialisation (they wait for their
@@ -619,9 +649,16 @@ static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const 
     cfg.numAttrs = 1;
     if (t.E > 0 && t.K > 0) {
         const int g = (int)(tiles < 2 * (int64_t)sms ? tiles : 2 * (int64_t)sms);
-        if (multi) k_bk_hist<true><<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
-        else k_bk_hist<false><<<g, kBkThreads, sizeof(unsigned) * (size_t)B.nb, s>>>(B, t.kernel_ptr, t.kernel_tensors);
-        count_launch();
+        {
+            cudaLaunchConfig_t c1 = cfg;
+            c1.gridDim = dim3((unsigned)g);
+            c1.dynamicSmemBytes = sizeof(unsigned) * (size_t)B.nb;
+            c1.numAttrs = pdl_first ? 1 : 0;
+            const int64_t *kp = t.kernel_ptr;
+            const int32_t *kt = t.kernel_tensors;
+            const cudaError_t e1 = multi ? cudaLaunchKernelEx(&c1, k_bk_hist<true>, B, kp, kt) : cudaLaunchKernelEx(&c1, k_bk_hist<false>, B, kp, kt);
+            if (e1 != cudaSuccess) return e1;
+        }
         // Shared memory of the partition kernel: three bucket tables and ten bytes per staged event; two blocks per SM.
         const size_t tables = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8;
         int64_t cap = ((int64_t)(100 << 10) - (int64_t)tables) / 10 / kBkThreads * kBkThreads;
@@ -651,16 +688,19 @@ static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const 
         if (e != cudaSuccess) return e;
     }
     const size_t sm3 = sizeof(int) * (size_t)(bk_pad(B.nb) + 3 * bk_pad(B.bt) + kBkCap) + sizeof(unsigned short) * (size_t)B.bt;
-    cudaError_t e = cudaFuncSetAttribute(k_bk_emit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
+    const bool fused = out.tl_diff != nullptr;
+    cudaError_t e = fused ? cudaFuncSetAttribute(k_bk_emit<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3)
+                          : cudaFuncSetAttribute(k_bk_emit<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
     const int g3 = B.nb < 2 * sms ? B.nb : 2 * sms;
     cfg.gridDim = dim3((unsigned)g3);
     cfg.dynamicSmemBytes = sm3;
-    if ((e = cudaLaunchKernelEx(&cfg, k_bk_emit, B, out)) != cudaSuccess) return e;
+    e = fused ? cudaLaunchKernelEx(&cfg, k_bk_emit<true>, B, out) : cudaLaunchKernelEx(&cfg, k_bk_emit<false>, B, out);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
-cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s, int64_t *status_out)
+cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s, int64_t *status_out, bool pdl_first)
 {
     if (!vitality_buckets_supported(t.N, t.E)) return cudaErrorInvalidValue;
     const int sms = current_sm_count();
@@ -687,7 +727,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
             if ((e = cudaMemsetAsync(w.bk_words, 0, sizeof(ull) * 2 * 4096, s)) != cudaSuccess) return e;
             if ((e = cudaMemsetAsync(w.emit_scan.ticket, 0, sizeof(unsigned), s)) != cudaSuccess) return e;
         }
-        const cudaError_t e = launch_bucket_pass(B, t, out, sms, passes > 1, s);
+        const cudaError_t e = launch_bucket_pass(B, t, out, sms, passes > 1, pdl_first && p == 0, s);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

@@ -56,7 +56,7 @@ def test_traffic_constants_carry_the_hash_of_the_sources_they_were_captured_on()
 
     now = bench.kernel_sources_sha256()
     assert len(now) == 64 and int(now, 16) >= 0
-    assert set(bench.TRAFFIC) == {"vitality", "timeline", "timeline_given", "captured_at", "sources_sha256"}
+    assert set(bench.TRAFFIC) == {"vitality", "timeline", "timeline_given", "fused", "captured_at", "sources_sha256"}
     assert len(bench.TRAFFIC["sources_sha256"]) == 64, "the traffic constants carry no source hash"
     assert bench.TRAFFIC["vitality"] > 0 and bench.TRAFFIC["timeline"] > 0
     if now != bench.TRAFFIC["sources_sha256"]:

@@ -58,6 +58,19 @@ def check_timeline(gpu, oracle, tr, tb):
     assert int(tg.status.item()) == 0
     assert np.array_equal(_np(tg.kernel_start_ns)[:tr.K + 1], start) and np.array_equal(_np(tg.pressure)[:tr.K], P0)
     assert int(tg.peak_bytes.item()) == peak and int(tg.peak_slot.item()) == slot
+    # ... and both analyses from one call (the vitality kernels book the sizes on their way)
+    vf = gpu.g10_vitality(tb, timeline=True)
+    torch.cuda.synchronize()
+    tf = vf.timeline
+    assert int(tf.status.item()) == 0 and _np(vf.counts).tolist() == _np(v.counts).tolist()
+    for name, cnt in (("first_use", tr.N), ("last_use", tr.N), ("num_uses", tr.N), ("use_ptr", tr.N + 1), ("period_ptr", tr.N + 1)):
+        assert np.array_equal(_np(getattr(vf, name))[:cnt], _np(getattr(v, name))[:cnt]), name
+    nu, npd = int(_np(v.counts)[0]), int(_np(v.counts)[1])
+    assert np.array_equal(_np(vf.uses)[:nu], _np(v.uses)[:nu])
+    for name in ("period_tensor", "period_prev_use", "period_next_use"):
+        assert np.array_equal(_np(getattr(vf, name))[:npd], _np(getattr(v, name))[:npd]), name
+    assert np.array_equal(_np(tf.kernel_start_ns)[:tr.K + 1], start) and np.array_equal(_np(tf.pressure)[:tr.K], P0)
+    assert int(tf.peak_bytes.item()) == peak and int(tf.peak_slot.item()) == slot
     return tl, (start, P0, peak, slot)
 
 
@@ -303,6 +316,11 @@ def test_bad_trace_sets_status_bits(gpu):
     assert _np(v.counts)[2] & 0x1
     st = int(tl.status.item())
     assert (st & 0x1) and (st & 0x8) and (st & 0x4)
+    vf = gpu.g10_vitality(tb, timeline=True)                 # both analyses from one call: the same bits in both status words
+    torch.cuda.synchronize()
+    for word in (int(vf.timeline.status.item()), int(_np(vf.counts)[2])):
+        assert (word & 0x1) and (word & 0x8) and (word & 0x4)
+    assert np.array_equal(_np(vf.timeline.pressure), _np(tl.pressure)) and np.array_equal(_np(vf.first_use), _np(v.first_use))
     # first / last use handed over but wrong (last before first, last beyond the trace): flagged, skipped, in bounds
     good = traces.config0_mlp_chain()
     tbg = gpu.upload(good)
