@@ -322,7 +322,8 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
     Workspace w;
     DeviceTrace d;
     const bool buckets = vitality_buckets_supported(trace->num_tensors, trace->num_events);
-    rc = begin_call(wsk, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | (to ? kZeroDiffPoint : 0));
+    // (bucketed formulation with the timeline: its counting kernel clears the difference array and the point masses itself)
+    rc = begin_call(wsk, trace, ws, w, d, s, (buckets ? 0 : kZeroCounts) | (to && !buckets ? kZeroDiffPoint : 0));
     if (rc != G10_OK) return rc;
     const bool host = trace->mem == G10_MEM_HOST;
     VitalityBuffers vb;

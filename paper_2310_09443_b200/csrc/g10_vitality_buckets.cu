@@ -47,6 +47,8 @@ struct BucketArgs {
     ull *words;                // [2 * nb] tagged totals of each bucket: distinct uses, periods
     int32_t *spill;            // [E] per-tensor segments of buckets too large for shared memory
     unsigned *ticket;
+    int64_t *zero_diff, *zero_point;   // timeline wanted from the same call: difference array [K + 1] and point masses [K] that
+                                       // the counting kernel of the first pass clears on its way (nullptr: nothing to clear)
     unsigned *done;            // blocks of the last kernel that have finished (starts at zero)
     int64_t *status_out;       // receives the status word when the last of them finishes the last pass (nullptr: nobody asked)
     ull *status;
@@ -136,6 +138,11 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
 {
     extern __shared__ unsigned s_hist[];
     for (int b = threadIdx.x; b < B.nb; b += kBkThreads) s_hist[b] = 0;
+    if (B.zero_diff != nullptr)
+        for (int64_t k = (int64_t)blockIdx.x * kBkThreads + threadIdx.x; k <= B.K; k += (int64_t)gridDim.x * kBkThreads) {
+            B.zero_diff[k] = 0;
+            if (k < B.K) B.zero_point[k] = 0;
+        }
     __syncthreads();
     ull bad = 0;
     // the partition walks the events kernel by kernel: kernel_ptr has to be a monotone map onto [0, E]
@@ -720,6 +727,15 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         if (!choose_buckets(B.N, e_share, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
         B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
         B.ticket = w.emit_scan.ticket; B.done = w.emit_scan.done; B.status_out = status_out; B.status = w.status; B.spill = w.raw_uses;
+        B.zero_diff = nullptr; B.zero_point = nullptr;
+        if (p == 0 && out.tl_diff != nullptr) {
+            if (t.E > 0 && t.K > 0) { B.zero_diff = (int64_t *)out.tl_diff; B.zero_point = (int64_t *)out.tl_point; }
+            else {                                     // (no counting kernel will run: clear them here)
+                cudaError_t e0;
+                if ((e0 = cudaMemsetAsync(out.tl_diff, 0, sizeof(int64_t) * (size_t)(t.K + 1), s)) != cudaSuccess) return e0;
+                if (t.K > 0 && (e0 = cudaMemsetAsync(out.tl_point, 0, sizeof(int64_t) * (size_t)t.K, s)) != cudaSuccess) return e0;
+            }
+        }
         if (p > 0) {                                   // what the call's opening memset cleared for the first pass
             cudaError_t e;
             if ((e = cudaMemsetAsync(w.bk_count, 0, sizeof(unsigned) * 4096, s)) != cudaSuccess) return e;
