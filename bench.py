@@ -2,8 +2,8 @@
 """Benchmark of the G10 planning path on B200.
 
 Headline (`value`): trace events per second through the analysis passes S1-S3 -- slot clock, tensor vitality
-and pressure timeline, i.e. one g10_vitality call plus one g10_pressure_timeline call -- on the 1M-kernel /
-4M-tensor stress trace (config 4), the largest single-GPU workload and the only one whose arrays are large enough
+and pressure timeline, i.e. one g10_vitality call with its timeline output (the e2e leg: one g10_vitality plus one
+g10_pressure_timeline call through host pointers) -- on the 1M-kernel / 4M-tensor stress trace (config 4), the largest single-GPU workload and the only one whose arrays are large enough
 for an HBM fraction to mean something.  A step is one such pass with the trace resident in HBM; the L2 is flushed
 between steps.  Second headline (`plan_ms`): one whole g10_plan_migrations call (S1-S7) on the ResNet-152-shaped
 trace (config 1).  The same line carries the plan of every configuration (`plans`), the two analysis calls on a
@@ -536,7 +536,7 @@ def run_ours(args):
         "metric": "trace_events_per_s", "value": value, "unit": "events/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "step": "S1-S3: one g10_vitality call + one g10_pressure_timeline call, trace resident in HBM",
+        "config": {"workload": WORKLOAD, "step": "S1-S3: one g10_vitality call with its timeline output (uses, periods, slot clock, pressure, peak), trace resident in HBM",
                    "trace_sha256": tr.sha256(), "K": K, "N": N, "E": E, "uses": uses, "periods": periods,
                    "l2": "flushed between timed iterations (%d MiB write)" % (L2_FLUSH_BYTES >> 20),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
