@@ -97,8 +97,8 @@ typedef struct g10_vitality_out {
     int32_t *period_tensor, *period_prev_use, *period_next_use;   /* [periods_cap] (E always suffices) */
     int64_t periods_cap;
     int64_t *counts;                            /* [3]: number of uses E', number of periods Pn, device status word */
-    /* Optional (NULL = no): the memory-pressure timeline of the same trace from the same call (device traces
-       only; workspace G10_WS_ANALYSIS).  The kernel that writes first / last use books every tensor's size
+    /* Optional (NULL = no): the memory-pressure timeline of the same trace from the same call (workspace
+       G10_WS_ANALYSIS; with a host trace the trace is staged once for both).  The kernel that writes first / last use books every tensor's size
        on the way, so that S1 - S3 walk the events once and only the slot clock and the pressure scan are
        left.  Its first_use / last_use inputs must be NULL; its outputs and status word are those of
        g10_pressure_timeline. */

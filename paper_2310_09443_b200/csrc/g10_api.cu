@@ -312,7 +312,7 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
         return G10_ERR_ARG;
     g10_timeline_out *to = out->timeline;                  // the pressure timeline from the same call, if wanted
     if (to) {
-        if (trace->mem != G10_MEM_DEVICE || to->first_use || to->last_use) return G10_ERR_ARG;
+        if (to->first_use || to->last_use) return G10_ERR_ARG;
         if (!to->kernel_start_ns || !to->peak_bytes || !to->peak_slot || !to->status || (trace->num_kernels > 0 && !to->pressure)) return G10_ERR_ARG;
     }
     const int32_t wsk = to ? G10_WS_ANALYSIS : G10_WS_VITALITY;
@@ -335,17 +335,21 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
         vb = VitalityBuffers{w.first_use, w.last_use, w.num_uses, w.use_ptr, w.uses, ucap, w.period_ptr,
                              w.period_tensor, w.period_prev_use, w.period_next_use, pcap, w.counts};
     }
+    // (host traces: the timeline's results stay in the workspace too and are copied out below)
+    int64_t *tl_start = to ? (host ? w.start : to->kernel_start_ns) : nullptr, *tl_P = to ? (host ? w.pressure : to->pressure) : nullptr;
+    int64_t *tl_pk = to ? (host ? w.peak_bytes : to->peak_bytes) : nullptr, *tl_st = to ? (host ? w.counts + 3 : to->status) : nullptr;
+    int32_t *tl_ps = to ? (host ? w.peak_slot : to->peak_slot) : nullptr;
     if (to && buckets) {
         // slot clock; beside it the vitality kernels, the last of which books the tensors' sizes; then the pressure scan alone
-        CU(launch_slot_clock(d, w, to->kernel_start_ns, s));
+        CU(launch_slot_clock(d, w, tl_start, s));
         vb.tl_diff = (ull *)w.diff; vb.tl_point = (ull *)w.tl_point; vb.tl_bytes = d.tensor_bytes; vb.tl_glob = d.tensor_global; vb.tl_K = d.K;
         CU(launch_vitality_buckets(d, w, vb, s, vb.counts + 2, true));
-        CU(launch_pressure_scan(d, w, w.tl_point, to->pressure, to->peak_bytes, to->peak_slot, to->status, s));
+        CU(launch_pressure_scan(d, w, w.tl_point, tl_P, tl_pk, tl_ps, tl_st, s));
     } else if (buckets) CU(launch_vitality_buckets(d, w, vb, s, vb.counts + 2));     // (its last block publishes the status word)
     else {
         CU(launch_vitality(d, w, vb, s));
         CU(launch_publish_status(w, vb.counts + 2, s));
-        if (to) CU(launch_timeline_given(d, w, to->kernel_start_ns, vb.first_use, vb.last_use, w.tl_point, to->pressure, to->peak_bytes, to->peak_slot, to->status, s));
+        if (to) CU(launch_timeline_given(d, w, tl_start, vb.first_use, vb.last_use, w.tl_point, tl_P, tl_pk, tl_ps, tl_st, s));
     }
     if (host) {
         int64_t counts[3];
@@ -364,6 +368,13 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
         CU(d2h(out->period_tensor, w.period_tensor, np, s));
         CU(d2h(out->period_prev_use, w.period_prev_use, np, s));
         CU(d2h(out->period_next_use, w.period_next_use, np, s));
+        if (to) {
+            CU(d2h(to->kernel_start_ns, w.start, (size_t)d.K + 1, s));
+            CU(d2h(to->pressure, w.pressure, (size_t)d.K, s));
+            CU(d2h(to->peak_bytes, w.peak_bytes, 1, s));
+            CU(d2h(to->peak_slot, w.peak_slot, 1, s));
+            CU(d2h(to->status, w.counts + 3, 1, s));
+        }
         CU(cudaStreamSynchronize(s));
     }
     return G10_OK;

@@ -376,6 +376,13 @@ def test_host_pointer_mode(gpu, oracle):
     start, P0, peak, slot = oracle.timeline(tr)
     assert np.array_equal(tl.pressure.numpy(), P0) and int(tl.peak_bytes) == peak and int(tl.peak_slot) == slot
     assert np.array_equal(tl.kernel_start_ns.numpy(), start)
+    vf = gpu.g10_vitality(tb, timeline=True)                 # both analyses from one call: the trace is staged once
+    assert int(vf.counts[2]) == 0 and int(vf.timeline.status) == 0
+    for name, n in (("first_use", None), ("last_use", None), ("num_uses", None), ("use_ptr", None), ("period_ptr", None),
+                    ("uses", e2), ("period_tensor", pn), ("period_prev_use", pn), ("period_next_use", pn)):
+        assert np.array_equal(getattr(vf, name).numpy()[:n], getattr(ov, name)), name
+    assert np.array_equal(vf.timeline.pressure.numpy(), P0) and int(vf.timeline.peak_bytes) == peak and int(vf.timeline.peak_slot) == slot
+    assert np.array_equal(vf.timeline.kernel_start_ns.numpy(), start)
     ref = oracle.plan(tr, tr.capacity_from_peak(peak))
     plan = gpu.g10_plan_migrations(tb, tr.capacity_from_peak(int(tl.peak_bytes)), tr.host_bw, tr.ssd_bw)
     assert np.array_equal(plan.summary.numpy()[:7], ref.summary[:7]) and int(plan.summary[7]) == 0
