@@ -16,6 +16,11 @@
  *     no device memory, keeps no state between calls and frees nothing.  The workspace `ws` is ALWAYS
  *     device memory, 256-byte aligned, of at least g10_workspace_bytes(...) bytes; its contents are
  *     scratch.  Two calls may run concurrently only on different workspaces.
+ *   - Stream capture: a G10_MEM_DEVICE call of g10_vitality, g10_pressure_timeline, g10_candidate_geometry,
+ *     g10_characterize or g10_emit_instructions enqueues only kernels and memsets (with programmatic
+ *     dependencies between them) and may be captured in a CUDA graph, after one ordinary call of the same
+ *     entry point (which sets kernel attributes).  The planner calls launch cooperative kernels and
+ *     g10_plan_batch may synchronise: they are not meant for capture.
  *   - Errors: the return value is 0 (enqueued) or a negative G10_ERR_* found on the host before any
  *     launch.  Errors that depend on the data (tensor id out of range, non-monotone kernel_ptr,
  *     sizes or durations outside their limits, an output array too small, a grid barrier that timed

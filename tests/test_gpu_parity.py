@@ -872,3 +872,34 @@ def test_crowded_ties_and_conflicts(gpu, oracle):
         for flags in (0, gpu.FLAG_GLOBAL_STATE, gpu.FLAG_MULTI_BLOCK, gpu.FLAG_RESCORE_ALL):
             check_plan(gpu, tr, tb, cap, ref, flags=flags)
         check_cyclic(gpu, oracle, tr, cap)
+
+
+@pytest.mark.gpu
+def test_analysis_call_in_a_cuda_graph(gpu, oracle):
+    """The device-mode calls only enqueue work on the caller's stream (kernels, memsets; programmatic dependencies between
+    them): they can be captured in a CUDA graph and replayed.  The one-call analysis of config 1, captured once, replayed
+    three times into cleared outputs, against the oracle."""
+    import torch
+    tr = traces.config1_resnet152()
+    tb = gpu.upload(tr)
+    ws = torch.empty(gpu.g10_workspace_bytes(gpu.WS_ANALYSIS, tb.K, tb.N, tb.E), dtype=torch.uint8, device="cuda")
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        v = gpu.g10_vitality(tb, ws=ws, timeline=True, stream=s)             # (first call outside the capture: attributes get set)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            gpu.g10_vitality(tb, ws=ws, out=v, timeline=v.timeline, stream=torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+    start, P0, peak, slot = oracle.timeline(tr)
+    for _ in range(3):
+        for t in (v.first_use, v.last_use, v.period_tensor, v.timeline.pressure, v.counts, v.timeline.peak_bytes):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        pn = int(v.counts[1].item())
+        assert int(v.counts[2].item()) == 0 and int(v.timeline.status.item()) == 0 and pn == len(ov.period_tensor)
+        assert np.array_equal(_np(v.first_use), ov.first_use) and np.array_equal(_np(v.last_use), ov.last_use)
+        assert np.array_equal(_np(v.period_tensor)[:pn], ov.period_tensor)
+        assert np.array_equal(_np(v.timeline.pressure)[:tr.K], P0) and int(v.timeline.peak_bytes.item()) == peak
