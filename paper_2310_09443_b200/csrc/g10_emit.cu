@@ -248,18 +248,32 @@ __global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int6
                     s_pay[slot] = ((rk[q] >> 31) & 1u) ? gp[j] : -1;       // (PRE_EVICT = 1 and PREFETCH = 3 come from a plan record)
                 }
             __syncthreads();
-            for (int bd = threadIdx.x; bd < bw_eff; bd += kEmitThreads) {
-                const int o = s_cnt[bd], m = s_cnt[bd + 1] - o;
-                if (m > kEmitWide) { const int q = atomicAdd(&s_nwide, 1); if (q < 64) s_wide[q] = bd; }
-                else {
-                    for (int a = 1; a < m; ++a) {
-                        const ull x = s_keys[o + a];
-                        const int32_t px = s_pay[o + a];
-                        int c = a - 1;
-                        while (c >= 0 && s_keys[o + c] > x) { s_keys[o + c + 1] = s_keys[o + c]; s_pay[o + c + 1] = s_pay[o + c]; --c; }
-                        s_keys[o + c + 1] = x; s_pay[o + c + 1] = px;
+            // Inside a boundary the keys go in key order.  Every thread takes back the instructions at its slots, finds for
+            // each its rank among the instructions of its boundary by counting the smaller keys (a boundary holds a handful;
+            // keys are unique, so ranks are too), and puts it where it belongs.  One thread sorting one boundary, as before,
+            // makes the whole block wait for the boundary with the most instructions.
+            {
+                ull ik[kEmitRegs];
+                int ip[kEmitRegs], dst[kEmitRegs];
+#pragma unroll
+                for (int q = 0; q < kEmitRegs; ++q) {
+                    const int j = q * kEmitThreads + threadIdx.x;
+                    dst[q] = -1;
+                    if (j < n) {
+                        ik[q] = s_keys[j]; ip[q] = s_pay[j];
+                        const int bd = (int)((ik[q] >> 33) - b0);
+                        const int o = s_cnt[bd], m = s_cnt[bd + 1] - o;
+                        if (m <= kEmitWide) {
+                            int r = 0;
+                            for (int a = 0; a < m; ++a) r += s_keys[o + a] < ik[q] ? 1 : 0;
+                            dst[q] = o + r;
+                        } else if (j == o) { const int w2 = atomicAdd(&s_nwide, 1); if (w2 < 64) s_wide[w2] = bd; }   // (its first slot reports it)
                     }
                 }
+                __syncthreads();
+#pragma unroll
+                for (int q = 0; q < kEmitRegs; ++q)
+                    if (dst[q] >= 0) { s_keys[dst[q]] = ik[q]; s_pay[dst[q]] = ip[q]; }
             }
             __syncthreads();
             const int nwide = s_nwide;
