@@ -185,7 +185,7 @@ constexpr int kSmallMaxBlocks = 160;       // blocks of the small-trace planner 
 constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock fit in shared memory
 
 // passes (g10_passes.cu)
-cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s);
+cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s, bool check_kernel_ptr = true);
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 // bucketed formulation (g10_vitality_buckets.cu); 4096 buckets of 4096 tensors per pass over the events, up to 16 passes
 bool vitality_buckets_supported(int64_t N, int64_t E);

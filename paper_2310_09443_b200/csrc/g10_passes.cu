@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
         for (int j = 0; j < 4; ++j) {                      // all loads of the batch in flight together
             const int64_t k = k0 + (int64_t)j * kSegThreads;
             v[j] = k < hi ? in[k] : (kind == 0 ? 1 : 0);
-            if (kind == 0) { p0[j] = k < hi ? kptr[k] : 0; p1[j] = k < hi ? kptr[k + 1] : 0; }
+            if (kind == 0 && kptr != nullptr) { p0[j] = k < hi ? kptr[k] : 0; p1[j] = k < hi ? kptr[k + 1] : 0; }
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
             if (k < hi) {
                 if (kind == 0) {
                     if (v[j] < 1 || v[j] >= ((long long)1 << 44)) { bad |= G10_DEV_BAD_DURATION; v[j] = 1; }
-                    if (p0[j] > p1[j] || p0[j] < 0 || p1[j] > E || (k == 0 && p0[j] != 0) || (k == n - 1 && p1[j] != E))
+                    if (kptr != nullptr && (p0[j] > p1[j] || p0[j] < 0 || p1[j] > E || (k == 0 && p0[j] != 0) || (k == n - 1 && p1[j] != E)))
                         bad |= G10_DEV_BAD_KERNEL_PTR;
                 }
                 sum += v[j];
@@ -222,10 +222,11 @@ static int seg_scan_blocks(int64_t n)
     return g < 1 ? 1 : (int)g;
 }
 
-cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s)
+cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s, bool check_kernel_ptr)
 {
     const int G = seg_scan_blocks(t.K);
-    k_seg_scan<0><<<G, kSegThreads, 0, s>>>(t.K, t.E, t.kernel_ns, t.kernel_ptr, start, w.clock_scan.ticket, w.clock_scan.done,
+    // (check_kernel_ptr false: another kernel of the same call makes the same check of kernel_ptr; this one then reads a third)
+    k_seg_scan<0><<<G, kSegThreads, 0, s>>>(t.K, t.E, t.kernel_ns, check_kernel_ptr ? t.kernel_ptr : nullptr, start, w.clock_scan.ticket, w.clock_scan.done,
                                           w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status, nullptr); count_launch();
     return cudaGetLastError();
 }
