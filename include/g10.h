@@ -363,7 +363,8 @@ int32_t g10_characterize(int64_t num_kernels, int64_t num_tensors, const int64_t
    It takes no workspace: its scratch is a fixed 1.5 MiB array inside the library image, present on every GPU
    that loads the library until the process exits.  Consequences the caller must know:
      - device pointers only (trace->mem must be G10_MEM_DEVICE); same outputs, same device status word and the
-       same stream semantics as g10_pressure_timeline;
+       same stream semantics as g10_pressure_timeline (the optional first_use / last_use inputs of the output
+       struct are not looked at: first and last use always come from the trace);
      - traces up to G10_STATIC_MAX_KERNELS kernels and G10_STATIC_MAX_TENSORS tensors; anything larger is
        refused with G10_ERR_LIMIT before any work is enqueued;
      - the first call on each device looks the array's address up (cudaGetSymbolAddress, with that device
