@@ -117,35 +117,40 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
     if (lane == 0) s_w[warp] = pre;
     __syncthreads();
     long long carry = seg_warp_totals(s_w, lane, warp, &unused);
-    // ---- pass 2: scan the segment chunk by chunk (each thread kSegItems consecutive elements)
+    // ---- pass 2: scan the segment chunk by chunk.  A warp takes 32 * kSegItems consecutive elements as kSegItems rows of 32,
+    // lane l the l-th of each row: every load and store of a warp is one contiguous 256-byte run (a thread with kSegItems
+    // consecutive elements of its own would touch each 32-byte sector four times, and the stores reach the L2 one by one).
     long long mx = 0;
     int sl = -1;
     for (int64_t c0 = lo; c0 < hi; c0 += kSegChunk) {
-        const int64_t base = c0 + (int64_t)threadIdx.x * kSegItems;
-        long long v[kSegItems];
-        long long tsum = 0;
+        const int64_t base = c0 + (int64_t)warp * (32 * kSegItems) + lane;
+        long long v[kSegItems], inc[kSegItems], pt[kSegItems];
 #pragma unroll
         for (int j = 0; j < kSegItems; ++j) {
-            const int64_t k = base + j;
+            const int64_t k = base + j * 32;
             v[j] = k < hi ? in[k] : 0;
             if (kind == 0 && k < hi && (v[j] < 1 || v[j] >= ((long long)1 << 44))) v[j] = 1;
-            tsum += v[j];
+            pt[j] = (kind == 1 && kptr != nullptr && k < hi) ? kptr[k] : 0;   // (kind 1: kptr = bytes alive in slot k only, or null)
         }
-        const long long incl = warp_inclusive_scan_i64(tsum, lane);
+        long long rows = 0;                                // the rows before row j, then the warp's total
+#pragma unroll
+        for (int j = 0; j < kSegItems; ++j) {
+            inc[j] = warp_inclusive_scan_i64(v[j], lane) + rows;
+            rows = __shfl_sync(0xffffffffu, inc[j], 31);
+        }
         __syncthreads();                                   // s_w has been read by every warp
-        if (lane == 31) s_w[warp] = incl;
+        if (lane == 0) s_w[warp] = rows;
         __syncthreads();
         long long wpre;
         const long long ctot = seg_warp_totals(s_w, lane, warp, &wpre);
-        long long run = carry + wpre + incl - tsum;
+        const long long before = carry + wpre;
 #pragma unroll
         for (int j = 0; j < kSegItems; ++j) {
-            const int64_t k = base + j;
-            if (kind == 0) { if (k < hi) out[k] = run; run += v[j]; }
-            else {
-                run += v[j];
-                if (k < hi) {
-                    const long long p = kptr != nullptr ? run + kptr[k] : run;     // (kind 1: kptr = bytes alive in slot k only, or null)
+            const int64_t k = base + j * 32;
+            if (k < hi) {
+                if (kind == 0) out[k] = before + inc[j] - v[j];
+                else {
+                    const long long p = before + inc[j] + pt[j];
                     out[k] = p;
                     if (sl < 0 || p > mx) { mx = p; sl = (int)k; }
                 }

@@ -1,6 +1,6 @@
 // Tensor vitality (Section 4.2: born / dead / inactive periods) in three kernels that keep the random
-// accesses on chip.  Tensors are cut into buckets of `bt` consecutive ids (a power of two, chosen so that a
-// bucket holds a few thousand trace events):
+// accesses on chip.  Tensors are cut into buckets of `bt` consecutive ids (chosen so that a bucket holds a few
+// thousand trace events and the buckets come to whole rounds of the last kernel's grid):
 //   1. k_bk_hist     counts the events of every bucket (shared-memory histogram per block);
 //   2. k_bk_scatter  partitions the events by bucket: each event becomes one 64-bit key
 //                    (tensor id inside the bucket << 32 | kernel) written into its bucket's slice; the events are
@@ -36,7 +36,7 @@ struct BucketArgs {
     int last_pass;
     const long long *carry_in; // [2] distinct uses and periods of all tensors before the pass (nullptr: none)
     long long *carry_out;      // [2] the same after the pass
-    int shift;                 // log2(bt)
+    ull magic;                 // ceil(2^40 / bt): (x * magic) >> 40 == x / bt for every tensor number x of a pass (bk_bucket)
     int bt;                    // tensors per bucket
     int nb;                    // number of buckets
     int tile_kernels;          // kernels per partition tile (at most 32768)
@@ -53,6 +53,11 @@ struct BucketArgs {
     int64_t *status_out;       // receives the status word when the last of them finishes the last pass (nullptr: nobody asked)
     ull *status;
 };
+
+// Bucket of tensor number x (inside a pass: 0 <= x < 2^24) for buckets of bt tensors, 64 <= bt <= 4096, without a division:
+// with magic = ceil(2^40 / bt) the product x * magic / 2^40 exceeds x / bt by less than 2^-16, and x / bt is at least
+// 1 / bt >= 2^-12 short of the next integer.
+__device__ __forceinline__ int bk_bucket(int x, ull magic) { return (int)(((ull)(unsigned)x * magic) >> 40); }
 
 // Block-wide exclusive scans over at most kBkThreads * 8 = 4096 entries, eight consecutive entries per thread.
 // in[0..n) -> out[0..n), out[n] = total (in == out allowed).  NA = 1 or 2 arrays scanned together.
@@ -164,11 +169,11 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
             if (id[j] == -2) continue;
             if (!kMulti) {
                 if (id[j] < 0 || id[j] >= B.N) bad |= G10_DEV_BAD_TENSOR_ID;
-                else atomicAdd(&s_hist[id[j] >> B.shift], 1u);
+                else atomicAdd(&s_hist[bk_bucket(id[j], B.magic)], 1u);
             } else if (id[j] < 0 || id[j] >= B.N_total) { if (B.t_begin == 0) bad |= G10_DEV_BAD_TENSOR_ID; }
             else {
                 const int64_t rel = (int64_t)id[j] - B.t_begin;
-                if (rel >= 0 && rel < B.N) atomicAdd(&s_hist[rel >> B.shift], 1u);
+                if (rel >= 0 && rel < B.N) atomicAdd(&s_hist[bk_bucket((int)rel, B.magic)], 1u);
             }
         }
     }
@@ -255,11 +260,11 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_scatter(BucketArgs B, cons
             for (int j = 0; j < kPtMaxItems; ++j) {
                 rank[j] = 0;
                 if (!kMulti) {
-                    if (id[j] >= 0 && id[j] < B.N) rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1);
+                    if (id[j] >= 0 && id[j] < B.N) rank[j] = atomicAdd(&s_cnt[bk_bucket(id[j], B.magic)], 1);
                     else id[j] = -1;
                 } else {
                     const int64_t rel = (int64_t)id[j] - B.t_begin;          // (the tensor's number inside the pass from here on)
-                    if (id[j] >= 0 && rel >= 0 && rel < B.N) { id[j] = (int)rel; rank[j] = atomicAdd(&s_cnt[id[j] >> B.shift], 1); }
+                    if (id[j] >= 0 && rel >= 0 && rel < B.N) { id[j] = (int)rel; rank[j] = atomicAdd(&s_cnt[bk_bucket(id[j], B.magic)], 1); }
                     else id[j] = -1;
                 }
             }
@@ -283,9 +288,9 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_scatter(BucketArgs B, cons
             for (int j = 0; j < kPtMaxItems; ++j) {
                 if (id[j] >= 0) {
                     const int p = j * kBkThreads + threadIdx.x;
-                    const int b = id[j] >> B.shift;
+                    const int b = bk_bucket(id[j], B.magic);
                     const unsigned k = (unsigned)(tk0 + s_krel[p]);
-                    s_key[s_cnt[b] + rank[j]] = ((ull)(unsigned)b << 48) | ((ull)(unsigned)(id[j] & (B.bt - 1)) << 32) | k;
+                    s_key[s_cnt[b] + rank[j]] = ((ull)(unsigned)b << 48) | ((ull)(unsigned)(id[j] - b * B.bt) << 32) | k;
                 }
             }
             __syncthreads();
@@ -618,16 +623,27 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
 }
 
 // Picks the bucket width for (a pass over) N tensors with about E events; false if that is outside what the bucket path handles.
-static bool choose_buckets(int64_t N, int64_t E, int *shift, int *bt, int *nb)
+static bool choose_buckets(int64_t N, int64_t E, int sms, int *bt, int *nb, ull *magic)
 {
     if (N <= 0) return false;
     int64_t want = E > 0 ? (6000 * N) / E : 4096;        // tensors per bucket for about 4000-6000 events
     int s = 6;
     while (s < 12 && ((int64_t)1 << (s + 1)) <= want) ++s;
     while (s < 12 && ((N + ((int64_t)1 << s) - 1) >> s) > 4096) ++s;
-    const int64_t buckets = (N + ((int64_t)1 << s) - 1) >> s;
+    int64_t width = (int64_t)1 << s;
+    int64_t buckets = (N + width - 1) / width;
     if (buckets > 4096) return false;
-    *shift = s; *bt = 1 << s; *nb = (int)buckets;
+    // k_bk_emit takes the buckets one per block at a time with two blocks per SM, and what a bucket costs depends little on
+    // its width: when there are more buckets than blocks, somewhat narrower buckets that come to whole rounds of the grid
+    // finish sooner than a last round that a quarter of the blocks take part in.
+    const int64_t G = 2 * (int64_t)sms;
+    if (buckets > G) {
+        const int64_t target = (buckets + G - 1) / G * G;
+        const int64_t narrower = (N + target - 1) / target;
+        if (target <= 4096 && narrower >= 64) { width = narrower; buckets = (N + width - 1) / width; }
+    }
+    *bt = (int)width; *nb = (int)buckets;
+    *magic = (((ull)1 << 40) + (ull)width - 1) / (ull)width;
     return true;
 }
 
@@ -724,7 +740,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         B.carry_out = w.bk_carry + 2 * (p & 1);
         // (bucket width from the pass's share of the events, taken as proportional to its share of the tensors)
         const int64_t e_share = passes > 1 ? (int64_t)((double)t.E * (double)B.N / (double)t.N) : t.E;
-        if (!choose_buckets(B.N, e_share, &B.shift, &B.bt, &B.nb)) return cudaErrorInvalidValue;
+        if (!choose_buckets(B.N, e_share, sms, &B.bt, &B.nb, &B.magic)) return cudaErrorInvalidValue;
         B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
         B.ticket = w.emit_scan.ticket; B.done = w.emit_scan.done; B.status_out = status_out; B.status = w.status; B.spill = w.raw_uses;
         B.zero_diff = nullptr; B.zero_point = nullptr;
