@@ -341,7 +341,10 @@ int32_t g10_vitality(const g10_trace *trace, g10_vitality_out *out, void *ws, si
     int32_t *tl_ps = to ? (host ? w.peak_slot : to->peak_slot) : nullptr;
     if (to && buckets) {
         // slot clock; beside it the vitality kernels, the last of which books the tensors' sizes; then the pressure scan alone
-        CU(launch_slot_clock(d, w, tl_start, s, !(d.E > 0 && d.K > 0)));       // (k_bk_hist, which runs whenever there are events, checks kernel_ptr)
+        // (k_bk_hist, which runs whenever there are events, checks kernel_ptr; the slot clock, the lighter of the two, clears
+        // the difference array and the point masses for the bookings of k_bk_emit)
+        CU(launch_slot_clock(d, w, tl_start, s, !(d.E > 0 && d.K > 0), w.diff, w.tl_point));
+        vb.tl_cleared = true;
         vb.tl_diff = (ull *)w.diff; vb.tl_point = (ull *)w.tl_point; vb.tl_bytes = d.tensor_bytes; vb.tl_glob = d.tensor_global; vb.tl_K = d.K;
         CU(launch_vitality_buckets(d, w, vb, s, vb.counts + 2, true));
         CU(launch_pressure_scan(d, w, w.tl_point, tl_P, tl_pk, tl_ps, tl_st, s));

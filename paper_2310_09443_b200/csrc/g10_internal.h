@@ -165,6 +165,7 @@ struct VitalityBuffers {
     // first / last use also books every tensor's size into the difference array [K + 1] and the point masses [K] (both
     // cleared beforehand), so that only the scan is left to do.  All null otherwise.
     ull *tl_diff = nullptr, *tl_point = nullptr;
+    bool tl_cleared = false;     // tl_diff and tl_point have been cleared by an earlier kernel of the stream
     const int64_t *tl_bytes = nullptr;
     const uint8_t *tl_glob = nullptr;
     int64_t tl_K = 0;
@@ -185,7 +186,9 @@ constexpr int kSmallMaxBlocks = 160;       // blocks of the small-trace planner 
 constexpr int64_t kSmallMaxSlots = 12000;  // largest K whose pressure + clock fit in shared memory
 
 // passes (g10_passes.cu)
-cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s, bool check_kernel_ptr = true);
+// (zero_diff [K + 1], zero_point [K]: arrays the kernel clears on its way, for a later kernel of the same call)
+cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s, bool check_kernel_ptr = true,
+                              int64_t *zero_diff = nullptr, int64_t *zero_point = nullptr);
 cudaError_t launch_vitality(const DeviceTrace &t, const Workspace &w, const VitalityBuffers &out, cudaStream_t s);
 // bucketed formulation (g10_vitality_buckets.cu); 4096 buckets of 4096 tensors per pass over the events, up to 16 passes
 bool vitality_buckets_supported(int64_t N, int64_t E);

@@ -51,7 +51,7 @@ template <int kind>
 __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t E, const int64_t *__restrict__ in, const int64_t *__restrict__ kptr,
                                                              int64_t *__restrict__ out, unsigned *ticket, unsigned *done, ull *words,
                                                              int64_t *blk_max, int32_t *blk_slot, int64_t *peak_bytes, int32_t *peak_slot, ull *status,
-                                                             int64_t *status_out)
+                                                             int64_t *status_out, int64_t *zero_a = nullptr, int64_t *zero_b = nullptr)
 {
     __shared__ long long s_w[kSegWarps];
     __shared__ int s_sl[kSegWarps];
@@ -64,6 +64,13 @@ __global__ void __launch_bounds__(kSegThreads, 2) k_seg_scan(int64_t n, int64_t 
     // while the predecessor still runs)
     const int g = next_tile(ticket);
     if (kind != 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // (the difference array is complete; see k_diff_scatter)
+    // (kind 0, when the same call goes on to the pressure timeline: this kernel, the lighter of the two that open the call
+    // side by side, clears the difference array [n + 1] and the point masses [n] on its way)
+    if (kind == 0 && zero_a != nullptr)
+        for (int64_t k = (int64_t)blockIdx.x * kSegThreads + threadIdx.x; k <= n; k += (int64_t)G * kSegThreads) {
+            zero_a[k] = 0;
+            if (k < n) zero_b[k] = 0;
+        }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t seg = ((n + G - 1) / G + kSegChunk - 1) / kSegChunk * kSegChunk;
     const int64_t lo = (int64_t)g * seg, hi = lo + seg < n ? lo + seg : n;
@@ -227,12 +234,13 @@ static int seg_scan_blocks(int64_t n)
     return g < 1 ? 1 : (int)g;
 }
 
-cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s, bool check_kernel_ptr)
+cudaError_t launch_slot_clock(const DeviceTrace &t, const Workspace &w, int64_t *start, cudaStream_t s, bool check_kernel_ptr, int64_t *zero_diff,
+                              int64_t *zero_point)
 {
     const int G = seg_scan_blocks(t.K);
     // (check_kernel_ptr false: another kernel of the same call makes the same check of kernel_ptr; this one then reads a third)
     k_seg_scan<0><<<G, kSegThreads, 0, s>>>(t.K, t.E, t.kernel_ns, check_kernel_ptr ? t.kernel_ptr : nullptr, start, w.clock_scan.ticket, w.clock_scan.done,
-                                          w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status, nullptr); count_launch();
+                                          w.seg_words, nullptr, nullptr, nullptr, nullptr, w.status, nullptr, zero_diff, zero_point); count_launch();
     return cudaGetLastError();
 }
 
@@ -861,7 +869,7 @@ cudaError_t launch_pressure(const DeviceTrace &t, const Workspace &w, const int3
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);
     e = cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)nullptr, pressure, w.pressure_scan.ticket,
-                           w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, (int64_t *)nullptr);
+                           w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, (int64_t *)nullptr, (int64_t *)nullptr, (int64_t *)nullptr);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
@@ -901,7 +909,7 @@ cudaError_t launch_timeline_pairs(const DeviceTrace &t, const Workspace &w, int6
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);
     return cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)point, pressure, w.pressure_scan.ticket,
-                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out);
+                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out, (int64_t *)nullptr, (int64_t *)nullptr);
 }
 
 cudaError_t launch_pressure_scan(const DeviceTrace &t, const Workspace &w, const int64_t *point, int64_t *pressure, int64_t *peak_bytes,
@@ -918,7 +926,7 @@ cudaError_t launch_pressure_scan(const DeviceTrace &t, const Workspace &w, const
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);
     return cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, point, pressure, w.pressure_scan.ticket,
-                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out);
+                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out, (int64_t *)nullptr, (int64_t *)nullptr);
 }
 
 // The timeline call when the caller hands first / last use over: slot clock, then (beside it) the bookings, then the scan.
@@ -946,7 +954,7 @@ cudaError_t launch_timeline_given(const DeviceTrace &t, const Workspace &w, int6
     cfg.gridDim = dim3((unsigned)seg_scan_blocks(t.K));
     cfg.blockDim = dim3(kSegThreads);
     return cudaLaunchKernelEx(&cfg, k_seg_scan<1>, t.K, (int64_t)0, (const int64_t *)w.diff, (const int64_t *)point, pressure, w.pressure_scan.ticket,
-                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out);
+                              w.pressure_scan.done, w.seg_words2, w.tile_max, w.tile_slot, peak_bytes, peak_slot, w.status, status_out, (int64_t *)nullptr, (int64_t *)nullptr);
 }
 
 // =============================================================================================

@@ -151,21 +151,34 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
     __syncthreads();
     ull bad = 0;
     // the partition walks the events kernel by kernel: kernel_ptr has to be a monotone map onto [0, E]
-    for (int64_t k = (int64_t)blockIdx.x * kBkThreads + threadIdx.x; k < B.K; k += (int64_t)gridDim.x * kBkThreads) {
-        const int64_t p0 = kptr[k], p1 = kptr[k + 1];
-        if (p0 > p1 || p0 < 0 || p1 > B.E || (k == 0 && p0 != 0) || (k == B.K - 1 && p1 != B.E)) bad |= G10_DEV_BAD_KERNEL_PTR;
-    }
-    const int64_t tiles = (B.E + kBkTile - 1) / kBkTile;
-    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        const int64_t base = tile * kBkTile;
-        int32_t id[kBkItems];
+    // (both walks are short chains of memory latencies: four steps of the first and two tiles of the second have their loads
+    // in flight together)
+    for (int64_t k0 = (int64_t)blockIdx.x * kBkThreads + threadIdx.x; k0 < B.K; k0 += 4 * (int64_t)gridDim.x * kBkThreads) {
+        int64_t p0[4], p1[4];
 #pragma unroll
-        for (int j = 0; j < kBkItems; ++j) {
-            const int64_t e = base + (int64_t)j * kBkThreads + threadIdx.x;
-            id[j] = e < B.E ? kt[e] : -2;
+        for (int q = 0; q < 4; ++q) {
+            const int64_t k = k0 + q * (int64_t)gridDim.x * kBkThreads;
+            p0[q] = k < B.K ? kptr[k] : 0; p1[q] = k < B.K ? kptr[k + 1] : 0;
         }
 #pragma unroll
-        for (int j = 0; j < kBkItems; ++j) {
+        for (int q = 0; q < 4; ++q) {
+            const int64_t k = k0 + q * (int64_t)gridDim.x * kBkThreads;
+            if (k < B.K && (p0[q] > p1[q] || p0[q] < 0 || p1[q] > B.E || (k == 0 && p0[q] != 0) || (k == B.K - 1 && p1[q] != B.E)))
+                bad |= G10_DEV_BAD_KERNEL_PTR;
+        }
+    }
+    const int64_t tiles = (B.E + kBkTile - 1) / kBkTile;
+    constexpr int kHistItems = 2 * kBkItems;
+    for (int64_t tile = blockIdx.x; tile < tiles; tile += 2 * (int64_t)gridDim.x) {
+        int32_t id[kHistItems];
+#pragma unroll
+        for (int j = 0; j < kHistItems; ++j) {
+            const int64_t t2 = tile + (j / kBkItems) * (int64_t)gridDim.x;
+            const int64_t e = t2 * kBkTile + (int64_t)(j % kBkItems) * kBkThreads + threadIdx.x;
+            id[j] = (t2 < tiles && e < B.E) ? kt[e] : -2;
+        }
+#pragma unroll
+        for (int j = 0; j < kHistItems; ++j) {
             if (id[j] == -2) continue;
             if (!kMulti) {
                 if (id[j] < 0 || id[j] >= B.N) bad |= G10_DEV_BAD_TENSOR_ID;
@@ -744,7 +757,7 @@ cudaError_t launch_vitality_buckets(const DeviceTrace &t, const Workspace &w, co
         B.bucket_count = w.bk_count; B.bucket_cursor = w.bk_cursor; B.pairs = w.bk_pairs; B.words = w.bk_words;
         B.ticket = w.emit_scan.ticket; B.done = w.emit_scan.done; B.status_out = status_out; B.status = w.status; B.spill = w.raw_uses;
         B.zero_diff = nullptr; B.zero_point = nullptr;
-        if (p == 0 && out.tl_diff != nullptr) {
+        if (p == 0 && out.tl_diff != nullptr && !out.tl_cleared) {
             if (t.E > 0 && t.K > 0) { B.zero_diff = (int64_t *)out.tl_diff; B.zero_point = (int64_t *)out.tl_point; }
             else {                                     // (no counting kernel will run: clear them here)
                 cudaError_t e0;
