@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_hist(BucketArgs B, const int6
 // registers; (c) the counters are scanned and the round's room in every bucket it touches is reserved with one
 // global atomic per bucket; (d) the keys are staged in bucket order in shared memory and (e) written out in
 // coalesced runs.
-constexpr int kPtMaxItems = 16;                     // events per thread and round, at most (tile_cap <= 16 * kBkThreads)
+constexpr int kPtMaxItems = 18;                     // events per thread and round, at most (tile_cap <= 18 * kBkThreads)
 
 template <bool kMulti>
 __global__ void __launch_bounds__(kBkThreads, 2) k_bk_scatter(BucketArgs B, const int64_t *__restrict__ kptr, const int32_t *__restrict__ kt)
@@ -697,13 +697,14 @@ static cudaError_t launch_bucket_pass(BucketArgs B, const DeviceTrace &t, const 
         }
         // Shared memory of the partition kernel: three bucket tables and ten bytes per staged event; two blocks per SM.
         const size_t tables = sizeof(int) * (size_t)(3 * bk_pad(B.nb)) + 8;
-        int64_t cap = ((int64_t)(100 << 10) - (int64_t)tables) / 10 / kBkThreads * kBkThreads;
+        int64_t cap = ((int64_t)(108 << 10) - (int64_t)tables) / 10 / kBkThreads * kBkThreads;
         cap = cap < kBkThreads ? kBkThreads : (cap > (int64_t)kPtMaxItems * kBkThreads ? (int64_t)kPtMaxItems * kBkThreads : cap);
         B.tile_cap = (int)cap;
-        // Kernels per tile: as many as fill nine tenths of a round on average (so that few tiles need a second round),
+        // Kernels per tile: as many as fill 92 % of a round on average (so that few tiles need a second round; a round has costs
+        // of its own, so few full rounds beat many light ones: config 4 takes two rounds per block this way, not three),
         // then evened out so that every block of the grid gets the same number of tiles.
         const int g2max = 2 * sms;
-        int64_t tk = (cap * 9 / 10) * t.K / t.E;
+        int64_t tk = (cap * 92 / 100) * t.K / t.E;
         tk = tk < 32 ? 32 : (tk > 32768 ? 32768 : tk);
         const int64_t per_block = (t.K + tk * g2max - 1) / (tk * g2max);
         tk = (t.K + per_block * g2max - 1) / (per_block * g2max);
