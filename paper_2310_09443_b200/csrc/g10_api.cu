@@ -446,8 +446,9 @@ int32_t g10_emit_instructions(int64_t K, int64_t N, const int32_t *first_use, co
     if (N > 0 && (!first_use || !last_use || !tensor_bytes)) return G10_ERR_ARG;
     if (n > 0 && !migrations) return G10_ERR_ARG;
     if (out->instructions_cap < 0 || (out->instructions_cap > 0 && !out->instructions)) return G10_ERR_ARG;
-    int shift = 0, nb = 0;
-    if (!emit_choose_buckets(K, 2 * N + 2 * n, &shift, &nb)) return G10_ERR_LIMIT;
+    int bw = 0, nb = 0;
+    ull magic = 0;
+    if (!emit_choose_buckets(K, 2 * N + 2 * n, 0, &bw, &nb, &magic)) return G10_ERR_LIMIT;
     EmitLaunch L;
     char *zb = nullptr;
     size_t zbytes = 0;

@@ -12,6 +12,7 @@
 // A bucket too large for shared memory (very many tensors allocated at one boundary) is sorted in global memory.
 #include "g10_device.cuh"
 #include "g10_internal.h"
+#include <cstddef>
 
 namespace g10 {
 
@@ -27,7 +28,8 @@ struct EmitArgs {
     const int64_t *start;
     const g10_migration *mig;
     const int64_t *new_issue;
-    int shift, nb;                        // boundaries per bucket = 1 << shift
+    int bw, nb;                           // boundaries per bucket, buckets
+    ull magic;                            // ceil(2^64 / bw) (0 when bw == 1): the bucket of boundary x is the high half of x * magic
     unsigned *bucket_count, *bucket_cursor;
     unsigned *block_count;                // [nb][G] per bucket: what each block of the counting kernel saw, then the running sums
     int G;                                // blocks of the counting and of the scatter kernel (the same items go to the same block)
@@ -66,6 +68,13 @@ __device__ __forceinline__ bool emit_item(const EmitArgs &A, int64_t item, int64
     return true;
 }
 
+// Bucket of a boundary.  With magic = (2^64 + e) / bw, 0 <= e < bw, the product x * magic / 2^64 exceeds x / bw by less than
+// 2^-32 for x < 2^32, and x / bw is at least 1 / bw short of the next integer: the high half is the quotient exactly.
+__device__ __forceinline__ int emit_bucket(const EmitArgs &A, int64_t boundary)
+{
+    return A.magic ? (int)__umul64hi((ull)boundary, A.magic) : (int)boundary;
+}
+
 __device__ __forceinline__ ull emit_key(int64_t boundary, int opcode, int tensor)
 {
     return ((ull)boundary << 33) | ((ull)opcode << 31) | (ull)(unsigned)tensor;
@@ -79,7 +88,7 @@ __global__ void __launch_bounds__(kEmitThreads) k_emit_hist(EmitArgs A)
     const int64_t total = 2 * A.N + 2 * A.n;
     for (int64_t item = (int64_t)blockIdx.x * kEmitThreads + threadIdx.x; item < total; item += (int64_t)gridDim.x * kEmitThreads) {
         int64_t bd; int op, tn, rc;
-        if (emit_item(A, item, &bd, &op, &tn, &rc)) atomicAdd(&s_hist[bd >> A.shift], 1u);
+        if (emit_item(A, item, &bd, &op, &tn, &rc)) atomicAdd(&s_hist[emit_bucket(A, bd)], 1u);
     }
     __syncthreads();
     // what this block saw of every bucket: the scatter kernel, whose blocks walk the same items, gets from it the block's own
@@ -141,7 +150,7 @@ __global__ void __launch_bounds__(kEmitThreads) k_emit_scatter(EmitArgs A)
     for (int64_t item = (int64_t)blockIdx.x * kEmitThreads + threadIdx.x; item < total; item += (int64_t)gridDim.x * kEmitThreads) {
         int64_t bd; int op, tn, rc;
         if (emit_item(A, item, &bd, &op, &tn, &rc)) {
-            const int b = (int)(bd >> A.shift);
+            const int b = emit_bucket(A, bd);
             const long long pos = s_base[b] + atomicAdd(&s_next[b], 1u);       // (shared memory: the block's own run of the bucket)
             A.keys[pos] = emit_key(bd, op, tn);
             if (rc >= 0) A.payload[pos] = rc;          // (only the few instructions that come from a plan record carry one: the
@@ -172,6 +181,10 @@ __device__ void emit_bitonic(ull *k, int32_t *p, int n)
     }
 }
 
+static_assert(sizeof(g10_instruction) == 32 && offsetof(g10_instruction, opcode) == 0 && offsetof(g10_instruction, tensor) == 4 &&
+              offsetof(g10_instruction, target) == 8 && offsetof(g10_instruction, record) == 12 && offsetof(g10_instruction, bytes) == 16 &&
+              offsetof(g10_instruction, time_ns) == 24, "k_emit_write assembles the record from four 64-bit words");
+constexpr int kEmitStageStride = 36;      // (32 + 4: the four word planes of a warp's tile fall into different banks)
 constexpr int kEmitRegs = kEmitCap / kEmitThreads;   // keys a thread keeps in registers between the two passes
 constexpr int kEmitWide = 32;                        // a boundary with more instructions is sorted by the whole block
 
@@ -180,13 +193,14 @@ __global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int6
     extern __shared__ long long s_dyn[];
     long long *s_base = s_dyn;                                   // [nb + 1]
     int *s_cnt = (int *)(s_base + A.nb + 1);                     // [bw + 1] instructions per boundary of the bucket, then their offsets
-    int *s_cur = s_cnt + (1 << A.shift) + 1;                     // [bw] fill cursors
-    ull *s_keys = (ull *)(((uintptr_t)(s_cur + (1 << A.shift)) + 7) & ~(uintptr_t)7);   // [kEmitCap]
+    int *s_cur = s_cnt + A.bw + 1;                               // [bw] fill cursors
+    ull *s_keys = (ull *)(((uintptr_t)(s_cur + A.bw) + 7) & ~(uintptr_t)7);               // [kEmitCap]
     int32_t *s_pay = (int32_t *)(s_keys + kEmitCap);              // [kEmitCap]
+    ull *s_stage = (ull *)(s_pay + kEmitCap);                     // [warps][4][kEmitStageStride] the records of a warp on their way out
     __shared__ long long s_w[kEmitThreads / 32];
     __shared__ int s_bucket, s_nwide;
     __shared__ int s_wide[64];
-    const int bw = 1 << A.shift;
+    const int bw = A.bw;
     emit_scan_buckets(A.bucket_count, A.nb, s_base, s_w);
     for (;;) {
         __syncthreads();
@@ -198,7 +212,7 @@ __global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int6
         const int n = (int)(s_base[b + 1] - base);
         ull *gk = A.keys + base;
         int32_t *gp = A.payload + base;
-        const int64_t b0 = (int64_t)b << A.shift;
+        const int64_t b0 = (int64_t)b * bw;
         const int bw_eff = (int)((A.K + 1 - b0) < bw ? (A.K + 1 - b0) : bw);
         for (int j = threadIdx.x; j <= bw_eff; j += kEmitThreads) { s_cnt[j] = 0; if (j < bw_eff) s_cur[j] = 0; }
         __syncthreads();
@@ -316,37 +330,68 @@ __global__ void __launch_bounds__(kEmitThreads, 2) k_emit_write(EmitArgs A, int6
             counts[0] = s_base[A.nb];
             if (s_base[A.nb] > inst_cap) raise_status(A.status, G10_DEV_PLAN_OVERFLOW);
         }
-        // the records, in order
-        for (int j = threadIdx.x; j < n; j += kEmitThreads) {
-            const long long pos = base + j;
-            if (pos >= inst_cap) continue;
-            const ull key = kp[j];
-            const int64_t boundary = (int64_t)(key >> 33);
-            g10_instruction ins;
-            ins.opcode = (int)((key >> 31) & 3u); ins.tensor = (int)(key & 0x7fffffffu); ins.record = (ins.opcode & 1) ? pp[j] : -1; ins.target = -1;
-            ins.bytes = A.bytes[ins.tensor];
-            ins.time_ns = A.start[boundary];
-            if (ins.opcode == kOpPreEvict) { ins.target = A.mig[ins.record].dest; ins.time_ns = A.mig[ins.record].evict_issue_ns; }
-            if (ins.opcode == kOpPrefetch) {
-                ins.time_ns = A.new_issue ? A.new_issue[ins.record] : A.mig[ins.record].prefetch_issue_ns;
-                if (ins.time_ns >= A.start[A.K]) ins.time_ns -= A.start[A.K];      // (steady-state plans: see emit_item)
+        // the records, in order.  A thread that stored its own 32-byte record would write every 32-byte sector in four pieces
+        // (four 8-byte stores at a stride of 32 bytes across the warp); the 32 records of a warp go through a small
+        // shared-memory tile instead and leave as four contiguous 256-byte runs.
+        {
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            ull *st = s_stage + warp * (4 * kEmitStageStride);
+            for (int j0 = 0; j0 < n; j0 += kEmitThreads) {
+                const int j = j0 + threadIdx.x;
+                ull w0 = 0, w1 = 0, w2 = 0, w3 = 0;
+                if (j < n && base + j < inst_cap) {
+                    const ull key = kp[j];
+                    const int64_t boundary = (int64_t)(key >> 33);
+                    const int opcode = (int)((key >> 31) & 3u), tensor = (int)(key & 0x7fffffffu), record = (opcode & 1) ? pp[j] : -1;
+                    int target = -1;
+                    int64_t time_ns = A.start[boundary];
+                    if (opcode == kOpPreEvict) { target = A.mig[record].dest; time_ns = A.mig[record].evict_issue_ns; }
+                    if (opcode == kOpPrefetch) {
+                        time_ns = A.new_issue ? A.new_issue[record] : A.mig[record].prefetch_issue_ns;
+                        if (time_ns >= A.start[A.K]) time_ns -= A.start[A.K];      // (steady-state plans: see emit_item)
+                    }
+                    w0 = (ull)(unsigned)opcode | ((ull)(unsigned)tensor << 32);
+                    w1 = (ull)(unsigned)target | ((ull)(unsigned)record << 32);
+                    w2 = (ull)A.bytes[tensor];
+                    w3 = (ull)time_ns;
+                }
+                st[0 * kEmitStageStride + lane] = w0; st[1 * kEmitStageStride + lane] = w1;
+                st[2 * kEmitStageStride + lane] = w2; st[3 * kEmitStageStride + lane] = w3;
+                __syncwarp();
+                const long long first = base + j0 + warp * 32;              // the warp's first record
+                long long nrec = n - (j0 + warp * 32);
+                if (inst_cap - first < nrec) nrec = inst_cap - first;
+                if (nrec > 32) nrec = 32;
+                ull *dst = reinterpret_cast<ull *>(inst + first);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int i = q * 32 + lane;                          // 8-byte word of the warp's 1024 bytes
+                    if ((i >> 2) < nrec) dst[i] = st[(i & 3) * kEmitStageStride + (i >> 2)];
+                }
+                __syncwarp();
             }
-            inst[pos] = ins;
         }
     }
 }
 
-bool emit_choose_buckets(int64_t K, int64_t total_items, int *shift, int *nb)
+bool emit_choose_buckets(int64_t K, int64_t total_items, int sms, int *bw, int *nb, ull *magic)
 {
-    // boundaries per bucket so that a bucket holds about 2000 instructions; at most 4096 buckets of 4096 boundaries
+    // boundaries per bucket so that a bucket holds about 3000 instructions (kEmitCap = 4096 are sorted in shared memory; a
+    // fuller bucket goes the slow way); at most 4096 buckets of 4096 boundaries.  k_emit_write takes the buckets one per block
+    // at a time with two blocks per SM: with more buckets than blocks they are narrowed to whole rounds of its grid (sms > 0).
     const int64_t B = K + 1;
-    int64_t want = total_items > 0 ? (2000 * B) / total_items : 4096;
-    int s = 0;
-    while (s < 12 && ((int64_t)1 << (s + 1)) <= want) ++s;
-    while (s < 12 && ((B + ((int64_t)1 << s) - 1) >> s) > 4096) ++s;
-    const int64_t buckets = (B + ((int64_t)1 << s) - 1) >> s;
-    if (buckets > 4096) return false;
-    *shift = s; *nb = (int)buckets;
+    int64_t w = total_items > 0 ? (3000 * B) / total_items : 4096;
+    w = w < 1 ? 1 : (w > 4096 ? 4096 : w);
+    int64_t buckets = (B + w - 1) / w;
+    if (buckets > 4096) { w = (B + 4095) / 4096; buckets = (B + w - 1) / w; }
+    if (w > 4096) return false;
+    const int64_t G = 2 * (int64_t)sms;
+    if (G > 0 && buckets > G) {
+        const int64_t target = (buckets + G - 1) / G * G;
+        if (target <= 4096) { w = (B + target - 1) / target; buckets = (B + w - 1) / w; }
+    }
+    *bw = (int)w; *nb = (int)buckets;
+    *magic = w == 1 ? 0 : ~(ull)0 / (ull)w + 1;
     return true;
 }
 
@@ -356,11 +401,11 @@ cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s)
     A.K = L.K; A.N = L.N; A.n = L.n;
     A.first_use = L.first_use; A.last_use = L.last_use; A.bytes = L.bytes; A.glob = L.glob; A.start = L.start;
     A.mig = L.mig; A.new_issue = L.new_issue;
-    if (!emit_choose_buckets(L.K, 2 * L.N + 2 * L.n, &A.shift, &A.nb)) return cudaErrorInvalidValue;
     A.bucket_count = L.bucket_count; A.bucket_cursor = L.bucket_cursor; A.keys = L.keys; A.payload = L.payload;
     A.ticket = L.ticket; A.status = L.status;
     const int sms = current_sm_count();
     if (sms <= 0) return cudaErrorInvalidDevice;
+    if (!emit_choose_buckets(L.K, 2 * L.N + 2 * L.n, sms, &A.bw, &A.nb, &A.magic)) return cudaErrorInvalidValue;
     const int64_t total = 2 * L.N + 2 * L.n;
     int64_t g = (total + kEmitThreads - 1) / kEmitThreads;
     if (g > 4 * (int64_t)sms) g = 4 * (int64_t)sms;
@@ -373,8 +418,8 @@ cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s)
     cudaError_t e2 = cudaFuncSetAttribute(k_emit_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2);
     if (e2 != cudaSuccess) return e2;
     k_emit_scatter<<<(int)g, kEmitThreads, sm2, s>>>(A); count_launch();
-    const size_t sm3 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(int) * (size_t)(2 * (1 << A.shift) + 2) + 8 +
-                       (sizeof(ull) + sizeof(int32_t)) * kEmitCap;
+    const size_t sm3 = sizeof(long long) * (size_t)(A.nb + 1) + sizeof(int) * (size_t)(2 * A.bw + 2) + 8 +
+                       (sizeof(ull) + sizeof(int32_t)) * kEmitCap + sizeof(ull) * (kEmitThreads / 32) * 4 * kEmitStageStride;
     cudaError_t e = cudaFuncSetAttribute(k_emit_write, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
     if (e != cudaSuccess) return e;
     const int g3 = A.nb < 2 * sms ? A.nb : 2 * sms;

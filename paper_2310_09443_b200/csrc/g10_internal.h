@@ -248,7 +248,7 @@ struct EmitLaunch {
     int64_t inst_cap;
     int64_t *counts;
 };
-bool emit_choose_buckets(int64_t K, int64_t total_items, int *shift, int *nb);
+bool emit_choose_buckets(int64_t K, int64_t total_items, int sms, int *bw, int *nb, ull *magic);
 cudaError_t launch_emit(const EmitLaunch &L, cudaStream_t s);
 cudaError_t launch_characterize(int64_t K, int64_t N, const int64_t *use_ptr, const int32_t *uses, const int64_t *bytes, const int64_t *start,
                                 int64_t Pn, const int32_t *per_t, const int32_t *per_u, const int32_t *per_v, uint64_t host_bw, uint64_t ssd_bw,
