@@ -198,10 +198,13 @@ def _csr_trace(name, rng, K, N, degrees):
                         tensor_global=(rng.random(N) < 0.01).astype(np.uint8), capacity_frac=(1, 2))
 
 
-@pytest.mark.parametrize("shape", ["one_event_per_kernel", "mostly_empty_kernels", "few_tensors_many_uses", "every_kernel_wide", "many_tensors"])
+@pytest.mark.parametrize("shape", ["one_event_per_kernel", "mostly_empty_kernels", "few_tensors_many_uses", "every_kernel_wide", "many_tensors",
+                                   "odd_narrow_buckets", "odd_wide_buckets"])
 def test_pass_shapes(gpu, oracle, shape):
     """Vitality and timeline on traces whose shape drives the partition differently: the widest and the narrowest tiles,
-    empty kernels, buckets that overflow shared memory, kernels all wider than a warp row, thousands of buckets."""
+    empty kernels, buckets that overflow shared memory, kernels all wider than a warp row, thousands of buckets, and bucket
+    widths that are no powers of two (more buckets than the last kernel has blocks: 113 and 2534 tensors per bucket on a
+    148-SM part), with many and with few events per tensor."""
     rng = np.random.default_rng(1000 + len(shape))
     if shape == "one_event_per_kernel":
         K, N = 200_000, 50_000
@@ -215,6 +218,12 @@ def test_pass_shapes(gpu, oracle, shape):
     elif shape == "every_kernel_wide":
         K, N = 600, 40_000
         tr = _csr_trace(shape, rng, K, N, rng.integers(65, 400, size=K))
+    elif shape == "odd_narrow_buckets":
+        K, N = 60_000, 100_000
+        tr = _csr_trace(shape, rng, K, N, rng.integers(30, 70, size=K))
+    elif shape == "odd_wide_buckets":
+        K, N = 250_000, 1_500_000
+        tr = _csr_trace(shape, rng, K, N, rng.integers(4, 12, size=K))
     else:
         K, N = 50_000, 3_000_000
         tr = _csr_trace(shape, rng, K, N, rng.integers(0, 9, size=K))
