@@ -346,9 +346,10 @@ __device__ void bk_bitonic_sort_i32(int32_t *a, int n)    // arbitrary n: the ne
 __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
 
 
-// (kTimeline: the call also wants the pressure timeline; the outputs loop then books every tensor's size, see VitalityBuffers)
+// (kTimeline: the call also wants the pressure timeline; the outputs loop then books every tensor's size, see VitalityBuffers.
+// Two blocks share an SM -- shared memory is sized for that -- so the kernel must stay within 64 registers.)
 template <bool kTimeline>
-__global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBuffers out)
+__global__ void __launch_bounds__(kBkThreads, 2) k_bk_emit(BucketArgs B, VitalityBuffers out)
 {
     extern __shared__ __align__(16) int s_mem[];
     int *s_base = s_mem;                       // [nb + 1] first key of each bucket
@@ -388,9 +389,9 @@ __global__ void __launch_bounds__(kBkThreads) k_bk_emit(BucketArgs B, VitalityBu
         for (int tl = threadIdx.x; tl <= bt_eff; tl += kBkThreads) { t_off[tl] = 0; t_d[tl] = 0; }
         __syncthreads();
         // ---- raw events per tensor, segment offsets, scatter.  The first keys of the bucket stay in registers between the
-        // counting and the scatter; the rest is read again (from L2).  Six per thread: with twelve -- every key of a usual
-        // bucket -- the kernel needs more than the 64 registers that let two blocks share an SM, and spills.
-        constexpr int kRegKeys = kTimeline ? 4 : 6;          // (the bookings of the timeline form need registers of their own)
+        // counting and the scatter; the rest is read again (from L2).  Eight per thread, about a usual bucket's share: with
+        // twelve the kernel needs more than the 64 registers that let two blocks share an SM, and spills.
+        constexpr int kRegKeys = kTimeline ? 4 : 8;          // (the bookings of the timeline form need registers of their own)
         ull rk[kRegKeys];
 #pragma unroll
         for (int q = 0; q < kRegKeys; ++q) {
