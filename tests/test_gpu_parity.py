@@ -578,6 +578,30 @@ def test_instruction_stream(gpu, oracle):
     check_emit(gpu, oracle, big, 10**9, False)
 
 
+@pytest.mark.gpu
+def test_instruction_stream_in_whole_rounds(gpu, oracle):
+    """The stream of allocations and frees of a 200 000-kernel trace (no plan): 1.1 M instructions in more buckets than the
+    writing kernel has blocks, so that the buckets are narrowed to whole rounds of its grid (592 buckets of 338 boundaries
+    on a 148-SM part: a width that is no power of two)."""
+    import torch
+    tr = traces.config4_stress_dag(K=200_000, N=800_000)
+    tb = gpu.upload(tr)
+    v = gpu.g10_vitality(tb)
+    tl = gpu.g10_pressure_timeline(tb)
+    em = gpu.g10_emit_instructions(tr.K, tr.N, v.first_use, v.last_use, tb.tensor_bytes, tb.tensor_global, tl.kernel_start_ns, 0, None, None)
+    torch.cuda.synchronize()
+    assert int(em.counts[1].item()) == 0
+    ov = oracle.vitality(tr.kernel_ptr, tr.kernel_tensors, tr.N)
+    start = oracle.slot_clock(tr.kernel_ns)
+    oe = oracle.emit_instructions(tr.K, ov.first_use, ov.last_use, tr.tensor_bytes, tr.tensor_global, start,
+                                  np.zeros(0, oracle.MIGRATION_DTYPE), None)
+    assert int(em.counts[0].item()) == len(oe.instructions) > 1_000_000
+    assert np.array_equal(_np(em.inst_ptr), oe.inst_ptr)
+    got = gpu.instructions_numpy(em)
+    for name in got.dtype.names:
+        assert np.array_equal(got[name], oe.instructions[name]), name
+
+
 def check_stats(gpu, oracle, tr):
     """Characterisation statistics (Section 3, Figures 2-4) from the GPU's own vitality + slot clock."""
     import torch
