@@ -441,17 +441,37 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_emit(BucketArgs B, Vitalit
             const int tl = s_mid[q];
             const int m = t_off[tl + 1] - t_off[tl];
             int32_t *seg = ks + t_off[tl];
-            for (int a = 1; a < m; ++a) {
-                const int32_t x = seg[a];
-                int c = a - 1;
-                while (c >= 0 && seg[c] > x) { seg[c + 1] = seg[c]; --c; }
-                seg[c + 1] = x;
-            }
-            int32_t prev = seg[0];
             int dd = 1, pp = 0;
-            for (int a = 1; a < m; ++a) {
-                const int32_t x = seg[a];
-                if (x != prev) { if (x - prev >= 2) ++pp; seg[dd++] = x; prev = x; }
+            if (m <= 8) {
+                // up to eight raw uses (nearly all of the list): loaded together, put in order by a 19-comparator network in
+                // registers (the padding sorts to the end), then de-duplicated on the way back -- one round trip to shared
+                // memory instead of an insertion sort's chain of them
+                int32_t v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = j < m ? seg[j] : 0x7fffffff;
+#define G10_CE(a, b) { const int32_t lo = min(v[a], v[b]), hi = max(v[a], v[b]); v[a] = lo; v[b] = hi; }
+                G10_CE(0, 1) G10_CE(2, 3) G10_CE(4, 5) G10_CE(6, 7) G10_CE(0, 2) G10_CE(1, 3) G10_CE(4, 6) G10_CE(5, 7) G10_CE(1, 2) G10_CE(5, 6)
+                G10_CE(0, 4) G10_CE(1, 5) G10_CE(2, 6) G10_CE(3, 7) G10_CE(2, 4) G10_CE(3, 5) G10_CE(1, 2) G10_CE(3, 4) G10_CE(5, 6)
+#undef G10_CE
+                int32_t prev = v[0];
+                seg[0] = prev;
+#pragma unroll
+                for (int a = 1; a < 8; ++a) {
+                    const int32_t x = v[a];
+                    if (a < m && x != prev) { if (x - prev >= 2) ++pp; seg[dd++] = x; prev = x; }
+                }
+            } else {
+                for (int a = 1; a < m; ++a) {
+                    const int32_t x = seg[a];
+                    int c = a - 1;
+                    while (c >= 0 && seg[c] > x) { seg[c + 1] = seg[c]; --c; }
+                    seg[c + 1] = x;
+                }
+                int32_t prev = seg[0];
+                for (int a = 1; a < m; ++a) {
+                    const int32_t x = seg[a];
+                    if (x != prev) { if (x - prev >= 2) ++pp; seg[dd++] = x; prev = x; }
+                }
             }
             t_d[tl] = dd; t_np[tl] = pp;
             my_d += dd; my_p += pp;
