@@ -41,8 +41,8 @@ L2_FLUSH_BYTES = 512 << 20
 # caches alone between launches, as this program does: the write-back of the L2 flush's dirty lines is part of it).
 # "sources_sha256" is the hash of the kernel sources at the time of the capture: when the sources have changed since, the
 # bench line says so ("traffic_stale") instead of passing old traffic off as current, and a CPU test warns.
-TRAFFIC = {"vitality": 227_700_000, "timeline": 124_000_000, "timeline_given": 135_700_000, "fused": 337_700_000, "captured_at": "2026-11-25",
-           "sources_sha256": "3025ada8c83b46c5e231ea4ecee75191e583e2bdba296f448e49db9c68afb0fb"}
+TRAFFIC = {"vitality": 227_100_000, "timeline": 117_800_000, "timeline_given": 135_500_000, "fused": 337_200_000, "captured_at": "2026-11-25",
+           "sources_sha256": "ebb78cb31457e2e2a3b2906af1e995c64e1459826260a1eb9c5a0bb878efadf8"}
 
 
 PASS_SOURCES = ("g10_passes.cu", "g10_vitality_buckets.cu")     # the kernels of g10_vitality and g10_pressure_timeline

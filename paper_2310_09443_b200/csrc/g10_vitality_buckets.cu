@@ -346,7 +346,7 @@ __device__ void bk_bitonic_sort_i32(int32_t *a, int n)    // arbitrary n: the ne
 __device__ __forceinline__ ull bk_pack(long long v) { return (1ull << 62) | ((ull)v & ((1ull << 62) - 1)); }
 
 
-// (kTimeline: the call also wants the pressure timeline; the outputs loop then books every tensor's size, see VitalityBuffers.
+// (kTimeline: the call also wants the pressure timeline; the kernel then books every tensor's size itself, see VitalityBuffers.
 // Two blocks share an SM -- shared memory is sized for that -- so the kernel must stay within 64 registers.)
 template <bool kTimeline>
 __global__ void __launch_bounds__(kBkThreads, 2) k_bk_emit(BucketArgs B, VitalityBuffers out)
@@ -391,7 +391,7 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_emit(BucketArgs B, Vitalit
         // ---- raw events per tensor, segment offsets, scatter.  The first keys of the bucket stay in registers between the
         // counting and the scatter; the rest is read again (from L2).  Eight per thread, about a usual bucket's share: with
         // twelve the kernel needs more than the 64 registers that let two blocks share an SM, and spills.
-        constexpr int kRegKeys = kTimeline ? 4 : 8;          // (the bookings of the timeline form need registers of their own)
+        constexpr int kRegKeys = 8;
         ull rk[kRegKeys];
 #pragma unroll
         for (int q = 0; q < kRegKeys; ++q) {
@@ -525,6 +525,43 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_emit(BucketArgs B, Vitalit
                 asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(&B.words[2 * b + 1]), "l"(bk_pack(tp)) : "memory");
             }
         }
+        // ---- the pressure timeline is wanted from the same call: every tensor's size is booked where it is born and where it
+        // dies (a tensor of one kernel in that slot's point mass; a global tensor in slot 0, summed per thread first).  First
+        // and last use are known since the segments were sorted.  Done here, in a loop of their own behind the publication of
+        // the totals, the reductions go out while the totals of the earlier buckets come in; inside the outputs loop their
+        // requests to the L2 came on top of that loop's stores, and the loop's registers cost the kernel its keys in registers.
+        if (kTimeline) {
+            constexpr int kBook = 4;                           // (tensors of a thread whose loads are in flight together; 2, 3 and 8 were slower)
+            for (int tl0 = threadIdx.x; tl0 < bt_eff; tl0 += kBook * kBkThreads) {
+                long long bz4[kBook];
+                int dd4[kBook], of4[kBook];
+#pragma unroll
+                for (int q = 0; q < kBook; ++q) {
+                    const int tl = tl0 + q * kBkThreads;
+                    bz4[q] = 1; dd4[q] = -1; of4[q] = 0;
+                    if (tl < bt_eff) {
+                        bz4[q] = out.tl_bytes[t0 + tl]; dd4[q] = t_d[tl]; of4[q] = t_off[tl];
+                        if (out.tl_glob != nullptr && out.tl_glob[t0 + tl]) dd4[q] = -2 - dd4[q];   // (a global tensor: -2 - its uses)
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < kBook; ++q) {
+                    if (dd4[q] == -1) continue;
+                    const long long bsz = bz4[q];
+                    if (bsz < 1 || bsz >= ((long long)1 << 40)) tl_bad = true;
+                    if (dd4[q] < -2) tl_gsum += bsz;                   // (global and used)
+                    else if (dd4[q] > 0) {
+                        const int64_t f = ks[of4[q]], l = ks[of4[q] + dd4[q] - 1];
+                        if (f == l) atomicAdd(&out.tl_point[f], (ull)bsz);
+                        else {
+                            atomicAdd(&out.tl_diff[f], (ull)bsz);
+                            if (l + 1 < out.tl_K) atomicAdd(&out.tl_diff[l + 1], (ull)(-bsz));
+                        }
+                    }
+                }
+            }
+            // (no barrier: the scan below writes t_d only behind a barrier of its own, which every thread reaches after this loop)
+        }
         bk_block_scan<2>(t_d, t_d, t_np, t_np, bt_eff, s_scan);
         const long long D = t_d[bt_eff], PC = t_np[bt_eff];
         long long pu = 0, pq = 0;
@@ -578,15 +615,11 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_emit(BucketArgs B, Vitalit
         for (int tl0 = threadIdx.x; tl0 < bt_eff; tl0 += 2 * kBkThreads) {
             int d04[2], dd4[2], of4[2], np4[2];
             int32_t f4[2], l4[2];
-            long long bz4[2];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int tl = tl0 + q * kBkThreads;
-                d04[q] = 0; dd4[q] = -1; of4[q] = 0; np4[q] = 0; bz4[q] = 1;
-                if (tl < bt_eff) {
-                    d04[q] = t_d[tl]; dd4[q] = t_d[tl + 1] - d04[q]; of4[q] = t_off[tl]; np4[q] = t_np[tl];
-                    if (kTimeline) bz4[q] = out.tl_bytes[t0 + tl];
-                }
+                d04[q] = 0; dd4[q] = -1; of4[q] = 0; np4[q] = 0;
+                if (tl < bt_eff) { d04[q] = t_d[tl]; dd4[q] = t_d[tl + 1] - d04[q]; of4[q] = t_off[tl]; np4[q] = t_np[tl]; }
             }
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
@@ -605,21 +638,6 @@ __global__ void __launch_bounds__(kBkThreads, 2) k_bk_emit(BucketArgs B, Vitalit
             out.num_uses[t] = dd;
             out.use_ptr[t] = U + d04[q];
             out.period_ptr[t] = PB + np4[q];
-            if (kTimeline) {
-                // the pressure timeline is wanted from the same call: the tensor's size is booked where it is born and where it dies
-                // (a tensor of one kernel in that slot's point mass; a global tensor in slot 0, summed per thread first)
-                const long long bsz = bz4[q];
-                if (bsz < 1 || bsz >= ((long long)1 << 40)) tl_bad = true;
-                if (dd > 0) {
-                    const int64_t f = f4[q], l = l4[q];
-                    if (out.tl_glob != nullptr && out.tl_glob[t]) tl_gsum += bsz;
-                    else if (f == l) atomicAdd(&out.tl_point[f], (ull)bsz);
-                    else {
-                        atomicAdd(&out.tl_diff[f], (ull)bsz);
-                        if (l + 1 < out.tl_K) atomicAdd(&out.tl_diff[l + 1], (ull)(-bsz));
-                    }
-                }
-            }
             long long uo = U + d04[q], po = PB + np4[q];
             for (int a = dense ? 1 : 0; a < dd; ++a) {
                 const int32_t x = seg[a];
