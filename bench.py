@@ -69,7 +69,10 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi (every 20 ms, a process of its own: a sampling thread in this
+    process would delay the launches) from some untimed steps before the timed region to its end.  The timed region of the
+    default run lasts a few milliseconds, less than nvidia-smi needs to come up: it is started a moment earlier, the same
+    step runs untimed until it has answered a few times, and the timed steps follow at once."""
 
     def __init__(self, gpu_index: int):
         self.rows = []
@@ -81,7 +84,7 @@ class ClockSampler:
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -92,10 +95,14 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
-    def stop(self):
+    def count(self) -> int:
+        return len(self.rows)
+
+    def stop(self, first_timed_row: int = 0):
+        """first_timed_row: how many rows there were when the timed region began (the rest came during it)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        in_timed = len(self.rows) - first_timed_row
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -114,7 +121,8 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "samples_in_timed_region": max(0, in_timed),
+                "window": "untimed steps right before the timed region and the timed region itself"}
 
 
 
@@ -352,6 +360,17 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    # (more untimed steps, paced by the GPU, until the sampler has answered a few times -- at most half a second; every rank
+    # does the same so that the ranks stay under the same load)
+    t_settle = time.time()
+    while time.time() - t_settle < 0.5 and (rank != 0 or sampler.proc is None or sampler.count() < 4 or time.time() - t_settle < 0.1):
+        flush.fill_(1)
+        step()
+        torch.cuda.synchronize()
+        if rank == 0 and sampler.proc is None:
+            break
+    barrier()
+    first_timed_row = sampler.count()
     launches0 = binding.g10_launch_count()
     total_ms = 0.0
     for _ in range(args.steps):
@@ -364,7 +383,7 @@ def run_ours(args):
         total_ms += a.elapsed_time(b)
     gpu_launches = binding.g10_launch_count() - launches0
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(first_timed_row) if rank == 0 else None
     total_ms = max_over_ranks(torch, dist, world, total_ms, dev)
     value = aggregate_events_per_s(world, E, args.steps, total_ms)
     step_s = total_ms / args.steps / 1e3
@@ -601,7 +620,7 @@ def cpu_baseline(tr):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)      # (0.3 ms each with the L2 flush: long enough for a few clock samples)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline, plans and per-call rooflines only")
